@@ -1,0 +1,243 @@
+"""TEST INFRASTRUCTURE -- Algorithm 1 (RSD) of the paper, batched over independent rows.
+
+For every live row and step i (Algorithm 1, loop body):
+    draft step   y^_i <- m(x, y_{1:i-1})
+    reward       r_i  <- r(y^_i | x, y_{1:i-1})          (the listing prints y_i; the prose around
+                                                           it scores the draft step)
+    if A_omega(r_i):  y_i <- y^_i                          (Algorithm 2, Table 1)
+    else:             y_i <- M(x, y_{1:i-1})
+    stop the row when the EOS token s is in y_i, or after N steps.
+
+A "step" is a run of tokens that ends with the step delimiter (Section 3, "Default Setting": a
+generation ending in a blank line is one reasoning step), with EOS, or at a token cap.
+
+Besides the token-level results the loop keeps the integer book-keeping a paged implementation
+needs, under one deterministic policy, so it can be compared bit for bit:
+  * per model a cursor kv_len[b] = number of positions whose keys/values are cached.  The newest
+    committed token may be un-cached; it is the first input of the next decode;
+  * 16-token pages handed out by a bump counter, in ascending row order, when a phase needs
+    capacity: draft (live rows) up to |z_i|-1+cap at step start, PRM (live rows) up to
+    |z_i|+len(y^_i) before scoring, target (rejected rows) up to |z_i|-1+cap after the gate;
+    pages stay with their row until reset;
+  * the ascending list of rejected rows, and token / FLOPs counters (Section 3.3: 2N FLOPs per
+    inference token of an N-parameter model, PRM included).
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+
+import numpy as np
+
+from . import OracleModel, sample, accept as _accept, uniform as _uniform
+
+DRAFT, PRM, TARGET = 0, 1, 2
+STREAM_ACCEPT = 3  # Philox stream of the acceptance uniform of Algorithm 2
+
+
+@dataclass
+class LoopConfig:
+    max_step_tokens: int
+    max_steps: int
+    max_seq_tokens: int
+    step_end_id: int
+    eos_id: int = -1
+    step_end_mod: int = 0          # >0: a token ends a step iff id % mod == step_end_id % mod
+    temperature: float = 0.0
+    seed: int = 0
+    page_tokens: int = 16
+    omega_kind: int = 1            # Table 1 row: 0 constant, 1 binary step, 2 clip, 3 r/(1+r), 4 logistic
+    omega_b: float = 0.0           # alpha of the logistic; the first parameter is the delta of each step
+    pool_pages: tuple = (1 << 30, 1 << 30, 1 << 30)
+    keep_logits: bool = False
+
+
+@dataclass
+class Row:
+    z: list                         # committed tokens: prompt x followed by y_{1:i-1}
+    live: bool = True
+    n_steps: int = 0
+    kv_len: list = field(default_factory=lambda: [0, 0, 0])
+    caches: list = field(default_factory=lambda: [None, None, None])
+    pages: list = field(default_factory=lambda: [[], [], []])
+
+
+class OracleRSD:
+    def __init__(self, draft: OracleModel, prm: OracleModel, target: OracleModel, cfg: LoopConfig):
+        self.models = [draft, prm, target]
+        self.cfg = cfg
+        self.v_limit = min(m.shape.vocab for m in self.models)  # ids valid for all three embeddings
+        self.rows: list[Row] = []
+        self.next_page = [0, 0, 0]
+        self.counters = dict(gen_tokens=[0, 0, 0], ingest_tokens=[0, 0, 0], score_tokens=0, steps=0,
+                             accepted_steps=0, rejected_steps=0, discarded_draft_tokens=0)
+
+    # -- book-keeping ---------------------------------------------------------------------
+    def _reserve(self, which: int, b: int, need_tokens: int):
+        row = self.rows[b]
+        pt = self.cfg.page_tokens
+        while len(row.pages[which]) * pt < need_tokens:
+            if self.next_page[which] >= self.cfg.pool_pages[which]:
+                raise MemoryError("page pool exhausted")
+            row.pages[which].append(self.next_page[which])
+            self.next_page[which] += 1
+
+    def _ends_step(self, tok: int) -> bool:
+        c = self.cfg
+        if c.eos_id >= 0 and tok == c.eos_id:
+            return True
+        if c.step_end_mod > 0:
+            return tok % c.step_end_mod == c.step_end_id % c.step_end_mod
+        return tok == c.step_end_id
+
+    def _ingest(self, which: int, b: int, upto: int, tokens: list) -> np.ndarray | None:
+        """Cache positions [kv_len, upto) of `tokens` in model `which`; returns their hidden states."""
+        row = self.rows[b]
+        start = row.kv_len[which]
+        if upto <= start:
+            return None
+        h = self.models[which].forward(row.caches[which], tokens[start:upto], start)
+        row.kv_len[which] = upto
+        return h
+
+    # -- entry points -----------------------------------------------------------------------
+    def prefill(self, prompts: list):
+        """Rows start with z_1 = x.  The draft caches x without its last token, the PRM all of x;
+        the target is left untouched until a row is first rejected."""
+        self.rows = []
+        for b, p in enumerate(prompts):
+            row = Row(z=[int(t) for t in p])
+            for which in (DRAFT, PRM, TARGET):
+                row.caches[which] = self.models[which].new_cache(self.cfg.max_seq_tokens)
+            self.rows.append(row)
+        for b, row in enumerate(self.rows):
+            self._reserve(DRAFT, b, len(row.z) - 1)
+        for b, row in enumerate(self.rows):
+            self._reserve(PRM, b, len(row.z))
+        for b, row in enumerate(self.rows):
+            n = len(row.z)
+            self._ingest(DRAFT, b, n - 1, row.z)
+            self._ingest(PRM, b, n, row.z)
+            self.counters["ingest_tokens"][DRAFT] += n - 1
+            self.counters["ingest_tokens"][PRM] += n
+            if n + self.cfg.max_step_tokens > self.cfg.max_seq_tokens:
+                row.live = False
+
+    def _generate_step(self, which: int, b: int, forced=None, trace=None) -> list:
+        """One step from model `which` given the row's context z (Algorithm 1: m(x, y_{1:i-1}) or
+        M(x, y_{1:i-1})): cache what of z is missing, then decode token by token."""
+        row, cfg, model = self.rows[b], self.cfg, self.models[which]
+        z = row.z
+        before = row.kv_len[which]
+        self._ingest(which, b, len(z) - 1, z)
+        self.counters["ingest_tokens"][which] += (len(z) - 1) - before
+        out, cur, pos = [], z[-1], len(z) - 1
+        for j in range(cfg.max_step_tokens):
+            h = model.forward(row.caches[which], [cur], pos)
+            row.kv_len[which] = pos + 1
+            logits = model.logits(h[0])
+            tok, margin = sample(logits, self.v_limit, cfg.temperature, cfg.seed, which, b, pos + 1)
+            if trace is not None:
+                trace["sampled"].append(tok)
+                trace["margin"].append(margin)
+                if cfg.keep_logits:
+                    trace["logits"].append(logits.copy())
+            if forced is not None:
+                tok = int(forced[j])
+            out.append(tok)
+            self.counters["gen_tokens"][which] += 1
+            if self._ends_step(tok) or (forced is not None and j + 1 == len(forced)):
+                break
+            cur, pos = tok, pos + 1
+        return out
+
+    def step(self, delta: float, forced_draft=None, forced_target=None, forced_accept=None) -> dict:
+        """One pass of the loop body of Algorithm 1 over all rows.  `forced_*` (per-row lists, or
+        None entries) replace sampled tokens / gate decisions; what was sampled is still reported."""
+        cfg, B = self.cfg, len(self.rows)
+        res = dict(step_tokens=[[] for _ in range(B)], step_len=np.zeros(B, np.int32),
+                   rewards=np.zeros(B, np.float64), accept=np.zeros(B, np.uint8), live=np.zeros(B, np.uint8),
+                   draft_tokens=[[] for _ in range(B)], target_tokens=[[] for _ in range(B)],
+                   draft_trace=[None] * B, target_trace=[None] * B, rej_idx=[], z_len_before=np.zeros(B, np.int32))
+        live_rows = [b for b in range(B) if self.rows[b].live]
+        for b in range(B):
+            res["z_len_before"][b] = len(self.rows[b].z)
+
+        # draft step y^_i for every live row
+        for b in live_rows:
+            self._reserve(DRAFT, b, len(self.rows[b].z) - 1 + cfg.max_step_tokens)
+        for b in live_rows:
+            tr = dict(sampled=[], margin=[], logits=[])
+            f = forced_draft[b] if forced_draft is not None else None
+            res["draft_tokens"][b] = self._generate_step(DRAFT, b, f, tr)
+            res["draft_trace"][b] = tr
+
+        # reward r_i = r(y^_i | z_i), read at the last token of the draft step
+        for b in live_rows:
+            self._reserve(PRM, b, len(self.rows[b].z) + len(res["draft_tokens"][b]))
+        for b in live_rows:
+            row = self.rows[b]
+            seq = row.z + res["draft_tokens"][b]
+            n_known = len(row.z) - row.kv_len[PRM]      # committed tokens the PRM has not cached yet
+            h = self._ingest(PRM, b, len(seq), seq)
+            res["rewards"][b] = self.models[PRM].reward(h[-1])
+            self.counters["ingest_tokens"][PRM] += n_known
+            self.counters["score_tokens"] += len(res["draft_tokens"][b])
+
+        # acceptance criterion A_omega(r_i)  (Algorithm 2; binary step: accept iff r_i >= delta)
+        for b in live_rows:
+            u = _uniform(cfg.seed, STREAM_ACCEPT, b, len(self.rows[b].z), 0)
+            a = _accept(cfg.omega_kind, res["rewards"][b], float(delta), cfg.omega_b, u)
+            if forced_accept is not None and forced_accept[b] is not None:
+                a = int(forced_accept[b])
+            res["accept"][b] = a
+        res["rej_idx"] = [b for b in live_rows if not res["accept"][b]]
+
+        # rejected rows: drop the draft step from the draft and PRM caches, let the target write y_i
+        for b in res["rej_idx"]:
+            row = self.rows[b]
+            row.kv_len[DRAFT] = len(row.z) - 1
+            row.kv_len[PRM] = len(row.z)
+            self.counters["discarded_draft_tokens"] += len(res["draft_tokens"][b])
+        for b in res["rej_idx"]:
+            self._reserve(TARGET, b, len(self.rows[b].z) - 1 + cfg.max_step_tokens)
+        for b in res["rej_idx"]:
+            tr = dict(sampled=[], margin=[], logits=[])
+            f = forced_target[b] if forced_target is not None else None
+            res["target_tokens"][b] = self._generate_step(TARGET, b, f, tr)
+            res["target_trace"][b] = tr
+
+        # commit y_i, stop rows that produced EOS or ran out of steps / room
+        for b in live_rows:
+            row = self.rows[b]
+            y = res["draft_tokens"][b] if res["accept"][b] else res["target_tokens"][b]
+            row.z = row.z + y
+            row.n_steps += 1
+            res["step_tokens"][b] = y
+            res["step_len"][b] = len(y)
+            self.counters["steps"] += 1
+            self.counters["accepted_steps" if res["accept"][b] else "rejected_steps"] += 1
+            if (cfg.eos_id >= 0 and cfg.eos_id in y) or row.n_steps >= cfg.max_steps \
+                    or len(row.z) + cfg.max_step_tokens > cfg.max_seq_tokens:
+                row.live = False
+        for b in range(B):
+            res["live"][b] = 1 if self.rows[b].live else 0
+        return res
+
+    # -- reporting --------------------------------------------------------------------------
+    def flops_paper(self) -> float:
+        """2N per inference token (Section 3.3): every token the draft or the target generated
+        (discarded draft tokens included) and every token the PRM processed."""
+        c = self.counters
+        n = [m.n_params for m in self.models]
+        return 2.0 * n[DRAFT] * c["gen_tokens"][DRAFT] + 2.0 * n[TARGET] * c["gen_tokens"][TARGET] \
+            + 2.0 * n[PRM] * (c["score_tokens"] + c["ingest_tokens"][PRM])
+
+    def state(self) -> dict:
+        B = len(self.rows)
+        return dict(z_len=np.array([len(r.z) for r in self.rows], np.int32),
+                    kv_len=np.array([[r.kv_len[w] for r in self.rows] for w in range(3)], np.int32),
+                    n_pages=np.array([[len(r.pages[w]) for r in self.rows] for w in range(3)], np.int32),
+                    pages=[[list(r.pages[w]) for r in self.rows] for w in range(3)],
+                    next_page=list(self.next_page),
+                    live=np.array([r.live for r in self.rows], np.uint8),
+                    n_steps=np.array([r.n_steps for r in self.rows], np.int32))
