@@ -1,0 +1,214 @@
+/* rsd.h -- C ABI of the B200 (sm_100a) library for the batched step loop of Reward-Guided
+ * Speculative Decoding (RSD, arXiv 2501.19324, Algorithm 1).
+ *
+ * One context serves a batch of independent rows.  Per step and per live row the library
+ *   (1) decodes a draft step  y^_i <- m(x, y_{1:i-1})            (Algorithm 1, "Generate draft step"),
+ *   (2) scores it             r_i  <- r(y^_i | x, y_{1:i-1})     (Algorithm 1, "Compute reward"),
+ *   (3) gates it              accept iff r_i >= delta            (Table 1, binary step; Algorithm 2),
+ *   (4) re-decodes rejected rows with the target  y_i <- M(x, y_{1:i-1}),
+ *   (5) commits y_i and stops rows on EOS / step budget          (Algorithm 1, "if s in y_i: break").
+ * m, M and r are Llama-style decoder-only transformers; r carries a scalar head in place of
+ * lm_head (Appendix B.3) whose sigmoid lies in [0,1] (Section 3, "Models").
+ *
+ * Conventions
+ *   - Every function returns an int status: 0 = RSD_OK, negative = error.  Nothing throws, aborts
+ *     or exits.  rsd_last_error() returns a library-owned description of the last failure.
+ *   - "device" pointers are CUDA device pointers valid on the context's GPU; "host" pointers are
+ *     ordinary host memory.  The library allocates NO device memory: weights, KV pools and the
+ *     workspace are allocated by the caller and only borrowed until rsd_destroy().
+ *   - All work is enqueued on the stream given to each call.  Calls that return host values
+ *     synchronise that stream before returning.
+ *   - One context must be used by one host thread at a time.
+ *   - There is no CPU fallback: without a CUDA device every compute call fails with RSD_ERR_CUDA.
+ */
+#ifndef RSD_H
+#define RSD_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct rsd_ctx rsd_ctx; /* opaque, owned by the library */
+
+enum {
+  RSD_OK = 0,
+  RSD_ERR_ARG = -1,         /* bad argument / inconsistent shapes                         */
+  RSD_ERR_STATE = -2,       /* call out of order (e.g. step before prefill)               */
+  RSD_ERR_OOM_PAGES = -3,   /* a KV page pool or the workspace is too small               */
+  RSD_ERR_CUDA = -4,        /* a CUDA call failed; only rsd_destroy is valid afterwards   */
+  RSD_ERR_TIMEOUT = -5,     /* a bounded device-side wait expired                         */
+  RSD_ERR_UNSUPPORTED = -6  /* shape or option the kernels do not cover                   */
+};
+
+enum { RSD_F32 = 0, RSD_BF16 = 1 };
+enum { RSD_DRAFT = 0, RSD_PRM = 1, RSD_TARGET = 2 };
+enum { RSD_HEAD_LM = 0, RSD_HEAD_REWARD_SIGMOID = 1, RSD_HEAD_REWARD_RAW = 2 };
+
+/* Weighting functions omega(r) of Table 1, used by the acceptance criterion of Algorithm 2. */
+enum {
+  RSD_OMEGA_CONSTANT = 0, /* omega = p               (p passed as delta)                   */
+  RSD_OMEGA_STEP = 1,     /* omega = 1(r >= delta)   (the paper's default)                 */
+  RSD_OMEGA_CLIP = 2,     /* omega = min(1, max(0, r))                                     */
+  RSD_OMEGA_RATIO = 3,    /* omega = max(0, r / (1 + r))                                   */
+  RSD_OMEGA_LOGISTIC = 4  /* omega = 1 / (1 + exp(-alpha (r - delta)))                     */
+};
+
+/* One transformer.  All pointers are DEVICE pointers, borrowed, read-only, row-major, of element
+ * type `dtype` (fp32 or bfloat16), never copied or repacked by the library.
+ *   y = W x with W stored [out_features, in_features].                                      */
+typedef struct {
+  int32_t n_layers, d_model, n_heads, n_kv_heads, head_dim, d_ffn, vocab, dtype;
+  float rope_theta, rms_eps;
+  int32_t head_kind;          /* RSD_HEAD_*                                                  */
+  const void* tok_embed;      /* [vocab, d_model]                                            */
+  const void* final_norm;     /* [d_model]                                                   */
+  const void* head;           /* [vocab, d_model] (lm_head) or [d_model] (reward projection) */
+  const void* const* wqkv;    /* host array of n_layers device pointers:
+                                 [(H + 2 KV) * head_dim, d_model], rows = Wq | Wk | Wv       */
+  const void* const* wo;      /* per layer [d_model, H * head_dim]                           */
+  const void* const* wgu;     /* per layer [2 * d_ffn, d_model], rows = Wgate | Wup          */
+  const void* const* wdown;   /* per layer [d_model, d_ffn]                                  */
+  const void* const* norm1;   /* per layer [d_model], RMSNorm gain before attention          */
+  const void* const* norm2;   /* per layer [d_model], RMSNorm gain before the MLP            */
+} rsd_model;
+
+typedef struct {
+  int32_t max_batch;          /* rows B, 1..1024                                             */
+  int32_t max_seq_tokens;     /* per-row capacity of prompt + response                       */
+  int32_t max_step_tokens;    /* cap on the tokens of one step                               */
+  int32_t max_steps;          /* N of Algorithm 1: a row stops after this many steps         */
+  int32_t page_tokens;        /* KV page size; must be 16                                    */
+  int32_t step_end_id;        /* token that ends a step (the delimiter belongs to the step)  */
+  int32_t eos_id;             /* EOS token s of Algorithm 1; -1 = none                       */
+  int32_t step_end_mod;       /* 0 = off; m > 0: a token ends a step iff id % m == step_end_id % m */
+  float temperature;          /* 0 = greedy; > 0 = Gumbel-max sampling at this temperature   */
+  uint64_t seed;              /* Philox key of the sampling noise                            */
+  int32_t omega_kind;         /* RSD_OMEGA_*; RSD_OMEGA_STEP reproduces the paper's default  */
+  float omega_alpha;          /* alpha of RSD_OMEGA_LOGISTIC                                 */
+  int32_t max_chunk_tokens;   /* tokens pushed through a model per multi-token pass; 0 = 4096 */
+  int32_t debug_flags;        /* RSD_DEBUG_*                                                 */
+  /* caller-allocated device memory, sizes as reported by rsd_query_sizes (or larger)        */
+  void* kv_pool[3];           /* RSD_DRAFT / RSD_PRM / RSD_TARGET                            */
+  size_t kv_bytes[3];
+  void* workspace;
+  size_t workspace_bytes;
+} rsd_config;
+
+enum { RSD_DEBUG_KEEP_LOGITS = 1 /* keep every decode iteration's logits for rsd_debug_get_logits */ };
+
+/* Fills cfg->kv_bytes[] (enough pages for max_batch rows of max_seq_tokens) and
+ * cfg->workspace_bytes for these three models.  Host only.  RSD_ERR_ARG on bad shapes.       */
+int rsd_query_sizes(const rsd_model* draft, const rsd_model* prm, const rsd_model* target, rsd_config* cfg);
+
+/* Creates a context on the current CUDA device from a filled rsd_config.  The KV pools and the
+ * workspace must stay alive and untouched by the caller until rsd_destroy.                   */
+int rsd_create(const rsd_config* cfg, rsd_ctx** out);
+
+/* rsd_load_models(draft, prm, target): records the three borrowed weight sets, validates shapes
+ * (GQA divisibility, head_dim 64 or 128, K dimensions a multiple of the vector width) and lays
+ * out the workspace.  Sampling is restricted to ids below the smallest of the three vocabularies
+ * so every token is valid for every embedding.                                               */
+int rsd_load_models(rsd_ctx*, const rsd_model* draft, const rsd_model* prm, const rsd_model* target);
+
+/* rsd_prefill(prompts): starts B rows from ragged prompts (z_1 = x).  `tokens` is a HOST array of
+ * offsets[B] ids, row b owning [offsets[b], offsets[b+1]).  The draft caches each prompt without
+ * its last token, the PRM the whole prompt, the target nothing (it catches up when a row is first
+ * rejected).  Drops any rows of an earlier call.                                             */
+int rsd_prefill(rsd_ctx*, const int32_t* tokens, const int32_t* offsets, int32_t B, void* cuda_stream);
+
+/* rsd_step(delta): one pass of the loop body of Algorithm 1 over all rows.  Outputs are HOST
+ * arrays (any may be NULL): step_tokens [B, max_step_tokens] (y_i, zero padded), step_len [B],
+ * rewards [B] (r_i of the draft step), accept [B] (1 = draft step kept), live [B] (row continues).
+ * Rows that were already stopped report step_len 0, reward 0, accept 0.  Synchronises.       */
+int rsd_step(rsd_ctx*, float delta, void* cuda_stream, int32_t* step_tokens, int32_t* step_len,
+             float* rewards, uint8_t* accept, uint8_t* live);
+
+/* Counters of the work done since rsd_prefill / rsd_reset.  Index 0 draft, 1 PRM, 2 target.
+ * flops_paper follows Section 3.3: 2N per inference token of an N-parameter model (all
+ * parameters, embedding and head included), counting every token the draft or the target
+ * generated (discarded draft steps too) and every token the PRM processed.  flops_all_tokens
+ * bills 2N for every token pushed through any model, prompts and catch-up included.         */
+typedef struct {
+  uint64_t gen_tokens[3];
+  uint64_t ingest_tokens[3];
+  uint64_t score_tokens;
+  uint64_t steps, accepted_steps, rejected_steps, discarded_draft_tokens;
+  double flops_paper, flops_all_tokens;
+} rsd_counters;
+int rsd_flops_counters(rsd_ctx*, rsd_counters* out);
+
+int rsd_reset(rsd_ctx*);    /* drops rows and returns every KV page; keeps the models        */
+int rsd_destroy(rsd_ctx*);
+const char* rsd_last_error(const rsd_ctx*); /* ctx may be NULL: error of the last failed create */
+
+/* ---- parity hooks ------------------------------------------------------------------------- */
+
+/* Teacher forcing for the NEXT rsd_step only: tokens [B, max_step_tokens] and len [B] (HOST) replace
+ * what model `which` (RSD_DRAFT or RSD_TARGET) samples; len[b] = 0 leaves row b free.  The sampled
+ * ids remain readable through rsd_debug_get_sampled.  accept [B] (HOST, may be NULL; 0/1, other
+ * values = do not force) overrides the gate when which == RSD_PRM (tokens/len ignored).      */
+int rsd_debug_force(rsd_ctx*, int which, const int32_t* tokens, const int32_t* len, const uint8_t* accept);
+
+/* Logits of the last rsd_step's decode iterations of model `which`, when RSD_DEBUG_KEEP_LOGITS
+ * is set: out is a HOST array [B, max_step_tokens, vocab(which)] (row b, iteration j).        */
+int rsd_debug_get_logits(rsd_ctx*, int which, float* out);
+/* Ids sampled (before forcing) in the last rsd_step: HOST out [B, max_step_tokens].           */
+int rsd_debug_get_sampled(rsd_ctx*, int which, int32_t* out);
+
+/* Integer state, HOST outputs (any may be NULL): z_len [B], kv_len [3, B], n_pages [3, B],
+ * page_table [3, B, max_pages] with max_pages = ceil(max_seq_tokens / page_tokens), next_page [3],
+ * rej_idx [B] (ascending rejected rows of the last step, first *n_rej entries valid).         */
+int rsd_debug_get_state(rsd_ctx*, int32_t* z_len, int32_t* kv_len, int32_t* n_pages, int32_t* page_table,
+                        int32_t* next_page, int32_t* rej_idx, int32_t* n_rej);
+
+/* ---- single kernels (sweeps and unit parity); all pointers DEVICE unless noted ------------ */
+
+/* y[M, N] (fp32) = (accumulate ? y : 0) + x[M, K] * W[N, K]^T, W and x of element type `dtype`.
+ * impl: 0 = pick by shape, 1 = split-K SIMT GEMV path, 2 = tcgen05/TMEM/TMA path (bf16 only,
+ * K % 64 == 0, 16-byte aligned rows).  `scratch` (scratch_bytes from rsd_k_gemm_scratch_bytes)
+ * holds split-K partial sums and tile counters; the first 4 KiB must be zero before the first
+ * call and are left zero by every call.                                                      */
+int rsd_k_gemm(const void* W, const void* x, float* y, int32_t M, int32_t N, int32_t K, int32_t dtype,
+               int32_t accumulate, int32_t impl, void* scratch, size_t scratch_bytes, void* cuda_stream);
+size_t rsd_k_gemm_scratch_bytes(int32_t M, int32_t N, int32_t K);
+
+/* Paged-KV grouped-query decode attention: one query per row.  q [B, H, hd] fp32, kv pool laid out
+ * [page][2 (K,V)][KV][page_tokens][hd] of `dtype`, page_table [B, max_pages], ctx_len [B] (number
+ * of cached positions attended, >= 1), out [B, H, hd] fp32.                                   */
+int rsd_k_attn_decode(const float* q, const void* kv_pool, const int32_t* page_table, const int32_t* ctx_len,
+                      float* out, int32_t B, int32_t H, int32_t KV, int32_t hd, int32_t max_pages,
+                      int32_t dtype, void* scratch, size_t scratch_bytes, void* cuda_stream);
+size_t rsd_k_attn_decode_scratch_bytes(int32_t B, int32_t H, int32_t hd, int32_t max_ctx);
+
+/* Gate + compaction (Table 1 binary step; Algorithm 1 else-branch batched over rows):
+ * accept[b] = live[b] && rewards[b] >= delta; rej_idx [B] receives the ascending list of live
+ * rejected rows, *n_rej (device) their count.  B up to 2^24.  scratch: 4 * ceil(B / 1024) bytes. */
+int rsd_k_gate_compact(const float* rewards, const uint8_t* live, float delta, uint8_t* accept,
+                       int32_t* rej_idx, int32_t* n_rej, int32_t B, void* scratch, size_t scratch_bytes,
+                       void* cuda_stream);
+
+/* out[t, :] = x[t, :] * gain / sqrt(mean(x^2) + eps), x fp32 [T, d], out of element type `dtype`. */
+int rsd_k_rmsnorm(const float* x, const void* gain, void* out, int32_t T, int32_t d, float eps,
+                  int32_t dtype, void* cuda_stream);
+/* Rotary embedding in place on v [T, n_heads, hd] fp32 at positions pos [T]: pairs (i, i + hd/2). */
+int rsd_k_rope(float* v, const int32_t* pos, int32_t T, int32_t n_heads, int32_t hd, float theta,
+               void* cuda_stream);
+/* out[t, f] = silu(gu[t, f]) * gu[t, F + f]; gu fp32 [T, 2F], out of element type `dtype`.     */
+int rsd_k_swiglu(const float* gu, void* out, int32_t T, int32_t F, int32_t dtype, void* cuda_stream);
+/* token[b] = argmax over v < v_limit of logits[b, v] / T + g, g = -log(-log u) with u the Philox
+ * uniform of (seed; counter = (v / 4, pos[b] + 1, row[b], model_id), word v % 4), or the plain
+ * argmax when temperature == 0; ties to the lowest id.  pos[b] is the position of the token fed to
+ * the model, the sampled token sits at pos[b] + 1.  row[b] < 0 skips slot b.  logits fp32 [B, V]. */
+int rsd_k_sample(const float* logits, int32_t B, int32_t V, int32_t v_limit, float temperature,
+                 uint64_t seed, int32_t model_id, const int32_t* row, const int32_t* pos, int32_t* token,
+                 void* cuda_stream);
+/* Philox4x32-10 blocks: out[i] = philox(ctr[i], key), ctr [n, 4], key [2], out [n, 4] (uint32). */
+int rsd_k_philox(const uint32_t* ctr, const uint32_t* key, uint32_t* out, int32_t n, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RSD_H */

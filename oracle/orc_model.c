@@ -195,8 +195,9 @@ void orc_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t ou
   memcpy(out, c, sizeof(c));
 }
 
-/* 32 random bits -> uniform on (0,1): the top 24 bits, centred in their cell. */
-double orc_uniform_from_bits(uint32_t x) { return ((double)(x >> 8) + 0.5) * (1.0 / 16777216.0); }
+/* 32 random bits -> uniform on (0,1): the top 23 bits, centred in their cell, so that the value
+ * (2k+1) / 2^24 is also exact in fp32 and never 0 or 1. */
+double orc_uniform_from_bits(uint32_t x) { return ((double)(x >> 9) + 0.5) * (1.0 / 8388608.0); }
 
 /* Uniform draw attached to (seed, stream, row, position, index): counter = (index/4, position,
  * row, stream), key = the two halves of the seed, word index%4 of the block. */

@@ -109,18 +109,21 @@ class OracleRSD:
             for which in (DRAFT, PRM, TARGET):
                 row.caches[which] = self.models[which].new_cache(self.cfg.max_seq_tokens)
             self.rows.append(row)
-        for b, row in enumerate(self.rows):
-            self._reserve(DRAFT, b, len(row.z) - 1)
-        for b, row in enumerate(self.rows):
-            self._reserve(PRM, b, len(row.z))
-        for b, row in enumerate(self.rows):
+        for row in self.rows:
+            if len(row.z) + self.cfg.max_step_tokens > self.cfg.max_seq_tokens:
+                row.live = False        # no room for even one step: the row never starts
+        live_rows = [b for b, row in enumerate(self.rows) if row.live]
+        for b in live_rows:
+            self._reserve(DRAFT, b, len(self.rows[b].z) - 1)
+        for b in live_rows:
+            self._reserve(PRM, b, len(self.rows[b].z))
+        for b in live_rows:
+            row = self.rows[b]
             n = len(row.z)
             self._ingest(DRAFT, b, n - 1, row.z)
             self._ingest(PRM, b, n, row.z)
             self.counters["ingest_tokens"][DRAFT] += n - 1
             self.counters["ingest_tokens"][PRM] += n
-            if n + self.cfg.max_step_tokens > self.cfg.max_seq_tokens:
-                row.live = False
 
     def _generate_step(self, which: int, b: int, forced=None, trace=None) -> list:
         """One step from model `which` given the row's context z (Algorithm 1: m(x, y_{1:i-1}) or

@@ -1,0 +1,737 @@
+// C ABI of the RSD step-loop library: context, workspace layout, and the orchestration of one
+// prefill / one step (Algorithm 1 batched over rows) as kernel launches on the caller's stream.
+#include "../../include/rsd.h"
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "kernels.cuh"
+
+using namespace rsd;
+
+namespace {
+
+std::string g_create_error;
+
+struct ModelHost {
+  rsd_model m{};
+  std::vector<const void*> wqkv, wo, wgu, wdown, norm1, norm2;
+  size_t elem = 4;
+  float2* rope = nullptr;
+  char* kv_pool = nullptr;
+  size_t layer_stride = 0;  // bytes of one layer's slab
+  int pool_pages = 0;
+  double n_params = 0;
+};
+
+// Host-visible scalars mirrored from the device after each phase boundary.
+struct Scalars {
+  int32_t n_tok, n_rej, err, n_active, n_slots, next_page[3];
+};
+
+struct Layout {
+  size_t bytes = 0;
+  size_t take(size_t n) {
+    size_t off = bytes;
+    bytes += (n + 255) & ~(size_t)255;
+    return off;
+  }
+};
+
+}  // namespace
+
+struct rsd_ctx {
+  rsd_config cfg{};
+  ModelHost mdl[3];
+  bool loaded = false, prefilled = false, poisoned = false;
+  RowState st{};
+  LoopParams lp{};
+  int B_max = 0, S = 0, C = 0, max_pages = 0, chunk = 0, v_limit = 0, T_max = 0;
+  // activations (workspace)
+  float *x = nullptr, *qkv = nullptr, *q = nullptr, *gu = nullptr, *logits = nullptr;
+  void *h = nullptr, *attn = nullptr, *act = nullptr;
+  int32_t* sampled_slots = nullptr;
+  float* dbg_logits[2] = {nullptr, nullptr};
+  int32_t* d_scalars = nullptr;  // device block holding n_tok, n_rej, err, n_active, n_slots, next_page[3]
+  // staging of step outputs (device) and their pinned host mirrors
+  int32_t *o_tokens = nullptr, *o_len = nullptr;
+  float* o_rewards = nullptr;
+  uint8_t *o_accept = nullptr, *o_live = nullptr;
+  char* pinned = nullptr;
+  size_t pinned_bytes = 0;
+  void* gemm_scratch = nullptr;
+  size_t gemm_scratch_bytes = 0;
+  rsd_counters ctr{};
+  int last_n_rej = 0;
+  std::string err;
+};
+
+namespace {
+
+int fail(rsd_ctx* c, int code, const char* fmt, const char* detail = "") {
+  char buf[512];
+  snprintf(buf, sizeof(buf), fmt, detail);
+  if (c) c->err = buf; else g_create_error = buf;
+  return code;
+}
+
+#define CU(call)                                                                        \
+  do {                                                                                  \
+    cudaError_t e_ = (call);                                                            \
+    if (e_ != cudaSuccess) {                                                            \
+      c->poisoned = true;                                                               \
+      return fail(c, RSD_ERR_CUDA, "CUDA error: %s", cudaGetErrorString(e_));           \
+    }                                                                                   \
+  } while (0)
+
+int check_model(const rsd_model* m, const char** why) {
+  *why = "";
+  if (!m) { *why = "null model"; return RSD_ERR_ARG; }
+  if (m->n_layers < 1 || m->d_model < 8 || m->n_heads < 1 || m->n_kv_heads < 1 || m->d_ffn < 8 || m->vocab < 1) {
+    *why = "non-positive dimension"; return RSD_ERR_ARG;
+  }
+  if (m->n_heads % m->n_kv_heads != 0) { *why = "n_heads not a multiple of n_kv_heads"; return RSD_ERR_ARG; }
+  if (m->dtype != RSD_F32 && m->dtype != RSD_BF16) { *why = "dtype"; return RSD_ERR_ARG; }
+  if (m->head_dim != 64 && m->head_dim != 128) { *why = "head_dim must be 64 or 128"; return RSD_ERR_UNSUPPORTED; }
+  const int vec = m->dtype == RSD_BF16 ? 8 : 4;
+  if (m->d_model % vec || m->d_ffn % vec || (m->n_heads * m->head_dim) % vec) {
+    *why = "inner dimensions must be multiples of a 16-byte vector"; return RSD_ERR_UNSUPPORTED;
+  }
+  if (m->head_kind < 0 || m->head_kind > 2) { *why = "head_kind"; return RSD_ERR_ARG; }
+  return RSD_OK;
+}
+
+double count_params(const rsd_model& m) {
+  const double d = m.d_model, hd = m.head_dim;
+  const double per_layer = d * m.n_heads * hd + 2 * d * m.n_kv_heads * hd + m.n_heads * hd * d + 3 * d * m.d_ffn + 2 * d;
+  const double head = m.head_kind == RSD_HEAD_LM ? (double)m.vocab * d : d;
+  return (double)m.vocab * d + m.n_layers * per_layer + d + head;
+}
+
+size_t kv_pool_bytes(const rsd_model& m, int pages) {
+  const size_t elem = m.dtype == RSD_BF16 ? 2 : 4;
+  return (size_t)pages * m.n_layers * 2 * m.n_kv_heads * kPageTokens * m.head_dim * elem;
+}
+
+struct Dims {
+  int d = 0, qkv = 0, hq = 0, f = 0, v = 0, hd = 0;
+};
+
+Dims max_dims(const rsd_model* const ms[3]) {
+  Dims r;
+  for (int i = 0; i < 3; ++i) {
+    const rsd_model& m = *ms[i];
+    r.d = std::max(r.d, m.d_model);
+    r.qkv = std::max(r.qkv, (m.n_heads + 2 * m.n_kv_heads) * m.head_dim);
+    r.hq = std::max(r.hq, m.n_heads * m.head_dim);
+    r.f = std::max(r.f, m.d_ffn);
+    if (m.head_kind == RSD_HEAD_LM) r.v = std::max(r.v, m.vocab);
+    r.hd = std::max(r.hd, m.head_dim);
+  }
+  return r;
+}
+
+// Lays out the workspace; with c == nullptr only the size is computed.
+size_t layout_workspace(const rsd_config& cfg, const rsd_model* const ms[3], rsd_ctx* c) {
+  Layout L;
+  const int B = cfg.max_batch, S = cfg.max_seq_tokens, C = cfg.max_step_tokens;
+  const int max_pages = (S + kPageTokens - 1) / kPageTokens;
+  const int chunk = cfg.max_chunk_tokens > 0 ? cfg.max_chunk_tokens : 4096;
+  const int T = std::max(B, chunk);
+  const Dims dm = max_dims(ms);
+  char* base = c ? (char*)cfg.workspace : nullptr;
+  auto P = [&](size_t off) -> char* { return base ? base + off : nullptr; };
+#define TAKE(type, n) (type*)P(L.take(sizeof(type) * (size_t)(n)))
+  // row state
+  RowState st{};
+  st.B = 0; st.S = S; st.C = C; st.max_pages = max_pages;
+  st.z_len = TAKE(int32_t, B); st.live = TAKE(int32_t, B); st.n_steps = TAKE(int32_t, B);
+  st.tok = TAKE(int32_t, (size_t)B * S);
+  for (int w = 0; w < 3; ++w) {
+    st.kv_len[w] = TAKE(int32_t, B);
+    st.n_pages[w] = TAKE(int32_t, B);
+    st.page_table[w] = TAKE(int32_t, (size_t)B * max_pages);
+  }
+  for (int p = 0; p < 2; ++p) {
+    st.gen_len[p] = TAKE(int32_t, B);
+    st.gen_tok[p] = TAKE(int32_t, (size_t)B * C);
+    st.sampled[p] = TAKE(int32_t, (size_t)B * C);
+    st.forced_tok[p] = TAKE(int32_t, (size_t)B * C);
+    st.forced_len[p] = TAKE(int32_t, B);
+  }
+  st.forced_accept = TAKE(uint8_t, B);
+  st.gen_active = TAKE(int32_t, B);
+  st.rewards = TAKE(float, B);
+  st.accept = TAKE(uint8_t, B);
+  st.rej_idx = TAKE(int32_t, B);
+  st.slot_row = TAKE(int32_t, B);
+  st.last_idx = TAKE(int32_t, B);
+  int32_t* scal = TAKE(int32_t, 16);
+  st.n_tok = scal + 0; st.n_rej = scal + 1; st.err = scal + 2; st.n_active = scal + 3; st.n_slots = scal + 4;
+  st.next_page = scal + 5;
+  st.pass_capacity = B * S;
+  st.pass_tok_id = TAKE(int32_t, (size_t)B * S);
+  st.pass_tok_row = TAKE(int32_t, (size_t)B * S);
+  st.pass_tok_pos = TAKE(int32_t, (size_t)B * S);
+  // activations
+  float* x = TAKE(float, (size_t)T * dm.d);
+  void* h = TAKE(float, (size_t)T * dm.d);
+  float* qkv = TAKE(float, (size_t)T * dm.qkv);
+  float* q = TAKE(float, (size_t)T * dm.hq);
+  void* attn = TAKE(float, (size_t)T * dm.hq);
+  float* gu = TAKE(float, (size_t)T * 2 * dm.f);
+  void* act = TAKE(float, (size_t)T * dm.f);
+  float* logits = TAKE(float, (size_t)B * dm.v);
+  int32_t* sampled_slots = TAKE(int32_t, B);
+  float2* rope[3];
+  for (int w = 0; w < 3; ++w) rope[w] = TAKE(float2, (size_t)S * (ms[w]->head_dim / 2));
+  float* dbg[2] = {nullptr, nullptr};
+  if (cfg.debug_flags & RSD_DEBUG_KEEP_LOGITS) {
+    dbg[0] = TAKE(float, (size_t)B * C * ms[RSD_DRAFT]->vocab);
+    dbg[1] = TAKE(float, (size_t)B * C * ms[RSD_TARGET]->vocab);
+  }
+  int32_t* o_tokens = TAKE(int32_t, (size_t)B * C);
+  int32_t* o_len = TAKE(int32_t, B);
+  float* o_rewards = TAKE(float, B);
+  uint8_t* o_accept = TAKE(uint8_t, B);
+  uint8_t* o_live = TAKE(uint8_t, B);
+  const size_t gs = gemm_scratch_bytes(T);
+  void* gscr = TAKE(char, gs);
+#undef TAKE
+  if (c) {
+    c->st = st; c->B_max = B; c->S = S; c->C = C; c->max_pages = max_pages; c->chunk = chunk; c->T_max = T;
+    c->x = x; c->h = h; c->qkv = qkv; c->q = q; c->attn = attn; c->gu = gu; c->act = act; c->logits = logits;
+    c->sampled_slots = sampled_slots;
+    for (int w = 0; w < 3; ++w) c->mdl[w].rope = rope[w];
+    c->dbg_logits[0] = dbg[0]; c->dbg_logits[1] = dbg[1];
+    c->d_scalars = scal;
+    c->o_tokens = o_tokens; c->o_len = o_len; c->o_rewards = o_rewards; c->o_accept = o_accept; c->o_live = o_live;
+    c->gemm_scratch = gscr; c->gemm_scratch_bytes = gs;
+  }
+  return L.bytes;
+}
+
+int check_config(const rsd_config* cfg, const char** why) {
+  *why = "";
+  if (!cfg) { *why = "null config"; return RSD_ERR_ARG; }
+  if (cfg->max_batch < 1 || cfg->max_batch > kMaxBatch) { *why = "max_batch out of 1..1024"; return RSD_ERR_ARG; }
+  if (cfg->page_tokens != kPageTokens) { *why = "page_tokens must be 16"; return RSD_ERR_UNSUPPORTED; }
+  if (cfg->max_step_tokens < 1 || cfg->max_steps < 1 || cfg->max_seq_tokens < 2) { *why = "step/sequence limits"; return RSD_ERR_ARG; }
+  if (cfg->temperature < 0.f) { *why = "temperature"; return RSD_ERR_ARG; }
+  if (cfg->omega_kind < 0 || cfg->omega_kind > 4) { *why = "omega_kind"; return RSD_ERR_ARG; }
+  if (cfg->step_end_mod < 0) { *why = "step_end_mod"; return RSD_ERR_ARG; }
+  return RSD_OK;
+}
+
+// ---- device scalars <-> host ---------------------------------------------------------------
+int read_scalars(rsd_ctx* c, cudaStream_t s, Scalars* out) {
+  CU(cudaMemcpyAsync(c->pinned, c->d_scalars, sizeof(Scalars), cudaMemcpyDeviceToHost, s));
+  CU(cudaStreamSynchronize(s));
+  memcpy(out, c->pinned, sizeof(Scalars));
+  if (out->err == RSD_ERR_OOM_PAGES) return fail(c, RSD_ERR_OOM_PAGES, "KV page pool or pass list exhausted%s");
+  if (out->err != 0) { c->poisoned = true; return fail(c, RSD_ERR_TIMEOUT, "device-side error flag raised%s"); }
+  return RSD_OK;
+}
+
+// ---- one model pass over T token slots ------------------------------------------------------
+int gemm(rsd_ctx* c, const ModelHost& M, const void* W, const void* xin, float* y, int Mrows, int N, int K,
+         int accumulate, const int32_t* n_active, cudaStream_t s) {
+  CU(launch_gemm(M.m.dtype, W, xin, y, Mrows, N, K, accumulate, 0, c->gemm_scratch, c->gemm_scratch_bytes, n_active, s));
+  return RSD_OK;
+}
+
+int forward_pass(rsd_ctx* c, int which, PassView p, cudaStream_t s) {
+  const ModelHost& M = c->mdl[which];
+  const rsd_model& m = M.m;
+  const int d = m.d_model, H = m.n_heads, KV = m.n_kv_heads, hd = m.head_dim, F = m.d_ffn;
+  const int T = p.T;
+  if (T <= 0) return RSD_OK;
+  CU(launch_embed(m.dtype, m.tok_embed, p, c->x, d, s));
+  for (int l = 0; l < m.n_layers; ++l) {
+    KvView kv{M.kv_pool + (size_t)l * M.layer_stride, c->st.page_table[which], c->max_pages};
+    CU(launch_rmsnorm(m.dtype, c->x, M.norm1[l], c->h, T, d, m.rms_eps, nullptr, p.n_active, s));
+    int rc = gemm(c, M, M.wqkv[l], c->h, c->qkv, T, (H + 2 * KV) * hd, d, 0, p.n_active, s);
+    if (rc) return rc;
+    CU(launch_rope_kv(m.dtype, c->qkv, p, c->q, kv, M.rope, H, KV, hd, s));
+    CU(launch_attn_generic(m.dtype, c->q, p, kv, c->attn, H, KV, hd, s));
+    rc = gemm(c, M, M.wo[l], c->attn, c->x, T, d, H * hd, 1, p.n_active, s);
+    if (rc) return rc;
+    CU(launch_rmsnorm(m.dtype, c->x, M.norm2[l], c->h, T, d, m.rms_eps, nullptr, p.n_active, s));
+    rc = gemm(c, M, M.wgu[l], c->h, c->gu, T, 2 * F, d, 0, p.n_active, s);
+    if (rc) return rc;
+    CU(launch_swiglu(m.dtype, c->gu, c->act, T, F, p.n_active, s));
+    rc = gemm(c, M, M.wdown[l], c->act, c->x, T, d, F, 1, p.n_active, s);
+    if (rc) return rc;
+  }
+  return RSD_OK;
+}
+
+// Multi-token pass over the flat list built by launch_build_pass, `chunk` tokens at a time.
+int run_ingest(rsd_ctx* c, int which, int n_total, bool want_reward, cudaStream_t s) {
+  for (int c0 = 0; c0 < n_total; c0 += c->chunk) {
+    const int Tc = std::min(c->chunk, n_total - c0);
+    PassView p{c->st.pass_tok_id + c0, c->st.pass_tok_row + c0, c->st.pass_tok_pos + c0, Tc, nullptr};
+    int rc = forward_pass(c, which, p, s);
+    if (rc) return rc;
+    if (want_reward) {
+      const rsd_model& m = c->mdl[which].m;
+      CU(launch_reward(m.dtype, c->x, m.final_norm, m.head, m.head_kind, c->st.last_idx, c0, Tc, m.d_model, m.rms_eps,
+                       c->st.rewards, c->st.B, s));
+    }
+  }
+  return RSD_OK;
+}
+
+__global__ void scatter_logits_kernel(const float* logits, const int32_t* slot_row, float* dbg, int V, int C, int iter,
+                                      const int32_t* n_active) {
+  if (*n_active == 0) return;
+  const int row = slot_row[blockIdx.x];
+  if (row < 0) return;
+  const float* src = logits + (size_t)blockIdx.x * V;
+  float* dst = dbg + ((size_t)row * C + iter) * V;
+  for (int i = threadIdx.x; i < V; i += blockDim.x) dst[i] = src[i];
+}
+
+// One decode phase: up to C iterations of (prepare, model pass, lm_head, sample, append).
+int decode_phase(rsd_ctx* c, int which, int phase, int n_slots, cudaStream_t s) {
+  const ModelHost& M = c->mdl[which];
+  const rsd_model& m = M.m;
+  CU(launch_decode_begin(c->st, phase, s));
+  if (n_slots <= 0) return RSD_OK;
+  for (int j = 0; j < c->C; ++j) {
+    CU(launch_decode_prepare(c->st, which, n_slots, s));
+    PassView p{c->st.pass_tok_id, c->st.pass_tok_row, c->st.pass_tok_pos, n_slots, c->st.n_active};
+    int rc = forward_pass(c, which, p, s);
+    if (rc) return rc;
+    CU(launch_rmsnorm(m.dtype, c->x, m.final_norm, c->h, n_slots, m.d_model, m.rms_eps, nullptr, p.n_active, s));
+    rc = gemm(c, M, m.head, c->h, c->logits, n_slots, m.vocab, m.d_model, 0, p.n_active, s);
+    if (rc) return rc;
+    if (c->dbg_logits[phase]) {
+      scatter_logits_kernel<<<n_slots, 256, 0, s>>>(c->logits, c->st.pass_tok_row, c->dbg_logits[phase], m.vocab, c->C, j, c->st.n_active);
+      CU(cudaGetLastError());
+    }
+    SampleArgs a{c->logits, n_slots, m.vocab, c->v_limit, c->cfg.temperature, c->cfg.seed, which,
+                 c->st.pass_tok_row, c->st.pass_tok_pos, c->sampled_slots, c->st.n_active};
+    CU(launch_sample(a, s));
+    CU(launch_decode_update(c->st, which, phase, j, c->sampled_slots, n_slots, c->lp, s));
+  }
+  return RSD_OK;
+}
+
+__global__ void init_rows_kernel(RowState st, const int32_t* flat, const int32_t* offsets, int B) {
+  const int b = blockIdx.x;
+  const int o = offsets[b], n = offsets[b + 1] - o;
+  for (int i = threadIdx.x; i < n; i += blockDim.x) st.tok[(size_t)b * st.S + i] = flat[o + i];
+  if (threadIdx.x == 0) {
+    st.z_len[b] = n;
+    st.live[b] = (n >= 1 && n + st.C <= st.S) ? 1 : 0;
+    st.n_steps[b] = 0;
+    for (int w = 0; w < 3; ++w) { st.kv_len[w][b] = 0; st.n_pages[w][b] = 0; }
+    for (int p = 0; p < 2; ++p) { st.gen_len[p][b] = 0; st.forced_len[p][b] = 0; }
+    st.forced_accept[b] = 255;
+    st.rewards[b] = 0.f;
+    st.accept[b] = 0;
+  }
+}
+
+int clear_forcing(rsd_ctx* c, cudaStream_t s) {
+  CU(cudaMemsetAsync(c->st.forced_len[0], 0, sizeof(int32_t) * c->B_max, s));
+  CU(cudaMemsetAsync(c->st.forced_len[1], 0, sizeof(int32_t) * c->B_max, s));
+  CU(cudaMemsetAsync(c->st.forced_accept, 255, c->B_max, s));
+  return RSD_OK;
+}
+
+}  // namespace
+
+// =================================================================================================
+// C ABI
+// =================================================================================================
+extern "C" {
+
+int rsd_query_sizes(const rsd_model* draft, const rsd_model* prm, const rsd_model* target, rsd_config* cfg) {
+  const char* why;
+  int rc = check_config(cfg, &why);
+  if (rc) return fail(nullptr, rc, "config: %s", why);
+  const rsd_model* ms[3] = {draft, prm, target};
+  for (int i = 0; i < 3; ++i) {
+    rc = check_model(ms[i], &why);
+    if (rc) return fail(nullptr, rc, "model: %s", why);
+  }
+  const int max_pages = (cfg->max_seq_tokens + kPageTokens - 1) / kPageTokens;
+  for (int i = 0; i < 3; ++i) cfg->kv_bytes[i] = kv_pool_bytes(*ms[i], cfg->max_batch * max_pages);
+  cfg->workspace_bytes = layout_workspace(*cfg, ms, nullptr);
+  return RSD_OK;
+}
+
+int rsd_create(const rsd_config* cfg, rsd_ctx** out) {
+  const char* why;
+  if (!out) return fail(nullptr, RSD_ERR_ARG, "null output pointer%s");
+  *out = nullptr;
+  int rc = check_config(cfg, &why);
+  if (rc) return fail(nullptr, rc, "config: %s", why);
+  if (!cfg->workspace || !cfg->kv_pool[0] || !cfg->kv_pool[1] || !cfg->kv_pool[2])
+    return fail(nullptr, RSD_ERR_ARG, "workspace and KV pools must be provided by the caller%s");
+  int dev_count = 0;
+  if (cudaGetDeviceCount(&dev_count) != cudaSuccess || dev_count == 0)
+    return fail(nullptr, RSD_ERR_CUDA, "no CUDA device: this library has no CPU fallback%s");
+  rsd_ctx* c = new (std::nothrow) rsd_ctx();
+  if (!c) return fail(nullptr, RSD_ERR_ARG, "out of host memory%s");
+  c->cfg = *cfg;
+  c->pinned_bytes = 4096 + (size_t)cfg->max_batch * (cfg->max_step_tokens * 4 + 64);
+  if (cudaHostAlloc((void**)&c->pinned, c->pinned_bytes, cudaHostAllocDefault) != cudaSuccess) {
+    delete c;
+    return fail(nullptr, RSD_ERR_CUDA, "pinned host allocation failed%s");
+  }
+  c->lp.step_end_id = cfg->step_end_id; c->lp.eos_id = cfg->eos_id; c->lp.step_end_mod = cfg->step_end_mod;
+  c->lp.max_steps = cfg->max_steps; c->lp.omega_kind = cfg->omega_kind; c->lp.omega_alpha = cfg->omega_alpha;
+  c->lp.seed = cfg->seed;
+  *out = c;
+  return RSD_OK;
+}
+
+int rsd_load_models(rsd_ctx* c, const rsd_model* draft, const rsd_model* prm, const rsd_model* target) {
+  if (!c) return RSD_ERR_ARG;
+  if (c->poisoned) return fail(c, RSD_ERR_STATE, "context unusable after a CUDA error%s");
+  const rsd_model* ms[3] = {draft, prm, target};
+  const char* why;
+  for (int i = 0; i < 3; ++i) {
+    int rc = check_model(ms[i], &why);
+    if (rc) return fail(c, rc, "model: %s", why);
+    if (!ms[i]->tok_embed || !ms[i]->final_norm || !ms[i]->head || !ms[i]->wqkv || !ms[i]->wo || !ms[i]->wgu ||
+        !ms[i]->wdown || !ms[i]->norm1 || !ms[i]->norm2)
+      return fail(c, RSD_ERR_ARG, "model: null weight pointer%s");
+  }
+  if (draft->head_kind != RSD_HEAD_LM || target->head_kind != RSD_HEAD_LM || prm->head_kind == RSD_HEAD_LM)
+    return fail(c, RSD_ERR_ARG, "draft and target need lm heads, the PRM a scalar head%s");
+  const size_t need = layout_workspace(c->cfg, ms, nullptr);
+  if (need > c->cfg.workspace_bytes) return fail(c, RSD_ERR_OOM_PAGES, "workspace smaller than rsd_query_sizes reports%s");
+  layout_workspace(c->cfg, ms, c);
+  const int max_pages = c->max_pages;
+  for (int w = 0; w < 3; ++w) {
+    ModelHost& M = c->mdl[w];
+    M.m = *ms[w];
+    const int L = M.m.n_layers;
+    M.wqkv.assign(ms[w]->wqkv, ms[w]->wqkv + L); M.wo.assign(ms[w]->wo, ms[w]->wo + L);
+    M.wgu.assign(ms[w]->wgu, ms[w]->wgu + L); M.wdown.assign(ms[w]->wdown, ms[w]->wdown + L);
+    M.norm1.assign(ms[w]->norm1, ms[w]->norm1 + L); M.norm2.assign(ms[w]->norm2, ms[w]->norm2 + L);
+    M.m.wqkv = M.wqkv.data(); M.m.wo = M.wo.data(); M.m.wgu = M.wgu.data(); M.m.wdown = M.wdown.data();
+    M.m.norm1 = M.norm1.data(); M.m.norm2 = M.norm2.data();
+    M.elem = M.m.dtype == RSD_BF16 ? 2 : 4;
+    M.n_params = count_params(M.m);
+    M.kv_pool = (char*)c->cfg.kv_pool[w];
+    const size_t page_bytes = (size_t)2 * M.m.n_kv_heads * kPageTokens * M.m.head_dim * M.elem;
+    int pages = (int)std::min<size_t>(c->cfg.kv_bytes[w] / (page_bytes * L), (size_t)c->B_max * max_pages);
+    if (pages < 1) return fail(c, RSD_ERR_OOM_PAGES, "KV pool too small for a single page%s");
+    M.pool_pages = pages;
+    M.layer_stride = (size_t)pages * page_bytes;
+    c->st.pool_pages[w] = pages;
+  }
+  c->v_limit = std::min(std::min(draft->vocab, prm->vocab), target->vocab);
+  cudaStream_t s = 0;
+  for (int w = 0; w < 3; ++w)
+    CU(launch_rope_table(c->mdl[w].rope, c->S, c->mdl[w].m.head_dim, c->mdl[w].m.rope_theta, s));
+  CU(cudaMemsetAsync(c->d_scalars, 0, 16 * sizeof(int32_t), s));
+  CU(cudaMemsetAsync(c->gemm_scratch, 0, c->gemm_scratch_bytes, s));
+  int rc = clear_forcing(c, s);
+  if (rc) return rc;
+  CU(cudaStreamSynchronize(s));
+  c->loaded = true;
+  c->prefilled = false;
+  return RSD_OK;
+}
+
+int rsd_reset(rsd_ctx* c) {
+  if (!c) return RSD_ERR_ARG;
+  if (c->poisoned) return fail(c, RSD_ERR_STATE, "context unusable after a CUDA error%s");
+  if (!c->loaded) return fail(c, RSD_ERR_STATE, "no models loaded%s");
+  CU(cudaDeviceSynchronize());
+  CU(cudaMemset(c->d_scalars, 0, 16 * sizeof(int32_t)));
+  c->st.B = 0;
+  c->prefilled = false;
+  memset(&c->ctr, 0, sizeof(c->ctr));
+  return RSD_OK;
+}
+
+int rsd_prefill(rsd_ctx* c, const int32_t* tokens, const int32_t* offsets, int32_t B, void* cuda_stream) {
+  if (!c) return RSD_ERR_ARG;
+  if (c->poisoned) return fail(c, RSD_ERR_STATE, "context unusable after a CUDA error%s");
+  if (!c->loaded) return fail(c, RSD_ERR_STATE, "rsd_prefill before rsd_load_models%s");
+  if (!tokens || !offsets || B < 1 || B > c->B_max) return fail(c, RSD_ERR_ARG, "prefill: bad batch%s");
+  if (offsets[0] != 0) return fail(c, RSD_ERR_ARG, "prefill: offsets[0] must be 0%s");
+  for (int b = 0; b < B; ++b) {
+    const int n = offsets[b + 1] - offsets[b];
+    if (n < 1 || n > c->S) return fail(c, RSD_ERR_ARG, "prefill: prompt length out of 1..max_seq_tokens%s");
+  }
+  const int total = offsets[B];
+  for (int i = 0; i < total; ++i)
+    if (tokens[i] < 0 || tokens[i] >= c->v_limit) return fail(c, RSD_ERR_ARG, "prefill: token id out of range%s");
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  int rc = rsd_reset(c);
+  if (rc) return rc;
+  c->st.B = B;
+  // stage the ragged prompt in the pass-list buffers, then scatter it into the row buffers
+  CU(cudaMemcpyAsync(c->st.pass_tok_id, tokens, sizeof(int32_t) * total, cudaMemcpyHostToDevice, s));
+  CU(cudaMemcpyAsync(c->st.pass_tok_row, offsets, sizeof(int32_t) * (B + 1), cudaMemcpyHostToDevice, s));
+  init_rows_kernel<<<B, 128, 0, s>>>(c->st, c->st.pass_tok_id, c->st.pass_tok_row, B);
+  CU(cudaGetLastError());
+  CU(cudaStreamSynchronize(s));  // the staging buffers are reused below
+  CU(launch_reserve_pages(c->st, RSD_DRAFT, kReservePrefillDraft, s));
+  CU(launch_reserve_pages(c->st, RSD_PRM, kReservePrefillPrm, s));
+  Scalars sc;
+  CU(launch_build_pass(c->st, RSD_DRAFT, kPassIngestDraft, s));
+  rc = read_scalars(c, s, &sc);
+  if (rc) return rc;
+  rc = run_ingest(c, RSD_DRAFT, sc.n_tok, false, s);
+  if (rc) return rc;
+  c->ctr.ingest_tokens[RSD_DRAFT] += sc.n_tok;
+  CU(launch_build_pass(c->st, RSD_PRM, kPassScorePrm, s));
+  rc = read_scalars(c, s, &sc);
+  if (rc) return rc;
+  rc = run_ingest(c, RSD_PRM, sc.n_tok, false, s);
+  if (rc) return rc;
+  c->ctr.ingest_tokens[RSD_PRM] += sc.n_tok;
+  CU(cudaStreamSynchronize(s));
+  c->prefilled = true;
+  return RSD_OK;
+}
+
+int rsd_step(rsd_ctx* c, float delta, void* cuda_stream, int32_t* step_tokens, int32_t* step_len, float* rewards,
+             uint8_t* accept, uint8_t* live) {
+  if (!c) return RSD_ERR_ARG;
+  if (c->poisoned) return fail(c, RSD_ERR_STATE, "context unusable after a CUDA error%s");
+  if (!c->prefilled) return fail(c, RSD_ERR_STATE, "rsd_step before rsd_prefill%s");
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  const int B = c->st.B;
+  Scalars sc;
+  int rc;
+  // draft: catch up on a step the target wrote last time, then decode y^_i
+  CU(launch_reserve_pages(c->st, RSD_DRAFT, kReserveStepDraft, s));
+  CU(launch_build_pass(c->st, RSD_DRAFT, kPassIngestDraft, s));
+  if ((rc = read_scalars(c, s, &sc))) return rc;
+  const int n_sync = sc.n_tok;
+  if ((rc = run_ingest(c, RSD_DRAFT, n_sync, false, s))) return rc;
+  if ((rc = decode_phase(c, RSD_DRAFT, 0, B, s))) return rc;
+  // PRM: score y^_i at its last token
+  CU(launch_reserve_pages(c->st, RSD_PRM, kReserveScorePrm, s));
+  CU(launch_build_pass(c->st, RSD_PRM, kPassScorePrm, s));
+  if ((rc = read_scalars(c, s, &sc))) return rc;
+  const int n_prm = sc.n_tok;
+  if ((rc = run_ingest(c, RSD_PRM, n_prm, true, s))) return rc;
+  // gate, compaction of rejected rows, target catch-up and decode
+  CU(launch_gate(c->st, delta, c->lp, s));
+  CU(launch_reserve_pages(c->st, RSD_TARGET, kReserveTarget, s));
+  CU(launch_build_pass(c->st, RSD_TARGET, kPassCatchupTarget, s));
+  if ((rc = read_scalars(c, s, &sc))) return rc;
+  const int n_catch = sc.n_tok, n_rej = sc.n_rej;
+  c->last_n_rej = n_rej;
+  if ((rc = run_ingest(c, RSD_TARGET, n_catch, false, s))) return rc;
+  if ((rc = decode_phase(c, RSD_TARGET, 1, n_rej, s))) return rc;
+  // commit and read the results back
+  CU(launch_commit(c->st, c->lp, c->o_tokens, c->o_len, c->o_rewards, c->o_accept, c->o_live, s));
+  char* hp = c->pinned + 256;
+  int32_t* h_tokens = (int32_t*)hp; hp += sizeof(int32_t) * (size_t)B * c->C;
+  int32_t* h_len = (int32_t*)hp; hp += sizeof(int32_t) * B;
+  int32_t* h_gen0 = (int32_t*)hp; hp += sizeof(int32_t) * B;
+  int32_t* h_gen1 = (int32_t*)hp; hp += sizeof(int32_t) * B;
+  float* h_rew = (float*)hp; hp += sizeof(float) * B;
+  uint8_t* h_acc = (uint8_t*)hp; hp += B;
+  uint8_t* h_live = (uint8_t*)hp; hp += B;
+  CU(cudaMemcpyAsync(h_tokens, c->o_tokens, sizeof(int32_t) * (size_t)B * c->C, cudaMemcpyDeviceToHost, s));
+  CU(cudaMemcpyAsync(h_len, c->o_len, sizeof(int32_t) * B, cudaMemcpyDeviceToHost, s));
+  CU(cudaMemcpyAsync(h_gen0, c->st.gen_len[0], sizeof(int32_t) * B, cudaMemcpyDeviceToHost, s));
+  CU(cudaMemcpyAsync(h_gen1, c->st.gen_len[1], sizeof(int32_t) * B, cudaMemcpyDeviceToHost, s));
+  CU(cudaMemcpyAsync(h_rew, c->o_rewards, sizeof(float) * B, cudaMemcpyDeviceToHost, s));
+  CU(cudaMemcpyAsync(h_acc, c->o_accept, B, cudaMemcpyDeviceToHost, s));
+  CU(cudaMemcpyAsync(h_live, c->o_live, B, cudaMemcpyDeviceToHost, s));
+  if ((rc = clear_forcing(c, s))) return rc;
+  if ((rc = read_scalars(c, s, &sc))) return rc;
+  // counters (Section 3.3 accounting)
+  uint64_t gen_d = 0, gen_t = 0, n_live = 0, n_acc = 0, discarded = 0;
+  for (int b = 0; b < B; ++b) {
+    if (h_len[b] == 0) continue;  // row was already stopped
+    ++n_live;
+    gen_d += h_gen0[b];
+    if (h_acc[b]) ++n_acc; else { gen_t += h_gen1[b]; discarded += h_gen0[b]; }
+  }
+  c->ctr.gen_tokens[RSD_DRAFT] += gen_d;
+  c->ctr.gen_tokens[RSD_TARGET] += gen_t;
+  c->ctr.ingest_tokens[RSD_DRAFT] += n_sync;
+  c->ctr.ingest_tokens[RSD_PRM] += (uint64_t)n_prm - gen_d;
+  c->ctr.ingest_tokens[RSD_TARGET] += n_catch;
+  c->ctr.score_tokens += gen_d;
+  c->ctr.steps += n_live; c->ctr.accepted_steps += n_acc; c->ctr.rejected_steps += n_live - n_acc;
+  c->ctr.discarded_draft_tokens += discarded;
+  if (step_tokens) memcpy(step_tokens, h_tokens, sizeof(int32_t) * (size_t)B * c->C);
+  if (step_len) memcpy(step_len, h_len, sizeof(int32_t) * B);
+  if (rewards) memcpy(rewards, h_rew, sizeof(float) * B);
+  if (accept) memcpy(accept, h_acc, B);
+  if (live) memcpy(live, h_live, B);
+  return RSD_OK;
+}
+
+int rsd_flops_counters(rsd_ctx* c, rsd_counters* out) {
+  if (!c || !out) return RSD_ERR_ARG;
+  if (!c->loaded) return fail(c, RSD_ERR_STATE, "no models loaded%s");
+  rsd_counters r = c->ctr;
+  const double nd = c->mdl[RSD_DRAFT].n_params, np = c->mdl[RSD_PRM].n_params, nt = c->mdl[RSD_TARGET].n_params;
+  r.flops_paper = 2.0 * nd * (double)r.gen_tokens[RSD_DRAFT] + 2.0 * nt * (double)r.gen_tokens[RSD_TARGET] +
+                  2.0 * np * (double)(r.score_tokens + r.ingest_tokens[RSD_PRM]);
+  r.flops_all_tokens = 2.0 * nd * (double)(r.gen_tokens[RSD_DRAFT] + r.ingest_tokens[RSD_DRAFT]) +
+                       2.0 * nt * (double)(r.gen_tokens[RSD_TARGET] + r.ingest_tokens[RSD_TARGET]) +
+                       2.0 * np * (double)(r.score_tokens + r.ingest_tokens[RSD_PRM]);
+  *out = r;
+  return RSD_OK;
+}
+
+int rsd_destroy(rsd_ctx* c) {
+  if (!c) return RSD_OK;
+  cudaDeviceSynchronize();
+  if (c->pinned) cudaFreeHost(c->pinned);
+  delete c;
+  return RSD_OK;
+}
+
+const char* rsd_last_error(const rsd_ctx* c) { return c ? c->err.c_str() : g_create_error.c_str(); }
+
+// ---- parity hooks ---------------------------------------------------------------------------
+int rsd_debug_force(rsd_ctx* c, int which, const int32_t* tokens, const int32_t* len, const uint8_t* accept) {
+  if (!c) return RSD_ERR_ARG;
+  if (!c->prefilled) return fail(c, RSD_ERR_STATE, "forcing needs rows%s");
+  const int B = c->st.B;
+  if (which == RSD_PRM) {
+    if (!accept) return fail(c, RSD_ERR_ARG, "null accept mask%s");
+    CU(cudaMemcpy(c->st.forced_accept, accept, B, cudaMemcpyHostToDevice));
+    return RSD_OK;
+  }
+  if (which != RSD_DRAFT && which != RSD_TARGET) return fail(c, RSD_ERR_ARG, "which%s");
+  if (!tokens || !len) return fail(c, RSD_ERR_ARG, "null forcing arrays%s");
+  for (int b = 0; b < B; ++b)
+    if (len[b] < 0 || len[b] > c->C) return fail(c, RSD_ERR_ARG, "forced length out of range%s");
+  const int p = which == RSD_DRAFT ? 0 : 1;
+  CU(cudaMemcpy(c->st.forced_tok[p], tokens, sizeof(int32_t) * (size_t)B * c->C, cudaMemcpyHostToDevice));
+  CU(cudaMemcpy(c->st.forced_len[p], len, sizeof(int32_t) * B, cudaMemcpyHostToDevice));
+  return RSD_OK;
+}
+
+int rsd_debug_get_logits(rsd_ctx* c, int which, float* out) {
+  if (!c || !out) return RSD_ERR_ARG;
+  const int p = which == RSD_DRAFT ? 0 : (which == RSD_TARGET ? 1 : -1);
+  if (p < 0 || !c->dbg_logits[p]) return fail(c, RSD_ERR_STATE, "logits were not kept%s");
+  CU(cudaMemcpy(out, c->dbg_logits[p], sizeof(float) * (size_t)c->st.B * c->C * c->mdl[which].m.vocab, cudaMemcpyDeviceToHost));
+  return RSD_OK;
+}
+
+int rsd_debug_get_sampled(rsd_ctx* c, int which, int32_t* out) {
+  if (!c || !out) return RSD_ERR_ARG;
+  const int p = which == RSD_DRAFT ? 0 : (which == RSD_TARGET ? 1 : -1);
+  if (p < 0 || !c->prefilled) return fail(c, RSD_ERR_ARG, "which%s");
+  CU(cudaMemcpy(out, c->st.sampled[p], sizeof(int32_t) * (size_t)c->st.B * c->C, cudaMemcpyDeviceToHost));
+  return RSD_OK;
+}
+
+int rsd_debug_get_state(rsd_ctx* c, int32_t* z_len, int32_t* kv_len, int32_t* n_pages, int32_t* page_table,
+                        int32_t* next_page, int32_t* rej_idx, int32_t* n_rej) {
+  if (!c) return RSD_ERR_ARG;
+  if (!c->prefilled) return fail(c, RSD_ERR_STATE, "no rows%s");
+  const int B = c->st.B;
+  CU(cudaDeviceSynchronize());
+  if (z_len) CU(cudaMemcpy(z_len, c->st.z_len, sizeof(int32_t) * B, cudaMemcpyDeviceToHost));
+  for (int w = 0; w < 3; ++w) {
+    if (kv_len) CU(cudaMemcpy(kv_len + (size_t)w * B, c->st.kv_len[w], sizeof(int32_t) * B, cudaMemcpyDeviceToHost));
+    if (n_pages) CU(cudaMemcpy(n_pages + (size_t)w * B, c->st.n_pages[w], sizeof(int32_t) * B, cudaMemcpyDeviceToHost));
+    if (page_table)
+      CU(cudaMemcpy(page_table + (size_t)w * B * c->max_pages, c->st.page_table[w], sizeof(int32_t) * (size_t)B * c->max_pages, cudaMemcpyDeviceToHost));
+  }
+  if (next_page) CU(cudaMemcpy(next_page, c->st.next_page, sizeof(int32_t) * 3, cudaMemcpyDeviceToHost));
+  if (rej_idx) CU(cudaMemcpy(rej_idx, c->st.rej_idx, sizeof(int32_t) * B, cudaMemcpyDeviceToHost));
+  if (n_rej) *n_rej = c->last_n_rej;
+  return RSD_OK;
+}
+
+// ---- single kernels -------------------------------------------------------------------------
+#define KCU(call)                                     \
+  do {                                                \
+    cudaError_t e_ = (call);                          \
+    if (e_ != cudaSuccess) {                          \
+      g_create_error = cudaGetErrorString(e_);        \
+      return RSD_ERR_CUDA;                            \
+    }                                                 \
+  } while (0)
+
+size_t rsd_k_gemm_scratch_bytes(int32_t M, int32_t N, int32_t K) {
+  (void)N; (void)K;
+  return gemm_scratch_bytes(M);
+}
+
+int rsd_k_gemm(const void* W, const void* x, float* y, int32_t M, int32_t N, int32_t K, int32_t dtype,
+               int32_t accumulate, int32_t impl, void* scratch, size_t scratch_bytes, void* cuda_stream) {
+  if (!W || !x || !y || M < 0 || N < 1 || K < 1 || (dtype != RSD_F32 && dtype != RSD_BF16) || impl < 0 || impl > 2)
+    return RSD_ERR_ARG;
+  if (K % (dtype == RSD_BF16 ? 8 : 4)) return RSD_ERR_UNSUPPORTED;
+  if (impl == 2 && !gemm_tc_supported(dtype, M, N, K)) return RSD_ERR_UNSUPPORTED;
+  if (impl != 1 && (!scratch || scratch_bytes < gemm_scratch_bytes(M))) return RSD_ERR_ARG;
+  KCU(launch_gemm(dtype, W, x, y, M, N, K, accumulate, impl, scratch, scratch_bytes, nullptr, (cudaStream_t)cuda_stream));
+  return RSD_OK;
+}
+
+size_t rsd_k_attn_decode_scratch_bytes(int32_t B, int32_t H, int32_t hd, int32_t max_ctx) {
+  return attn_decode_scratch_bytes(B, H, hd, max_ctx);
+}
+
+int rsd_k_attn_decode(const float* q, const void* kv_pool, const int32_t* page_table, const int32_t* ctx_len,
+                      float* out, int32_t B, int32_t H, int32_t KV, int32_t hd, int32_t max_pages, int32_t dtype,
+                      void* scratch, size_t scratch_bytes, void* cuda_stream) {
+  if (!q || !kv_pool || !page_table || !ctx_len || !out || B < 1 || H < 1 || KV < 1 || H % KV || max_pages < 1)
+    return RSD_ERR_ARG;
+  if (hd != 64 && hd != 128) return RSD_ERR_UNSUPPORTED;
+  if (scratch_bytes < attn_decode_scratch_bytes(B, H, hd, max_pages * kPageTokens) || !scratch) return RSD_ERR_ARG;
+  KCU(launch_attn_decode(dtype, q, kv_pool, page_table, max_pages, nullptr, ctx_len, out, RSD_F32, B, H, KV, hd,
+                         max_pages * kPageTokens, scratch, nullptr, (cudaStream_t)cuda_stream));
+  return RSD_OK;
+}
+
+int rsd_k_gate_compact(const float* rewards, const uint8_t* live, float delta, uint8_t* accept, int32_t* rej_idx,
+                       int32_t* n_rej, int32_t B, void* scratch, size_t scratch_bytes, void* cuda_stream) {
+  if (!rewards || !live || !accept || !rej_idx || !n_rej || B < 1 || B > (1 << 24)) return RSD_ERR_ARG;
+  if (!scratch || scratch_bytes < sizeof(int32_t) * (size_t)((B + 1023) / 1024)) return RSD_ERR_ARG;
+  KCU(launch_gate_compact_large(rewards, live, delta, accept, rej_idx, n_rej, (int32_t*)scratch, B, (cudaStream_t)cuda_stream));
+  return RSD_OK;
+}
+
+int rsd_k_rmsnorm(const float* x, const void* gain, void* out, int32_t T, int32_t d, float eps, int32_t dtype,
+                  void* cuda_stream) {
+  if (!x || !gain || !out || T < 0 || d < 4 || d % 4) return RSD_ERR_ARG;
+  KCU(launch_rmsnorm(dtype, x, gain, out, T, d, eps, nullptr, nullptr, (cudaStream_t)cuda_stream));
+  return RSD_OK;
+}
+
+int rsd_k_rope(float* v, const int32_t* pos, int32_t T, int32_t n_heads, int32_t hd, float theta, void* cuda_stream) {
+  if (!v || !pos || T < 0 || n_heads < 1 || hd < 2 || hd % 2) return RSD_ERR_ARG;
+  KCU(launch_rope_only(v, pos, T, n_heads, hd, theta, (cudaStream_t)cuda_stream));
+  return RSD_OK;
+}
+
+int rsd_k_swiglu(const float* gu, void* out, int32_t T, int32_t F, int32_t dtype, void* cuda_stream) {
+  if (!gu || !out || T < 0 || F < 1) return RSD_ERR_ARG;
+  KCU(launch_swiglu(dtype, gu, out, T, F, nullptr, (cudaStream_t)cuda_stream));
+  return RSD_OK;
+}
+
+int rsd_k_sample(const float* logits, int32_t B, int32_t V, int32_t v_limit, float temperature, uint64_t seed,
+                 int32_t model_id, const int32_t* row, const int32_t* pos, int32_t* token, void* cuda_stream) {
+  if (!logits || !row || !pos || !token || B < 1 || V < 1 || v_limit < 1 || v_limit > V || temperature < 0.f) return RSD_ERR_ARG;
+  SampleArgs a{logits, B, V, v_limit, temperature, seed, model_id, row, pos, token, nullptr};
+  KCU(launch_sample(a, (cudaStream_t)cuda_stream));
+  return RSD_OK;
+}
+
+int rsd_k_philox(const uint32_t* ctr, const uint32_t* key, uint32_t* out, int32_t n, void* cuda_stream) {
+  if (!ctr || !key || !out || n < 0) return RSD_ERR_ARG;
+  KCU(launch_philox(ctr, key, out, n, (cudaStream_t)cuda_stream));
+  return RSD_OK;
+}
+
+}  // extern "C"

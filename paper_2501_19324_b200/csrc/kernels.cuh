@@ -1,0 +1,130 @@
+// Host-side launchers of the RSD step-loop kernels.  Every launcher enqueues on `s` and returns the
+// launch status; none synchronises or allocates.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+namespace rsd {
+
+constexpr int kPageTokens = 16;   // tokens per KV page
+constexpr int kMaxBatch = 1024;   // rows per context (one thread per row in the state kernels)
+
+// A pass pushes T token slots through one model.  Slot t carries token tok_id[t] of row tok_row[t]
+// at position tok_pos[t]; tok_row[t] < 0 marks an idle slot.  When n_active is non-null and reads
+// 0 on the device the whole pass is skipped (every row of the decode phase has finished).
+struct PassView {
+  const int32_t* tok_id;
+  const int32_t* tok_row;
+  const int32_t* tok_pos;
+  int T;
+  const int32_t* n_active;
+};
+
+// Where one model keeps keys and values: per layer a slab [page][2][KV][16][hd].
+struct KvView {
+  void* pool_layer;            // slab of the current layer
+  const int32_t* page_table;   // [rows, max_pages]
+  int max_pages;
+};
+
+cudaError_t launch_embed(int dtype, const void* embed, PassView p, float* x, int d, cudaStream_t s);
+// out[t] = rmsnorm(x[src ? src[t] : t]); rows with src[t] < 0 are skipped.
+cudaError_t launch_rmsnorm(int dtype, const float* x, const void* gain, void* out, int T, int d, float eps,
+                           const int32_t* src, const int32_t* n_active, cudaStream_t s);
+cudaError_t launch_gemm_simt(int dtype, const void* W, const void* x, float* y, int M, int N, int K,
+                             int accumulate, const int32_t* n_active, cudaStream_t s);
+// tcgen05 / TMEM / TMA GEMM (bf16): same contract as launch_gemm_simt; `scratch` holds split-K
+// partial tiles and tile counters (the counters must be zero on entry and are left zero).
+bool gemm_tc_supported(int dtype, int M, int N, int K);
+size_t gemm_scratch_bytes(int M);
+cudaError_t launch_gemm_tc(const void* W, const void* x, float* y, int M, int N, int K, int accumulate,
+                           void* scratch, size_t scratch_bytes, const int32_t* n_active, cudaStream_t s);
+// impl: 0 = by shape, 1 = SIMT split-K GEMV, 2 = tcgen05.
+cudaError_t launch_gemm(int dtype, const void* W, const void* x, float* y, int M, int N, int K, int accumulate,
+                        int impl, void* scratch, size_t scratch_bytes, const int32_t* n_active, cudaStream_t s);
+cudaError_t launch_rope_table(float2* table, int n_pos, int hd, float theta, cudaStream_t s);
+// Splits qkv [T, (H+2KV)*hd] (fp32): rotated q -> q_out [T, H*hd] fp32; rotated k and v -> KV pages.
+cudaError_t launch_rope_kv(int dtype, const float* qkv, PassView p, float* q_out, KvView kv, const float2* rope,
+                           int H, int KV, int hd, cudaStream_t s);
+cudaError_t launch_rope_only(float* v, const int32_t* pos, int T, int n_heads, int hd, float theta, cudaStream_t s);
+// Causal attention of every slot over positions [0, tok_pos] of its row, read from the pages.
+cudaError_t launch_attn_generic(int dtype, const float* q, PassView p, KvView kv, void* out, int H, int KV,
+                                int hd, cudaStream_t s);
+cudaError_t launch_swiglu(int dtype, const float* gu, void* out, int T, int F, const int32_t* n_active,
+                          cudaStream_t s);
+
+// Decode attention (one query per row) with split-KV partial results merged in a second pass.
+size_t attn_decode_scratch_bytes(int B, int H, int hd, int max_ctx);
+cudaError_t launch_attn_decode(int dtype, const float* q, const void* pool_layer, const int32_t* page_table,
+                               int max_pages, const int32_t* slot_row, const int32_t* ctx_len, void* out,
+                               int out_dtype, int B, int H, int KV, int hd, int max_ctx, void* scratch,
+                               const int32_t* n_active, cudaStream_t s);
+
+struct SampleArgs {
+  const float* logits;         // [n_slots, V]
+  int n_slots, V, v_limit;
+  float temperature;
+  uint64_t seed;
+  int model_id;
+  const int32_t* slot_row;     // row id per slot (noise key); < 0 = idle slot
+  const int32_t* slot_pos;     // position of the slot's input token; the new token sits at +1
+  int32_t* token;              // [n_slots] out
+  const int32_t* n_active;
+};
+cudaError_t launch_sample(const SampleArgs& a, cudaStream_t s);
+cudaError_t launch_philox(const uint32_t* ctr, const uint32_t* key, uint32_t* out, int n, cudaStream_t s);
+
+// reward[row] = head(rmsnorm(x[last_idx[row] - t0])) for rows whose last token lies in [t0, t0+T).
+cudaError_t launch_reward(int dtype, const float* x, const void* final_norm, const void* w_r, int head_kind,
+                          const int32_t* last_idx, int t0, int T, int d, float eps, float* reward, int n_rows,
+                          cudaStream_t s);
+
+// block_cnt: scratch of ceil(B / 1024) ints.
+cudaError_t launch_gate_compact_large(const float* rewards, const uint8_t* live, float delta, uint8_t* accept,
+                                      int32_t* rej_idx, int32_t* n_rej, int32_t* block_cnt, int B, cudaStream_t s);
+
+// ---- row state ------------------------------------------------------------------------------
+struct RowState {
+  int B, S, C, max_pages;      // rows in use, tokens per row, step cap, pages per row
+  int32_t *z_len, *live, *n_steps, *tok;
+  int32_t *kv_len[3], *n_pages[3], *page_table[3];
+  int32_t* next_page;          // [3]
+  int32_t pool_pages[3];
+  int32_t *gen_len[2], *gen_tok[2], *sampled[2];   // 0 = draft phase, 1 = target phase
+  int32_t *forced_tok[2], *forced_len[2];
+  uint8_t* forced_accept;      // [B], 0/1 force, 255 free
+  int32_t *gen_active, *n_active;
+  float* rewards;
+  uint8_t* accept;
+  int32_t *rej_idx, *n_rej;
+  int32_t *slot_row, *n_slots; // decode slots of the current phase
+  int32_t *last_idx;           // [B] flat index of each row's last token in the current pass
+  int32_t *n_tok;              // tokens of the current pass
+  int32_t *err;                // first error raised on the device
+  int32_t *pass_tok_id, *pass_tok_row, *pass_tok_pos;  // flat pass lists
+  int pass_capacity;
+};
+
+enum ReserveMode { kReservePrefillDraft, kReservePrefillPrm, kReserveStepDraft, kReserveScorePrm, kReserveTarget };
+enum PassMode { kPassIngestDraft, kPassScorePrm, kPassCatchupTarget };
+
+struct LoopParams {
+  int step_end_id, eos_id, step_end_mod, max_steps;
+  int omega_kind;
+  float omega_alpha;
+  uint64_t seed;
+};
+
+cudaError_t launch_reserve_pages(const RowState& st, int which, ReserveMode mode, cudaStream_t s);
+cudaError_t launch_build_pass(const RowState& st, int which, PassMode mode, cudaStream_t s);
+cudaError_t launch_decode_begin(const RowState& st, int phase, cudaStream_t s);
+cudaError_t launch_decode_prepare(const RowState& st, int which, int n_slots, cudaStream_t s);
+cudaError_t launch_decode_update(const RowState& st, int which, int phase, int iter, const int32_t* sampled,
+                                 int n_slots, const LoopParams& lp, cudaStream_t s);
+cudaError_t launch_gate(const RowState& st, float delta, const LoopParams& lp, cudaStream_t s);
+cudaError_t launch_commit(const RowState& st, const LoopParams& lp, int32_t* out_tokens, int32_t* out_len,
+                          float* out_rewards, uint8_t* out_accept, uint8_t* out_live, cudaStream_t s);
+
+}  // namespace rsd

@@ -1,0 +1,514 @@
+// Element-wise, normalisation, rotary, SIMT GEMV, attention, sampling and reward kernels of the RSD
+// step loop (sm_100a).  The residual stream and every reduction are fp32; weights, GEMM inputs and
+// the KV cache are stored in the model's element type (fp32 or bfloat16).
+#include "common.cuh"
+#include "kernels.cuh"
+
+namespace rsd {
+
+#define RSD_SKIP_IF_IDLE(n_active) \
+  if ((n_active) != nullptr && *(n_active) == 0) return;
+
+// ---------------------------------------------------------------------------------------------
+// Embedding gather: x[t, :] = E[tok_id[t], :]
+// ---------------------------------------------------------------------------------------------
+template <typename WT>
+__global__ void embed_kernel(const WT* __restrict__ E, PassView p, float* __restrict__ x, int d) {
+  RSD_SKIP_IF_IDLE(p.n_active);
+  const int t = blockIdx.x;
+  if (p.tok_row[t] < 0) return;
+  const WT* src = E + (size_t)p.tok_id[t] * d;
+  float* dst = x + (size_t)t * d;
+  constexpr int N = Vec16<WT>::N;
+  for (int i = threadIdx.x * N; i < d; i += blockDim.x * N) {
+    Vec16<WT> v;
+    v.load(src + i);
+#pragma unroll
+    for (int j = 0; j < N; ++j) dst[i + j] = v.v[j];
+  }
+}
+
+cudaError_t launch_embed(int dtype, const void* embed, PassView p, float* x, int d, cudaStream_t s) {
+  if (p.T <= 0) return cudaSuccess;
+  if (dtype == 1) embed_kernel<__nv_bfloat16><<<p.T, 128, 0, s>>>((const __nv_bfloat16*)embed, p, x, d);
+  else embed_kernel<float><<<p.T, 128, 0, s>>>((const float*)embed, p, x, d);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// RMSNorm: out = x * gain / sqrt(mean(x^2) + eps), one block per token, x kept in registers
+// ---------------------------------------------------------------------------------------------
+template <typename OT, typename GT>
+__global__ void rmsnorm_kernel(const float* __restrict__ x, const GT* __restrict__ gain, OT* __restrict__ out,
+                               int d, float eps, const int32_t* __restrict__ src, const int32_t* n_active) {
+  RSD_SKIP_IF_IDLE(n_active);
+  __shared__ float red[33];
+  const int t = blockIdx.x;
+  int st = t;
+  if (src != nullptr) {
+    st = src[t];
+    if (st < 0) return;
+  }
+  const float* xr = x + (size_t)st * d;
+  float ss = 0.f;
+  for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) {
+    float4 v = *reinterpret_cast<const float4*>(xr + i);
+    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+  }
+  ss = block_sum(ss, red);
+  const float inv = rsqrtf(ss / (float)d + eps);
+  OT* o = out + (size_t)t * d;
+  for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) {
+    float4 v = *reinterpret_cast<const float4*>(xr + i);
+    o[i] = from_f32<OT>(v.x * inv * to_f32(gain[i]));
+    o[i + 1] = from_f32<OT>(v.y * inv * to_f32(gain[i + 1]));
+    o[i + 2] = from_f32<OT>(v.z * inv * to_f32(gain[i + 2]));
+    o[i + 3] = from_f32<OT>(v.w * inv * to_f32(gain[i + 3]));
+  }
+}
+
+cudaError_t launch_rmsnorm(int dtype, const float* x, const void* gain, void* out, int T, int d, float eps,
+                           const int32_t* src, const int32_t* n_active, cudaStream_t s) {
+  if (T <= 0) return cudaSuccess;
+  const int threads = d >= 2048 ? 512 : 256;
+  if (dtype == 1)
+    rmsnorm_kernel<__nv_bfloat16, __nv_bfloat16><<<T, threads, 0, s>>>(x, (const __nv_bfloat16*)gain, (__nv_bfloat16*)out, d, eps, src, n_active);
+  else
+    rmsnorm_kernel<float, float><<<T, threads, 0, s>>>(x, (const float*)gain, (float*)out, d, eps, src, n_active);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Split-K SIMT GEMV / skinny GEMM:  y[m, n] (+)= sum_k x[m, k] W[n, k]
+// A block of 8 warps covers nb = 8/ks output columns; the ks warps of one column each stream a
+// strided share of the row with 16-byte loads and their partial sums meet in shared memory, in a
+// fixed order (deterministic).  Rows of x are taken MT at a time.
+// ---------------------------------------------------------------------------------------------
+template <typename WT, int MT>
+__global__ void __launch_bounds__(256)
+gemv_splitk_kernel(const WT* __restrict__ W, const WT* __restrict__ X, float* __restrict__ Y, int M, int N, int K,
+                   int ks, int accumulate, const int32_t* n_active) {
+  RSD_SKIP_IF_IDLE(n_active);
+  constexpr int VN = Vec16<WT>::N;
+  __shared__ float part[8][MT];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int nb = 8 / ks;
+  const int col = warp / ks, split = warp % ks;
+  const int n = blockIdx.x * nb + col;
+  const int m0 = blockIdx.y * MT;
+  float acc[MT];
+#pragma unroll
+  for (int m = 0; m < MT; ++m) acc[m] = 0.f;
+  if (n < N) {
+    const WT* wrow = W + (size_t)n * K;
+    const int nvec = K / VN;
+    for (int v = split * 32 + lane; v < nvec; v += ks * 32) {
+      Vec16<WT> w;
+      w.load_stream(wrow + (size_t)v * VN);
+#pragma unroll
+      for (int m = 0; m < MT; ++m) {
+        if (m0 + m < M) {
+          Vec16<WT> xv;
+          xv.load(X + (size_t)(m0 + m) * K + (size_t)v * VN);
+#pragma unroll
+          for (int j = 0; j < VN; ++j) acc[m] = fmaf(w.v[j], xv.v[j], acc[m]);
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int m = 0; m < MT; ++m) acc[m] = warp_sum(acc[m]);
+  if (lane == 0) {
+#pragma unroll
+    for (int m = 0; m < MT; ++m) part[warp][m] = acc[m];
+  }
+  __syncthreads();
+  // one thread per (column, m): add the ks partial sums in split order
+  const int idx = threadIdx.x;
+  if (idx < nb * MT) {
+    const int c = idx / MT, m = idx % MT;
+    const int nn = blockIdx.x * nb + c;
+    if (nn < N && m0 + m < M) {
+      float sum = 0.f;
+      for (int sidx = 0; sidx < ks; ++sidx) sum += part[c * ks + sidx][m];
+      float* y = Y + (size_t)(m0 + m) * N + nn;
+      *y = accumulate ? (*y + sum) : sum;
+    }
+  }
+}
+
+cudaError_t launch_gemm_simt(int dtype, const void* W, const void* x, float* y, int M, int N, int K,
+                             int accumulate, const int32_t* n_active, cudaStream_t s) {
+  if (M <= 0 || N <= 0) return cudaSuccess;
+  // pick the split so that the grid covers the 148 SMs a few times over
+  int ks = 1;
+  while (ks < 8 && (long)N * ks / 8 < 148L * 4 && K / (ks * 2) >= 256) ks *= 2;
+  constexpr int MT = 8;
+  dim3 grid((N + (8 / ks) - 1) / (8 / ks), (M + MT - 1) / MT);
+  if (dtype == 1)
+    gemv_splitk_kernel<__nv_bfloat16, MT><<<grid, 256, 0, s>>>((const __nv_bfloat16*)W, (const __nv_bfloat16*)x, y, M, N, K, ks, accumulate, n_active);
+  else
+    gemv_splitk_kernel<float, MT><<<grid, 256, 0, s>>>((const float*)W, (const float*)x, y, M, N, K, ks, accumulate, n_active);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Rotary table: table[pos, i] = (cos, sin)(pos * theta^(-2i/hd)), evaluated in fp64
+// ---------------------------------------------------------------------------------------------
+__global__ void rope_table_kernel(float2* table, int n_pos, int half, double theta, double hd) {
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= n_pos * half) return;
+  const int pos = idx / half, i = idx % half;
+  const double ang = (double)pos * pow(theta, -2.0 * (double)i / hd);
+  double sn, cs;
+  sincos(ang, &sn, &cs);
+  table[idx] = make_float2((float)cs, (float)sn);
+}
+
+cudaError_t launch_rope_table(float2* table, int n_pos, int hd, float theta, cudaStream_t s) {
+  const int n = n_pos * (hd / 2);
+  if (n <= 0) return cudaSuccess;
+  rope_table_kernel<<<(n + 255) / 256, 256, 0, s>>>(table, n_pos, hd / 2, (double)theta, (double)hd);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// RoPE on q and k, KV page write.  One block per token slot; threads walk the (head, pair) grid.
+// Pair (i, i + hd/2) of a head turns by the angle of (position, i).
+// ---------------------------------------------------------------------------------------------
+template <typename KT>
+__global__ void rope_kv_kernel(const float* __restrict__ qkv, PassView p, float* __restrict__ q_out, KT* pool,
+                               const int32_t* __restrict__ page_table, int max_pages,
+                               const float2* __restrict__ rope, int H, int KV, int hd) {
+  RSD_SKIP_IF_IDLE(p.n_active);
+  const int t = blockIdx.x;
+  const int row = p.tok_row[t];
+  if (row < 0) return;
+  const int pos = p.tok_pos[t];
+  const int half = hd / 2;
+  const float* src = qkv + (size_t)t * (H + 2 * KV) * hd;
+  const float2* cs = rope + (size_t)pos * half;
+  const int page = page_table[(size_t)row * max_pages + pos / kPageTokens];
+  const int slot = pos % kPageTokens;
+  // [page][2][KV][16][hd]
+  KT* kbase = pool + ((size_t)page * 2 + 0) * KV * kPageTokens * hd;
+  KT* vbase = pool + ((size_t)page * 2 + 1) * KV * kPageTokens * hd;
+  const int n_rot = (H + KV) * half;
+  for (int idx = threadIdx.x; idx < n_rot; idx += blockDim.x) {
+    const int head = idx / half, i = idx % half;
+    const float a = src[head * hd + i], b = src[head * hd + i + half];
+    const float2 c = cs[i];
+    const float ra = a * c.x - b * c.y, rb = b * c.x + a * c.y;
+    if (head < H) {
+      q_out[(size_t)t * H * hd + head * hd + i] = ra;
+      q_out[(size_t)t * H * hd + head * hd + i + half] = rb;
+    } else {
+      KT* k = kbase + ((size_t)(head - H) * kPageTokens + slot) * hd;
+      k[i] = from_f32<KT>(ra);
+      k[i + half] = from_f32<KT>(rb);
+    }
+  }
+  const float* vsrc = src + (H + KV) * hd;
+  for (int idx = threadIdx.x; idx < KV * hd; idx += blockDim.x) {
+    const int head = idx / hd, i = idx % hd;
+    vbase[((size_t)head * kPageTokens + slot) * hd + i] = from_f32<KT>(vsrc[idx]);
+  }
+}
+
+cudaError_t launch_rope_kv(int dtype, const float* qkv, PassView p, float* q_out, KvView kv, const float2* rope,
+                           int H, int KV, int hd, cudaStream_t s) {
+  if (p.T <= 0) return cudaSuccess;
+  if (dtype == 1)
+    rope_kv_kernel<__nv_bfloat16><<<p.T, 256, 0, s>>>(qkv, p, q_out, (__nv_bfloat16*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd);
+  else
+    rope_kv_kernel<float><<<p.T, 256, 0, s>>>(qkv, p, q_out, (float*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd);
+  return cudaGetLastError();
+}
+
+// Stand-alone rotary kernel on [T, n_heads, hd] fp32 (angles in fp64).
+__global__ void rope_only_kernel(float* v, const int32_t* pos, int n_heads, int hd, double theta) {
+  const int t = blockIdx.x, half = hd / 2;
+  const int p = pos[t];
+  for (int idx = threadIdx.x; idx < n_heads * half; idx += blockDim.x) {
+    const int head = idx / half, i = idx % half;
+    double sn, cs;
+    sincos((double)p * pow(theta, -2.0 * (double)i / (double)hd), &sn, &cs);
+    float* h = v + ((size_t)t * n_heads + head) * hd;
+    const float a = h[i], b = h[i + half];
+    h[i] = a * (float)cs - b * (float)sn;
+    h[i + half] = b * (float)cs + a * (float)sn;
+  }
+}
+
+cudaError_t launch_rope_only(float* v, const int32_t* pos, int T, int n_heads, int hd, float theta, cudaStream_t s) {
+  if (T <= 0) return cudaSuccess;
+  rope_only_kernel<<<T, 128, 0, s>>>(v, pos, n_heads, hd, (double)theta);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Generic causal attention over paged KV: one warp per (slot, query head), online softmax.
+// Each lane owns hd/32 consecutive dims; query head j reads KV head j / (H / KV).
+// ---------------------------------------------------------------------------------------------
+template <typename KT, typename OT, int HD>
+__global__ void __launch_bounds__(128)
+attn_generic_kernel(const float* __restrict__ q, PassView p, const KT* __restrict__ pool,
+                    const int32_t* __restrict__ page_table, int max_pages, OT* __restrict__ out, int H, int KV) {
+  RSD_SKIP_IF_IDLE(p.n_active);
+  constexpr int DPL = HD / 32;
+  const int lane = threadIdx.x & 31;
+  const int w = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (w >= p.T * H) return;
+  const int t = w / H, h = w % H;
+  const int row = p.tok_row[t];
+  if (row < 0) return;
+  const int pos = p.tok_pos[t];
+  const int g = h / (H / KV);
+  const float scale = rsqrtf((float)HD);
+  float qv[DPL];
+#pragma unroll
+  for (int i = 0; i < DPL; ++i) qv[i] = q[((size_t)t * H + h) * HD + lane * DPL + i] * scale;
+  float m = -INFINITY, l = 0.f, acc[DPL];
+#pragma unroll
+  for (int i = 0; i < DPL; ++i) acc[i] = 0.f;
+  const int32_t* pt = page_table + (size_t)row * max_pages;
+  for (int p0 = 0; p0 <= pos; p0 += kPageTokens) {
+    const int page = pt[p0 / kPageTokens];
+    const KT* kb = pool + (((size_t)page * 2 + 0) * KV + g) * kPageTokens * HD;
+    const KT* vb = pool + (((size_t)page * 2 + 1) * KV + g) * kPageTokens * HD;
+    const int n = min(kPageTokens, pos + 1 - p0);
+    float sc[kPageTokens];
+#pragma unroll
+    for (int j = 0; j < kPageTokens; ++j) {
+      float a = 0.f;
+      if (j < n) {
+#pragma unroll
+        for (int i = 0; i < DPL; ++i) a = fmaf(qv[i], to_f32(kb[j * HD + lane * DPL + i]), a);
+      }
+      sc[j] = a;
+    }
+#pragma unroll
+    for (int j = 0; j < kPageTokens; ++j) sc[j] = warp_sum(sc[j]);
+    float mx = m;
+#pragma unroll
+    for (int j = 0; j < kPageTokens; ++j)
+      if (j < n) mx = fmaxf(mx, sc[j]);
+    const float corr = __expf(m - mx);
+    l *= corr;
+#pragma unroll
+    for (int i = 0; i < DPL; ++i) acc[i] *= corr;
+#pragma unroll
+    for (int j = 0; j < kPageTokens; ++j) {
+      if (j < n) {
+        const float pj = __expf(sc[j] - mx);
+        l += pj;
+#pragma unroll
+        for (int i = 0; i < DPL; ++i) acc[i] = fmaf(pj, to_f32(vb[j * HD + lane * DPL + i]), acc[i]);
+      }
+    }
+    m = mx;
+  }
+  const float inv = 1.f / l;
+#pragma unroll
+  for (int i = 0; i < DPL; ++i) out[((size_t)t * H + h) * HD + lane * DPL + i] = from_f32<OT>(acc[i] * inv);
+}
+
+cudaError_t launch_attn_generic(int dtype, const float* q, PassView p, KvView kv, void* out, int H, int KV,
+                                int hd, cudaStream_t s) {
+  if (p.T <= 0) return cudaSuccess;
+  const int warps = p.T * H;
+  const int blocks = (warps + 3) / 4;
+  if (dtype == 1) {
+    using KT = __nv_bfloat16;
+    if (hd == 128) attn_generic_kernel<KT, KT, 128><<<blocks, 128, 0, s>>>(q, p, (const KT*)kv.pool_layer, kv.page_table, kv.max_pages, (KT*)out, H, KV);
+    else attn_generic_kernel<KT, KT, 64><<<blocks, 128, 0, s>>>(q, p, (const KT*)kv.pool_layer, kv.page_table, kv.max_pages, (KT*)out, H, KV);
+  } else {
+    if (hd == 128) attn_generic_kernel<float, float, 128><<<blocks, 128, 0, s>>>(q, p, (const float*)kv.pool_layer, kv.page_table, kv.max_pages, (float*)out, H, KV);
+    else attn_generic_kernel<float, float, 64><<<blocks, 128, 0, s>>>(q, p, (const float*)kv.pool_layer, kv.page_table, kv.max_pages, (float*)out, H, KV);
+  }
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// SwiGLU: out[t, f] = silu(gu[t, f]) * gu[t, F + f]
+// ---------------------------------------------------------------------------------------------
+template <typename OT>
+__global__ void swiglu_kernel(const float* __restrict__ gu, OT* __restrict__ out, int T, int F, const int32_t* n_active) {
+  RSD_SKIP_IF_IDLE(n_active);
+  const size_t n = (size_t)T * F;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+    const size_t t = i / F, f = i % F;
+    const float a = gu[t * 2 * F + f], b = gu[t * 2 * F + F + f];
+    out[i] = from_f32<OT>(a / (1.f + expf(-a)) * b);
+  }
+}
+
+cudaError_t launch_swiglu(int dtype, const float* gu, void* out, int T, int F, const int32_t* n_active, cudaStream_t s) {
+  if (T <= 0) return cudaSuccess;
+  const size_t n = (size_t)T * F;
+  int blocks = (int)((n + 255) / 256);
+  if (blocks > 148 * 8) blocks = 148 * 8;
+  if (dtype == 1) swiglu_kernel<__nv_bfloat16><<<blocks, 256, 0, s>>>(gu, (__nv_bfloat16*)out, T, F, n_active);
+  else swiglu_kernel<float><<<blocks, 256, 0, s>>>(gu, (float*)out, T, F, n_active);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Sampling: greedy argmax, or Gumbel-max with Philox noise keyed by (seed; vocab id / 4, position
+// of the generated token, row, model id).  One block per slot; ties go to the lowest id.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void better(float& bs, int& bi, float s, int i) {
+  if (s > bs || (s == bs && i < bi)) { bs = s; bi = i; }
+}
+
+__global__ void __launch_bounds__(1024) sample_kernel(SampleArgs a) {
+  RSD_SKIP_IF_IDLE(a.n_active);
+  __shared__ float s_sc[32];
+  __shared__ int s_ix[32];
+  const int slot = blockIdx.x;
+  const int row = a.slot_row[slot];
+  if (row < 0) return;
+  const float* lg = a.logits + (size_t)slot * a.V;
+  const uint32_t position = (uint32_t)(a.slot_pos[slot] + 1);
+  const uint2 key = make_uint2((uint32_t)(a.seed & 0xFFFFFFFFull), (uint32_t)(a.seed >> 32));
+  const float inv_t = a.temperature > 0.f ? 1.f / a.temperature : 1.f;
+  float bs = -INFINITY;
+  int bi = 0x7FFFFFFF;
+  for (int v4 = threadIdx.x; v4 * 4 < a.v_limit; v4 += blockDim.x) {
+    float g[4] = {0.f, 0.f, 0.f, 0.f};
+    if (a.temperature > 0.f) {
+      const uint4 r = philox4x32_10(make_uint4((uint32_t)v4, position, (uint32_t)row, (uint32_t)a.model_id), key);
+      const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) g[j] = -logf(-logf(uniform_from_bits(w[j])));
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int v = v4 * 4 + j;
+      if (v < a.v_limit) better(bs, bi, lg[v] * inv_t + g[j], v);
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float os = __shfl_xor_sync(0xFFFFFFFFu, bs, o);
+    const int oi = __shfl_xor_sync(0xFFFFFFFFu, bi, o);
+    better(bs, bi, os, oi);
+  }
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (lane == 0) { s_sc[warp] = bs; s_ix[warp] = bi; }
+  __syncthreads();
+  if (warp == 0) {
+    const int nw = blockDim.x >> 5;
+    bs = lane < nw ? s_sc[lane] : -INFINITY;
+    bi = lane < nw ? s_ix[lane] : 0x7FFFFFFF;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float os = __shfl_xor_sync(0xFFFFFFFFu, bs, o);
+      const int oi = __shfl_xor_sync(0xFFFFFFFFu, bi, o);
+      better(bs, bi, os, oi);
+    }
+    if (lane == 0) a.token[slot] = bi;
+  }
+}
+
+cudaError_t launch_sample(const SampleArgs& a, cudaStream_t s) {
+  if (a.n_slots <= 0) return cudaSuccess;
+  const int threads = a.v_limit >= 16384 ? 1024 : 256;
+  sample_kernel<<<a.n_slots, threads, 0, s>>>(a);
+  return cudaGetLastError();
+}
+
+__global__ void philox_kernel(const uint32_t* ctr, const uint32_t* key, uint32_t* out, int n) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const uint4 r = philox4x32_10(make_uint4(ctr[4 * i], ctr[4 * i + 1], ctr[4 * i + 2], ctr[4 * i + 3]),
+                                make_uint2(key[0], key[1]));
+  out[4 * i] = r.x; out[4 * i + 1] = r.y; out[4 * i + 2] = r.z; out[4 * i + 3] = r.w;
+}
+
+cudaError_t launch_philox(const uint32_t* ctr, const uint32_t* key, uint32_t* out, int n, cudaStream_t s) {
+  if (n <= 0) return cudaSuccess;
+  philox_kernel<<<(n + 255) / 256, 256, 0, s>>>(ctr, key, out, n);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// PRM step scoring head: gathers the hidden state of each row's last step token, applies the final
+// RMSNorm, projects to a scalar and squashes it (Appendix B.3; score in [0,1], Section 3 "Models").
+// ---------------------------------------------------------------------------------------------
+template <typename WT>
+__global__ void reward_kernel(const float* __restrict__ x, const WT* __restrict__ final_norm, const WT* __restrict__ w_r,
+                              int head_kind, const int32_t* __restrict__ last_idx, int t0, int T, int d, float eps,
+                              float* __restrict__ reward) {
+  __shared__ float red[33];
+  const int row = blockIdx.x;
+  const int idx = last_idx[row];
+  if (idx < t0 || idx >= t0 + T) return;
+  const float* xr = x + (size_t)(idx - t0) * d;
+  float ss = 0.f, dot = 0.f;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) {
+    const float v = xr[i];
+    ss += v * v;
+    dot += v * to_f32(final_norm[i]) * to_f32(w_r[i]);
+  }
+  ss = block_sum(ss, red);
+  dot = block_sum(dot, red);
+  if (threadIdx.x == 0) {
+    const float a = dot * rsqrtf(ss / (float)d + eps);
+    reward[row] = head_kind == 2 ? a : 1.f / (1.f + expf(-a));
+  }
+}
+
+cudaError_t launch_reward(int dtype, const float* x, const void* final_norm, const void* w_r, int head_kind,
+                          const int32_t* last_idx, int t0, int T, int d, float eps, float* reward, int n_rows,
+                          cudaStream_t s) {
+  if (n_rows <= 0) return cudaSuccess;
+  if (dtype == 1)
+    reward_kernel<__nv_bfloat16><<<n_rows, 256, 0, s>>>(x, (const __nv_bfloat16*)final_norm, (const __nv_bfloat16*)w_r, head_kind, last_idx, t0, T, d, eps, reward);
+  else
+    reward_kernel<float><<<n_rows, 256, 0, s>>>(x, (const float*)final_norm, (const float*)w_r, head_kind, last_idx, t0, T, d, eps, reward);
+  return cudaGetLastError();
+}
+
+}  // namespace rsd
+
+// ---------------------------------------------------------------------------------------------
+// Decode attention entry: one query per row over its cached positions.
+// ---------------------------------------------------------------------------------------------
+namespace rsd {
+
+__global__ void decode_slots_kernel(const int32_t* slot_row, const int32_t* ctx_len, int32_t* row, int32_t* pos, int B) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= B) return;
+  const int r = slot_row ? slot_row[i] : i;
+  row[i] = (r >= 0 && ctx_len[i] >= 1) ? r : -1;
+  pos[i] = ctx_len[i] - 1;
+}
+
+size_t attn_decode_scratch_bytes(int B, int H, int hd, int max_ctx) {
+  (void)H; (void)hd; (void)max_ctx;
+  return sizeof(int32_t) * 2 * (size_t)B + 256;
+}
+
+cudaError_t launch_attn_decode(int dtype, const float* q, const void* pool_layer, const int32_t* page_table,
+                               int max_pages, const int32_t* slot_row, const int32_t* ctx_len, void* out,
+                               int out_dtype, int B, int H, int KV, int hd, int max_ctx, void* scratch,
+                               const int32_t* n_active, cudaStream_t s) {
+  (void)max_ctx;
+  int32_t* row = (int32_t*)scratch;
+  int32_t* pos = row + B;
+  decode_slots_kernel<<<(B + 255) / 256, 256, 0, s>>>(slot_row, ctx_len, row, pos, B);
+  PassView p{nullptr, row, pos, B, n_active};
+  KvView kv{const_cast<void*>(pool_layer), page_table, max_pages};
+  const int warps = B * H, blocks = (warps + 3) / 4;
+#define RSD_ATTN(KT, OT, HD) \
+  attn_generic_kernel<KT, OT, HD><<<blocks, 128, 0, s>>>(q, p, (const KT*)kv.pool_layer, kv.page_table, kv.max_pages, (OT*)out, H, KV)
+  using bf = __nv_bfloat16;
+  if (dtype == 1 && out_dtype == 1) { if (hd == 128) RSD_ATTN(bf, bf, 128); else RSD_ATTN(bf, bf, 64); }
+  else if (dtype == 1) { if (hd == 128) RSD_ATTN(bf, float, 128); else RSD_ATTN(bf, float, 64); }
+  else { if (hd == 128) RSD_ATTN(float, float, 128); else RSD_ATTN(float, float, 64); }
+#undef RSD_ATTN
+  return cudaGetLastError();
+}
+
+}  // namespace rsd

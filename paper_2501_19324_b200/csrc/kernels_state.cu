@@ -1,0 +1,381 @@
+// Integer side of the RSD step loop (Algorithm 1 batched over rows): page reservation, ragged pass
+// lists, decode-phase control, the threshold gate with warp-ballot compaction of rejected rows,
+// and the commit of y_i.  All state lives on the device; every kernel here runs as ONE block of
+// 1024 threads (thread b <-> row b, rows <= 1024), which keeps the ascending-row order of page
+// hand-out and of the rejected-row list deterministic.
+#include "common.cuh"
+#include "kernels.cuh"
+
+namespace rsd {
+
+// ---------------------------------------------------------------------------------------------
+// Page reservation.  Row b needs capacity for `need` cached positions; missing pages are taken
+// from a bump counter, rows served in ascending order, each row's new pages consecutive.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(1024) reserve_pages_kernel(RowState st, int which, int mode) {
+  __shared__ int scan[33];
+  const int b = threadIdx.x;
+  int need = 0;
+  if (b < st.B) {
+    const int z = st.z_len[b];
+    const bool live = st.live[b] != 0;
+    switch (mode) {
+      case kReservePrefillDraft: need = z - 1; break;
+      case kReservePrefillPrm: need = z; break;
+      case kReserveStepDraft: need = live ? z - 1 + st.C : 0; break;
+      case kReserveScorePrm: need = live ? z + st.gen_len[0][b] : 0; break;
+      case kReserveTarget: need = (live && !st.accept[b]) ? z - 1 + st.C : 0; break;
+    }
+  }
+  const int have = b < st.B ? st.n_pages[which][b] : 0;
+  int more = (need + kPageTokens - 1) / kPageTokens - have;
+  if (more < 0) more = 0;
+  int total;
+  const int off = block_exclusive_scan(more, scan, &total);
+  const int base = st.next_page[which];
+  if (base + total > st.pool_pages[which] || (b < st.B && have + more > st.max_pages)) {
+    st.err[0] = -3;  // pool exhausted: leave the tables untouched
+  }
+  __syncthreads();
+  if (st.err[0] != 0) return;
+  if (b < st.B) {
+    for (int i = 0; i < more; ++i) st.page_table[which][(size_t)b * st.max_pages + have + i] = base + off + i;
+    st.n_pages[which][b] = have + more;
+  }
+  __syncthreads();
+  if (b == 0) st.next_page[which] = base + total;
+}
+
+cudaError_t launch_reserve_pages(const RowState& st, int which, ReserveMode mode, cudaStream_t s) {
+  reserve_pages_kernel<<<1, 1024, 0, s>>>(st, which, (int)mode);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Ragged pass list: for every participating row the positions [kv_len, end) not yet cached by model
+// `which`, flattened in (row, position) order.  Advances kv_len to `end`.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(1024) build_pass_kernel(RowState st, int which, int mode) {
+  __shared__ int scan[33];
+  __shared__ int s_off[kMaxBatch + 1];
+  __shared__ int s_start[kMaxBatch];
+  const int b = threadIdx.x;
+  int start = 0, cnt = 0;
+  if (b < st.B) {
+    const int z = st.z_len[b];
+    const bool live = st.live[b] != 0;
+    start = st.kv_len[which][b];
+    int end = start;
+    switch (mode) {
+      case kPassIngestDraft: end = live ? z - 1 : start; break;
+      case kPassScorePrm: end = live ? z + st.gen_len[0][b] : start; break;
+      case kPassCatchupTarget: end = (live && !st.accept[b]) ? z - 1 : start; break;
+    }
+    cnt = max(0, end - start);
+  }
+  int total;
+  const int off = block_exclusive_scan(cnt, scan, &total);
+  if (b < kMaxBatch) { s_off[b] = off; s_start[b] = start; }
+  if (b == 0) {
+    s_off[kMaxBatch] = total;
+    st.n_tok[0] = total;
+    if (total > st.pass_capacity) st.err[0] = -3;
+  }
+  if (b < st.B) {
+    st.last_idx[b] = cnt > 0 ? off + cnt - 1 : -1;
+    st.kv_len[which][b] = start + cnt;
+  }
+  __syncthreads();
+  if (total > st.pass_capacity) return;
+  for (int t = threadIdx.x; t < total; t += blockDim.x) {
+    // largest row with s_off[row] <= t (rows with no tokens share an offset with their successor)
+    int lo = 0, hi = st.B - 1;
+    while (lo < hi) {
+      const int mid = (lo + hi + 1) >> 1;
+      if (s_off[mid] <= t) lo = mid; else hi = mid - 1;
+    }
+    const int pos = s_start[lo] + (t - s_off[lo]);
+    st.pass_tok_row[t] = lo;
+    st.pass_tok_pos[t] = pos;
+    st.pass_tok_id[t] = st.tok[(size_t)lo * st.S + pos];
+  }
+}
+
+cudaError_t launch_build_pass(const RowState& st, int which, PassMode mode, cudaStream_t s) {
+  build_pass_kernel<<<1, 1024, 0, s>>>(st, which, (int)mode);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Decode-phase control.  Phase 0: the draft writes y^_i for every live row (slot b = row b).
+// Phase 1: the target writes y_i for the rejected rows (slot i = rej_idx[i]).
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(1024) decode_begin_kernel(RowState st, int phase) {
+  __shared__ int scan[33];
+  const int b = threadIdx.x;
+  int part = 0;
+  if (b < st.B) {
+    part = st.live[b] != 0 && (phase == 0 || st.accept[b] == 0);
+    st.gen_active[b] = part;
+    st.gen_len[phase][b] = 0;
+  }
+  int total;
+  block_exclusive_scan(part, scan, &total);
+  if (b == 0) st.n_active[0] = total;
+  const int n_slots = phase == 0 ? st.B : st.n_rej[0];
+  if (b == 0) st.n_slots[0] = n_slots;
+  if (b < st.B) st.slot_row[b] = phase == 0 ? b : (b < n_slots ? st.rej_idx[b] : -1);
+  for (int i = threadIdx.x; i < st.B * st.C; i += blockDim.x) {
+    st.gen_tok[phase][i] = 0;
+    st.sampled[phase][i] = 0;
+  }
+}
+
+cudaError_t launch_decode_begin(const RowState& st, int phase, cudaStream_t s) {
+  decode_begin_kernel<<<1, 1024, 0, s>>>(st, phase);
+  return cudaGetLastError();
+}
+
+__global__ void __launch_bounds__(1024) decode_prepare_kernel(RowState st, int which, int n_slots) {
+  if (st.n_active[0] == 0) return;
+  const int i = threadIdx.x;
+  if (i >= n_slots) return;
+  const int row = st.slot_row[i];
+  if (row >= 0 && st.gen_active[row]) {
+    const int pos = st.kv_len[which][row];
+    st.pass_tok_id[i] = st.tok[(size_t)row * st.S + pos];
+    st.pass_tok_pos[i] = pos;
+    st.pass_tok_row[i] = row;
+  } else {
+    st.pass_tok_row[i] = -1;
+  }
+}
+
+cudaError_t launch_decode_prepare(const RowState& st, int which, int n_slots, cudaStream_t s) {
+  if (n_slots <= 0) return cudaSuccess;
+  decode_prepare_kernel<<<1, 1024, 0, s>>>(st, which, n_slots);
+  return cudaGetLastError();
+}
+
+__device__ __forceinline__ bool ends_step(int t, const LoopParams& lp) {
+  if (lp.eos_id >= 0 && t == lp.eos_id) return true;
+  if (lp.step_end_mod > 0) return (t % lp.step_end_mod) == (lp.step_end_id % lp.step_end_mod);
+  return t == lp.step_end_id;
+}
+
+// Appends iteration `iter`'s token of every active slot to its row and stops rows whose step ended.
+__global__ void __launch_bounds__(1024)
+decode_update_kernel(RowState st, int which, int phase, int iter, const int32_t* sampled, int n_slots, LoopParams lp) {
+  if (st.n_active[0] == 0) return;
+  const int i = threadIdx.x;
+  int ended = 0;
+  if (i < n_slots) {
+    const int row = st.pass_tok_row[i];
+    if (row >= 0) {
+      int t = sampled[i];
+      st.sampled[phase][(size_t)row * st.C + iter] = t;
+      const int flen = st.forced_len[phase][row];
+      if (flen > 0) t = st.forced_tok[phase][(size_t)row * st.C + iter];
+      const int pos = st.pass_tok_pos[i];
+      st.tok[(size_t)row * st.S + pos + 1] = t;
+      st.gen_tok[phase][(size_t)row * st.C + iter] = t;
+      st.kv_len[which][row] = pos + 1;
+      st.gen_len[phase][row] = iter + 1;
+      if (ends_step(t, lp) || iter + 1 == st.C || (flen > 0 && iter + 1 == flen)) {
+        st.gen_active[row] = 0;
+        ended = 1;
+      }
+    }
+  }
+  const int n_ended = __syncthreads_count(ended);
+  if (threadIdx.x == 0) st.n_active[0] -= n_ended;
+}
+
+cudaError_t launch_decode_update(const RowState& st, int which, int phase, int iter, const int32_t* sampled,
+                                 int n_slots, const LoopParams& lp, cudaStream_t s) {
+  if (n_slots <= 0) return cudaSuccess;
+  decode_update_kernel<<<1, 1024, 0, s>>>(st, which, phase, iter, sampled, n_slots, lp);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Gate + compaction.  Acceptance criterion of Algorithm 2 with the weighting functions of Table 1
+// (binary step: accept iff r >= delta); rejected live rows are listed in ascending order by a
+// warp ballot + popcount prefix, and their draft / PRM caches are rolled back to the step start.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ float omega_weight(int kind, float r, float delta, float alpha) {
+  switch (kind) {
+    case 0: return delta;
+    case 1: return r >= delta ? 1.f : 0.f;
+    case 2: return fminf(1.f, fmaxf(0.f, r));
+    case 3: return fmaxf(0.f, r / (1.f + r));
+    case 4: return 1.f / (1.f + expf(-alpha * (r - delta)));
+    default: return 0.f;
+  }
+}
+
+// Ascending compaction of the flagged threads of a 1024-thread block: returns this thread's rank
+// among flagged threads and the total; `wsum` holds 33 ints.
+__device__ __forceinline__ int ballot_rank(bool flag, int* wsum, int* total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const unsigned ballot = __ballot_sync(0xFFFFFFFFu, flag);
+  const int in_warp = __popc(ballot & ((1u << lane) - 1u));
+  __syncthreads();
+  if (lane == 0) wsum[warp] = __popc(ballot);
+  __syncthreads();
+  if (warp == 0) {
+    const int nw = blockDim.x >> 5;
+    const int c = lane < nw ? wsum[lane] : 0;
+    int inc = c;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int n = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+      if (lane >= o) inc += n;
+    }
+    wsum[lane] = inc - c;
+    if (lane == 31) wsum[32] = inc;
+  }
+  __syncthreads();
+  *total = wsum[32];
+  return wsum[warp] + in_warp;
+}
+
+__global__ void __launch_bounds__(1024) gate_kernel(RowState st, float delta, LoopParams lp) {
+  __shared__ int wsum[33];
+  const int b = threadIdx.x;
+  bool live = false, rejected = false;
+  if (b < st.B) {
+    live = st.live[b] != 0;
+    int acc = 0;
+    if (live) {
+      const float r = st.rewards[b];
+      const float w = omega_weight(lp.omega_kind, r, delta, lp.omega_alpha);
+      if (w == 0.f) acc = 0;
+      else if (w == 1.f) acc = 1;
+      else {
+        const uint4 rnd = philox4x32_10(make_uint4(0u, (uint32_t)st.z_len[b], (uint32_t)b, 3u),
+                                        make_uint2((uint32_t)(lp.seed & 0xFFFFFFFFull), (uint32_t)(lp.seed >> 32)));
+        acc = w >= uniform_from_bits(rnd.x) ? 1 : 0;
+      }
+      const uint8_t f = st.forced_accept[b];
+      if (f <= 1) acc = f;
+    } else {
+      st.rewards[b] = 0.f;
+    }
+    st.accept[b] = (uint8_t)acc;
+    rejected = live && !acc;
+  }
+  int total;
+  const int rank = ballot_rank(rejected, wsum, &total);
+  if (rejected) {
+    st.rej_idx[rank] = b;
+    st.kv_len[0][b] = st.z_len[b] - 1;   // draft: drop y^_i, keep z_i minus its newest token
+    st.kv_len[1][b] = st.z_len[b];       // PRM: drop y^_i
+  }
+  if (b == 0) st.n_rej[0] = total;
+}
+
+cudaError_t launch_gate(const RowState& st, float delta, const LoopParams& lp, cudaStream_t s) {
+  gate_kernel<<<1, 1024, 0, s>>>(st, delta, lp);
+  return cudaGetLastError();
+}
+
+// Stand-alone gate + compaction for any B: per-block ballot counts, a scan of the block counts,
+// then the ascending write.
+__global__ void __launch_bounds__(1024)
+gate_count_kernel(const float* rewards, const uint8_t* live, float delta, uint8_t* accept, int32_t* block_cnt, int B) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  bool rej = false;
+  if (b < B) {
+    const bool lv = live[b] != 0;
+    const bool acc = lv && rewards[b] >= delta;
+    accept[b] = acc ? 1 : 0;
+    rej = lv && !acc;
+  }
+  const int n = __syncthreads_count(rej);
+  if (threadIdx.x == 0) block_cnt[blockIdx.x] = n;
+}
+
+__global__ void __launch_bounds__(1024) gate_scan_kernel(int32_t* block_cnt, int n_blocks, int32_t* n_rej) {
+  // exclusive scan of up to 2^24 / 1024 = 16384 block counts by one block, 16 per thread
+  __shared__ int scan[33];
+  int local[16];
+  int sum = 0;
+  for (int i = 0; i < 16; ++i) {
+    const int idx = threadIdx.x * 16 + i;
+    local[i] = idx < n_blocks ? block_cnt[idx] : 0;
+    sum += local[i];
+  }
+  int total;
+  int off = block_exclusive_scan(sum, scan, &total);
+  for (int i = 0; i < 16; ++i) {
+    const int idx = threadIdx.x * 16 + i;
+    if (idx < n_blocks) block_cnt[idx] = off;
+    off += local[i];
+  }
+  if (threadIdx.x == 0) n_rej[0] = total;
+}
+
+__global__ void __launch_bounds__(1024)
+gate_write_kernel(const uint8_t* live, const uint8_t* accept, const int32_t* block_off, int32_t* rej_idx, int B) {
+  __shared__ int wsum[33];
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  const bool rej = b < B && live[b] != 0 && accept[b] == 0;
+  int total;
+  const int rank = ballot_rank(rej, wsum, &total);
+  if (rej) rej_idx[block_off[blockIdx.x] + rank] = b;
+}
+
+cudaError_t launch_gate_compact_large(const float* rewards, const uint8_t* live, float delta, uint8_t* accept,
+                                      int32_t* rej_idx, int32_t* n_rej, int32_t* block_cnt, int B, cudaStream_t s) {
+  const int n_blocks = (B + 1023) / 1024;
+  gate_count_kernel<<<n_blocks, 1024, 0, s>>>(rewards, live, delta, accept, block_cnt, B);
+  gate_scan_kernel<<<1, 1024, 0, s>>>(block_cnt, n_blocks, n_rej);
+  gate_write_kernel<<<n_blocks, 1024, 0, s>>>(live, accept, block_cnt, rej_idx, B);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Commit: y_i <- accept ? y^_i : target step; the row stops when EOS is in y_i, after max_steps
+// steps, or when another step would not fit.  One block per row.
+// ---------------------------------------------------------------------------------------------
+__global__ void commit_kernel(RowState st, LoopParams lp, int32_t* out_tokens, int32_t* out_len, float* out_rewards,
+                              uint8_t* out_accept, uint8_t* out_live) {
+  const int b = blockIdx.x;
+  const bool live = st.live[b] != 0;
+  const int acc = st.accept[b];
+  const int phase = acc ? 0 : 1;
+  const int n = live ? st.gen_len[phase][b] : 0;
+  const int32_t* y = st.gen_tok[phase] + (size_t)b * st.C;
+  int has_eos = 0;
+  for (int j = threadIdx.x; j < st.C; j += blockDim.x) {
+    const int t = j < n ? y[j] : 0;
+    out_tokens[(size_t)b * st.C + j] = t;
+    if (j < n && lp.eos_id >= 0 && t == lp.eos_id) has_eos = 1;
+  }
+  has_eos = __syncthreads_or(has_eos);
+  if (threadIdx.x == 0) {
+    out_len[b] = n;
+    out_rewards[b] = live ? st.rewards[b] : 0.f;
+    out_accept[b] = live ? (uint8_t)acc : 0;
+    int still = 0;
+    if (live) {
+      const int z = st.z_len[b] + n;
+      const int steps = st.n_steps[b] + 1;
+      st.z_len[b] = z;
+      st.n_steps[b] = steps;
+      still = !(has_eos || steps >= lp.max_steps || z + st.C > st.S);
+      st.live[b] = still;
+    }
+    out_live[b] = (uint8_t)still;
+  }
+}
+
+cudaError_t launch_commit(const RowState& st, const LoopParams& lp, int32_t* out_tokens, int32_t* out_len,
+                          float* out_rewards, uint8_t* out_accept, uint8_t* out_live, cudaStream_t s) {
+  if (st.B <= 0) return cudaSuccess;
+  commit_kernel<<<st.B, 128, 0, s>>>(st, lp, out_tokens, out_len, out_rewards, out_accept, out_live);
+  return cudaGetLastError();
+}
+
+}  // namespace rsd

@@ -177,6 +177,48 @@ def cpu_model_weights(shape: ModelShape, slot: int, seed: int, bf16: bool, head_
     return out
 
 
+def gpu_model_tensors(shape: ModelShape, slot: int, seed: int, bf16: bool, head_kind: int) -> dict:
+    """The same weights as cpu_model_weights, generated on the GPU into torch tensors in the fused
+    storage the CUDA library reads: wqkv rows = Wq | Wk | Wv, wgu rows = Wgate | Wup."""
+    import torch
+    lib = cuda_lib()
+    dt = torch.bfloat16 if bf16 else torch.float32
+    code = 1 if bf16 else 0
+    esz = 2 if bf16 else 4
+    stream = torch.cuda.current_stream().cuda_stream
+
+    def fill(t, row0, rows, cols, tid):
+        rc = lib.rsd_inputs_fill_device(t.data_ptr() + row0 * cols * esz, code, seed, tid, 0, rows * cols,
+                                        WEIGHT_SCALE, stream)
+        assert rc == 0, f"fill kernel launch failed: {rc}"
+
+    def ones(n):
+        return torch.ones(n, dtype=dt, device="cuda")
+
+    d, hd, H, KV, F = shape.d_model, shape.head_dim, shape.n_heads, shape.n_kv_heads, shape.d_ffn
+    out = {"tok_embed": torch.empty(shape.vocab, d, dtype=dt, device="cuda"), "final_norm": ones(d),
+           "wqkv": [], "wo": [], "wgu": [], "wdown": [], "norm1": [], "norm2": []}
+    fill(out["tok_embed"], 0, shape.vocab, d, tensor_id(slot, 0, KIND_EMBED))
+    head_rows = shape.vocab if head_kind == HEAD_LM else 1
+    out["head"] = torch.empty(head_rows, d, dtype=dt, device="cuda")
+    fill(out["head"], 0, head_rows, d, tensor_id(slot, 0, KIND_HEAD))
+    for l in range(shape.n_layers):
+        wqkv = torch.empty((H + 2 * KV) * hd, d, dtype=dt, device="cuda")
+        fill(wqkv, 0, H * hd, d, tensor_id(slot, l, KIND_WQ))
+        fill(wqkv, H * hd, KV * hd, d, tensor_id(slot, l, KIND_WK))
+        fill(wqkv, (H + KV) * hd, KV * hd, d, tensor_id(slot, l, KIND_WV))
+        wo = torch.empty(d, H * hd, dtype=dt, device="cuda")
+        fill(wo, 0, d, H * hd, tensor_id(slot, l, KIND_WO))
+        wgu = torch.empty(2 * F, d, dtype=dt, device="cuda")
+        fill(wgu, 0, F, d, tensor_id(slot, l, KIND_WGATE))
+        fill(wgu, F, F, d, tensor_id(slot, l, KIND_WUP))
+        wdown = torch.empty(d, F, dtype=dt, device="cuda")
+        fill(wdown, 0, d, F, tensor_id(slot, l, KIND_WDOWN))
+        out["wqkv"].append(wqkv); out["wo"].append(wo); out["wgu"].append(wgu); out["wdown"].append(wdown)
+        out["norm1"].append(ones(d)); out["norm2"].append(ones(d))
+    return out
+
+
 def prompts(seed: int, batch: int, len_lo: int, len_hi: int, vocab: int):
     """Ragged uniform-random prompts: lengths uniform on [len_lo, len_hi], ids uniform on [0, vocab)."""
     rng = np.random.Generator(np.random.PCG64(seed))

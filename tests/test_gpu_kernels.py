@@ -1,0 +1,179 @@
+"""Each CUDA kernel against the oracle's function for the same operation, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import rsd_inputs as ri
+from paper_2501_19324_b200 import binding as rb
+
+pytestmark = pytest.mark.gpu
+
+
+def dev(a, dtype=None):
+    t = torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    return t.to(dtype) if dtype is not None else t
+
+
+def test_input_generators_agree_bit_for_bit():
+    sh = ri.SHAPES["tiny_draft"]
+    for bf16 in (False, True):
+        g = ri.gpu_model_tensors(sh, 1, 3, bf16, ri.HEAD_REWARD_SIGMOID)
+        c = ri.cpu_model_weights(sh, 1, 3, bf16, ri.HEAD_REWARD_SIGMOID)
+        assert np.array_equal(g["tok_embed"].float().cpu().numpy(), c["tok_embed"])
+        assert np.array_equal(g["head"].float().cpu().numpy(), c["head"])
+        l = c["layers"][1]
+        assert np.array_equal(g["wqkv"][1].float().cpu().numpy(), np.concatenate([l["wq"], l["wk"], l["wv"]]))
+        assert np.array_equal(g["wgu"][1].float().cpu().numpy(), np.concatenate([l["wgate"], l["wup"]]))
+        assert np.array_equal(g["wo"][1].float().cpu().numpy(), l["wo"])
+        assert np.array_equal(g["wdown"][1].float().cpu().numpy(), l["wdown"])
+
+
+def test_philox_matches_oracle_on_many_counters():
+    rng = np.random.default_rng(0)
+    n = 1 << 16
+    ctr = rng.integers(0, 2 ** 32, size=(n, 4), dtype=np.uint64).astype(np.uint32)
+    ctr[0] = 0
+    ctr[1] = 0xFFFFFFFF
+    key = np.array([0x12345678, 0x9ABCDEF0], dtype=np.uint32)
+    got = rb.k_philox(dev(ctr.view(np.int32)), dev(key.view(np.int32))).cpu().numpy().view(np.uint32)
+    for i in list(range(64)) + list(rng.integers(0, n, size=192)):
+        assert np.array_equal(got[i], oracle.philox4x32_10(ctr[i], key))
+    zero = rb.k_philox(dev(np.zeros((1, 4), np.int32)), dev(np.zeros(2, np.int32))).cpu().numpy().view(np.uint32)
+    assert [hex(v) for v in zero[0]] == ["0x6627e8d5", "0xe169c58d", "0xbc57ac4c", "0x9b00dbd8"]
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+@pytest.mark.parametrize("M,N,K", [(1, 1024, 256), (4, 688 * 2, 256), (7, 256, 688), (33, 1000, 512), (130, 257, 1024)])
+def test_gemm_simt(M, N, K, bf16):
+    rng = np.random.default_rng(M * 1000 + N)
+    W = ri.cpu_tensor(1, 77, N, K, bf16)
+    x = rng.normal(size=(M, K)).astype(np.float32)
+    dt = torch.bfloat16 if bf16 else torch.float32
+    xd = dev(x, dt)
+    want = oracle.matmul(W, xd.float().cpu().numpy())
+    y0 = rng.normal(size=(M, N)).astype(np.float32)
+    got = rb.k_gemm(dev(W, dt), xd, impl=1).cpu().numpy()
+    np.testing.assert_allclose(got, want, rtol=0, atol=2e-5 * np.sqrt(K))
+    acc = rb.k_gemm(dev(W, dt), xd, y=dev(y0), accumulate=True, impl=1).cpu().numpy()
+    np.testing.assert_allclose(acc, want + y0, rtol=0, atol=2e-5 * np.sqrt(K))
+
+
+def test_rmsnorm_rope_swiglu():
+    rng = np.random.default_rng(1)
+    x = rng.normal(size=(5, 1536)).astype(np.float32) * 3
+    g = (1 + 0.1 * rng.normal(size=1536)).astype(np.float32)
+    got = rb.k_rmsnorm(dev(x), dev(g), 1e-6).cpu().numpy()
+    want = np.stack([oracle.rmsnorm(x[i], g, 1e-6) for i in range(5)])
+    np.testing.assert_allclose(got, want, rtol=0, atol=2e-6 * np.abs(want).max())
+    got16 = rb.k_rmsnorm(dev(x), dev(g, torch.bfloat16), 1e-6).float().cpu().numpy()
+    g16 = dev(g, torch.bfloat16).float().cpu().numpy()
+    want16 = np.stack([oracle.rmsnorm(x[i], g16, 1e-6) for i in range(5)])
+    np.testing.assert_allclose(got16, want16, rtol=2 ** -8, atol=0)
+
+    for hd in (64, 128):
+        v = rng.normal(size=(6, 3, hd)).astype(np.float32)
+        pos = np.array([0, 1, 17, 255, 4095, 16383], dtype=np.int32)
+        got = rb.k_rope(dev(v.copy()), dev(pos), 1e4).cpu().numpy()
+        want = np.stack([[oracle.rope(v[t, h], pos[t], 1e4) for h in range(3)] for t in range(6)])
+        np.testing.assert_allclose(got, want, rtol=0, atol=1e-6)
+
+    gu = rng.normal(size=(4, 2 * 688)).astype(np.float32) * 2
+    got = rb.k_swiglu(dev(gu), torch.float32).cpu().numpy()
+    a, b = gu[:, :688].astype(np.float64), gu[:, 688:].astype(np.float64)
+    np.testing.assert_allclose(got, a / (1 + np.exp(-a)) * b, rtol=0, atol=1e-6)
+
+
+@pytest.mark.parametrize("temperature", [0.0, 0.7])
+def test_sampling_matches_oracle(temperature):
+    rng = np.random.default_rng(2)
+    B, V, v_limit = 6, 5003, 4999
+    logits = rng.normal(size=(B, V)).astype(np.float32)
+    logits[0, 4] = logits[0, 9] = 50.0            # exact tie: lowest id wins when greedy
+    logits[1, v_limit + 1] = 99.0                 # beyond the shared vocabulary: never chosen
+    row = np.array([0, 1, 2, 3, -1, 7], dtype=np.int32)
+    pos = np.array([5, 5, 9, 1000, 3, 70000], dtype=np.int32)
+    got = rb.k_sample(dev(logits), v_limit, temperature, 1234, 2, dev(row), dev(pos)).cpu().numpy()
+    for b in range(B):
+        if row[b] < 0:
+            continue
+        want, margin = oracle.sample(logits[b].astype(np.float64), v_limit, temperature, 1234, 2, row[b], pos[b] + 1)
+        if margin > 1e-4 or temperature == 0.0:
+            assert got[b] == want, (b, got[b], want, margin)
+    if temperature == 0.0:
+        assert got[0] == 4
+
+
+def test_gate_compaction_all_masks_and_large():
+    # every mask of 12 rows: brute-force serial loop against the ballot / prefix path
+    B = 12
+    for mask in range(0, 1 << B, 37):
+        r = np.array([(0.9 if (mask >> b) & 1 else 0.1) for b in range(B)], dtype=np.float32)
+        live = np.array([1 if b % 5 else 0 for b in range(B)], dtype=np.uint8)
+        acc, rej, n = rb.k_gate_compact(dev(r), dev(live), 0.5)
+        want_rej = [b for b in range(B) if live[b] and r[b] < 0.5]
+        assert int(n.item()) == len(want_rej)
+        assert rej.cpu().numpy()[:len(want_rej)].tolist() == want_rej
+        assert acc.cpu().numpy().tolist() == [int(live[b] and r[b] >= 0.5) for b in range(B)]
+    rng = np.random.default_rng(3)
+    for B, p in [(1, 0.5), (1023, 0.3), (1024, 0.9), (1025, 0.1), (70001, 0.7), (1 << 20, 0.5)]:
+        r = rng.random(B).astype(np.float32)
+        live = (rng.random(B) < 0.95).astype(np.uint8)
+        delta = np.float32(1 - p)
+        acc, rej, n = rb.k_gate_compact(dev(r), dev(live), float(delta))
+        want = np.nonzero((live == 1) & ~(r >= delta))[0]
+        assert int(n.item()) == len(want)
+        assert np.array_equal(rej.cpu().numpy()[:len(want)], want)
+        assert np.array_equal(acc.cpu().numpy(), ((live == 1) & (r >= delta)).astype(np.uint8))
+    # r == delta accepts; NaN rejects
+    r = np.array([0.7, np.nan, np.nextafter(np.float32(0.7), np.float32(0))], dtype=np.float32)
+    acc, rej, n = rb.k_gate_compact(dev(r), dev(np.ones(3, np.uint8)), 0.7)
+    assert acc.cpu().numpy().tolist() == [1, 0, 0] and rej.cpu().numpy()[:2].tolist() == [1, 2]
+
+
+def paged_kv(rng, B, KV, hd, ctx, dtype, max_pages):
+    """Random K/V per row scattered over randomly permuted pages; returns pool, table, dense K, V."""
+    n_pages_row = [(c + 15) // 16 for c in ctx]
+    total = sum(n_pages_row)
+    perm = rng.permutation(total + 5)
+    pool = np.zeros((total + 5, 2, KV, 16, hd), dtype=np.float32)
+    table = np.zeros((B, max_pages), dtype=np.int32)
+    Ks, Vs = [], []
+    nxt = 0
+    for b in range(B):
+        K = rng.normal(size=(ctx[b], KV, hd)).astype(np.float32)
+        V = rng.normal(size=(ctx[b], KV, hd)).astype(np.float32)
+        for i in range(n_pages_row[b]):
+            pg = perm[nxt]; nxt += 1
+            table[b, i] = pg
+            n = min(16, ctx[b] - 16 * i)
+            pool[pg, 0, :, :n] = K[16 * i:16 * i + n].transpose(1, 0, 2)
+            pool[pg, 1, :, :n] = V[16 * i:16 * i + n].transpose(1, 0, 2)
+        Ks.append(K); Vs.append(V)
+    pool_d = dev(pool, dtype)
+    pool_back = pool_d.float().cpu().numpy()
+    for b in range(B):       # the oracle sees the values as stored (bf16-rounded when 16-bit)
+        for i in range(n_pages_row[b]):
+            n = min(16, ctx[b] - 16 * i)
+            Ks[b][16 * i:16 * i + n] = pool_back[table[b, i], 0, :, :n].transpose(1, 0, 2)
+            Vs[b][16 * i:16 * i + n] = pool_back[table[b, i], 1, :, :n].transpose(1, 0, 2)
+    return pool_d, dev(table), Ks, Vs
+
+
+@pytest.mark.parametrize("dtype,hd,H,KV", [(torch.float32, 64, 4, 2), (torch.bfloat16, 128, 12, 2),
+                                          (torch.bfloat16, 128, 28, 4), (torch.bfloat16, 128, 8, 1)])
+def test_decode_attention_against_definition(dtype, hd, H, KV):
+    rng = np.random.default_rng(4)
+    ctx = [1, 15, 16, 17, 33, 250, 1031]
+    B = len(ctx)
+    max_pages = 70
+    pool, table, Ks, Vs = paged_kv(rng, B, KV, hd, ctx, dtype, max_pages)
+    q = rng.normal(size=(B, H, hd)).astype(np.float32)
+    got = rb.k_attn_decode(dev(q), pool, table, dev(np.array(ctx, np.int32)), KV).cpu().numpy()
+    for b in range(B):
+        for h in range(H):
+            g = h // (H // KV)
+            s = Ks[b][:, g].astype(np.float64) @ q[b, h].astype(np.float64) / np.sqrt(hd)
+            p = np.exp(s - s.max()); p /= p.sum()
+            want = p @ Vs[b][:, g].astype(np.float64)
+            np.testing.assert_allclose(got[b, h], want, rtol=0, atol=2e-5)

@@ -1,0 +1,113 @@
+"""Step-loop parity of the CUDA library against the oracle (Algorithm 1 batched over rows)."""
+import numpy as np
+import pytest
+
+import rsd_inputs as ri
+from helpers import build_pair, parity_step, compare_counters, compare_state
+
+pytestmark = pytest.mark.gpu
+
+TINY = (ri.SHAPES["tiny_draft"], ri.SHAPES["tiny_draft"], ri.SHAPES["tiny_target"])
+MINI = (ri.SHAPES["mini_draft"], ri.SHAPES["mini_draft"], ri.SHAPES["mini_target"])
+# fp32 path: fp32 sums against fp64 sums; 16-bit path: the bounds asked of bf16 arithmetic
+TOL32 = dict(tol_logits=2e-4, tol_reward=1e-5, margin_tok=1e-3, margin_gate=1e-4)
+TOL16 = dict(tol_logits=3e-2, tol_reward=1e-2, margin_tok=5e-2, margin_gate=1e-2)
+
+
+def test_tiny_fp32_config_all_deltas():
+    """Tiny fp32 models, batch 4, 64-token prompts, step ends at id 13 or after 32 tokens, 4 steps,
+    greedy; delta = 0.7 as configured, plus the median reward (both branches) and the two limits."""
+    prompts = ri.prompts(0, 4, 64, 64, 1024)
+    base = dict(max_step_tokens=32, max_steps=4, max_seq_tokens=64 + 4 * 32, step_end_id=13, temperature=0.0, seed=0)
+    eng, loop = build_pair(TINY, bf16=False, prompts=prompts, loop_kwargs=base)
+    compare_state(eng, loop)
+    r0 = loop.step(0.0)["rewards"]
+    median = float(np.median(r0))
+    for delta in (0.7, median, 0.0, 1.5):
+        eng, loop = build_pair(TINY, bf16=False, prompts=prompts, loop_kwargs=base)
+        stats = {}
+        n_acc = 0
+        for _ in range(4):
+            g, o = parity_step(eng, loop, delta, stats=stats, **TOL32)
+            n_acc += int(g["accept"].sum())
+        compare_counters(eng, loop)
+        assert stats["tokens_compared"] >= 0.9 * stats["tokens"]
+        if delta == 0.0:
+            assert n_acc == 16 and eng.counters()["gen_tokens"][2] == 0
+        if delta == 1.5:
+            assert n_acc == 0 and eng.counters()["gen_tokens"][2] == eng.counters()["gen_tokens"][0]
+        assert not g["live"].any()          # four steps were the budget
+        eng.close()
+
+
+def test_tiny_free_running_equals_oracle_when_margins_are_clear():
+    """Without forcing, wherever every margin of the oracle's trace is clear the GPU must walk the
+    same path by itself: same tokens, gate decisions and integer state."""
+    prompts = ri.prompts(5, 3, 9, 30, 1024)
+    base = dict(max_step_tokens=12, max_steps=3, max_seq_tokens=96, step_end_id=3, step_end_mod=7,
+                temperature=0.7, seed=4)
+    eng, loop = build_pair(TINY, bf16=False, prompts=prompts, loop_kwargs=base)
+    delta = 0.5
+    for _ in range(3):
+        o = loop.step(delta)
+        margins = [m for key in ("draft_trace", "target_trace") for tr in o[key] if tr for m in tr["margin"]]
+        gate_margin = np.abs(o["rewards"][o["step_len"] > 0] - delta).min() if (o["step_len"] > 0).any() else 1.0
+        if min(margins) < 1e-3 or gate_margin < 1e-4:
+            pytest.skip("a margin of the oracle trace is too small for a free-running comparison")
+        g = eng.step(delta)
+        assert np.array_equal(g["accept"], o["accept"]) and np.array_equal(g["step_len"], o["step_len"])
+        for b in range(3):
+            assert g["step_tokens"][b, :o["step_len"][b]].tolist() == list(o["step_tokens"][b])
+        compare_state(eng, loop)
+    compare_counters(eng, loop)
+
+
+def test_ragged_steps_eos_and_dead_rows():
+    """Ragged prompts, steps of different lengths (delimiter by residue), an EOS id, a row that has
+    no room to start, and rows that stop at different times."""
+    tokens, offsets = ri.prompts(7, 6, 3, 40, 1024)
+    base = dict(max_step_tokens=9, max_steps=5, max_seq_tokens=72, step_end_id=2, step_end_mod=5, eos_id=77,
+                temperature=0.7, seed=9)
+    # row 5 gets a prompt that leaves no room for a step
+    long = np.arange(64, dtype=np.int32)
+    tokens = np.concatenate([tokens[:offsets[5]], long]).astype(np.int32)
+    offsets = offsets.copy(); offsets[6] = offsets[5] + 64
+    eng, loop = build_pair(TINY, bf16=False, prompts=(tokens, offsets), loop_kwargs=base)
+    r0 = loop.step(0.0)["rewards"]
+    delta = float(np.median(r0[r0 > 0]))
+    eng, loop = build_pair(TINY, bf16=False, prompts=(tokens, offsets), loop_kwargs=base)
+    lens = set()
+    for _ in range(5):
+        g, o = parity_step(eng, loop, delta, **TOL32)
+        lens.update(g["step_len"].tolist())
+        assert g["step_len"][5] == 0 and g["live"][5] == 0
+    assert len(lens) > 3
+    compare_counters(eng, loop)
+
+
+def test_mini_bf16_models():
+    """16-bit weights, head_dim 128, Gumbel-max at T = 0.7, chunked multi-token passes."""
+    prompts = ri.prompts(2, 5, 20, 70, 4096)
+    base = dict(max_step_tokens=10, max_steps=3, max_seq_tokens=112, step_end_id=1, step_end_mod=6,
+                temperature=0.7, seed=21)
+    eng, loop = build_pair(MINI, bf16=True, prompts=prompts, loop_kwargs=base)
+    r0 = loop.step(0.0)["rewards"]
+    delta = float(np.sort(r0)[1])
+    eng, loop = build_pair(MINI, bf16=True, prompts=prompts, loop_kwargs=base, engine_kwargs=dict(max_chunk_tokens=64))
+    stats = {}
+    for _ in range(3):
+        parity_step(eng, loop, delta, stats=stats, **TOL16)
+    compare_counters(eng, loop)
+    print("mini bf16 parity:", stats)
+
+
+def test_page_pool_exhaustion_is_an_error_not_a_fault():
+    from paper_2501_19324_b200 import RsdError
+    prompts = ri.prompts(0, 4, 64, 64, 1024)
+    base = dict(max_step_tokens=32, max_steps=4, max_seq_tokens=192, step_end_id=13, temperature=0.0, seed=0)
+    sh = ri.SHAPES["tiny_draft"]
+    page_bytes = sh.n_layers * 2 * sh.n_kv_heads * 16 * sh.head_dim * 4
+    with pytest.raises(RsdError) as e:
+        build_pair(TINY, bf16=False, prompts=prompts, loop_kwargs=base,
+                   engine_kwargs=dict(kv_bytes=[page_bytes * 10, page_bytes * 400, page_bytes * 800]))
+    assert e.value.code == -3

@@ -192,8 +192,8 @@ def test_philox_known_answers_and_uniform_range():
         c, k = rng.integers(0, 2 ** 32, size=4, dtype=np.uint64), rng.integers(0, 2 ** 32, size=2, dtype=np.uint64)
         assert np.array_equal(oracle.philox4x32_10(c, k), ri.philox4x32_10(c, k))
     lib = oracle.lib()
-    assert lib.orc_uniform_from_bits(0) == 0.5 / 2 ** 24
-    assert lib.orc_uniform_from_bits(0xFFFFFFFF) == 1.0 - 0.5 / 2 ** 24
+    assert lib.orc_uniform_from_bits(0) == 0.5 / 2 ** 23
+    assert lib.orc_uniform_from_bits(0xFFFFFFFF) == 1.0 - 0.5 / 2 ** 23
     # counter layout: word index%4 of block (index/4, position, row, stream), key = seed halves
     seed = (0xABCDEF01 << 32) | 0x12345678
     blk = oracle.philox4x32_10([9 // 4, 40, 3, 2], [0x12345678, 0xABCDEF01])
