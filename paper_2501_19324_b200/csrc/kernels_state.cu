@@ -20,8 +20,8 @@ __global__ void __launch_bounds__(1024) reserve_pages_kernel(RowState st, int wh
     const int z = st.z_len[b];
     const bool live = st.live[b] != 0;
     switch (mode) {
-      case kReservePrefillDraft: need = z - 1; break;
-      case kReservePrefillPrm: need = z; break;
+      case kReservePrefillDraft: need = live ? z - 1 : 0; break;
+      case kReservePrefillPrm: need = live ? z : 0; break;
       case kReserveStepDraft: need = live ? z - 1 + st.C : 0; break;
       case kReserveScorePrm: need = live ? z + st.gen_len[0][b] : 0; break;
       case kReserveTarget: need = (live && !st.accept[b]) ? z - 1 + st.C : 0; break;
