@@ -1,0 +1,316 @@
+#!/usr/bin/env python
+"""Benchmark of the RSD step loop on B200: tokens committed per second by rsd_step.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload cfg2|mini]
+
+A "step" is one rsd_step: draft decode of one reasoning step for every live row, PRM scoring, the
+threshold gate, target re-decode of the rejected rows, commit.  The default workload is the
+1.5B-shape draft and PRM with the 7B-shape target in bf16, batch 32, prompts of 128..512 uniform
+random tokens, steps of at most 128 tokens, Gumbel-max sampling at temperature 0.7, delta set on a
+calibration pass to the reward quantile that accepts about 70 % of the draft steps.  All inputs are
+seeded and synthetic (random-init weights, random prompts).
+
+With N > 1 (torchrun) every rank runs an independent replica of the workload on its own GPU with its
+own prompts; there is no collective on the data path.  `--impl reference` times the CPU oracle on a
+bounded sample of the same workload on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import rsd_inputs as ri  # noqa: E402
+
+METRIC = "rsd_step_tokens_per_sec"
+UNIT = "tokens/s"
+
+WORKLOADS = {
+    # name: (draft, prm, target shapes, batch, prompt lo, hi, step cap)
+    "cfg2": ("1.5b", "1.5b", "7b", 32, 128, 512, 128),
+    "mini": ("mini_draft", "mini_draft", "mini_target", 8, 32, 96, 16),
+}
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return d["hbm_gbs"], d["bf16_tflops_sustained"], "measured"
+    return 6650.0, 1400.0, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 7:
+                continue
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def cpu_cores() -> int:
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+def mem_available_gb() -> float:
+    try:
+        for line in open("/proc/meminfo"):
+            if line.startswith("MemAvailable"):
+                return int(line.split()[1]) / 1e6
+    except OSError:
+        pass
+    return 0.0
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle on a bounded sample of the workload
+# ------------------------------------------------------------------------------------------------
+class OracleSample:
+    """One row of the workload pushed through the oracle's step loop for one short step.
+
+    level 0: 8-token prompt, 2-token step, forced rejection, so draft, PRM and target all run;
+    level 1: 4-token prompt, 1-token step, accepted (draft and PRM only) -- used when many steps are
+    requested or the host has too little memory for the target's fp32 weights."""
+
+    def __init__(self, workload: str, level: int):
+        from oracle import OracleModel
+        d, p, t, _, _, _, _ = WORKLOADS[workload]
+        self.level = level
+        self.shapes = [ri.SHAPES[d], ri.SHAPES[p], ri.SHAPES[t]]
+        heads = (ri.HEAD_LM, ri.HEAD_REWARD_SIGMOID, ri.HEAD_LM)
+        self.models = []
+        for slot, (sh, hk) in enumerate(zip(self.shapes, heads)):
+            with_layers = not (slot == 2 and level == 1)
+            self.models.append(OracleModel(ri.cpu_model_weights(sh, slot, 0, True, hk, with_layers=with_layers), slot))
+        self.prompt_len, self.cap = (8, 2) if level == 0 else (4, 1)
+        self.delta = 2.0 if level == 0 else 0.0
+        self.desc = (f"1 row, {self.prompt_len}-token prompt, one step of {self.cap} token(s), "
+                     + ("delta above the PRM range so the target re-decodes it" if level == 0 else
+                        "delta 0 so the step is accepted (target not run)")
+                     + "; full depth and vocabulary, bf16-rounded weights, fp64 arithmetic")
+
+    def run_once(self, seed: int) -> tuple:
+        from oracle.rsd_loop import OracleRSD, LoopConfig
+        tokens, offsets = ri.prompts(100 + seed, 1, self.prompt_len, self.prompt_len, self.shapes[0].vocab)
+        cfg = LoopConfig(max_step_tokens=self.cap, max_steps=1, max_seq_tokens=self.prompt_len + self.cap,
+                         step_end_id=13, temperature=0.7, seed=seed)
+        loop = OracleRSD(*self.models, cfg)
+        t0 = time.perf_counter()
+        loop.prefill([tokens.tolist()])
+        r = loop.step(self.delta)
+        dt = time.perf_counter() - t0
+        return int(r["step_len"].sum()), dt
+
+
+def run_reference(args, rank: int):
+    if rank != 0:
+        return
+    level = 0 if (args.steps + args.warmup) <= 10 and mem_available_gb() > 60 else 1
+    if args.workload != "cfg2":
+        level = 0
+    sample = OracleSample(args.workload, level)
+    for i in range(args.warmup):
+        sample.run_once(i)
+    toks, secs = 0, 0.0
+    for i in range(args.steps):
+        n, dt = sample.run_once(args.warmup + i)
+        toks += n
+        secs += dt
+    value = toks / secs
+    out = {"metric": METRIC, "value": value, "unit": UNIT, "impl": "reference", "n_gpus": args.gpus,
+           "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * secs / args.steps,
+           "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+           "data": "synthetic", "config": workload_config(args),
+           "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_cores(), "kind": "oracle", "sample": sample.desc},
+           "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+           "gpu_launches": 0}
+    print(json.dumps(out), flush=True)
+
+
+def workload_config(args) -> dict:
+    d, p, t, B, lo, hi, cap = WORKLOADS[args.workload]
+    return {"workload": f"{args.workload}: draft {d} / PRM {p} / target {t} shapes, batch {B}, prompts {lo}-{hi} tokens, "
+                        f"step <= {cap} tokens, Gumbel-max T=0.7, delta at the 70% accept quantile",
+            "batch": B, "max_step_tokens": cap, "replicas": args.gpus,
+            "l2": "weights and KV read per decode iteration exceed the 126 MB L2 (no flush needed)"}
+
+
+# ------------------------------------------------------------------------------------------------
+# GPU arm
+# ------------------------------------------------------------------------------------------------
+def run_ours(args, rank: int, world: int):
+    import torch
+    import torch.distributed as dist
+    from paper_2501_19324_b200 import Engine, Model, lib
+
+    local = int(os.environ.get("LOCAL_RANK", 0))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    d, p, t, B, lo, hi, cap = WORKLOADS[args.workload]
+    shapes = [ri.SHAPES[d], ri.SHAPES[p], ri.SHAPES[t]]
+    heads = (ri.HEAD_LM, ri.HEAD_REWARD_SIGMOID, ri.HEAD_LM)
+    models = [Model(sh, ri.gpu_model_tensors(sh, slot, 0, True, hk), hk)
+              for slot, (sh, hk) in enumerate(zip(shapes, heads))]
+    n_steps = args.warmup + args.steps
+    S = hi + n_steps * cap
+    eng = Engine(*models, max_batch=B, max_seq_tokens=S, max_step_tokens=cap, max_steps=n_steps + 1,
+                 step_end_id=13, temperature=0.7, seed=0)
+    tokens, offsets = ri.prompts(1 + rank, B, lo, hi, shapes[0].vocab)
+    pinned_tokens = torch.from_numpy(tokens).pin_memory()
+
+    # calibration pass: rewards of the first step decide delta (30th percentile -> ~70 % accepted)
+    eng.prefill(tokens, offsets)
+    r0 = eng.step(0.0)["rewards"]
+    delta = float(np.sort(r0)[int(0.3 * B)])
+    eng.reset()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(local)
+    launches0 = lib().rsd_debug_launch_count()
+    barrier()
+    sampler.start()
+    e2e_t0 = time.perf_counter()
+    e2e_start = torch.cuda.Event(enable_timing=True); e2e_end = torch.cuda.Event(enable_timing=True)
+    e2e_start.record()
+    eng.prefill(pinned_tokens.numpy(), offsets)          # host prompts -> device inside the call
+    e2e_tokens = 0
+    accepted = live_steps = 0
+    for _ in range(args.warmup):
+        r = eng.step(delta)
+        e2e_tokens += int(r["step_len"].sum())
+    eng.gemm_timing(args.time_stride)
+    barrier()
+    launches1 = lib().rsd_debug_launch_count()
+    t_start = torch.cuda.Event(enable_timing=True); t_end = torch.cuda.Event(enable_timing=True)
+    t_start.record()
+    timed_tokens = 0
+    for _ in range(args.steps):
+        r = eng.step(delta)                                # host outputs: D2H inside the call
+        timed_tokens += int(r["step_len"].sum())
+        accepted += int(r["accept"].sum())
+        live_steps += int((r["step_len"] > 0).sum())
+    t_end.record()
+    barrier()
+    e2e_end.record()
+    torch.cuda.synchronize()
+    launches2 = lib().rsd_debug_launch_count()
+    clocks = sampler.stop()
+    gt = eng.gemm_timing(0)
+    e2e_tokens += timed_tokens
+    ms = t_start.elapsed_time(t_end)
+    e2e_ms = e2e_start.elapsed_time(e2e_end)
+    stats = torch.tensor([ms, e2e_ms, float(timed_tokens), float(e2e_tokens)], dtype=torch.float64, device="cuda")
+    if world > 1:
+        mx = stats.clone(); dist.all_reduce(mx, op=dist.ReduceOp.MAX)
+        sm = stats.clone(); dist.all_reduce(sm, op=dist.ReduceOp.SUM)
+        ms, e2e_ms = float(mx[0]), float(mx[1])
+        timed_tokens, e2e_tokens = float(sm[2]), float(sm[3])
+    counters = eng.counters()
+
+    if rank == 0:
+        hbm, tf, how = peaks()
+        achieved = gt["bytes"] / (gt["ms"] * 1e-3) / 1e9 if gt["ms"] > 0 else None
+        out = {"metric": METRIC, "value": timed_tokens / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
+               "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
+               "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+               "data": "synthetic", "config": workload_config(args),
+               "accept_rate": accepted / max(1, live_steps), "delta": delta,
+               "e2e": {"value": e2e_tokens / (e2e_ms * 1e-3), "unit": UNIT,
+                       "h2d_bytes_per_step": int(tokens.nbytes + offsets.nbytes) // n_steps,
+                       "d2h_bytes_per_step": B * (cap * 4 + 4 + 4 + 1 + 1) + 3 * 32,
+                       "covers": "prefill from host prompts + all warm-up and timed steps"},
+               "gpu_launches": int(launches2 - launches1),
+               "roofline": {"bound": "hbm", "kernel": "weight GEMM (decode, prefill, scoring)", "achieved": achieved,
+                            "peak": hbm, "unit": "GB/s", "frac": (achieved / hbm) if achieved else None,
+                            "traffic": None, "peak_source": how, "timed_launches": gt["launches"],
+                            "timing": f"CUDA events around every {args.time_stride}th GEMM launch of the timed steps"},
+               "flops_paper": counters["flops_paper"], "clocks": clocks,
+               "gen_tokens": counters["gen_tokens"]}
+        if world == 1 and not args.no_cpu_baseline:
+            level = 0 if mem_available_gb() > 60 and args.workload == "cfg2" else (1 if args.workload == "cfg2" else 0)
+            smp = OracleSample(args.workload, level)
+            n, dt = smp.run_once(0)
+            out["cpu_baseline"] = {"value": n / dt, "unit": UNIT, "cores": cpu_cores(), "kind": "oracle",
+                                   "sample": smp.desc, "seconds": dt}
+        print(json.dumps(out), flush=True)
+    eng.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=6)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2", choices=sorted(WORKLOADS))
+    ap.add_argument("--time-stride", type=int, default=16, dest="time_stride")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+    rank = int(os.environ.get("RANK", 0))
+    world = int(os.environ.get("WORLD_SIZE", 1))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+    run_ours(args, rank, world)
+
+
+if __name__ == "__main__":
+    main()

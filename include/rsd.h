@@ -164,6 +164,17 @@ int rsd_debug_get_sampled(rsd_ctx*, int which, int32_t* out);
 int rsd_debug_get_state(rsd_ctx*, int32_t* z_len, int32_t* kv_len, int32_t* n_pages, int32_t* page_table,
                         int32_t* next_page, int32_t* rej_idx, int32_t* n_rej);
 
+/* Timing of the weight GEMMs inside rsd_prefill / rsd_step with CUDA events on the caller's stream:
+ * every `stride`-th GEMM launch is bracketed by two events (stride 0 switches timing off; at most
+ * 8192 launches are held between two synchronisation points of a step).  Each call first returns
+ * what was gathered since the previous call -- summed device time in ms, summed algorithmic bytes
+ * (weights + input read once, output written once, or read and written when accumulated into) and
+ * the number of timed launches -- then clears the totals and installs the new stride.  HOST outputs,
+ * any may be NULL.  Synchronises the device.                                                   */
+int rsd_debug_gemm_timing(rsd_ctx*, int32_t stride, double* ms, double* bytes, uint64_t* launches);
+/* Number of kernels this library has enqueued in this process so far.                          */
+uint64_t rsd_debug_launch_count(void);
+
 /* ---- single kernels (sweeps and unit parity); all pointers DEVICE unless noted ------------ */
 
 /* y[M, N] (fp32) = (accumulate ? y : 0) + x[M, K] * W[N, K]^T, W and x of element type `dtype`.

@@ -51,7 +51,7 @@ class rsd_counters(ctypes.Structure):
 
 EXPORTS = ["rsd_query_sizes", "rsd_create", "rsd_load_models", "rsd_prefill", "rsd_step", "rsd_flops_counters",
            "rsd_reset", "rsd_destroy", "rsd_last_error", "rsd_debug_force", "rsd_debug_get_logits",
-           "rsd_debug_get_sampled", "rsd_debug_get_state", "rsd_k_gemm", "rsd_k_gemm_scratch_bytes",
+           "rsd_debug_get_sampled", "rsd_debug_get_state", "rsd_debug_gemm_timing", "rsd_debug_launch_count", "rsd_k_gemm", "rsd_k_gemm_scratch_bytes",
            "rsd_k_attn_decode", "rsd_k_attn_decode_scratch_bytes", "rsd_k_gate_compact", "rsd_k_rmsnorm",
            "rsd_k_rope", "rsd_k_swiglu", "rsd_k_sample", "rsd_k_philox"]
 
@@ -80,6 +80,9 @@ def lib():
         L.rsd_debug_get_logits.argtypes = [vp, c_int32, vp]
         L.rsd_debug_get_sampled.argtypes = [vp, c_int32, vp]
         L.rsd_debug_get_state.argtypes = [vp] * 8
+        L.rsd_debug_gemm_timing.argtypes = [vp, c_int32, vp, vp, vp]
+        L.rsd_debug_launch_count.argtypes = []
+        L.rsd_debug_launch_count.restype = c_uint64
         L.rsd_k_gemm.argtypes = [vp, vp, vp, c_int32, c_int32, c_int32, c_int32, c_int32, c_int32, vp, c_size_t, vp]
         L.rsd_k_gemm_scratch_bytes.argtypes = [c_int32, c_int32, c_int32]
         L.rsd_k_gemm_scratch_bytes.restype = c_size_t
@@ -201,6 +204,13 @@ class Engine:
     def reset(self):
         _check(lib().rsd_reset(self.ctx), self.ctx)
         self.B = 0
+
+    def gemm_timing(self, stride: int) -> dict:
+        """Returns {ms, bytes, launches} gathered since the last call and installs a new stride."""
+        ms, by, n = c_double(0), c_double(0), c_uint64(0)
+        _check(lib().rsd_debug_gemm_timing(self.ctx, stride, ctypes.addressof(ms), ctypes.addressof(by),
+                                           ctypes.addressof(n)), self.ctx)
+        return dict(ms=ms.value, bytes=by.value, launches=n.value)
 
     # -- parity hooks ---------------------------------------------------------------------------
     def force_tokens(self, which: int, steps: list):

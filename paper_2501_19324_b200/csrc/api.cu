@@ -66,6 +66,14 @@ struct rsd_ctx {
   size_t gemm_scratch_bytes = 0;
   rsd_counters ctr{};
   int last_n_rej = 0;
+  // sampled GEMM timing (rsd_debug_gemm_timing)
+  int time_stride = 0;
+  uint64_t gemm_calls = 0;
+  std::vector<cudaEvent_t> ev;          // pairs: start, stop
+  std::vector<double> ev_bytes;
+  size_t ev_used = 0;
+  double timed_ms = 0, timed_bytes = 0;
+  uint64_t timed_launches = 0;
   std::string err;
 };
 
@@ -226,10 +234,13 @@ int check_config(const rsd_config* cfg, const char** why) {
   return RSD_OK;
 }
 
+int drain_gemm_events(rsd_ctx* c);
+
 // ---- device scalars <-> host ---------------------------------------------------------------
 int read_scalars(rsd_ctx* c, cudaStream_t s, Scalars* out) {
   CU(cudaMemcpyAsync(c->pinned, c->d_scalars, sizeof(Scalars), cudaMemcpyDeviceToHost, s));
   CU(cudaStreamSynchronize(s));
+  if (c->ev_used) { int rc_ = drain_gemm_events(c); if (rc_) return rc_; }
   memcpy(out, c->pinned, sizeof(Scalars));
   if (out->err == RSD_ERR_OOM_PAGES) return fail(c, RSD_ERR_OOM_PAGES, "KV page pool or pass list exhausted%s");
   if (out->err != 0) { c->poisoned = true; return fail(c, RSD_ERR_TIMEOUT, "device-side error flag raised%s"); }
@@ -237,9 +248,32 @@ int read_scalars(rsd_ctx* c, cudaStream_t s, Scalars* out) {
 }
 
 // ---- one model pass over T token slots ------------------------------------------------------
+// Folds the finished event pairs into the running totals.  The stream must be idle.
+int drain_gemm_events(rsd_ctx* c) {
+  for (size_t i = 0; i < c->ev_used; ++i) {
+    float ms = 0.f;
+    CU(cudaEventElapsedTime(&ms, c->ev[2 * i], c->ev[2 * i + 1]));
+    c->timed_ms += ms;
+    c->timed_bytes += c->ev_bytes[i];
+    ++c->timed_launches;
+  }
+  c->ev_used = 0;
+  return RSD_OK;
+}
+
 int gemm(rsd_ctx* c, const ModelHost& M, const void* W, const void* xin, float* y, int Mrows, int N, int K,
          int accumulate, const int32_t* n_active, cudaStream_t s) {
+  const bool timed = c->time_stride > 0 && (c->gemm_calls++ % (uint64_t)c->time_stride) == 0 &&
+                     c->ev_used < c->ev_bytes.size();
+  if (timed) CU(cudaEventRecord(c->ev[2 * c->ev_used], s));
   CU(launch_gemm(M.m.dtype, W, xin, y, Mrows, N, K, accumulate, 0, c->gemm_scratch, c->gemm_scratch_bytes, n_active, s));
+  if (timed) {
+    CU(cudaEventRecord(c->ev[2 * c->ev_used + 1], s));
+    // algorithmic bytes: the weight matrix and the input once, the output once (twice when added to)
+    c->ev_bytes[c->ev_used] = (double)N * K * M.elem + (double)Mrows * K * M.elem +
+                              (double)Mrows * N * 4.0 * (accumulate ? 2.0 : 1.0);
+    ++c->ev_used;
+  }
   return RSD_OK;
 }
 
@@ -311,7 +345,7 @@ int decode_phase(rsd_ctx* c, int which, int phase, int n_slots, cudaStream_t s) 
     if (rc) return rc;
     if (c->dbg_logits[phase]) {
       scatter_logits_kernel<<<n_slots, 256, 0, s>>>(c->logits, c->st.pass_tok_row, c->dbg_logits[phase], m.vocab, c->C, j, c->st.n_active);
-      CU(cudaGetLastError());
+      CU(launched(1));
     }
     SampleArgs a{c->logits, n_slots, m.vocab, c->v_limit, c->cfg.temperature, c->cfg.seed, which,
                  c->st.pass_tok_row, c->st.pass_tok_pos, c->sampled_slots, c->st.n_active};
@@ -476,7 +510,7 @@ int rsd_prefill(rsd_ctx* c, const int32_t* tokens, const int32_t* offsets, int32
   CU(cudaMemcpyAsync(c->st.pass_tok_id, tokens, sizeof(int32_t) * total, cudaMemcpyHostToDevice, s));
   CU(cudaMemcpyAsync(c->st.pass_tok_row, offsets, sizeof(int32_t) * (B + 1), cudaMemcpyHostToDevice, s));
   init_rows_kernel<<<B, 128, 0, s>>>(c->st, c->st.pass_tok_id, c->st.pass_tok_row, B);
-  CU(cudaGetLastError());
+  CU(launched(1));
   CU(cudaStreamSynchronize(s));  // the staging buffers are reused below
   CU(launch_reserve_pages(c->st, RSD_DRAFT, kReservePrefillDraft, s));
   CU(launch_reserve_pages(c->st, RSD_PRM, kReservePrefillPrm, s));
@@ -589,6 +623,7 @@ int rsd_flops_counters(rsd_ctx* c, rsd_counters* out) {
 int rsd_destroy(rsd_ctx* c) {
   if (!c) return RSD_OK;
   cudaDeviceSynchronize();
+  for (cudaEvent_t e : c->ev) cudaEventDestroy(e);
   if (c->pinned) cudaFreeHost(c->pinned);
   delete c;
   return RSD_OK;
@@ -650,6 +685,28 @@ int rsd_debug_get_state(rsd_ctx* c, int32_t* z_len, int32_t* kv_len, int32_t* n_
   if (n_rej) *n_rej = c->last_n_rej;
   return RSD_OK;
 }
+
+int rsd_debug_gemm_timing(rsd_ctx* c, int32_t stride, double* ms, double* bytes, uint64_t* launches) {
+  if (!c || stride < 0) return RSD_ERR_ARG;
+  CU(cudaDeviceSynchronize());
+  int rc = drain_gemm_events(c);
+  if (rc) return rc;
+  if (ms) *ms = c->timed_ms;
+  if (bytes) *bytes = c->timed_bytes;
+  if (launches) *launches = c->timed_launches;
+  c->timed_ms = 0; c->timed_bytes = 0; c->timed_launches = 0;
+  c->gemm_calls = 0;
+  if (stride > 0 && c->ev.empty()) {
+    const size_t pairs = 8192;
+    c->ev.resize(2 * pairs);
+    for (auto& e : c->ev) CU(cudaEventCreate(&e));
+    c->ev_bytes.assign(pairs, 0.0);
+  }
+  c->time_stride = stride;
+  return RSD_OK;
+}
+
+uint64_t rsd_debug_launch_count(void) { return launches_total(); }
 
 // ---- single kernels -------------------------------------------------------------------------
 #define KCU(call)                                     \

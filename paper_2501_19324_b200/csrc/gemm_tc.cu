@@ -2,7 +2,16 @@
 #include "common.cuh"
 #include "kernels.cuh"
 
+#include <atomic>
+
 namespace rsd {
+
+static std::atomic<uint64_t> g_launches{0};
+cudaError_t launched(int n_kernels) {
+  g_launches.fetch_add((uint64_t)n_kernels, std::memory_order_relaxed);
+  return cudaGetLastError();
+}
+uint64_t launches_total() { return g_launches.load(std::memory_order_relaxed); }
 
 bool gemm_tc_supported(int dtype, int M, int N, int K) { (void)dtype; (void)M; (void)N; (void)K; return false; }
 size_t gemm_scratch_bytes(int M) { (void)M; return 4096; }

@@ -8,6 +8,11 @@
 
 namespace rsd {
 
+// Every launcher reports the kernels it enqueued; the total is what a caller can claim as its own
+// GPU launches.
+cudaError_t launched(int n_kernels);   // adds to the count and returns cudaGetLastError()
+uint64_t launches_total();
+
 constexpr int kPageTokens = 16;   // tokens per KV page
 constexpr int kMaxBatch = 1024;   // rows per context (one thread per row in the state kernels)
 

@@ -32,7 +32,7 @@ cudaError_t launch_embed(int dtype, const void* embed, PassView p, float* x, int
   if (p.T <= 0) return cudaSuccess;
   if (dtype == 1) embed_kernel<__nv_bfloat16><<<p.T, 128, 0, s>>>((const __nv_bfloat16*)embed, p, x, d);
   else embed_kernel<float><<<p.T, 128, 0, s>>>((const float*)embed, p, x, d);
-  return cudaGetLastError();
+  return launched(1);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -75,7 +75,7 @@ cudaError_t launch_rmsnorm(int dtype, const float* x, const void* gain, void* ou
     rmsnorm_kernel<__nv_bfloat16, __nv_bfloat16><<<T, threads, 0, s>>>(x, (const __nv_bfloat16*)gain, (__nv_bfloat16*)out, d, eps, src, n_active);
   else
     rmsnorm_kernel<float, float><<<T, threads, 0, s>>>(x, (const float*)gain, (float*)out, d, eps, src, n_active);
-  return cudaGetLastError();
+  return launched(1);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -149,7 +149,7 @@ cudaError_t launch_gemm_simt(int dtype, const void* W, const void* x, float* y, 
     gemv_splitk_kernel<__nv_bfloat16, MT><<<grid, 256, 0, s>>>((const __nv_bfloat16*)W, (const __nv_bfloat16*)x, y, M, N, K, ks, accumulate, n_active);
   else
     gemv_splitk_kernel<float, MT><<<grid, 256, 0, s>>>((const float*)W, (const float*)x, y, M, N, K, ks, accumulate, n_active);
-  return cudaGetLastError();
+  return launched(1);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -169,7 +169,7 @@ cudaError_t launch_rope_table(float2* table, int n_pos, int hd, float theta, cud
   const int n = n_pos * (hd / 2);
   if (n <= 0) return cudaSuccess;
   rope_table_kernel<<<(n + 255) / 256, 256, 0, s>>>(table, n_pos, hd / 2, (double)theta, (double)hd);
-  return cudaGetLastError();
+  return launched(1);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -222,7 +222,7 @@ cudaError_t launch_rope_kv(int dtype, const float* qkv, PassView p, float* q_out
     rope_kv_kernel<__nv_bfloat16><<<p.T, 256, 0, s>>>(qkv, p, q_out, (__nv_bfloat16*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd);
   else
     rope_kv_kernel<float><<<p.T, 256, 0, s>>>(qkv, p, q_out, (float*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd);
-  return cudaGetLastError();
+  return launched(1);
 }
 
 // Stand-alone rotary kernel on [T, n_heads, hd] fp32 (angles in fp64).
@@ -243,7 +243,7 @@ __global__ void rope_only_kernel(float* v, const int32_t* pos, int n_heads, int 
 cudaError_t launch_rope_only(float* v, const int32_t* pos, int T, int n_heads, int hd, float theta, cudaStream_t s) {
   if (T <= 0) return cudaSuccess;
   rope_only_kernel<<<T, 128, 0, s>>>(v, pos, n_heads, hd, (double)theta);
-  return cudaGetLastError();
+  return launched(1);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -326,7 +326,7 @@ cudaError_t launch_attn_generic(int dtype, const float* q, PassView p, KvView kv
     if (hd == 128) attn_generic_kernel<float, float, 128><<<blocks, 128, 0, s>>>(q, p, (const float*)kv.pool_layer, kv.page_table, kv.max_pages, (float*)out, H, KV);
     else attn_generic_kernel<float, float, 64><<<blocks, 128, 0, s>>>(q, p, (const float*)kv.pool_layer, kv.page_table, kv.max_pages, (float*)out, H, KV);
   }
-  return cudaGetLastError();
+  return launched(1);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -350,7 +350,7 @@ cudaError_t launch_swiglu(int dtype, const float* gu, void* out, int T, int F, c
   if (blocks > 148 * 8) blocks = 148 * 8;
   if (dtype == 1) swiglu_kernel<__nv_bfloat16><<<blocks, 256, 0, s>>>(gu, (__nv_bfloat16*)out, T, F, n_active);
   else swiglu_kernel<float><<<blocks, 256, 0, s>>>(gu, (float*)out, T, F, n_active);
-  return cudaGetLastError();
+  return launched(1);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -415,7 +415,7 @@ cudaError_t launch_sample(const SampleArgs& a, cudaStream_t s) {
   if (a.n_slots <= 0) return cudaSuccess;
   const int threads = a.v_limit >= 16384 ? 1024 : 256;
   sample_kernel<<<a.n_slots, threads, 0, s>>>(a);
-  return cudaGetLastError();
+  return launched(1);
 }
 
 __global__ void philox_kernel(const uint32_t* ctr, const uint32_t* key, uint32_t* out, int n) {
@@ -429,7 +429,7 @@ __global__ void philox_kernel(const uint32_t* ctr, const uint32_t* key, uint32_t
 cudaError_t launch_philox(const uint32_t* ctr, const uint32_t* key, uint32_t* out, int n, cudaStream_t s) {
   if (n <= 0) return cudaSuccess;
   philox_kernel<<<(n + 255) / 256, 256, 0, s>>>(ctr, key, out, n);
-  return cudaGetLastError();
+  return launched(1);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -467,7 +467,7 @@ cudaError_t launch_reward(int dtype, const float* x, const void* final_norm, con
     reward_kernel<__nv_bfloat16><<<n_rows, 256, 0, s>>>(x, (const __nv_bfloat16*)final_norm, (const __nv_bfloat16*)w_r, head_kind, last_idx, t0, T, d, eps, reward);
   else
     reward_kernel<float><<<n_rows, 256, 0, s>>>(x, (const float*)final_norm, (const float*)w_r, head_kind, last_idx, t0, T, d, eps, reward);
-  return cudaGetLastError();
+  return launched(1);
 }
 
 }  // namespace rsd
@@ -508,7 +508,7 @@ cudaError_t launch_attn_decode(int dtype, const float* q, const void* pool_layer
   else if (dtype == 1) { if (hd == 128) RSD_ATTN(bf, float, 128); else RSD_ATTN(bf, float, 64); }
   else { if (hd == 128) RSD_ATTN(float, float, 128); else RSD_ATTN(float, float, 64); }
 #undef RSD_ATTN
-  return cudaGetLastError();
+  return launched(2);
 }
 
 }  // namespace rsd

@@ -48,7 +48,7 @@ __global__ void __launch_bounds__(1024) reserve_pages_kernel(RowState st, int wh
 
 cudaError_t launch_reserve_pages(const RowState& st, int which, ReserveMode mode, cudaStream_t s) {
   reserve_pages_kernel<<<1, 1024, 0, s>>>(st, which, (int)mode);
-  return cudaGetLastError();
+  return launched(1);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -103,7 +103,7 @@ __global__ void __launch_bounds__(1024) build_pass_kernel(RowState st, int which
 
 cudaError_t launch_build_pass(const RowState& st, int which, PassMode mode, cudaStream_t s) {
   build_pass_kernel<<<1, 1024, 0, s>>>(st, which, (int)mode);
-  return cudaGetLastError();
+  return launched(1);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -133,7 +133,7 @@ __global__ void __launch_bounds__(1024) decode_begin_kernel(RowState st, int pha
 
 cudaError_t launch_decode_begin(const RowState& st, int phase, cudaStream_t s) {
   decode_begin_kernel<<<1, 1024, 0, s>>>(st, phase);
-  return cudaGetLastError();
+  return launched(1);
 }
 
 __global__ void __launch_bounds__(1024) decode_prepare_kernel(RowState st, int which, int n_slots) {
@@ -154,7 +154,7 @@ __global__ void __launch_bounds__(1024) decode_prepare_kernel(RowState st, int w
 cudaError_t launch_decode_prepare(const RowState& st, int which, int n_slots, cudaStream_t s) {
   if (n_slots <= 0) return cudaSuccess;
   decode_prepare_kernel<<<1, 1024, 0, s>>>(st, which, n_slots);
-  return cudaGetLastError();
+  return launched(1);
 }
 
 __device__ __forceinline__ bool ends_step(int t, const LoopParams& lp) {
@@ -195,7 +195,7 @@ cudaError_t launch_decode_update(const RowState& st, int which, int phase, int i
                                  int n_slots, const LoopParams& lp, cudaStream_t s) {
   if (n_slots <= 0) return cudaSuccess;
   decode_update_kernel<<<1, 1024, 0, s>>>(st, which, phase, iter, sampled, n_slots, lp);
-  return cudaGetLastError();
+  return launched(1);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -277,7 +277,7 @@ __global__ void __launch_bounds__(1024) gate_kernel(RowState st, float delta, Lo
 
 cudaError_t launch_gate(const RowState& st, float delta, const LoopParams& lp, cudaStream_t s) {
   gate_kernel<<<1, 1024, 0, s>>>(st, delta, lp);
-  return cudaGetLastError();
+  return launched(1);
 }
 
 // Stand-alone gate + compaction for any B: per-block ballot counts, a scan of the block counts,
@@ -332,7 +332,7 @@ cudaError_t launch_gate_compact_large(const float* rewards, const uint8_t* live,
   gate_count_kernel<<<n_blocks, 1024, 0, s>>>(rewards, live, delta, accept, block_cnt, B);
   gate_scan_kernel<<<1, 1024, 0, s>>>(block_cnt, n_blocks, n_rej);
   gate_write_kernel<<<n_blocks, 1024, 0, s>>>(live, accept, block_cnt, rej_idx, B);
-  return cudaGetLastError();
+  return launched(3);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -375,7 +375,7 @@ cudaError_t launch_commit(const RowState& st, const LoopParams& lp, int32_t* out
                           float* out_rewards, uint8_t* out_accept, uint8_t* out_live, cudaStream_t s) {
   if (st.B <= 0) return cudaSuccess;
   commit_kernel<<<st.B, 128, 0, s>>>(st, lp, out_tokens, out_len, out_rewards, out_accept, out_live);
-  return cudaGetLastError();
+  return launched(1);
 }
 
 }  // namespace rsd
