@@ -201,6 +201,26 @@ int rsd_k_gate_compact(const float* rewards, const uint8_t* live, float delta, u
                        int32_t* rej_idx, int32_t* n_rej, int32_t B, void* scratch, size_t scratch_bytes,
                        void* cuda_stream);
 
+/* The same gate + compaction for callers that cannot allocate device memory -- a serving process
+ * whose GPU memory was handed out once at start-up, a tenant held to a fixed memory budget, code in
+ * a section where an allocation (which may stall the device) is not allowed.  (The paper has no
+ * counterpart to this call: it is a packaging variant of rsd_k_gate_compact, not part of the method.)
+ * Its scratch is a fixed 4 KiB array inside the library's device image, present on every GPU that
+ * loads the library until the process ends, so the caller passes only inputs and outputs and the
+ * call performs no cudaMalloc / cudaFree.  B must lie in 1..RSD_GATE_STATIC_MAX_ROWS, otherwise
+ * RSD_ERR_ARG is returned and rsd_k_gate_compact_static_error() says why.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current); make that first call before starting any stream capture.
+ *   - All calls share the one array, which keeps the previous call's contents; none of it needs
+ *     clearing between calls (every counter a call reads is written by that call first).  Two
+ *     calls that overlap on the GPU -- different streams without ordering, or different host
+ *     threads -- race on it and give wrong lists: order them on one stream or with events.
+ *   - Pointers are DEVICE pointers as for rsd_k_gate_compact; results are identical to it.       */
+#define RSD_GATE_STATIC_MAX_ROWS (1 << 20)
+int rsd_k_gate_compact_static(const float* rewards, const uint8_t* live, float delta, uint8_t* accept,
+                              int32_t* rej_idx, int32_t* n_rej, int32_t B, void* cuda_stream);
+const char* rsd_k_gate_compact_static_error(void); /* library-owned text of its last failure      */
+
 /* out[t, :] = x[t, :] * gain / sqrt(mean(x^2) + eps), x fp32 [T, d], out of element type `dtype`. */
 int rsd_k_rmsnorm(const float* x, const void* gain, void* out, int32_t T, int32_t d, float eps,
                   int32_t dtype, void* cuda_stream);

@@ -52,7 +52,7 @@ class rsd_counters(ctypes.Structure):
 EXPORTS = ["rsd_query_sizes", "rsd_create", "rsd_load_models", "rsd_prefill", "rsd_step", "rsd_flops_counters",
            "rsd_reset", "rsd_destroy", "rsd_last_error", "rsd_debug_force", "rsd_debug_get_logits",
            "rsd_debug_get_sampled", "rsd_debug_get_state", "rsd_debug_gemm_timing", "rsd_debug_launch_count", "rsd_k_gemm", "rsd_k_gemm_scratch_bytes",
-           "rsd_k_attn_decode", "rsd_k_attn_decode_scratch_bytes", "rsd_k_gate_compact", "rsd_k_rmsnorm",
+           "rsd_k_attn_decode", "rsd_k_attn_decode_scratch_bytes", "rsd_k_gate_compact", "rsd_k_gate_compact_static", "rsd_k_gate_compact_static_error", "rsd_k_rmsnorm",
            "rsd_k_rope", "rsd_k_swiglu", "rsd_k_sample", "rsd_k_philox"]
 
 _lib = None
@@ -91,6 +91,9 @@ def lib():
         L.rsd_k_attn_decode_scratch_bytes.argtypes = [c_int32] * 4
         L.rsd_k_attn_decode_scratch_bytes.restype = c_size_t
         L.rsd_k_gate_compact.argtypes = [vp, vp, c_float, vp, vp, vp, c_int32, vp, c_size_t, vp]
+        L.rsd_k_gate_compact_static.argtypes = [vp, vp, c_float, vp, vp, vp, c_int32, vp]
+        L.rsd_k_gate_compact_static_error.argtypes = []
+        L.rsd_k_gate_compact_static_error.restype = ctypes.c_char_p
         L.rsd_k_rmsnorm.argtypes = [vp, vp, vp, c_int32, c_int32, c_float, c_int32, vp]
         L.rsd_k_rope.argtypes = [vp, vp, c_int32, c_int32, c_int32, c_float, vp]
         L.rsd_k_swiglu.argtypes = [vp, vp, c_int32, c_int32, c_int32, vp]
@@ -290,6 +293,13 @@ def k_gate_compact(rewards, live, delta):
     _check(lib().rsd_k_gate_compact(_ptr(rewards), _ptr(live), float(delta), _ptr(accept), _ptr(rej), _ptr(n_rej), B,
                                     _ptr(scratch), scratch.numel(), _stream()))
     return accept, rej, n_rej
+
+
+def k_gate_compact_static(rewards, live, delta, accept, rej, n_rej):
+    """Gate + compaction with the library's built-in scratch: the caller supplies every buffer and the
+    call itself allocates nothing (for hosts that cannot call cudaMalloc).  Returns the status code."""
+    return lib().rsd_k_gate_compact_static(_ptr(rewards), _ptr(live), float(delta), _ptr(accept), _ptr(rej),
+                                           _ptr(n_rej), rewards.numel(), _stream())
 
 
 def k_rmsnorm(x, gain, eps):
