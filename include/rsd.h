@@ -180,8 +180,9 @@ uint64_t rsd_debug_launch_count(void);
 /* y[M, N] (fp32) = (accumulate ? y : 0) + x[M, K] * W[N, K]^T, W and x of element type `dtype`.
  * impl: 0 = pick by shape, 1 = split-K SIMT GEMV path, 2 = tcgen05/TMEM/TMA path (bf16 only,
  * K % 64 == 0, 16-byte aligned rows).  `scratch` (scratch_bytes from rsd_k_gemm_scratch_bytes)
- * holds split-K partial sums and tile counters; the first 4 KiB must be zero before the first
- * call and are left zero by every call.                                                      */
+ * holds split-K partial sums and tile counters; its first 4 KiB + 256 B must be zero before the
+ * first call; the counters are left zero by every call and the int at byte 4096 becomes non-zero
+ * if a bounded device-side wait of the tcgen05 path expired (RSD_ERR_TIMEOUT condition).                                                      */
 int rsd_k_gemm(const void* W, const void* x, float* y, int32_t M, int32_t N, int32_t K, int32_t dtype,
                int32_t accumulate, int32_t impl, void* scratch, size_t scratch_bytes, void* cuda_stream);
 size_t rsd_k_gemm_scratch_bytes(int32_t M, int32_t N, int32_t K);

@@ -267,6 +267,8 @@ def k_gemm(W, x, y=None, accumulate=False, impl=0):
     dt = RSD_BF16 if W.dtype == torch.bfloat16 else RSD_F32
     _check(lib().rsd_k_gemm(_ptr(W), _ptr(x), _ptr(y), M, N, K, dt, int(accumulate), impl, _ptr(scratch), nbytes,
                             _stream()))
+    if nbytes >= 4100 and int(scratch[4096:4100].view(torch.int32).item()) != 0:
+        raise RsdError(-5, "a bounded wait inside the tensor-core GEMM expired")
     return y
 
 

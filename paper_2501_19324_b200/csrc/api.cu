@@ -239,7 +239,13 @@ int drain_gemm_events(rsd_ctx* c);
 // ---- device scalars <-> host ---------------------------------------------------------------
 int read_scalars(rsd_ctx* c, cudaStream_t s, Scalars* out) {
   CU(cudaMemcpyAsync(c->pinned, c->d_scalars, sizeof(Scalars), cudaMemcpyDeviceToHost, s));
+  // the tensor-core GEMM raises its own flag (bounded waits) at byte 4096 of its scratch
+  CU(cudaMemcpyAsync(c->pinned + 128, (char*)c->gemm_scratch + 4096, sizeof(int32_t), cudaMemcpyDeviceToHost, s));
   CU(cudaStreamSynchronize(s));
+  if (*(int32_t*)(c->pinned + 128) != 0) {
+    c->poisoned = true;
+    return fail(c, RSD_ERR_TIMEOUT, "a bounded wait inside the tensor-core GEMM expired%s");
+  }
   if (c->ev_used) { int rc_ = drain_gemm_events(c); if (rc_) return rc_; }
   memcpy(out, c->pinned, sizeof(Scalars));
   if (out->err == RSD_ERR_OOM_PAGES) return fail(c, RSD_ERR_OOM_PAGES, "KV page pool or pass list exhausted%s");

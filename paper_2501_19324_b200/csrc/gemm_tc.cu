@@ -1,8 +1,25 @@
-// GEMM dispatch.  (The tcgen05 path is added in this file.)
-#include "common.cuh"
-#include "kernels.cuh"
+// bf16 weight GEMM on the 5th-generation tensor cores (sm_100a): y[M, N] (+)= x[M, K] * W[N, K]^T.
+//
+// The weight matrix is the streamed operand, so it takes the 128-row side of the instruction:
+// each CTA owns a tile of 128 output features (rows of W) and MT rows of x, and computes
+// D^T[128, MT] = W_tile[128, K] * x_tile[MT, K]^T with tcgen05.mma (A = W tile, B = x tile, both
+// K-major in shared memory under the 128-byte swizzle, staged by TMA; accumulator in TMEM).  With
+// MT = 16..64 the same kernel is a bandwidth-bound skinny GEMM for decode (weights read once, MMA
+// cost hidden); with MT = 256 it is the dense GEMM of prefill / PRM scoring / catch-up.
+//
+// Roles inside a CTA of 6 warps: warps 0-3 read the accumulator out of TMEM (lane = output feature,
+// column = x row) and write y, warp 4 issues TMA loads through a ring of shared-memory stages,
+// warp 5 allocates TMEM and issues the MMAs.  Small problems are split along K across CTAs; the
+// partial tiles go to scratch and the last CTA to arrive adds them in split order (deterministic).
+// Every wait on an mbarrier is bounded; on expiry the CTA raises an error flag and leaves cleanly.
+#include <cuda.h>
 
 #include <atomic>
+#include <mutex>
+#include <unordered_map>
+
+#include "common.cuh"
+#include "kernels.cuh"
 
 namespace rsd {
 
@@ -13,16 +30,380 @@ cudaError_t launched(int n_kernels) {
 }
 uint64_t launches_total() { return g_launches.load(std::memory_order_relaxed); }
 
-bool gemm_tc_supported(int dtype, int M, int N, int K) { (void)dtype; (void)M; (void)N; (void)K; return false; }
-size_t gemm_scratch_bytes(int M) { (void)M; return 4096; }
+namespace {
 
-cudaError_t launch_gemm_tc(const void*, const void*, float*, int, int, int, int, void*, size_t, const int32_t*, cudaStream_t) {
-  return cudaErrorNotSupported;
+constexpr int kTileN = 128;        // W rows per CTA (UMMA M)
+constexpr int kTileK = 64;         // bf16 elements per 128-byte swizzled row
+constexpr int kUmmaK = 16;
+constexpr int kCounterBytes = 4096;
+constexpr int kMaxSplitTiles = kCounterBytes / 4;
+constexpr int kMaxSplitCtas = 640;
+constexpr uint32_t kWaitLimit = 1u << 22;
+
+// ---- PTX wrappers ---------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait: false when the limit is hit.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+  for (uint32_t i = 0; i < kWaitLimit; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  return false;
+}
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t* dst_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(ncols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
+}
+// Arrives on the mbarrier once every MMA issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void epilogue_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major tile under the 128-byte swizzle: rows of 128 bytes,
+// groups of 8 rows 1024 bytes apart (stride byte offset), leading byte offset unused (1), version 1.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
+  return (uint64_t)((saddr >> 4) & 0x3FFFu) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+
+template <int MT> struct TcCfg {
+  static constexpr int kStages = MT <= 64 ? 8 : (MT == 128 ? 6 : 4);
+  static constexpr int kABytes = kTileN * kTileK * 2;
+  static constexpr int kBBytes = MT * kTileK * 2;
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kTmemCols = MT < 32 ? 32 : MT;
+  static constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + 256;
+  // instruction descriptor: fp32 accumulate, bf16 A and B, both K-major, N = MT, M = 128
+  static constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(MT >> 3) << 17) | ((uint32_t)(kTileN >> 4) << 24);
+};
+
+template <int MT>
+__global__ void __launch_bounds__(192, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x, float* __restrict__ Y,
+               int M, int N, int K, int accumulate, int splits, int kb_per_split, float* __restrict__ partials,
+               int* __restrict__ counters, int* __restrict__ err, const int32_t* __restrict__ n_active) {
+  if (n_active != nullptr && *n_active == 0) return;
+  using Cfg = TcCfg<MT>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  uint64_t* full = (uint64_t*)(smem + (size_t)Cfg::kStages * Cfg::kStageBytes);
+  uint64_t* empty = full + Cfg::kStages;
+  uint64_t* tmem_full = empty + Cfg::kStages;
+  uint32_t* tmem_slot = (uint32_t*)(tmem_full + 1);
+  volatile uint32_t* flags = tmem_slot + 1;   // [0] abort, [1] last-arriver flag
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n0 = blockIdx.x * kTileN, m0 = blockIdx.y * MT, split = blockIdx.z;
+  const int total_kb = (K + kTileK - 1) / kTileK;
+  const int kb0 = split * kb_per_split;
+  const int kb1 = min(total_kb, kb0 + kb_per_split);
+  const int n_kb = kb1 - kb0;   // >= 1 by construction of the grid
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < Cfg::kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    mbar_init(tmem_full, 1);
+    flags[0] = 0; flags[1] = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 5) tmem_alloc(tmem_slot, Cfg::kTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 4) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      int issued = 0;
+      bool ok = true;
+      for (int i = 0; i < n_kb && ok; ++i) {
+        const int s = i % Cfg::kStages;
+        if (i >= Cfg::kStages) ok = mbar_wait(&empty[s], ((i / Cfg::kStages) - 1) & 1);
+        if (!ok || flags[0]) { ok = false; break; }
+        uint8_t* a = smem + (size_t)s * Cfg::kStageBytes;
+        mbar_expect_tx(&full[s], Cfg::kStageBytes);
+        tma_load_2d(a, &tm_w, &full[s], (kb0 + i) * kTileK, n0);
+        tma_load_2d(a + Cfg::kABytes, &tm_x, &full[s], (kb0 + i) * kTileK, m0);
+        issued = i + 1;
+      }
+      if (!ok) {
+        if (err) atomicCAS(err, 0, -5);
+        flags[0] = 1;
+        // let the copies already in flight land before the CTA goes away
+        for (int i = max(0, issued - Cfg::kStages); i < issued; ++i)
+          mbar_wait(&full[i % Cfg::kStages], (i / Cfg::kStages) & 1);
+      }
+    }
+  } else if (warp == 5) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      bool ok = true;
+      for (int i = 0; i < n_kb; ++i) {
+        const int s = i % Cfg::kStages;
+        ok = mbar_wait(&full[s], (i / Cfg::kStages) & 1);
+        if (!ok || flags[0]) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t a = smem_u32(smem + (size_t)s * Cfg::kStageBytes);
+        const uint32_t b = a + Cfg::kABytes;
+#pragma unroll
+        for (int k = 0; k < kTileK / kUmmaK; ++k) {
+          umma_bf16(tmem_base, smem_desc_sw128(a + k * kUmmaK * 2), smem_desc_sw128(b + k * kUmmaK * 2), Cfg::kIdesc,
+                    (i > 0 || k > 0) ? 1u : 0u);
+        }
+        umma_commit(&empty[s]);   // frees the stage once these MMAs have read it
+      }
+      if (ok) {
+        umma_commit(tmem_full);
+      } else {
+        if (err) atomicCAS(err, 0, -5);
+        flags[0] = 1;
+      }
+    }
+  } else {
+    // ---------------- epilogue: TMEM -> registers -> global ----------------
+    bool ok = mbar_wait(tmem_full, 0);
+    if (!ok && err) atomicCAS(err, 0, -5);
+    if (!ok) flags[0] = 1;
+    tc_fence_after();
+    const int n_local = warp * 32 + lane;
+    const int n = n0 + n_local;
+    const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16);
+    const int m_valid = min(MT, M - m0);
+    const int tile = blockIdx.y * gridDim.x + blockIdx.x;
+    const size_t tile_elems = (size_t)kTileN * MT;
+    if (ok) {
+      float* part = partials + ((size_t)split * gridDim.x * gridDim.y + tile) * tile_elems;
+      for (int c = 0; c < m_valid; c += 16) {
+        float v[16];
+        tmem_ld16(taddr + c, v);
+        if (splits == 1) {
+          if (n < N) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              if (c + j < m_valid) {
+                float* y = Y + (size_t)(m0 + c + j) * N + n;
+                *y = accumulate ? (*y + v[j]) : v[j];
+              }
+            }
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 16; ++j)
+            if (c + j < m_valid) part[(size_t)(c + j) * kTileN + n_local] = v[j];
+        }
+      }
+    }
+    if (splits > 1) {
+      __threadfence();
+      epilogue_barrier();
+      if (threadIdx.x == 0) {
+        const int old = atomicAdd(&counters[tile], 1);
+        flags[1] = (old == splits - 1) ? 1u : 0u;
+      }
+      epilogue_barrier();
+      if (flags[1]) {
+        __threadfence();
+        if (n < N && !flags[0]) {
+          for (int m = 0; m < m_valid; ++m) {
+            float sum = 0.f;
+            for (int sidx = 0; sidx < splits; ++sidx)
+              sum += __ldcg(partials + ((size_t)sidx * gridDim.x * gridDim.y + tile) * tile_elems + (size_t)m * kTileN + n_local);
+            float* y = Y + (size_t)(m0 + m) * N + n;
+            *y = accumulate ? (*y + sum) : sum;
+          }
+        }
+        if (threadIdx.x == 0) counters[tile] = 0;
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 5) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, Cfg::kTmemCols);
+  }
+}
+
+// ---- tensor maps (host) -----------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)p;
+  });
+  return fn;
+}
+
+struct MapKey {
+  const void* ptr; int rows, cols, box_rows;
+  bool operator==(const MapKey& o) const { return ptr == o.ptr && rows == o.rows && cols == o.cols && box_rows == o.box_rows; }
+};
+struct MapKeyHash {
+  size_t operator()(const MapKey& k) const {
+    size_t h = std::hash<const void*>()(k.ptr);
+    h ^= std::hash<long long>()(((long long)k.rows << 32) ^ ((long long)k.cols << 8) ^ k.box_rows) + 0x9e3779b97f4a7c15ull + (h << 6) + (h >> 2);
+    return h;
+  }
+};
+
+// Row-major bf16 matrix [rows, cols]; box = 64 columns x box_rows rows; 128-byte swizzle.  Maps are
+// cached by (pointer, shape): weights and activation buffers keep their addresses for a context's life.
+bool get_map(const void* ptr, int rows, int cols, int box_rows, CUtensorMap* out) {
+  static std::mutex mu;
+  static std::unordered_map<MapKey, CUtensorMap, MapKeyHash> cache;
+  std::lock_guard<std::mutex> lock(mu);
+  MapKey key{ptr, rows, cols, box_rows};
+  auto it = cache.find(key);
+  if (it != cache.end()) { *out = it->second; return true; }
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  CUtensorMap m;
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  cuuint32_t box[2] = {(cuuint32_t)kTileK, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return false;
+  if (cache.size() > 65536) cache.clear();
+  cache.emplace(key, m);
+  *out = m;
+  return true;
+}
+
+int pick_mt(int M) {
+  if (M <= 16) return 16;
+  if (M <= 32) return 32;
+  if (M <= 64) return 64;
+  if (M <= 128) return 128;
+  return 256;
+}
+
+struct TcPlan { int mt, n_tiles, m_tiles, splits, kb_per_split; };
+
+TcPlan plan_tc(int M, int N, int K) {
+  TcPlan p;
+  p.mt = pick_mt(M);
+  p.n_tiles = (N + kTileN - 1) / kTileN;
+  p.m_tiles = (M + p.mt - 1) / p.mt;
+  const int tiles = p.n_tiles * p.m_tiles;
+  const int total_kb = (K + kTileK - 1) / kTileK;
+  int splits = 1;
+  if (tiles < 148 && tiles <= kMaxSplitTiles && p.mt <= 64) {
+    splits = (2 * 148 + tiles - 1) / tiles;
+    splits = std::min(splits, std::max(1, total_kb / 2));
+    splits = std::min(splits, kMaxSplitCtas / tiles);
+    splits = std::max(splits, 1);
+  }
+  p.kb_per_split = (total_kb + splits - 1) / splits;
+  p.splits = (total_kb + p.kb_per_split - 1) / p.kb_per_split;   // no empty split
+  return p;
+}
+
+template <int MT>
+cudaError_t launch_mt(const CUtensorMap& tw, const CUtensorMap& tx, float* y, int M, int N, int K, int accumulate,
+                      const TcPlan& p, float* partials, int* counters, int* err, const int32_t* n_active, cudaStream_t s) {
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<MT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TcCfg<MT>::kSmemBytes);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  dim3 grid(p.n_tiles, p.m_tiles, p.splits);
+  gemm_tc_kernel<MT><<<grid, 192, TcCfg<MT>::kSmemBytes, s>>>(tw, tx, y, M, N, K, accumulate, p.splits, p.kb_per_split,
+                                                              partials, counters, err, n_active);
+  return launched(1);
+}
+
+}  // namespace
+
+bool gemm_tc_supported(int dtype, int M, int N, int K) {
+  return dtype == 1 && M >= 1 && N >= 1 && K >= 8 && K % 8 == 0;
+}
+
+// Layout of the scratch: [0, 4096) tile counters (kept zero between launches), then one int error
+// flag region of 256 bytes, then split-K partial tiles.
+size_t gemm_scratch_bytes(int M) {
+  const int mt = pick_mt(M);
+  const size_t part = mt <= 64 ? (size_t)kMaxSplitCtas * kTileN * mt * 4 : 0;
+  return kCounterBytes + 256 + part;
+}
+
+cudaError_t launch_gemm_tc(const void* W, const void* x, float* y, int M, int N, int K, int accumulate,
+                           void* scratch, size_t scratch_bytes, const int32_t* n_active, cudaStream_t s) {
+  if (M <= 0) return cudaSuccess;
+  if (!scratch || scratch_bytes < gemm_scratch_bytes(M)) return cudaErrorInvalidValue;
+  if (((uintptr_t)W & 15) || ((uintptr_t)x & 15)) return cudaErrorMisalignedAddress;
+  const TcPlan p = plan_tc(M, N, K);
+  CUtensorMap tw, tx;
+  if (!get_map(W, N, K, kTileN, &tw) || !get_map(x, M, K, p.mt, &tx)) return cudaErrorNotSupported;
+  int* counters = (int*)scratch;
+  int* err = (int*)((char*)scratch + kCounterBytes);
+  float* partials = (float*)((char*)scratch + kCounterBytes + 256);
+  switch (p.mt) {
+    case 16: return launch_mt<16>(tw, tx, y, M, N, K, accumulate, p, partials, counters, err, n_active, s);
+    case 32: return launch_mt<32>(tw, tx, y, M, N, K, accumulate, p, partials, counters, err, n_active, s);
+    case 64: return launch_mt<64>(tw, tx, y, M, N, K, accumulate, p, partials, counters, err, n_active, s);
+    case 128: return launch_mt<128>(tw, tx, y, M, N, K, accumulate, p, partials, counters, err, n_active, s);
+    default: return launch_mt<256>(tw, tx, y, M, N, K, accumulate, p, partials, counters, err, n_active, s);
+  }
 }
 
 cudaError_t launch_gemm(int dtype, const void* W, const void* x, float* y, int M, int N, int K, int accumulate,
                         int impl, void* scratch, size_t scratch_bytes, const int32_t* n_active, cudaStream_t s) {
-  if (impl == 2 || (impl == 0 && gemm_tc_supported(dtype, M, N, K)))
+  const bool tc_ok = gemm_tc_supported(dtype, M, N, K) && scratch && scratch_bytes >= gemm_scratch_bytes(M);
+  if (impl == 2 || (impl == 0 && tc_ok && M > 4))
     return launch_gemm_tc(W, x, y, M, N, K, accumulate, scratch, scratch_bytes, n_active, s);
   return launch_gemm_simt(dtype, W, x, y, M, N, K, accumulate, n_active, s);
 }

@@ -59,6 +59,28 @@ def test_gemm_simt(M, N, K, bf16):
     np.testing.assert_allclose(acc, want + y0, rtol=0, atol=2e-5 * np.sqrt(K))
 
 
+@pytest.mark.parametrize("M,N,K", [(16, 128, 64), (5, 256, 512), (17, 1536, 1536), (32, 2048, 1536), (33, 1000, 520),
+                                   (64, 1536, 8960), (100, 384, 1408), (128, 640, 768), (129, 256, 2048),
+                                   (300, 4096, 512), (1000, 1280, 768), (8, 17920, 1536)])
+def test_gemm_tcgen05(M, N, K):
+    """Tensor-core path: ragged M, N not a multiple of the 128-row tile, K not a multiple of 64,
+    split-K with the last-arriver reduction, several x tiles, accumulate into y."""
+    rng = np.random.default_rng(M * 7 + N)
+    W = ri.cpu_tensor(2, 5, N, K, True)
+    x = rng.normal(size=(M, K)).astype(np.float32)
+    xd = dev(x, torch.bfloat16)
+    want = oracle.matmul(W, xd.float().cpu().numpy())
+    Wd = dev(W, torch.bfloat16)
+    got = rb.k_gemm(Wd, xd, impl=2).cpu().numpy()
+    tol = 3e-5 * np.sqrt(K)
+    np.testing.assert_allclose(got, want, rtol=0, atol=tol)
+    y0 = rng.normal(size=(M, N)).astype(np.float32)
+    acc = rb.k_gemm(Wd, xd, y=dev(y0), accumulate=True, impl=2).cpu().numpy()
+    np.testing.assert_allclose(acc, want + y0, rtol=0, atol=tol)
+    again = rb.k_gemm(Wd, xd, impl=2).cpu().numpy()
+    assert np.array_equal(again, got)          # deterministic, whatever order the split CTAs finish in
+
+
 def test_rmsnorm_rope_swiglu():
     rng = np.random.default_rng(1)
     x = rng.normal(size=(5, 1536)).astype(np.float32) * 3
