@@ -234,6 +234,7 @@ def run_ours(args, rank: int, world: int):
         r = eng.step(delta)
         e2e_tokens += int(r["step_len"].sum())
     eng.gemm_timing(args.time_stride)
+    eng.phase_ms(True)
     barrier()
     launches1 = lib().rsd_debug_launch_count()
     t_start = torch.cuda.Event(enable_timing=True); t_end = torch.cuda.Event(enable_timing=True)
@@ -251,6 +252,7 @@ def run_ours(args, rank: int, world: int):
     launches2 = lib().rsd_debug_launch_count()
     clocks = sampler.stop()
     gt = eng.gemm_timing(0)
+    phases = {k: v / args.steps for k, v in eng.phase_ms(False).items()}
     e2e_tokens += timed_tokens
     ms = t_start.elapsed_time(t_end)
     e2e_ms = e2e_start.elapsed_time(e2e_end)
@@ -279,6 +281,7 @@ def run_ours(args, rank: int, world: int):
                             "peak": hbm, "unit": "GB/s", "frac": (achieved / hbm) if achieved else None,
                             "traffic": None, "peak_source": how, "timed_launches": gt["launches"],
                             "timing": f"CUDA events around every {args.time_stride}th GEMM launch of the timed steps"},
+               "phase_ms_per_step": phases,
                "flops_paper": counters["flops_paper"], "clocks": clocks,
                "gen_tokens": counters["gen_tokens"]}
         if world == 1 and not args.no_cpu_baseline:

@@ -172,6 +172,11 @@ int rsd_debug_get_state(rsd_ctx*, int32_t* z_len, int32_t* kv_len, int32_t* n_pa
  * the number of timed launches -- then clears the totals and installs the new stride.  HOST outputs,
  * any may be NULL.  Synchronises the device.                                                   */
 int rsd_debug_gemm_timing(rsd_ctx*, int32_t stride, double* ms, double* bytes, uint64_t* launches);
+/* Device time of the phases of rsd_step, from CUDA events on the caller's stream, summed over the
+ * steps since the previous call: out[7] (HOST, may be NULL) = draft sync, draft decode, PRM scoring,
+ * gate + routing, target catch-up, target decode, commit, in ms.  Each call returns and clears the
+ * sums, then switches the timing on (enable != 0) or off.                                       */
+int rsd_debug_phase_ms(rsd_ctx*, int32_t enable, double* out);
 /* Number of kernels this library has enqueued in this process so far.                          */
 uint64_t rsd_debug_launch_count(void);
 
@@ -187,9 +192,11 @@ int rsd_k_gemm(const void* W, const void* x, float* y, int32_t M, int32_t N, int
                int32_t accumulate, int32_t impl, void* scratch, size_t scratch_bytes, void* cuda_stream);
 size_t rsd_k_gemm_scratch_bytes(int32_t M, int32_t N, int32_t K);
 
-/* Paged-KV grouped-query decode attention: one query per row.  q [B, H, hd] fp32, kv pool laid out
- * [page][2 (K,V)][KV][page_tokens][hd] of `dtype`, page_table [B, max_pages], ctx_len [B] (number
- * of cached positions attended, >= 1), out [B, H, hd] fp32.                                   */
+/* Paged-KV grouped-query decode attention: one query per row.  q [B, H, hd] fp32; kv pool of pages,
+ * each page = keys [KV][16 tokens][hd] followed by values transposed [KV][hd][16 tokens], of
+ * `dtype`; page_table [B, max_pages]; ctx_len [B] (number of cached positions attended; rows with
+ * ctx_len < 1 are skipped); out [B, H, hd] fp32.  bf16 caches with H / KV <= 8 take the tensor-core
+ * split-context kernel, everything else a generic kernel.                                   */
 int rsd_k_attn_decode(const float* q, const void* kv_pool, const int32_t* page_table, const int32_t* ctx_len,
                       float* out, int32_t B, int32_t H, int32_t KV, int32_t hd, int32_t max_pages,
                       int32_t dtype, void* scratch, size_t scratch_bytes, void* cuda_stream);

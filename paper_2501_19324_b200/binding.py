@@ -51,7 +51,7 @@ class rsd_counters(ctypes.Structure):
 
 EXPORTS = ["rsd_query_sizes", "rsd_create", "rsd_load_models", "rsd_prefill", "rsd_step", "rsd_flops_counters",
            "rsd_reset", "rsd_destroy", "rsd_last_error", "rsd_debug_force", "rsd_debug_get_logits",
-           "rsd_debug_get_sampled", "rsd_debug_get_state", "rsd_debug_gemm_timing", "rsd_debug_launch_count", "rsd_k_gemm", "rsd_k_gemm_scratch_bytes",
+           "rsd_debug_get_sampled", "rsd_debug_get_state", "rsd_debug_gemm_timing", "rsd_debug_launch_count", "rsd_debug_phase_ms", "rsd_k_gemm", "rsd_k_gemm_scratch_bytes",
            "rsd_k_attn_decode", "rsd_k_attn_decode_scratch_bytes", "rsd_k_gate_compact", "rsd_k_gate_compact_static", "rsd_k_gate_compact_static_error", "rsd_k_rmsnorm",
            "rsd_k_rope", "rsd_k_swiglu", "rsd_k_sample", "rsd_k_philox"]
 
@@ -81,6 +81,7 @@ def lib():
         L.rsd_debug_get_sampled.argtypes = [vp, c_int32, vp]
         L.rsd_debug_get_state.argtypes = [vp] * 8
         L.rsd_debug_gemm_timing.argtypes = [vp, c_int32, vp, vp, vp]
+        L.rsd_debug_phase_ms.argtypes = [vp, c_int32, vp]
         L.rsd_debug_launch_count.argtypes = []
         L.rsd_debug_launch_count.restype = c_uint64
         L.rsd_k_gemm.argtypes = [vp, vp, vp, c_int32, c_int32, c_int32, c_int32, c_int32, c_int32, vp, c_size_t, vp]
@@ -214,6 +215,14 @@ class Engine:
         _check(lib().rsd_debug_gemm_timing(self.ctx, stride, ctypes.addressof(ms), ctypes.addressof(by),
                                            ctypes.addressof(n)), self.ctx)
         return dict(ms=ms.value, bytes=by.value, launches=n.value)
+
+    PHASES = ("draft_sync", "draft_decode", "prm_scoring", "gate_routing", "target_catchup", "target_decode", "commit")
+
+    def phase_ms(self, enable: bool) -> dict:
+        """Per-phase device time (ms) summed since the last call; switches the timing on or off."""
+        out = (c_double * 7)()
+        _check(lib().rsd_debug_phase_ms(self.ctx, int(enable), out), self.ctx)
+        return dict(zip(self.PHASES, list(out)))
 
     # -- parity hooks ---------------------------------------------------------------------------
     def force_tokens(self, which: int, steps: list):

@@ -64,8 +64,14 @@ struct rsd_ctx {
   size_t pinned_bytes = 0;
   void* gemm_scratch = nullptr;
   size_t gemm_scratch_bytes = 0;
+  void* attn_scratch = nullptr;
+  size_t attn_scratch_bytes = 0;
   rsd_counters ctr{};
   int last_n_rej = 0;
+  // per-phase timing of rsd_step (rsd_debug_phase_ms)
+  bool time_phases = false;
+  cudaEvent_t ph_ev[8] = {};
+  double ph_ms[7] = {};
   // sampled GEMM timing (rsd_debug_gemm_timing)
   int time_stride = 0;
   uint64_t gemm_calls = 0;
@@ -206,8 +212,12 @@ size_t layout_workspace(const rsd_config& cfg, const rsd_model* const ms[3], rsd
   float* o_rewards = TAKE(float, B);
   uint8_t* o_accept = TAKE(uint8_t, B);
   uint8_t* o_live = TAKE(uint8_t, B);
-  const size_t gs = gemm_scratch_bytes(T);
+  const size_t gs = gemm_scratch_bytes_any();
   void* gscr = TAKE(char, gs);
+  int h_max = 0;
+  for (int w = 0; w < 3; ++w) h_max = std::max(h_max, ms[w]->n_heads);
+  const size_t as = attn_decode_scratch_bytes(B, h_max, dm.hd, S);
+  void* ascr = TAKE(char, as);
 #undef TAKE
   if (c) {
     c->st = st; c->B_max = B; c->S = S; c->C = C; c->max_pages = max_pages; c->chunk = chunk; c->T_max = T;
@@ -218,6 +228,7 @@ size_t layout_workspace(const rsd_config& cfg, const rsd_model* const ms[3], rsd
     c->d_scalars = scal;
     c->o_tokens = o_tokens; c->o_len = o_len; c->o_rewards = o_rewards; c->o_accept = o_accept; c->o_live = o_live;
     c->gemm_scratch = gscr; c->gemm_scratch_bytes = gs;
+    c->attn_scratch = ascr; c->attn_scratch_bytes = as;
   }
   return L.bytes;
 }
@@ -296,7 +307,13 @@ int forward_pass(rsd_ctx* c, int which, PassView p, cudaStream_t s) {
     int rc = gemm(c, M, M.wqkv[l], c->h, c->qkv, T, (H + 2 * KV) * hd, d, 0, p.n_active, s);
     if (rc) return rc;
     CU(launch_rope_kv(m.dtype, c->qkv, p, c->q, kv, M.rope, H, KV, hd, s));
-    CU(launch_attn_generic(m.dtype, c->q, p, kv, c->attn, H, KV, hd, s));
+    if (p.n_active != nullptr) {
+      // decode pass: one query per row slot
+      CU(launch_attn_decode(m.dtype, c->q, kv.pool_layer, kv.page_table, kv.max_pages, p.tok_row, p.tok_pos, 1, c->attn,
+                            m.dtype, T, H, KV, hd, c->S, c->attn_scratch, c->attn_scratch_bytes, p.n_active, s));
+    } else {
+      CU(launch_attn_generic(m.dtype, c->q, p, kv, c->attn, m.dtype, H, KV, hd, s));
+    }
     rc = gemm(c, M, M.wo[l], c->attn, c->x, T, d, H * hd, 1, p.n_active, s);
     if (rc) return rc;
     CU(launch_rmsnorm(m.dtype, c->x, M.norm2[l], c->h, T, d, m.rms_eps, nullptr, p.n_active, s));
@@ -547,19 +564,24 @@ int rsd_step(rsd_ctx* c, float delta, void* cuda_stream, int32_t* step_tokens, i
   const int B = c->st.B;
   Scalars sc;
   int rc;
+#define PHASE(i) do { if (c->time_phases) CU(cudaEventRecord(c->ph_ev[i], s)); } while (0)
+  PHASE(0);
   // draft: catch up on a step the target wrote last time, then decode y^_i
   CU(launch_reserve_pages(c->st, RSD_DRAFT, kReserveStepDraft, s));
   CU(launch_build_pass(c->st, RSD_DRAFT, kPassIngestDraft, s));
   if ((rc = read_scalars(c, s, &sc))) return rc;
   const int n_sync = sc.n_tok;
   if ((rc = run_ingest(c, RSD_DRAFT, n_sync, false, s))) return rc;
+  PHASE(1);
   if ((rc = decode_phase(c, RSD_DRAFT, 0, B, s))) return rc;
+  PHASE(2);
   // PRM: score y^_i at its last token
   CU(launch_reserve_pages(c->st, RSD_PRM, kReserveScorePrm, s));
   CU(launch_build_pass(c->st, RSD_PRM, kPassScorePrm, s));
   if ((rc = read_scalars(c, s, &sc))) return rc;
   const int n_prm = sc.n_tok;
   if ((rc = run_ingest(c, RSD_PRM, n_prm, true, s))) return rc;
+  PHASE(3);
   // gate, compaction of rejected rows, target catch-up and decode
   CU(launch_gate(c->st, delta, c->lp, s));
   CU(launch_reserve_pages(c->st, RSD_TARGET, kReserveTarget, s));
@@ -567,8 +589,11 @@ int rsd_step(rsd_ctx* c, float delta, void* cuda_stream, int32_t* step_tokens, i
   if ((rc = read_scalars(c, s, &sc))) return rc;
   const int n_catch = sc.n_tok, n_rej = sc.n_rej;
   c->last_n_rej = n_rej;
+  PHASE(4);
   if ((rc = run_ingest(c, RSD_TARGET, n_catch, false, s))) return rc;
+  PHASE(5);
   if ((rc = decode_phase(c, RSD_TARGET, 1, n_rej, s))) return rc;
+  PHASE(6);
   // commit and read the results back
   CU(launch_commit(c->st, c->lp, c->o_tokens, c->o_len, c->o_rewards, c->o_accept, c->o_live, s));
   char* hp = c->pinned + 256;
@@ -587,7 +612,16 @@ int rsd_step(rsd_ctx* c, float delta, void* cuda_stream, int32_t* step_tokens, i
   CU(cudaMemcpyAsync(h_acc, c->o_accept, B, cudaMemcpyDeviceToHost, s));
   CU(cudaMemcpyAsync(h_live, c->o_live, B, cudaMemcpyDeviceToHost, s));
   if ((rc = clear_forcing(c, s))) return rc;
+  PHASE(7);
+#undef PHASE
   if ((rc = read_scalars(c, s, &sc))) return rc;
+  if (c->time_phases) {
+    for (int i = 0; i < 7; ++i) {
+      float ms = 0.f;
+      CU(cudaEventElapsedTime(&ms, c->ph_ev[i], c->ph_ev[i + 1]));
+      c->ph_ms[i] += ms;
+    }
+  }
   // counters (Section 3.3 accounting)
   uint64_t gen_d = 0, gen_t = 0, n_live = 0, n_acc = 0, discarded = 0;
   for (int b = 0; b < B; ++b) {
@@ -630,6 +664,7 @@ int rsd_destroy(rsd_ctx* c) {
   if (!c) return RSD_OK;
   cudaDeviceSynchronize();
   for (cudaEvent_t e : c->ev) cudaEventDestroy(e);
+  for (cudaEvent_t e : c->ph_ev) if (e) cudaEventDestroy(e);
   if (c->pinned) cudaFreeHost(c->pinned);
   delete c;
   return RSD_OK;
@@ -714,6 +749,16 @@ int rsd_debug_gemm_timing(rsd_ctx* c, int32_t stride, double* ms, double* bytes,
 
 uint64_t rsd_debug_launch_count(void) { return launches_total(); }
 
+int rsd_debug_phase_ms(rsd_ctx* c, int32_t enable, double* out) {
+  if (!c) return RSD_ERR_ARG;
+  if (out) memcpy(out, c->ph_ms, sizeof(c->ph_ms));
+  memset(c->ph_ms, 0, sizeof(c->ph_ms));
+  if (enable && !c->ph_ev[0])
+    for (auto& e : c->ph_ev) CU(cudaEventCreate(&e));
+  c->time_phases = enable != 0;
+  return RSD_OK;
+}
+
 // ---- single kernels -------------------------------------------------------------------------
 #define KCU(call)                                     \
   do {                                                \
@@ -751,8 +796,8 @@ int rsd_k_attn_decode(const float* q, const void* kv_pool, const int32_t* page_t
     return RSD_ERR_ARG;
   if (hd != 64 && hd != 128) return RSD_ERR_UNSUPPORTED;
   if (scratch_bytes < attn_decode_scratch_bytes(B, H, hd, max_pages * kPageTokens) || !scratch) return RSD_ERR_ARG;
-  KCU(launch_attn_decode(dtype, q, kv_pool, page_table, max_pages, nullptr, ctx_len, out, RSD_F32, B, H, KV, hd,
-                         max_pages * kPageTokens, scratch, nullptr, (cudaStream_t)cuda_stream));
+  KCU(launch_attn_decode(dtype, q, kv_pool, page_table, max_pages, nullptr, ctx_len, 0, out, RSD_F32, B, H, KV, hd,
+                         max_pages * kPageTokens, scratch, scratch_bytes, nullptr, (cudaStream_t)cuda_stream));
   return RSD_OK;
 }
 

@@ -1,0 +1,244 @@
+// Paged-KV grouped-query decode attention (one query token per row), sm_100a.
+//
+// A CTA of 4 warps serves one (row slot, KV head, context split): the G = H / KV query heads that
+// share the KV head are the rows of a 16-row MMA tile, so every key / value is read once from HBM for
+// the whole group.  Each warp walks its share of the 16-token pages:
+//   S  = Q K^T   with mma.sync m16n8k16 (bf16 in, fp32 out): keys stream from global memory straight
+//        into B fragments with 128-bit loads (the order of the head dims inside a 32-dim block is
+//        permuted identically for Q and K, which a dot product does not see);
+//   softmax statistics per head are kept on line (running max / sum), reduced over the 4 lanes that
+//        share a row with warp shuffles;
+//   O += P V     with the same MMA: values are stored transposed inside a page ([hd][16 tokens]), so a
+//        B fragment is one 64-bit load; the order of the tokens inside a page is permuted identically
+//        for P and V.
+// The warps' partial (max, sum, O) meet in shared memory; with several context splits the CTA writes
+// its partial to scratch and a second kernel merges the splits.
+#include "common.cuh"
+#include "kernels.cuh"
+
+namespace rsd {
+
+namespace {
+
+constexpr int kMaxSplits = 32;
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+__device__ __forceinline__ void mma_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// part_o: [slot][head][split][HD] un-normalised outputs; part_ml: [slot][head][split][2] (max, sum).
+template <int HD, typename OT>
+__global__ void __launch_bounds__(128)
+attn_decode_kernel(const float* __restrict__ q, const __nv_bfloat16* __restrict__ pool, const int32_t* __restrict__ page_table,
+                   int max_pages, const int32_t* __restrict__ slot_row, const int32_t* __restrict__ len_or_pos, int len_offset,
+                   OT* __restrict__ out, float* __restrict__ part_o, float* __restrict__ part_ml, int H, int KV, int n_splits,
+                   const int32_t* __restrict__ n_active) {
+  if (n_active != nullptr && *n_active == 0) return;
+  constexpr int KB = HD / 32;    // 32-dim blocks of the head dimension
+  constexpr int NT = HD / 8;     // 8-dim output tiles
+  __shared__ float s_m[4][8], s_l[4][8];
+  __shared__ float s_o[4][8][HD];
+  const int kvh = blockIdx.x, slot = blockIdx.y, split = blockIdx.z;
+  const int row = slot_row ? slot_row[slot] : slot;
+  if (row < 0) return;
+  const int ctx = len_or_pos[slot] + len_offset;
+  if (ctx <= 0) return;
+  const int G = H / KV, h0 = kvh * G;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, t = lane & 3;
+  const float scale = rsqrtf((float)HD);
+
+  const int n_pages = (ctx + kPageTokens - 1) / kPageTokens;
+  const int pps = (n_pages + n_splits - 1) / n_splits;
+  const int p_begin = split * pps, p_end = min(n_pages, p_begin + pps);
+
+  // Q fragments (rows 8..15 of the tile are padding): dims 32j + 8t + e of head h0 + g
+  uint32_t qa[KB][2][2];
+#pragma unroll
+  for (int j = 0; j < KB; ++j) {
+    float v[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) v[e] = g < G ? q[((size_t)slot * H + h0 + g) * HD + 32 * j + 8 * t + e] : 0.f;
+    qa[j][0][0] = pack_bf16(v[0], v[1]); qa[j][0][1] = pack_bf16(v[2], v[3]);
+    qa[j][1][0] = pack_bf16(v[4], v[5]); qa[j][1][1] = pack_bf16(v[6], v[7]);
+  }
+  float o[NT][4];
+#pragma unroll
+  for (int i = 0; i < NT; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
+  float m_run = -INFINITY, l_run = 0.f;
+
+  const int32_t* pt = page_table + (size_t)row * max_pages;
+  const size_t page_elems = (size_t)2 * KV * kPageTokens * HD;
+  // tokens whose keys this lane loads: tile 0 -> 4(g/2) + g%2, tile 1 -> that + 2
+  const int tok0 = 4 * (g >> 1) + (g & 1), tok1 = tok0 + 2;
+  for (int p = p_begin + warp; p < p_end; p += 4) {
+    const __nv_bfloat16* kb = pool + (size_t)pt[p] * page_elems + (size_t)kvh * kPageTokens * HD;
+    const __nv_bfloat16* vb = pool + (size_t)pt[p] * page_elems + (size_t)KV * kPageTokens * HD + (size_t)kvh * HD * kPageTokens;
+    float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int j = 0; j < KB; ++j) {
+      const uint4 k0 = *reinterpret_cast<const uint4*>(kb + tok0 * HD + 32 * j + 8 * t);
+      const uint4 k1 = *reinterpret_cast<const uint4*>(kb + tok1 * HD + 32 * j + 8 * t);
+      mma_16816(s0, qa[j][0][0], 0u, qa[j][0][1], 0u, k0.x, k0.y);
+      mma_16816(s0, qa[j][1][0], 0u, qa[j][1][1], 0u, k0.z, k0.w);
+      mma_16816(s1, qa[j][0][0], 0u, qa[j][0][1], 0u, k1.x, k1.y);
+      mma_16816(s1, qa[j][1][0], 0u, qa[j][1][1], 0u, k1.z, k1.w);
+    }
+    // this lane's scores of head g: tokens 4t, 4t+1 (tile 0) and 4t+2, 4t+3 (tile 1) of the page
+    const int n_valid = min(kPageTokens, ctx - p * kPageTokens);
+    float sc[4] = {s0[0] * scale, s0[1] * scale, s1[0] * scale, s1[1] * scale};
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+      if (4 * t + e >= n_valid) sc[e] = -INFINITY;
+    float mx = fmaxf(fmaxf(sc[0], sc[1]), fmaxf(sc[2], sc[3]));
+    mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 1));
+    mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 2));
+    const float m_new = fmaxf(m_run, mx);          // finite: token 0 of the page is always valid
+    const float corr = __expf(m_run - m_new);
+    float pr[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) pr[e] = __expf(sc[e] - m_new);
+    l_run = l_run * corr + (pr[0] + pr[1] + pr[2] + pr[3]);
+    m_run = m_new;
+    const uint32_t pa0 = pack_bf16(pr[0], pr[1]), pa2 = pack_bf16(pr[2], pr[3]);
+    // mask of the 16-bit halves of a value fragment that belong to cached tokens
+    uint32_t mlo = 0xFFFFFFFFu, mhi = 0xFFFFFFFFu;
+    if (n_valid < kPageTokens) {
+      mlo = (4 * t < n_valid ? 0x0000FFFFu : 0u) | (4 * t + 1 < n_valid ? 0xFFFF0000u : 0u);
+      mhi = (4 * t + 2 < n_valid ? 0x0000FFFFu : 0u) | (4 * t + 3 < n_valid ? 0xFFFF0000u : 0u);
+    }
+#pragma unroll
+    for (int i = 0; i < NT; ++i) {
+      const uint2 vv = *reinterpret_cast<const uint2*>(vb + (size_t)(8 * i + g) * kPageTokens + 4 * t);
+      o[i][0] *= corr; o[i][1] *= corr;
+      mma_16816(o[i], pa0, 0u, pa2, 0u, vv.x & mlo, vv.y & mhi);
+    }
+  }
+  // the 4 lanes of a row hold partial sums of l
+  l_run += __shfl_xor_sync(0xFFFFFFFFu, l_run, 1);
+  l_run += __shfl_xor_sync(0xFFFFFFFFu, l_run, 2);
+  if (t == 0) { s_m[warp][g] = m_run; s_l[warp][g] = l_run; }
+#pragma unroll
+  for (int i = 0; i < NT; ++i) {
+    s_o[warp][g][8 * i + 2 * t] = o[i][0];
+    s_o[warp][g][8 * i + 2 * t + 1] = o[i][1];
+  }
+  __syncthreads();
+  for (int idx = threadIdx.x; idx < G * HD; idx += blockDim.x) {
+    const int gg = idx / HD, dd = idx % HD;
+    float M = fmaxf(fmaxf(s_m[0][gg], s_m[1][gg]), fmaxf(s_m[2][gg], s_m[3][gg]));
+    float L = 0.f, O = 0.f;
+    if (M > -INFINITY) {
+#pragma unroll
+      for (int w = 0; w < 4; ++w) {
+        const float e = __expf(s_m[w][gg] - M);
+        L += s_l[w][gg] * e;
+        O += s_o[w][gg][dd] * e;
+      }
+    }
+    const int h = h0 + gg;
+    if (n_splits == 1) {
+      out[((size_t)slot * H + h) * HD + dd] = from_f32<OT>(O / L);
+    } else {
+      const size_t base = ((size_t)slot * H + h) * n_splits + split;
+      part_o[base * HD + dd] = O;
+      if (dd == 0) { part_ml[base * 2] = M; part_ml[base * 2 + 1] = L; }
+    }
+  }
+}
+
+template <int HD, typename OT>
+__global__ void __launch_bounds__(HD)
+attn_merge_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml, const int32_t* __restrict__ slot_row,
+                  const int32_t* __restrict__ len_or_pos, int len_offset, OT* __restrict__ out, int H, int n_splits,
+                  const int32_t* __restrict__ n_active) {
+  if (n_active != nullptr && *n_active == 0) return;
+  const int slot = blockIdx.y, h = blockIdx.x, dd = threadIdx.x;
+  if ((slot_row && slot_row[slot] < 0) || len_or_pos[slot] + len_offset <= 0) return;
+  const size_t base = ((size_t)slot * H + h) * n_splits;
+  float M = -INFINITY;
+  for (int s = 0; s < n_splits; ++s) M = fmaxf(M, part_ml[(base + s) * 2]);
+  float L = 0.f, O = 0.f;
+  for (int s = 0; s < n_splits; ++s) {
+    const float m = part_ml[(base + s) * 2];
+    if (m > -INFINITY) {
+      const float e = __expf(m - M);
+      L += part_ml[(base + s) * 2 + 1] * e;
+      O += part_o[(base + s) * HD + dd] * e;
+    }
+  }
+  out[((size_t)slot * H + h) * HD + dd] = from_f32<OT>(O / L);
+}
+
+__global__ void decode_slots_kernel(const int32_t* slot_row, const int32_t* len_or_pos, int len_offset, int32_t* row,
+                                    int32_t* pos, int B) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= B) return;
+  const int r = slot_row ? slot_row[i] : i;
+  const int ctx = len_or_pos[i] + len_offset;
+  row[i] = (r >= 0 && ctx >= 1) ? r : -1;
+  pos[i] = ctx - 1;
+}
+
+int pick_splits(int B, int KV, int max_ctx) {
+  const int ctas = B * KV;
+  int splits = (2 * 148 + ctas - 1) / ctas;
+  const int max_by_ctx = std::max(1, (max_ctx / kPageTokens) / 8);   // at least 8 pages per split
+  splits = std::min(splits, max_by_ctx);
+  return std::max(1, std::min(splits, kMaxSplits));
+}
+
+}  // namespace
+
+size_t attn_decode_scratch_bytes(int B, int H, int hd, int max_ctx) {
+  (void)max_ctx;
+  const size_t partials = (size_t)B * H * kMaxSplits * (hd + 2) * sizeof(float);
+  return sizeof(int32_t) * 2 * (size_t)B + 256 + partials;
+}
+
+cudaError_t launch_attn_decode(int dtype, const float* q, const void* pool_layer, const int32_t* page_table,
+                               int max_pages, const int32_t* slot_row, const int32_t* len_or_pos, int len_offset,
+                               void* out, int out_dtype, int B, int H, int KV, int hd, int max_ctx, void* scratch,
+                               size_t scratch_bytes, const int32_t* n_active, cudaStream_t s) {
+  if (B <= 0) return cudaSuccess;
+  if (!scratch || scratch_bytes < attn_decode_scratch_bytes(B, H, hd, max_ctx)) return cudaErrorInvalidValue;
+  const int G = H / KV;
+  int32_t* row = (int32_t*)scratch;
+  int32_t* pos = row + B;
+  if (dtype != 1 || G > 8) {
+    // fp32 caches and wide groups take the generic kernel
+    decode_slots_kernel<<<(B + 255) / 256, 256, 0, s>>>(slot_row, len_or_pos, len_offset, row, pos, B);
+    launched(1);
+    PassView p{nullptr, row, pos, B, n_active};
+    KvView kv{const_cast<void*>(pool_layer), page_table, max_pages};
+    return launch_attn_generic(dtype, q, p, kv, out, out_dtype, H, KV, hd, s);
+  }
+  const size_t head = ((sizeof(int32_t) * 2 * (size_t)B + 255) / 256) * 256;
+  float* part_ml = (float*)((char*)scratch + head);
+  float* part_o = part_ml + (size_t)B * H * kMaxSplits * 2;
+  const int splits = pick_splits(B, KV, max_ctx);
+  dim3 grid(KV, B, splits);
+  const __nv_bfloat16* pool = (const __nv_bfloat16*)pool_layer;
+#define RSD_DEC(HD, OT)                                                                                             \
+  do {                                                                                                              \
+    attn_decode_kernel<HD, OT><<<grid, 128, 0, s>>>(q, pool, page_table, max_pages, slot_row, len_or_pos, len_offset, \
+                                                    (OT*)out, part_o, part_ml, H, KV, splits, n_active);             \
+    if (splits > 1)                                                                                                 \
+      attn_merge_kernel<HD, OT><<<dim3(H, B), HD, 0, s>>>(part_o, part_ml, slot_row, len_or_pos, len_offset, (OT*)out, \
+                                                          H, splits, n_active);                                     \
+  } while (0)
+  if (hd == 128) { if (out_dtype == 1) RSD_DEC(128, __nv_bfloat16); else RSD_DEC(128, float); }
+  else { if (out_dtype == 1) RSD_DEC(64, __nv_bfloat16); else RSD_DEC(64, float); }
+#undef RSD_DEC
+  return launched(splits > 1 ? 2 : 1);
+}
+
+}  // namespace rsd

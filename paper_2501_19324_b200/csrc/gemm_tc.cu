@@ -380,6 +380,9 @@ size_t gemm_scratch_bytes(int M) {
   return kCounterBytes + 256 + part;
 }
 
+// Enough for any M (split-K is only used with tiles of at most 64 rows of x).
+size_t gemm_scratch_bytes_any() { return gemm_scratch_bytes(64); }
+
 cudaError_t launch_gemm_tc(const void* W, const void* x, float* y, int M, int N, int K, int accumulate,
                            void* scratch, size_t scratch_bytes, const int32_t* n_active, cudaStream_t s) {
   if (M <= 0) return cudaSuccess;

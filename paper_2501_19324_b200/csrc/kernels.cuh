@@ -27,7 +27,8 @@ struct PassView {
   const int32_t* n_active;
 };
 
-// Where one model keeps keys and values: per layer a slab [page][2][KV][16][hd].
+// Where one model keeps keys and values: per layer a slab of pages, each page holding the keys
+// [KV][16 tokens][hd] followed by the values transposed [KV][hd][16 tokens].
 struct KvView {
   void* pool_layer;            // slab of the current layer
   const int32_t* page_table;   // [rows, max_pages]
@@ -44,6 +45,7 @@ cudaError_t launch_gemm_simt(int dtype, const void* W, const void* x, float* y, 
 // partial tiles and tile counters (the counters must be zero on entry and are left zero).
 bool gemm_tc_supported(int dtype, int M, int N, int K);
 size_t gemm_scratch_bytes(int M);
+size_t gemm_scratch_bytes_any();
 cudaError_t launch_gemm_tc(const void* W, const void* x, float* y, int M, int N, int K, int accumulate,
                            void* scratch, size_t scratch_bytes, const int32_t* n_active, cudaStream_t s);
 // impl: 0 = by shape, 1 = SIMT split-K GEMV, 2 = tcgen05.
@@ -55,17 +57,19 @@ cudaError_t launch_rope_kv(int dtype, const float* qkv, PassView p, float* q_out
                            int H, int KV, int hd, cudaStream_t s);
 cudaError_t launch_rope_only(float* v, const int32_t* pos, int T, int n_heads, int hd, float theta, cudaStream_t s);
 // Causal attention of every slot over positions [0, tok_pos] of its row, read from the pages.
-cudaError_t launch_attn_generic(int dtype, const float* q, PassView p, KvView kv, void* out, int H, int KV,
-                                int hd, cudaStream_t s);
+cudaError_t launch_attn_generic(int dtype, const float* q, PassView p, KvView kv, void* out, int out_dtype, int H,
+                                int KV, int hd, cudaStream_t s);
 cudaError_t launch_swiglu(int dtype, const float* gu, void* out, int T, int F, const int32_t* n_active,
                           cudaStream_t s);
 
 // Decode attention (one query per row) with split-KV partial results merged in a second pass.
 size_t attn_decode_scratch_bytes(int B, int H, int hd, int max_ctx);
+// Slot i attends positions [0, len_or_pos[i] + len_offset) of row slot_row[i] (slot i itself when
+// slot_row is null); slot_row[i] < 0 skips the slot.
 cudaError_t launch_attn_decode(int dtype, const float* q, const void* pool_layer, const int32_t* page_table,
-                               int max_pages, const int32_t* slot_row, const int32_t* ctx_len, void* out,
-                               int out_dtype, int B, int H, int KV, int hd, int max_ctx, void* scratch,
-                               const int32_t* n_active, cudaStream_t s);
+                               int max_pages, const int32_t* slot_row, const int32_t* len_or_pos, int len_offset,
+                               void* out, int out_dtype, int B, int H, int KV, int hd, int max_ctx, void* scratch,
+                               size_t scratch_bytes, const int32_t* n_active, cudaStream_t s);
 
 struct SampleArgs {
   const float* logits;         // [n_slots, V]

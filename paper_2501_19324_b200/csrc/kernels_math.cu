@@ -190,7 +190,7 @@ __global__ void rope_kv_kernel(const float* __restrict__ qkv, PassView p, float*
   const float2* cs = rope + (size_t)pos * half;
   const int page = page_table[(size_t)row * max_pages + pos / kPageTokens];
   const int slot = pos % kPageTokens;
-  // [page][2][KV][16][hd]
+  // page = K block [KV][16][hd] followed by V block [KV][hd][16] (V transposed within the page)
   KT* kbase = pool + ((size_t)page * 2 + 0) * KV * kPageTokens * hd;
   KT* vbase = pool + ((size_t)page * 2 + 1) * KV * kPageTokens * hd;
   const int n_rot = (H + KV) * half;
@@ -211,7 +211,7 @@ __global__ void rope_kv_kernel(const float* __restrict__ qkv, PassView p, float*
   const float* vsrc = src + (H + KV) * hd;
   for (int idx = threadIdx.x; idx < KV * hd; idx += blockDim.x) {
     const int head = idx / hd, i = idx % hd;
-    vbase[((size_t)head * kPageTokens + slot) * hd + i] = from_f32<KT>(vsrc[idx]);
+    vbase[((size_t)head * hd + i) * kPageTokens + slot] = from_f32<KT>(vsrc[idx]);
   }
 }
 
@@ -303,7 +303,7 @@ attn_generic_kernel(const float* __restrict__ q, PassView p, const KT* __restric
         const float pj = __expf(sc[j] - mx);
         l += pj;
 #pragma unroll
-        for (int i = 0; i < DPL; ++i) acc[i] = fmaf(pj, to_f32(vb[j * HD + lane * DPL + i]), acc[i]);
+        for (int i = 0; i < DPL; ++i) acc[i] = fmaf(pj, to_f32(vb[(lane * DPL + i) * kPageTokens + j]), acc[i]);
       }
     }
     m = mx;
@@ -313,19 +313,18 @@ attn_generic_kernel(const float* __restrict__ q, PassView p, const KT* __restric
   for (int i = 0; i < DPL; ++i) out[((size_t)t * H + h) * HD + lane * DPL + i] = from_f32<OT>(acc[i] * inv);
 }
 
-cudaError_t launch_attn_generic(int dtype, const float* q, PassView p, KvView kv, void* out, int H, int KV,
-                                int hd, cudaStream_t s) {
+cudaError_t launch_attn_generic(int dtype, const float* q, PassView p, KvView kv, void* out, int out_dtype, int H,
+                                int KV, int hd, cudaStream_t s) {
   if (p.T <= 0) return cudaSuccess;
   const int warps = p.T * H;
   const int blocks = (warps + 3) / 4;
-  if (dtype == 1) {
-    using KT = __nv_bfloat16;
-    if (hd == 128) attn_generic_kernel<KT, KT, 128><<<blocks, 128, 0, s>>>(q, p, (const KT*)kv.pool_layer, kv.page_table, kv.max_pages, (KT*)out, H, KV);
-    else attn_generic_kernel<KT, KT, 64><<<blocks, 128, 0, s>>>(q, p, (const KT*)kv.pool_layer, kv.page_table, kv.max_pages, (KT*)out, H, KV);
-  } else {
-    if (hd == 128) attn_generic_kernel<float, float, 128><<<blocks, 128, 0, s>>>(q, p, (const float*)kv.pool_layer, kv.page_table, kv.max_pages, (float*)out, H, KV);
-    else attn_generic_kernel<float, float, 64><<<blocks, 128, 0, s>>>(q, p, (const float*)kv.pool_layer, kv.page_table, kv.max_pages, (float*)out, H, KV);
-  }
+#define RSD_ATTN(KT, OT, HD) \
+  attn_generic_kernel<KT, OT, HD><<<blocks, 128, 0, s>>>(q, p, (const KT*)kv.pool_layer, kv.page_table, kv.max_pages, (OT*)out, H, KV)
+  using bf = __nv_bfloat16;
+  if (dtype == 1 && out_dtype == 1) { if (hd == 128) RSD_ATTN(bf, bf, 128); else RSD_ATTN(bf, bf, 64); }
+  else if (dtype == 1) { if (hd == 128) RSD_ATTN(bf, float, 128); else RSD_ATTN(bf, float, 64); }
+  else { if (hd == 128) RSD_ATTN(float, float, 128); else RSD_ATTN(float, float, 64); }
+#undef RSD_ATTN
   return launched(1);
 }
 
@@ -468,47 +467,6 @@ cudaError_t launch_reward(int dtype, const float* x, const void* final_norm, con
   else
     reward_kernel<float><<<n_rows, 256, 0, s>>>(x, (const float*)final_norm, (const float*)w_r, head_kind, last_idx, t0, T, d, eps, reward);
   return launched(1);
-}
-
-}  // namespace rsd
-
-// ---------------------------------------------------------------------------------------------
-// Decode attention entry: one query per row over its cached positions.
-// ---------------------------------------------------------------------------------------------
-namespace rsd {
-
-__global__ void decode_slots_kernel(const int32_t* slot_row, const int32_t* ctx_len, int32_t* row, int32_t* pos, int B) {
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= B) return;
-  const int r = slot_row ? slot_row[i] : i;
-  row[i] = (r >= 0 && ctx_len[i] >= 1) ? r : -1;
-  pos[i] = ctx_len[i] - 1;
-}
-
-size_t attn_decode_scratch_bytes(int B, int H, int hd, int max_ctx) {
-  (void)H; (void)hd; (void)max_ctx;
-  return sizeof(int32_t) * 2 * (size_t)B + 256;
-}
-
-cudaError_t launch_attn_decode(int dtype, const float* q, const void* pool_layer, const int32_t* page_table,
-                               int max_pages, const int32_t* slot_row, const int32_t* ctx_len, void* out,
-                               int out_dtype, int B, int H, int KV, int hd, int max_ctx, void* scratch,
-                               const int32_t* n_active, cudaStream_t s) {
-  (void)max_ctx;
-  int32_t* row = (int32_t*)scratch;
-  int32_t* pos = row + B;
-  decode_slots_kernel<<<(B + 255) / 256, 256, 0, s>>>(slot_row, ctx_len, row, pos, B);
-  PassView p{nullptr, row, pos, B, n_active};
-  KvView kv{const_cast<void*>(pool_layer), page_table, max_pages};
-  const int warps = B * H, blocks = (warps + 3) / 4;
-#define RSD_ATTN(KT, OT, HD) \
-  attn_generic_kernel<KT, OT, HD><<<blocks, 128, 0, s>>>(q, p, (const KT*)kv.pool_layer, kv.page_table, kv.max_pages, (OT*)out, H, KV)
-  using bf = __nv_bfloat16;
-  if (dtype == 1 && out_dtype == 1) { if (hd == 128) RSD_ATTN(bf, bf, 128); else RSD_ATTN(bf, bf, 64); }
-  else if (dtype == 1) { if (hd == 128) RSD_ATTN(bf, float, 128); else RSD_ATTN(bf, float, 64); }
-  else { if (hd == 128) RSD_ATTN(float, float, 128); else RSD_ATTN(float, float, 64); }
-#undef RSD_ATTN
-  return launched(2);
 }
 
 }  // namespace rsd
