@@ -43,7 +43,7 @@ enum {
   RSD_ERR_UNSUPPORTED = -6  /* shape or option the kernels do not cover                   */
 };
 
-enum { RSD_F32 = 0, RSD_BF16 = 1 };
+enum { RSD_F32 = 0, RSD_BF16 = 1, RSD_F16 = 2 /* KV caches only */ };
 enum { RSD_DRAFT = 0, RSD_PRM = 1, RSD_TARGET = 2 };
 enum { RSD_HEAD_LM = 0, RSD_HEAD_REWARD_SIGMOID = 1, RSD_HEAD_REWARD_RAW = 2 };
 
@@ -182,21 +182,24 @@ uint64_t rsd_debug_launch_count(void);
 
 /* ---- single kernels (sweeps and unit parity); all pointers DEVICE unless noted ------------ */
 
-/* y[M, N] (fp32) = (accumulate ? y : 0) + x[M, K] * W[N, K]^T, W and x of element type `dtype`.
+/* y[M, N] (fp32) = (accumulate ? y : 0) + (x + x_lo)[M, K] * W[N, K]^T, W and x of element type `dtype`.
+ * x_lo (bf16 only, may be NULL) is the low half of a split-precision activation: x = bf16(a),
+ * x_lo = bf16(a - x), both multiplied on the tensor cores and added, so `a` enters with ~16 bits.
  * impl: 0 = pick by shape, 1 = split-K SIMT GEMV path, 2 = tcgen05/TMEM/TMA path (bf16 only,
  * K % 64 == 0, 16-byte aligned rows).  `scratch` (scratch_bytes from rsd_k_gemm_scratch_bytes)
  * holds split-K partial sums and tile counters; its first 4 KiB + 256 B must be zero before the
  * first call; the counters are left zero by every call and the int at byte 4096 becomes non-zero
  * if a bounded device-side wait of the tcgen05 path expired (RSD_ERR_TIMEOUT condition).                                                      */
-int rsd_k_gemm(const void* W, const void* x, float* y, int32_t M, int32_t N, int32_t K, int32_t dtype,
+int rsd_k_gemm(const void* W, const void* x, const void* x_lo, float* y, int32_t M, int32_t N, int32_t K, int32_t dtype,
                int32_t accumulate, int32_t impl, void* scratch, size_t scratch_bytes, void* cuda_stream);
 size_t rsd_k_gemm_scratch_bytes(int32_t M, int32_t N, int32_t K);
 
 /* Paged-KV grouped-query decode attention: one query per row.  q [B, H, hd] fp32; kv pool of pages,
  * each page = keys [KV][16 tokens][hd] followed by values transposed [KV][hd][16 tokens], of
- * `dtype`; page_table [B, max_pages]; ctx_len [B] (number of cached positions attended; rows with
- * ctx_len < 1 are skipped); out [B, H, hd] fp32.  bf16 caches with H / KV <= 8 take the tensor-core
- * split-context kernel, everything else a generic kernel.                                   */
+ * `dtype` (RSD_F32, RSD_BF16 or RSD_F16); page_table [B, max_pages]; ctx_len [B] (number of cached
+ * positions attended; rows with ctx_len < 1 are skipped); out [B, H, hd] fp32.  16-bit caches with
+ * H / KV <= 8 take the tensor-core split-context kernel, everything else a generic kernel.  The
+ * step loop keeps fp16 caches for bf16 models (same bytes, three more mantissa bits).                                   */
 int rsd_k_attn_decode(const float* q, const void* kv_pool, const int32_t* page_table, const int32_t* ctx_len,
                       float* out, int32_t B, int32_t H, int32_t KV, int32_t hd, int32_t max_pages,
                       int32_t dtype, void* scratch, size_t scratch_bytes, void* cuda_stream);

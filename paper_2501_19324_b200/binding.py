@@ -84,7 +84,7 @@ def lib():
         L.rsd_debug_phase_ms.argtypes = [vp, c_int32, vp]
         L.rsd_debug_launch_count.argtypes = []
         L.rsd_debug_launch_count.restype = c_uint64
-        L.rsd_k_gemm.argtypes = [vp, vp, vp, c_int32, c_int32, c_int32, c_int32, c_int32, c_int32, vp, c_size_t, vp]
+        L.rsd_k_gemm.argtypes = [vp, vp, vp, vp, c_int32, c_int32, c_int32, c_int32, c_int32, c_int32, vp, c_size_t, vp]
         L.rsd_k_gemm_scratch_bytes.argtypes = [c_int32, c_int32, c_int32]
         L.rsd_k_gemm_scratch_bytes.restype = c_size_t
         L.rsd_k_attn_decode.argtypes = [vp, vp, vp, vp, vp, c_int32, c_int32, c_int32, c_int32, c_int32, c_int32,
@@ -264,8 +264,8 @@ class Engine:
 
 # ---- single kernels ---------------------------------------------------------------------------
 
-def k_gemm(W, x, y=None, accumulate=False, impl=0):
-    """y[M, N] (fp32) (+)= x[M, K] @ W[N, K]^T on CUDA tensors."""
+def k_gemm(W, x, y=None, accumulate=False, impl=0, x_lo=None):
+    """y[M, N] (fp32) (+)= (x + x_lo)[M, K] @ W[N, K]^T on CUDA tensors."""
     import torch
     M, K = x.shape
     N = W.shape[0]
@@ -274,7 +274,7 @@ def k_gemm(W, x, y=None, accumulate=False, impl=0):
     nbytes = lib().rsd_k_gemm_scratch_bytes(M, N, K)
     scratch = torch.zeros(nbytes, dtype=torch.uint8, device=x.device)
     dt = RSD_BF16 if W.dtype == torch.bfloat16 else RSD_F32
-    _check(lib().rsd_k_gemm(_ptr(W), _ptr(x), _ptr(y), M, N, K, dt, int(accumulate), impl, _ptr(scratch), nbytes,
+    _check(lib().rsd_k_gemm(_ptr(W), _ptr(x), _ptr(x_lo) if x_lo is not None else None, _ptr(y), M, N, K, dt, int(accumulate), impl, _ptr(scratch), nbytes,
                             _stream()))
     if nbytes >= 4100 and int(scratch[4096:4100].view(torch.int32).item()) != 0:
         raise RsdError(-5, "a bounded wait inside the tensor-core GEMM expired")
@@ -288,7 +288,7 @@ def k_attn_decode(q, kv_pool, page_table, ctx_len, KV):
     out = torch.empty_like(q)
     nbytes = lib().rsd_k_attn_decode_scratch_bytes(B, H, hd, max_pages * 16)
     scratch = torch.zeros(nbytes, dtype=torch.uint8, device=q.device)
-    dt = RSD_BF16 if kv_pool.dtype == torch.bfloat16 else RSD_F32
+    dt = {torch.bfloat16: RSD_BF16, torch.float16: 2, torch.float32: RSD_F32}[kv_pool.dtype]
     _check(lib().rsd_k_attn_decode(_ptr(q), _ptr(kv_pool), _ptr(page_table), _ptr(ctx_len), _ptr(out), B, H, KV, hd,
                                    max_pages, dt, _ptr(scratch), nbytes, _stream()))
     return out

@@ -20,6 +20,8 @@ struct ModelHost {
   rsd_model m{};
   std::vector<const void*> wqkv, wo, wgu, wdown, norm1, norm2;
   size_t elem = 4;
+  int kv_dtype = 0;      // element type of this model's KV cache: 0 fp32, 2 fp16 (for bf16 weights)
+  bool split = false;    // bf16 GEMM inputs are kept as hi + lo pairs
   float2* rope = nullptr;
   char* kv_pool = nullptr;
   size_t layer_stride = 0;  // bytes of one layer's slab
@@ -53,6 +55,7 @@ struct rsd_ctx {
   // activations (workspace)
   float *x = nullptr, *qkv = nullptr, *q = nullptr, *gu = nullptr, *logits = nullptr;
   void *h = nullptr, *attn = nullptr, *act = nullptr;
+  void *h_lo = nullptr, *attn_lo = nullptr, *act_lo = nullptr;   // low halves (bf16 models)
   int32_t* sampled_slots = nullptr;
   float* dbg_logits[2] = {nullptr, nullptr};
   int32_t* d_scalars = nullptr;  // device block holding n_tok, n_rej, err, n_active, n_slots, next_page[3]
@@ -222,6 +225,10 @@ size_t layout_workspace(const rsd_config& cfg, const rsd_model* const ms[3], rsd
   if (c) {
     c->st = st; c->B_max = B; c->S = S; c->C = C; c->max_pages = max_pages; c->chunk = chunk; c->T_max = T;
     c->x = x; c->h = h; c->qkv = qkv; c->q = q; c->attn = attn; c->gu = gu; c->act = act; c->logits = logits;
+    // each operand buffer was sized at 4 bytes per element: a bf16 hi array followed by its lo array
+    c->h_lo = (char*)h + (size_t)T * dm.d * 2;
+    c->attn_lo = (char*)attn + (size_t)T * dm.hq * 2;
+    c->act_lo = (char*)act + (size_t)T * dm.f * 2;
     c->sampled_slots = sampled_slots;
     for (int w = 0; w < 3; ++w) c->mdl[w].rope = rope[w];
     c->dbg_logits[0] = dbg[0]; c->dbg_logits[1] = dbg[1];
@@ -278,12 +285,13 @@ int drain_gemm_events(rsd_ctx* c) {
   return RSD_OK;
 }
 
-int gemm(rsd_ctx* c, const ModelHost& M, const void* W, const void* xin, float* y, int Mrows, int N, int K,
-         int accumulate, const int32_t* n_active, cudaStream_t s) {
+int gemm(rsd_ctx* c, const ModelHost& M, const void* W, const void* xin, const void* xin_lo, float* y, int Mrows, int N,
+         int K, int accumulate, const int32_t* n_active, cudaStream_t s) {
   const bool timed = c->time_stride > 0 && (c->gemm_calls++ % (uint64_t)c->time_stride) == 0 &&
                      c->ev_used < c->ev_bytes.size();
   if (timed) CU(cudaEventRecord(c->ev[2 * c->ev_used], s));
-  CU(launch_gemm(M.m.dtype, W, xin, y, Mrows, N, K, accumulate, 0, c->gemm_scratch, c->gemm_scratch_bytes, n_active, s));
+  CU(launch_gemm(M.m.dtype, W, xin, M.split ? xin_lo : nullptr, y, Mrows, N, K, accumulate, 0, c->gemm_scratch,
+                 c->gemm_scratch_bytes, n_active, s));
   if (timed) {
     CU(cudaEventRecord(c->ev[2 * c->ev_used + 1], s));
     // algorithmic bytes: the weight matrix and the input once, the output once (twice when added to)
@@ -301,26 +309,30 @@ int forward_pass(rsd_ctx* c, int which, PassView p, cudaStream_t s) {
   const int T = p.T;
   if (T <= 0) return RSD_OK;
   CU(launch_embed(m.dtype, m.tok_embed, p, c->x, d, s));
+  void* h_lo = M.split ? c->h_lo : nullptr;
+  void* attn_lo = M.split ? c->attn_lo : nullptr;
+  void* act_lo = M.split ? c->act_lo : nullptr;
   for (int l = 0; l < m.n_layers; ++l) {
     KvView kv{M.kv_pool + (size_t)l * M.layer_stride, c->st.page_table[which], c->max_pages};
-    CU(launch_rmsnorm(m.dtype, c->x, M.norm1[l], c->h, T, d, m.rms_eps, nullptr, p.n_active, s));
-    int rc = gemm(c, M, M.wqkv[l], c->h, c->qkv, T, (H + 2 * KV) * hd, d, 0, p.n_active, s);
+    CU(launch_rmsnorm(m.dtype, c->x, M.norm1[l], c->h, h_lo, T, d, m.rms_eps, nullptr, p.n_active, s));
+    int rc = gemm(c, M, M.wqkv[l], c->h, h_lo, c->qkv, T, (H + 2 * KV) * hd, d, 0, p.n_active, s);
     if (rc) return rc;
-    CU(launch_rope_kv(m.dtype, c->qkv, p, c->q, kv, M.rope, H, KV, hd, s));
+    CU(launch_rope_kv(M.kv_dtype, c->qkv, p, c->q, kv, M.rope, H, KV, hd, s));
     if (p.n_active != nullptr) {
       // decode pass: one query per row slot
-      CU(launch_attn_decode(m.dtype, c->q, kv.pool_layer, kv.page_table, kv.max_pages, p.tok_row, p.tok_pos, 1, c->attn,
-                            m.dtype, T, H, KV, hd, c->S, c->attn_scratch, c->attn_scratch_bytes, p.n_active, s));
+      CU(launch_attn_decode(M.kv_dtype, c->q, kv.pool_layer, kv.page_table, kv.max_pages, p.tok_row, p.tok_pos, 1,
+                            c->attn, attn_lo, m.dtype, T, H, KV, hd, c->S, c->attn_scratch, c->attn_scratch_bytes,
+                            p.n_active, s));
     } else {
-      CU(launch_attn_generic(m.dtype, c->q, p, kv, c->attn, m.dtype, H, KV, hd, s));
+      CU(launch_attn_generic(M.kv_dtype, c->q, p, kv, c->attn, attn_lo, m.dtype, H, KV, hd, s));
     }
-    rc = gemm(c, M, M.wo[l], c->attn, c->x, T, d, H * hd, 1, p.n_active, s);
+    rc = gemm(c, M, M.wo[l], c->attn, attn_lo, c->x, T, d, H * hd, 1, p.n_active, s);
     if (rc) return rc;
-    CU(launch_rmsnorm(m.dtype, c->x, M.norm2[l], c->h, T, d, m.rms_eps, nullptr, p.n_active, s));
-    rc = gemm(c, M, M.wgu[l], c->h, c->gu, T, 2 * F, d, 0, p.n_active, s);
+    CU(launch_rmsnorm(m.dtype, c->x, M.norm2[l], c->h, h_lo, T, d, m.rms_eps, nullptr, p.n_active, s));
+    rc = gemm(c, M, M.wgu[l], c->h, h_lo, c->gu, T, 2 * F, d, 0, p.n_active, s);
     if (rc) return rc;
-    CU(launch_swiglu(m.dtype, c->gu, c->act, T, F, p.n_active, s));
-    rc = gemm(c, M, M.wdown[l], c->act, c->x, T, d, F, 1, p.n_active, s);
+    CU(launch_swiglu(m.dtype, c->gu, c->act, act_lo, T, F, p.n_active, s));
+    rc = gemm(c, M, M.wdown[l], c->act, act_lo, c->x, T, d, F, 1, p.n_active, s);
     if (rc) return rc;
   }
   return RSD_OK;
@@ -363,8 +375,9 @@ int decode_phase(rsd_ctx* c, int which, int phase, int n_slots, cudaStream_t s) 
     PassView p{c->st.pass_tok_id, c->st.pass_tok_row, c->st.pass_tok_pos, n_slots, c->st.n_active};
     int rc = forward_pass(c, which, p, s);
     if (rc) return rc;
-    CU(launch_rmsnorm(m.dtype, c->x, m.final_norm, c->h, n_slots, m.d_model, m.rms_eps, nullptr, p.n_active, s));
-    rc = gemm(c, M, m.head, c->h, c->logits, n_slots, m.vocab, m.d_model, 0, p.n_active, s);
+    CU(launch_rmsnorm(m.dtype, c->x, m.final_norm, c->h, M.split ? c->h_lo : nullptr, n_slots, m.d_model, m.rms_eps,
+                      nullptr, p.n_active, s));
+    rc = gemm(c, M, m.head, c->h, c->h_lo, c->logits, n_slots, m.vocab, m.d_model, 0, p.n_active, s);
     if (rc) return rc;
     if (c->dbg_logits[phase]) {
       scatter_logits_kernel<<<n_slots, 256, 0, s>>>(c->logits, c->st.pass_tok_row, c->dbg_logits[phase], m.vocab, c->C, j, c->st.n_active);
@@ -477,6 +490,8 @@ int rsd_load_models(rsd_ctx* c, const rsd_model* draft, const rsd_model* prm, co
     M.m.wqkv = M.wqkv.data(); M.m.wo = M.wo.data(); M.m.wgu = M.wgu.data(); M.m.wdown = M.wdown.data();
     M.m.norm1 = M.norm1.data(); M.m.norm2 = M.norm2.data();
     M.elem = M.m.dtype == RSD_BF16 ? 2 : 4;
+    M.kv_dtype = M.m.dtype == RSD_BF16 ? 2 : 0;
+    M.split = M.m.dtype == RSD_BF16;
     M.n_params = count_params(M.m);
     M.kv_pool = (char*)c->cfg.kv_pool[w];
     const size_t page_bytes = (size_t)2 * M.m.n_kv_heads * kPageTokens * M.m.head_dim * M.elem;
@@ -774,14 +789,15 @@ size_t rsd_k_gemm_scratch_bytes(int32_t M, int32_t N, int32_t K) {
   return gemm_scratch_bytes(M);
 }
 
-int rsd_k_gemm(const void* W, const void* x, float* y, int32_t M, int32_t N, int32_t K, int32_t dtype,
+int rsd_k_gemm(const void* W, const void* x, const void* x_lo, float* y, int32_t M, int32_t N, int32_t K, int32_t dtype,
                int32_t accumulate, int32_t impl, void* scratch, size_t scratch_bytes, void* cuda_stream) {
   if (!W || !x || !y || M < 0 || N < 1 || K < 1 || (dtype != RSD_F32 && dtype != RSD_BF16) || impl < 0 || impl > 2)
     return RSD_ERR_ARG;
   if (K % (dtype == RSD_BF16 ? 8 : 4)) return RSD_ERR_UNSUPPORTED;
   if (impl == 2 && !gemm_tc_supported(dtype, M, N, K)) return RSD_ERR_UNSUPPORTED;
   if (impl != 1 && (!scratch || scratch_bytes < gemm_scratch_bytes(M))) return RSD_ERR_ARG;
-  KCU(launch_gemm(dtype, W, x, y, M, N, K, accumulate, impl, scratch, scratch_bytes, nullptr, (cudaStream_t)cuda_stream));
+  if (x_lo && dtype != RSD_BF16) return RSD_ERR_ARG;
+  KCU(launch_gemm(dtype, W, x, x_lo, y, M, N, K, accumulate, impl, scratch, scratch_bytes, nullptr, (cudaStream_t)cuda_stream));
   return RSD_OK;
 }
 
@@ -796,7 +812,8 @@ int rsd_k_attn_decode(const float* q, const void* kv_pool, const int32_t* page_t
     return RSD_ERR_ARG;
   if (hd != 64 && hd != 128) return RSD_ERR_UNSUPPORTED;
   if (scratch_bytes < attn_decode_scratch_bytes(B, H, hd, max_pages * kPageTokens) || !scratch) return RSD_ERR_ARG;
-  KCU(launch_attn_decode(dtype, q, kv_pool, page_table, max_pages, nullptr, ctx_len, 0, out, RSD_F32, B, H, KV, hd,
+  if (dtype < 0 || dtype > 2) return RSD_ERR_ARG;
+  KCU(launch_attn_decode(dtype, q, kv_pool, page_table, max_pages, nullptr, ctx_len, 0, out, nullptr, RSD_F32, B, H, KV, hd,
                          max_pages * kPageTokens, scratch, scratch_bytes, nullptr, (cudaStream_t)cuda_stream));
   return RSD_OK;
 }
@@ -812,7 +829,7 @@ int rsd_k_gate_compact(const float* rewards, const uint8_t* live, float delta, u
 int rsd_k_rmsnorm(const float* x, const void* gain, void* out, int32_t T, int32_t d, float eps, int32_t dtype,
                   void* cuda_stream) {
   if (!x || !gain || !out || T < 0 || d < 4 || d % 4) return RSD_ERR_ARG;
-  KCU(launch_rmsnorm(dtype, x, gain, out, T, d, eps, nullptr, nullptr, (cudaStream_t)cuda_stream));
+  KCU(launch_rmsnorm(dtype, x, gain, out, nullptr, T, d, eps, nullptr, nullptr, (cudaStream_t)cuda_stream));
   return RSD_OK;
 }
 
@@ -824,7 +841,7 @@ int rsd_k_rope(float* v, const int32_t* pos, int32_t T, int32_t n_heads, int32_t
 
 int rsd_k_swiglu(const float* gu, void* out, int32_t T, int32_t F, int32_t dtype, void* cuda_stream) {
   if (!gu || !out || T < 0 || F < 1) return RSD_ERR_ARG;
-  KCU(launch_swiglu(dtype, gu, out, T, F, nullptr, (cudaStream_t)cuda_stream));
+  KCU(launch_swiglu(dtype, gu, out, nullptr, T, F, nullptr, (cudaStream_t)cuda_stream));
   return RSD_OK;
 }
 

@@ -22,24 +22,40 @@ namespace {
 
 constexpr int kMaxSplits = 32;
 
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+// Two fp32 values rounded to the cache's 16-bit type and packed into one MMA operand register.
+template <typename KT> __device__ __forceinline__ uint32_t pack2(float lo, float hi);
+template <> __device__ __forceinline__ uint32_t pack2<__nv_bfloat16>(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
 }
+template <> __device__ __forceinline__ uint32_t pack2<__half>(float lo, float hi) {
+  __half2 v = __floats2half2_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
 
-__device__ __forceinline__ void mma_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+template <typename KT>
+__device__ __forceinline__ void mma_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1);
+template <>
+__device__ __forceinline__ void mma_16816<__nv_bfloat16>(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
   asm volatile(
       "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
+template <>
+__device__ __forceinline__ void mma_16816<__half>(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
 
 // part_o: [slot][head][split][HD] un-normalised outputs; part_ml: [slot][head][split][2] (max, sum).
-template <int HD, typename OT>
+template <int HD, typename KT, typename OT>
 __global__ void __launch_bounds__(128)
-attn_decode_kernel(const float* __restrict__ q, const __nv_bfloat16* __restrict__ pool, const int32_t* __restrict__ page_table,
+attn_decode_kernel(const float* __restrict__ q, const KT* __restrict__ pool, const int32_t* __restrict__ page_table,
                    int max_pages, const int32_t* __restrict__ slot_row, const int32_t* __restrict__ len_or_pos, int len_offset,
-                   OT* __restrict__ out, float* __restrict__ part_o, float* __restrict__ part_ml, int H, int KV, int n_splits,
+                   OT* __restrict__ out, OT* __restrict__ out_lo, float* __restrict__ part_o, float* __restrict__ part_ml, int H, int KV, int n_splits,
                    const int32_t* __restrict__ n_active) {
   if (n_active != nullptr && *n_active == 0) return;
   constexpr int KB = HD / 32;    // 32-dim blocks of the head dimension
@@ -67,8 +83,8 @@ attn_decode_kernel(const float* __restrict__ q, const __nv_bfloat16* __restrict_
     float v[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) v[e] = g < G ? q[((size_t)slot * H + h0 + g) * HD + 32 * j + 8 * t + e] : 0.f;
-    qa[j][0][0] = pack_bf16(v[0], v[1]); qa[j][0][1] = pack_bf16(v[2], v[3]);
-    qa[j][1][0] = pack_bf16(v[4], v[5]); qa[j][1][1] = pack_bf16(v[6], v[7]);
+    qa[j][0][0] = pack2<KT>(v[0], v[1]); qa[j][0][1] = pack2<KT>(v[2], v[3]);
+    qa[j][1][0] = pack2<KT>(v[4], v[5]); qa[j][1][1] = pack2<KT>(v[6], v[7]);
   }
   float o[NT][4];
 #pragma unroll
@@ -80,17 +96,17 @@ attn_decode_kernel(const float* __restrict__ q, const __nv_bfloat16* __restrict_
   // tokens whose keys this lane loads: tile 0 -> 4(g/2) + g%2, tile 1 -> that + 2
   const int tok0 = 4 * (g >> 1) + (g & 1), tok1 = tok0 + 2;
   for (int p = p_begin + warp; p < p_end; p += 4) {
-    const __nv_bfloat16* kb = pool + (size_t)pt[p] * page_elems + (size_t)kvh * kPageTokens * HD;
-    const __nv_bfloat16* vb = pool + (size_t)pt[p] * page_elems + (size_t)KV * kPageTokens * HD + (size_t)kvh * HD * kPageTokens;
+    const KT* kb = pool + (size_t)pt[p] * page_elems + (size_t)kvh * kPageTokens * HD;
+    const KT* vb = pool + (size_t)pt[p] * page_elems + (size_t)KV * kPageTokens * HD + (size_t)kvh * HD * kPageTokens;
     float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
     for (int j = 0; j < KB; ++j) {
       const uint4 k0 = *reinterpret_cast<const uint4*>(kb + tok0 * HD + 32 * j + 8 * t);
       const uint4 k1 = *reinterpret_cast<const uint4*>(kb + tok1 * HD + 32 * j + 8 * t);
-      mma_16816(s0, qa[j][0][0], 0u, qa[j][0][1], 0u, k0.x, k0.y);
-      mma_16816(s0, qa[j][1][0], 0u, qa[j][1][1], 0u, k0.z, k0.w);
-      mma_16816(s1, qa[j][0][0], 0u, qa[j][0][1], 0u, k1.x, k1.y);
-      mma_16816(s1, qa[j][1][0], 0u, qa[j][1][1], 0u, k1.z, k1.w);
+      mma_16816<KT>(s0, qa[j][0][0], 0u, qa[j][0][1], 0u, k0.x, k0.y);
+      mma_16816<KT>(s0, qa[j][1][0], 0u, qa[j][1][1], 0u, k0.z, k0.w);
+      mma_16816<KT>(s1, qa[j][0][0], 0u, qa[j][0][1], 0u, k1.x, k1.y);
+      mma_16816<KT>(s1, qa[j][1][0], 0u, qa[j][1][1], 0u, k1.z, k1.w);
     }
     // this lane's scores of head g: tokens 4t, 4t+1 (tile 0) and 4t+2, 4t+3 (tile 1) of the page
     const int n_valid = min(kPageTokens, ctx - p * kPageTokens);
@@ -108,7 +124,7 @@ attn_decode_kernel(const float* __restrict__ q, const __nv_bfloat16* __restrict_
     for (int e = 0; e < 4; ++e) pr[e] = __expf(sc[e] - m_new);
     l_run = l_run * corr + (pr[0] + pr[1] + pr[2] + pr[3]);
     m_run = m_new;
-    const uint32_t pa0 = pack_bf16(pr[0], pr[1]), pa2 = pack_bf16(pr[2], pr[3]);
+    const uint32_t pa0 = pack2<KT>(pr[0], pr[1]), pa2 = pack2<KT>(pr[2], pr[3]);
     // mask of the 16-bit halves of a value fragment that belong to cached tokens
     uint32_t mlo = 0xFFFFFFFFu, mhi = 0xFFFFFFFFu;
     if (n_valid < kPageTokens) {
@@ -119,7 +135,7 @@ attn_decode_kernel(const float* __restrict__ q, const __nv_bfloat16* __restrict_
     for (int i = 0; i < NT; ++i) {
       const uint2 vv = *reinterpret_cast<const uint2*>(vb + (size_t)(8 * i + g) * kPageTokens + 4 * t);
       o[i][0] *= corr; o[i][1] *= corr;
-      mma_16816(o[i], pa0, 0u, pa2, 0u, vv.x & mlo, vv.y & mhi);
+      mma_16816<KT>(o[i], pa0, 0u, pa2, 0u, vv.x & mlo, vv.y & mhi);
     }
   }
   // the 4 lanes of a row hold partial sums of l
@@ -146,7 +162,7 @@ attn_decode_kernel(const float* __restrict__ q, const __nv_bfloat16* __restrict_
     }
     const int h = h0 + gg;
     if (n_splits == 1) {
-      out[((size_t)slot * H + h) * HD + dd] = from_f32<OT>(O / L);
+      store_operand<OT>(out, out_lo, ((size_t)slot * H + h) * HD + dd, O / L);
     } else {
       const size_t base = ((size_t)slot * H + h) * n_splits + split;
       part_o[base * HD + dd] = O;
@@ -158,8 +174,8 @@ attn_decode_kernel(const float* __restrict__ q, const __nv_bfloat16* __restrict_
 template <int HD, typename OT>
 __global__ void __launch_bounds__(HD)
 attn_merge_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml, const int32_t* __restrict__ slot_row,
-                  const int32_t* __restrict__ len_or_pos, int len_offset, OT* __restrict__ out, int H, int n_splits,
-                  const int32_t* __restrict__ n_active) {
+                  const int32_t* __restrict__ len_or_pos, int len_offset, OT* __restrict__ out, OT* __restrict__ out_lo,
+                  int H, int n_splits, const int32_t* __restrict__ n_active) {
   if (n_active != nullptr && *n_active == 0) return;
   const int slot = blockIdx.y, h = blockIdx.x, dd = threadIdx.x;
   if ((slot_row && slot_row[slot] < 0) || len_or_pos[slot] + len_offset <= 0) return;
@@ -175,7 +191,7 @@ attn_merge_kernel(const float* __restrict__ part_o, const float* __restrict__ pa
       O += part_o[(base + s) * HD + dd] * e;
     }
   }
-  out[((size_t)slot * H + h) * HD + dd] = from_f32<OT>(O / L);
+  store_operand<OT>(out, out_lo, ((size_t)slot * H + h) * HD + dd, O / L);
 }
 
 __global__ void decode_slots_kernel(const int32_t* slot_row, const int32_t* len_or_pos, int len_offset, int32_t* row,
@@ -204,39 +220,41 @@ size_t attn_decode_scratch_bytes(int B, int H, int hd, int max_ctx) {
   return sizeof(int32_t) * 2 * (size_t)B + 256 + partials;
 }
 
-cudaError_t launch_attn_decode(int dtype, const float* q, const void* pool_layer, const int32_t* page_table,
+cudaError_t launch_attn_decode(int kv_dtype, const float* q, const void* pool_layer, const int32_t* page_table,
                                int max_pages, const int32_t* slot_row, const int32_t* len_or_pos, int len_offset,
-                               void* out, int out_dtype, int B, int H, int KV, int hd, int max_ctx, void* scratch,
-                               size_t scratch_bytes, const int32_t* n_active, cudaStream_t s) {
+                               void* out, void* out_lo, int out_dtype, int B, int H, int KV, int hd, int max_ctx,
+                               void* scratch, size_t scratch_bytes, const int32_t* n_active, cudaStream_t s) {
   if (B <= 0) return cudaSuccess;
   if (!scratch || scratch_bytes < attn_decode_scratch_bytes(B, H, hd, max_ctx)) return cudaErrorInvalidValue;
   const int G = H / KV;
   int32_t* row = (int32_t*)scratch;
   int32_t* pos = row + B;
-  if (dtype != 1 || G > 8) {
+  if (kv_dtype == 0 || G > 8) {
     // fp32 caches and wide groups take the generic kernel
     decode_slots_kernel<<<(B + 255) / 256, 256, 0, s>>>(slot_row, len_or_pos, len_offset, row, pos, B);
     launched(1);
     PassView p{nullptr, row, pos, B, n_active};
     KvView kv{const_cast<void*>(pool_layer), page_table, max_pages};
-    return launch_attn_generic(dtype, q, p, kv, out, out_dtype, H, KV, hd, s);
+    return launch_attn_generic(kv_dtype, q, p, kv, out, out_lo, out_dtype, H, KV, hd, s);
   }
   const size_t head = ((sizeof(int32_t) * 2 * (size_t)B + 255) / 256) * 256;
   float* part_ml = (float*)((char*)scratch + head);
   float* part_o = part_ml + (size_t)B * H * kMaxSplits * 2;
   const int splits = pick_splits(B, KV, max_ctx);
   dim3 grid(KV, B, splits);
-  const __nv_bfloat16* pool = (const __nv_bfloat16*)pool_layer;
-#define RSD_DEC(HD, OT)                                                                                             \
-  do {                                                                                                              \
-    attn_decode_kernel<HD, OT><<<grid, 128, 0, s>>>(q, pool, page_table, max_pages, slot_row, len_or_pos, len_offset, \
-                                                    (OT*)out, part_o, part_ml, H, KV, splits, n_active);             \
-    if (splits > 1)                                                                                                 \
+#define RSD_DEC(HD, KT, OT)                                                                                          \
+  do {                                                                                                               \
+    attn_decode_kernel<HD, KT, OT><<<grid, 128, 0, s>>>(q, (const KT*)pool_layer, page_table, max_pages, slot_row,     \
+                                                        len_or_pos, len_offset, (OT*)out, (OT*)out_lo, part_o, part_ml, \
+                                                        H, KV, splits, n_active);                                    \
+    if (splits > 1)                                                                                                  \
       attn_merge_kernel<HD, OT><<<dim3(H, B), HD, 0, s>>>(part_o, part_ml, slot_row, len_or_pos, len_offset, (OT*)out, \
-                                                          H, splits, n_active);                                     \
+                                                          (OT*)out_lo, H, splits, n_active);                         \
   } while (0)
-  if (hd == 128) { if (out_dtype == 1) RSD_DEC(128, __nv_bfloat16); else RSD_DEC(128, float); }
-  else { if (out_dtype == 1) RSD_DEC(64, __nv_bfloat16); else RSD_DEC(64, float); }
+#define RSD_DEC_O(HD, KT) do { if (out_dtype == 1) RSD_DEC(HD, KT, __nv_bfloat16); else RSD_DEC(HD, KT, float); } while (0)
+  if (kv_dtype == 2) { if (hd == 128) RSD_DEC_O(128, __half); else RSD_DEC_O(64, __half); }
+  else { if (hd == 128) RSD_DEC_O(128, __nv_bfloat16); else RSD_DEC_O(64, __nv_bfloat16); }
+#undef RSD_DEC_O
 #undef RSD_DEC
   return launched(splits > 1 ? 2 : 1);
 }

@@ -2,6 +2,7 @@
 #pragma once
 
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -10,9 +11,23 @@ namespace rsd {
 // ---- element conversion ---------------------------------------------------------------------
 __device__ __forceinline__ float to_f32(float v) { return v; }
 __device__ __forceinline__ float to_f32(__nv_bfloat16 v) { return __bfloat162float(v); }
+__device__ __forceinline__ float to_f32(__half v) { return __half2float(v); }
 template <typename T> __device__ __forceinline__ T from_f32(float v);
 template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
 template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+template <> __device__ __forceinline__ __half from_f32<__half>(float v) { return __float2half_rn(v); }
+
+// Stores v as a GEMM operand.  fp32 operands are stored as they are.  bf16 operands are stored as a
+// pair hi = bf16(v), lo = bf16(v - hi) when a second array is given, so that the tensor-core product
+// with bf16 weights sees the activation to about 16 mantissa bits (hi and lo are two rows of the same
+// GEMM whose results are added).
+template <typename T> __device__ __forceinline__ void store_operand(T* hi, T* lo, size_t i, float v);
+template <> __device__ __forceinline__ void store_operand<float>(float* hi, float*, size_t i, float v) { hi[i] = v; }
+template <> __device__ __forceinline__ void store_operand<__nv_bfloat16>(__nv_bfloat16* hi, __nv_bfloat16* lo, size_t i, float v) {
+  const __nv_bfloat16 h = __float2bfloat16_rn(v);
+  hi[i] = h;
+  if (lo != nullptr) lo[i] = __float2bfloat16_rn(v - __bfloat162float(h));
+}
 
 // 16-byte vector of elements of type T, unpacked to fp32.
 template <typename T> struct Vec16;

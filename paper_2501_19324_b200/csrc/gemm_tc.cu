@@ -108,7 +108,10 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
 }
 
 template <int MT> struct TcCfg {
-  static constexpr int kStages = MT <= 64 ? 8 : (MT == 128 ? 6 : 4);
+  // tiles of up to 128 x-rows leave room for two CTAs per SM (one streams while the other starts
+  // up or drains); the 256-row tile of the dense regime takes the SM alone
+  static constexpr int kCtasPerSm = MT <= 128 ? 2 : 1;
+  static constexpr int kStages = MT <= 32 ? 5 : (MT == 64 ? 4 : (MT == 128 ? 3 : 4));
   static constexpr int kABytes = kTileN * kTileK * 2;
   static constexpr int kBBytes = MT * kTileK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
@@ -118,13 +121,17 @@ template <int MT> struct TcCfg {
   static constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(MT >> 3) << 17) | ((uint32_t)(kTileN >> 4) << 24);
 };
 
-template <int MT>
-__global__ void __launch_bounds__(192, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x, float* __restrict__ Y,
+// SPLIT: the x operand is a pair (hi, lo) of bf16 matrices whose sum is the activation; the tile
+// holds MT/2 rows of hi followed by the same MT/2 rows of lo, and the epilogue adds the two halves.
+template <int MT, bool SPLIT>
+__global__ void __launch_bounds__(192, TcCfg<MT>::kCtasPerSm)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x,
+               const __grid_constant__ CUtensorMap tm_x_lo, float* __restrict__ Y,
                int M, int N, int K, int accumulate, int splits, int kb_per_split, float* __restrict__ partials,
                int* __restrict__ counters, int* __restrict__ err, const int32_t* __restrict__ n_active) {
   if (n_active != nullptr && *n_active == 0) return;
   using Cfg = TcCfg<MT>;
+  constexpr int kRows = SPLIT ? MT / 2 : MT;   // distinct x rows per tile
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint64_t* full = (uint64_t*)(smem + (size_t)Cfg::kStages * Cfg::kStageBytes);
@@ -134,7 +141,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
   volatile uint32_t* flags = tmem_slot + 1;   // [0] abort, [1] last-arriver flag
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n0 = blockIdx.x * kTileN, m0 = blockIdx.y * MT, split = blockIdx.z;
+  const int n0 = blockIdx.x * kTileN, m0 = blockIdx.y * kRows, split = blockIdx.z;
   const int total_kb = (K + kTileK - 1) / kTileK;
   const int kb0 = split * kb_per_split;
   const int kb1 = min(total_kb, kb0 + kb_per_split);
@@ -165,6 +172,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
         mbar_expect_tx(&full[s], Cfg::kStageBytes);
         tma_load_2d(a, &tm_w, &full[s], (kb0 + i) * kTileK, n0);
         tma_load_2d(a + Cfg::kABytes, &tm_x, &full[s], (kb0 + i) * kTileK, m0);
+        if (SPLIT) tma_load_2d(a + Cfg::kABytes + kRows * kTileK * 2, &tm_x_lo, &full[s], (kb0 + i) * kTileK, m0);
         issued = i + 1;
       }
       if (!ok) {
@@ -209,14 +217,25 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
     const int n_local = warp * 32 + lane;
     const int n = n0 + n_local;
     const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16);
-    const int m_valid = min(MT, M - m0);
+    const int m_valid = min(kRows, M - m0);
     const int tile = blockIdx.y * gridDim.x + blockIdx.x;
-    const size_t tile_elems = (size_t)kTileN * MT;
+    const size_t tile_elems = (size_t)kTileN * kRows;
     if (ok) {
       float* part = partials + ((size_t)split * gridDim.x * gridDim.y + tile) * tile_elems;
       for (int c = 0; c < m_valid; c += 16) {
         float v[16];
         tmem_ld16(taddr + c, v);
+        if (SPLIT) {
+          if (kRows == 8) {          // hi in columns 0..7, lo in columns 8..15 of the same load
+#pragma unroll
+            for (int j = 0; j < 8; ++j) v[j] += v[j + 8];
+          } else {
+            float w[16];
+            tmem_ld16(taddr + kRows + c, w);
+#pragma unroll
+            for (int j = 0; j < 16; ++j) v[j] += w[j];
+          }
+        }
         if (splits == 1) {
           if (n < N) {
 #pragma unroll
@@ -322,26 +341,30 @@ bool get_map(const void* ptr, int rows, int cols, int box_rows, CUtensorMap* out
   return true;
 }
 
-int pick_mt(int M) {
+// Rows of x per tile: the smallest tile that holds M, up to 128 (split operand) or 256 (plain).
+int pick_rows(int M, bool split_operand) {
+  if (split_operand && M <= 8) return 8;
   if (M <= 16) return 16;
   if (M <= 32) return 32;
   if (M <= 64) return 64;
-  if (M <= 128) return 128;
+  if (M <= 128 || split_operand) return 128;
   return 256;
 }
 
-struct TcPlan { int mt, n_tiles, m_tiles, splits, kb_per_split; };
+struct TcPlan { int rows, mt, n_tiles, m_tiles, splits, kb_per_split; };
 
-TcPlan plan_tc(int M, int N, int K) {
+TcPlan plan_tc(int M, int N, int K, bool split_operand) {
   TcPlan p;
-  p.mt = pick_mt(M);
+  p.rows = pick_rows(M, split_operand);
+  p.mt = split_operand ? 2 * p.rows : p.rows;
   p.n_tiles = (N + kTileN - 1) / kTileN;
-  p.m_tiles = (M + p.mt - 1) / p.mt;
+  p.m_tiles = (M + p.rows - 1) / p.rows;
   const int tiles = p.n_tiles * p.m_tiles;
   const int total_kb = (K + kTileK - 1) / kTileK;
   int splits = 1;
-  if (tiles < 148 && tiles <= kMaxSplitTiles && p.mt <= 64) {
-    splits = (2 * 148 + tiles - 1) / tiles;
+  if (tiles < 148 && tiles <= kMaxSplitTiles && p.rows <= 64) {
+    // aim at one wave of two CTAs per SM, each with at least two k-blocks
+    splits = std::max(1, (2 * 148) / tiles);
     splits = std::min(splits, std::max(1, total_kb / 2));
     splits = std::min(splits, kMaxSplitCtas / tiles);
     splits = std::max(splits, 1);
@@ -351,18 +374,19 @@ TcPlan plan_tc(int M, int N, int K) {
   return p;
 }
 
-template <int MT>
-cudaError_t launch_mt(const CUtensorMap& tw, const CUtensorMap& tx, float* y, int M, int N, int K, int accumulate,
-                      const TcPlan& p, float* partials, int* counters, int* err, const int32_t* n_active, cudaStream_t s) {
+template <int MT, bool SPLIT>
+cudaError_t launch_mt(const CUtensorMap& tw, const CUtensorMap& tx, const CUtensorMap& txl, float* y, int M, int N, int K,
+                      int accumulate, const TcPlan& p, float* partials, int* counters, int* err, const int32_t* n_active,
+                      cudaStream_t s) {
   static bool configured = false;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<MT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TcCfg<MT>::kSmemBytes);
+    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<MT, SPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TcCfg<MT>::kSmemBytes);
     if (e != cudaSuccess) return e;
     configured = true;
   }
   dim3 grid(p.n_tiles, p.m_tiles, p.splits);
-  gemm_tc_kernel<MT><<<grid, 192, TcCfg<MT>::kSmemBytes, s>>>(tw, tx, y, M, N, K, accumulate, p.splits, p.kb_per_split,
-                                                              partials, counters, err, n_active);
+  gemm_tc_kernel<MT, SPLIT><<<grid, 192, TcCfg<MT>::kSmemBytes, s>>>(tw, tx, txl, y, M, N, K, accumulate, p.splits,
+                                                                     p.kb_per_split, partials, counters, err, n_active);
   return launched(1);
 }
 
@@ -375,40 +399,55 @@ bool gemm_tc_supported(int dtype, int M, int N, int K) {
 // Layout of the scratch: [0, 4096) tile counters (kept zero between launches), then one int error
 // flag region of 256 bytes, then split-K partial tiles.
 size_t gemm_scratch_bytes(int M) {
-  const int mt = pick_mt(M);
-  const size_t part = mt <= 64 ? (size_t)kMaxSplitCtas * kTileN * mt * 4 : 0;
+  const int rows = pick_rows(M, false);
+  const size_t part = rows <= 64 ? (size_t)kMaxSplitCtas * kTileN * std::min(64, std::max(rows, 16)) * 4 : 0;
   return kCounterBytes + 256 + part;
 }
 
 // Enough for any M (split-K is only used with tiles of at most 64 rows of x).
 size_t gemm_scratch_bytes_any() { return gemm_scratch_bytes(64); }
 
-cudaError_t launch_gemm_tc(const void* W, const void* x, float* y, int M, int N, int K, int accumulate,
+cudaError_t launch_gemm_tc(const void* W, const void* x, const void* x_lo, float* y, int M, int N, int K, int accumulate,
                            void* scratch, size_t scratch_bytes, const int32_t* n_active, cudaStream_t s) {
   if (M <= 0) return cudaSuccess;
   if (!scratch || scratch_bytes < gemm_scratch_bytes(M)) return cudaErrorInvalidValue;
-  if (((uintptr_t)W & 15) || ((uintptr_t)x & 15)) return cudaErrorMisalignedAddress;
-  const TcPlan p = plan_tc(M, N, K);
-  CUtensorMap tw, tx;
-  if (!get_map(W, N, K, kTileN, &tw) || !get_map(x, M, K, p.mt, &tx)) return cudaErrorNotSupported;
+  if (((uintptr_t)W & 15) || ((uintptr_t)x & 15) || ((uintptr_t)x_lo & 15)) return cudaErrorMisalignedAddress;
+  const bool split_operand = x_lo != nullptr;
+  const TcPlan p = plan_tc(M, N, K, split_operand);
+  CUtensorMap tw, tx, txl;
+  if (!get_map(W, N, K, kTileN, &tw) || !get_map(x, M, K, p.rows, &tx)) return cudaErrorNotSupported;
+  if (split_operand) { if (!get_map(x_lo, M, K, p.rows, &txl)) return cudaErrorNotSupported; }
+  else txl = tx;
   int* counters = (int*)scratch;
   int* err = (int*)((char*)scratch + kCounterBytes);
   float* partials = (float*)((char*)scratch + kCounterBytes + 256);
-  switch (p.mt) {
-    case 16: return launch_mt<16>(tw, tx, y, M, N, K, accumulate, p, partials, counters, err, n_active, s);
-    case 32: return launch_mt<32>(tw, tx, y, M, N, K, accumulate, p, partials, counters, err, n_active, s);
-    case 64: return launch_mt<64>(tw, tx, y, M, N, K, accumulate, p, partials, counters, err, n_active, s);
-    case 128: return launch_mt<128>(tw, tx, y, M, N, K, accumulate, p, partials, counters, err, n_active, s);
-    default: return launch_mt<256>(tw, tx, y, M, N, K, accumulate, p, partials, counters, err, n_active, s);
+#define RSD_TC(MT, SP) return launch_mt<MT, SP>(tw, tx, txl, y, M, N, K, accumulate, p, partials, counters, err, n_active, s)
+  if (split_operand) {
+    switch (p.mt) {
+      case 16: RSD_TC(16, true);
+      case 32: RSD_TC(32, true);
+      case 64: RSD_TC(64, true);
+      case 128: RSD_TC(128, true);
+      default: RSD_TC(256, true);
+    }
   }
+  switch (p.mt) {
+    case 16: RSD_TC(16, false);
+    case 32: RSD_TC(32, false);
+    case 64: RSD_TC(64, false);
+    case 128: RSD_TC(128, false);
+    default: RSD_TC(256, false);
+  }
+#undef RSD_TC
 }
 
-cudaError_t launch_gemm(int dtype, const void* W, const void* x, float* y, int M, int N, int K, int accumulate,
-                        int impl, void* scratch, size_t scratch_bytes, const int32_t* n_active, cudaStream_t s) {
+cudaError_t launch_gemm(int dtype, const void* W, const void* x, const void* x_lo, float* y, int M, int N, int K,
+                        int accumulate, int impl, void* scratch, size_t scratch_bytes, const int32_t* n_active,
+                        cudaStream_t s) {
   const bool tc_ok = gemm_tc_supported(dtype, M, N, K) && scratch && scratch_bytes >= gemm_scratch_bytes(M);
   if (impl == 2 || (impl == 0 && tc_ok && M > 4))
-    return launch_gemm_tc(W, x, y, M, N, K, accumulate, scratch, scratch_bytes, n_active, s);
-  return launch_gemm_simt(dtype, W, x, y, M, N, K, accumulate, n_active, s);
+    return launch_gemm_tc(W, x, x_lo, y, M, N, K, accumulate, scratch, scratch_bytes, n_active, s);
+  return launch_gemm_simt(dtype, W, x, dtype == 1 ? x_lo : nullptr, y, M, N, K, accumulate, n_active, s);
 }
 
 }  // namespace rsd

@@ -37,38 +37,42 @@ struct KvView {
 
 cudaError_t launch_embed(int dtype, const void* embed, PassView p, float* x, int d, cudaStream_t s);
 // out[t] = rmsnorm(x[src ? src[t] : t]); rows with src[t] < 0 are skipped.
-cudaError_t launch_rmsnorm(int dtype, const float* x, const void* gain, void* out, int T, int d, float eps,
+// out (and out_lo when given, bf16 only: the low half of a split-precision operand)
+cudaError_t launch_rmsnorm(int dtype, const float* x, const void* gain, void* out, void* out_lo, int T, int d, float eps,
                            const int32_t* src, const int32_t* n_active, cudaStream_t s);
-cudaError_t launch_gemm_simt(int dtype, const void* W, const void* x, float* y, int M, int N, int K,
+// x_lo (nullable, bf16 only): second operand matrix added to x (split-precision activations).
+cudaError_t launch_gemm_simt(int dtype, const void* W, const void* x, const void* x_lo, float* y, int M, int N, int K,
                              int accumulate, const int32_t* n_active, cudaStream_t s);
 // tcgen05 / TMEM / TMA GEMM (bf16): same contract as launch_gemm_simt; `scratch` holds split-K
 // partial tiles and tile counters (the counters must be zero on entry and are left zero).
 bool gemm_tc_supported(int dtype, int M, int N, int K);
 size_t gemm_scratch_bytes(int M);
 size_t gemm_scratch_bytes_any();
-cudaError_t launch_gemm_tc(const void* W, const void* x, float* y, int M, int N, int K, int accumulate,
+cudaError_t launch_gemm_tc(const void* W, const void* x, const void* x_lo, float* y, int M, int N, int K, int accumulate,
                            void* scratch, size_t scratch_bytes, const int32_t* n_active, cudaStream_t s);
 // impl: 0 = by shape, 1 = SIMT split-K GEMV, 2 = tcgen05.
-cudaError_t launch_gemm(int dtype, const void* W, const void* x, float* y, int M, int N, int K, int accumulate,
-                        int impl, void* scratch, size_t scratch_bytes, const int32_t* n_active, cudaStream_t s);
+cudaError_t launch_gemm(int dtype, const void* W, const void* x, const void* x_lo, float* y, int M, int N, int K,
+                        int accumulate, int impl, void* scratch, size_t scratch_bytes, const int32_t* n_active,
+                        cudaStream_t s);
 cudaError_t launch_rope_table(float2* table, int n_pos, int hd, float theta, cudaStream_t s);
 // Splits qkv [T, (H+2KV)*hd] (fp32): rotated q -> q_out [T, H*hd] fp32; rotated k and v -> KV pages.
-cudaError_t launch_rope_kv(int dtype, const float* qkv, PassView p, float* q_out, KvView kv, const float2* rope,
+// kv_dtype: element type of the cache: 0 fp32, 1 bf16, 2 fp16.
+cudaError_t launch_rope_kv(int kv_dtype, const float* qkv, PassView p, float* q_out, KvView kv, const float2* rope,
                            int H, int KV, int hd, cudaStream_t s);
 cudaError_t launch_rope_only(float* v, const int32_t* pos, int T, int n_heads, int hd, float theta, cudaStream_t s);
 // Causal attention of every slot over positions [0, tok_pos] of its row, read from the pages.
-cudaError_t launch_attn_generic(int dtype, const float* q, PassView p, KvView kv, void* out, int out_dtype, int H,
-                                int KV, int hd, cudaStream_t s);
-cudaError_t launch_swiglu(int dtype, const float* gu, void* out, int T, int F, const int32_t* n_active,
+cudaError_t launch_attn_generic(int kv_dtype, const float* q, PassView p, KvView kv, void* out, void* out_lo,
+                                int out_dtype, int H, int KV, int hd, cudaStream_t s);
+cudaError_t launch_swiglu(int dtype, const float* gu, void* out, void* out_lo, int T, int F, const int32_t* n_active,
                           cudaStream_t s);
 
 // Decode attention (one query per row) with split-KV partial results merged in a second pass.
 size_t attn_decode_scratch_bytes(int B, int H, int hd, int max_ctx);
 // Slot i attends positions [0, len_or_pos[i] + len_offset) of row slot_row[i] (slot i itself when
 // slot_row is null); slot_row[i] < 0 skips the slot.
-cudaError_t launch_attn_decode(int dtype, const float* q, const void* pool_layer, const int32_t* page_table,
+cudaError_t launch_attn_decode(int kv_dtype, const float* q, const void* pool_layer, const int32_t* page_table,
                                int max_pages, const int32_t* slot_row, const int32_t* len_or_pos, int len_offset,
-                               void* out, int out_dtype, int B, int H, int KV, int hd, int max_ctx, void* scratch,
+                               void* out, void* out_lo, int out_dtype, int B, int H, int KV, int hd, int max_ctx, void* scratch,
                                size_t scratch_bytes, const int32_t* n_active, cudaStream_t s);
 
 struct SampleArgs {

@@ -40,7 +40,8 @@ cudaError_t launch_embed(int dtype, const void* embed, PassView p, float* x, int
 // ---------------------------------------------------------------------------------------------
 template <typename OT, typename GT>
 __global__ void rmsnorm_kernel(const float* __restrict__ x, const GT* __restrict__ gain, OT* __restrict__ out,
-                               int d, float eps, const int32_t* __restrict__ src, const int32_t* n_active) {
+                               OT* __restrict__ out_lo, int d, float eps, const int32_t* __restrict__ src,
+                               const int32_t* n_active) {
   RSD_SKIP_IF_IDLE(n_active);
   __shared__ float red[33];
   const int t = blockIdx.x;
@@ -57,24 +58,24 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, const GT* __restrict
   }
   ss = block_sum(ss, red);
   const float inv = rsqrtf(ss / (float)d + eps);
-  OT* o = out + (size_t)t * d;
+  const size_t o = (size_t)t * d;
   for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) {
     float4 v = *reinterpret_cast<const float4*>(xr + i);
-    o[i] = from_f32<OT>(v.x * inv * to_f32(gain[i]));
-    o[i + 1] = from_f32<OT>(v.y * inv * to_f32(gain[i + 1]));
-    o[i + 2] = from_f32<OT>(v.z * inv * to_f32(gain[i + 2]));
-    o[i + 3] = from_f32<OT>(v.w * inv * to_f32(gain[i + 3]));
+    store_operand<OT>(out, out_lo, o + i, v.x * inv * to_f32(gain[i]));
+    store_operand<OT>(out, out_lo, o + i + 1, v.y * inv * to_f32(gain[i + 1]));
+    store_operand<OT>(out, out_lo, o + i + 2, v.z * inv * to_f32(gain[i + 2]));
+    store_operand<OT>(out, out_lo, o + i + 3, v.w * inv * to_f32(gain[i + 3]));
   }
 }
 
-cudaError_t launch_rmsnorm(int dtype, const float* x, const void* gain, void* out, int T, int d, float eps,
+cudaError_t launch_rmsnorm(int dtype, const float* x, const void* gain, void* out, void* out_lo, int T, int d, float eps,
                            const int32_t* src, const int32_t* n_active, cudaStream_t s) {
   if (T <= 0) return cudaSuccess;
   const int threads = d >= 2048 ? 512 : 256;
   if (dtype == 1)
-    rmsnorm_kernel<__nv_bfloat16, __nv_bfloat16><<<T, threads, 0, s>>>(x, (const __nv_bfloat16*)gain, (__nv_bfloat16*)out, d, eps, src, n_active);
+    rmsnorm_kernel<__nv_bfloat16, __nv_bfloat16><<<T, threads, 0, s>>>(x, (const __nv_bfloat16*)gain, (__nv_bfloat16*)out, (__nv_bfloat16*)out_lo, d, eps, src, n_active);
   else
-    rmsnorm_kernel<float, float><<<T, threads, 0, s>>>(x, (const float*)gain, (float*)out, d, eps, src, n_active);
+    rmsnorm_kernel<float, float><<<T, threads, 0, s>>>(x, (const float*)gain, (float*)out, nullptr, d, eps, src, n_active);
   return launched(1);
 }
 
@@ -86,8 +87,8 @@ cudaError_t launch_rmsnorm(int dtype, const float* x, const void* gain, void* ou
 // ---------------------------------------------------------------------------------------------
 template <typename WT, int MT>
 __global__ void __launch_bounds__(256)
-gemv_splitk_kernel(const WT* __restrict__ W, const WT* __restrict__ X, float* __restrict__ Y, int M, int N, int K,
-                   int ks, int accumulate, const int32_t* n_active) {
+gemv_splitk_kernel(const WT* __restrict__ W, const WT* __restrict__ X, const WT* __restrict__ X_lo, float* __restrict__ Y,
+                   int M, int N, int K, int ks, int accumulate, const int32_t* n_active) {
   RSD_SKIP_IF_IDLE(n_active);
   constexpr int VN = Vec16<WT>::N;
   __shared__ float part[8][MT];
@@ -110,6 +111,12 @@ gemv_splitk_kernel(const WT* __restrict__ W, const WT* __restrict__ X, float* __
         if (m0 + m < M) {
           Vec16<WT> xv;
           xv.load(X + (size_t)(m0 + m) * K + (size_t)v * VN);
+          if (X_lo != nullptr) {
+            Vec16<WT> xl;
+            xl.load(X_lo + (size_t)(m0 + m) * K + (size_t)v * VN);
+#pragma unroll
+            for (int j = 0; j < VN; ++j) xv.v[j] += xl.v[j];
+          }
 #pragma unroll
           for (int j = 0; j < VN; ++j) acc[m] = fmaf(w.v[j], xv.v[j], acc[m]);
         }
@@ -137,7 +144,7 @@ gemv_splitk_kernel(const WT* __restrict__ W, const WT* __restrict__ X, float* __
   }
 }
 
-cudaError_t launch_gemm_simt(int dtype, const void* W, const void* x, float* y, int M, int N, int K,
+cudaError_t launch_gemm_simt(int dtype, const void* W, const void* x, const void* x_lo, float* y, int M, int N, int K,
                              int accumulate, const int32_t* n_active, cudaStream_t s) {
   if (M <= 0 || N <= 0) return cudaSuccess;
   // pick the split so that the grid covers the 148 SMs a few times over
@@ -146,9 +153,9 @@ cudaError_t launch_gemm_simt(int dtype, const void* W, const void* x, float* y, 
   constexpr int MT = 8;
   dim3 grid((N + (8 / ks) - 1) / (8 / ks), (M + MT - 1) / MT);
   if (dtype == 1)
-    gemv_splitk_kernel<__nv_bfloat16, MT><<<grid, 256, 0, s>>>((const __nv_bfloat16*)W, (const __nv_bfloat16*)x, y, M, N, K, ks, accumulate, n_active);
+    gemv_splitk_kernel<__nv_bfloat16, MT><<<grid, 256, 0, s>>>((const __nv_bfloat16*)W, (const __nv_bfloat16*)x, (const __nv_bfloat16*)x_lo, y, M, N, K, ks, accumulate, n_active);
   else
-    gemv_splitk_kernel<float, MT><<<grid, 256, 0, s>>>((const float*)W, (const float*)x, y, M, N, K, ks, accumulate, n_active);
+    gemv_splitk_kernel<float, MT><<<grid, 256, 0, s>>>((const float*)W, (const float*)x, nullptr, y, M, N, K, ks, accumulate, n_active);
   return launched(1);
 }
 
@@ -215,10 +222,12 @@ __global__ void rope_kv_kernel(const float* __restrict__ qkv, PassView p, float*
   }
 }
 
-cudaError_t launch_rope_kv(int dtype, const float* qkv, PassView p, float* q_out, KvView kv, const float2* rope,
+cudaError_t launch_rope_kv(int kv_dtype, const float* qkv, PassView p, float* q_out, KvView kv, const float2* rope,
                            int H, int KV, int hd, cudaStream_t s) {
   if (p.T <= 0) return cudaSuccess;
-  if (dtype == 1)
+  if (kv_dtype == 2)
+    rope_kv_kernel<__half><<<p.T, 256, 0, s>>>(qkv, p, q_out, (__half*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd);
+  else if (kv_dtype == 1)
     rope_kv_kernel<__nv_bfloat16><<<p.T, 256, 0, s>>>(qkv, p, q_out, (__nv_bfloat16*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd);
   else
     rope_kv_kernel<float><<<p.T, 256, 0, s>>>(qkv, p, q_out, (float*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd);
@@ -253,7 +262,8 @@ cudaError_t launch_rope_only(float* v, const int32_t* pos, int T, int n_heads, i
 template <typename KT, typename OT, int HD>
 __global__ void __launch_bounds__(128)
 attn_generic_kernel(const float* __restrict__ q, PassView p, const KT* __restrict__ pool,
-                    const int32_t* __restrict__ page_table, int max_pages, OT* __restrict__ out, int H, int KV) {
+                    const int32_t* __restrict__ page_table, int max_pages, OT* __restrict__ out, OT* __restrict__ out_lo,
+                    int H, int KV) {
   RSD_SKIP_IF_IDLE(p.n_active);
   constexpr int DPL = HD / 32;
   const int lane = threadIdx.x & 31;
@@ -310,20 +320,22 @@ attn_generic_kernel(const float* __restrict__ q, PassView p, const KT* __restric
   }
   const float inv = 1.f / l;
 #pragma unroll
-  for (int i = 0; i < DPL; ++i) out[((size_t)t * H + h) * HD + lane * DPL + i] = from_f32<OT>(acc[i] * inv);
+  for (int i = 0; i < DPL; ++i) store_operand<OT>(out, out_lo, ((size_t)t * H + h) * HD + lane * DPL + i, acc[i] * inv);
 }
 
-cudaError_t launch_attn_generic(int dtype, const float* q, PassView p, KvView kv, void* out, int out_dtype, int H,
-                                int KV, int hd, cudaStream_t s) {
+cudaError_t launch_attn_generic(int kv_dtype, const float* q, PassView p, KvView kv, void* out, void* out_lo,
+                                int out_dtype, int H, int KV, int hd, cudaStream_t s) {
   if (p.T <= 0) return cudaSuccess;
   const int warps = p.T * H;
   const int blocks = (warps + 3) / 4;
 #define RSD_ATTN(KT, OT, HD) \
-  attn_generic_kernel<KT, OT, HD><<<blocks, 128, 0, s>>>(q, p, (const KT*)kv.pool_layer, kv.page_table, kv.max_pages, (OT*)out, H, KV)
+  attn_generic_kernel<KT, OT, HD><<<blocks, 128, 0, s>>>(q, p, (const KT*)kv.pool_layer, kv.page_table, kv.max_pages, (OT*)out, (OT*)out_lo, H, KV)
+#define RSD_ATTN_HD(KT, OT) do { if (hd == 128) RSD_ATTN(KT, OT, 128); else RSD_ATTN(KT, OT, 64); } while (0)
   using bf = __nv_bfloat16;
-  if (dtype == 1 && out_dtype == 1) { if (hd == 128) RSD_ATTN(bf, bf, 128); else RSD_ATTN(bf, bf, 64); }
-  else if (dtype == 1) { if (hd == 128) RSD_ATTN(bf, float, 128); else RSD_ATTN(bf, float, 64); }
-  else { if (hd == 128) RSD_ATTN(float, float, 128); else RSD_ATTN(float, float, 64); }
+  if (kv_dtype == 2) { if (out_dtype == 1) RSD_ATTN_HD(__half, bf); else RSD_ATTN_HD(__half, float); }
+  else if (kv_dtype == 1) { if (out_dtype == 1) RSD_ATTN_HD(bf, bf); else RSD_ATTN_HD(bf, float); }
+  else RSD_ATTN_HD(float, float);
+#undef RSD_ATTN_HD
 #undef RSD_ATTN
   return launched(1);
 }
@@ -332,23 +344,25 @@ cudaError_t launch_attn_generic(int dtype, const float* q, PassView p, KvView kv
 // SwiGLU: out[t, f] = silu(gu[t, f]) * gu[t, F + f]
 // ---------------------------------------------------------------------------------------------
 template <typename OT>
-__global__ void swiglu_kernel(const float* __restrict__ gu, OT* __restrict__ out, int T, int F, const int32_t* n_active) {
+__global__ void swiglu_kernel(const float* __restrict__ gu, OT* __restrict__ out, OT* __restrict__ out_lo, int T, int F,
+                              const int32_t* n_active) {
   RSD_SKIP_IF_IDLE(n_active);
   const size_t n = (size_t)T * F;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
     const size_t t = i / F, f = i % F;
     const float a = gu[t * 2 * F + f], b = gu[t * 2 * F + F + f];
-    out[i] = from_f32<OT>(a / (1.f + expf(-a)) * b);
+    store_operand<OT>(out, out_lo, i, a / (1.f + expf(-a)) * b);
   }
 }
 
-cudaError_t launch_swiglu(int dtype, const float* gu, void* out, int T, int F, const int32_t* n_active, cudaStream_t s) {
+cudaError_t launch_swiglu(int dtype, const float* gu, void* out, void* out_lo, int T, int F, const int32_t* n_active,
+                          cudaStream_t s) {
   if (T <= 0) return cudaSuccess;
   const size_t n = (size_t)T * F;
   int blocks = (int)((n + 255) / 256);
   if (blocks > 148 * 8) blocks = 148 * 8;
-  if (dtype == 1) swiglu_kernel<__nv_bfloat16><<<blocks, 256, 0, s>>>(gu, (__nv_bfloat16*)out, T, F, n_active);
-  else swiglu_kernel<float><<<blocks, 256, 0, s>>>(gu, (float*)out, T, F, n_active);
+  if (dtype == 1) swiglu_kernel<__nv_bfloat16><<<blocks, 256, 0, s>>>(gu, (__nv_bfloat16*)out, (__nv_bfloat16*)out_lo, T, F, n_active);
+  else swiglu_kernel<float><<<blocks, 256, 0, s>>>(gu, (float*)out, nullptr, T, F, n_active);
   return launched(1);
 }
 

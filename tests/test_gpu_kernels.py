@@ -79,6 +79,17 @@ def test_gemm_tcgen05(M, N, K):
     np.testing.assert_allclose(acc, want + y0, rtol=0, atol=tol)
     again = rb.k_gemm(Wd, xd, impl=2).cpu().numpy()
     assert np.array_equal(again, got)          # deterministic, whatever order the split CTAs finish in
+    # split-precision activations: x = hi + lo, both bf16, both multiplied on the tensor cores
+    xf = dev(x)
+    hi = xf.to(torch.bfloat16)
+    lo = (xf - hi.float()).to(torch.bfloat16)
+    want2 = oracle.matmul(W, (hi.float() + lo.float()).cpu().numpy())
+    got2 = rb.k_gemm(Wd, hi, impl=2, x_lo=lo).cpu().numpy()
+    np.testing.assert_allclose(got2, want2, rtol=0, atol=tol)
+    assert np.abs(want2 - oracle.matmul(W, x)).max() < 1e-3 * np.sqrt(K) * 0.02 + 1e-4   # hi + lo ~ x
+    if M <= 4 or True:
+        got3 = rb.k_gemm(Wd, hi, impl=1, x_lo=lo).cpu().numpy()                # SIMT path, same operands
+        np.testing.assert_allclose(got3, want2, rtol=0, atol=tol)
 
 
 def test_rmsnorm_rope_swiglu():
@@ -188,7 +199,8 @@ def paged_kv(rng, B, KV, hd, ctx, dtype, max_pages):
 @pytest.mark.parametrize("dtype,hd,H,KV", [(torch.float32, 64, 4, 2), (torch.bfloat16, 128, 12, 2),
                                           (torch.bfloat16, 128, 28, 4), (torch.bfloat16, 128, 8, 1),
                                           (torch.bfloat16, 64, 6, 2), (torch.bfloat16, 128, 16, 1),
-                                          (torch.bfloat16, 128, 64, 8)])
+                                          (torch.bfloat16, 128, 64, 8), (torch.float16, 128, 12, 2),
+                                          (torch.float16, 64, 4, 2), (torch.float16, 128, 28, 4)])
 def test_decode_attention_against_definition(dtype, hd, H, KV):
     rng = np.random.default_rng(4)
     ctx = [1, 15, 16, 17, 33, 250, 1031, 2049]
@@ -196,7 +208,7 @@ def test_decode_attention_against_definition(dtype, hd, H, KV):
     max_pages = 130
     # fp32 caches: fp32 arithmetic.  bf16 caches: the query and the softmax weights are rounded to
     # bf16 for the tensor-core products (relative 2^-9 each) on values of order one
-    tol = 2e-5 if dtype == torch.float32 else 1.5e-2
+    tol = {torch.float32: 2e-5, torch.bfloat16: 1.5e-2, torch.float16: 2e-3}[dtype]
     pool, table, Ks, Vs = paged_kv(rng, B, KV, hd, ctx, dtype, max_pages)
     q = rng.normal(size=(B, H, hd)).astype(np.float32)
     got = rb.k_attn_decode(dev(q), pool, table, dev(np.array(ctx, np.int32)), KV).cpu().numpy()
