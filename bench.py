@@ -181,7 +181,7 @@ def workload_config(args) -> dict:
     d, p, t, B, lo, hi, cap = WORKLOADS[args.workload]
     return {"workload": f"{args.workload}: draft {d} / PRM {p} / target {t} shapes, batch {B}, prompts {lo}-{hi} tokens, "
                         f"step <= {cap} tokens, Gumbel-max T=0.7, delta at the 70% accept quantile",
-            "batch": B, "max_step_tokens": cap, "replicas": args.gpus,
+            "batch": B, "max_step_tokens": args.cap or cap, "replicas": args.gpus,
             "l2": "weights and KV read per decode iteration exceed the 126 MB L2 (no flush needed)"}
 
 
@@ -198,6 +198,8 @@ def run_ours(args, rank: int, world: int):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     d, p, t, B, lo, hi, cap = WORKLOADS[args.workload]
+    if args.cap:
+        cap = args.cap          # profiling aid: shorter steps (recorded in the config line)
     shapes = [ri.SHAPES[d], ri.SHAPES[p], ri.SHAPES[t]]
     heads = (ri.HEAD_LM, ri.HEAD_REWARD_SIGMOID, ri.HEAD_LM)
     models = [Model(sh, ri.gpu_model_tensors(sh, slot, 0, True, hk), hk)
@@ -305,6 +307,7 @@ def main():
     ap.add_argument("--workload", default="cfg2", choices=sorted(WORKLOADS))
     ap.add_argument("--time-stride", type=int, default=16, dest="time_stride")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cap", type=int, default=0, help="override the step cap (profiling aid)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
     rank = int(os.environ.get("RANK", 0))
