@@ -97,7 +97,10 @@ typedef struct {
   size_t workspace_bytes;
 } rsd_config;
 
-enum { RSD_DEBUG_KEEP_LOGITS = 1 /* keep every decode iteration's logits for rsd_debug_get_logits */ };
+enum {
+  RSD_DEBUG_KEEP_LOGITS = 1, /* keep every decode iteration's logits for rsd_debug_get_logits      */
+  RSD_DEBUG_NO_GRAPHS = 2    /* launch decode iterations kernel by kernel instead of as CUDA graphs */
+};
 
 /* Fills cfg->kv_bytes[] (enough pages for max_batch rows of max_seq_tokens) and
  * cfg->workspace_bytes for these three models.  Host only.  RSD_ERR_ARG on bad shapes.       */

@@ -71,6 +71,12 @@ struct rsd_ctx {
   size_t attn_scratch_bytes = 0;
   rsd_counters ctr{};
   int last_n_rej = 0;
+  // one CUDA graph per decode phase (draft, target): a whole decode iteration, replayed per token
+  cudaStream_t cap_stream = nullptr;
+  cudaGraphExec_t dec_graph[2] = {nullptr, nullptr};
+  int dec_graph_B[2] = {0, 0};
+  uint64_t dec_graph_kernels[2] = {0, 0};
+  bool time_this_iter = false, in_decode = false;
   // per-phase timing of rsd_step (rsd_debug_phase_ms)
   bool time_phases = false;
   cudaEvent_t ph_ev[8] = {};
@@ -187,7 +193,7 @@ size_t layout_workspace(const rsd_config& cfg, const rsd_model* const ms[3], rsd
   st.slot_row = TAKE(int32_t, B);
   st.last_idx = TAKE(int32_t, B);
   int32_t* scal = TAKE(int32_t, 16);
-  st.n_tok = scal + 0; st.n_rej = scal + 1; st.err = scal + 2; st.n_active = scal + 3; st.n_slots = scal + 4;
+  st.n_tok = scal + 0; st.n_rej = scal + 1; st.err = scal + 2; st.n_active = scal + 3; st.n_slots = scal + 4; st.iter = scal + 8;
   st.next_page = scal + 5;
   st.pass_capacity = B * S;
   st.pass_tok_id = TAKE(int32_t, (size_t)B * S);
@@ -287,8 +293,10 @@ int drain_gemm_events(rsd_ctx* c) {
 
 int gemm(rsd_ctx* c, const ModelHost& M, const void* W, const void* xin, const void* xin_lo, float* y, int Mrows, int N,
          int K, int accumulate, const int32_t* n_active, cudaStream_t s) {
-  const bool timed = c->time_stride > 0 && (c->gemm_calls++ % (uint64_t)c->time_stride) == 0 &&
-                     c->ev_used < c->ev_bytes.size();
+  // ragged passes: every stride-th GEMM; decode: every GEMM of the iterations chosen by decode_phase
+  const bool pick = c->in_decode ? c->time_this_iter
+                                 : (c->time_stride > 0 && (c->gemm_calls++ % (uint64_t)c->time_stride) == 0);
+  const bool timed = pick && c->ev_used < c->ev_bytes.size();
   if (timed) CU(cudaEventRecord(c->ev[2 * c->ev_used], s));
   CU(launch_gemm(M.m.dtype, W, xin, M.split ? xin_lo : nullptr, y, Mrows, N, K, accumulate, 0, c->gemm_scratch,
                  c->gemm_scratch_bytes, n_active, s));
@@ -354,41 +362,100 @@ int run_ingest(rsd_ctx* c, int which, int n_total, bool want_reward, cudaStream_
   return RSD_OK;
 }
 
-__global__ void scatter_logits_kernel(const float* logits, const int32_t* slot_row, float* dbg, int V, int C, int iter,
-                                      const int32_t* n_active) {
+__global__ void scatter_logits_kernel(const float* logits, const int32_t* slot_row, float* dbg, int V, int C,
+                                      const int32_t* iter, const int32_t* n_active) {
   if (*n_active == 0) return;
   const int row = slot_row[blockIdx.x];
   if (row < 0) return;
   const float* src = logits + (size_t)blockIdx.x * V;
-  float* dst = dbg + ((size_t)row * C + iter) * V;
+  float* dst = dbg + ((size_t)row * C + *iter) * V;
   for (int i = threadIdx.x; i < V; i += blockDim.x) dst[i] = src[i];
 }
 
-// One decode phase: up to C iterations of (prepare, model pass, lm_head, sample, append).
-int decode_phase(rsd_ctx* c, int which, int phase, int n_slots, cudaStream_t s) {
+// Enqueues one decode iteration: (prepare, model pass, final norm, lm_head, sample, append).
+int decode_iteration(rsd_ctx* c, int which, int phase, int n_slots, cudaStream_t s) {
   const ModelHost& M = c->mdl[which];
   const rsd_model& m = M.m;
+  CU(launch_decode_prepare(c->st, which, n_slots, s));
+  PassView p{c->st.pass_tok_id, c->st.pass_tok_row, c->st.pass_tok_pos, n_slots, c->st.n_active};
+  int rc = forward_pass(c, which, p, s);
+  if (rc) return rc;
+  CU(launch_rmsnorm(m.dtype, c->x, m.final_norm, c->h, M.split ? c->h_lo : nullptr, n_slots, m.d_model, m.rms_eps,
+                    nullptr, p.n_active, s));
+  rc = gemm(c, M, m.head, c->h, c->h_lo, c->logits, n_slots, m.vocab, m.d_model, 0, p.n_active, s);
+  if (rc) return rc;
+  if (c->dbg_logits[phase]) {
+    scatter_logits_kernel<<<n_slots, 256, 0, s>>>(c->logits, c->st.pass_tok_row, c->dbg_logits[phase], m.vocab, c->C,
+                                                  c->st.iter, c->st.n_active);
+    CU(launched(1));
+  }
+  SampleArgs a{c->logits, n_slots, m.vocab, c->v_limit, c->cfg.temperature, c->cfg.seed, which,
+               c->st.pass_tok_row, c->st.pass_tok_pos, c->sampled_slots, c->st.n_active};
+  CU(launch_sample(a, s));
+  CU(launch_decode_update(c->st, which, phase, c->sampled_slots, n_slots, c->lp, s));
+  return RSD_OK;
+}
+
+// Captures one decode iteration of `which` over all B slots into a graph (idle slots are skipped
+// inside the kernels), so that a token costs one graph launch instead of some 300 kernel launches.
+int ensure_decode_graph(rsd_ctx* c, int which, int phase) {
+  const int B = c->st.B;
+  if (c->dec_graph[phase] && c->dec_graph_B[phase] == B) return RSD_OK;
+  if (c->dec_graph[phase]) { cudaGraphExecDestroy(c->dec_graph[phase]); c->dec_graph[phase] = nullptr; }
+  if (!c->cap_stream) CU(cudaStreamCreateWithFlags(&c->cap_stream, cudaStreamNonBlocking));
+  const uint64_t before = launches_total();
+  CU(cudaStreamBeginCapture(c->cap_stream, cudaStreamCaptureModeThreadLocal));
+  const bool was_in_decode = c->in_decode, was_timed = c->time_this_iter;
+  c->in_decode = true; c->time_this_iter = false;          // no event records inside the capture
+  const int rc = decode_iteration(c, which, phase, B, c->cap_stream);
+  c->in_decode = was_in_decode; c->time_this_iter = was_timed;
+  cudaGraph_t graph = nullptr;
+  cudaError_t e = cudaStreamEndCapture(c->cap_stream, &graph);
+  if (rc) { if (graph) cudaGraphDestroy(graph); return rc; }
+  CU(e);
+  c->dec_graph_kernels[phase] = launches_total() - before;
+  e = cudaGraphInstantiate(&c->dec_graph[phase], graph, 0);
+  cudaGraphDestroy(graph);
+  CU(e);
+  c->dec_graph_B[phase] = B;
+  return RSD_OK;
+}
+
+// One decode phase: up to C iterations; every 16 iterations the host looks at the number of rows
+// still decoding and stops early when none is left.
+int decode_phase(rsd_ctx* c, int which, int phase, int n_slots, cudaStream_t s) {
   CU(launch_decode_begin(c->st, phase, s));
   if (n_slots <= 0) return RSD_OK;
-  for (int j = 0; j < c->C; ++j) {
-    CU(launch_decode_prepare(c->st, which, n_slots, s));
-    PassView p{c->st.pass_tok_id, c->st.pass_tok_row, c->st.pass_tok_pos, n_slots, c->st.n_active};
-    int rc = forward_pass(c, which, p, s);
-    if (rc) return rc;
-    CU(launch_rmsnorm(m.dtype, c->x, m.final_norm, c->h, M.split ? c->h_lo : nullptr, n_slots, m.d_model, m.rms_eps,
-                      nullptr, p.n_active, s));
-    rc = gemm(c, M, m.head, c->h, c->h_lo, c->logits, n_slots, m.vocab, m.d_model, 0, p.n_active, s);
-    if (rc) return rc;
-    if (c->dbg_logits[phase]) {
-      scatter_logits_kernel<<<n_slots, 256, 0, s>>>(c->logits, c->st.pass_tok_row, c->dbg_logits[phase], m.vocab, c->C, j, c->st.n_active);
-      CU(launched(1));
+  const bool graphs = !(c->cfg.debug_flags & RSD_DEBUG_NO_GRAPHS);
+  if (graphs) n_slots = c->st.B;   // fixed shape: slots beyond the phase's rows are idle
+  c->in_decode = true;
+  int rc = RSD_OK;
+  for (int j = 0; j < c->C && rc == RSD_OK; ++j) {
+    const bool timed_iter = c->time_stride > 0 && (j % 16) == 5;
+    // the first iteration ever runs kernel by kernel (it also sets every kernel's attributes), then
+    // the iteration is captured once and replayed
+    const bool have_graph = graphs && c->dec_graph[phase] && c->dec_graph_B[phase] == c->st.B;
+    if (graphs && !have_graph && j > 0) {
+      rc = ensure_decode_graph(c, which, phase);
+      if (rc) break;
     }
-    SampleArgs a{c->logits, n_slots, m.vocab, c->v_limit, c->cfg.temperature, c->cfg.seed, which,
-                 c->st.pass_tok_row, c->st.pass_tok_pos, c->sampled_slots, c->st.n_active};
-    CU(launch_sample(a, s));
-    CU(launch_decode_update(c->st, which, phase, j, c->sampled_slots, n_slots, c->lp, s));
+    if (graphs && !timed_iter && c->dec_graph[phase] && c->dec_graph_B[phase] == c->st.B) {
+      cudaError_t e = cudaGraphLaunch(c->dec_graph[phase], s);
+      if (e != cudaSuccess) { c->in_decode = false; CU(e); }
+      note_replayed_launches(c->dec_graph_kernels[phase]);
+    } else {
+      c->time_this_iter = timed_iter;
+      rc = decode_iteration(c, which, phase, n_slots, s);
+      c->time_this_iter = false;
+    }
+    if (rc == RSD_OK && (j & 15) == 15 && j + 1 < c->C) {
+      Scalars sc;
+      rc = read_scalars(c, s, &sc);
+      if (rc == RSD_OK && sc.n_active == 0) break;
+    }
   }
-  return RSD_OK;
+  c->in_decode = false;
+  return rc;
 }
 
 __global__ void init_rows_kernel(RowState st, const int32_t* flat, const int32_t* offsets, int B) {
@@ -680,6 +747,8 @@ int rsd_destroy(rsd_ctx* c) {
   cudaDeviceSynchronize();
   for (cudaEvent_t e : c->ev) cudaEventDestroy(e);
   for (cudaEvent_t e : c->ph_ev) if (e) cudaEventDestroy(e);
+  for (auto& g : c->dec_graph) if (g) cudaGraphExecDestroy(g);
+  if (c->cap_stream) cudaStreamDestroy(c->cap_stream);
   if (c->pinned) cudaFreeHost(c->pinned);
   delete c;
   return RSD_OK;

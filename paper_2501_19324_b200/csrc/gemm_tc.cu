@@ -29,6 +29,7 @@ cudaError_t launched(int n_kernels) {
   return cudaGetLastError();
 }
 uint64_t launches_total() { return g_launches.load(std::memory_order_relaxed); }
+void note_replayed_launches(uint64_t n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
 namespace {
 

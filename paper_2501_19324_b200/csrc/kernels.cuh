@@ -12,6 +12,7 @@ namespace rsd {
 // GPU launches.
 cudaError_t launched(int n_kernels);   // adds to the count and returns cudaGetLastError()
 uint64_t launches_total();
+void note_replayed_launches(uint64_t n);   // kernels run by replaying a captured graph
 
 constexpr int kPageTokens = 16;   // tokens per KV page
 constexpr int kMaxBatch = 1024;   // rows per context (one thread per row in the state kernels)
@@ -116,6 +117,7 @@ struct RowState {
   uint8_t* accept;
   int32_t *rej_idx, *n_rej;
   int32_t *slot_row, *n_slots; // decode slots of the current phase
+  int32_t *iter;               // iteration counter of the current decode phase
   int32_t *last_idx;           // [B] flat index of each row's last token in the current pass
   int32_t *n_tok;              // tokens of the current pass
   int32_t *err;                // first error raised on the device
@@ -137,7 +139,7 @@ cudaError_t launch_reserve_pages(const RowState& st, int which, ReserveMode mode
 cudaError_t launch_build_pass(const RowState& st, int which, PassMode mode, cudaStream_t s);
 cudaError_t launch_decode_begin(const RowState& st, int phase, cudaStream_t s);
 cudaError_t launch_decode_prepare(const RowState& st, int which, int n_slots, cudaStream_t s);
-cudaError_t launch_decode_update(const RowState& st, int which, int phase, int iter, const int32_t* sampled,
+cudaError_t launch_decode_update(const RowState& st, int which, int phase, const int32_t* sampled,
                                  int n_slots, const LoopParams& lp, cudaStream_t s);
 cudaError_t launch_gate(const RowState& st, float delta, const LoopParams& lp, cudaStream_t s);
 cudaError_t launch_commit(const RowState& st, const LoopParams& lp, int32_t* out_tokens, int32_t* out_len,

@@ -121,7 +121,7 @@ __global__ void __launch_bounds__(1024) decode_begin_kernel(RowState st, int pha
   }
   int total;
   block_exclusive_scan(part, scan, &total);
-  if (b == 0) st.n_active[0] = total;
+  if (b == 0) { st.n_active[0] = total; st.iter[0] = 0; }
   const int n_slots = phase == 0 ? st.B : st.n_rej[0];
   if (b == 0) st.n_slots[0] = n_slots;
   if (b < st.B) st.slot_row[b] = phase == 0 ? b : (b < n_slots ? st.rej_idx[b] : -1);
@@ -163,10 +163,11 @@ __device__ __forceinline__ bool ends_step(int t, const LoopParams& lp) {
   return t == lp.step_end_id;
 }
 
-// Appends iteration `iter`'s token of every active slot to its row and stops rows whose step ended.
+// Appends the current iteration's token of every active slot to its row and stops rows whose step ended.
 __global__ void __launch_bounds__(1024)
-decode_update_kernel(RowState st, int which, int phase, int iter, const int32_t* sampled, int n_slots, LoopParams lp) {
+decode_update_kernel(RowState st, int which, int phase, const int32_t* sampled, int n_slots, LoopParams lp) {
   if (st.n_active[0] == 0) return;
+  const int iter = st.iter[0];   // iteration of the current decode phase, kept on the device
   const int i = threadIdx.x;
   int ended = 0;
   if (i < n_slots) {
@@ -188,13 +189,16 @@ decode_update_kernel(RowState st, int which, int phase, int iter, const int32_t*
     }
   }
   const int n_ended = __syncthreads_count(ended);
-  if (threadIdx.x == 0) st.n_active[0] -= n_ended;
+  if (threadIdx.x == 0) {
+    st.n_active[0] -= n_ended;
+    st.iter[0] = iter + 1;
+  }
 }
 
-cudaError_t launch_decode_update(const RowState& st, int which, int phase, int iter, const int32_t* sampled,
+cudaError_t launch_decode_update(const RowState& st, int which, int phase, const int32_t* sampled,
                                  int n_slots, const LoopParams& lp, cudaStream_t s) {
   if (n_slots <= 0) return cudaSuccess;
-  decode_update_kernel<<<1, 1024, 0, s>>>(st, which, phase, iter, sampled, n_slots, lp);
+  decode_update_kernel<<<1, 1024, 0, s>>>(st, which, phase, sampled, n_slots, lp);
   return launched(1);
 }
 
