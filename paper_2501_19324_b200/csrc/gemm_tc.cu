@@ -100,7 +100,6 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
 #pragma unroll
   for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
-__device__ __forceinline__ void epilogue_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 // Shared-memory matrix descriptor of a K-major tile under the 128-byte swizzle: rows of 128 bytes,
 // groups of 8 rows 1024 bytes apart (stride byte offset), leading byte offset unused (1), version 1.
@@ -129,7 +128,7 @@ __global__ void __launch_bounds__(192, TcCfg<MT>::kCtasPerSm)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x,
                const __grid_constant__ CUtensorMap tm_x_lo, float* __restrict__ Y,
                int M, int N, int K, int accumulate, int splits, int kb_per_split, float* __restrict__ partials,
-               int* __restrict__ counters, int* __restrict__ err, const int32_t* __restrict__ n_active) {
+               int* __restrict__ err, const int32_t* __restrict__ n_active) {
   if (n_active != nullptr && *n_active == 0) return;
   using Cfg = TcCfg<MT>;
   constexpr int kRows = SPLIT ? MT / 2 : MT;   // distinct x rows per tile
@@ -139,7 +138,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
   uint64_t* empty = full + Cfg::kStages;
   uint64_t* tmem_full = empty + Cfg::kStages;
   uint32_t* tmem_slot = (uint32_t*)(tmem_full + 1);
-  volatile uint32_t* flags = tmem_slot + 1;   // [0] abort, [1] last-arriver flag
+  volatile uint32_t* flags = tmem_slot + 1;   // [0] abort
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n0 = blockIdx.x * kTileN, m0 = blockIdx.y * kRows, split = blockIdx.z;
@@ -219,10 +218,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
     const int n = n0 + n_local;
     const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16);
     const int m_valid = min(kRows, M - m0);
-    const int tile = blockIdx.y * gridDim.x + blockIdx.x;
-    const size_t tile_elems = (size_t)kTileN * kRows;
     if (ok) {
-      float* part = partials + ((size_t)split * gridDim.x * gridDim.y + tile) * tile_elems;
+      // with several K-splits each CTA stores its partial sums as rows of a [split][M][N] array;
+      // a reduction kernel adds the splits in order afterwards (deterministic)
+      float* dst = splits == 1 ? Y : partials + (size_t)split * M * N;
       for (int c = 0; c < m_valid; c += 16) {
         float v[16];
         tmem_ld16(taddr + c, v);
@@ -237,43 +236,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
             for (int j = 0; j < 16; ++j) v[j] += w[j];
           }
         }
-        if (splits == 1) {
-          if (n < N) {
+        if (n < N) {
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              if (c + j < m_valid) {
-                float* y = Y + (size_t)(m0 + c + j) * N + n;
-                *y = accumulate ? (*y + v[j]) : v[j];
-              }
+          for (int j = 0; j < 16; ++j) {
+            if (c + j < m_valid) {
+              float* y = dst + (size_t)(m0 + c + j) * N + n;
+              *y = (accumulate && splits == 1) ? (*y + v[j]) : v[j];
             }
           }
-        } else {
-#pragma unroll
-          for (int j = 0; j < 16; ++j)
-            if (c + j < m_valid) part[(size_t)(c + j) * kTileN + n_local] = v[j];
         }
-      }
-    }
-    if (splits > 1) {
-      __threadfence();
-      epilogue_barrier();
-      if (threadIdx.x == 0) {
-        const int old = atomicAdd(&counters[tile], 1);
-        flags[1] = (old == splits - 1) ? 1u : 0u;
-      }
-      epilogue_barrier();
-      if (flags[1]) {
-        __threadfence();
-        if (n < N && !flags[0]) {
-          for (int m = 0; m < m_valid; ++m) {
-            float sum = 0.f;
-            for (int sidx = 0; sidx < splits; ++sidx)
-              sum += __ldcg(partials + ((size_t)sidx * gridDim.x * gridDim.y + tile) * tile_elems + (size_t)m * kTileN + n_local);
-            float* y = Y + (size_t)(m0 + m) * N + n;
-            *y = accumulate ? (*y + sum) : sum;
-          }
-        }
-        if (threadIdx.x == 0) counters[tile] = 0;
       }
     }
   }
@@ -283,6 +254,33 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
     __syncwarp();
     tc_fence_after();
     tmem_dealloc(tmem_base, Cfg::kTmemCols);
+  }
+}
+
+// y[m, n] (+)= sum over splits of partials[s][m][n], splits added in order; 4 columns per thread.
+__global__ void __launch_bounds__(256)
+splitk_reduce_kernel(const float* __restrict__ partials, float* __restrict__ Y, int M, int N, int splits, int accumulate,
+                     const int32_t* __restrict__ n_active) {
+  if (n_active != nullptr && *n_active == 0) return;
+  const size_t total4 = (size_t)M * N / 4, stride = (size_t)M * N / 4;
+  const float4* p4 = reinterpret_cast<const float4*>(partials);
+  float4* y4 = reinterpret_cast<float4*>(Y);
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total4; i += (size_t)gridDim.x * blockDim.x) {
+    float4 acc = accumulate ? y4[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+    int sidx = 0;
+    for (; sidx + 4 <= splits; sidx += 4) {
+      const float4 a = __ldcg(p4 + (size_t)sidx * stride + i), b = __ldcg(p4 + (size_t)(sidx + 1) * stride + i);
+      const float4 c = __ldcg(p4 + (size_t)(sidx + 2) * stride + i), d = __ldcg(p4 + (size_t)(sidx + 3) * stride + i);
+      acc.x += a.x; acc.y += a.y; acc.z += a.z; acc.w += a.w;
+      acc.x += b.x; acc.y += b.y; acc.z += b.z; acc.w += b.w;
+      acc.x += c.x; acc.y += c.y; acc.z += c.z; acc.w += c.w;
+      acc.x += d.x; acc.y += d.y; acc.z += d.z; acc.w += d.w;
+    }
+    for (; sidx < splits; ++sidx) {
+      const float4 a = __ldcg(p4 + (size_t)sidx * stride + i);
+      acc.x += a.x; acc.y += a.y; acc.z += a.z; acc.w += a.w;
+    }
+    y4[i] = acc;
   }
 }
 
@@ -363,7 +361,7 @@ TcPlan plan_tc(int M, int N, int K, bool split_operand) {
   const int tiles = p.n_tiles * p.m_tiles;
   const int total_kb = (K + kTileK - 1) / kTileK;
   int splits = 1;
-  if (tiles < 148 && tiles <= kMaxSplitTiles && p.rows <= 64) {
+  if (tiles < 148 && tiles <= kMaxSplitTiles && p.rows <= 64 && N % 4 == 0) {
     // aim at one wave of two CTAs per SM, each with at least two k-blocks
     splits = std::max(1, (2 * 148) / tiles);
     splits = std::min(splits, std::max(1, total_kb / 2));
@@ -377,7 +375,7 @@ TcPlan plan_tc(int M, int N, int K, bool split_operand) {
 
 template <int MT, bool SPLIT>
 cudaError_t launch_mt(const CUtensorMap& tw, const CUtensorMap& tx, const CUtensorMap& txl, float* y, int M, int N, int K,
-                      int accumulate, const TcPlan& p, float* partials, int* counters, int* err, const int32_t* n_active,
+                      int accumulate, const TcPlan& p, float* partials, int* err, const int32_t* n_active,
                       cudaStream_t s) {
   static bool configured = false;
   if (!configured) {
@@ -387,7 +385,13 @@ cudaError_t launch_mt(const CUtensorMap& tw, const CUtensorMap& tx, const CUtens
   }
   dim3 grid(p.n_tiles, p.m_tiles, p.splits);
   gemm_tc_kernel<MT, SPLIT><<<grid, 192, TcCfg<MT>::kSmemBytes, s>>>(tw, tx, txl, y, M, N, K, accumulate, p.splits,
-                                                                     p.kb_per_split, partials, counters, err, n_active);
+                                                                     p.kb_per_split, partials, err, n_active);
+  if (p.splits > 1) {
+    const size_t total4 = (size_t)M * N / 4;
+    const int blocks = (int)std::min<size_t>((total4 + 255) / 256, 148 * 8);
+    splitk_reduce_kernel<<<blocks, 256, 0, s>>>(partials, y, M, N, p.splits, accumulate, n_active);
+    return launched(2);
+  }
   return launched(1);
 }
 
@@ -419,10 +423,9 @@ cudaError_t launch_gemm_tc(const void* W, const void* x, const void* x_lo, float
   if (!get_map(W, N, K, kTileN, &tw) || !get_map(x, M, K, p.rows, &tx)) return cudaErrorNotSupported;
   if (split_operand) { if (!get_map(x_lo, M, K, p.rows, &txl)) return cudaErrorNotSupported; }
   else txl = tx;
-  int* counters = (int*)scratch;
   int* err = (int*)((char*)scratch + kCounterBytes);
   float* partials = (float*)((char*)scratch + kCounterBytes + 256);
-#define RSD_TC(MT, SP) return launch_mt<MT, SP>(tw, tx, txl, y, M, N, K, accumulate, p, partials, counters, err, n_active, s)
+#define RSD_TC(MT, SP) return launch_mt<MT, SP>(tw, tx, txl, y, M, N, K, accumulate, p, partials, err, n_active, s)
   if (split_operand) {
     switch (p.mt) {
       case 16: RSD_TC(16, true);
