@@ -246,10 +246,11 @@ int rsd_k_swiglu(const float* gu, void* out, int32_t T, int32_t F, int32_t dtype
 /* token[b] = argmax over v < v_limit of logits[b, v] / T + g, g = -log(-log u) with u the Philox
  * uniform of (seed; counter = (v / 4, pos[b] + 1, row[b], model_id), word v % 4), or the plain
  * argmax when temperature == 0; ties to the lowest id.  pos[b] is the position of the token fed to
- * the model, the sampled token sits at pos[b] + 1.  row[b] < 0 skips slot b.  logits fp32 [B, V]. */
+ * the model, the sampled token sits at pos[b] + 1.  row[b] < 0 skips slot b.  logits fp32 [B, V].
+ * scratch: 8 * B bytes, 8-byte aligned (per-slot packed maxima the vocabulary chunks fold into).  */
 int rsd_k_sample(const float* logits, int32_t B, int32_t V, int32_t v_limit, float temperature,
                  uint64_t seed, int32_t model_id, const int32_t* row, const int32_t* pos, int32_t* token,
-                 void* cuda_stream);
+                 void* scratch, size_t scratch_bytes, void* cuda_stream);
 /* Philox4x32-10 blocks: out[i] = philox(ctr[i], key), ctr [n, 4], key [2], out [n, 4] (uint32). */
 int rsd_k_philox(const uint32_t* ctr, const uint32_t* key, uint32_t* out, int32_t n, void* cuda_stream);
 

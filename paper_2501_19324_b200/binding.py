@@ -98,7 +98,7 @@ def lib():
         L.rsd_k_rmsnorm.argtypes = [vp, vp, vp, c_int32, c_int32, c_float, c_int32, vp]
         L.rsd_k_rope.argtypes = [vp, vp, c_int32, c_int32, c_int32, c_float, vp]
         L.rsd_k_swiglu.argtypes = [vp, vp, c_int32, c_int32, c_int32, vp]
-        L.rsd_k_sample.argtypes = [vp, c_int32, c_int32, c_int32, c_float, c_uint64, c_int32, vp, vp, vp, vp]
+        L.rsd_k_sample.argtypes = [vp, c_int32, c_int32, c_int32, c_float, c_uint64, c_int32, vp, vp, vp, vp, c_size_t, vp]
         L.rsd_k_philox.argtypes = [vp, vp, vp, c_int32, vp]
         _lib = L
     return _lib
@@ -340,8 +340,9 @@ def k_sample(logits, v_limit, temperature, seed, model_id, row, pos):
     import torch
     B, V = logits.shape
     tok = torch.zeros(B, dtype=torch.int32, device=logits.device)
+    scratch = torch.zeros(B, dtype=torch.int64, device=logits.device)
     _check(lib().rsd_k_sample(_ptr(logits), B, V, v_limit, temperature, seed, model_id, _ptr(row), _ptr(pos), _ptr(tok),
-                              _stream()))
+                              _ptr(scratch), 8 * B, _stream()))
     return tok
 
 

@@ -56,7 +56,7 @@ struct rsd_ctx {
   float *x = nullptr, *qkv = nullptr, *q = nullptr, *gu = nullptr, *logits = nullptr;
   void *h = nullptr, *attn = nullptr, *act = nullptr;
   void *h_lo = nullptr, *attn_lo = nullptr, *act_lo = nullptr;   // low halves (bf16 models)
-  int32_t* sampled_slots = nullptr;
+  unsigned long long* sample_best = nullptr;   // packed sampling winners, one per slot
   float* dbg_logits[2] = {nullptr, nullptr};
   int32_t* d_scalars = nullptr;  // device block holding n_tok, n_rej, err, n_active, n_slots, next_page[3]
   // staging of step outputs (device) and their pinned host mirrors
@@ -208,7 +208,7 @@ size_t layout_workspace(const rsd_config& cfg, const rsd_model* const ms[3], rsd
   float* gu = TAKE(float, (size_t)T * 2 * dm.f);
   void* act = TAKE(float, (size_t)T * dm.f);
   float* logits = TAKE(float, (size_t)B * dm.v);
-  int32_t* sampled_slots = TAKE(int32_t, B);
+  unsigned long long* sample_best = TAKE(unsigned long long, B);
   float2* rope[3];
   for (int w = 0; w < 3; ++w) rope[w] = TAKE(float2, (size_t)S * (ms[w]->head_dim / 2));
   float* dbg[2] = {nullptr, nullptr};
@@ -235,7 +235,7 @@ size_t layout_workspace(const rsd_config& cfg, const rsd_model* const ms[3], rsd
     c->h_lo = (char*)h + (size_t)T * dm.d * 2;
     c->attn_lo = (char*)attn + (size_t)T * dm.hq * 2;
     c->act_lo = (char*)act + (size_t)T * dm.f * 2;
-    c->sampled_slots = sampled_slots;
+    c->sample_best = sample_best;
     for (int w = 0; w < 3; ++w) c->mdl[w].rope = rope[w];
     c->dbg_logits[0] = dbg[0]; c->dbg_logits[1] = dbg[1];
     c->d_scalars = scal;
@@ -291,15 +291,19 @@ int drain_gemm_events(rsd_ctx* c) {
   return RSD_OK;
 }
 
+// `pending` (nullable): the caller's next kernel adds up K-split partial sums itself, so the GEMM may
+// leave them in the scratch; *pending then describes them (splits == 1: y is complete).
 int gemm(rsd_ctx* c, const ModelHost& M, const void* W, const void* xin, const void* xin_lo, float* y, int Mrows, int N,
-         int K, int accumulate, const int32_t* n_active, cudaStream_t s) {
+         int K, int accumulate, const int32_t* n_active, SplitSum* pending, cudaStream_t s) {
   // ragged passes: every stride-th GEMM; decode: every GEMM of the iterations chosen by decode_phase
   const bool pick = c->in_decode ? c->time_this_iter
                                  : (c->time_stride > 0 && (c->gemm_calls++ % (uint64_t)c->time_stride) == 0);
   const bool timed = pick && c->ev_used < c->ev_bytes.size();
   if (timed) CU(cudaEventRecord(c->ev[2 * c->ev_used], s));
+  int splits = 1;
   CU(launch_gemm(M.m.dtype, W, xin, M.split ? xin_lo : nullptr, y, Mrows, N, K, accumulate, 0, c->gemm_scratch,
-                 c->gemm_scratch_bytes, n_active, s));
+                 c->gemm_scratch_bytes, n_active, pending ? &splits : nullptr, s));
+  if (pending) { pending->splits = splits; pending->partials = gemm_partials(c->gemm_scratch); }
   if (timed) {
     CU(cudaEventRecord(c->ev[2 * c->ev_used + 1], s));
     // algorithmic bytes: the weight matrix and the input once, the output once (twice when added to)
@@ -320,12 +324,18 @@ int forward_pass(rsd_ctx* c, int which, PassView p, cudaStream_t s) {
   void* h_lo = M.split ? c->h_lo : nullptr;
   void* attn_lo = M.split ? c->attn_lo : nullptr;
   void* act_lo = M.split ? c->act_lo : nullptr;
+  // K-split partial sums can be left for the consumer kernel to add up.  That pays where the
+  // consumer runs many blocks (SwiGLU); RMSNorm and RoPE run one block per token, too few to pull
+  // the partials in quickly, so those GEMMs reduce with their own kernel.
+  const bool defer_small = false;
+  SplitSum x_pending;   // partial sums of the last GEMM that adds into the residual stream
   for (int l = 0; l < m.n_layers; ++l) {
     KvView kv{M.kv_pool + (size_t)l * M.layer_stride, c->st.page_table[which], c->max_pages};
-    CU(launch_rmsnorm(m.dtype, c->x, M.norm1[l], c->h, h_lo, T, d, m.rms_eps, nullptr, p.n_active, s));
-    int rc = gemm(c, M, M.wqkv[l], c->h, h_lo, c->qkv, T, (H + 2 * KV) * hd, d, 0, p.n_active, s);
+    CU(launch_rmsnorm(m.dtype, c->x, M.norm1[l], c->h, h_lo, T, d, m.rms_eps, nullptr, p.n_active, x_pending, s));
+    SplitSum qkv_pending;
+    int rc = gemm(c, M, M.wqkv[l], c->h, h_lo, c->qkv, T, (H + 2 * KV) * hd, d, 0, p.n_active, defer_small ? &qkv_pending : nullptr, s);
     if (rc) return rc;
-    CU(launch_rope_kv(M.kv_dtype, c->qkv, p, c->q, kv, M.rope, H, KV, hd, s));
+    CU(launch_rope_kv(M.kv_dtype, c->qkv, qkv_pending, p, c->q, kv, M.rope, H, KV, hd, s));
     if (p.n_active != nullptr) {
       // decode pass: one query per row slot
       CU(launch_attn_decode(M.kv_dtype, c->q, kv.pool_layer, kv.page_table, kv.max_pages, p.tok_row, p.tok_pos, 1,
@@ -334,13 +344,17 @@ int forward_pass(rsd_ctx* c, int which, PassView p, cudaStream_t s) {
     } else {
       CU(launch_attn_chunk(M.kv_dtype, c->q, p, kv, c->attn, attn_lo, m.dtype, H, KV, hd, s));
     }
-    rc = gemm(c, M, M.wo[l], c->attn, attn_lo, c->x, T, d, H * hd, 1, p.n_active, s);
+    rc = gemm(c, M, M.wo[l], c->attn, attn_lo, c->x, T, d, H * hd, 1, p.n_active, defer_small ? &x_pending : nullptr, s);
     if (rc) return rc;
-    CU(launch_rmsnorm(m.dtype, c->x, M.norm2[l], c->h, h_lo, T, d, m.rms_eps, nullptr, p.n_active, s));
-    rc = gemm(c, M, M.wgu[l], c->h, h_lo, c->gu, T, 2 * F, d, 0, p.n_active, s);
+    CU(launch_rmsnorm(m.dtype, c->x, M.norm2[l], c->h, h_lo, T, d, m.rms_eps, nullptr, p.n_active, x_pending, s));
+    SplitSum gu_pending;
+    rc = gemm(c, M, M.wgu[l], c->h, h_lo, c->gu, T, 2 * F, d, 0, p.n_active, &gu_pending, s);
     if (rc) return rc;
-    CU(launch_swiglu(m.dtype, c->gu, c->act, act_lo, T, F, p.n_active, s));
-    rc = gemm(c, M, M.wdown[l], c->act, act_lo, c->x, T, d, F, 1, p.n_active, s);
+    CU(launch_swiglu(m.dtype, c->gu, gu_pending, c->act, act_lo, T, F, p.n_active, s));
+    // the last layer's result must be complete in x when the pass ends
+    const bool last = l + 1 == m.n_layers;
+    x_pending = SplitSum();
+    rc = gemm(c, M, M.wdown[l], c->act, act_lo, c->x, T, d, F, 1, p.n_active, (last || !defer_small) ? nullptr : &x_pending, s);
     if (rc) return rc;
   }
   return RSD_OK;
@@ -381,8 +395,8 @@ int decode_iteration(rsd_ctx* c, int which, int phase, int n_slots, cudaStream_t
   int rc = forward_pass(c, which, p, s);
   if (rc) return rc;
   CU(launch_rmsnorm(m.dtype, c->x, m.final_norm, c->h, M.split ? c->h_lo : nullptr, n_slots, m.d_model, m.rms_eps,
-                    nullptr, p.n_active, s));
-  rc = gemm(c, M, m.head, c->h, c->h_lo, c->logits, n_slots, m.vocab, m.d_model, 0, p.n_active, s);
+                    nullptr, p.n_active, SplitSum(), s));
+  rc = gemm(c, M, m.head, c->h, c->h_lo, c->logits, n_slots, m.vocab, m.d_model, 0, p.n_active, nullptr, s);
   if (rc) return rc;
   if (c->dbg_logits[phase]) {
     scatter_logits_kernel<<<n_slots, 256, 0, s>>>(c->logits, c->st.pass_tok_row, c->dbg_logits[phase], m.vocab, c->C,
@@ -390,9 +404,9 @@ int decode_iteration(rsd_ctx* c, int which, int phase, int n_slots, cudaStream_t
     CU(launched(1));
   }
   SampleArgs a{c->logits, n_slots, m.vocab, c->v_limit, c->cfg.temperature, c->cfg.seed, which,
-               c->st.pass_tok_row, c->st.pass_tok_pos, c->sampled_slots, c->st.n_active};
+               c->st.pass_tok_row, c->st.pass_tok_pos, nullptr, c->st.n_active, c->sample_best};
   CU(launch_sample(a, s));
-  CU(launch_decode_update(c->st, which, phase, c->sampled_slots, n_slots, c->lp, s));
+  CU(launch_decode_update(c->st, which, phase, c->sample_best, n_slots, c->lp, s));
   return RSD_OK;
 }
 
@@ -574,6 +588,7 @@ int rsd_load_models(rsd_ctx* c, const rsd_model* draft, const rsd_model* prm, co
     CU(launch_rope_table(c->mdl[w].rope, c->S, c->mdl[w].m.head_dim, c->mdl[w].m.rope_theta, s));
   CU(cudaMemsetAsync(c->d_scalars, 0, 16 * sizeof(int32_t), s));
   CU(cudaMemsetAsync(c->gemm_scratch, 0, c->gemm_scratch_bytes, s));
+  CU(cudaMemsetAsync(c->sample_best, 0, sizeof(unsigned long long) * c->B_max, s));
   int rc = clear_forcing(c, s);
   if (rc) return rc;
   CU(cudaStreamSynchronize(s));
@@ -866,7 +881,7 @@ int rsd_k_gemm(const void* W, const void* x, const void* x_lo, float* y, int32_t
   if (impl == 2 && !gemm_tc_supported(dtype, M, N, K)) return RSD_ERR_UNSUPPORTED;
   if (impl != 1 && (!scratch || scratch_bytes < gemm_scratch_bytes(M))) return RSD_ERR_ARG;
   if (x_lo && dtype != RSD_BF16) return RSD_ERR_ARG;
-  KCU(launch_gemm(dtype, W, x, x_lo, y, M, N, K, accumulate, impl, scratch, scratch_bytes, nullptr, (cudaStream_t)cuda_stream));
+  KCU(launch_gemm(dtype, W, x, x_lo, y, M, N, K, accumulate, impl, scratch, scratch_bytes, nullptr, nullptr, (cudaStream_t)cuda_stream));
   return RSD_OK;
 }
 
@@ -898,7 +913,7 @@ int rsd_k_gate_compact(const float* rewards, const uint8_t* live, float delta, u
 int rsd_k_rmsnorm(const float* x, const void* gain, void* out, int32_t T, int32_t d, float eps, int32_t dtype,
                   void* cuda_stream) {
   if (!x || !gain || !out || T < 0 || d < 4 || d % 4) return RSD_ERR_ARG;
-  KCU(launch_rmsnorm(dtype, x, gain, out, nullptr, T, d, eps, nullptr, nullptr, (cudaStream_t)cuda_stream));
+  KCU(launch_rmsnorm(dtype, const_cast<float*>(x), gain, out, nullptr, T, d, eps, nullptr, nullptr, SplitSum(), (cudaStream_t)cuda_stream));
   return RSD_OK;
 }
 
@@ -910,14 +925,17 @@ int rsd_k_rope(float* v, const int32_t* pos, int32_t T, int32_t n_heads, int32_t
 
 int rsd_k_swiglu(const float* gu, void* out, int32_t T, int32_t F, int32_t dtype, void* cuda_stream) {
   if (!gu || !out || T < 0 || F < 1) return RSD_ERR_ARG;
-  KCU(launch_swiglu(dtype, gu, out, nullptr, T, F, nullptr, (cudaStream_t)cuda_stream));
+  KCU(launch_swiglu(dtype, gu, SplitSum(), out, nullptr, T, F, nullptr, (cudaStream_t)cuda_stream));
   return RSD_OK;
 }
 
 int rsd_k_sample(const float* logits, int32_t B, int32_t V, int32_t v_limit, float temperature, uint64_t seed,
-                 int32_t model_id, const int32_t* row, const int32_t* pos, int32_t* token, void* cuda_stream) {
+                 int32_t model_id, const int32_t* row, const int32_t* pos, int32_t* token, void* scratch,
+                 size_t scratch_bytes, void* cuda_stream) {
   if (!logits || !row || !pos || !token || B < 1 || V < 1 || v_limit < 1 || v_limit > V || temperature < 0.f) return RSD_ERR_ARG;
-  SampleArgs a{logits, B, V, v_limit, temperature, seed, model_id, row, pos, token, nullptr};
+  if (!scratch || scratch_bytes < sizeof(unsigned long long) * (size_t)B || ((uintptr_t)scratch & 7)) return RSD_ERR_ARG;
+  KCU(cudaMemsetAsync(scratch, 0, sizeof(unsigned long long) * (size_t)B, (cudaStream_t)cuda_stream));
+  SampleArgs a{logits, B, V, v_limit, temperature, seed, model_id, row, pos, token, nullptr, (unsigned long long*)scratch};
   KCU(launch_sample(a, (cudaStream_t)cuda_stream));
   return RSD_OK;
 }

@@ -376,7 +376,7 @@ TcPlan plan_tc(int M, int N, int K, bool split_operand) {
 template <int MT, bool SPLIT>
 cudaError_t launch_mt(const CUtensorMap& tw, const CUtensorMap& tx, const CUtensorMap& txl, float* y, int M, int N, int K,
                       int accumulate, const TcPlan& p, float* partials, int* err, const int32_t* n_active,
-                      cudaStream_t s) {
+                      bool defer_reduce, cudaStream_t s) {
   static bool configured = false;
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<MT, SPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TcCfg<MT>::kSmemBytes);
@@ -386,7 +386,7 @@ cudaError_t launch_mt(const CUtensorMap& tw, const CUtensorMap& tx, const CUtens
   dim3 grid(p.n_tiles, p.m_tiles, p.splits);
   gemm_tc_kernel<MT, SPLIT><<<grid, 192, TcCfg<MT>::kSmemBytes, s>>>(tw, tx, txl, y, M, N, K, accumulate, p.splits,
                                                                      p.kb_per_split, partials, err, n_active);
-  if (p.splits > 1) {
+  if (p.splits > 1 && !defer_reduce) {
     const size_t total4 = (size_t)M * N / 4;
     const int blocks = (int)std::min<size_t>((total4 + 255) / 256, 148 * 8);
     splitk_reduce_kernel<<<blocks, 256, 0, s>>>(partials, y, M, N, p.splits, accumulate, n_active);
@@ -412,20 +412,26 @@ size_t gemm_scratch_bytes(int M) {
 // Enough for any M (split-K is only used with tiles of at most 64 rows of x).
 size_t gemm_scratch_bytes_any() { return gemm_scratch_bytes(64); }
 
+const float* gemm_partials(const void* scratch) { return (const float*)((const char*)scratch + kCounterBytes + 256); }
+
 cudaError_t launch_gemm_tc(const void* W, const void* x, const void* x_lo, float* y, int M, int N, int K, int accumulate,
-                           void* scratch, size_t scratch_bytes, const int32_t* n_active, cudaStream_t s) {
+                           void* scratch, size_t scratch_bytes, const int32_t* n_active, int* deferred_splits,
+                           cudaStream_t s) {
+  if (deferred_splits) *deferred_splits = 1;
   if (M <= 0) return cudaSuccess;
   if (!scratch || scratch_bytes < gemm_scratch_bytes(M)) return cudaErrorInvalidValue;
   if (((uintptr_t)W & 15) || ((uintptr_t)x & 15) || ((uintptr_t)x_lo & 15)) return cudaErrorMisalignedAddress;
   const bool split_operand = x_lo != nullptr;
   const TcPlan p = plan_tc(M, N, K, split_operand);
+  if (deferred_splits) *deferred_splits = p.splits;
+  const bool defer = deferred_splits != nullptr;
   CUtensorMap tw, tx, txl;
   if (!get_map(W, N, K, kTileN, &tw) || !get_map(x, M, K, p.rows, &tx)) return cudaErrorNotSupported;
   if (split_operand) { if (!get_map(x_lo, M, K, p.rows, &txl)) return cudaErrorNotSupported; }
   else txl = tx;
   int* err = (int*)((char*)scratch + kCounterBytes);
   float* partials = (float*)((char*)scratch + kCounterBytes + 256);
-#define RSD_TC(MT, SP) return launch_mt<MT, SP>(tw, tx, txl, y, M, N, K, accumulate, p, partials, err, n_active, s)
+#define RSD_TC(MT, SP) return launch_mt<MT, SP>(tw, tx, txl, y, M, N, K, accumulate, p, partials, err, n_active, defer, s)
   if (split_operand) {
     switch (p.mt) {
       case 16: RSD_TC(16, true);
@@ -447,10 +453,11 @@ cudaError_t launch_gemm_tc(const void* W, const void* x, const void* x_lo, float
 
 cudaError_t launch_gemm(int dtype, const void* W, const void* x, const void* x_lo, float* y, int M, int N, int K,
                         int accumulate, int impl, void* scratch, size_t scratch_bytes, const int32_t* n_active,
-                        cudaStream_t s) {
+                        int* deferred_splits, cudaStream_t s) {
+  if (deferred_splits) *deferred_splits = 1;
   const bool tc_ok = gemm_tc_supported(dtype, M, N, K) && scratch && scratch_bytes >= gemm_scratch_bytes(M);
   if (impl == 2 || (impl == 0 && tc_ok && M > 4))
-    return launch_gemm_tc(W, x, x_lo, y, M, N, K, accumulate, scratch, scratch_bytes, n_active, s);
+    return launch_gemm_tc(W, x, x_lo, y, M, N, K, accumulate, scratch, scratch_bytes, n_active, deferred_splits, s);
   return launch_gemm_simt(dtype, W, x, dtype == 1 ? x_lo : nullptr, y, M, N, K, accumulate, n_active, s);
 }
 

@@ -17,6 +17,12 @@ void note_replayed_launches(uint64_t n);   // kernels run by replaying a capture
 constexpr int kPageTokens = 16;   // tokens per KV page
 constexpr int kMaxBatch = 1024;   // rows per context (one thread per row in the state kernels)
 
+// A GEMM result that may still be spread over K-split partial sums: value = y (+) sum_s partials[s].
+struct SplitSum {
+  const float* partials = nullptr;
+  int splits = 1;
+};
+
 // A pass pushes T token slots through one model.  Slot t carries token tok_id[t] of row tok_row[t]
 // at position tok_pos[t]; tok_row[t] < 0 marks an idle slot.  When n_active is non-null and reads
 // 0 on the device the whole pass is skipped (every row of the decode phase has finished).
@@ -39,8 +45,9 @@ struct KvView {
 cudaError_t launch_embed(int dtype, const void* embed, PassView p, float* x, int d, cudaStream_t s);
 // out[t] = rmsnorm(x[src ? src[t] : t]); rows with src[t] < 0 are skipped.
 // out (and out_lo when given, bf16 only: the low half of a split-precision operand)
-cudaError_t launch_rmsnorm(int dtype, const float* x, const void* gain, void* out, void* out_lo, int T, int d, float eps,
-                           const int32_t* src, const int32_t* n_active, cudaStream_t s);
+// pending (splits > 1): x[t] += sum of the partial sums [splits][T][d] first (x is written back).
+cudaError_t launch_rmsnorm(int dtype, float* x, const void* gain, void* out, void* out_lo, int T, int d, float eps,
+                           const int32_t* src, const int32_t* n_active, SplitSum pending, cudaStream_t s);
 // x_lo (nullable, bf16 only): second operand matrix added to x (split-precision activations).
 cudaError_t launch_gemm_simt(int dtype, const void* W, const void* x, const void* x_lo, float* y, int M, int N, int K,
                              int accumulate, const int32_t* n_active, cudaStream_t s);
@@ -49,16 +56,23 @@ cudaError_t launch_gemm_simt(int dtype, const void* W, const void* x, const void
 bool gemm_tc_supported(int dtype, int M, int N, int K);
 size_t gemm_scratch_bytes(int M);
 size_t gemm_scratch_bytes_any();
+// deferred_splits (nullable): when given, a K-split launch leaves its partial sums in the scratch as
+// [splits][M][N] (gemm_partials) for the consumer kernel to add up, and reports the split count;
+// 1 means y holds the finished result.
 cudaError_t launch_gemm_tc(const void* W, const void* x, const void* x_lo, float* y, int M, int N, int K, int accumulate,
-                           void* scratch, size_t scratch_bytes, const int32_t* n_active, cudaStream_t s);
+                           void* scratch, size_t scratch_bytes, const int32_t* n_active, int* deferred_splits,
+                           cudaStream_t s);
+const float* gemm_partials(const void* scratch);
+
 // impl: 0 = by shape, 1 = SIMT split-K GEMV, 2 = tcgen05.
 cudaError_t launch_gemm(int dtype, const void* W, const void* x, const void* x_lo, float* y, int M, int N, int K,
                         int accumulate, int impl, void* scratch, size_t scratch_bytes, const int32_t* n_active,
-                        cudaStream_t s);
+                        int* deferred_splits, cudaStream_t s);
 cudaError_t launch_rope_table(float2* table, int n_pos, int hd, float theta, cudaStream_t s);
 // Splits qkv [T, (H+2KV)*hd] (fp32): rotated q -> q_out [T, H*hd] fp32; rotated k and v -> KV pages.
 // kv_dtype: element type of the cache: 0 fp32, 1 bf16, 2 fp16.
-cudaError_t launch_rope_kv(int kv_dtype, const float* qkv, PassView p, float* q_out, KvView kv, const float2* rope,
+// pending (splits > 1): qkv is the sum of the partial sums instead of the qkv array.
+cudaError_t launch_rope_kv(int kv_dtype, const float* qkv, SplitSum pending, PassView p, float* q_out, KvView kv, const float2* rope,
                            int H, int KV, int hd, cudaStream_t s);
 cudaError_t launch_rope_only(float* v, const int32_t* pos, int T, int n_heads, int hd, float theta, cudaStream_t s);
 // Causal attention of every slot over positions [0, tok_pos] of its row, read from the pages.
@@ -67,8 +81,8 @@ cudaError_t launch_attn_generic(int kv_dtype, const float* q, PassView p, KvView
 // Tensor-core version of the above for 16-bit caches with H / KV <= 8 (falls back otherwise).
 cudaError_t launch_attn_chunk(int kv_dtype, const float* q, PassView p, KvView kv, void* out, void* out_lo,
                               int out_dtype, int H, int KV, int hd, cudaStream_t s);
-cudaError_t launch_swiglu(int dtype, const float* gu, void* out, void* out_lo, int T, int F, const int32_t* n_active,
-                          cudaStream_t s);
+cudaError_t launch_swiglu(int dtype, const float* gu, SplitSum pending, void* out, void* out_lo, int T, int F,
+                          const int32_t* n_active, cudaStream_t s);
 
 // Decode attention (one query per row) with split-KV partial results merged in a second pass.
 size_t attn_decode_scratch_bytes(int B, int H, int hd, int max_ctx);
@@ -87,8 +101,9 @@ struct SampleArgs {
   int model_id;
   const int32_t* slot_row;     // row id per slot (noise key); < 0 = idle slot
   const int32_t* slot_pos;     // position of the slot's input token; the new token sits at +1
-  int32_t* token;              // [n_slots] out
+  int32_t* token;              // [n_slots] out; null = leave the packed winners in `best`
   const int32_t* n_active;
+  unsigned long long* best;    // [n_slots] scratch, zero on entry: packed (score, id) maxima
 };
 cudaError_t launch_sample(const SampleArgs& a, cudaStream_t s);
 cudaError_t launch_philox(const uint32_t* ctr, const uint32_t* key, uint32_t* out, int n, cudaStream_t s);
@@ -139,7 +154,8 @@ cudaError_t launch_reserve_pages(const RowState& st, int which, ReserveMode mode
 cudaError_t launch_build_pass(const RowState& st, int which, PassMode mode, cudaStream_t s);
 cudaError_t launch_decode_begin(const RowState& st, int phase, cudaStream_t s);
 cudaError_t launch_decode_prepare(const RowState& st, int which, int n_slots, cudaStream_t s);
-cudaError_t launch_decode_update(const RowState& st, int which, int phase, const int32_t* sampled,
+// best: packed winners left by launch_sample (cleared here).
+cudaError_t launch_decode_update(const RowState& st, int which, int phase, unsigned long long* best,
                                  int n_slots, const LoopParams& lp, cudaStream_t s);
 cudaError_t launch_gate(const RowState& st, float delta, const LoopParams& lp, cudaStream_t s);
 cudaError_t launch_commit(const RowState& st, const LoopParams& lp, int32_t* out_tokens, int32_t* out_len,

@@ -39,9 +39,9 @@ cudaError_t launch_embed(int dtype, const void* embed, PassView p, float* x, int
 // RMSNorm: out = x * gain / sqrt(mean(x^2) + eps), one block per token, x kept in registers
 // ---------------------------------------------------------------------------------------------
 template <typename OT, typename GT>
-__global__ void rmsnorm_kernel(const float* __restrict__ x, const GT* __restrict__ gain, OT* __restrict__ out,
+__global__ void rmsnorm_kernel(float* __restrict__ x, const GT* __restrict__ gain, OT* __restrict__ out,
                                OT* __restrict__ out_lo, int d, float eps, const int32_t* __restrict__ src,
-                               const int32_t* n_active) {
+                               const int32_t* n_active, const float* __restrict__ partials, int splits, int T) {
   RSD_SKIP_IF_IDLE(n_active);
   __shared__ float red[33];
   const int t = blockIdx.x;
@@ -50,10 +50,26 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, const GT* __restrict
     st = src[t];
     if (st < 0) return;
   }
-  const float* xr = x + (size_t)st * d;
+  float* xr = x + (size_t)st * d;
   float ss = 0.f;
   for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) {
     float4 v = *reinterpret_cast<const float4*>(xr + i);
+    if (splits > 1) {
+      // the producing GEMM left K-split partial sums: fold them into the residual stream here
+      int sidx = 0;
+      for (; sidx + 8 <= splits; sidx += 8) {
+        float4 a[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) a[u] = __ldcg(reinterpret_cast<const float4*>(partials + ((size_t)(sidx + u) * T + st) * d + i));
+#pragma unroll
+        for (int u = 0; u < 8; ++u) { v.x += a[u].x; v.y += a[u].y; v.z += a[u].z; v.w += a[u].w; }
+      }
+      for (; sidx < splits; ++sidx) {
+        const float4 a = __ldcg(reinterpret_cast<const float4*>(partials + ((size_t)sidx * T + st) * d + i));
+        v.x += a.x; v.y += a.y; v.z += a.z; v.w += a.w;
+      }
+      *reinterpret_cast<float4*>(xr + i) = v;
+    }
     ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
   }
   ss = block_sum(ss, red);
@@ -68,14 +84,14 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, const GT* __restrict
   }
 }
 
-cudaError_t launch_rmsnorm(int dtype, const float* x, const void* gain, void* out, void* out_lo, int T, int d, float eps,
-                           const int32_t* src, const int32_t* n_active, cudaStream_t s) {
+cudaError_t launch_rmsnorm(int dtype, float* x, const void* gain, void* out, void* out_lo, int T, int d, float eps,
+                           const int32_t* src, const int32_t* n_active, SplitSum pending, cudaStream_t s) {
   if (T <= 0) return cudaSuccess;
   const int threads = d >= 2048 ? 512 : 256;
   if (dtype == 1)
-    rmsnorm_kernel<__nv_bfloat16, __nv_bfloat16><<<T, threads, 0, s>>>(x, (const __nv_bfloat16*)gain, (__nv_bfloat16*)out, (__nv_bfloat16*)out_lo, d, eps, src, n_active);
+    rmsnorm_kernel<__nv_bfloat16, __nv_bfloat16><<<T, threads, 0, s>>>(x, (const __nv_bfloat16*)gain, (__nv_bfloat16*)out, (__nv_bfloat16*)out_lo, d, eps, src, n_active, pending.partials, pending.splits, T);
   else
-    rmsnorm_kernel<float, float><<<T, threads, 0, s>>>(x, (const float*)gain, (float*)out, nullptr, d, eps, src, n_active);
+    rmsnorm_kernel<float, float><<<T, threads, 0, s>>>(x, (const float*)gain, (float*)out, nullptr, d, eps, src, n_active, pending.partials, pending.splits, T);
   return launched(1);
 }
 
@@ -183,8 +199,26 @@ cudaError_t launch_rope_table(float2* table, int n_pos, int hd, float theta, cud
 // RoPE on q and k, KV page write.  One block per token slot; threads walk the (head, pair) grid.
 // Pair (i, i + hd/2) of a head turns by the angle of (position, i).
 // ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ float split_sum(const float* __restrict__ direct, const float* __restrict__ partials, int splits,
+                                           size_t idx, size_t stride) {
+  if (splits <= 1) return direct[idx];
+  // loads go out eight at a time so their latencies overlap; the sums stay in split order
+  float v = 0.f;
+  int sidx = 0;
+  for (; sidx + 8 <= splits; sidx += 8) {
+    float t[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) t[u] = __ldcg(partials + (size_t)(sidx + u) * stride + idx);
+#pragma unroll
+    for (int u = 0; u < 8; ++u) v += t[u];
+  }
+  for (; sidx < splits; ++sidx) v += __ldcg(partials + (size_t)sidx * stride + idx);
+  return v;
+}
+
 template <typename KT>
-__global__ void rope_kv_kernel(const float* __restrict__ qkv, PassView p, float* __restrict__ q_out, KT* pool,
+__global__ void rope_kv_kernel(const float* __restrict__ qkv, const float* __restrict__ partials, int splits,
+                               PassView p, float* __restrict__ q_out, KT* pool,
                                const int32_t* __restrict__ page_table, int max_pages,
                                const float2* __restrict__ rope, int H, int KV, int hd) {
   RSD_SKIP_IF_IDLE(p.n_active);
@@ -193,7 +227,9 @@ __global__ void rope_kv_kernel(const float* __restrict__ qkv, PassView p, float*
   if (row < 0) return;
   const int pos = p.tok_pos[t];
   const int half = hd / 2;
-  const float* src = qkv + (size_t)t * (H + 2 * KV) * hd;
+  const int width = (H + 2 * KV) * hd;
+  const size_t src0 = (size_t)t * width;                 // offset of this token's row in qkv / a partial
+  const size_t sstride = (size_t)gridDim.x * width;      // one partial array = [T][width]
   const float2* cs = rope + (size_t)pos * half;
   const int page = page_table[(size_t)row * max_pages + pos / kPageTokens];
   const int slot = pos % kPageTokens;
@@ -203,7 +239,8 @@ __global__ void rope_kv_kernel(const float* __restrict__ qkv, PassView p, float*
   const int n_rot = (H + KV) * half;
   for (int idx = threadIdx.x; idx < n_rot; idx += blockDim.x) {
     const int head = idx / half, i = idx % half;
-    const float a = src[head * hd + i], b = src[head * hd + i + half];
+    const float a = split_sum(qkv, partials, splits, src0 + head * hd + i, sstride);
+    const float b = split_sum(qkv, partials, splits, src0 + head * hd + i + half, sstride);
     const float2 c = cs[i];
     const float ra = a * c.x - b * c.y, rb = b * c.x + a * c.y;
     if (head < H) {
@@ -215,22 +252,22 @@ __global__ void rope_kv_kernel(const float* __restrict__ qkv, PassView p, float*
       k[i + half] = from_f32<KT>(rb);
     }
   }
-  const float* vsrc = src + (H + KV) * hd;
   for (int idx = threadIdx.x; idx < KV * hd; idx += blockDim.x) {
     const int head = idx / hd, i = idx % hd;
-    vbase[((size_t)head * hd + i) * kPageTokens + slot] = from_f32<KT>(vsrc[idx]);
+    const float v = split_sum(qkv, partials, splits, src0 + (H + KV) * hd + idx, sstride);
+    vbase[((size_t)head * hd + i) * kPageTokens + slot] = from_f32<KT>(v);
   }
 }
 
-cudaError_t launch_rope_kv(int kv_dtype, const float* qkv, PassView p, float* q_out, KvView kv, const float2* rope,
-                           int H, int KV, int hd, cudaStream_t s) {
+cudaError_t launch_rope_kv(int kv_dtype, const float* qkv, SplitSum pending, PassView p, float* q_out, KvView kv,
+                           const float2* rope, int H, int KV, int hd, cudaStream_t s) {
   if (p.T <= 0) return cudaSuccess;
   if (kv_dtype == 2)
-    rope_kv_kernel<__half><<<p.T, 256, 0, s>>>(qkv, p, q_out, (__half*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd);
+    rope_kv_kernel<__half><<<p.T, 256, 0, s>>>(qkv, pending.partials, pending.splits, p, q_out, (__half*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd);
   else if (kv_dtype == 1)
-    rope_kv_kernel<__nv_bfloat16><<<p.T, 256, 0, s>>>(qkv, p, q_out, (__nv_bfloat16*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd);
+    rope_kv_kernel<__nv_bfloat16><<<p.T, 256, 0, s>>>(qkv, pending.partials, pending.splits, p, q_out, (__nv_bfloat16*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd);
   else
-    rope_kv_kernel<float><<<p.T, 256, 0, s>>>(qkv, p, q_out, (float*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd);
+    rope_kv_kernel<float><<<p.T, 256, 0, s>>>(qkv, pending.partials, pending.splits, p, q_out, (float*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd);
   return launched(1);
 }
 
@@ -344,25 +381,27 @@ cudaError_t launch_attn_generic(int kv_dtype, const float* q, PassView p, KvView
 // SwiGLU: out[t, f] = silu(gu[t, f]) * gu[t, F + f]
 // ---------------------------------------------------------------------------------------------
 template <typename OT>
-__global__ void swiglu_kernel(const float* __restrict__ gu, OT* __restrict__ out, OT* __restrict__ out_lo, int T, int F,
-                              const int32_t* n_active) {
+__global__ void swiglu_kernel(const float* __restrict__ gu, const float* __restrict__ partials, int splits,
+                              OT* __restrict__ out, OT* __restrict__ out_lo, int T, int F, const int32_t* n_active) {
   RSD_SKIP_IF_IDLE(n_active);
   const size_t n = (size_t)T * F;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
     const size_t t = i / F, f = i % F;
-    const float a = gu[t * 2 * F + f], b = gu[t * 2 * F + F + f];
+    const size_t sstride = (size_t)T * 2 * F;
+    const float a = split_sum(gu, partials, splits, t * 2 * F + f, sstride);
+    const float b = split_sum(gu, partials, splits, t * 2 * F + F + f, sstride);
     store_operand<OT>(out, out_lo, i, a / (1.f + expf(-a)) * b);
   }
 }
 
-cudaError_t launch_swiglu(int dtype, const float* gu, void* out, void* out_lo, int T, int F, const int32_t* n_active,
-                          cudaStream_t s) {
+cudaError_t launch_swiglu(int dtype, const float* gu, SplitSum pending, void* out, void* out_lo, int T, int F,
+                          const int32_t* n_active, cudaStream_t s) {
   if (T <= 0) return cudaSuccess;
   const size_t n = (size_t)T * F;
   int blocks = (int)((n + 255) / 256);
   if (blocks > 148 * 8) blocks = 148 * 8;
-  if (dtype == 1) swiglu_kernel<__nv_bfloat16><<<blocks, 256, 0, s>>>(gu, (__nv_bfloat16*)out, (__nv_bfloat16*)out_lo, T, F, n_active);
-  else swiglu_kernel<float><<<blocks, 256, 0, s>>>(gu, (float*)out, nullptr, T, F, n_active);
+  if (dtype == 1) swiglu_kernel<__nv_bfloat16><<<blocks, 256, 0, s>>>(gu, pending.partials, pending.splits, (__nv_bfloat16*)out, (__nv_bfloat16*)out_lo, T, F, n_active);
+  else swiglu_kernel<float><<<blocks, 256, 0, s>>>(gu, pending.partials, pending.splits, (float*)out, nullptr, T, F, n_active);
   return launched(1);
 }
 
@@ -374,6 +413,16 @@ __device__ __forceinline__ void better(float& bs, int& bi, float s, int i) {
   if (s > bs || (s == bs && i < bi)) { bs = s; bi = i; }
 }
 
+// (score, id) packed so that an unsigned 64-bit maximum picks the highest score and, among equal
+// scores, the lowest id: high word = order-preserving image of the float, low word = ~id.
+__device__ __forceinline__ unsigned long long pack_best(float sc, int id) {
+  const uint32_t b = __float_as_uint(sc);
+  const uint32_t key = (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+  return ((unsigned long long)key << 32) | (uint32_t)(0xFFFFFFFFu - (uint32_t)id);
+}
+
+// Grid (slots, chunks): every block scans one chunk of the vocabulary and folds its best candidate
+// into best[slot] with an atomic maximum (order-independent, hence deterministic).
 __global__ void __launch_bounds__(1024) sample_kernel(SampleArgs a) {
   RSD_SKIP_IF_IDLE(a.n_active);
   __shared__ float s_sc[32];
@@ -387,7 +436,10 @@ __global__ void __launch_bounds__(1024) sample_kernel(SampleArgs a) {
   const float inv_t = a.temperature > 0.f ? 1.f / a.temperature : 1.f;
   float bs = -INFINITY;
   int bi = 0x7FFFFFFF;
-  for (int v4 = threadIdx.x; v4 * 4 < a.v_limit; v4 += blockDim.x) {
+  const int n_v4 = (a.v_limit + 3) / 4;
+  const int per_chunk = (n_v4 + gridDim.y - 1) / gridDim.y;
+  const int v4_end = min(n_v4, (int)(blockIdx.y + 1) * per_chunk);
+  for (int v4 = blockIdx.y * per_chunk + threadIdx.x; v4 < v4_end; v4 += blockDim.x) {
     float g[4] = {0.f, 0.f, 0.f, 0.f};
     if (a.temperature > 0.f) {
       const uint4 r = philox4x32_10(make_uint4((uint32_t)v4, position, (uint32_t)row, (uint32_t)a.model_id), key);
@@ -420,15 +472,29 @@ __global__ void __launch_bounds__(1024) sample_kernel(SampleArgs a) {
       const int oi = __shfl_xor_sync(0xFFFFFFFFu, bi, o);
       better(bs, bi, os, oi);
     }
-    if (lane == 0) a.token[slot] = bi;
+    if (lane == 0 && bi != 0x7FFFFFFF) atomicMax(a.best + slot, pack_best(bs, bi));
   }
 }
 
+// token[slot] = id held in best[slot]; best is cleared for the next use.
+__global__ void sample_finalize_kernel(unsigned long long* best, const int32_t* slot_row, int32_t* token, int n) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  if (slot_row[i] >= 0) token[i] = (int32_t)(0xFFFFFFFFu - (uint32_t)(best[i] & 0xFFFFFFFFull));
+  best[i] = 0ull;
+}
+
+int sample_chunks(int v_limit) { return v_limit >= 65536 ? 16 : (v_limit >= 8192 ? 4 : 1); }
+
+// Leaves the winners packed in a.best (which must be zero on entry); when a.token is given a second
+// kernel unpacks them into a.token and clears a.best.
 cudaError_t launch_sample(const SampleArgs& a, cudaStream_t s) {
   if (a.n_slots <= 0) return cudaSuccess;
   const int threads = a.v_limit >= 16384 ? 1024 : 256;
-  sample_kernel<<<a.n_slots, threads, 0, s>>>(a);
-  return launched(1);
+  sample_kernel<<<dim3(a.n_slots, sample_chunks(a.v_limit)), threads, 0, s>>>(a);
+  if (a.token == nullptr) return launched(1);
+  sample_finalize_kernel<<<(a.n_slots + 255) / 256, 256, 0, s>>>(a.best, a.slot_row, a.token, a.n_slots);
+  return launched(2);
 }
 
 __global__ void philox_kernel(const uint32_t* ctr, const uint32_t* key, uint32_t* out, int n) {

@@ -165,15 +165,18 @@ __device__ __forceinline__ bool ends_step(int t, const LoopParams& lp) {
 
 // Appends the current iteration's token of every active slot to its row and stops rows whose step ended.
 __global__ void __launch_bounds__(1024)
-decode_update_kernel(RowState st, int which, int phase, const int32_t* sampled, int n_slots, LoopParams lp) {
+decode_update_kernel(RowState st, int which, int phase, unsigned long long* best, int n_slots, LoopParams lp) {
   if (st.n_active[0] == 0) return;
   const int iter = st.iter[0];   // iteration of the current decode phase, kept on the device
   const int i = threadIdx.x;
   int ended = 0;
   if (i < n_slots) {
     const int row = st.pass_tok_row[i];
+    const unsigned long long packed = best[i];
+    best[i] = 0ull;
     if (row >= 0) {
-      int t = sampled[i];
+      // packed == 0: no candidate was comparable (all scores NaN); fall back to id 0
+      int t = packed ? (int)(0xFFFFFFFFu - (uint32_t)(packed & 0xFFFFFFFFull)) : 0;
       st.sampled[phase][(size_t)row * st.C + iter] = t;
       const int flen = st.forced_len[phase][row];
       if (flen > 0) t = st.forced_tok[phase][(size_t)row * st.C + iter];
@@ -195,10 +198,10 @@ decode_update_kernel(RowState st, int which, int phase, const int32_t* sampled, 
   }
 }
 
-cudaError_t launch_decode_update(const RowState& st, int which, int phase, const int32_t* sampled,
+cudaError_t launch_decode_update(const RowState& st, int which, int phase, unsigned long long* best,
                                  int n_slots, const LoopParams& lp, cudaStream_t s) {
   if (n_slots <= 0) return cudaSuccess;
-  decode_update_kernel<<<1, 1024, 0, s>>>(st, which, phase, sampled, n_slots, lp);
+  decode_update_kernel<<<1, 1024, 0, s>>>(st, which, phase, best, n_slots, lp);
   return launched(1);
 }
 
