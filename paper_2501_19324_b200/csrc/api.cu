@@ -8,6 +8,7 @@
 #include <string>
 #include <vector>
 
+#include "common.cuh"
 #include "kernels.cuh"
 
 using namespace rsd;
@@ -378,6 +379,7 @@ int run_ingest(rsd_ctx* c, int which, int n_total, bool want_reward, cudaStream_
 
 __global__ void scatter_logits_kernel(const float* logits, const int32_t* slot_row, float* dbg, int V, int C,
                                       const int32_t* iter, const int32_t* n_active) {
+  RSD_PDL_SYNC();
   if (*n_active == 0) return;
   const int row = slot_row[blockIdx.x];
   if (row < 0) return;
@@ -399,7 +401,7 @@ int decode_iteration(rsd_ctx* c, int which, int phase, int n_slots, cudaStream_t
   rc = gemm(c, M, m.head, c->h, c->h_lo, c->logits, n_slots, m.vocab, m.d_model, 0, p.n_active, nullptr, s);
   if (rc) return rc;
   if (c->dbg_logits[phase]) {
-    scatter_logits_kernel<<<n_slots, 256, 0, s>>>(c->logits, c->st.pass_tok_row, c->dbg_logits[phase], m.vocab, c->C,
+    RSD_LAUNCH((scatter_logits_kernel), n_slots, 256, 0, s, c->logits, c->st.pass_tok_row, c->dbg_logits[phase], m.vocab, c->C,
                                                   c->st.iter, c->st.n_active);
     CU(launched(1));
   }
@@ -473,6 +475,7 @@ int decode_phase(rsd_ctx* c, int which, int phase, int n_slots, cudaStream_t s) 
 }
 
 __global__ void init_rows_kernel(RowState st, const int32_t* flat, const int32_t* offsets, int B) {
+  RSD_PDL_SYNC();
   const int b = blockIdx.x;
   const int o = offsets[b], n = offsets[b + 1] - o;
   for (int i = threadIdx.x; i < n; i += blockDim.x) st.tok[(size_t)b * st.S + i] = flat[o + i];
@@ -629,7 +632,7 @@ int rsd_prefill(rsd_ctx* c, const int32_t* tokens, const int32_t* offsets, int32
   // stage the ragged prompt in the pass-list buffers, then scatter it into the row buffers
   CU(cudaMemcpyAsync(c->st.pass_tok_id, tokens, sizeof(int32_t) * total, cudaMemcpyHostToDevice, s));
   CU(cudaMemcpyAsync(c->st.pass_tok_row, offsets, sizeof(int32_t) * (B + 1), cudaMemcpyHostToDevice, s));
-  init_rows_kernel<<<B, 128, 0, s>>>(c->st, c->st.pass_tok_id, c->st.pass_tok_row, B);
+  RSD_LAUNCH((init_rows_kernel), B, 128, 0, s, c->st, c->st.pass_tok_id, c->st.pass_tok_row, B);
   CU(launched(1));
   CU(cudaStreamSynchronize(s));  // the staging buffers are reused below
   CU(launch_reserve_pages(c->st, RSD_DRAFT, kReservePrefillDraft, s));

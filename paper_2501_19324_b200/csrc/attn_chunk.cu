@@ -48,6 +48,7 @@ template <int HD, typename KT, typename OT>
 __global__ void __launch_bounds__(256)
 attn_chunk_kernel(const float* __restrict__ q, PassView p, const KT* __restrict__ pool, const int32_t* __restrict__ page_table,
                   int max_pages, OT* __restrict__ out, OT* __restrict__ out_lo, int H, int KV) {
+  RSD_PDL_SYNC();
   constexpr int KB = HD / 32, NT = HD / 8;
   const int G = H / KV;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -174,7 +175,7 @@ cudaError_t launch_attn_chunk(int kv_dtype, const float* q, PassView p, KvView k
   dim3 grid((p.T + 15) / 16, KV);
   const int threads = 32 * G;
 #define RSD_CH(HD, KT, OT) \
-  attn_chunk_kernel<HD, KT, OT><<<grid, threads, 0, s>>>(q, p, (const KT*)kv.pool_layer, kv.page_table, kv.max_pages, (OT*)out, (OT*)out_lo, H, KV)
+  RSD_LAUNCH((attn_chunk_kernel<HD, KT, OT>), grid, threads, 0, s, q, p, (const KT*)kv.pool_layer, kv.page_table, kv.max_pages, (OT*)out, (OT*)out_lo, H, KV)
 #define RSD_CH_O(HD, KT) do { if (out_dtype == 1) RSD_CH(HD, KT, __nv_bfloat16); else RSD_CH(HD, KT, float); } while (0)
   if (kv_dtype == 2) { if (hd == 128) RSD_CH_O(128, __half); else RSD_CH_O(64, __half); }
   else { if (hd == 128) RSD_CH_O(128, __nv_bfloat16); else RSD_CH_O(64, __nv_bfloat16); }

@@ -57,6 +57,7 @@ attn_decode_kernel(const float* __restrict__ q, const KT* __restrict__ pool, con
                    int max_pages, const int32_t* __restrict__ slot_row, const int32_t* __restrict__ len_or_pos, int len_offset,
                    OT* __restrict__ out, OT* __restrict__ out_lo, float* __restrict__ part_o, float* __restrict__ part_ml, int H, int KV, int n_splits,
                    const int32_t* __restrict__ n_active) {
+  RSD_PDL_SYNC();
   if (n_active != nullptr && *n_active == 0) return;
   constexpr int KB = HD / 32;    // 32-dim blocks of the head dimension
   constexpr int NT = HD / 8;     // 8-dim output tiles
@@ -176,6 +177,7 @@ __global__ void __launch_bounds__(HD)
 attn_merge_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml, const int32_t* __restrict__ slot_row,
                   const int32_t* __restrict__ len_or_pos, int len_offset, OT* __restrict__ out, OT* __restrict__ out_lo,
                   int H, int n_splits, const int32_t* __restrict__ n_active) {
+  RSD_PDL_SYNC();
   if (n_active != nullptr && *n_active == 0) return;
   const int slot = blockIdx.y, h = blockIdx.x, dd = threadIdx.x;
   if ((slot_row && slot_row[slot] < 0) || len_or_pos[slot] + len_offset <= 0) return;
@@ -196,6 +198,7 @@ attn_merge_kernel(const float* __restrict__ part_o, const float* __restrict__ pa
 
 __global__ void decode_slots_kernel(const int32_t* slot_row, const int32_t* len_or_pos, int len_offset, int32_t* row,
                                     int32_t* pos, int B) {
+  RSD_PDL_SYNC();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= B) return;
   const int r = slot_row ? slot_row[i] : i;
@@ -231,7 +234,7 @@ cudaError_t launch_attn_decode(int kv_dtype, const float* q, const void* pool_la
   int32_t* pos = row + B;
   if (kv_dtype == 0 || G > 8) {
     // fp32 caches and wide groups take the generic kernel
-    decode_slots_kernel<<<(B + 255) / 256, 256, 0, s>>>(slot_row, len_or_pos, len_offset, row, pos, B);
+    RSD_LAUNCH((decode_slots_kernel), (B + 255) / 256, 256, 0, s, slot_row, len_or_pos, len_offset, row, pos, B);
     launched(1);
     PassView p{nullptr, row, pos, B, n_active};
     KvView kv{const_cast<void*>(pool_layer), page_table, max_pages};
@@ -244,11 +247,11 @@ cudaError_t launch_attn_decode(int kv_dtype, const float* q, const void* pool_la
   dim3 grid(KV, B, splits);
 #define RSD_DEC(HD, KT, OT)                                                                                          \
   do {                                                                                                               \
-    attn_decode_kernel<HD, KT, OT><<<grid, 128, 0, s>>>(q, (const KT*)pool_layer, page_table, max_pages, slot_row,     \
+    RSD_LAUNCH((attn_decode_kernel<HD, KT, OT>), grid, 128, 0, s, q, (const KT*)pool_layer, page_table, max_pages, slot_row,     \
                                                         len_or_pos, len_offset, (OT*)out, (OT*)out_lo, part_o, part_ml, \
                                                         H, KV, splits, n_active);                                    \
     if (splits > 1)                                                                                                  \
-      attn_merge_kernel<HD, OT><<<dim3(H, B), HD, 0, s>>>(part_o, part_ml, slot_row, len_or_pos, len_offset, (OT*)out, \
+      RSD_LAUNCH((attn_merge_kernel<HD, OT>), dim3(H, B), HD, 0, s, part_o, part_ml, slot_row, len_or_pos, len_offset, (OT*)out, \
                                                           (OT*)out_lo, H, splits, n_active);                         \
   } while (0)
 #define RSD_DEC_O(HD, KT) do { if (out_dtype == 1) RSD_DEC(HD, KT, __nv_bfloat16); else RSD_DEC(HD, KT, float); } while (0)

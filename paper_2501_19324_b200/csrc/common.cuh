@@ -6,7 +6,38 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <utility>
+
 namespace rsd {
+
+// ---- programmatic dependent launch ------------------------------------------------------------------
+// Every kernel starts with RSD_PDL_SYNC(): it lets the next kernel in the stream be scheduled early
+// (launch_dependents) and then waits until the kernels before it have completed and their writes
+// are visible (wait).  Launched through launch_pdl, a kernel's blocks can therefore be resident and
+// past their set-up while the previous kernel drains, instead of paying the launch gap after it.
+// Without the launch attribute both instructions do nothing.
+#define RSD_PDL_SYNC()                                             \
+  do {                                                             \
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); \
+    asm volatile("griddepcontrol.wait;" ::: "memory");             \
+  } while (0)
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(std::forward<Args>(args))...);
+}
+#define RSD_LAUNCH(kernel, grid, block, smem, stream, ...) \
+  (void)::rsd::launch_pdl(kernel, dim3(grid), dim3(block), (size_t)(smem), stream, __VA_ARGS__)
 
 // ---- element conversion ---------------------------------------------------------------------
 __device__ __forceinline__ float to_f32(float v) { return v; }

@@ -129,6 +129,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
                const __grid_constant__ CUtensorMap tm_x_lo, float* __restrict__ Y,
                int M, int N, int K, int accumulate, int splits, int kb_per_split, float* __restrict__ partials,
                int* __restrict__ err, const int32_t* __restrict__ n_active) {
+  RSD_PDL_SYNC();
   if (n_active != nullptr && *n_active == 0) return;
   using Cfg = TcCfg<MT>;
   constexpr int kRows = SPLIT ? MT / 2 : MT;   // distinct x rows per tile
@@ -261,6 +262,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
 __global__ void __launch_bounds__(256)
 splitk_reduce_kernel(const float* __restrict__ partials, float* __restrict__ Y, int M, int N, int splits, int accumulate,
                      const int32_t* __restrict__ n_active) {
+  RSD_PDL_SYNC();
   if (n_active != nullptr && *n_active == 0) return;
   const size_t total4 = (size_t)M * N / 4, stride = (size_t)M * N / 4;
   const float4* p4 = reinterpret_cast<const float4*>(partials);
@@ -384,12 +386,12 @@ cudaError_t launch_mt(const CUtensorMap& tw, const CUtensorMap& tx, const CUtens
     configured = true;
   }
   dim3 grid(p.n_tiles, p.m_tiles, p.splits);
-  gemm_tc_kernel<MT, SPLIT><<<grid, 192, TcCfg<MT>::kSmemBytes, s>>>(tw, tx, txl, y, M, N, K, accumulate, p.splits,
+  RSD_LAUNCH((gemm_tc_kernel<MT, SPLIT>), grid, 192, TcCfg<MT>::kSmemBytes, s, tw, tx, txl, y, M, N, K, accumulate, p.splits,
                                                                      p.kb_per_split, partials, err, n_active);
   if (p.splits > 1 && !defer_reduce) {
     const size_t total4 = (size_t)M * N / 4;
     const int blocks = (int)std::min<size_t>((total4 + 255) / 256, 148 * 8);
-    splitk_reduce_kernel<<<blocks, 256, 0, s>>>(partials, y, M, N, p.splits, accumulate, n_active);
+    RSD_LAUNCH((splitk_reduce_kernel), blocks, 256, 0, s, partials, y, M, N, p.splits, accumulate, n_active);
     return launched(2);
   }
   return launched(1);

@@ -14,6 +14,7 @@ namespace rsd {
 // ---------------------------------------------------------------------------------------------
 template <typename WT>
 __global__ void embed_kernel(const WT* __restrict__ E, PassView p, float* __restrict__ x, int d) {
+  RSD_PDL_SYNC();
   RSD_SKIP_IF_IDLE(p.n_active);
   const int t = blockIdx.x;
   if (p.tok_row[t] < 0) return;
@@ -30,8 +31,8 @@ __global__ void embed_kernel(const WT* __restrict__ E, PassView p, float* __rest
 
 cudaError_t launch_embed(int dtype, const void* embed, PassView p, float* x, int d, cudaStream_t s) {
   if (p.T <= 0) return cudaSuccess;
-  if (dtype == 1) embed_kernel<__nv_bfloat16><<<p.T, 128, 0, s>>>((const __nv_bfloat16*)embed, p, x, d);
-  else embed_kernel<float><<<p.T, 128, 0, s>>>((const float*)embed, p, x, d);
+  if (dtype == 1) RSD_LAUNCH((embed_kernel<__nv_bfloat16>), p.T, 128, 0, s, (const __nv_bfloat16*)embed, p, x, d);
+  else RSD_LAUNCH((embed_kernel<float>), p.T, 128, 0, s, (const float*)embed, p, x, d);
   return launched(1);
 }
 
@@ -42,6 +43,7 @@ template <typename OT, typename GT>
 __global__ void rmsnorm_kernel(float* __restrict__ x, const GT* __restrict__ gain, OT* __restrict__ out,
                                OT* __restrict__ out_lo, int d, float eps, const int32_t* __restrict__ src,
                                const int32_t* n_active, const float* __restrict__ partials, int splits, int T) {
+  RSD_PDL_SYNC();
   RSD_SKIP_IF_IDLE(n_active);
   __shared__ float red[33];
   const int t = blockIdx.x;
@@ -89,9 +91,9 @@ cudaError_t launch_rmsnorm(int dtype, float* x, const void* gain, void* out, voi
   if (T <= 0) return cudaSuccess;
   const int threads = d >= 2048 ? 512 : 256;
   if (dtype == 1)
-    rmsnorm_kernel<__nv_bfloat16, __nv_bfloat16><<<T, threads, 0, s>>>(x, (const __nv_bfloat16*)gain, (__nv_bfloat16*)out, (__nv_bfloat16*)out_lo, d, eps, src, n_active, pending.partials, pending.splits, T);
+    RSD_LAUNCH((rmsnorm_kernel<__nv_bfloat16, __nv_bfloat16>), T, threads, 0, s, x, (const __nv_bfloat16*)gain, (__nv_bfloat16*)out, (__nv_bfloat16*)out_lo, d, eps, src, n_active, pending.partials, pending.splits, T);
   else
-    rmsnorm_kernel<float, float><<<T, threads, 0, s>>>(x, (const float*)gain, (float*)out, nullptr, d, eps, src, n_active, pending.partials, pending.splits, T);
+    RSD_LAUNCH((rmsnorm_kernel<float, float>), T, threads, 0, s, x, (const float*)gain, (float*)out, nullptr, d, eps, src, n_active, pending.partials, pending.splits, T);
   return launched(1);
 }
 
@@ -105,6 +107,7 @@ template <typename WT, int MT>
 __global__ void __launch_bounds__(256)
 gemv_splitk_kernel(const WT* __restrict__ W, const WT* __restrict__ X, const WT* __restrict__ X_lo, float* __restrict__ Y,
                    int M, int N, int K, int ks, int accumulate, const int32_t* n_active) {
+  RSD_PDL_SYNC();
   RSD_SKIP_IF_IDLE(n_active);
   constexpr int VN = Vec16<WT>::N;
   __shared__ float part[8][MT];
@@ -169,9 +172,9 @@ cudaError_t launch_gemm_simt(int dtype, const void* W, const void* x, const void
   constexpr int MT = 8;
   dim3 grid((N + (8 / ks) - 1) / (8 / ks), (M + MT - 1) / MT);
   if (dtype == 1)
-    gemv_splitk_kernel<__nv_bfloat16, MT><<<grid, 256, 0, s>>>((const __nv_bfloat16*)W, (const __nv_bfloat16*)x, (const __nv_bfloat16*)x_lo, y, M, N, K, ks, accumulate, n_active);
+    RSD_LAUNCH((gemv_splitk_kernel<__nv_bfloat16, MT>), grid, 256, 0, s, (const __nv_bfloat16*)W, (const __nv_bfloat16*)x, (const __nv_bfloat16*)x_lo, y, M, N, K, ks, accumulate, n_active);
   else
-    gemv_splitk_kernel<float, MT><<<grid, 256, 0, s>>>((const float*)W, (const float*)x, nullptr, y, M, N, K, ks, accumulate, n_active);
+    RSD_LAUNCH((gemv_splitk_kernel<float, MT>), grid, 256, 0, s, (const float*)W, (const float*)x, nullptr, y, M, N, K, ks, accumulate, n_active);
   return launched(1);
 }
 
@@ -179,6 +182,7 @@ cudaError_t launch_gemm_simt(int dtype, const void* W, const void* x, const void
 // Rotary table: table[pos, i] = (cos, sin)(pos * theta^(-2i/hd)), evaluated in fp64
 // ---------------------------------------------------------------------------------------------
 __global__ void rope_table_kernel(float2* table, int n_pos, int half, double theta, double hd) {
+  RSD_PDL_SYNC();
   const int idx = blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= n_pos * half) return;
   const int pos = idx / half, i = idx % half;
@@ -191,7 +195,7 @@ __global__ void rope_table_kernel(float2* table, int n_pos, int half, double the
 cudaError_t launch_rope_table(float2* table, int n_pos, int hd, float theta, cudaStream_t s) {
   const int n = n_pos * (hd / 2);
   if (n <= 0) return cudaSuccess;
-  rope_table_kernel<<<(n + 255) / 256, 256, 0, s>>>(table, n_pos, hd / 2, (double)theta, (double)hd);
+  RSD_LAUNCH((rope_table_kernel), (n + 255) / 256, 256, 0, s, table, n_pos, hd / 2, (double)theta, (double)hd);
   return launched(1);
 }
 
@@ -221,6 +225,7 @@ __global__ void rope_kv_kernel(const float* __restrict__ qkv, const float* __res
                                PassView p, float* __restrict__ q_out, KT* pool,
                                const int32_t* __restrict__ page_table, int max_pages,
                                const float2* __restrict__ rope, int H, int KV, int hd) {
+  RSD_PDL_SYNC();
   RSD_SKIP_IF_IDLE(p.n_active);
   const int t = blockIdx.x;
   const int row = p.tok_row[t];
@@ -263,16 +268,17 @@ cudaError_t launch_rope_kv(int kv_dtype, const float* qkv, SplitSum pending, Pas
                            const float2* rope, int H, int KV, int hd, cudaStream_t s) {
   if (p.T <= 0) return cudaSuccess;
   if (kv_dtype == 2)
-    rope_kv_kernel<__half><<<p.T, 256, 0, s>>>(qkv, pending.partials, pending.splits, p, q_out, (__half*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd);
+    RSD_LAUNCH((rope_kv_kernel<__half>), p.T, 256, 0, s, qkv, pending.partials, pending.splits, p, q_out, (__half*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd);
   else if (kv_dtype == 1)
-    rope_kv_kernel<__nv_bfloat16><<<p.T, 256, 0, s>>>(qkv, pending.partials, pending.splits, p, q_out, (__nv_bfloat16*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd);
+    RSD_LAUNCH((rope_kv_kernel<__nv_bfloat16>), p.T, 256, 0, s, qkv, pending.partials, pending.splits, p, q_out, (__nv_bfloat16*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd);
   else
-    rope_kv_kernel<float><<<p.T, 256, 0, s>>>(qkv, pending.partials, pending.splits, p, q_out, (float*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd);
+    RSD_LAUNCH((rope_kv_kernel<float>), p.T, 256, 0, s, qkv, pending.partials, pending.splits, p, q_out, (float*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd);
   return launched(1);
 }
 
 // Stand-alone rotary kernel on [T, n_heads, hd] fp32 (angles in fp64).
 __global__ void rope_only_kernel(float* v, const int32_t* pos, int n_heads, int hd, double theta) {
+  RSD_PDL_SYNC();
   const int t = blockIdx.x, half = hd / 2;
   const int p = pos[t];
   for (int idx = threadIdx.x; idx < n_heads * half; idx += blockDim.x) {
@@ -288,7 +294,7 @@ __global__ void rope_only_kernel(float* v, const int32_t* pos, int n_heads, int 
 
 cudaError_t launch_rope_only(float* v, const int32_t* pos, int T, int n_heads, int hd, float theta, cudaStream_t s) {
   if (T <= 0) return cudaSuccess;
-  rope_only_kernel<<<T, 128, 0, s>>>(v, pos, n_heads, hd, (double)theta);
+  RSD_LAUNCH((rope_only_kernel), T, 128, 0, s, v, pos, n_heads, hd, (double)theta);
   return launched(1);
 }
 
@@ -301,6 +307,7 @@ __global__ void __launch_bounds__(128)
 attn_generic_kernel(const float* __restrict__ q, PassView p, const KT* __restrict__ pool,
                     const int32_t* __restrict__ page_table, int max_pages, OT* __restrict__ out, OT* __restrict__ out_lo,
                     int H, int KV) {
+  RSD_PDL_SYNC();
   RSD_SKIP_IF_IDLE(p.n_active);
   constexpr int DPL = HD / 32;
   const int lane = threadIdx.x & 31;
@@ -366,7 +373,7 @@ cudaError_t launch_attn_generic(int kv_dtype, const float* q, PassView p, KvView
   const int warps = p.T * H;
   const int blocks = (warps + 3) / 4;
 #define RSD_ATTN(KT, OT, HD) \
-  attn_generic_kernel<KT, OT, HD><<<blocks, 128, 0, s>>>(q, p, (const KT*)kv.pool_layer, kv.page_table, kv.max_pages, (OT*)out, (OT*)out_lo, H, KV)
+  RSD_LAUNCH((attn_generic_kernel<KT, OT, HD>), blocks, 128, 0, s, q, p, (const KT*)kv.pool_layer, kv.page_table, kv.max_pages, (OT*)out, (OT*)out_lo, H, KV)
 #define RSD_ATTN_HD(KT, OT) do { if (hd == 128) RSD_ATTN(KT, OT, 128); else RSD_ATTN(KT, OT, 64); } while (0)
   using bf = __nv_bfloat16;
   if (kv_dtype == 2) { if (out_dtype == 1) RSD_ATTN_HD(__half, bf); else RSD_ATTN_HD(__half, float); }
@@ -383,6 +390,7 @@ cudaError_t launch_attn_generic(int kv_dtype, const float* q, PassView p, KvView
 template <typename OT>
 __global__ void swiglu_kernel(const float* __restrict__ gu, const float* __restrict__ partials, int splits,
                               OT* __restrict__ out, OT* __restrict__ out_lo, int T, int F, const int32_t* n_active) {
+  RSD_PDL_SYNC();
   RSD_SKIP_IF_IDLE(n_active);
   const size_t n = (size_t)T * F;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
@@ -400,8 +408,8 @@ cudaError_t launch_swiglu(int dtype, const float* gu, SplitSum pending, void* ou
   const size_t n = (size_t)T * F;
   int blocks = (int)((n + 255) / 256);
   if (blocks > 148 * 8) blocks = 148 * 8;
-  if (dtype == 1) swiglu_kernel<__nv_bfloat16><<<blocks, 256, 0, s>>>(gu, pending.partials, pending.splits, (__nv_bfloat16*)out, (__nv_bfloat16*)out_lo, T, F, n_active);
-  else swiglu_kernel<float><<<blocks, 256, 0, s>>>(gu, pending.partials, pending.splits, (float*)out, nullptr, T, F, n_active);
+  if (dtype == 1) RSD_LAUNCH((swiglu_kernel<__nv_bfloat16>), blocks, 256, 0, s, gu, pending.partials, pending.splits, (__nv_bfloat16*)out, (__nv_bfloat16*)out_lo, T, F, n_active);
+  else RSD_LAUNCH((swiglu_kernel<float>), blocks, 256, 0, s, gu, pending.partials, pending.splits, (float*)out, nullptr, T, F, n_active);
   return launched(1);
 }
 
@@ -424,6 +432,7 @@ __device__ __forceinline__ unsigned long long pack_best(float sc, int id) {
 // Grid (slots, chunks): every block scans one chunk of the vocabulary and folds its best candidate
 // into best[slot] with an atomic maximum (order-independent, hence deterministic).
 __global__ void __launch_bounds__(1024) sample_kernel(SampleArgs a) {
+  RSD_PDL_SYNC();
   RSD_SKIP_IF_IDLE(a.n_active);
   __shared__ float s_sc[32];
   __shared__ int s_ix[32];
@@ -478,6 +487,7 @@ __global__ void __launch_bounds__(1024) sample_kernel(SampleArgs a) {
 
 // token[slot] = id held in best[slot]; best is cleared for the next use.
 __global__ void sample_finalize_kernel(unsigned long long* best, const int32_t* slot_row, int32_t* token, int n) {
+  RSD_PDL_SYNC();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n) return;
   if (slot_row[i] >= 0) token[i] = (int32_t)(0xFFFFFFFFu - (uint32_t)(best[i] & 0xFFFFFFFFull));
@@ -491,13 +501,14 @@ int sample_chunks(int v_limit) { return v_limit >= 65536 ? 16 : (v_limit >= 8192
 cudaError_t launch_sample(const SampleArgs& a, cudaStream_t s) {
   if (a.n_slots <= 0) return cudaSuccess;
   const int threads = a.v_limit >= 16384 ? 1024 : 256;
-  sample_kernel<<<dim3(a.n_slots, sample_chunks(a.v_limit)), threads, 0, s>>>(a);
+  RSD_LAUNCH((sample_kernel), dim3(a.n_slots, sample_chunks(a.v_limit)), threads, 0, s, a);
   if (a.token == nullptr) return launched(1);
-  sample_finalize_kernel<<<(a.n_slots + 255) / 256, 256, 0, s>>>(a.best, a.slot_row, a.token, a.n_slots);
+  RSD_LAUNCH((sample_finalize_kernel), (a.n_slots + 255) / 256, 256, 0, s, a.best, a.slot_row, a.token, a.n_slots);
   return launched(2);
 }
 
 __global__ void philox_kernel(const uint32_t* ctr, const uint32_t* key, uint32_t* out, int n) {
+  RSD_PDL_SYNC();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n) return;
   const uint4 r = philox4x32_10(make_uint4(ctr[4 * i], ctr[4 * i + 1], ctr[4 * i + 2], ctr[4 * i + 3]),
@@ -507,7 +518,7 @@ __global__ void philox_kernel(const uint32_t* ctr, const uint32_t* key, uint32_t
 
 cudaError_t launch_philox(const uint32_t* ctr, const uint32_t* key, uint32_t* out, int n, cudaStream_t s) {
   if (n <= 0) return cudaSuccess;
-  philox_kernel<<<(n + 255) / 256, 256, 0, s>>>(ctr, key, out, n);
+  RSD_LAUNCH((philox_kernel), (n + 255) / 256, 256, 0, s, ctr, key, out, n);
   return launched(1);
 }
 
@@ -519,6 +530,7 @@ template <typename WT>
 __global__ void reward_kernel(const float* __restrict__ x, const WT* __restrict__ final_norm, const WT* __restrict__ w_r,
                               int head_kind, const int32_t* __restrict__ last_idx, int t0, int T, int d, float eps,
                               float* __restrict__ reward) {
+  RSD_PDL_SYNC();
   __shared__ float red[33];
   const int row = blockIdx.x;
   const int idx = last_idx[row];
@@ -543,9 +555,9 @@ cudaError_t launch_reward(int dtype, const float* x, const void* final_norm, con
                           cudaStream_t s) {
   if (n_rows <= 0) return cudaSuccess;
   if (dtype == 1)
-    reward_kernel<__nv_bfloat16><<<n_rows, 256, 0, s>>>(x, (const __nv_bfloat16*)final_norm, (const __nv_bfloat16*)w_r, head_kind, last_idx, t0, T, d, eps, reward);
+    RSD_LAUNCH((reward_kernel<__nv_bfloat16>), n_rows, 256, 0, s, x, (const __nv_bfloat16*)final_norm, (const __nv_bfloat16*)w_r, head_kind, last_idx, t0, T, d, eps, reward);
   else
-    reward_kernel<float><<<n_rows, 256, 0, s>>>(x, (const float*)final_norm, (const float*)w_r, head_kind, last_idx, t0, T, d, eps, reward);
+    RSD_LAUNCH((reward_kernel<float>), n_rows, 256, 0, s, x, (const float*)final_norm, (const float*)w_r, head_kind, last_idx, t0, T, d, eps, reward);
   return launched(1);
 }
 

@@ -13,6 +13,7 @@ namespace rsd {
 // from a bump counter, rows served in ascending order, each row's new pages consecutive.
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(1024) reserve_pages_kernel(RowState st, int which, int mode) {
+  RSD_PDL_SYNC();
   __shared__ int scan[33];
   const int b = threadIdx.x;
   int need = 0;
@@ -47,7 +48,7 @@ __global__ void __launch_bounds__(1024) reserve_pages_kernel(RowState st, int wh
 }
 
 cudaError_t launch_reserve_pages(const RowState& st, int which, ReserveMode mode, cudaStream_t s) {
-  reserve_pages_kernel<<<1, 1024, 0, s>>>(st, which, (int)mode);
+  RSD_LAUNCH((reserve_pages_kernel), 1, 1024, 0, s, st, which, (int)mode);
   return launched(1);
 }
 
@@ -56,6 +57,7 @@ cudaError_t launch_reserve_pages(const RowState& st, int which, ReserveMode mode
 // `which`, flattened in (row, position) order.  Advances kv_len to `end`.
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(1024) build_pass_kernel(RowState st, int which, int mode) {
+  RSD_PDL_SYNC();
   __shared__ int scan[33];
   __shared__ int s_off[kMaxBatch + 1];
   __shared__ int s_start[kMaxBatch];
@@ -102,7 +104,7 @@ __global__ void __launch_bounds__(1024) build_pass_kernel(RowState st, int which
 }
 
 cudaError_t launch_build_pass(const RowState& st, int which, PassMode mode, cudaStream_t s) {
-  build_pass_kernel<<<1, 1024, 0, s>>>(st, which, (int)mode);
+  RSD_LAUNCH((build_pass_kernel), 1, 1024, 0, s, st, which, (int)mode);
   return launched(1);
 }
 
@@ -111,6 +113,7 @@ cudaError_t launch_build_pass(const RowState& st, int which, PassMode mode, cuda
 // Phase 1: the target writes y_i for the rejected rows (slot i = rej_idx[i]).
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(1024) decode_begin_kernel(RowState st, int phase) {
+  RSD_PDL_SYNC();
   __shared__ int scan[33];
   const int b = threadIdx.x;
   int part = 0;
@@ -132,11 +135,12 @@ __global__ void __launch_bounds__(1024) decode_begin_kernel(RowState st, int pha
 }
 
 cudaError_t launch_decode_begin(const RowState& st, int phase, cudaStream_t s) {
-  decode_begin_kernel<<<1, 1024, 0, s>>>(st, phase);
+  RSD_LAUNCH((decode_begin_kernel), 1, 1024, 0, s, st, phase);
   return launched(1);
 }
 
 __global__ void __launch_bounds__(1024) decode_prepare_kernel(RowState st, int which, int n_slots) {
+  RSD_PDL_SYNC();
   if (st.n_active[0] == 0) return;
   const int i = threadIdx.x;
   if (i >= n_slots) return;
@@ -153,7 +157,7 @@ __global__ void __launch_bounds__(1024) decode_prepare_kernel(RowState st, int w
 
 cudaError_t launch_decode_prepare(const RowState& st, int which, int n_slots, cudaStream_t s) {
   if (n_slots <= 0) return cudaSuccess;
-  decode_prepare_kernel<<<1, 1024, 0, s>>>(st, which, n_slots);
+  RSD_LAUNCH((decode_prepare_kernel), 1, 1024, 0, s, st, which, n_slots);
   return launched(1);
 }
 
@@ -166,6 +170,7 @@ __device__ __forceinline__ bool ends_step(int t, const LoopParams& lp) {
 // Appends the current iteration's token of every active slot to its row and stops rows whose step ended.
 __global__ void __launch_bounds__(1024)
 decode_update_kernel(RowState st, int which, int phase, unsigned long long* best, int n_slots, LoopParams lp) {
+  RSD_PDL_SYNC();
   if (st.n_active[0] == 0) return;
   const int iter = st.iter[0];   // iteration of the current decode phase, kept on the device
   const int i = threadIdx.x;
@@ -201,7 +206,7 @@ decode_update_kernel(RowState st, int which, int phase, unsigned long long* best
 cudaError_t launch_decode_update(const RowState& st, int which, int phase, unsigned long long* best,
                                  int n_slots, const LoopParams& lp, cudaStream_t s) {
   if (n_slots <= 0) return cudaSuccess;
-  decode_update_kernel<<<1, 1024, 0, s>>>(st, which, phase, best, n_slots, lp);
+  RSD_LAUNCH((decode_update_kernel), 1, 1024, 0, s, st, which, phase, best, n_slots, lp);
   return launched(1);
 }
 
@@ -248,6 +253,7 @@ __device__ __forceinline__ int ballot_rank(bool flag, int* wsum, int* total) {
 }
 
 __global__ void __launch_bounds__(1024) gate_kernel(RowState st, float delta, LoopParams lp) {
+  RSD_PDL_SYNC();
   __shared__ int wsum[33];
   const int b = threadIdx.x;
   bool live = false, rejected = false;
@@ -283,7 +289,7 @@ __global__ void __launch_bounds__(1024) gate_kernel(RowState st, float delta, Lo
 }
 
 cudaError_t launch_gate(const RowState& st, float delta, const LoopParams& lp, cudaStream_t s) {
-  gate_kernel<<<1, 1024, 0, s>>>(st, delta, lp);
+  RSD_LAUNCH((gate_kernel), 1, 1024, 0, s, st, delta, lp);
   return launched(1);
 }
 
@@ -291,6 +297,7 @@ cudaError_t launch_gate(const RowState& st, float delta, const LoopParams& lp, c
 // then the ascending write.
 __global__ void __launch_bounds__(1024)
 gate_count_kernel(const float* rewards, const uint8_t* live, float delta, uint8_t* accept, int32_t* block_cnt, int B) {
+  RSD_PDL_SYNC();
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   bool rej = false;
   if (b < B) {
@@ -304,6 +311,7 @@ gate_count_kernel(const float* rewards, const uint8_t* live, float delta, uint8_
 }
 
 __global__ void __launch_bounds__(1024) gate_scan_kernel(int32_t* block_cnt, int n_blocks, int32_t* n_rej) {
+  RSD_PDL_SYNC();
   // exclusive scan of up to 2^24 / 1024 = 16384 block counts by one block, 16 per thread
   __shared__ int scan[33];
   int local[16];
@@ -325,6 +333,7 @@ __global__ void __launch_bounds__(1024) gate_scan_kernel(int32_t* block_cnt, int
 
 __global__ void __launch_bounds__(1024)
 gate_write_kernel(const uint8_t* live, const uint8_t* accept, const int32_t* block_off, int32_t* rej_idx, int B) {
+  RSD_PDL_SYNC();
   __shared__ int wsum[33];
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   const bool rej = b < B && live[b] != 0 && accept[b] == 0;
@@ -336,9 +345,9 @@ gate_write_kernel(const uint8_t* live, const uint8_t* accept, const int32_t* blo
 cudaError_t launch_gate_compact_large(const float* rewards, const uint8_t* live, float delta, uint8_t* accept,
                                       int32_t* rej_idx, int32_t* n_rej, int32_t* block_cnt, int B, cudaStream_t s) {
   const int n_blocks = (B + 1023) / 1024;
-  gate_count_kernel<<<n_blocks, 1024, 0, s>>>(rewards, live, delta, accept, block_cnt, B);
-  gate_scan_kernel<<<1, 1024, 0, s>>>(block_cnt, n_blocks, n_rej);
-  gate_write_kernel<<<n_blocks, 1024, 0, s>>>(live, accept, block_cnt, rej_idx, B);
+  RSD_LAUNCH((gate_count_kernel), n_blocks, 1024, 0, s, rewards, live, delta, accept, block_cnt, B);
+  RSD_LAUNCH((gate_scan_kernel), 1, 1024, 0, s, block_cnt, n_blocks, n_rej);
+  RSD_LAUNCH((gate_write_kernel), n_blocks, 1024, 0, s, live, accept, block_cnt, rej_idx, B);
   return launched(3);
 }
 
@@ -348,6 +357,7 @@ cudaError_t launch_gate_compact_large(const float* rewards, const uint8_t* live,
 // ---------------------------------------------------------------------------------------------
 __global__ void commit_kernel(RowState st, LoopParams lp, int32_t* out_tokens, int32_t* out_len, float* out_rewards,
                               uint8_t* out_accept, uint8_t* out_live) {
+  RSD_PDL_SYNC();
   const int b = blockIdx.x;
   const bool live = st.live[b] != 0;
   const int acc = st.accept[b];
@@ -381,7 +391,7 @@ __global__ void commit_kernel(RowState st, LoopParams lp, int32_t* out_tokens, i
 cudaError_t launch_commit(const RowState& st, const LoopParams& lp, int32_t* out_tokens, int32_t* out_len,
                           float* out_rewards, uint8_t* out_accept, uint8_t* out_live, cudaStream_t s) {
   if (st.B <= 0) return cudaSuccess;
-  commit_kernel<<<st.B, 128, 0, s>>>(st, lp, out_tokens, out_len, out_rewards, out_accept, out_live);
+  RSD_LAUNCH((commit_kernel), st.B, 128, 0, s, st, lp, out_tokens, out_len, out_rewards, out_accept, out_live);
   return launched(1);
 }
 
