@@ -298,6 +298,142 @@ def run_ours(args, rank: int, world: int):
         dist.destroy_process_group()
 
 
+# ------------------------------------------------------------------------------------------------
+# Kernel sweeps: each point is one JSON line with its fraction of the HBM or bf16 roofline
+# ------------------------------------------------------------------------------------------------
+def _graph_time_us(fn, variants, iters=20):
+    """Device time per call of fn(v), v cycling over `variants` (distinct buffers, so that repeated
+    calls do not hit L2), measured by replaying a CUDA graph of `iters` calls."""
+    import torch
+    torch.cuda.synchronize()          # inputs were filled on the default stream: finish before the side stream reads them
+    side = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        for v in variants:
+            fn(v)
+        torch.cuda.synchronize()
+        with torch.cuda.graph(g, stream=side):
+            for i in range(iters):
+                fn(variants[i % len(variants)])
+    torch.cuda.synchronize()
+    g.replay()
+    torch.cuda.synchronize()
+    s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s.record(); g.replay(); e.record()
+    torch.cuda.synchronize()
+    return s.elapsed_time(e) * 1e3 / iters
+
+
+def sweep_gemm(args):
+    import torch
+    from paper_2501_19324_b200 import binding as rb
+    hbm, tf, how = peaks()
+    for K, N in ((1536, 8960), (3584, 18944)):
+        nbuf = max(2, int(400e6 // (N * K * 2)))
+        Ws = [(torch.randn(N, K, device="cuda") * 0.02).to(torch.bfloat16) for _ in range(nbuf)]
+        for M in (1, 2, 4, 8, 16, 32, 64, 128, 256, 512):
+            x = torch.randn(M, K, device="cuda")
+            hi = x.to(torch.bfloat16)
+            lo = (x - hi.float()).to(torch.bfloat16)
+            y = torch.zeros(M, N, device="cuda")
+            nbytes = rb.lib().rsd_k_gemm_scratch_bytes(M, N, K)
+            scratch = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
+
+            def call(W):
+                rb._check(rb.lib().rsd_k_gemm(rb._ptr(W), rb._ptr(hi), rb._ptr(lo), rb._ptr(y), M, N, K, 1, 0, 0,
+                                              rb._ptr(scratch), nbytes, rb._stream()))
+            us = _graph_time_us(call, Ws)
+            byts = N * K * 2 + 2 * M * K * 2 + M * N * 4
+            flops = 2.0 * 2 * M * N * K          # hi and lo rows both go through the tensor cores
+            print(json.dumps({"sweep": "gemm", "M": M, "K": K, "N": N, "us": us, "GBps": byts / us * 1e-3,
+                              "hbm_frac": byts / us * 1e-3 / hbm, "TFLOPs_mma": flops / us * 1e-6,
+                              "bf16_frac": flops / us * 1e-6 / tf, "peak_source": how}), flush=True)
+
+
+def sweep_attn(args):
+    import torch
+    from paper_2501_19324_b200 import binding as rb
+    hbm, _, how = peaks()
+    hd = 128
+    for H, KV in ((12, 2), (28, 4)):
+        for ctx in (512, 1024, 2048, 4096, 8192, 16384):
+            for B in (1, 2, 4, 8, 16, 32, 64, 128, 256):
+                n_pages = B * (ctx // 16)
+                pool_bytes = n_pages * 2 * KV * 16 * hd * 2
+                if pool_bytes > 24e9:
+                    continue
+                reps = max(1, min(4, int(300e6 // pool_bytes) + 1))
+                pools = [torch.randn(n_pages * 2 * KV * 16 * hd, device="cuda", dtype=torch.float16) for _ in range(reps)]
+                table = torch.randperm(n_pages, device="cuda", dtype=torch.int32).view(B, ctx // 16).contiguous()
+                q = torch.randn(B, H, hd, device="cuda")
+                ctx_len = torch.full((B,), ctx, dtype=torch.int32, device="cuda")
+                out = torch.empty_like(q)
+                nbytes = rb.lib().rsd_k_attn_decode_scratch_bytes(B, H, hd, ctx)
+                scratch = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
+
+                def call(pool):
+                    rb._check(rb.lib().rsd_k_attn_decode(rb._ptr(q), rb._ptr(pool), rb._ptr(table), rb._ptr(ctx_len),
+                                                         rb._ptr(out), B, H, KV, hd, ctx // 16, 2, rb._ptr(scratch),
+                                                         nbytes, rb._stream()))
+                us = _graph_time_us(call, pools, iters=10)
+                print(json.dumps({"sweep": "attn_decode", "H": H, "KV": KV, "ctx": ctx, "batch": B, "us": us,
+                                  "GBps": pool_bytes / us * 1e-3, "hbm_frac": pool_bytes / us * 1e-3 / hbm,
+                                  "pages": "randomly permuted", "peak_source": how}), flush=True)
+                del pools
+
+
+def sweep_gate(args):
+    import torch
+    from paper_2501_19324_b200 import binding as rb
+    hbm, _, how = peaks()
+    for B in (256, 1 << 20):
+        for p in (0.1, 0.3, 0.5, 0.7, 0.9):
+            r = torch.rand(B, device="cuda")
+            live = torch.ones(B, dtype=torch.uint8, device="cuda")
+            acc = torch.empty(B, dtype=torch.uint8, device="cuda")
+            rej = torch.empty(B, dtype=torch.int32, device="cuda")
+            n = torch.zeros(1, dtype=torch.int32, device="cuda")
+            scratch = torch.zeros(4 * ((B + 1023) // 1024) + 16, dtype=torch.uint8, device="cuda")
+
+            def call(_):
+                rb._check(rb.lib().rsd_k_gate_compact(rb._ptr(r), rb._ptr(live), float(1 - p), rb._ptr(acc), rb._ptr(rej),
+                                                      rb._ptr(n), B, rb._ptr(scratch), scratch.numel(), rb._stream()))
+            us = _graph_time_us(call, [0])
+            byts = B * (4 + 1 + 1) + int(B * (1 - p)) * 4
+            print(json.dumps({"sweep": "gate_compact", "rows": B, "accept_p": p, "us": us, "GBps": byts / us * 1e-3,
+                              "hbm_frac": byts / us * 1e-3 / hbm, "bound": "latency" if B <= 1024 else "hbm",
+                              "peak_source": how}), flush=True)
+
+
+def sweep_score(args):
+    """PRM scoring of 128-token steps: the 1.5B-shape PRM behind small draft / target models; the time is
+    the PRM-scoring phase of one rsd_step."""
+    import torch
+    from paper_2501_19324_b200 import Engine, Model
+    _, tf, how = peaks()
+    small_d, small_t, prm = ri.SHAPES["mini_draft"], ri.SHAPES["mini_target"], ri.SHAPES["1.5b"]
+    models = [Model(small_d, ri.gpu_model_tensors(small_d, 0, 0, True, ri.HEAD_LM), ri.HEAD_LM),
+              Model(prm, ri.gpu_model_tensors(prm, 1, 0, True, ri.HEAD_REWARD_SIGMOID), ri.HEAD_REWARD_SIGMOID),
+              Model(small_t, ri.gpu_model_tensors(small_t, 2, 0, True, ri.HEAD_LM), ri.HEAD_LM)]
+    layer_params = prm.n_params(ri.HEAD_REWARD_SIGMOID) - prm.vocab * prm.d_model
+    for B in (1, 2, 4, 8, 16, 32, 64, 128):
+        eng = Engine(*models, max_batch=B, max_seq_tokens=256 + 3 * 128, max_step_tokens=128, max_steps=4,
+                     step_end_id=13, temperature=0.7, seed=0)
+        tokens, offsets = ri.prompts(3, B, 256, 256, small_d.vocab)
+        eng.prefill(tokens, offsets)
+        eng.step(0.0)
+        eng.phase_ms(True)
+        eng.step(0.0)
+        ms = eng.phase_ms(False)["prm_scoring"]
+        T = B * 128
+        flops = 2.0 * layer_params * T
+        print(json.dumps({"sweep": "prm_scoring", "batch": B, "step_tokens": 128, "ms": ms,
+                          "TFLOPs_algorithmic": flops / ms * 1e-9, "bf16_frac_algorithmic": flops / ms * 1e-9 / tf,
+                          "note": "split-precision operands double the tensor-core work per algorithmic flop",
+                          "peak_source": how}), flush=True)
+        eng.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -308,7 +444,12 @@ def main():
     ap.add_argument("--time-stride", type=int, default=16, dest="time_stride")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cap", type=int, default=0, help="override the step cap (profiling aid)")
+    ap.add_argument("--sweep", default="", choices=["", "gemm", "attn", "gate", "score"],
+                    help="kernel sweep on config-2 shapes instead of the step-loop benchmark")
     args = ap.parse_args()
+    if args.sweep:
+        {"gemm": sweep_gemm, "attn": sweep_attn, "gate": sweep_gate, "score": sweep_score}[args.sweep](args)
+        return
     args.warmup = max(args.warmup, 0)
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))
