@@ -185,6 +185,24 @@ def workload_config(args) -> dict:
             "l2": "weights and KV read per decode iteration exceed the 126 MB L2 (no flush needed)"}
 
 
+def combine_ranks(ms, e2e_ms, tokens, e2e_tokens, world, device):
+    """Whole-job figures of N independent replicas: the slowest rank's time, the sum of the tokens."""
+    if world <= 1:
+        return ms, e2e_ms, float(tokens), float(e2e_tokens)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms, e2e_ms], dtype=torch.float64, device=device)
+    n = torch.tensor([float(tokens), float(e2e_tokens)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(n, op=dist.ReduceOp.SUM)
+    return float(t[0]), float(t[1]), float(n[0]), float(n[1])
+
+
+def rank_prompts(rank, B, lo, hi, vocab):
+    """Every replica works on its own prompts (seed 1 + rank)."""
+    return ri.prompts(1 + rank, B, lo, hi, vocab)
+
+
 # ------------------------------------------------------------------------------------------------
 # GPU arm
 # ------------------------------------------------------------------------------------------------
@@ -208,7 +226,7 @@ def run_ours(args, rank: int, world: int):
     S = hi + n_steps * cap
     eng = Engine(*models, max_batch=B, max_seq_tokens=S, max_step_tokens=cap, max_steps=n_steps + 1,
                  step_end_id=13, temperature=0.7, seed=0)
-    tokens, offsets = ri.prompts(1 + rank, B, lo, hi, shapes[0].vocab)
+    tokens, offsets = rank_prompts(rank, B, lo, hi, shapes[0].vocab)
     pinned_tokens = torch.from_numpy(tokens).pin_memory()
 
     # calibration pass: rewards of the first step decide delta (30th percentile -> ~70 % accepted)
@@ -258,12 +276,7 @@ def run_ours(args, rank: int, world: int):
     e2e_tokens += timed_tokens
     ms = t_start.elapsed_time(t_end)
     e2e_ms = e2e_start.elapsed_time(e2e_end)
-    stats = torch.tensor([ms, e2e_ms, float(timed_tokens), float(e2e_tokens)], dtype=torch.float64, device="cuda")
-    if world > 1:
-        mx = stats.clone(); dist.all_reduce(mx, op=dist.ReduceOp.MAX)
-        sm = stats.clone(); dist.all_reduce(sm, op=dist.ReduceOp.SUM)
-        ms, e2e_ms = float(mx[0]), float(mx[1])
-        timed_tokens, e2e_tokens = float(sm[2]), float(sm[3])
+    ms, e2e_ms, timed_tokens, e2e_tokens = combine_ranks(ms, e2e_ms, timed_tokens, e2e_tokens, world, "cuda")
     counters = eng.counters()
 
     if rank == 0:

@@ -23,6 +23,7 @@ def build_pair(shapes, *, bf16, seed=0, prompts, loop_kwargs, engine_kwargs=None
     kw = dict(max_batch=B, debug_flags=RSD_DEBUG_KEEP_LOGITS)
     kw.update({k: loop_kwargs[k] for k in ("max_seq_tokens", "max_step_tokens", "max_steps", "step_end_id",
                                            "eos_id", "step_end_mod", "temperature", "seed") if k in loop_kwargs})
+    # loop_kwargs may also carry oracle-only settings (omega_kind, omega_b); the engine takes its own
     kw.update(engine_kwargs or {})
     eng = Engine(*gpu_models, **kw)
     loop = OracleRSD(*cpu_models, LoopConfig(keep_logits=True, **loop_kwargs))

@@ -111,3 +111,21 @@ def test_page_pool_exhaustion_is_an_error_not_a_fault():
         build_pair(TINY, bf16=False, prompts=prompts, loop_kwargs=base,
                    engine_kwargs=dict(kv_bytes=[page_bytes * 10, page_bytes * 400, page_bytes * 800]))
     assert e.value.code == -3
+
+
+@pytest.mark.parametrize("omega_kind,delta,alpha", [(0, 0.6, 0.0), (2, 0.0, 0.0), (3, 0.0, 0.0), (4, 0.5, 30.0)])
+def test_general_acceptance_criterion_on_gpu(omega_kind, delta, alpha):
+    """Algorithm 2 with the other weighting functions of Table 1 (constant, clip, r/(1+r), logistic):
+    the GPU draws the same Philox uniform per (row, |z_i|) and takes the same decision as the oracle."""
+    prompts = ri.prompts(11, 8, 10, 24, 1024)
+    base = dict(max_step_tokens=6, max_steps=4, max_seq_tokens=64, step_end_id=3, step_end_mod=4,
+                temperature=0.7, seed=17, omega_kind=omega_kind, omega_b=alpha)
+    eng, loop = build_pair(TINY, bf16=False, prompts=prompts, loop_kwargs=base,
+                           engine_kwargs=dict(omega_kind=omega_kind, omega_alpha=alpha))
+    seen = set()
+    for _ in range(4):
+        tol = dict(TOL32, margin_gate=0.0)            # never force the gate: it must agree by itself
+        g, o = parity_step(eng, loop, delta, **tol)
+        seen.update(g["accept"][g["step_len"] > 0].tolist())
+    assert seen == {0, 1}                             # both outcomes occurred
+    compare_counters(eng, loop)
