@@ -34,25 +34,28 @@ template <> __device__ __forceinline__ uint32_t pack2<__half>(float lo, float hi
 }
 
 template <typename KT>
-__device__ __forceinline__ void mma_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1);
+__device__ __forceinline__ void mma_16816(float& d0, float& d1, float& d2, float& d3, uint32_t a0, uint32_t a1, uint32_t a2,
+                                          uint32_t a3, uint32_t b0, uint32_t b1);
 template <>
-__device__ __forceinline__ void mma_16816<__nv_bfloat16>(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+__device__ __forceinline__ void mma_16816<__nv_bfloat16>(float& d0, float& d1, float& d2, float& d3, uint32_t a0, uint32_t a1,
+                                                         uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
   asm volatile(
       "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "+f"(d0), "+f"(d1), "+f"(d2), "+f"(d3)
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 template <>
-__device__ __forceinline__ void mma_16816<__half>(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+__device__ __forceinline__ void mma_16816<__half>(float& d0, float& d1, float& d2, float& d3, uint32_t a0, uint32_t a1,
+                                                  uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
   asm volatile(
       "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "+f"(d0), "+f"(d1), "+f"(d2), "+f"(d3)
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
 // part_o: [slot][head][split][HD] un-normalised outputs; part_ml: [slot][head][split][2] (max, sum).
 template <int HD, typename KT, typename OT>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(128, 4)
 attn_decode_kernel(const float* __restrict__ q, const KT* __restrict__ pool, const int32_t* __restrict__ page_table,
                    int max_pages, const int32_t* __restrict__ slot_row, const int32_t* __restrict__ len_or_pos, int len_offset,
                    OT* __restrict__ out, OT* __restrict__ out_lo, float* __restrict__ part_o, float* __restrict__ part_ml, int H, int KV, int n_splits,
@@ -87,27 +90,40 @@ attn_decode_kernel(const float* __restrict__ q, const KT* __restrict__ pool, con
     qa[j][0][0] = pack2<KT>(v[0], v[1]); qa[j][0][1] = pack2<KT>(v[2], v[3]);
     qa[j][1][0] = pack2<KT>(v[4], v[5]); qa[j][1][1] = pack2<KT>(v[6], v[7]);
   }
-  float o[NT][4];
+  // Rows 8..15 of every MMA tile are padding (their A rows are zero), so all tiles share two dump
+  // registers for those rows instead of carrying 2 x (NT + 2) dead accumulators.
+  float o[NT][2];
 #pragma unroll
-  for (int i = 0; i < NT; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
+  for (int i = 0; i < NT; ++i) { o[i][0] = o[i][1] = 0.f; }
+  float dump0 = 0.f, dump1 = 0.f;
   float m_run = -INFINITY, l_run = 0.f;
 
   const int32_t* pt = page_table + (size_t)row * max_pages;
   const size_t page_elems = (size_t)2 * KV * kPageTokens * HD;
   // tokens whose keys this lane loads: tile 0 -> 4(g/2) + g%2, tile 1 -> that + 2
   const int tok0 = 4 * (g >> 1) + (g & 1), tok1 = tok0 + 2;
+  int page = (p_begin + warp < p_end) ? pt[p_begin + warp] : 0;
   for (int p = p_begin + warp; p < p_end; p += 4) {
-    const KT* kb = pool + (size_t)pt[p] * page_elems + (size_t)kvh * kPageTokens * HD;
-    const KT* vb = pool + (size_t)pt[p] * page_elems + (size_t)KV * kPageTokens * HD + (size_t)kvh * HD * kPageTokens;
-    float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+    const KT* kb = pool + (size_t)page * page_elems + (size_t)kvh * kPageTokens * HD;
+    const KT* vb = pool + (size_t)page * page_elems + (size_t)KV * kPageTokens * HD + (size_t)kvh * HD * kPageTokens;
+    if (p + 4 < p_end) page = pt[p + 4];     // next page's index is fetched while this page is worked on
+    // all of the page's keys and values are requested up front (8 KB per warp in flight)
+    uint4 k0[KB], k1[KB];
+    uint2 vv[NT];
 #pragma unroll
     for (int j = 0; j < KB; ++j) {
-      const uint4 k0 = *reinterpret_cast<const uint4*>(kb + tok0 * HD + 32 * j + 8 * t);
-      const uint4 k1 = *reinterpret_cast<const uint4*>(kb + tok1 * HD + 32 * j + 8 * t);
-      mma_16816<KT>(s0, qa[j][0][0], 0u, qa[j][0][1], 0u, k0.x, k0.y);
-      mma_16816<KT>(s0, qa[j][1][0], 0u, qa[j][1][1], 0u, k0.z, k0.w);
-      mma_16816<KT>(s1, qa[j][0][0], 0u, qa[j][0][1], 0u, k1.x, k1.y);
-      mma_16816<KT>(s1, qa[j][1][0], 0u, qa[j][1][1], 0u, k1.z, k1.w);
+      k0[j] = *reinterpret_cast<const uint4*>(kb + tok0 * HD + 32 * j + 8 * t);
+      k1[j] = *reinterpret_cast<const uint4*>(kb + tok1 * HD + 32 * j + 8 * t);
+    }
+#pragma unroll
+    for (int i = 0; i < NT; ++i) vv[i] = *reinterpret_cast<const uint2*>(vb + (size_t)(8 * i + g) * kPageTokens + 4 * t);
+    float s0[2] = {0.f, 0.f}, s1[2] = {0.f, 0.f};
+#pragma unroll
+    for (int j = 0; j < KB; ++j) {
+      mma_16816<KT>(s0[0], s0[1], dump0, dump1, qa[j][0][0], 0u, qa[j][0][1], 0u, k0[j].x, k0[j].y);
+      mma_16816<KT>(s0[0], s0[1], dump0, dump1, qa[j][1][0], 0u, qa[j][1][1], 0u, k0[j].z, k0[j].w);
+      mma_16816<KT>(s1[0], s1[1], dump0, dump1, qa[j][0][0], 0u, qa[j][0][1], 0u, k1[j].x, k1[j].y);
+      mma_16816<KT>(s1[0], s1[1], dump0, dump1, qa[j][1][0], 0u, qa[j][1][1], 0u, k1[j].z, k1[j].w);
     }
     // this lane's scores of head g: tokens 4t, 4t+1 (tile 0) and 4t+2, 4t+3 (tile 1) of the page
     const int n_valid = min(kPageTokens, ctx - p * kPageTokens);
@@ -134,9 +150,8 @@ attn_decode_kernel(const float* __restrict__ q, const KT* __restrict__ pool, con
     }
 #pragma unroll
     for (int i = 0; i < NT; ++i) {
-      const uint2 vv = *reinterpret_cast<const uint2*>(vb + (size_t)(8 * i + g) * kPageTokens + 4 * t);
       o[i][0] *= corr; o[i][1] *= corr;
-      mma_16816<KT>(o[i], pa0, 0u, pa2, 0u, vv.x & mlo, vv.y & mhi);
+      mma_16816<KT>(o[i][0], o[i][1], dump0, dump1, pa0, 0u, pa2, 0u, vv[i].x & mlo, vv[i].y & mhi);
     }
   }
   // the 4 lanes of a row hold partial sums of l
@@ -209,8 +224,8 @@ __global__ void decode_slots_kernel(const int32_t* slot_row, const int32_t* len_
 
 int pick_splits(int B, int KV, int max_ctx) {
   const int ctas = B * KV;
-  int splits = (2 * 148 + ctas - 1) / ctas;
-  const int max_by_ctx = std::max(1, (max_ctx / kPageTokens) / 8);   // at least 8 pages per split
+  int splits = (4 * 148) / ctas;   // one wave of at most four CTAs per SM: a second, partial wave would double the time
+  const int max_by_ctx = std::max(1, (max_ctx / kPageTokens) / 4);   // at least 4 pages per split (one per warp)
   splits = std::min(splits, max_by_ctx);
   return std::max(1, std::min(splits, kMaxSplits));
 }

@@ -458,7 +458,8 @@ cudaError_t launch_gemm(int dtype, const void* W, const void* x, const void* x_l
                         int* deferred_splits, cudaStream_t s) {
   if (deferred_splits) *deferred_splits = 1;
   const bool tc_ok = gemm_tc_supported(dtype, M, N, K) && scratch && scratch_bytes >= gemm_scratch_bytes(M);
-  if (impl == 2 || (impl == 0 && tc_ok && M > 4))
+  // the tensor-core path wins for every M (an M = 1 GEMV included: TMA streaming beats the SIMT loads)
+  if (impl == 2 || (impl == 0 && tc_ok))
     return launch_gemm_tc(W, x, x_lo, y, M, N, K, accumulate, scratch, scratch_bytes, n_active, deferred_splits, s);
   return launch_gemm_simt(dtype, W, x, dtype == 1 ? x_lo : nullptr, y, M, N, K, accumulate, n_active, s);
 }
