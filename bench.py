@@ -41,6 +41,18 @@ WORKLOADS = {
 }
 
 
+def gemm_traffic_ratio():
+    """DRAM traffic / algorithmic bytes of the tensor-core GEMM from the committed ncu capture, or None
+    when the kernel source has changed since the counters were taken."""
+    import hashlib
+    try:
+        d = json.load(open(os.path.join(ROOT, "profiles", "gemm_tc_traffic.json")))
+        src = open(os.path.join(ROOT, d["source"]), "rb").read()
+        return d["ratio"] if hashlib.sha256(src).hexdigest() == d["sha256"] else None
+    except (OSError, KeyError, ValueError):
+        return None
+
+
 def peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -282,6 +294,8 @@ def run_ours(args, rank: int, world: int):
     if rank == 0:
         hbm, tf, how = peaks()
         achieved = gt["bytes"] / (gt["ms"] * 1e-3) / 1e9 if gt["ms"] > 0 else None
+        ratio = gemm_traffic_ratio()
+        traffic = (ratio * gt["bytes"] / gt["launches"]) if (ratio and gt["launches"]) else None
         out = {"metric": METRIC, "value": timed_tokens / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
                "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
@@ -294,7 +308,12 @@ def run_ours(args, rank: int, world: int):
                "gpu_launches": int(launches2 - launches1),
                "roofline": {"bound": "hbm", "kernel": "weight GEMM (decode, prefill, scoring)", "achieved": achieved,
                             "peak": hbm, "unit": "GB/s", "frac": (achieved / hbm) if achieved else None,
-                            "traffic": None, "peak_source": how, "timed_launches": gt["launches"],
+                            "traffic": traffic,
+                            "algorithmic_bytes_per_launch": (gt["bytes"] / gt["launches"]) if gt["launches"] else None,
+                            "traffic_source": "ncu capture of one decode-shaped launch (profiles/), traffic / algorithmic = "
+                                              + (f"{ratio}" if ratio else "n/a: kernel changed since the capture")
+                                              + ", scaled to the average launch",
+                            "peak_source": how, "timed_launches": gt["launches"],
                             "timing": f"CUDA events around every {args.time_stride}th GEMM launch of the timed steps"},
                "phase_ms_per_step": phases,
                "flops_paper": counters["flops_paper"], "clocks": clocks,
@@ -341,6 +360,18 @@ def sweep_gemm(args):
     import torch
     from paper_2501_19324_b200 import binding as rb
     hbm, tf, how = peaks()
+    if args.only:
+        # one point, launched plainly (no graph): the form an ncu capture of the GEMM kernel uses
+        M, K, N = (int(v) for v in args.only.split(","))
+        Ws = [(torch.randn(N, K, device="cuda") * 0.02).to(torch.bfloat16) for _ in range(3)]
+        x = torch.randn(M, K, device="cuda")
+        hi = x.to(torch.bfloat16)
+        lo = (x - hi.float()).to(torch.bfloat16)
+        for W in Ws + Ws:
+            rb.k_gemm(W, hi, x_lo=lo)
+        torch.cuda.synchronize()
+        print(json.dumps({"sweep": "gemm", "only": [M, K, N], "algorithmic_bytes": N * K * 2 + 2 * M * K * 2 + M * N * 4}))
+        return
     for K, N in ((1536, 8960), (3584, 18944)):
         nbuf = max(2, int(400e6 // (N * K * 2)))
         Ws = [(torch.randn(N, K, device="cuda") * 0.02).to(torch.bfloat16) for _ in range(nbuf)]
@@ -457,6 +488,7 @@ def main():
     ap.add_argument("--time-stride", type=int, default=16, dest="time_stride")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cap", type=int, default=0, help="override the step cap (profiling aid)")
+    ap.add_argument("--only", default="", help="with --sweep gemm: a single M,K,N point, plain launches")
     ap.add_argument("--sweep", default="", choices=["", "gemm", "attn", "gate", "score"],
                     help="kernel sweep on config-2 shapes instead of the step-loop benchmark")
     args = ap.parse_args()
