@@ -38,6 +38,10 @@ WORKLOADS = {
     # name: (draft, prm, target shapes, batch, prompt lo, hi, step cap)
     "cfg2": ("1.5b", "1.5b", "7b", 32, 128, 512, 128),
     "mini": ("mini_draft", "mini_draft", "mini_target", 8, 32, 96, 16),
+    # PRM at the target's shape, batch 64, 256-token prompts, steps of up to 256 tokens (delta sweep via --delta)
+    "cfg3": ("1.5b", "7b", "7b", 64, 256, 256, 256),
+    # 72B-shape target (about 145 GB of bf16 weights), batch 8, 256-token prompts, steps of up to 256 tokens
+    "cfg4": ("1.5b", "1.5b", "72b", 8, 256, 256, 256),
 }
 
 
@@ -168,8 +172,10 @@ def run_reference(args, rank: int):
     if rank != 0:
         return
     level = 0 if (args.steps + args.warmup) <= 10 and mem_available_gb() > 60 else 1
-    if args.workload != "cfg2":
+    if args.workload == "mini":
         level = 0
+    if args.workload in ("cfg3", "cfg4"):
+        level = 1          # two 7B-shape or one 72B-shape fp32 weight set do not fit the host: draft + PRM only
     sample = OracleSample(args.workload, level)
     for i in range(args.warmup):
         sample.run_once(i)
@@ -192,7 +198,8 @@ def run_reference(args, rank: int):
 def workload_config(args) -> dict:
     d, p, t, B, lo, hi, cap = WORKLOADS[args.workload]
     return {"workload": f"{args.workload}: draft {d} / PRM {p} / target {t} shapes, batch {B}, prompts {lo}-{hi} tokens, "
-                        f"step <= {cap} tokens, Gumbel-max T=0.7, delta at the 70% accept quantile",
+                        f"step <= {cap} tokens, Gumbel-max T=0.7, "
+                        + (f"delta {args.delta}" if getattr(args, "delta", None) is not None else "delta at the 70% accept quantile"),
             "batch": B, "max_step_tokens": args.cap or cap, "replicas": args.gpus,
             "l2": "weights and KV read per decode iteration exceed the 126 MB L2 (no flush needed)"}
 
@@ -245,6 +252,8 @@ def run_ours(args, rank: int, world: int):
     eng.prefill(tokens, offsets)
     r0 = eng.step(0.0)["rewards"]
     delta = float(np.sort(r0)[int(0.3 * B)])
+    if args.delta is not None:
+        delta = args.delta         # fixed threshold (config 3 sweeps 0.5 / 0.7 / 0.9)
     eng.reset()
 
     def barrier():
@@ -319,7 +328,7 @@ def run_ours(args, rank: int, world: int):
                "flops_paper": counters["flops_paper"], "clocks": clocks,
                "gen_tokens": counters["gen_tokens"]}
         if world == 1 and not args.no_cpu_baseline:
-            level = 0 if mem_available_gb() > 60 and args.workload == "cfg2" else (1 if args.workload == "cfg2" else 0)
+            level = 0 if (args.workload == "mini" or (args.workload == "cfg2" and mem_available_gb() > 60)) else 1
             smp = OracleSample(args.workload, level)
             n, dt = smp.run_once(0)
             out["cpu_baseline"] = {"value": n / dt, "unit": UNIT, "cores": cpu_cores(), "kind": "oracle",
@@ -487,6 +496,7 @@ def main():
     ap.add_argument("--workload", default="cfg2", choices=sorted(WORKLOADS))
     ap.add_argument("--time-stride", type=int, default=16, dest="time_stride")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--delta", type=float, default=None, help="fixed threshold instead of the 70 %% accept quantile")
     ap.add_argument("--cap", type=int, default=0, help="override the step cap (profiling aid)")
     ap.add_argument("--only", default="", help="with --sweep gemm: a single M,K,N point, plain launches")
     ap.add_argument("--sweep", default="", choices=["", "gemm", "attn", "gate", "score"],
