@@ -129,8 +129,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
                const __grid_constant__ CUtensorMap tm_x_lo, float* __restrict__ Y,
                int M, int N, int K, int accumulate, int splits, int kb_per_split, float* __restrict__ partials,
                int* __restrict__ err, const int32_t* __restrict__ n_active) {
-  RSD_PDL_SYNC();
-  if (n_active != nullptr && *n_active == 0) return;
+  // Programmatic dependent launch: the next kernel may be scheduled at once; this kernel sets itself
+  // up and starts streaming its WEIGHT tiles (never written by any kernel) while its predecessors are
+  // still running, and only then waits for them (griddepcontrol.wait) before it touches activations,
+  // outputs or the idle flag.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   using Cfg = TcCfg<MT>;
   constexpr int kRows = SPLIT ? MT / 2 : MT;   // distinct x rows per tile
   extern __shared__ uint8_t smem_raw[];
@@ -165,23 +168,44 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
     if (lane == 0) {
       int issued = 0;
       bool ok = true;
-      for (int i = 0; i < n_kb && ok; ++i) {
-        const int s = i % Cfg::kStages;
-        if (i >= Cfg::kStages) ok = mbar_wait(&empty[s], ((i / Cfg::kStages) - 1) & 1);
-        if (!ok || flags[0]) { ok = false; break; }
-        uint8_t* a = smem + (size_t)s * Cfg::kStageBytes;
-        mbar_expect_tx(&full[s], Cfg::kStageBytes);
-        tma_load_2d(a, &tm_w, &full[s], (kb0 + i) * kTileK, n0);
-        tma_load_2d(a + Cfg::kABytes, &tm_x, &full[s], (kb0 + i) * kTileK, m0);
-        if (SPLIT) tma_load_2d(a + Cfg::kABytes + kRows * kTileK * 2, &tm_x_lo, &full[s], (kb0 + i) * kTileK, m0);
-        issued = i + 1;
+      // weight tiles of the first ring of stages go out before the predecessors have finished
+      const int pre = min(n_kb, Cfg::kStages);
+      for (int i = 0; i < pre; ++i) {
+        mbar_expect_tx(&full[i], Cfg::kStageBytes);
+        tma_load_2d(smem + (size_t)i * Cfg::kStageBytes, &tm_w, &full[i], (kb0 + i) * kTileK, n0);
       }
-      if (!ok) {
-        if (err) atomicCAS(err, 0, -5);
-        flags[0] = 1;
-        // let the copies already in flight land before the CTA goes away
-        for (int i = max(0, issued - Cfg::kStages); i < issued; ++i)
-          mbar_wait(&full[i % Cfg::kStages], (i / Cfg::kStages) & 1);
+      issued = pre;
+      asm volatile("griddepcontrol.wait;" ::: "memory");
+      // every row of the decode phase has finished: complete the copies that are in flight (their
+      // x halves are fetched too so that the stage barriers close), then leave without computing
+      const bool idle = n_active != nullptr && *n_active == 0;
+      if (idle) flags[0] = 2;
+      for (int i = 0; i < pre; ++i) {
+        uint8_t* a = smem + (size_t)i * Cfg::kStageBytes;
+        tma_load_2d(a + Cfg::kABytes, &tm_x, &full[i], (kb0 + i) * kTileK, m0);
+        if (SPLIT) tma_load_2d(a + Cfg::kABytes + kRows * kTileK * 2, &tm_x_lo, &full[i], (kb0 + i) * kTileK, m0);
+      }
+      if (idle) {
+        for (int i = 0; i < pre; ++i) mbar_wait(&full[i], 0);
+      } else {
+        for (int i = pre; i < n_kb && ok; ++i) {
+          const int s = i % Cfg::kStages;
+          ok = mbar_wait(&empty[s], ((i / Cfg::kStages) - 1) & 1);
+          if (!ok || flags[0]) { ok = false; break; }
+          uint8_t* a = smem + (size_t)s * Cfg::kStageBytes;
+          mbar_expect_tx(&full[s], Cfg::kStageBytes);
+          tma_load_2d(a, &tm_w, &full[s], (kb0 + i) * kTileK, n0);
+          tma_load_2d(a + Cfg::kABytes, &tm_x, &full[s], (kb0 + i) * kTileK, m0);
+          if (SPLIT) tma_load_2d(a + Cfg::kABytes + kRows * kTileK * 2, &tm_x_lo, &full[s], (kb0 + i) * kTileK, m0);
+          issued = i + 1;
+        }
+        if (!ok) {
+          if (err && flags[0] != 2) atomicCAS(err, 0, -5);
+          if (flags[0] == 0) flags[0] = 1;
+          // let the copies already in flight land before the CTA goes away
+          for (int i = max(0, issued - Cfg::kStages); i < issued; ++i)
+            mbar_wait(&full[i % Cfg::kStages], (i / Cfg::kStages) & 1);
+        }
       }
     }
   } else if (warp == 5) {
@@ -204,16 +228,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
       }
       if (ok) {
         umma_commit(tmem_full);
-      } else {
+      } else if (flags[0] == 0) {      // a wait of this thread expired (flags[0] != 0: someone else stopped the CTA)
         if (err) atomicCAS(err, 0, -5);
         flags[0] = 1;
       }
     }
   } else {
     // ---------------- epilogue: TMEM -> registers -> global ----------------
-    bool ok = mbar_wait(tmem_full, 0);
-    if (!ok && err) atomicCAS(err, 0, -5);
-    if (!ok) flags[0] = 1;
+    asm volatile("griddepcontrol.wait;" ::: "memory");   // y and the partial sums belong to earlier kernels until now
+    bool ok = false;
+    for (uint32_t i = 0; i < kWaitLimit && !ok; ++i) {
+      ok = mbar_try_wait(tmem_full, 0);
+      if (!ok && flags[0]) break;                        // the CTA was stopped (idle phase or an expired wait)
+    }
+    if (!ok && flags[0] == 0) {
+      if (err) atomicCAS(err, 0, -5);
+      flags[0] = 1;
+    }
     tc_fence_after();
     const int n_local = warp * 32 + lane;
     const int n = n0 + n_local;
