@@ -208,6 +208,15 @@ int rsd_k_attn_decode(const float* q, const void* kv_pool, const int32_t* page_t
                       int32_t dtype, void* scratch, size_t scratch_bytes, void* cuda_stream);
 size_t rsd_k_attn_decode_scratch_bytes(int32_t B, int32_t H, int32_t hd, int32_t max_ctx);
 
+/* Causal attention of a ragged list of T new tokens over the same paged cache (prefill, PRM step scoring,
+ * catch-up): entry t belongs to row tok_row[t] (entries sorted by row, then position; tok_row < 0 is
+ * skipped) and attends positions [0, tok_pos[t]] of that row, whose keys and values (those of the new
+ * tokens included) are already in the pages.  q and out are [T, H, hd] fp32.  16-bit caches with
+ * H / KV <= 8 take the tensor-core kernel, everything else the generic one.                        */
+int rsd_k_attn_chunk(const float* q, const void* kv_pool, const int32_t* page_table, const int32_t* tok_row,
+                     const int32_t* tok_pos, float* out, int32_t T, int32_t H, int32_t KV, int32_t hd,
+                     int32_t max_pages, int32_t dtype, void* cuda_stream);
+
 /* Gate + compaction (Table 1 binary step; Algorithm 1 else-branch batched over rows):
  * accept[b] = live[b] && rewards[b] >= delta; rej_idx [B] receives the ascending list of live
  * rejected rows, *n_rej (device) their count.  B up to 2^24.  scratch: 4 * ceil(B / 1024) bytes. */

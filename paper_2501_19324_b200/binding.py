@@ -52,7 +52,7 @@ class rsd_counters(ctypes.Structure):
 EXPORTS = ["rsd_query_sizes", "rsd_create", "rsd_load_models", "rsd_prefill", "rsd_step", "rsd_flops_counters",
            "rsd_reset", "rsd_destroy", "rsd_last_error", "rsd_debug_force", "rsd_debug_get_logits",
            "rsd_debug_get_sampled", "rsd_debug_get_state", "rsd_debug_gemm_timing", "rsd_debug_launch_count", "rsd_debug_phase_ms", "rsd_k_gemm", "rsd_k_gemm_scratch_bytes",
-           "rsd_k_attn_decode", "rsd_k_attn_decode_scratch_bytes", "rsd_k_gate_compact", "rsd_k_gate_compact_static", "rsd_k_gate_compact_static_error", "rsd_k_rmsnorm",
+           "rsd_k_attn_decode", "rsd_k_attn_decode_scratch_bytes", "rsd_k_attn_chunk", "rsd_k_gate_compact", "rsd_k_gate_compact_static", "rsd_k_gate_compact_static_error", "rsd_k_rmsnorm",
            "rsd_k_rope", "rsd_k_swiglu", "rsd_k_sample", "rsd_k_philox"]
 
 _lib = None
@@ -89,6 +89,7 @@ def lib():
         L.rsd_k_gemm_scratch_bytes.restype = c_size_t
         L.rsd_k_attn_decode.argtypes = [vp, vp, vp, vp, vp, c_int32, c_int32, c_int32, c_int32, c_int32, c_int32,
                                         vp, c_size_t, vp]
+        L.rsd_k_attn_chunk.argtypes = [vp, vp, vp, vp, vp, vp, c_int32, c_int32, c_int32, c_int32, c_int32, c_int32, vp]
         L.rsd_k_attn_decode_scratch_bytes.argtypes = [c_int32] * 4
         L.rsd_k_attn_decode_scratch_bytes.restype = c_size_t
         L.rsd_k_gate_compact.argtypes = [vp, vp, c_float, vp, vp, vp, c_int32, vp, c_size_t, vp]
@@ -291,6 +292,16 @@ def k_attn_decode(q, kv_pool, page_table, ctx_len, KV):
     dt = {torch.bfloat16: RSD_BF16, torch.float16: 2, torch.float32: RSD_F32}[kv_pool.dtype]
     _check(lib().rsd_k_attn_decode(_ptr(q), _ptr(kv_pool), _ptr(page_table), _ptr(ctx_len), _ptr(out), B, H, KV, hd,
                                    max_pages, dt, _ptr(scratch), nbytes, _stream()))
+    return out
+
+
+def k_attn_chunk(q, kv_pool, page_table, tok_row, tok_pos, KV):
+    import torch
+    T, H, hd = q.shape
+    out = torch.zeros_like(q)
+    dt = {torch.bfloat16: RSD_BF16, torch.float16: 2, torch.float32: RSD_F32}[kv_pool.dtype]
+    _check(lib().rsd_k_attn_chunk(_ptr(q), _ptr(kv_pool), _ptr(page_table), _ptr(tok_row), _ptr(tok_pos), _ptr(out), T, H, KV,
+                                  hd, page_table.shape[1], dt, _stream()))
     return out
 
 

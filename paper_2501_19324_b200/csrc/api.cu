@@ -907,6 +907,19 @@ int rsd_k_attn_decode(const float* q, const void* kv_pool, const int32_t* page_t
   return RSD_OK;
 }
 
+int rsd_k_attn_chunk(const float* q, const void* kv_pool, const int32_t* page_table, const int32_t* tok_row,
+                     const int32_t* tok_pos, float* out, int32_t T, int32_t H, int32_t KV, int32_t hd, int32_t max_pages,
+                     int32_t dtype, void* cuda_stream) {
+  if (!q || !kv_pool || !page_table || !tok_row || !tok_pos || !out || T < 1 || H < 1 || KV < 1 || H % KV || max_pages < 1)
+    return RSD_ERR_ARG;
+  if (hd != 64 && hd != 128) return RSD_ERR_UNSUPPORTED;
+  if (dtype < 0 || dtype > 2) return RSD_ERR_ARG;
+  PassView p{nullptr, tok_row, tok_pos, T, nullptr};
+  KvView kv{const_cast<void*>(kv_pool), page_table, max_pages};
+  KCU(launch_attn_chunk(dtype, q, p, kv, out, nullptr, RSD_F32, H, KV, hd, (cudaStream_t)cuda_stream));
+  return RSD_OK;
+}
+
 int rsd_k_gate_compact(const float* rewards, const uint8_t* live, float delta, uint8_t* accept, int32_t* rej_idx,
                        int32_t* n_rej, int32_t B, void* scratch, size_t scratch_bytes, void* cuda_stream) {
   if (!rewards || !live || !accept || !rej_idx || !n_rej || B < 1 || B > (1 << 24)) return RSD_ERR_ARG;

@@ -219,3 +219,35 @@ def test_decode_attention_against_definition(dtype, hd, H, KV):
             p = np.exp(s - s.max()); p /= p.sum()
             want = p @ Vs[b][:, g].astype(np.float64)
             np.testing.assert_allclose(got[b, h], want, rtol=0, atol=tol)
+
+
+@pytest.mark.parametrize("dtype,hd,H,KV", [(torch.float16, 128, 12, 2), (torch.float16, 128, 28, 4), (torch.float16, 64, 4, 2),
+                                          (torch.float32, 64, 4, 2), (torch.float16, 128, 64, 8)])
+def test_chunk_attention_against_definition(dtype, hd, H, KV):
+    """Ragged chunks of several rows in one list: tiles that straddle rows, a chunk that starts in the
+    middle of a page, long prefixes, one idle entry; every query against brute-force causal softmax."""
+    rng = np.random.default_rng(8)
+    ctx = [40, 1, 300, 17, 1031]                # cached positions per row after the chunk was written
+    new = [40, 1, 37, 5, 70]                    # the last `new` positions of each row are the chunk
+    B = len(ctx)
+    max_pages = 70
+    pool, table, Ks, Vs = paged_kv(rng, B, KV, hd, ctx, dtype, max_pages)
+    rows, poss = [], []
+    for b in range(B):
+        for p in range(ctx[b] - new[b], ctx[b]):
+            rows.append(b); poss.append(p)
+    rows.insert(45, -1); poss.insert(45, 0)     # an idle entry in the middle of the list
+    T = len(rows)
+    q = rng.normal(size=(T, H, hd)).astype(np.float32)
+    got = rb.k_attn_chunk(dev(q), pool, table, dev(np.array(rows, np.int32)), dev(np.array(poss, np.int32)), KV).cpu().numpy()
+    tol = 2e-5 if dtype == torch.float32 else 2e-3
+    for t in range(T):
+        b, p = rows[t], poss[t]
+        if b < 0:
+            continue
+        for h in range(0, H, max(1, H // 6)):
+            g = h // (H // KV)
+            s = Ks[b][:p + 1, g].astype(np.float64) @ q[t, h].astype(np.float64) / np.sqrt(hd)
+            w = np.exp(s - s.max()); w /= w.sum()
+            want = w @ Vs[b][:p + 1, g].astype(np.float64)
+            np.testing.assert_allclose(got[t, h], want, rtol=0, atol=tol)

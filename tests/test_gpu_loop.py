@@ -129,3 +129,47 @@ def test_general_acceptance_criterion_on_gpu(omega_kind, delta, alpha):
         seen.update(g["accept"][g["step_len"] > 0].tolist())
     assert seen == {0, 1}                             # both outcomes occurred
     compare_counters(eng, loop)
+
+
+def test_reset_and_new_batch_sizes_reuse_one_context():
+    """rsd_reset / a second rsd_prefill with another batch size on the same context: pages return to the
+    pool, the captured decode graphs are rebuilt for the new slot count, results match a fresh oracle."""
+    from oracle.rsd_loop import OracleRSD
+    base = dict(max_step_tokens=6, max_steps=3, max_seq_tokens=64, step_end_id=5, step_end_mod=9, temperature=0.7, seed=8)
+    p4 = ri.prompts(21, 4, 8, 20, 4096)
+    eng, loop = build_pair(MINI, bf16=True, prompts=p4, loop_kwargs=base, engine_kwargs=dict(max_batch=6))
+    for _ in range(2):
+        parity_step(eng, loop, 0.45, **TOL16)
+    for seed, B in ((22, 6), (23, 2)):
+        tokens, offsets = ri.prompts(seed, B, 8, 20, 4096)
+        eng.prefill(tokens, offsets)                     # drops the old rows
+        assert eng.counters()["steps"] == 0
+        loop = OracleRSD(*loop.models, loop.cfg)
+        loop.prefill([tokens[offsets[b]:offsets[b + 1]].tolist() for b in range(B)])
+        compare_state(eng, loop)
+        for _ in range(2):
+            parity_step(eng, loop, 0.45, **TOL16)
+        compare_counters(eng, loop)
+
+
+def test_call_order_and_argument_errors():
+    from paper_2501_19324_b200 import Engine, Model, RsdError
+    sh = ri.SHAPES["tiny_draft"]
+    models = [Model(sh, ri.gpu_model_tensors(sh, slot, 0, False, hk), hk)
+              for slot, hk in enumerate((ri.HEAD_LM, ri.HEAD_REWARD_SIGMOID, ri.HEAD_LM))]
+    eng = Engine(*models, max_batch=2, max_seq_tokens=48, max_step_tokens=8, max_steps=2, step_end_id=13)
+    eng.B = 2
+    with pytest.raises(RsdError) as e:
+        eng.step(0.5)                                    # step before prefill
+    assert e.value.code == -2
+    with pytest.raises(RsdError) as e:
+        eng.prefill(np.array([1, 2, 5000], np.int32), np.array([0, 2, 3], np.int32))    # id beyond the vocabulary
+    assert e.value.code == -1
+    with pytest.raises(RsdError) as e:
+        eng.prefill(np.arange(6, dtype=np.int32), np.array([0, 2, 4, 6], np.int32))      # more rows than max_batch
+    assert e.value.code == -1
+    eng.prefill(np.array([1, 2, 3, 4], np.int32), np.array([0, 2, 4], np.int32))          # still usable afterwards
+    r = eng.step(0.0)
+    assert r["accept"].all() and (r["step_len"] > 0).all()
+    with pytest.raises(RsdError):                        # a PRM must not carry an lm head, and vice versa
+        Engine(models[0], models[0], models[2], max_batch=2, max_seq_tokens=48, max_step_tokens=8, max_steps=2, step_end_id=13)
