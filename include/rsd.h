@@ -43,7 +43,8 @@ enum {
   RSD_ERR_UNSUPPORTED = -6  /* shape or option the kernels do not cover                   */
 };
 
-enum { RSD_F32 = 0, RSD_BF16 = 1, RSD_F16 = 2 /* KV caches only */ };
+enum { RSD_F32 = 0, RSD_BF16 = 1, RSD_F16 = 2 /* KV caches only */, RSD_F16_EXT = 3 /* fp16 cache whose pages carry
+       two more blocks with the low halves of keys and values; queries and softmax weights as hi + lo */ };
 enum { RSD_DRAFT = 0, RSD_PRM = 1, RSD_TARGET = 2 };
 enum { RSD_HEAD_LM = 0, RSD_HEAD_REWARD_SIGMOID = 1, RSD_HEAD_REWARD_RAW = 2 };
 
@@ -90,6 +91,11 @@ typedef struct {
   float omega_alpha;          /* alpha of RSD_OMEGA_LOGISTIC                                 */
   int32_t max_chunk_tokens;   /* tokens pushed through a model per multi-token pass; 0 = 4096 */
   int32_t debug_flags;        /* RSD_DEBUG_*                                                 */
+  int32_t kv_extended;        /* bf16 models only.  0: fp16 keys and values, fp16 queries and softmax
+                                 weights in the attention products.  1: keys and values are cached as
+                                 fp16 hi + lo pairs (twice the KV bytes) and queries / softmax weights
+                                 enter as hi + lo pairs (attention accurate to ~2^-20); for deep models
+                                 whose logits must stay within 3e-2 of an fp64 reference               */
   /* caller-allocated device memory, sizes as reported by rsd_query_sizes (or larger)        */
   void* kv_pool[3];           /* RSD_DRAFT / RSD_PRM / RSD_TARGET                            */
   size_t kv_bytes[3];
@@ -199,7 +205,8 @@ size_t rsd_k_gemm_scratch_bytes(int32_t M, int32_t N, int32_t K);
 
 /* Paged-KV grouped-query decode attention: one query per row.  q [B, H, hd] fp32; kv pool of pages,
  * each page = keys [KV][16 tokens][hd] followed by values transposed [KV][hd][16 tokens], of
- * `dtype` (RSD_F32, RSD_BF16 or RSD_F16); page_table [B, max_pages]; ctx_len [B] (number of cached
+ * `dtype` (RSD_F32, RSD_BF16, RSD_F16 or RSD_F16_EXT, which adds the blocks keys_lo and values_lo after the
+ * first two); page_table [B, max_pages]; ctx_len [B] (number of cached
  * positions attended; rows with ctx_len < 1 are skipped); out [B, H, hd] fp32.  16-bit caches with
  * H / KV <= 8 take the tensor-core split-context kernel, everything else a generic kernel.  The
  * step loop keeps fp16 caches for bf16 models (same bytes, three more mantissa bits).                                   */

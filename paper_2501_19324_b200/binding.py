@@ -38,7 +38,7 @@ class rsd_config(ctypes.Structure):
     _fields_ = [(n, c_int32) for n in ("max_batch", "max_seq_tokens", "max_step_tokens", "max_steps", "page_tokens",
                                         "step_end_id", "eos_id", "step_end_mod")] + \
                [("temperature", c_float), ("seed", c_uint64), ("omega_kind", c_int32), ("omega_alpha", c_float),
-                ("max_chunk_tokens", c_int32), ("debug_flags", c_int32),
+                ("max_chunk_tokens", c_int32), ("debug_flags", c_int32), ("kv_extended", c_int32),
                 ("kv_pool", c_void_p * 3), ("kv_bytes", c_size_t * 3), ("workspace", c_void_p),
                 ("workspace_bytes", c_size_t)]
 
@@ -152,7 +152,7 @@ class Engine:
 
     def __init__(self, draft: Model, prm: Model, target: Model, *, max_batch, max_seq_tokens, max_step_tokens,
                  max_steps, step_end_id, eos_id=-1, step_end_mod=0, temperature=0.0, seed=0, omega_kind=1,
-                 omega_alpha=0.0, max_chunk_tokens=0, debug_flags=0, kv_bytes=None):
+                 omega_alpha=0.0, max_chunk_tokens=0, debug_flags=0, kv_bytes=None, kv_extended=0):
         import torch
         if not torch.cuda.is_available():
             raise RsdError(-4, "no CUDA device: this library has no CPU fallback")
@@ -160,7 +160,7 @@ class Engine:
         self.B_max, self.S, self.C = max_batch, max_seq_tokens, max_step_tokens
         self.max_pages = (max_seq_tokens + 15) // 16
         cfg = rsd_config(max_batch, max_seq_tokens, max_step_tokens, max_steps, 16, step_end_id, eos_id, step_end_mod,
-                         temperature, seed, omega_kind, omega_alpha, max_chunk_tokens, debug_flags)
+                         temperature, seed, omega_kind, omega_alpha, max_chunk_tokens, debug_flags, kv_extended)
         _check(lib().rsd_query_sizes(draft.desc, prm.desc, target.desc, cfg))
         if kv_bytes is not None:
             for i in range(3):
@@ -282,7 +282,7 @@ def k_gemm(W, x, y=None, accumulate=False, impl=0, x_lo=None):
     return y
 
 
-def k_attn_decode(q, kv_pool, page_table, ctx_len, KV):
+def k_attn_decode(q, kv_pool, page_table, ctx_len, KV, ext=False):
     import torch
     B, H, hd = q.shape
     max_pages = page_table.shape[1]
@@ -290,16 +290,20 @@ def k_attn_decode(q, kv_pool, page_table, ctx_len, KV):
     nbytes = lib().rsd_k_attn_decode_scratch_bytes(B, H, hd, max_pages * 16)
     scratch = torch.zeros(nbytes, dtype=torch.uint8, device=q.device)
     dt = {torch.bfloat16: RSD_BF16, torch.float16: 2, torch.float32: RSD_F32}[kv_pool.dtype]
+    if ext:
+        dt = 3
     _check(lib().rsd_k_attn_decode(_ptr(q), _ptr(kv_pool), _ptr(page_table), _ptr(ctx_len), _ptr(out), B, H, KV, hd,
                                    max_pages, dt, _ptr(scratch), nbytes, _stream()))
     return out
 
 
-def k_attn_chunk(q, kv_pool, page_table, tok_row, tok_pos, KV):
+def k_attn_chunk(q, kv_pool, page_table, tok_row, tok_pos, KV, ext=False):
     import torch
     T, H, hd = q.shape
     out = torch.zeros_like(q)
     dt = {torch.bfloat16: RSD_BF16, torch.float16: 2, torch.float32: RSD_F32}[kv_pool.dtype]
+    if ext:
+        dt = 3
     _check(lib().rsd_k_attn_chunk(_ptr(q), _ptr(kv_pool), _ptr(page_table), _ptr(tok_row), _ptr(tok_pos), _ptr(out), T, H, KV,
                                   hd, page_table.shape[1], dt, _stream()))
     return out

@@ -135,9 +135,10 @@ double count_params(const rsd_model& m) {
   return (double)m.vocab * d + m.n_layers * per_layer + d + head;
 }
 
-size_t kv_pool_bytes(const rsd_model& m, int pages) {
+size_t kv_pool_bytes(const rsd_model& m, int pages, int kv_extended) {
   const size_t elem = m.dtype == RSD_BF16 ? 2 : 4;
-  return (size_t)pages * m.n_layers * 2 * m.n_kv_heads * kPageTokens * m.head_dim * elem;
+  const size_t blocks = (m.dtype == RSD_BF16 && kv_extended) ? 4 : 2;   // keys, values (, their low halves)
+  return (size_t)pages * m.n_layers * blocks * m.n_kv_heads * kPageTokens * m.head_dim * elem;
 }
 
 struct Dims {
@@ -331,7 +332,7 @@ int forward_pass(rsd_ctx* c, int which, PassView p, cudaStream_t s) {
   const bool defer_small = false;
   SplitSum x_pending;   // partial sums of the last GEMM that adds into the residual stream
   for (int l = 0; l < m.n_layers; ++l) {
-    KvView kv{M.kv_pool + (size_t)l * M.layer_stride, c->st.page_table[which], c->max_pages};
+    KvView kv{M.kv_pool + (size_t)l * M.layer_stride, c->st.page_table[which], c->max_pages, M.kv_dtype == 3 ? 1 : 0};
     CU(launch_rmsnorm(m.dtype, c->x, M.norm1[l], c->h, h_lo, T, d, m.rms_eps, nullptr, p.n_active, x_pending, s));
     SplitSum qkv_pending;
     int rc = gemm(c, M, M.wqkv[l], c->h, h_lo, c->qkv, T, (H + 2 * KV) * hd, d, 0, p.n_active, defer_small ? &qkv_pending : nullptr, s);
@@ -515,7 +516,7 @@ int rsd_query_sizes(const rsd_model* draft, const rsd_model* prm, const rsd_mode
     if (rc) return fail(nullptr, rc, "model: %s", why);
   }
   const int max_pages = (cfg->max_seq_tokens + kPageTokens - 1) / kPageTokens;
-  for (int i = 0; i < 3; ++i) cfg->kv_bytes[i] = kv_pool_bytes(*ms[i], cfg->max_batch * max_pages);
+  for (int i = 0; i < 3; ++i) cfg->kv_bytes[i] = kv_pool_bytes(*ms[i], cfg->max_batch * max_pages, cfg->kv_extended);
   cfg->workspace_bytes = layout_workspace(*cfg, ms, nullptr);
   return RSD_OK;
 }
@@ -574,13 +575,13 @@ int rsd_load_models(rsd_ctx* c, const rsd_model* draft, const rsd_model* prm, co
     M.m.wqkv = M.wqkv.data(); M.m.wo = M.wo.data(); M.m.wgu = M.wgu.data(); M.m.wdown = M.wdown.data();
     M.m.norm1 = M.norm1.data(); M.m.norm2 = M.norm2.data();
     M.elem = M.m.dtype == RSD_BF16 ? 2 : 4;
-    M.kv_dtype = M.m.dtype == RSD_BF16 ? 2 : 0;
+    M.kv_dtype = M.m.dtype == RSD_BF16 ? (c->cfg.kv_extended ? 3 : 2) : 0;
     // hi + lo operands for every bf16 model: with plain bf16 operands a 7B-shape PRM misses the
     // 1e-2 reward bound (1.1e-2 measured), a 1.5B-shape one would pass (1.5e-3)
     M.split = M.m.dtype == RSD_BF16;
     M.n_params = count_params(M.m);
     M.kv_pool = (char*)c->cfg.kv_pool[w];
-    const size_t page_bytes = (size_t)2 * M.m.n_kv_heads * kPageTokens * M.m.head_dim * M.elem;
+    const size_t page_bytes = (size_t)(M.kv_dtype == 3 ? 4 : 2) * M.m.n_kv_heads * kPageTokens * M.m.head_dim * M.elem;
     int pages = (int)std::min<size_t>(c->cfg.kv_bytes[w] / (page_bytes * L), (size_t)c->B_max * max_pages);
     if (pages < 1) return fail(c, RSD_ERR_OOM_PAGES, "KV pool too small for a single page%s");
     M.pool_pages = pages;
@@ -901,7 +902,7 @@ int rsd_k_attn_decode(const float* q, const void* kv_pool, const int32_t* page_t
     return RSD_ERR_ARG;
   if (hd != 64 && hd != 128) return RSD_ERR_UNSUPPORTED;
   if (scratch_bytes < attn_decode_scratch_bytes(B, H, hd, max_pages * kPageTokens) || !scratch) return RSD_ERR_ARG;
-  if (dtype < 0 || dtype > 2) return RSD_ERR_ARG;
+  if (dtype < 0 || dtype > 3) return RSD_ERR_ARG;
   KCU(launch_attn_decode(dtype, q, kv_pool, page_table, max_pages, nullptr, ctx_len, 0, out, nullptr, RSD_F32, B, H, KV, hd,
                          max_pages * kPageTokens, scratch, scratch_bytes, nullptr, (cudaStream_t)cuda_stream));
   return RSD_OK;
@@ -913,7 +914,7 @@ int rsd_k_attn_chunk(const float* q, const void* kv_pool, const int32_t* page_ta
   if (!q || !kv_pool || !page_table || !tok_row || !tok_pos || !out || T < 1 || H < 1 || KV < 1 || H % KV || max_pages < 1)
     return RSD_ERR_ARG;
   if (hd != 64 && hd != 128) return RSD_ERR_UNSUPPORTED;
-  if (dtype < 0 || dtype > 2) return RSD_ERR_ARG;
+  if (dtype < 0 || dtype > 3) return RSD_ERR_ARG;
   PassView p{nullptr, tok_row, tok_pos, T, nullptr};
   KvView kv{const_cast<void*>(kv_pool), page_table, max_pages};
   KCU(launch_attn_chunk(dtype, q, p, kv, out, nullptr, RSD_F32, H, KV, hd, (cudaStream_t)cuda_stream));

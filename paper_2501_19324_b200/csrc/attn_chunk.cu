@@ -27,6 +27,11 @@ template <> __device__ __forceinline__ uint32_t pack2c<__half>(float lo, float h
   __half2 v = __floats2half2_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
 }
+template <typename KT> __device__ __forceinline__ void pack2c_split(float a, float b, uint32_t& hi, uint32_t& lo) {
+  const KT ah = from_f32<KT>(a), bh = from_f32<KT>(b);
+  hi = pack2c<KT>(to_f32(ah), to_f32(bh));
+  lo = pack2c<KT>(a - to_f32(ah), b - to_f32(bh));
+}
 template <typename KT>
 __device__ __forceinline__ void mma_c(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1);
 template <>
@@ -44,7 +49,9 @@ __device__ __forceinline__ void mma_c<__half>(float (&d)[4], uint32_t a0, uint32
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-template <int HD, typename KT, typename OT>
+// EXT: hi + lo pairs for the queries and the softmax weights, low halves of the values in a third block
+// of every page (see the decode kernel).
+template <int HD, typename KT, typename OT, bool EXT>
 __global__ void __launch_bounds__(256)
 attn_chunk_kernel(const float* __restrict__ q, PassView p, const KT* __restrict__ pool, const int32_t* __restrict__ page_table,
                   int max_pages, OT* __restrict__ out, OT* __restrict__ out_lo, int H, int KV) {
@@ -58,7 +65,8 @@ attn_chunk_kernel(const float* __restrict__ q, PassView p, const KT* __restrict_
   const int n_tile = min(16, p.T - t0);
   const int g = lane >> 2, t = lane & 3;
   const float scale = rsqrtf((float)HD);
-  const size_t page_elems = (size_t)2 * KV * kPageTokens * HD;
+  const size_t block_elems = (size_t)KV * kPageTokens * HD;
+  const size_t page_elems = (EXT ? 4 : 2) * block_elems;
   // key tokens of a page whose scores this lane holds: 4t, 4t+1 (first MMA tile), 4t+2, 4t+3 (second)
   const int tok0 = 4 * (g >> 1) + (g & 1), tok1 = tok0 + 2;
 
@@ -75,7 +83,7 @@ attn_chunk_kernel(const float* __restrict__ q, PassView p, const KT* __restrict_
     // the two query rows of this lane
     const bool v0 = g >= seg && g < seg_end, v1 = g + 8 >= seg && g + 8 < seg_end;
     const int pq0 = v0 ? p.tok_pos[t0 + g] : pos_last, pq1 = v1 ? p.tok_pos[t0 + g + 8] : pos_last;
-    uint32_t qa[KB][2][4];
+    uint32_t qa[KB][2][4], ql[EXT ? KB : 1][2][4];
 #pragma unroll
     for (int j = 0; j < KB; ++j) {
       float a[8], b[8];
@@ -84,10 +92,17 @@ attn_chunk_kernel(const float* __restrict__ q, PassView p, const KT* __restrict_
         a[e] = v0 ? q[((size_t)(t0 + g) * H + h) * HD + 32 * j + 8 * t + e] : 0.f;
         b[e] = v1 ? q[((size_t)(t0 + g + 8) * H + h) * HD + 32 * j + 8 * t + e] : 0.f;
       }
-      qa[j][0][0] = pack2c<KT>(a[0], a[1]); qa[j][0][1] = pack2c<KT>(b[0], b[1]);
-      qa[j][0][2] = pack2c<KT>(a[2], a[3]); qa[j][0][3] = pack2c<KT>(b[2], b[3]);
-      qa[j][1][0] = pack2c<KT>(a[4], a[5]); qa[j][1][1] = pack2c<KT>(b[4], b[5]);
-      qa[j][1][2] = pack2c<KT>(a[6], a[7]); qa[j][1][3] = pack2c<KT>(b[6], b[7]);
+      if (EXT) {
+        pack2c_split<KT>(a[0], a[1], qa[j][0][0], ql[j][0][0]); pack2c_split<KT>(b[0], b[1], qa[j][0][1], ql[j][0][1]);
+        pack2c_split<KT>(a[2], a[3], qa[j][0][2], ql[j][0][2]); pack2c_split<KT>(b[2], b[3], qa[j][0][3], ql[j][0][3]);
+        pack2c_split<KT>(a[4], a[5], qa[j][1][0], ql[j][1][0]); pack2c_split<KT>(b[4], b[5], qa[j][1][1], ql[j][1][1]);
+        pack2c_split<KT>(a[6], a[7], qa[j][1][2], ql[j][1][2]); pack2c_split<KT>(b[6], b[7], qa[j][1][3], ql[j][1][3]);
+      } else {
+        qa[j][0][0] = pack2c<KT>(a[0], a[1]); qa[j][0][1] = pack2c<KT>(b[0], b[1]);
+        qa[j][0][2] = pack2c<KT>(a[2], a[3]); qa[j][0][3] = pack2c<KT>(b[2], b[3]);
+        qa[j][1][0] = pack2c<KT>(a[4], a[5]); qa[j][1][1] = pack2c<KT>(b[4], b[5]);
+        qa[j][1][2] = pack2c<KT>(a[6], a[7]); qa[j][1][3] = pack2c<KT>(b[6], b[7]);
+      }
     }
     float o[NT][4];
 #pragma unroll
@@ -107,6 +122,18 @@ attn_chunk_kernel(const float* __restrict__ q, PassView p, const KT* __restrict_
         mma_c<KT>(s0, qa[j][1][0], qa[j][1][1], qa[j][1][2], qa[j][1][3], k0.z, k0.w);
         mma_c<KT>(s1, qa[j][0][0], qa[j][0][1], qa[j][0][2], qa[j][0][3], k1.x, k1.y);
         mma_c<KT>(s1, qa[j][1][0], qa[j][1][1], qa[j][1][2], qa[j][1][3], k1.z, k1.w);
+        if (EXT) {
+          const uint4 e0 = *reinterpret_cast<const uint4*>(kb + 2 * block_elems + tok0 * HD + 32 * j + 8 * t);
+          const uint4 e1 = *reinterpret_cast<const uint4*>(kb + 2 * block_elems + tok1 * HD + 32 * j + 8 * t);
+          mma_c<KT>(s0, qa[j][0][0], qa[j][0][1], qa[j][0][2], qa[j][0][3], e0.x, e0.y);
+          mma_c<KT>(s0, qa[j][1][0], qa[j][1][1], qa[j][1][2], qa[j][1][3], e0.z, e0.w);
+          mma_c<KT>(s1, qa[j][0][0], qa[j][0][1], qa[j][0][2], qa[j][0][3], e1.x, e1.y);
+          mma_c<KT>(s1, qa[j][1][0], qa[j][1][1], qa[j][1][2], qa[j][1][3], e1.z, e1.w);
+          mma_c<KT>(s0, ql[j][0][0], ql[j][0][1], ql[j][0][2], ql[j][0][3], k0.x, k0.y);
+          mma_c<KT>(s0, ql[j][1][0], ql[j][1][1], ql[j][1][2], ql[j][1][3], k0.z, k0.w);
+          mma_c<KT>(s1, ql[j][0][0], ql[j][0][1], ql[j][0][2], ql[j][0][3], k1.x, k1.y);
+          mma_c<KT>(s1, ql[j][1][0], ql[j][1][1], ql[j][1][2], ql[j][1][3], k1.z, k1.w);
+        }
       }
       // scores of query g: sa[e], of query g+8: sb[e], for key tokens base + 4t + e
       const int base = pg * kPageTokens + 4 * t;
@@ -129,8 +156,14 @@ attn_chunk_kernel(const float* __restrict__ q, PassView p, const KT* __restrict_
       l0 = l0 * ca + (pa[0] + pa[1] + pa[2] + pa[3]);
       l1 = l1 * cb + (pb[0] + pb[1] + pb[2] + pb[3]);
       m0 = na; m1 = nb;
-      const uint32_t a0 = pack2c<KT>(pa[0], pa[1]), a1 = pack2c<KT>(pb[0], pb[1]);
-      const uint32_t a2 = pack2c<KT>(pa[2], pa[3]), a3 = pack2c<KT>(pb[2], pb[3]);
+      uint32_t a0, a1, a2, a3, l0p = 0u, l1p = 0u, l2p = 0u, l3p = 0u;
+      if (EXT) {
+        pack2c_split<KT>(pa[0], pa[1], a0, l0p); pack2c_split<KT>(pb[0], pb[1], a1, l1p);
+        pack2c_split<KT>(pa[2], pa[3], a2, l2p); pack2c_split<KT>(pb[2], pb[3], a3, l3p);
+      } else {
+        a0 = pack2c<KT>(pa[0], pa[1]); a1 = pack2c<KT>(pb[0], pb[1]);
+        a2 = pack2c<KT>(pa[2], pa[3]); a3 = pack2c<KT>(pb[2], pb[3]);
+      }
       // values of tokens beyond the last cached position of the row may be uninitialised memory
       const int n_valid = min(kPageTokens, pos_last + 1 - pg * kPageTokens);
       uint32_t mlo = 0xFFFFFFFFu, mhi = 0xFFFFFFFFu;
@@ -143,6 +176,11 @@ attn_chunk_kernel(const float* __restrict__ q, PassView p, const KT* __restrict_
         const uint2 vv = *reinterpret_cast<const uint2*>(vb + (size_t)(8 * i + g) * kPageTokens + 4 * t);
         o[i][0] *= ca; o[i][1] *= ca; o[i][2] *= cb; o[i][3] *= cb;
         mma_c<KT>(o[i], a0, a1, a2, a3, vv.x & mlo, vv.y & mhi);
+        if (EXT) {
+          const uint2 vl = *reinterpret_cast<const uint2*>(vb + 2 * block_elems + (size_t)(8 * i + g) * kPageTokens + 4 * t);
+          mma_c<KT>(o[i], l0p, l1p, l2p, l3p, vv.x & mlo, vv.y & mhi);
+          mma_c<KT>(o[i], a0, a1, a2, a3, vl.x & mlo, vl.y & mhi);
+        }
       }
     }
     l0 += __shfl_xor_sync(0xFFFFFFFFu, l0, 1); l0 += __shfl_xor_sync(0xFFFFFFFFu, l0, 2);
@@ -171,14 +209,17 @@ cudaError_t launch_attn_chunk(int kv_dtype, const float* q, PassView p, KvView k
                               int out_dtype, int H, int KV, int hd, cudaStream_t s) {
   if (p.T <= 0) return cudaSuccess;
   const int G = H / KV;
-  if (kv_dtype == 0 || G > 8) return launch_attn_generic(kv_dtype, q, p, kv, out, out_lo, out_dtype, H, KV, hd, s);
+  if (kv_dtype == 3) kv.v_extra = 1;
+  if (kv_dtype == 0 || G > 8)
+    return launch_attn_generic(kv_dtype == 3 ? 2 : kv_dtype, q, p, kv, out, out_lo, out_dtype, H, KV, hd, s);
   dim3 grid((p.T + 15) / 16, KV);
   const int threads = 32 * G;
-#define RSD_CH(HD, KT, OT) \
-  RSD_LAUNCH((attn_chunk_kernel<HD, KT, OT>), grid, threads, 0, s, q, p, (const KT*)kv.pool_layer, kv.page_table, kv.max_pages, (OT*)out, (OT*)out_lo, H, KV)
-#define RSD_CH_O(HD, KT) do { if (out_dtype == 1) RSD_CH(HD, KT, __nv_bfloat16); else RSD_CH(HD, KT, float); } while (0)
-  if (kv_dtype == 2) { if (hd == 128) RSD_CH_O(128, __half); else RSD_CH_O(64, __half); }
-  else { if (hd == 128) RSD_CH_O(128, __nv_bfloat16); else RSD_CH_O(64, __nv_bfloat16); }
+#define RSD_CH(HD, KT, OT, EXTV) \
+  RSD_LAUNCH((attn_chunk_kernel<HD, KT, OT, EXTV>), grid, threads, 0, s, q, p, (const KT*)kv.pool_layer, kv.page_table, kv.max_pages, (OT*)out, (OT*)out_lo, H, KV)
+#define RSD_CH_O(HD, KT, EXTV) do { if (out_dtype == 1) RSD_CH(HD, KT, __nv_bfloat16, EXTV); else RSD_CH(HD, KT, float, EXTV); } while (0)
+  if (kv_dtype == 3) { if (hd == 128) RSD_CH_O(128, __half, true); else RSD_CH_O(64, __half, true); }
+  else if (kv_dtype == 2) { if (hd == 128) RSD_CH_O(128, __half, false); else RSD_CH_O(64, __half, false); }
+  else { if (hd == 128) RSD_CH_O(128, __nv_bfloat16, false); else RSD_CH_O(64, __nv_bfloat16, false); }
 #undef RSD_CH_O
 #undef RSD_CH
   return launched(1);

@@ -33,6 +33,13 @@ template <> __device__ __forceinline__ uint32_t pack2<__half>(float lo, float hi
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
+// The same pair split into a high and a low 16-bit part: (a, b) = hi + lo up to ~2^-22 relative.
+template <typename KT> __device__ __forceinline__ void pack2_split(float a, float b, uint32_t& hi, uint32_t& lo) {
+  const KT ah = from_f32<KT>(a), bh = from_f32<KT>(b);
+  hi = pack2<KT>(to_f32(ah), to_f32(bh));
+  lo = pack2<KT>(a - to_f32(ah), b - to_f32(bh));
+}
+
 template <typename KT>
 __device__ __forceinline__ void mma_16816(float& d0, float& d1, float& d2, float& d3, uint32_t a0, uint32_t a1, uint32_t a2,
                                           uint32_t a3, uint32_t b0, uint32_t b1);
@@ -54,8 +61,10 @@ __device__ __forceinline__ void mma_16816<__half>(float& d0, float& d1, float& d
 }
 
 // part_o: [slot][head][split][HD] un-normalised outputs; part_ml: [slot][head][split][2] (max, sum).
-template <int HD, typename KT, typename OT>
-__global__ void __launch_bounds__(128, 4)
+// EXT: queries and softmax weights enter the products as hi + lo pairs and every page carries the low
+// halves of its keys and values in two more blocks: the attention is accurate to about 2^-20.
+template <int HD, typename KT, typename OT, bool EXT>
+__global__ void __launch_bounds__(128, EXT ? 2 : 4)
 attn_decode_kernel(const float* __restrict__ q, const KT* __restrict__ pool, const int32_t* __restrict__ page_table,
                    int max_pages, const int32_t* __restrict__ slot_row, const int32_t* __restrict__ len_or_pos, int len_offset,
                    OT* __restrict__ out, OT* __restrict__ out_lo, float* __restrict__ part_o, float* __restrict__ part_ml, int H, int KV, int n_splits,
@@ -81,14 +90,19 @@ attn_decode_kernel(const float* __restrict__ q, const KT* __restrict__ pool, con
   const int p_begin = split * pps, p_end = min(n_pages, p_begin + pps);
 
   // Q fragments (rows 8..15 of the tile are padding): dims 32j + 8t + e of head h0 + g
-  uint32_t qa[KB][2][2];
+  uint32_t qa[KB][2][2], ql[EXT ? KB : 1][2][2];
 #pragma unroll
   for (int j = 0; j < KB; ++j) {
     float v[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) v[e] = g < G ? q[((size_t)slot * H + h0 + g) * HD + 32 * j + 8 * t + e] : 0.f;
-    qa[j][0][0] = pack2<KT>(v[0], v[1]); qa[j][0][1] = pack2<KT>(v[2], v[3]);
-    qa[j][1][0] = pack2<KT>(v[4], v[5]); qa[j][1][1] = pack2<KT>(v[6], v[7]);
+    if (EXT) {
+      pack2_split<KT>(v[0], v[1], qa[j][0][0], ql[j][0][0]); pack2_split<KT>(v[2], v[3], qa[j][0][1], ql[j][0][1]);
+      pack2_split<KT>(v[4], v[5], qa[j][1][0], ql[j][1][0]); pack2_split<KT>(v[6], v[7], qa[j][1][1], ql[j][1][1]);
+    } else {
+      qa[j][0][0] = pack2<KT>(v[0], v[1]); qa[j][0][1] = pack2<KT>(v[2], v[3]);
+      qa[j][1][0] = pack2<KT>(v[4], v[5]); qa[j][1][1] = pack2<KT>(v[6], v[7]);
+    }
   }
   // Rows 8..15 of every MMA tile are padding (their A rows are zero), so all tiles share two dump
   // registers for those rows instead of carrying 2 x (NT + 2) dead accumulators.
@@ -99,7 +113,8 @@ attn_decode_kernel(const float* __restrict__ q, const KT* __restrict__ pool, con
   float m_run = -INFINITY, l_run = 0.f;
 
   const int32_t* pt = page_table + (size_t)row * max_pages;
-  const size_t page_elems = (size_t)2 * KV * kPageTokens * HD;
+  const size_t block_elems = (size_t)KV * kPageTokens * HD;
+  const size_t page_elems = (EXT ? 4 : 2) * block_elems;
   // tokens whose keys this lane loads: tile 0 -> 4(g/2) + g%2, tile 1 -> that + 2
   const int tok0 = 4 * (g >> 1) + (g & 1), tok1 = tok0 + 2;
   int page = (p_begin + warp < p_end) ? pt[p_begin + warp] : 0;
@@ -109,7 +124,7 @@ attn_decode_kernel(const float* __restrict__ q, const KT* __restrict__ pool, con
     if (p + 4 < p_end) page = pt[p + 4];     // next page's index is fetched while this page is worked on
     // all of the page's keys and values are requested up front (8 KB per warp in flight)
     uint4 k0[KB], k1[KB];
-    uint2 vv[NT];
+    uint2 vv[NT], vl[EXT ? NT : 1];
 #pragma unroll
     for (int j = 0; j < KB; ++j) {
       k0[j] = *reinterpret_cast<const uint4*>(kb + tok0 * HD + 32 * j + 8 * t);
@@ -117,6 +132,10 @@ attn_decode_kernel(const float* __restrict__ q, const KT* __restrict__ pool, con
     }
 #pragma unroll
     for (int i = 0; i < NT; ++i) vv[i] = *reinterpret_cast<const uint2*>(vb + (size_t)(8 * i + g) * kPageTokens + 4 * t);
+    if (EXT) {
+#pragma unroll
+      for (int i = 0; i < NT; ++i) vl[i] = *reinterpret_cast<const uint2*>(vb + 2 * block_elems + (size_t)(8 * i + g) * kPageTokens + 4 * t);
+    }
     float s0[2] = {0.f, 0.f}, s1[2] = {0.f, 0.f};
 #pragma unroll
     for (int j = 0; j < KB; ++j) {
@@ -124,6 +143,18 @@ attn_decode_kernel(const float* __restrict__ q, const KT* __restrict__ pool, con
       mma_16816<KT>(s0[0], s0[1], dump0, dump1, qa[j][1][0], 0u, qa[j][1][1], 0u, k0[j].z, k0[j].w);
       mma_16816<KT>(s1[0], s1[1], dump0, dump1, qa[j][0][0], 0u, qa[j][0][1], 0u, k1[j].x, k1[j].y);
       mma_16816<KT>(s1[0], s1[1], dump0, dump1, qa[j][1][0], 0u, qa[j][1][1], 0u, k1[j].z, k1[j].w);
+      if (EXT) {
+        const uint4 e0 = *reinterpret_cast<const uint4*>(kb + 2 * block_elems + tok0 * HD + 32 * j + 8 * t);
+        const uint4 e1 = *reinterpret_cast<const uint4*>(kb + 2 * block_elems + tok1 * HD + 32 * j + 8 * t);
+        mma_16816<KT>(s0[0], s0[1], dump0, dump1, qa[j][0][0], 0u, qa[j][0][1], 0u, e0.x, e0.y);
+        mma_16816<KT>(s0[0], s0[1], dump0, dump1, qa[j][1][0], 0u, qa[j][1][1], 0u, e0.z, e0.w);
+        mma_16816<KT>(s1[0], s1[1], dump0, dump1, qa[j][0][0], 0u, qa[j][0][1], 0u, e1.x, e1.y);
+        mma_16816<KT>(s1[0], s1[1], dump0, dump1, qa[j][1][0], 0u, qa[j][1][1], 0u, e1.z, e1.w);
+        mma_16816<KT>(s0[0], s0[1], dump0, dump1, ql[j][0][0], 0u, ql[j][0][1], 0u, k0[j].x, k0[j].y);
+        mma_16816<KT>(s0[0], s0[1], dump0, dump1, ql[j][1][0], 0u, ql[j][1][1], 0u, k0[j].z, k0[j].w);
+        mma_16816<KT>(s1[0], s1[1], dump0, dump1, ql[j][0][0], 0u, ql[j][0][1], 0u, k1[j].x, k1[j].y);
+        mma_16816<KT>(s1[0], s1[1], dump0, dump1, ql[j][1][0], 0u, ql[j][1][1], 0u, k1[j].z, k1[j].w);
+      }
     }
     // this lane's scores of head g: tokens 4t, 4t+1 (tile 0) and 4t+2, 4t+3 (tile 1) of the page
     const int n_valid = min(kPageTokens, ctx - p * kPageTokens);
@@ -141,7 +172,9 @@ attn_decode_kernel(const float* __restrict__ q, const KT* __restrict__ pool, con
     for (int e = 0; e < 4; ++e) pr[e] = __expf(sc[e] - m_new);
     l_run = l_run * corr + (pr[0] + pr[1] + pr[2] + pr[3]);
     m_run = m_new;
-    const uint32_t pa0 = pack2<KT>(pr[0], pr[1]), pa2 = pack2<KT>(pr[2], pr[3]);
+    uint32_t pa0, pa2, pl0 = 0u, pl2 = 0u;
+    if (EXT) { pack2_split<KT>(pr[0], pr[1], pa0, pl0); pack2_split<KT>(pr[2], pr[3], pa2, pl2); }
+    else { pa0 = pack2<KT>(pr[0], pr[1]); pa2 = pack2<KT>(pr[2], pr[3]); }
     // mask of the 16-bit halves of a value fragment that belong to cached tokens
     uint32_t mlo = 0xFFFFFFFFu, mhi = 0xFFFFFFFFu;
     if (n_valid < kPageTokens) {
@@ -152,6 +185,10 @@ attn_decode_kernel(const float* __restrict__ q, const KT* __restrict__ pool, con
     for (int i = 0; i < NT; ++i) {
       o[i][0] *= corr; o[i][1] *= corr;
       mma_16816<KT>(o[i][0], o[i][1], dump0, dump1, pa0, 0u, pa2, 0u, vv[i].x & mlo, vv[i].y & mhi);
+      if (EXT) {
+        mma_16816<KT>(o[i][0], o[i][1], dump0, dump1, pl0, 0u, pl2, 0u, vv[i].x & mlo, vv[i].y & mhi);
+        mma_16816<KT>(o[i][0], o[i][1], dump0, dump1, pa0, 0u, pa2, 0u, vl[i].x & mlo, vl[i].y & mhi);
+      }
     }
   }
   // the 4 lanes of a row hold partial sums of l
@@ -252,26 +289,27 @@ cudaError_t launch_attn_decode(int kv_dtype, const float* q, const void* pool_la
     RSD_LAUNCH((decode_slots_kernel), (B + 255) / 256, 256, 0, s, slot_row, len_or_pos, len_offset, row, pos, B);
     launched(1);
     PassView p{nullptr, row, pos, B, n_active};
-    KvView kv{const_cast<void*>(pool_layer), page_table, max_pages};
-    return launch_attn_generic(kv_dtype, q, p, kv, out, out_lo, out_dtype, H, KV, hd, s);
+    KvView kv{const_cast<void*>(pool_layer), page_table, max_pages, kv_dtype == 3 ? 1 : 0};
+    return launch_attn_generic(kv_dtype == 3 ? 2 : kv_dtype, q, p, kv, out, out_lo, out_dtype, H, KV, hd, s);
   }
   const size_t head = ((sizeof(int32_t) * 2 * (size_t)B + 255) / 256) * 256;
   float* part_ml = (float*)((char*)scratch + head);
   float* part_o = part_ml + (size_t)B * H * kMaxSplits * 2;
   const int splits = pick_splits(B, KV, max_ctx);
   dim3 grid(KV, B, splits);
-#define RSD_DEC(HD, KT, OT)                                                                                          \
+#define RSD_DEC(HD, KT, OT, EXTV)                                                                                          \
   do {                                                                                                               \
-    RSD_LAUNCH((attn_decode_kernel<HD, KT, OT>), grid, 128, 0, s, q, (const KT*)pool_layer, page_table, max_pages, slot_row,     \
+    RSD_LAUNCH((attn_decode_kernel<HD, KT, OT, EXTV>), grid, 128, 0, s, q, (const KT*)pool_layer, page_table, max_pages, slot_row,     \
                                                         len_or_pos, len_offset, (OT*)out, (OT*)out_lo, part_o, part_ml, \
                                                         H, KV, splits, n_active);                                    \
     if (splits > 1)                                                                                                  \
       RSD_LAUNCH((attn_merge_kernel<HD, OT>), dim3(H, B), HD, 0, s, part_o, part_ml, slot_row, len_or_pos, len_offset, (OT*)out, \
                                                           (OT*)out_lo, H, splits, n_active);                         \
   } while (0)
-#define RSD_DEC_O(HD, KT) do { if (out_dtype == 1) RSD_DEC(HD, KT, __nv_bfloat16); else RSD_DEC(HD, KT, float); } while (0)
-  if (kv_dtype == 2) { if (hd == 128) RSD_DEC_O(128, __half); else RSD_DEC_O(64, __half); }
-  else { if (hd == 128) RSD_DEC_O(128, __nv_bfloat16); else RSD_DEC_O(64, __nv_bfloat16); }
+#define RSD_DEC_O(HD, KT, EXTV) do { if (out_dtype == 1) RSD_DEC(HD, KT, __nv_bfloat16, EXTV); else RSD_DEC(HD, KT, float, EXTV); } while (0)
+  if (kv_dtype == 3) { if (hd == 128) RSD_DEC_O(128, __half, true); else RSD_DEC_O(64, __half, true); }
+  else if (kv_dtype == 2) { if (hd == 128) RSD_DEC_O(128, __half, false); else RSD_DEC_O(64, __half, false); }
+  else { if (hd == 128) RSD_DEC_O(128, __nv_bfloat16, false); else RSD_DEC_O(64, __nv_bfloat16, false); }
 #undef RSD_DEC_O
 #undef RSD_DEC
   return launched(splits > 1 ? 2 : 1);

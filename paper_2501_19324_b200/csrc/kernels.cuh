@@ -40,6 +40,8 @@ struct KvView {
   void* pool_layer;            // slab of the current layer
   const int32_t* page_table;   // [rows, max_pages]
   int max_pages;
+  int v_extra = 0;             // 1: every page carries two more blocks, the low halves of the keys and of
+                               // the values (x = hi + lo, both fp16), laid out like the first two
 };
 
 cudaError_t launch_embed(int dtype, const void* embed, PassView p, float* x, int d, cudaStream_t s);

@@ -224,7 +224,7 @@ template <typename KT>
 __global__ void rope_kv_kernel(const float* __restrict__ qkv, const float* __restrict__ partials, int splits,
                                PassView p, float* __restrict__ q_out, KT* pool,
                                const int32_t* __restrict__ page_table, int max_pages,
-                               const float2* __restrict__ rope, int H, int KV, int hd) {
+                               const float2* __restrict__ rope, int H, int KV, int hd, int pf) {
   RSD_PDL_SYNC();
   RSD_SKIP_IF_IDLE(p.n_active);
   const int t = blockIdx.x;
@@ -239,8 +239,10 @@ __global__ void rope_kv_kernel(const float* __restrict__ qkv, const float* __res
   const int page = page_table[(size_t)row * max_pages + pos / kPageTokens];
   const int slot = pos % kPageTokens;
   // page = K block [KV][16][hd] followed by V block [KV][hd][16] (V transposed within the page)
-  KT* kbase = pool + ((size_t)page * 2 + 0) * KV * kPageTokens * hd;
-  KT* vbase = pool + ((size_t)page * 2 + 1) * KV * kPageTokens * hd;
+  // (pf = 4: two more blocks hold the low halves of the keys and of the values)
+  const size_t block = (size_t)KV * kPageTokens * hd;
+  KT* kbase = pool + (size_t)page * pf * block;
+  KT* vbase = kbase + block;
   const int n_rot = (H + KV) * half;
   for (int idx = threadIdx.x; idx < n_rot; idx += blockDim.x) {
     const int head = idx / half, i = idx % half;
@@ -253,26 +255,33 @@ __global__ void rope_kv_kernel(const float* __restrict__ qkv, const float* __res
       q_out[(size_t)t * H * hd + head * hd + i + half] = rb;
     } else {
       KT* k = kbase + ((size_t)(head - H) * kPageTokens + slot) * hd;
-      k[i] = from_f32<KT>(ra);
-      k[i + half] = from_f32<KT>(rb);
+      const KT ka = from_f32<KT>(ra), kb2 = from_f32<KT>(rb);
+      k[i] = ka;
+      k[i + half] = kb2;
+      if (pf == 4) {
+        k[2 * block + i] = from_f32<KT>(ra - to_f32(ka));
+        k[2 * block + i + half] = from_f32<KT>(rb - to_f32(kb2));
+      }
     }
   }
   for (int idx = threadIdx.x; idx < KV * hd; idx += blockDim.x) {
     const int head = idx / hd, i = idx % hd;
     const float v = split_sum(qkv, partials, splits, src0 + (H + KV) * hd + idx, sstride);
-    vbase[((size_t)head * hd + i) * kPageTokens + slot] = from_f32<KT>(v);
+    const KT vh = from_f32<KT>(v);
+    vbase[((size_t)head * hd + i) * kPageTokens + slot] = vh;
+    if (pf == 4) vbase[2 * block + ((size_t)head * hd + i) * kPageTokens + slot] = from_f32<KT>(v - to_f32(vh));
   }
 }
 
 cudaError_t launch_rope_kv(int kv_dtype, const float* qkv, SplitSum pending, PassView p, float* q_out, KvView kv,
                            const float2* rope, int H, int KV, int hd, cudaStream_t s) {
   if (p.T <= 0) return cudaSuccess;
-  if (kv_dtype == 2)
-    RSD_LAUNCH((rope_kv_kernel<__half>), p.T, 256, 0, s, qkv, pending.partials, pending.splits, p, q_out, (__half*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd);
+  if (kv_dtype == 2 || kv_dtype == 3)
+    RSD_LAUNCH((rope_kv_kernel<__half>), p.T, 256, 0, s, qkv, pending.partials, pending.splits, p, q_out, (__half*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd, 2 + 2 * kv.v_extra);
   else if (kv_dtype == 1)
-    RSD_LAUNCH((rope_kv_kernel<__nv_bfloat16>), p.T, 256, 0, s, qkv, pending.partials, pending.splits, p, q_out, (__nv_bfloat16*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd);
+    RSD_LAUNCH((rope_kv_kernel<__nv_bfloat16>), p.T, 256, 0, s, qkv, pending.partials, pending.splits, p, q_out, (__nv_bfloat16*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd, 2 + 2 * kv.v_extra);
   else
-    RSD_LAUNCH((rope_kv_kernel<float>), p.T, 256, 0, s, qkv, pending.partials, pending.splits, p, q_out, (float*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd);
+    RSD_LAUNCH((rope_kv_kernel<float>), p.T, 256, 0, s, qkv, pending.partials, pending.splits, p, q_out, (float*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd, 2 + 2 * kv.v_extra);
   return launched(1);
 }
 
@@ -306,7 +315,7 @@ template <typename KT, typename OT, int HD>
 __global__ void __launch_bounds__(128)
 attn_generic_kernel(const float* __restrict__ q, PassView p, const KT* __restrict__ pool,
                     const int32_t* __restrict__ page_table, int max_pages, OT* __restrict__ out, OT* __restrict__ out_lo,
-                    int H, int KV) {
+                    int H, int KV, int pf) {
   RSD_PDL_SYNC();
   RSD_SKIP_IF_IDLE(p.n_active);
   constexpr int DPL = HD / 32;
@@ -328,8 +337,9 @@ attn_generic_kernel(const float* __restrict__ q, PassView p, const KT* __restric
   const int32_t* pt = page_table + (size_t)row * max_pages;
   for (int p0 = 0; p0 <= pos; p0 += kPageTokens) {
     const int page = pt[p0 / kPageTokens];
-    const KT* kb = pool + (((size_t)page * 2 + 0) * KV + g) * kPageTokens * HD;
-    const KT* vb = pool + (((size_t)page * 2 + 1) * KV + g) * kPageTokens * HD;
+    const size_t block = (size_t)KV * kPageTokens * HD;
+    const KT* kb = pool + (size_t)page * pf * block + (size_t)g * kPageTokens * HD;
+    const KT* vb = kb + block;
     const int n = min(kPageTokens, pos + 1 - p0);
     float sc[kPageTokens];
 #pragma unroll
@@ -337,7 +347,11 @@ attn_generic_kernel(const float* __restrict__ q, PassView p, const KT* __restric
       float a = 0.f;
       if (j < n) {
 #pragma unroll
-        for (int i = 0; i < DPL; ++i) a = fmaf(qv[i], to_f32(kb[j * HD + lane * DPL + i]), a);
+        for (int i = 0; i < DPL; ++i) {
+          float kk = to_f32(kb[j * HD + lane * DPL + i]);
+          if (pf == 4) kk += to_f32(kb[2 * block + j * HD + lane * DPL + i]);
+          a = fmaf(qv[i], kk, a);
+        }
       }
       sc[j] = a;
     }
@@ -357,7 +371,11 @@ attn_generic_kernel(const float* __restrict__ q, PassView p, const KT* __restric
         const float pj = __expf(sc[j] - mx);
         l += pj;
 #pragma unroll
-        for (int i = 0; i < DPL; ++i) acc[i] = fmaf(pj, to_f32(vb[(lane * DPL + i) * kPageTokens + j]), acc[i]);
+        for (int i = 0; i < DPL; ++i) {
+          float vv = to_f32(vb[(lane * DPL + i) * kPageTokens + j]);
+          if (pf == 4) vv += to_f32(vb[2 * block + (lane * DPL + i) * kPageTokens + j]);
+          acc[i] = fmaf(pj, vv, acc[i]);
+        }
       }
     }
     m = mx;
@@ -373,7 +391,7 @@ cudaError_t launch_attn_generic(int kv_dtype, const float* q, PassView p, KvView
   const int warps = p.T * H;
   const int blocks = (warps + 3) / 4;
 #define RSD_ATTN(KT, OT, HD) \
-  RSD_LAUNCH((attn_generic_kernel<KT, OT, HD>), blocks, 128, 0, s, q, p, (const KT*)kv.pool_layer, kv.page_table, kv.max_pages, (OT*)out, (OT*)out_lo, H, KV)
+  RSD_LAUNCH((attn_generic_kernel<KT, OT, HD>), blocks, 128, 0, s, q, p, (const KT*)kv.pool_layer, kv.page_table, kv.max_pages, (OT*)out, (OT*)out_lo, H, KV, 2 + 2 * kv.v_extra)
 #define RSD_ATTN_HD(KT, OT) do { if (hd == 128) RSD_ATTN(KT, OT, 128); else RSD_ATTN(KT, OT, 64); } while (0)
   using bf = __nv_bfloat16;
   if (kv_dtype == 2) { if (out_dtype == 1) RSD_ATTN_HD(__half, bf); else RSD_ATTN_HD(__half, float); }

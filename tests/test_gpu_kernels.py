@@ -164,13 +164,14 @@ def test_gate_compaction_all_masks_and_large():
     assert acc.cpu().numpy().tolist() == [1, 0, 0] and rej.cpu().numpy()[:2].tolist() == [1, 2]
 
 
-def paged_kv(rng, B, KV, hd, ctx, dtype, max_pages):
-    """Random K/V per row scattered over randomly permuted pages; returns pool, table, dense K, V."""
+def paged_kv(rng, B, KV, hd, ctx, dtype, max_pages, ext=False):
+    """Random K/V per row scattered over randomly permuted pages; returns pool, table, dense K, V.
+    ext: pages carry two more blocks with the low halves of keys and values (x = fp16 hi + fp16 lo)."""
     n_pages_row = [(c + 15) // 16 for c in ctx]
     total = sum(n_pages_row)
     perm = rng.permutation(total + 5)
     # page = keys [KV][16][hd] followed by values transposed [KV][hd][16]; unused slots hold NaN
-    pool = np.full((total + 5, 2, KV * 16 * hd), np.nan, dtype=np.float32)
+    pool = np.full((total + 5, 4 if ext else 2, KV * 16 * hd), np.nan, dtype=np.float32)
     table = np.zeros((B, max_pages), dtype=np.int32)
     Ks, Vs = [], []
     nxt = 0
@@ -183,8 +184,20 @@ def paged_kv(rng, B, KV, hd, ctx, dtype, max_pages):
             n = min(16, ctx[b] - 16 * i)
             kk = pool[pg, 0].reshape(KV, 16, hd)
             vv = pool[pg, 1].reshape(KV, hd, 16)
-            kk[:, :n] = K[16 * i:16 * i + n].transpose(1, 0, 2)
-            vv[:, :, :n] = V[16 * i:16 * i + n].transpose(1, 2, 0)
+            kblk = K[16 * i:16 * i + n].transpose(1, 0, 2)
+            if ext:
+                khi = kblk.astype(np.float16).astype(np.float32)
+                kk[:, :n] = khi
+                pool[pg, 2].reshape(KV, 16, hd)[:, :n] = kblk - khi
+            else:
+                kk[:, :n] = kblk
+            vblk = V[16 * i:16 * i + n].transpose(1, 2, 0)
+            if ext:
+                vhi = vblk.astype(np.float16).astype(np.float32)
+                vv[:, :, :n] = vhi
+                pool[pg, 3].reshape(KV, hd, 16)[:, :, :n] = vblk - vhi
+            else:
+                vv[:, :, :n] = vblk
         Ks.append(K); Vs.append(V)
     pool_d = dev(pool, dtype)
     pool_back = pool_d.float().cpu().numpy()
@@ -193,6 +206,9 @@ def paged_kv(rng, B, KV, hd, ctx, dtype, max_pages):
             n = min(16, ctx[b] - 16 * i)
             Ks[b][16 * i:16 * i + n] = pool_back[table[b, i], 0].reshape(KV, 16, hd)[:, :n].transpose(1, 0, 2)
             Vs[b][16 * i:16 * i + n] = pool_back[table[b, i], 1].reshape(KV, hd, 16)[:, :, :n].transpose(2, 0, 1)
+            if ext:
+                Ks[b][16 * i:16 * i + n] += pool_back[table[b, i], 2].reshape(KV, 16, hd)[:, :n].transpose(1, 0, 2)
+                Vs[b][16 * i:16 * i + n] += pool_back[table[b, i], 3].reshape(KV, hd, 16)[:, :, :n].transpose(2, 0, 1)
     return pool_d, dev(table), Ks, Vs
 
 
@@ -251,3 +267,31 @@ def test_chunk_attention_against_definition(dtype, hd, H, KV):
             w = np.exp(s - s.max()); w /= w.sum()
             want = w @ Vs[b][:p + 1, g].astype(np.float64)
             np.testing.assert_allclose(got[t, h], want, rtol=0, atol=tol)
+
+
+@pytest.mark.parametrize("hd,H,KV", [(128, 12, 2), (128, 64, 8), (64, 4, 2), (128, 16, 1)])
+def test_extended_precision_attention(hd, H, KV):
+    """fp16 cache with keys and values kept as hi + lo pairs, queries and softmax weights as hi + lo
+    pairs: decode and chunk kernels alike agree with the fp64 definition to fp32 accuracy."""
+    rng = np.random.default_rng(12)
+    ctx = [1, 16, 33, 250, 1031]
+    B = len(ctx)
+    pool, table, Ks, Vs = paged_kv(rng, B, KV, hd, ctx, torch.float16, 70, ext=True)
+    q = rng.normal(size=(B, H, hd)).astype(np.float32)
+    got = rb.k_attn_decode(dev(q), pool, table, dev(np.array(ctx, np.int32)), KV, ext=True).cpu().numpy()
+    rows = [b for b in range(B) for _ in range(min(ctx[b], 20))]
+    poss = [p for b in range(B) for p in range(ctx[b] - min(ctx[b], 20), ctx[b])]
+    qc = rng.normal(size=(len(rows), H, hd)).astype(np.float32)
+    gotc = rb.k_attn_chunk(dev(qc), pool, table, dev(np.array(rows, np.int32)), dev(np.array(poss, np.int32)), KV, ext=True).cpu().numpy()
+
+    def ref(b, p, qv, h):
+        g = h // (H // KV)
+        s = Ks[b][:p + 1, g].astype(np.float64) @ qv.astype(np.float64) / np.sqrt(hd)
+        w = np.exp(s - s.max()); w /= w.sum()
+        return w @ Vs[b][:p + 1, g].astype(np.float64)
+    for b in range(B):
+        for h in range(0, H, max(1, H // 4)):
+            np.testing.assert_allclose(got[b, h], ref(b, ctx[b] - 1, q[b, h], h), rtol=0, atol=2e-5)
+    for t in range(0, len(rows), 3):
+        for h in range(0, H, max(1, H // 4)):
+            np.testing.assert_allclose(gotc[t, h], ref(rows[t], poss[t], qc[t, h], h), rtol=0, atol=2e-5)

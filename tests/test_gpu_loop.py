@@ -85,20 +85,23 @@ def test_ragged_steps_eos_and_dead_rows():
     compare_counters(eng, loop)
 
 
-def test_mini_bf16_models():
-    """16-bit weights, head_dim 128, Gumbel-max at T = 0.7, chunked multi-token passes."""
+@pytest.mark.parametrize("kv_extended", [0, 1])
+def test_mini_bf16_models(kv_extended):
+    """16-bit weights, head_dim 128, Gumbel-max at T = 0.7, chunked multi-token passes; with the
+    16-bit KV cache and with the extended one (values as hi + lo pairs)."""
     prompts = ri.prompts(2, 5, 20, 70, 4096)
     base = dict(max_step_tokens=10, max_steps=3, max_seq_tokens=112, step_end_id=1, step_end_mod=6,
                 temperature=0.7, seed=21)
     eng, loop = build_pair(MINI, bf16=True, prompts=prompts, loop_kwargs=base)
     r0 = loop.step(0.0)["rewards"]
     delta = float(np.sort(r0)[1])
-    eng, loop = build_pair(MINI, bf16=True, prompts=prompts, loop_kwargs=base, engine_kwargs=dict(max_chunk_tokens=64))
+    eng, loop = build_pair(MINI, bf16=True, prompts=prompts, loop_kwargs=base,
+                           engine_kwargs=dict(max_chunk_tokens=64, kv_extended=kv_extended))
     stats = {}
     for _ in range(3):
         parity_step(eng, loop, delta, stats=stats, **TOL16)
     compare_counters(eng, loop)
-    print("mini bf16 parity:", stats)
+    print("mini bf16 parity, kv_extended =", kv_extended, stats)
 
 
 def test_page_pool_exhaustion_is_an_error_not_a_fault():
