@@ -21,6 +21,14 @@ needs, under one deterministic policy, so it can be compared bit for bit:
     pages stay with their row until reset;
   * the ascending list of rejected rows, and token / FLOPs counters (Section 3.3: 2N FLOPs per
     inference token of an N-parameter model, PRM included).
+
+Queued rejections (`min_target_rows` > 1).  Rows never interact, so nothing in Algorithm 1 says that
+all rows must take their i-th step together.  The paper counts the cost of the target by the tokens
+it generates (Section 3.3), but a batched target pass reads all of M's weights whether one row or
+the whole batch was rejected; to turn the saved FLOPs into saved time a rejected row may WAIT, its
+draft step dropped, while the accepted rows go on drafting, until `min_target_rows` rows wait (or
+nothing else is left to run); then the target writes y_i for all of them in one pass.  Each row's
+own sequence of steps is the one Algorithm 1 gives it: only the order in time changes.
 """
 from __future__ import annotations
 
@@ -55,6 +63,8 @@ class LoopConfig:
 class Row:
     z: list                         # committed tokens: prompt x followed by y_{1:i-1}
     live: bool = True
+    waiting: bool = False           # the row's draft step was rejected and the target has not written y_i yet
+    reward: float = 0.0             # reward of the row's latest draft step
     n_steps: int = 0
     kv_len: list = field(default_factory=lambda: [0, 0, 0])
     caches: list = field(default_factory=lambda: [None, None, None])
@@ -153,66 +163,90 @@ class OracleRSD:
             cur, pos = tok, pos + 1
         return out
 
-    def step(self, delta: float, forced_draft=None, forced_target=None, forced_accept=None) -> dict:
-        """One pass of the loop body of Algorithm 1 over all rows.  `forced_*` (per-row lists, or
-        None entries) replace sampled tokens / gate decisions; what was sampled is still reported."""
+    def step(self, delta: float, forced_draft=None, forced_target=None, forced_accept=None,
+             min_target_rows: int = 1) -> dict:
+        """One pass of the loop body of Algorithm 1 over the rows.  `forced_*` (per-row lists, or
+        None entries) replace sampled tokens / gate decisions; what was sampled is still reported.
+
+        min_target_rows = 1: every live row takes one step (draft, score, gate, target for the
+        rejected rows).  min_target_rows > 1: rows whose step is rejected wait until that many rows
+        wait, or until all live rows do; waiting rows take no part in the draft phase and report
+        step_len 0 until the target has written their step."""
         cfg, B = self.cfg, len(self.rows)
         res = dict(step_tokens=[[] for _ in range(B)], step_len=np.zeros(B, np.int32),
                    rewards=np.zeros(B, np.float64), accept=np.zeros(B, np.uint8), live=np.zeros(B, np.uint8),
                    draft_tokens=[[] for _ in range(B)], target_tokens=[[] for _ in range(B)],
-                   draft_trace=[None] * B, target_trace=[None] * B, rej_idx=[], z_len_before=np.zeros(B, np.int32))
-        live_rows = [b for b in range(B) if self.rows[b].live]
+                   draft_trace=[None] * B, target_trace=[None] * B, rej_idx=[], z_len_before=np.zeros(B, np.int32),
+                   drafted=np.zeros(B, np.uint8), waiting=np.zeros(B, np.uint8), flushed=False)
+        run_rows = [b for b in range(B) if self.rows[b].live and not self.rows[b].waiting]
         for b in range(B):
             res["z_len_before"][b] = len(self.rows[b].z)
+        for b in run_rows:
+            res["drafted"][b] = 1
 
-        # draft step y^_i for every live row
-        for b in live_rows:
+        # draft step y^_i for every live row that is not waiting for the target
+        for b in run_rows:
             self._reserve(DRAFT, b, len(self.rows[b].z) - 1 + cfg.max_step_tokens)
-        for b in live_rows:
+        for b in run_rows:
             tr = dict(sampled=[], margin=[], logits=[])
             f = forced_draft[b] if forced_draft is not None else None
             res["draft_tokens"][b] = self._generate_step(DRAFT, b, f, tr)
             res["draft_trace"][b] = tr
 
         # reward r_i = r(y^_i | z_i), read at the last token of the draft step
-        for b in live_rows:
+        for b in run_rows:
             self._reserve(PRM, b, len(self.rows[b].z) + len(res["draft_tokens"][b]))
-        for b in live_rows:
+        for b in run_rows:
             row = self.rows[b]
             seq = row.z + res["draft_tokens"][b]
             n_known = len(row.z) - row.kv_len[PRM]      # committed tokens the PRM has not cached yet
             h = self._ingest(PRM, b, len(seq), seq)
-            res["rewards"][b] = self.models[PRM].reward(h[-1])
+            row.reward = self.models[PRM].reward(h[-1])
             self.counters["ingest_tokens"][PRM] += n_known
             self.counters["score_tokens"] += len(res["draft_tokens"][b])
 
         # acceptance criterion A_omega(r_i)  (Algorithm 2; binary step: accept iff r_i >= delta)
-        for b in live_rows:
-            u = _uniform(cfg.seed, STREAM_ACCEPT, b, len(self.rows[b].z), 0)
-            a = _accept(cfg.omega_kind, res["rewards"][b], float(delta), cfg.omega_b, u)
+        for b in run_rows:
+            row = self.rows[b]
+            u = _uniform(cfg.seed, STREAM_ACCEPT, b, len(row.z), 0)
+            a = _accept(cfg.omega_kind, row.reward, float(delta), cfg.omega_b, u)
             if forced_accept is not None and forced_accept[b] is not None:
                 a = int(forced_accept[b])
             res["accept"][b] = a
-        res["rej_idx"] = [b for b in live_rows if not res["accept"][b]]
+            if not a:
+                # drop the draft step from the draft and PRM caches; the target will write y_i
+                row.waiting = True
+                row.kv_len[DRAFT] = len(row.z) - 1
+                row.kv_len[PRM] = len(row.z)
+                self.counters["discarded_draft_tokens"] += len(res["draft_tokens"][b])
+        wait_rows = [b for b in range(B) if self.rows[b].live and self.rows[b].waiting]
+        res["rej_idx"] = wait_rows
+        n_live = sum(1 for r in self.rows if r.live)
+        flush = len(wait_rows) > 0 and len(wait_rows) >= min(max(1, int(min_target_rows)), n_live)
+        res["flushed"] = flush
 
-        # rejected rows: drop the draft step from the draft and PRM caches, let the target write y_i
-        for b in res["rej_idx"]:
-            row = self.rows[b]
-            row.kv_len[DRAFT] = len(row.z) - 1
-            row.kv_len[PRM] = len(row.z)
-            self.counters["discarded_draft_tokens"] += len(res["draft_tokens"][b])
-        for b in res["rej_idx"]:
-            self._reserve(TARGET, b, len(self.rows[b].z) - 1 + cfg.max_step_tokens)
-        for b in res["rej_idx"]:
-            tr = dict(sampled=[], margin=[], logits=[])
-            f = forced_target[b] if forced_target is not None else None
-            res["target_tokens"][b] = self._generate_step(TARGET, b, f, tr)
-            res["target_trace"][b] = tr
+        if flush:
+            for b in wait_rows:
+                self._reserve(TARGET, b, len(self.rows[b].z) - 1 + cfg.max_step_tokens)
+            for b in wait_rows:
+                tr = dict(sampled=[], margin=[], logits=[])
+                f = forced_target[b] if forced_target is not None else None
+                res["target_tokens"][b] = self._generate_step(TARGET, b, f, tr)
+                res["target_trace"][b] = tr
 
         # commit y_i, stop rows that produced EOS or ran out of steps / room
-        for b in live_rows:
+        for b in range(B):
             row = self.rows[b]
-            y = res["draft_tokens"][b] if res["accept"][b] else res["target_tokens"][b]
+            if not row.live:
+                continue
+            res["rewards"][b] = row.reward
+            if res["accept"][b]:
+                y = res["draft_tokens"][b]
+            elif row.waiting and flush:
+                y = res["target_tokens"][b]
+                row.waiting = False
+            else:
+                continue                # waits for a later target pass
             row.z = row.z + y
             row.n_steps += 1
             res["step_tokens"][b] = y
@@ -224,6 +258,7 @@ class OracleRSD:
                 row.live = False
         for b in range(B):
             res["live"][b] = 1 if self.rows[b].live else 0
+            res["waiting"][b] = 1 if (self.rows[b].live and self.rows[b].waiting) else 0
         return res
 
     # -- reporting --------------------------------------------------------------------------
@@ -243,4 +278,5 @@ class OracleRSD:
                     pages=[[list(r.pages[w]) for r in self.rows] for w in range(3)],
                     next_page=list(self.next_page),
                     live=np.array([r.live for r in self.rows], np.uint8),
+                    waiting=np.array([r.live and r.waiting for r in self.rows], np.uint8),
                     n_steps=np.array([r.n_steps for r in self.rows], np.int32))

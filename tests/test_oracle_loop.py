@@ -226,3 +226,98 @@ def test_eos_stops_a_row_and_row_independence(tiny_weights):
     solo = OracleRSD(dm, pm, tm, LoopConfig(**base)); solo.prefill(prompts[:1])
     s = solo.step(0.5)
     assert list(s["step_tokens"][0]) == list(first["step_tokens"][0]) and s["rewards"][0] == first["rewards"][0]
+
+
+def run_to_end(loop, delta, min_target_rows, max_calls=200):
+    """Calls step until no row is live; returns per row the list of (tokens, accepted) in commit order."""
+    B = len(loop.rows)
+    hist = [[] for _ in range(B)]
+    flushes = calls = 0
+    for _ in range(max_calls):
+        if not any(r.live for r in loop.rows):
+            break
+        r = loop.step(delta, min_target_rows=min_target_rows)
+        calls += 1
+        flushes += int(r["flushed"])
+        for b in range(B):
+            if r["step_len"][b] > 0:
+                hist[b].append((list(r["step_tokens"][b]), int(r["accept"][b])))
+            else:
+                assert r["accept"][b] == 0
+        # a row that waits stays live, took no step, and keeps its reward
+        for b in range(B):
+            if r["waiting"][b]:
+                assert r["live"][b] == 1 and r["step_len"][b] == 0
+    assert not any(r.live for r in loop.rows)
+    return hist, flushes, calls
+
+
+@pytest.mark.parametrize("min_rows", [2, 3, 100])
+def test_queued_rejections_leave_every_rows_sequence_unchanged(tiny_weights, min_rows):
+    """Rows are independent in Algorithm 1, so letting rejected rows wait for a fuller target batch
+    changes when a step is written, never what is written: every row's committed steps, gate
+    decisions, final context and the token counters equal those of the lock-step loop; only the
+    number of target passes drops."""
+    dm, pm, tm = tiny_models(tiny_weights)
+    cfg = LoopConfig(max_step_tokens=5, max_steps=5, max_seq_tokens=80, step_end_id=2, step_end_mod=4,
+                     temperature=0.7, seed=21)
+    tok, off = ri.prompts(9, 5, 4, 9, 1024)
+    prompts = [tok[off[b]:off[b + 1]].tolist() for b in range(5)]
+    # a threshold near the median reward of the first step mixes accepted and rejected rows
+    probe = OracleRSD(dm, pm, tm, cfg)
+    probe.prefill(prompts)
+    delta = float(np.median(probe.step(0.0)["rewards"]))
+    lock = OracleRSD(dm, pm, tm, cfg)
+    lock.prefill(prompts)
+    want, flushes_lock, calls_lock = run_to_end(lock, delta, 1)
+    assert any(a for h in want for _, a in h) and any(not a for h in want for _, a in h)
+    queued = OracleRSD(dm, pm, tm, cfg)
+    queued.prefill(prompts)
+    got, flushes_q, calls_q = run_to_end(queued, delta, min_rows)
+    assert got == want
+    assert [r.z for r in queued.rows] == [r.z for r in lock.rows]
+    for key in ("gen_tokens", "score_tokens", "steps", "accepted_steps", "rejected_steps", "discarded_draft_tokens"):
+        assert queued.counters[key] == lock.counters[key], key
+    assert flushes_q <= flushes_lock and calls_q >= calls_lock
+
+
+def test_queued_flush_rule_and_cursors(tiny_weights):
+    """Forced gate decisions: rejected rows wait with their draft and PRM cursors rolled back and the
+    target untouched; the target pass happens in the call in which the number of waiting rows reaches
+    min_target_rows (or every live row waits), serves all of them in ascending order and hands out
+    their pages in that order."""
+    dm, pm, tm = tiny_models(tiny_weights)
+    cfg = LoopConfig(max_step_tokens=4, max_steps=6, max_seq_tokens=64, step_end_id=900, temperature=0.0, seed=2)
+    tok, off = ri.prompts(5, 4, 6, 6, 1024)
+    prompts = [tok[off[b]:off[b + 1]].tolist() for b in range(4)]
+    loop = OracleRSD(dm, pm, tm, cfg)
+    loop.prefill(prompts)
+    # call 1: row 2 rejected -> waits (1 < 3)
+    r = loop.step(0.5, forced_accept=[1, 1, 0, 1], min_target_rows=3)
+    assert not r["flushed"] and list(r["waiting"]) == [0, 0, 1, 0] and r["rej_idx"] == [2]
+    assert list(r["step_len"]) == [4, 4, 0, 4] and list(r["drafted"]) == [1, 1, 1, 1]
+    st = loop.state()
+    assert st["kv_len"][DRAFT][2] == 5 and st["kv_len"][PRM][2] == 6 and st["kv_len"][TARGET][2] == 0
+    assert st["n_pages"][TARGET].sum() == 0 and st["n_steps"][2] == 0
+    # call 2: row 0 rejected -> two wait (2 < 3); row 2 does not draft
+    r = loop.step(0.5, forced_accept=[0, 1, None, 1], min_target_rows=3)
+    assert not r["flushed"] and list(r["waiting"]) == [1, 0, 1, 0] and r["rej_idx"] == [0, 2]
+    assert list(r["drafted"]) == [1, 1, 0, 1] and list(r["step_len"]) == [0, 4, 0, 4]
+    assert r["draft_tokens"][2] == []
+    # call 3: row 3 rejected -> three wait: the target writes the step of rows 0, 2 and 3
+    r = loop.step(0.5, forced_accept=[None, 1, None, 0], min_target_rows=3)
+    assert r["flushed"] and r["rej_idx"] == [0, 2, 3] and list(r["waiting"]) == [0, 0, 0, 0]
+    assert list(r["step_len"]) == [4, 4, 4, 4] and list(r["accept"]) == [0, 1, 0, 0]
+    st = loop.state()
+    # target pages in ascending row order: rows 0, 2, 3 need ceil((z - 1 + 4) / 16) pages each
+    assert st["pages"][TARGET][0] == [0] and st["pages"][TARGET][1] == []
+    assert st["pages"][TARGET][2] == [1] and st["pages"][TARGET][3] == [2, 3]
+    assert list(st["n_steps"]) == [2, 3, 1, 3]
+    # each committed target step is what the target writes from the committed context alone
+    for b, ctx_len in ((0, 6 + 4), (2, 6), (3, 6 + 8)):
+        ctx = loop.rows[b].z[:ctx_len]
+        want = plain_decode(tm, TARGET, b, ctx, 4, cfg, 1024)
+        assert want == list(r["step_tokens"][b])
+    # every live row waits -> flush although fewer than min_target_rows wait
+    r = loop.step(0.5, forced_accept=[0, 0, 0, 0], min_target_rows=100)
+    assert r["flushed"] and r["rej_idx"] == [0, 1, 2, 3]
