@@ -209,6 +209,8 @@ def workload_config(args) -> dict:
                         + (f"delta {args.delta}" if getattr(args, "delta", None) is not None else "delta at the 70% accept quantile"),
             "batch": B, "max_step_tokens": args.cap or cap, "replicas": args.gpus,
             "kv_cache": "fp16 hi+lo pairs" if kv_extended(args) else "fp16",
+            "schedule": "lock-step rsd_step" if getattr(args, "queue", 1) == 1 else
+                        f"rsd_step_queued, target pass once {args.queue} rows wait",
             "l2": "weights and KV read per decode iteration exceed the 126 MB L2 (no flush needed)"}
 
 
@@ -280,7 +282,7 @@ def run_ours(args, rank: int, world: int):
     e2e_tokens = 0
     accepted = live_steps = 0
     for _ in range(args.warmup):
-        r = eng.step(delta)
+        r = eng.step(delta, args.queue)
         e2e_tokens += int(r["step_len"].sum())
     eng.gemm_timing(args.time_stride)
     eng.phase_ms(True)
@@ -290,7 +292,7 @@ def run_ours(args, rank: int, world: int):
     t_start.record()
     timed_tokens = 0
     for _ in range(args.steps):
-        r = eng.step(delta)                                # host outputs: D2H inside the call
+        r = eng.step(delta, args.queue)                    # host outputs: D2H inside the call
         timed_tokens += int(r["step_len"].sum())
         accepted += int(r["accept"].sum())
         live_steps += int((r["step_len"] > 0).sum())
@@ -506,6 +508,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--delta", type=float, default=None, help="fixed threshold instead of the 70 %% accept quantile")
     ap.add_argument("--cap", type=int, default=0, help="override the step cap (profiling aid)")
+    ap.add_argument("--queue", type=int, default=1,
+                    help="min_target_rows of rsd_step_queued (1 = rsd_step, the headline configuration)")
     ap.add_argument("--kv-extended", type=int, default=None, choices=[0, 1], dest="kv_extended",
                     help="KV cache as fp16 hi+lo pairs (default: on for cfg4 only)")
     ap.add_argument("--only", default="", help="with --sweep gemm: a single M,K,N point, plain launches")

@@ -135,6 +135,20 @@ int rsd_prefill(rsd_ctx*, const int32_t* tokens, const int32_t* offsets, int32_t
 int rsd_step(rsd_ctx*, float delta, void* cuda_stream, int32_t* step_tokens, int32_t* step_len,
              float* rewards, uint8_t* accept, uint8_t* live);
 
+/* rsd_step with queued rejections.  Rows are independent in Algorithm 1, and a batched target pass
+ * reads all of M's weights however few rows were rejected (the FLOPs of Section 3.3 count tokens, the
+ * clock counts weight passes).  Here a row whose draft step is rejected WAITS -- its draft step is
+ * dropped from the draft and PRM caches, it takes no part in later draft phases -- while accepted
+ * rows go on; in the call in which min_target_rows rows wait (or every live row does) the target
+ * catches up on and writes y_i for all waiting rows, in ascending row order.  Every row's own
+ * sequence of steps is the one rsd_step would give it; min_target_rows = 1 is rsd_step.
+ * Outputs as rsd_step, per call: a row that waits reports step_len 0, accept 0, live 1 and
+ * waiting 1 (HOST [B], may be NULL); rewards[b] is the reward of row b's latest draft step; a row
+ * served by the target reports its step with accept 0 in the call of that pass.
+ * RSD_ERR_ARG when min_target_rows < 1.                                                        */
+int rsd_step_queued(rsd_ctx*, float delta, int32_t min_target_rows, void* cuda_stream, int32_t* step_tokens,
+                    int32_t* step_len, float* rewards, uint8_t* accept, uint8_t* live, uint8_t* waiting);
+
 /* Counters of the work done since rsd_prefill / rsd_reset.  Index 0 draft, 1 PRM, 2 target.
  * flops_paper follows Section 3.3: 2N per inference token of an N-parameter model (all
  * parameters, embedding and head included), counting every token the draft or the target
@@ -169,7 +183,8 @@ int rsd_debug_get_sampled(rsd_ctx*, int which, int32_t* out);
 
 /* Integer state, HOST outputs (any may be NULL): z_len [B], kv_len [3, B], n_pages [3, B],
  * page_table [3, B, max_pages] with max_pages = ceil(max_seq_tokens / page_tokens), next_page [3],
- * rej_idx [B] (ascending rejected rows of the last step, first *n_rej entries valid).         */
+ * rej_idx [B] (ascending rows that waited for the target after the last step's gate -- with rsd_step
+ * the rows rejected in that step -- first *n_rej entries valid).                                */
 int rsd_debug_get_state(rsd_ctx*, int32_t* z_len, int32_t* kv_len, int32_t* n_pages, int32_t* page_table,
                         int32_t* next_page, int32_t* rej_idx, int32_t* n_rej);
 

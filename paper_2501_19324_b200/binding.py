@@ -49,7 +49,7 @@ class rsd_counters(ctypes.Structure):
                 ("discarded_draft_tokens", c_uint64), ("flops_paper", c_double), ("flops_all_tokens", c_double)]
 
 
-EXPORTS = ["rsd_query_sizes", "rsd_create", "rsd_load_models", "rsd_prefill", "rsd_step", "rsd_flops_counters",
+EXPORTS = ["rsd_query_sizes", "rsd_create", "rsd_load_models", "rsd_prefill", "rsd_step", "rsd_step_queued", "rsd_flops_counters",
            "rsd_reset", "rsd_destroy", "rsd_last_error", "rsd_debug_force", "rsd_debug_get_logits",
            "rsd_debug_get_sampled", "rsd_debug_get_state", "rsd_debug_gemm_timing", "rsd_debug_launch_count", "rsd_debug_phase_ms", "rsd_k_gemm", "rsd_k_gemm_scratch_bytes",
            "rsd_k_attn_decode", "rsd_k_attn_decode_scratch_bytes", "rsd_k_attn_chunk", "rsd_k_gate_compact", "rsd_k_gate_compact_static", "rsd_k_gate_compact_static_error", "rsd_k_rmsnorm",
@@ -71,6 +71,7 @@ def lib():
         L.rsd_load_models.argtypes = [vp] + [POINTER(rsd_model)] * 3
         L.rsd_prefill.argtypes = [vp, vp, vp, c_int32, vp]
         L.rsd_step.argtypes = [vp, c_float, vp, vp, vp, vp, vp, vp]
+        L.rsd_step_queued.argtypes = [vp, c_float, c_int32, vp, vp, vp, vp, vp, vp, vp]
         L.rsd_flops_counters.argtypes = [vp, POINTER(rsd_counters)]
         L.rsd_reset.argtypes = [vp]
         L.rsd_destroy.argtypes = [vp]
@@ -190,12 +191,19 @@ class Engine:
         self.B = len(offsets) - 1
         _check(lib().rsd_prefill(self.ctx, tokens.ctypes.data, offsets.ctypes.data, self.B, _stream()), self.ctx)
 
-    def step(self, delta: float) -> dict:
+    def step(self, delta: float, min_target_rows: int = 1) -> dict:
+        """rsd_step(delta); with min_target_rows > 1, rsd_step_queued: rejected rows wait (step_len 0,
+        waiting 1) until that many wait, then the target writes all their steps in one pass."""
         B, C = self.B, self.C
         out = dict(step_tokens=np.zeros((B, C), np.int32), step_len=np.zeros(B, np.int32),
-                   rewards=np.zeros(B, np.float32), accept=np.zeros(B, np.uint8), live=np.zeros(B, np.uint8))
-        _check(lib().rsd_step(self.ctx, delta, _stream(), out["step_tokens"].ctypes.data, out["step_len"].ctypes.data,
-                              out["rewards"].ctypes.data, out["accept"].ctypes.data, out["live"].ctypes.data), self.ctx)
+                   rewards=np.zeros(B, np.float32), accept=np.zeros(B, np.uint8), live=np.zeros(B, np.uint8),
+                   waiting=np.zeros(B, np.uint8))
+        ptrs = [out[k].ctypes.data for k in ("step_tokens", "step_len", "rewards", "accept", "live")]
+        if min_target_rows == 1:
+            _check(lib().rsd_step(self.ctx, delta, _stream(), *ptrs), self.ctx)
+        else:
+            _check(lib().rsd_step_queued(self.ctx, delta, min_target_rows, _stream(), *ptrs,
+                                         out["waiting"].ctypes.data), self.ctx)
         return out
 
     def counters(self) -> dict:

@@ -32,7 +32,7 @@ struct ModelHost {
 
 // Host-visible scalars mirrored from the device after each phase boundary.
 struct Scalars {
-  int32_t n_tok, n_rej, err, n_active, n_slots, next_page[3];
+  int32_t n_tok, n_rej, err, n_active, n_slots, next_page[3], iter, n_live;
 };
 
 struct Layout {
@@ -63,7 +63,7 @@ struct rsd_ctx {
   // staging of step outputs (device) and their pinned host mirrors
   int32_t *o_tokens = nullptr, *o_len = nullptr;
   float* o_rewards = nullptr;
-  uint8_t *o_accept = nullptr, *o_live = nullptr;
+  uint8_t *o_accept = nullptr, *o_live = nullptr, *o_role = nullptr, *o_waiting = nullptr;
   char* pinned = nullptr;
   size_t pinned_bytes = 0;
   void* gemm_scratch = nullptr;
@@ -191,12 +191,13 @@ size_t layout_workspace(const rsd_config& cfg, const rsd_model* const ms[3], rsd
   st.gen_active = TAKE(int32_t, B);
   st.rewards = TAKE(float, B);
   st.accept = TAKE(uint8_t, B);
+  st.waiting = TAKE(uint8_t, B);
   st.rej_idx = TAKE(int32_t, B);
   st.slot_row = TAKE(int32_t, B);
   st.last_idx = TAKE(int32_t, B);
   int32_t* scal = TAKE(int32_t, 16);
   st.n_tok = scal + 0; st.n_rej = scal + 1; st.err = scal + 2; st.n_active = scal + 3; st.n_slots = scal + 4; st.iter = scal + 8;
-  st.next_page = scal + 5;
+  st.next_page = scal + 5; st.n_live = scal + 9;
   st.pass_capacity = B * S;
   st.pass_tok_id = TAKE(int32_t, (size_t)B * S);
   st.pass_tok_row = TAKE(int32_t, (size_t)B * S);
@@ -223,6 +224,8 @@ size_t layout_workspace(const rsd_config& cfg, const rsd_model* const ms[3], rsd
   float* o_rewards = TAKE(float, B);
   uint8_t* o_accept = TAKE(uint8_t, B);
   uint8_t* o_live = TAKE(uint8_t, B);
+  uint8_t* o_role = TAKE(uint8_t, B);
+  uint8_t* o_waiting = TAKE(uint8_t, B);
   const size_t gs = gemm_scratch_bytes_any();
   void* gscr = TAKE(char, gs);
   int h_max = 0;
@@ -242,6 +245,7 @@ size_t layout_workspace(const rsd_config& cfg, const rsd_model* const ms[3], rsd
     c->dbg_logits[0] = dbg[0]; c->dbg_logits[1] = dbg[1];
     c->d_scalars = scal;
     c->o_tokens = o_tokens; c->o_len = o_len; c->o_rewards = o_rewards; c->o_accept = o_accept; c->o_live = o_live;
+    c->o_role = o_role; c->o_waiting = o_waiting;
     c->gemm_scratch = gscr; c->gemm_scratch_bytes = gs;
     c->attn_scratch = ascr; c->attn_scratch_bytes = as;
   }
@@ -489,6 +493,7 @@ __global__ void init_rows_kernel(RowState st, const int32_t* flat, const int32_t
     st.forced_accept[b] = 255;
     st.rewards[b] = 0.f;
     st.accept[b] = 0;
+    st.waiting[b] = 0;
   }
 }
 
@@ -638,16 +643,16 @@ int rsd_prefill(rsd_ctx* c, const int32_t* tokens, const int32_t* offsets, int32
   RSD_LAUNCH((init_rows_kernel), B, 128, 0, s, c->st, c->st.pass_tok_id, c->st.pass_tok_row, B);
   CU(launched(1));
   CU(cudaStreamSynchronize(s));  // the staging buffers are reused below
-  CU(launch_reserve_pages(c->st, RSD_DRAFT, kReservePrefillDraft, s));
-  CU(launch_reserve_pages(c->st, RSD_PRM, kReservePrefillPrm, s));
+  CU(launch_reserve_pages(c->st, RSD_DRAFT, kReservePrefillDraft, 1, s));
+  CU(launch_reserve_pages(c->st, RSD_PRM, kReservePrefillPrm, 1, s));
   Scalars sc;
-  CU(launch_build_pass(c->st, RSD_DRAFT, kPassIngestDraft, s));
+  CU(launch_build_pass(c->st, RSD_DRAFT, kPassIngestDraft, 1, s));
   rc = read_scalars(c, s, &sc);
   if (rc) return rc;
   rc = run_ingest(c, RSD_DRAFT, sc.n_tok, false, s);
   if (rc) return rc;
   c->ctr.ingest_tokens[RSD_DRAFT] += sc.n_tok;
-  CU(launch_build_pass(c->st, RSD_PRM, kPassScorePrm, s));
+  CU(launch_build_pass(c->st, RSD_PRM, kPassScorePrm, 1, s));
   rc = read_scalars(c, s, &sc);
   if (rc) return rc;
   rc = run_ingest(c, RSD_PRM, sc.n_tok, false, s);
@@ -658,20 +663,22 @@ int rsd_prefill(rsd_ctx* c, const int32_t* tokens, const int32_t* offsets, int32
   return RSD_OK;
 }
 
-int rsd_step(rsd_ctx* c, float delta, void* cuda_stream, int32_t* step_tokens, int32_t* step_len, float* rewards,
-             uint8_t* accept, uint8_t* live) {
+static int step_impl(rsd_ctx* c, float delta, int min_target_rows, void* cuda_stream, int32_t* step_tokens,
+                     int32_t* step_len, float* rewards, uint8_t* accept, uint8_t* live, uint8_t* waiting) {
   if (!c) return RSD_ERR_ARG;
   if (c->poisoned) return fail(c, RSD_ERR_STATE, "context unusable after a CUDA error%s");
   if (!c->prefilled) return fail(c, RSD_ERR_STATE, "rsd_step before rsd_prefill%s");
+  if (min_target_rows < 1) return fail(c, RSD_ERR_ARG, "min_target_rows must be at least 1%s");
   cudaStream_t s = (cudaStream_t)cuda_stream;
   const int B = c->st.B;
   Scalars sc;
   int rc;
 #define PHASE(i) do { if (c->time_phases) CU(cudaEventRecord(c->ph_ev[i], s)); } while (0)
   PHASE(0);
-  // draft: catch up on a step the target wrote last time, then decode y^_i
-  CU(launch_reserve_pages(c->st, RSD_DRAFT, kReserveStepDraft, s));
-  CU(launch_build_pass(c->st, RSD_DRAFT, kPassIngestDraft, s));
+  // draft: catch up on a step the target wrote last time, then decode y^_i (rows that wait for the
+  // target take no part)
+  CU(launch_reserve_pages(c->st, RSD_DRAFT, kReserveStepDraft, 1, s));
+  CU(launch_build_pass(c->st, RSD_DRAFT, kPassIngestDraft, 1, s));
   if ((rc = read_scalars(c, s, &sc))) return rc;
   const int n_sync = sc.n_tok;
   if ((rc = run_ingest(c, RSD_DRAFT, n_sync, false, s))) return rc;
@@ -679,26 +686,28 @@ int rsd_step(rsd_ctx* c, float delta, void* cuda_stream, int32_t* step_tokens, i
   if ((rc = decode_phase(c, RSD_DRAFT, 0, B, s))) return rc;
   PHASE(2);
   // PRM: score y^_i at its last token
-  CU(launch_reserve_pages(c->st, RSD_PRM, kReserveScorePrm, s));
-  CU(launch_build_pass(c->st, RSD_PRM, kPassScorePrm, s));
+  CU(launch_reserve_pages(c->st, RSD_PRM, kReserveScorePrm, 1, s));
+  CU(launch_build_pass(c->st, RSD_PRM, kPassScorePrm, 1, s));
   if ((rc = read_scalars(c, s, &sc))) return rc;
   const int n_prm = sc.n_tok;
   if ((rc = run_ingest(c, RSD_PRM, n_prm, true, s))) return rc;
   PHASE(3);
-  // gate, compaction of rejected rows, target catch-up and decode
+  // gate, compaction of the waiting rows; once enough of them wait: target catch-up and decode
   CU(launch_gate(c->st, delta, c->lp, s));
-  CU(launch_reserve_pages(c->st, RSD_TARGET, kReserveTarget, s));
-  CU(launch_build_pass(c->st, RSD_TARGET, kPassCatchupTarget, s));
+  CU(launch_reserve_pages(c->st, RSD_TARGET, kReserveTarget, min_target_rows, s));
+  CU(launch_build_pass(c->st, RSD_TARGET, kPassCatchupTarget, min_target_rows, s));
   if ((rc = read_scalars(c, s, &sc))) return rc;
   const int n_catch = sc.n_tok, n_rej = sc.n_rej;
+  const bool target_runs = target_pass_due(n_rej, sc.n_live, min_target_rows);
   c->last_n_rej = n_rej;
   PHASE(4);
-  if ((rc = run_ingest(c, RSD_TARGET, n_catch, false, s))) return rc;
+  if (target_runs && (rc = run_ingest(c, RSD_TARGET, n_catch, false, s))) return rc;
   PHASE(5);
-  if ((rc = decode_phase(c, RSD_TARGET, 1, n_rej, s))) return rc;
+  if (target_runs && (rc = decode_phase(c, RSD_TARGET, 1, n_rej, s))) return rc;
   PHASE(6);
   // commit and read the results back
-  CU(launch_commit(c->st, c->lp, c->o_tokens, c->o_len, c->o_rewards, c->o_accept, c->o_live, s));
+  CU(launch_commit(c->st, c->lp, target_runs ? 1 : 0, c->o_tokens, c->o_len, c->o_rewards, c->o_accept, c->o_live,
+                   c->o_role, c->o_waiting, s));
   char* hp = c->pinned + 256;
   int32_t* h_tokens = (int32_t*)hp; hp += sizeof(int32_t) * (size_t)B * c->C;
   int32_t* h_len = (int32_t*)hp; hp += sizeof(int32_t) * B;
@@ -707,6 +716,8 @@ int rsd_step(rsd_ctx* c, float delta, void* cuda_stream, int32_t* step_tokens, i
   float* h_rew = (float*)hp; hp += sizeof(float) * B;
   uint8_t* h_acc = (uint8_t*)hp; hp += B;
   uint8_t* h_live = (uint8_t*)hp; hp += B;
+  uint8_t* h_role = (uint8_t*)hp; hp += B;
+  uint8_t* h_wait = (uint8_t*)hp; hp += B;
   CU(cudaMemcpyAsync(h_tokens, c->o_tokens, sizeof(int32_t) * (size_t)B * c->C, cudaMemcpyDeviceToHost, s));
   CU(cudaMemcpyAsync(h_len, c->o_len, sizeof(int32_t) * B, cudaMemcpyDeviceToHost, s));
   CU(cudaMemcpyAsync(h_gen0, c->st.gen_len[0], sizeof(int32_t) * B, cudaMemcpyDeviceToHost, s));
@@ -714,6 +725,8 @@ int rsd_step(rsd_ctx* c, float delta, void* cuda_stream, int32_t* step_tokens, i
   CU(cudaMemcpyAsync(h_rew, c->o_rewards, sizeof(float) * B, cudaMemcpyDeviceToHost, s));
   CU(cudaMemcpyAsync(h_acc, c->o_accept, B, cudaMemcpyDeviceToHost, s));
   CU(cudaMemcpyAsync(h_live, c->o_live, B, cudaMemcpyDeviceToHost, s));
+  CU(cudaMemcpyAsync(h_role, c->o_role, B, cudaMemcpyDeviceToHost, s));
+  CU(cudaMemcpyAsync(h_wait, c->o_waiting, B, cudaMemcpyDeviceToHost, s));
   if ((rc = clear_forcing(c, s))) return rc;
   PHASE(7);
 #undef PHASE
@@ -725,28 +738,40 @@ int rsd_step(rsd_ctx* c, float delta, void* cuda_stream, int32_t* step_tokens, i
       c->ph_ms[i] += ms;
     }
   }
-  // counters (Section 3.3 accounting)
-  uint64_t gen_d = 0, gen_t = 0, n_live = 0, n_acc = 0, discarded = 0;
+  // counters (Section 3.3 accounting): draft tokens when they are generated, steps when they are committed
+  uint64_t gen_d = 0, gen_t = 0, n_acc = 0, n_tgt = 0, discarded = 0;
   for (int b = 0; b < B; ++b) {
-    if (h_len[b] == 0) continue;  // row was already stopped
-    ++n_live;
-    gen_d += h_gen0[b];
-    if (h_acc[b]) ++n_acc; else { gen_t += h_gen1[b]; discarded += h_gen0[b]; }
+    const int code = h_role[b] & 3;
+    if (code) gen_d += h_gen0[b];
+    if (code == 1) ++n_acc;
+    if (code == 2) discarded += h_gen0[b];
+    if (h_role[b] & 4) { gen_t += h_gen1[b]; ++n_tgt; }
   }
   c->ctr.gen_tokens[RSD_DRAFT] += gen_d;
   c->ctr.gen_tokens[RSD_TARGET] += gen_t;
   c->ctr.ingest_tokens[RSD_DRAFT] += n_sync;
   c->ctr.ingest_tokens[RSD_PRM] += (uint64_t)n_prm - gen_d;
-  c->ctr.ingest_tokens[RSD_TARGET] += n_catch;
+  c->ctr.ingest_tokens[RSD_TARGET] += target_runs ? n_catch : 0;
   c->ctr.score_tokens += gen_d;
-  c->ctr.steps += n_live; c->ctr.accepted_steps += n_acc; c->ctr.rejected_steps += n_live - n_acc;
+  c->ctr.steps += n_acc + n_tgt; c->ctr.accepted_steps += n_acc; c->ctr.rejected_steps += n_tgt;
   c->ctr.discarded_draft_tokens += discarded;
   if (step_tokens) memcpy(step_tokens, h_tokens, sizeof(int32_t) * (size_t)B * c->C);
   if (step_len) memcpy(step_len, h_len, sizeof(int32_t) * B);
   if (rewards) memcpy(rewards, h_rew, sizeof(float) * B);
   if (accept) memcpy(accept, h_acc, B);
   if (live) memcpy(live, h_live, B);
+  if (waiting) memcpy(waiting, h_wait, B);
   return RSD_OK;
+}
+
+int rsd_step(rsd_ctx* c, float delta, void* cuda_stream, int32_t* step_tokens, int32_t* step_len, float* rewards,
+             uint8_t* accept, uint8_t* live) {
+  return step_impl(c, delta, 1, cuda_stream, step_tokens, step_len, rewards, accept, live, nullptr);
+}
+
+int rsd_step_queued(rsd_ctx* c, float delta, int32_t min_target_rows, void* cuda_stream, int32_t* step_tokens,
+                    int32_t* step_len, float* rewards, uint8_t* accept, uint8_t* live, uint8_t* waiting) {
+  return step_impl(c, delta, min_target_rows, cuda_stream, step_tokens, step_len, rewards, accept, live, waiting);
 }
 
 int rsd_flops_counters(rsd_ctx* c, rsd_counters* out) {

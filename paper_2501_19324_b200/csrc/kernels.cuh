@@ -131,8 +131,10 @@ struct RowState {
   uint8_t* forced_accept;      // [B], 0/1 force, 255 free
   int32_t *gen_active, *n_active;
   float* rewards;
-  uint8_t* accept;
-  int32_t *rej_idx, *n_rej;
+  uint8_t* accept;             // [B] this call: 0 took no draft step, 1 accepted, 2 rejected
+  uint8_t* waiting;            // [B] 1: the row's draft step was rejected and the target has not written y_i yet
+  int32_t *rej_idx, *n_rej;    // ascending list of the waiting rows and its length
+  int32_t *n_live;             // live rows, counted by the gate
   int32_t *slot_row, *n_slots; // decode slots of the current phase
   int32_t *iter;               // iteration counter of the current decode phase
   int32_t *last_idx;           // [B] flat index of each row's last token in the current pass
@@ -152,15 +154,24 @@ struct LoopParams {
   uint64_t seed;
 };
 
-cudaError_t launch_reserve_pages(const RowState& st, int which, ReserveMode mode, cudaStream_t s);
-cudaError_t launch_build_pass(const RowState& st, int which, PassMode mode, cudaStream_t s);
+// min_target_rows: the target serves the waiting rows only once that many wait, or every live row does
+// (target_pass_due); it matters to the target modes alone.
+cudaError_t launch_reserve_pages(const RowState& st, int which, ReserveMode mode, int min_target_rows, cudaStream_t s);
+cudaError_t launch_build_pass(const RowState& st, int which, PassMode mode, int min_target_rows, cudaStream_t s);
+inline __host__ __device__ bool target_pass_due(int n_waiting, int n_live, int min_target_rows) {
+  const int want = min_target_rows < 1 ? 1 : min_target_rows;
+  return n_waiting > 0 && n_waiting >= (want < n_live ? want : n_live);
+}
 cudaError_t launch_decode_begin(const RowState& st, int phase, cudaStream_t s);
 cudaError_t launch_decode_prepare(const RowState& st, int which, int n_slots, cudaStream_t s);
 // best: packed winners left by launch_sample (cleared here).
 cudaError_t launch_decode_update(const RowState& st, int which, int phase, unsigned long long* best,
                                  int n_slots, const LoopParams& lp, cudaStream_t s);
 cudaError_t launch_gate(const RowState& st, float delta, const LoopParams& lp, cudaStream_t s);
-cudaError_t launch_commit(const RowState& st, const LoopParams& lp, int32_t* out_tokens, int32_t* out_len,
-                          float* out_rewards, uint8_t* out_accept, uint8_t* out_live, cudaStream_t s);
+// target_ran: the waiting rows' steps were written by the target in this call.  out_role[b]: bits 0-1 =
+// accept code of this call, bit 2 = the row committed a target step; out_waiting[b]: still waiting.
+cudaError_t launch_commit(const RowState& st, const LoopParams& lp, int target_ran, int32_t* out_tokens,
+                          int32_t* out_len, float* out_rewards, uint8_t* out_accept, uint8_t* out_live,
+                          uint8_t* out_role, uint8_t* out_waiting, cudaStream_t s);
 
 }  // namespace rsd

@@ -12,7 +12,7 @@ namespace rsd {
 // Page reservation.  Row b needs capacity for `need` cached positions; missing pages are taken
 // from a bump counter, rows served in ascending order, each row's new pages consecutive.
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(1024) reserve_pages_kernel(RowState st, int which, int mode) {
+__global__ void __launch_bounds__(1024) reserve_pages_kernel(RowState st, int which, int mode, int min_target_rows) {
   RSD_PDL_SYNC();
   __shared__ int scan[33];
   const int b = threadIdx.x;
@@ -20,12 +20,15 @@ __global__ void __launch_bounds__(1024) reserve_pages_kernel(RowState st, int wh
   if (b < st.B) {
     const int z = st.z_len[b];
     const bool live = st.live[b] != 0;
+    const bool runs = live && !st.waiting[b];     // takes a draft step in this call
     switch (mode) {
       case kReservePrefillDraft: need = live ? z - 1 : 0; break;
       case kReservePrefillPrm: need = live ? z : 0; break;
-      case kReserveStepDraft: need = live ? z - 1 + st.C : 0; break;
-      case kReserveScorePrm: need = live ? z + st.gen_len[0][b] : 0; break;
-      case kReserveTarget: need = (live && !st.accept[b]) ? z - 1 + st.C : 0; break;
+      case kReserveStepDraft: need = runs ? z - 1 + st.C : 0; break;
+      case kReserveScorePrm: need = runs ? z + st.gen_len[0][b] : 0; break;
+      case kReserveTarget:
+        need = (live && st.waiting[b] && target_pass_due(st.n_rej[0], st.n_live[0], min_target_rows)) ? z - 1 + st.C : 0;
+        break;
     }
   }
   const int have = b < st.B ? st.n_pages[which][b] : 0;
@@ -47,8 +50,8 @@ __global__ void __launch_bounds__(1024) reserve_pages_kernel(RowState st, int wh
   if (b == 0) st.next_page[which] = base + total;
 }
 
-cudaError_t launch_reserve_pages(const RowState& st, int which, ReserveMode mode, cudaStream_t s) {
-  RSD_LAUNCH((reserve_pages_kernel), 1, 1024, 0, s, st, which, (int)mode);
+cudaError_t launch_reserve_pages(const RowState& st, int which, ReserveMode mode, int min_target_rows, cudaStream_t s) {
+  RSD_LAUNCH((reserve_pages_kernel), 1, 1024, 0, s, st, which, (int)mode, min_target_rows);
   return launched(1);
 }
 
@@ -56,7 +59,7 @@ cudaError_t launch_reserve_pages(const RowState& st, int which, ReserveMode mode
 // Ragged pass list: for every participating row the positions [kv_len, end) not yet cached by model
 // `which`, flattened in (row, position) order.  Advances kv_len to `end`.
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(1024) build_pass_kernel(RowState st, int which, int mode) {
+__global__ void __launch_bounds__(1024) build_pass_kernel(RowState st, int which, int mode, int min_target_rows) {
   RSD_PDL_SYNC();
   __shared__ int scan[33];
   __shared__ int s_off[kMaxBatch + 1];
@@ -66,12 +69,15 @@ __global__ void __launch_bounds__(1024) build_pass_kernel(RowState st, int which
   if (b < st.B) {
     const int z = st.z_len[b];
     const bool live = st.live[b] != 0;
+    const bool runs = live && !st.waiting[b];
     start = st.kv_len[which][b];
     int end = start;
     switch (mode) {
-      case kPassIngestDraft: end = live ? z - 1 : start; break;
-      case kPassScorePrm: end = live ? z + st.gen_len[0][b] : start; break;
-      case kPassCatchupTarget: end = (live && !st.accept[b]) ? z - 1 : start; break;
+      case kPassIngestDraft: end = runs ? z - 1 : start; break;
+      case kPassScorePrm: end = runs ? z + st.gen_len[0][b] : start; break;
+      case kPassCatchupTarget:
+        end = (live && st.waiting[b] && target_pass_due(st.n_rej[0], st.n_live[0], min_target_rows)) ? z - 1 : start;
+        break;
     }
     cnt = max(0, end - start);
   }
@@ -103,14 +109,14 @@ __global__ void __launch_bounds__(1024) build_pass_kernel(RowState st, int which
   }
 }
 
-cudaError_t launch_build_pass(const RowState& st, int which, PassMode mode, cudaStream_t s) {
-  RSD_LAUNCH((build_pass_kernel), 1, 1024, 0, s, st, which, (int)mode);
+cudaError_t launch_build_pass(const RowState& st, int which, PassMode mode, int min_target_rows, cudaStream_t s) {
+  RSD_LAUNCH((build_pass_kernel), 1, 1024, 0, s, st, which, (int)mode, min_target_rows);
   return launched(1);
 }
 
 // ---------------------------------------------------------------------------------------------
-// Decode-phase control.  Phase 0: the draft writes y^_i for every live row (slot b = row b).
-// Phase 1: the target writes y_i for the rejected rows (slot i = rej_idx[i]).
+// Decode-phase control.  Phase 0: the draft writes y^_i for every live row that is not waiting for
+// the target (slot b = row b).  Phase 1: the target writes y_i for the waiting rows (slot i = rej_idx[i]).
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(1024) decode_begin_kernel(RowState st, int phase) {
   RSD_PDL_SYNC();
@@ -118,7 +124,7 @@ __global__ void __launch_bounds__(1024) decode_begin_kernel(RowState st, int pha
   const int b = threadIdx.x;
   int part = 0;
   if (b < st.B) {
-    part = st.live[b] != 0 && (phase == 0 || st.accept[b] == 0);
+    part = st.live[b] != 0 && (phase == 0 ? st.waiting[b] == 0 : st.waiting[b] != 0);
     st.gen_active[b] = part;
     st.gen_len[phase][b] = 0;
   }
@@ -212,8 +218,10 @@ cudaError_t launch_decode_update(const RowState& st, int which, int phase, unsig
 
 // ---------------------------------------------------------------------------------------------
 // Gate + compaction.  Acceptance criterion of Algorithm 2 with the weighting functions of Table 1
-// (binary step: accept iff r >= delta); rejected live rows are listed in ascending order by a
-// warp ballot + popcount prefix, and their draft / PRM caches are rolled back to the step start.
+// (binary step: accept iff r >= delta) for the rows that took a draft step; a rejected row starts
+// waiting for the target and its draft / PRM caches are rolled back to the step start.  All waiting
+// rows (those of earlier calls included) are listed in ascending order by a warp ballot + popcount
+// prefix.
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ float omega_weight(int kind, float r, float delta, float alpha) {
   switch (kind) {
@@ -256,13 +264,15 @@ __global__ void __launch_bounds__(1024) gate_kernel(RowState st, float delta, Lo
   RSD_PDL_SYNC();
   __shared__ int wsum[33];
   const int b = threadIdx.x;
-  bool live = false, rejected = false;
+  bool live = false, waits = false;
   if (b < st.B) {
     live = st.live[b] != 0;
-    int acc = 0;
-    if (live) {
+    waits = live && st.waiting[b] != 0;
+    int code = 0;                      // rows that took no draft step in this call keep 0
+    if (live && !waits) {
       const float r = st.rewards[b];
       const float w = omega_weight(lp.omega_kind, r, delta, lp.omega_alpha);
+      int acc;
       if (w == 0.f) acc = 0;
       else if (w == 1.f) acc = 1;
       else {
@@ -272,20 +282,23 @@ __global__ void __launch_bounds__(1024) gate_kernel(RowState st, float delta, Lo
       }
       const uint8_t f = st.forced_accept[b];
       if (f <= 1) acc = f;
-    } else {
+      code = acc ? 1 : 2;
+      if (!acc) {
+        waits = true;
+        st.waiting[b] = 1;
+        st.kv_len[0][b] = st.z_len[b] - 1;   // draft: drop y^_i, keep z_i minus its newest token
+        st.kv_len[1][b] = st.z_len[b];       // PRM: drop y^_i
+      }
+    } else if (!live) {
       st.rewards[b] = 0.f;
     }
-    st.accept[b] = (uint8_t)acc;
-    rejected = live && !acc;
+    st.accept[b] = (uint8_t)code;
   }
+  const int n_live = __syncthreads_count(live);
   int total;
-  const int rank = ballot_rank(rejected, wsum, &total);
-  if (rejected) {
-    st.rej_idx[rank] = b;
-    st.kv_len[0][b] = st.z_len[b] - 1;   // draft: drop y^_i, keep z_i minus its newest token
-    st.kv_len[1][b] = st.z_len[b];       // PRM: drop y^_i
-  }
-  if (b == 0) st.n_rej[0] = total;
+  const int rank = ballot_rank(waits, wsum, &total);
+  if (waits) st.rej_idx[rank] = b;
+  if (b == 0) { st.n_rej[0] = total; st.n_live[0] = n_live; }
 }
 
 cudaError_t launch_gate(const RowState& st, float delta, const LoopParams& lp, cudaStream_t s) {
@@ -355,15 +368,18 @@ cudaError_t launch_gate_compact_large(const float* rewards, const uint8_t* live,
 // Commit: y_i <- accept ? y^_i : target step; the row stops when EOS is in y_i, after max_steps
 // steps, or when another step would not fit.  One block per row.
 // ---------------------------------------------------------------------------------------------
-__global__ void commit_kernel(RowState st, LoopParams lp, int32_t* out_tokens, int32_t* out_len, float* out_rewards,
-                              uint8_t* out_accept, uint8_t* out_live) {
+__global__ void commit_kernel(RowState st, LoopParams lp, int target_ran, int32_t* out_tokens, int32_t* out_len,
+                              float* out_rewards, uint8_t* out_accept, uint8_t* out_live, uint8_t* out_role,
+                              uint8_t* out_waiting) {
   RSD_PDL_SYNC();
   const int b = blockIdx.x;
   const bool live = st.live[b] != 0;
-  const int acc = st.accept[b];
-  const int phase = acc ? 0 : 1;
-  const int n = live ? st.gen_len[phase][b] : 0;
-  const int32_t* y = st.gen_tok[phase] + (size_t)b * st.C;
+  const int code = st.accept[b];
+  const bool waits = live && st.waiting[b] != 0;
+  // the step this row commits now: the accepted draft step, the target's step, or none (it waits)
+  const int phase = (live && code == 1) ? 0 : (waits && target_ran) ? 1 : -1;
+  const int n = phase >= 0 ? st.gen_len[phase][b] : 0;
+  const int32_t* y = st.gen_tok[phase >= 0 ? phase : 0] + (size_t)b * st.C;
   int has_eos = 0;
   for (int j = threadIdx.x; j < st.C; j += blockDim.x) {
     const int t = j < n ? y[j] : 0;
@@ -374,24 +390,29 @@ __global__ void commit_kernel(RowState st, LoopParams lp, int32_t* out_tokens, i
   if (threadIdx.x == 0) {
     out_len[b] = n;
     out_rewards[b] = live ? st.rewards[b] : 0.f;
-    out_accept[b] = live ? (uint8_t)acc : 0;
-    int still = 0;
-    if (live) {
+    out_accept[b] = (live && code == 1) ? 1 : 0;
+    out_role[b] = (uint8_t)((live ? code : 0) | (phase == 1 ? 4 : 0));
+    int still = live ? 1 : 0, still_waits = waits ? 1 : 0;
+    if (phase >= 0) {
       const int z = st.z_len[b] + n;
       const int steps = st.n_steps[b] + 1;
       st.z_len[b] = z;
       st.n_steps[b] = steps;
       still = !(has_eos || steps >= lp.max_steps || z + st.C > st.S);
       st.live[b] = still;
+      if (phase == 1) { st.waiting[b] = 0; still_waits = 0; }
     }
     out_live[b] = (uint8_t)still;
+    out_waiting[b] = (uint8_t)(still && still_waits);
   }
 }
 
-cudaError_t launch_commit(const RowState& st, const LoopParams& lp, int32_t* out_tokens, int32_t* out_len,
-                          float* out_rewards, uint8_t* out_accept, uint8_t* out_live, cudaStream_t s) {
+cudaError_t launch_commit(const RowState& st, const LoopParams& lp, int target_ran, int32_t* out_tokens,
+                          int32_t* out_len, float* out_rewards, uint8_t* out_accept, uint8_t* out_live,
+                          uint8_t* out_role, uint8_t* out_waiting, cudaStream_t s) {
   if (st.B <= 0) return cudaSuccess;
-  RSD_LAUNCH((commit_kernel), st.B, 128, 0, s, st, lp, out_tokens, out_len, out_rewards, out_accept, out_live);
+  RSD_LAUNCH((commit_kernel), st.B, 128, 0, s, st, lp, target_ran, out_tokens, out_len, out_rewards, out_accept,
+             out_live, out_role, out_waiting);
   return launched(1);
 }
 

@@ -41,27 +41,29 @@ def compare_state(eng, loop):
     assert g["next_page"] == o["next_page"]
 
 
-def parity_step(eng, loop, delta, *, tol_logits, tol_reward, margin_tok, margin_gate, stats=None):
+def parity_step(eng, loop, delta, *, tol_logits, tol_reward, margin_tok, margin_gate, stats=None, min_target_rows=1):
     """One step on both sides.  The GPU is forced onto the oracle's tokens; its own samples and its
     own gate decisions are checked wherever the oracle's margins are clear."""
     B = len(loop.rows)
-    o = loop.step(delta)
+    o = loop.step(delta, min_target_rows=min_target_rows)
     eng.force_tokens(DRAFT, o["draft_tokens"])
     eng.force_tokens(TARGET, o["target_tokens"])
     # the gate is left to the GPU except where the oracle's reward sits within the margin of delta
     amb = [None] * B
     for b in range(B):
-        if o["step_len"][b] > 0 and abs(o["rewards"][b] - delta) <= margin_gate:
+        if o["drafted"][b] and abs(o["rewards"][b] - delta) <= margin_gate:
             amb[b] = int(o["accept"][b])
     eng.force_accept(amb)
-    g = eng.step(delta)
-    live_before = o["step_len"] > 0
+    g = eng.step(delta, min_target_rows)
+    live_before = (o["step_len"] > 0) | (o["drafted"] > 0) | (o["waiting"] > 0)
     # rewards, gate, outputs
     err_r = np.abs(g["rewards"].astype(np.float64) - o["rewards"])[live_before]
     assert err_r.size == 0 or err_r.max() <= tol_reward, f"reward error {err_r.max()}"
     assert np.array_equal(g["accept"], o["accept"])
     assert np.array_equal(g["step_len"], o["step_len"])
     assert np.array_equal(g["live"], o["live"])
+    if min_target_rows > 1:
+        assert np.array_equal(g["waiting"], o["waiting"])
     for b in range(B):
         n = o["step_len"][b]
         assert g["step_tokens"][b, :n].tolist() == list(o["step_tokens"][b])

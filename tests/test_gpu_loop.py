@@ -176,3 +176,52 @@ def test_call_order_and_argument_errors():
     assert r["accept"].all() and (r["step_len"] > 0).all()
     with pytest.raises(RsdError):                        # a PRM must not carry an lm head, and vice versa
         Engine(models[0], models[0], models[2], max_batch=2, max_seq_tokens=48, max_step_tokens=8, max_steps=2, step_end_id=13)
+
+
+@pytest.mark.parametrize("delta,min_rows", [(0.47, 3), (0.49, 4)])
+def test_queued_rejections_match_the_oracle(delta, min_rows):
+    """rsd_step_queued: rejected rows wait until min_rows wait, then one target pass serves all of
+    them.  Compared call by call with the oracle under the same rule (tokens, rewards, gate, waiting
+    flags, cursors, page tables, the list of waiting rows, counters), and at the end every row's
+    sequence equals the one the lock-step oracle loop writes."""
+    shapes = (ri.SHAPES["tiny_draft"], ri.SHAPES["tiny_draft"], ri.SHAPES["tiny_target"])
+    prompts = ri.prompts(31, 6, 5, 20, 1024)
+    # thresholds just under the tiny PRM's reward range (0.5 +- 0.08): a rejection every few steps
+    kw = dict(max_step_tokens=6, max_steps=6, max_seq_tokens=96, step_end_id=3, step_end_mod=5, temperature=0.7, seed=4)
+    eng, loop = build_pair(shapes, bf16=False, prompts=prompts, loop_kwargs=kw)
+    _, lock = build_pair(shapes, bf16=False, prompts=prompts, loop_kwargs=kw)
+    stats = {}
+    waited = flushed = 0
+    for _ in range(40):
+        if not any(r.live for r in loop.rows):
+            break
+        g, o = parity_step(eng, loop, delta, tol_logits=2e-4, tol_reward=1e-5, margin_tok=1e-3, margin_gate=1e-4,
+                           stats=stats, min_target_rows=min_rows)
+        waited += int(o["waiting"].sum())
+        flushed += int(o["flushed"])
+    assert not any(r.live for r in loop.rows)
+    assert waited > 0 and flushed > 0
+    compare_counters(eng, loop)
+    while any(r.live for r in lock.rows):
+        lock.step(delta)
+    assert [r.z for r in loop.rows] == [r.z for r in lock.rows]
+    print("queued rejections, min_rows", min_rows, stats)
+
+
+def test_queued_with_min_rows_one_is_rsd_step_and_bad_arguments():
+    from paper_2501_19324_b200 import lib
+    shapes = (ri.SHAPES["tiny_draft"], ri.SHAPES["tiny_draft"], ri.SHAPES["tiny_target"])
+    prompts = ri.prompts(32, 4, 5, 12, 1024)
+    kw = dict(max_step_tokens=5, max_steps=3, max_seq_tokens=64, step_end_id=3, temperature=0.7, seed=5)
+    a, _ = build_pair(shapes, bf16=False, prompts=prompts, loop_kwargs=kw)
+    b, _ = build_pair(shapes, bf16=False, prompts=prompts, loop_kwargs=kw)
+    for _ in range(3):
+        ra = a.step(0.5)
+        out = {k: np.zeros_like(v) for k, v in ra.items()}
+        ptr = [out[k].ctypes.data for k in ("step_tokens", "step_len", "rewards", "accept", "live", "waiting")]
+        assert lib().rsd_step_queued(b.ctx, 0.5, 1, None, *ptr) == 0
+        for k in ("step_tokens", "step_len", "rewards", "accept", "live"):
+            assert np.array_equal(ra[k], out[k]), k
+        assert not out["waiting"].any()
+    assert lib().rsd_step_queued(b.ctx, 0.5, 0, None, *ptr) == -1
+    assert b"min_target_rows" in lib().rsd_last_error(b.ctx)
