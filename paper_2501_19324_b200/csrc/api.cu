@@ -64,6 +64,7 @@ struct rsd_ctx {
   int32_t *o_tokens = nullptr, *o_len = nullptr;
   float* o_rewards = nullptr;
   uint8_t *o_accept = nullptr, *o_live = nullptr, *o_role = nullptr, *o_waiting = nullptr;
+  float* norm_ssq = nullptr;   // [B][chunks] sums of squares of the residual stream (decode path)
   char* pinned = nullptr;
   size_t pinned_bytes = 0;
   void* gemm_scratch = nullptr;
@@ -212,6 +213,7 @@ size_t layout_workspace(const rsd_config& cfg, const rsd_model* const ms[3], rsd
   void* act = TAKE(float, (size_t)T * dm.f);
   float* logits = TAKE(float, (size_t)B * dm.v);
   unsigned long long* sample_best = TAKE(unsigned long long, B);
+  float* norm_ssq = TAKE(float, (size_t)B * norm_chunks(dm.d));
   float2* rope[3];
   for (int w = 0; w < 3; ++w) rope[w] = TAKE(float2, (size_t)S * (ms[w]->head_dim / 2));
   float* dbg[2] = {nullptr, nullptr};
@@ -241,6 +243,7 @@ size_t layout_workspace(const rsd_config& cfg, const rsd_model* const ms[3], rsd
     c->attn_lo = (char*)attn + (size_t)T * dm.hq * 2;
     c->act_lo = (char*)act + (size_t)T * dm.f * 2;
     c->sample_best = sample_best;
+    c->norm_ssq = norm_ssq;
     for (int w = 0; w < 3; ++w) c->mdl[w].rope = rope[w];
     c->dbg_logits[0] = dbg[0]; c->dbg_logits[1] = dbg[1];
     c->d_scalars = scal;
@@ -300,7 +303,7 @@ int drain_gemm_events(rsd_ctx* c) {
 // `pending` (nullable): the caller's next kernel adds up K-split partial sums itself, so the GEMM may
 // leave them in the scratch; *pending then describes them (splits == 1: y is complete).
 int gemm(rsd_ctx* c, const ModelHost& M, const void* W, const void* xin, const void* xin_lo, float* y, int Mrows, int N,
-         int K, int accumulate, const int32_t* n_active, SplitSum* pending, cudaStream_t s) {
+         int K, int accumulate, const int32_t* n_active, SplitSum* pending, cudaStream_t s, RowScale rs = RowScale()) {
   // ragged passes: every stride-th GEMM; decode: every GEMM of the iterations chosen by decode_phase
   const bool pick = c->in_decode ? c->time_this_iter
                                  : (c->time_stride > 0 && (c->gemm_calls++ % (uint64_t)c->time_stride) == 0);
@@ -308,7 +311,7 @@ int gemm(rsd_ctx* c, const ModelHost& M, const void* W, const void* xin, const v
   if (timed) CU(cudaEventRecord(c->ev[2 * c->ev_used], s));
   int splits = 1;
   CU(launch_gemm(M.m.dtype, W, xin, M.split ? xin_lo : nullptr, y, Mrows, N, K, accumulate, 0, c->gemm_scratch,
-                 c->gemm_scratch_bytes, n_active, pending ? &splits : nullptr, s));
+                 c->gemm_scratch_bytes, n_active, pending ? &splits : nullptr, s, rs));
   if (pending) { pending->splits = splits; pending->partials = gemm_partials(c->gemm_scratch); }
   if (timed) {
     CU(cudaEventRecord(c->ev[2 * c->ev_used + 1], s));
@@ -366,6 +369,48 @@ int forward_pass(rsd_ctx* c, int which, PassView p, cudaStream_t s) {
   return RSD_OK;
 }
 
+// Decode pass of a bf16 model with RMSNorm folded into its neighbours: the kernel that completes the
+// residual stream (reduce_norm) also writes the next GEMM's operand x * gain and the sums of squares, and
+// that GEMM scales its result rows by the RMSNorm denominator; the K-split sums of the qkv product are
+// added up by the RoPE kernel.  Ten kernels per layer instead of thirteen.  On return h / h_lo hold
+// x * final_gain and norm_ssq the sums of squares of the final residual stream.
+bool fused_decode_ok(const ModelHost& M) { return M.m.dtype == RSD_BF16 && M.split && M.m.d_model % 4 == 0; }
+
+int forward_decode_fused(rsd_ctx* c, int which, PassView p, const void* final_gain, cudaStream_t s) {
+  const ModelHost& M = c->mdl[which];
+  const rsd_model& m = M.m;
+  const int d = m.d_model, H = m.n_heads, KV = m.n_kv_heads, hd = m.head_dim, F = m.d_ffn;
+  const int T = p.T;
+  if (T <= 0) return RSD_OK;
+  const RowScale rs{c->norm_ssq, norm_chunks(d), 1.f / (float)d, m.rms_eps};
+  CU(launch_embed(m.dtype, m.tok_embed, p, c->x, d, s));
+  CU(launch_reduce_norm(nullptr, 1, c->x, M.norm1[0], c->h, c->h_lo, c->norm_ssq, T, d, p.n_active, s));
+  for (int l = 0; l < m.n_layers; ++l) {
+    KvView kv{M.kv_pool + (size_t)l * M.layer_stride, c->st.page_table[which], c->max_pages, M.kv_dtype == 3 ? 1 : 0};
+    SplitSum qkv_pending, gu_pending, x_pending;
+    int rc = gemm(c, M, M.wqkv[l], c->h, c->h_lo, c->qkv, T, (H + 2 * KV) * hd, d, 0, p.n_active, &qkv_pending, s, rs);
+    if (rc) return rc;
+    CU(launch_rope_kv(M.kv_dtype, c->qkv, qkv_pending, p, c->q, kv, M.rope, H, KV, hd, s));
+    CU(launch_attn_decode(M.kv_dtype, c->q, kv.pool_layer, kv.page_table, kv.max_pages, p.tok_row, p.tok_pos, 1,
+                          c->attn, c->attn_lo, m.dtype, T, H, KV, hd, c->S, c->attn_scratch, c->attn_scratch_bytes,
+                          p.n_active, s));
+    rc = gemm(c, M, M.wo[l], c->attn, c->attn_lo, c->x, T, d, H * hd, 1, p.n_active, &x_pending, s);
+    if (rc) return rc;
+    CU(launch_reduce_norm(x_pending.partials, x_pending.splits, c->x, M.norm2[l], c->h, c->h_lo, c->norm_ssq, T, d,
+                          p.n_active, s));
+    rc = gemm(c, M, M.wgu[l], c->h, c->h_lo, c->gu, T, 2 * F, d, 0, p.n_active, &gu_pending, s, rs);
+    if (rc) return rc;
+    CU(launch_swiglu(m.dtype, c->gu, gu_pending, c->act, c->act_lo, T, F, p.n_active, s));
+    x_pending = SplitSum();
+    rc = gemm(c, M, M.wdown[l], c->act, c->act_lo, c->x, T, d, F, 1, p.n_active, &x_pending, s);
+    if (rc) return rc;
+    const void* next_gain = l + 1 < m.n_layers ? M.norm1[l + 1] : final_gain;
+    CU(launch_reduce_norm(x_pending.partials, x_pending.splits, c->x, next_gain, c->h, c->h_lo, c->norm_ssq, T, d,
+                          p.n_active, s));
+  }
+  return RSD_OK;
+}
+
 // Multi-token pass over the flat list built by launch_build_pass, `chunk` tokens at a time.
 int run_ingest(rsd_ctx* c, int which, int n_total, bool want_reward, cudaStream_t s) {
   for (int c0 = 0; c0 < n_total; c0 += c->chunk) {
@@ -399,11 +444,17 @@ int decode_iteration(rsd_ctx* c, int which, int phase, int n_slots, cudaStream_t
   const rsd_model& m = M.m;
   CU(launch_decode_prepare(c->st, which, n_slots, s));
   PassView p{c->st.pass_tok_id, c->st.pass_tok_row, c->st.pass_tok_pos, n_slots, c->st.n_active};
-  int rc = forward_pass(c, which, p, s);
-  if (rc) return rc;
-  CU(launch_rmsnorm(m.dtype, c->x, m.final_norm, c->h, M.split ? c->h_lo : nullptr, n_slots, m.d_model, m.rms_eps,
-                    nullptr, p.n_active, SplitSum(), s));
-  rc = gemm(c, M, m.head, c->h, c->h_lo, c->logits, n_slots, m.vocab, m.d_model, 0, p.n_active, nullptr, s);
+  int rc;
+  if (fused_decode_ok(M)) {
+    if ((rc = forward_decode_fused(c, which, p, m.final_norm, s))) return rc;
+    const RowScale rs{c->norm_ssq, norm_chunks(m.d_model), 1.f / (float)m.d_model, m.rms_eps};
+    rc = gemm(c, M, m.head, c->h, c->h_lo, c->logits, n_slots, m.vocab, m.d_model, 0, p.n_active, nullptr, s, rs);
+  } else {
+    if ((rc = forward_pass(c, which, p, s))) return rc;
+    CU(launch_rmsnorm(m.dtype, c->x, m.final_norm, c->h, M.split ? c->h_lo : nullptr, n_slots, m.d_model, m.rms_eps,
+                      nullptr, p.n_active, SplitSum(), s));
+    rc = gemm(c, M, m.head, c->h, c->h_lo, c->logits, n_slots, m.vocab, m.d_model, 0, p.n_active, nullptr, s);
+  }
   if (rc) return rc;
   if (c->dbg_logits[phase]) {
     RSD_LAUNCH((scatter_logits_kernel), n_slots, 256, 0, s, c->logits, c->st.pass_tok_row, c->dbg_logits[phase], m.vocab, c->C,

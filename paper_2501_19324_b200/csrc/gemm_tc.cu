@@ -116,7 +116,7 @@ template <int MT> struct TcCfg {
   static constexpr int kBBytes = MT * kTileK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
   static constexpr int kTmemCols = MT < 32 ? 32 : MT;
-  static constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + 256;
+  static constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + 256 + 512;   // barriers, row scales
   // instruction descriptor: fp32 accumulate, bf16 A and B, both K-major, N = MT, M = 128
   static constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(MT >> 3) << 17) | ((uint32_t)(kTileN >> 4) << 24);
 };
@@ -128,7 +128,7 @@ __global__ void __launch_bounds__(192, TcCfg<MT>::kCtasPerSm)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x,
                const __grid_constant__ CUtensorMap tm_x_lo, float* __restrict__ Y,
                int M, int N, int K, int accumulate, int splits, int kb_per_split, float* __restrict__ partials,
-               int* __restrict__ err, const int32_t* __restrict__ n_active) {
+               int* __restrict__ err, const int32_t* __restrict__ n_active, RowScale rs) {
   // Programmatic dependent launch: the next kernel may be scheduled at once; this kernel sets itself
   // up and starts streaming its WEIGHT tiles (never written by any kernel) while its predecessors are
   // still running, and only then waits for them (griddepcontrol.wait) before it touches activations,
@@ -143,6 +143,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
   uint64_t* tmem_full = empty + Cfg::kStages;
   uint32_t* tmem_slot = (uint32_t*)(tmem_full + 1);
   volatile uint32_t* flags = tmem_slot + 1;   // [0] abort
+  float* row_scale = (float*)(smem + (size_t)Cfg::kStages * Cfg::kStageBytes + 256);   // [kRows <= 128]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n0 = blockIdx.x * kTileN, m0 = blockIdx.y * kRows, split = blockIdx.z;
@@ -236,6 +237,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
   } else {
     // ---------------- epilogue: TMEM -> registers -> global ----------------
     asm volatile("griddepcontrol.wait;" ::: "memory");   // y and the partial sums belong to earlier kernels until now
+    if (rs.ssq != nullptr) {
+      // RMSNorm denominators of this tile's x rows, one per epilogue thread, while the MMAs run
+      const int r = threadIdx.x;
+      if (r < kRows && m0 + r < M) {
+        float sum = 0.f;
+        for (int c = 0; c < rs.n_chunks; ++c) sum += rs.ssq[(size_t)(m0 + r) * rs.n_chunks + c];
+        row_scale[r] = rsqrtf(sum * rs.inv_d + rs.eps);
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");   // the four epilogue warps only
+    }
     bool ok = false;
     for (uint32_t i = 0; i < kWaitLimit && !ok; ++i) {
       ok = mbar_try_wait(tmem_full, 0);
@@ -267,6 +278,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
 #pragma unroll
             for (int j = 0; j < 16; ++j) v[j] += w[j];
           }
+        }
+        if (rs.ssq != nullptr) {
+#pragma unroll
+          for (int j = 0; j < 16; ++j)
+            if (c + j < m_valid) v[j] *= row_scale[c + j];
         }
         if (n < N) {
 #pragma unroll
@@ -409,7 +425,7 @@ TcPlan plan_tc(int M, int N, int K, bool split_operand) {
 template <int MT, bool SPLIT>
 cudaError_t launch_mt(const CUtensorMap& tw, const CUtensorMap& tx, const CUtensorMap& txl, float* y, int M, int N, int K,
                       int accumulate, const TcPlan& p, float* partials, int* err, const int32_t* n_active,
-                      bool defer_reduce, cudaStream_t s) {
+                      bool defer_reduce, RowScale rs, cudaStream_t s) {
   static bool configured = false;
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<MT, SPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TcCfg<MT>::kSmemBytes);
@@ -418,7 +434,7 @@ cudaError_t launch_mt(const CUtensorMap& tw, const CUtensorMap& tx, const CUtens
   }
   dim3 grid(p.n_tiles, p.m_tiles, p.splits);
   RSD_LAUNCH((gemm_tc_kernel<MT, SPLIT>), grid, 192, TcCfg<MT>::kSmemBytes, s, tw, tx, txl, y, M, N, K, accumulate, p.splits,
-                                                                     p.kb_per_split, partials, err, n_active);
+                                                                     p.kb_per_split, partials, err, n_active, rs);
   if (p.splits > 1 && !defer_reduce) {
     const size_t total4 = (size_t)M * N / 4;
     const int blocks = (int)std::min<size_t>((total4 + 255) / 256, 148 * 8);
@@ -449,13 +465,15 @@ const float* gemm_partials(const void* scratch) { return (const float*)((const c
 
 cudaError_t launch_gemm_tc(const void* W, const void* x, const void* x_lo, float* y, int M, int N, int K, int accumulate,
                            void* scratch, size_t scratch_bytes, const int32_t* n_active, int* deferred_splits,
-                           cudaStream_t s) {
+                           cudaStream_t s, RowScale rs) {
   if (deferred_splits) *deferred_splits = 1;
   if (M <= 0) return cudaSuccess;
+  if (rs.ssq != nullptr && accumulate) return cudaErrorInvalidValue;
   if (!scratch || scratch_bytes < gemm_scratch_bytes(M)) return cudaErrorInvalidValue;
   if (((uintptr_t)W & 15) || ((uintptr_t)x & 15) || ((uintptr_t)x_lo & 15)) return cudaErrorMisalignedAddress;
   const bool split_operand = x_lo != nullptr;
   const TcPlan p = plan_tc(M, N, K, split_operand);
+  if (rs.ssq != nullptr && p.rows > 128) return cudaErrorInvalidValue;   // one epilogue thread per x row of the tile
   if (deferred_splits) *deferred_splits = p.splits;
   const bool defer = deferred_splits != nullptr;
   CUtensorMap tw, tx, txl;
@@ -464,7 +482,7 @@ cudaError_t launch_gemm_tc(const void* W, const void* x, const void* x_lo, float
   else txl = tx;
   int* err = (int*)((char*)scratch + kCounterBytes);
   float* partials = (float*)((char*)scratch + kCounterBytes + 256);
-#define RSD_TC(MT, SP) return launch_mt<MT, SP>(tw, tx, txl, y, M, N, K, accumulate, p, partials, err, n_active, defer, s)
+#define RSD_TC(MT, SP) return launch_mt<MT, SP>(tw, tx, txl, y, M, N, K, accumulate, p, partials, err, n_active, defer, rs, s)
   if (split_operand) {
     switch (p.mt) {
       case 16: RSD_TC(16, true);
@@ -486,12 +504,13 @@ cudaError_t launch_gemm_tc(const void* W, const void* x, const void* x_lo, float
 
 cudaError_t launch_gemm(int dtype, const void* W, const void* x, const void* x_lo, float* y, int M, int N, int K,
                         int accumulate, int impl, void* scratch, size_t scratch_bytes, const int32_t* n_active,
-                        int* deferred_splits, cudaStream_t s) {
+                        int* deferred_splits, cudaStream_t s, RowScale rs) {
   if (deferred_splits) *deferred_splits = 1;
   const bool tc_ok = gemm_tc_supported(dtype, M, N, K) && scratch && scratch_bytes >= gemm_scratch_bytes(M);
   // the tensor-core path wins for every M (an M = 1 GEMV included: TMA streaming beats the SIMT loads)
   if (impl == 2 || (impl == 0 && tc_ok))
-    return launch_gemm_tc(W, x, x_lo, y, M, N, K, accumulate, scratch, scratch_bytes, n_active, deferred_splits, s);
+    return launch_gemm_tc(W, x, x_lo, y, M, N, K, accumulate, scratch, scratch_bytes, n_active, deferred_splits, s, rs);
+  if (rs.ssq != nullptr) return cudaErrorNotSupported;
   return launch_gemm_simt(dtype, W, x, dtype == 1 ? x_lo : nullptr, y, M, N, K, accumulate, n_active, s);
 }
 

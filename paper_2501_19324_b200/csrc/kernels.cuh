@@ -23,6 +23,15 @@ struct SplitSum {
   int splits = 1;
 };
 
+// Per-row scale of a GEMM whose input rows were left un-normalised: row m of the result is multiplied by
+// rsqrt(sum_c ssq[m * n_chunks + c] * inv_d + eps), i.e. the RMSNorm denominator of input row m whose
+// squares were summed chunk by chunk by the producer of the input (reduce_norm).  ssq == nullptr: no scale.
+struct RowScale {
+  const float* ssq = nullptr;
+  int n_chunks = 0;
+  float inv_d = 0.f, eps = 0.f;
+};
+
 // A pass pushes T token slots through one model.  Slot t carries token tok_id[t] of row tok_row[t]
 // at position tok_pos[t]; tok_row[t] < 0 marks an idle slot.  When n_active is non-null and reads
 // 0 on the device the whole pass is skipped (every row of the decode phase has finished).
@@ -63,13 +72,19 @@ size_t gemm_scratch_bytes_any();
 // 1 means y holds the finished result.
 cudaError_t launch_gemm_tc(const void* W, const void* x, const void* x_lo, float* y, int M, int N, int K, int accumulate,
                            void* scratch, size_t scratch_bytes, const int32_t* n_active, int* deferred_splits,
-                           cudaStream_t s);
+                           cudaStream_t s, RowScale rs = RowScale());
 const float* gemm_partials(const void* scratch);
 
 // impl: 0 = by shape, 1 = SIMT split-K GEMV, 2 = tcgen05.
 cudaError_t launch_gemm(int dtype, const void* W, const void* x, const void* x_lo, float* y, int M, int N, int K,
                         int accumulate, int impl, void* scratch, size_t scratch_bytes, const int32_t* n_active,
-                        int* deferred_splits, cudaStream_t s);
+                        int* deferred_splits, cudaStream_t s, RowScale rs = RowScale());
+// x (+)= sum of the K-split partial sums [splits][M][d] (splits == 1: x is complete already); then the
+// un-normalised RMSNorm operand of the next GEMM: hi + lo = x * gain as two bf16 arrays, and the sums of
+// squares of x per 256-column chunk, ssq [M][ceil(d / 256)], for that GEMM's RowScale.
+cudaError_t launch_reduce_norm(const float* partials, int splits, float* x, const void* gain, void* hi, void* lo,
+                               float* ssq, int M, int d, const int32_t* n_active, cudaStream_t s);
+inline int norm_chunks(int d) { return (d + 255) / 256; }
 cudaError_t launch_rope_table(float2* table, int n_pos, int hd, float theta, cudaStream_t s);
 // Splits qkv [T, (H+2KV)*hd] (fp32): rotated q -> q_out [T, H*hd] fp32; rotated k and v -> KV pages.
 // kv_dtype: element type of the cache: 0 fp32, 1 bf16, 2 fp16.

@@ -98,6 +98,65 @@ cudaError_t launch_rmsnorm(int dtype, float* x, const void* gain, void* out, voi
 }
 
 // ---------------------------------------------------------------------------------------------
+// Residual update + un-normalised RMSNorm operand (decode path of bf16 models).  One block per (row,
+// 256-column chunk): x (+)= sum of the K-split partial sums of the GEMM that feeds the residual stream;
+// hi + lo = x * gain (two bf16 arrays, the operand of the next GEMM); ssq[row][chunk] = sum of x^2
+// over the chunk.  The next GEMM multiplies its result rows by rsqrt(sum_chunk ssq / d + eps)
+// (RowScale), which is RMSNorm applied after the product instead of before it.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(64)
+reduce_norm_kernel(const float* __restrict__ partials, int splits, float* __restrict__ x,
+                   const __nv_bfloat16* __restrict__ gain, __nv_bfloat16* __restrict__ hi,
+                   __nv_bfloat16* __restrict__ lo, float* __restrict__ ssq, int M, int d, int n_chunks,
+                   const int32_t* n_active) {
+  RSD_PDL_SYNC();
+  RSD_SKIP_IF_IDLE(n_active);
+  __shared__ float red[2];
+  const int m = blockIdx.y, c = blockIdx.x;
+  const int col = c * 256 + threadIdx.x * 4;
+  float ss = 0.f;
+  if (col < d) {
+    const size_t o = (size_t)m * d + col;
+    float4 v = *reinterpret_cast<const float4*>(x + o);
+    if (splits > 1) {
+      const size_t stride = (size_t)M * d;
+      int sidx = 0;
+      for (; sidx + 4 <= splits; sidx += 4) {
+        float4 a[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) a[u] = __ldcg(reinterpret_cast<const float4*>(partials + (size_t)(sidx + u) * stride + o));
+#pragma unroll
+        for (int u = 0; u < 4; ++u) { v.x += a[u].x; v.y += a[u].y; v.z += a[u].z; v.w += a[u].w; }
+      }
+      for (; sidx < splits; ++sidx) {
+        const float4 a = __ldcg(reinterpret_cast<const float4*>(partials + (size_t)sidx * stride + o));
+        v.x += a.x; v.y += a.y; v.z += a.z; v.w += a.w;
+      }
+      *reinterpret_cast<float4*>(x + o) = v;
+    }
+    ss = v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+    store_operand<__nv_bfloat16>(hi, lo, o, v.x * to_f32(gain[col]));
+    store_operand<__nv_bfloat16>(hi, lo, o + 1, v.y * to_f32(gain[col + 1]));
+    store_operand<__nv_bfloat16>(hi, lo, o + 2, v.z * to_f32(gain[col + 2]));
+    store_operand<__nv_bfloat16>(hi, lo, o + 3, v.w * to_f32(gain[col + 3]));
+  }
+  ss = warp_sum(ss);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  if (threadIdx.x == 0) ssq[(size_t)m * n_chunks + c] = red[0] + red[1];
+}
+
+cudaError_t launch_reduce_norm(const float* partials, int splits, float* x, const void* gain, void* hi, void* lo,
+                               float* ssq, int M, int d, const int32_t* n_active, cudaStream_t s) {
+  if (M <= 0) return cudaSuccess;
+  if (d % 4 != 0) return cudaErrorInvalidValue;
+  const int n_chunks = norm_chunks(d);
+  RSD_LAUNCH((reduce_norm_kernel), dim3(n_chunks, M), 64, 0, s, partials, splits, x, (const __nv_bfloat16*)gain,
+             (__nv_bfloat16*)hi, (__nv_bfloat16*)lo, ssq, M, d, n_chunks, n_active);
+  return launched(1);
+}
+
+// ---------------------------------------------------------------------------------------------
 // Split-K SIMT GEMV / skinny GEMM:  y[m, n] (+)= sum_k x[m, k] W[n, k]
 // A block of 8 warps covers nb = 8/ks output columns; the ks warps of one column each stream a
 // strided share of the row with 16-byte loads and their partial sums meet in shared memory, in a
@@ -243,33 +302,36 @@ __global__ void rope_kv_kernel(const float* __restrict__ qkv, const float* __res
   const size_t block = (size_t)KV * kPageTokens * hd;
   KT* kbase = pool + (size_t)page * pf * block;
   KT* vbase = kbase + block;
-  const int n_rot = (H + KV) * half;
-  for (int idx = threadIdx.x; idx < n_rot; idx += blockDim.x) {
-    const int head = idx / half, i = idx % half;
-    const float a = split_sum(qkv, partials, splits, src0 + head * hd + i, sstride);
-    const float b = split_sum(qkv, partials, splits, src0 + head * hd + i + half, sstride);
-    const float2 c = cs[i];
-    const float ra = a * c.x - b * c.y, rb = b * c.x + a * c.y;
-    if (head < H) {
-      q_out[(size_t)t * H * hd + head * hd + i] = ra;
-      q_out[(size_t)t * H * hd + head * hd + i + half] = rb;
-    } else {
-      KT* k = kbase + ((size_t)(head - H) * kPageTokens + slot) * hd;
-      const KT ka = from_f32<KT>(ra), kb2 = from_f32<KT>(rb);
-      k[i] = ka;
-      k[i + half] = kb2;
-      if (pf == 4) {
-        k[2 * block + i] = from_f32<KT>(ra - to_f32(ka));
-        k[2 * block + i + half] = from_f32<KT>(rb - to_f32(kb2));
+  // one block per (token, head): query and key heads are rotated, value heads copied
+  const int head = blockIdx.y;
+  if (head < H + KV) {
+    for (int i = threadIdx.x; i < half; i += blockDim.x) {
+      const float a = split_sum(qkv, partials, splits, src0 + head * hd + i, sstride);
+      const float b = split_sum(qkv, partials, splits, src0 + head * hd + i + half, sstride);
+      const float2 c = cs[i];
+      const float ra = a * c.x - b * c.y, rb = b * c.x + a * c.y;
+      if (head < H) {
+        q_out[(size_t)t * H * hd + head * hd + i] = ra;
+        q_out[(size_t)t * H * hd + head * hd + i + half] = rb;
+      } else {
+        KT* k = kbase + ((size_t)(head - H) * kPageTokens + slot) * hd;
+        const KT ka = from_f32<KT>(ra), kb2 = from_f32<KT>(rb);
+        k[i] = ka;
+        k[i + half] = kb2;
+        if (pf == 4) {
+          k[2 * block + i] = from_f32<KT>(ra - to_f32(ka));
+          k[2 * block + i + half] = from_f32<KT>(rb - to_f32(kb2));
+        }
       }
     }
-  }
-  for (int idx = threadIdx.x; idx < KV * hd; idx += blockDim.x) {
-    const int head = idx / hd, i = idx % hd;
-    const float v = split_sum(qkv, partials, splits, src0 + (H + KV) * hd + idx, sstride);
-    const KT vh = from_f32<KT>(v);
-    vbase[((size_t)head * hd + i) * kPageTokens + slot] = vh;
-    if (pf == 4) vbase[2 * block + ((size_t)head * hd + i) * kPageTokens + slot] = from_f32<KT>(v - to_f32(vh));
+  } else {
+    const int vh_idx = head - H - KV;
+    for (int i = threadIdx.x; i < hd; i += blockDim.x) {
+      const float v = split_sum(qkv, partials, splits, src0 + (size_t)head * hd + i, sstride);
+      const KT vh = from_f32<KT>(v);
+      vbase[((size_t)vh_idx * hd + i) * kPageTokens + slot] = vh;
+      if (pf == 4) vbase[2 * block + ((size_t)vh_idx * hd + i) * kPageTokens + slot] = from_f32<KT>(v - to_f32(vh));
+    }
   }
 }
 
@@ -277,11 +339,11 @@ cudaError_t launch_rope_kv(int kv_dtype, const float* qkv, SplitSum pending, Pas
                            const float2* rope, int H, int KV, int hd, cudaStream_t s) {
   if (p.T <= 0) return cudaSuccess;
   if (kv_dtype == 2 || kv_dtype == 3)
-    RSD_LAUNCH((rope_kv_kernel<__half>), p.T, 256, 0, s, qkv, pending.partials, pending.splits, p, q_out, (__half*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd, 2 + 2 * kv.v_extra);
+    RSD_LAUNCH((rope_kv_kernel<__half>), dim3(p.T, H + 2 * KV), 64, 0, s, qkv, pending.partials, pending.splits, p, q_out, (__half*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd, 2 + 2 * kv.v_extra);
   else if (kv_dtype == 1)
-    RSD_LAUNCH((rope_kv_kernel<__nv_bfloat16>), p.T, 256, 0, s, qkv, pending.partials, pending.splits, p, q_out, (__nv_bfloat16*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd, 2 + 2 * kv.v_extra);
+    RSD_LAUNCH((rope_kv_kernel<__nv_bfloat16>), dim3(p.T, H + 2 * KV), 64, 0, s, qkv, pending.partials, pending.splits, p, q_out, (__nv_bfloat16*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd, 2 + 2 * kv.v_extra);
   else
-    RSD_LAUNCH((rope_kv_kernel<float>), p.T, 256, 0, s, qkv, pending.partials, pending.splits, p, q_out, (float*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd, 2 + 2 * kv.v_extra);
+    RSD_LAUNCH((rope_kv_kernel<float>), dim3(p.T, H + 2 * KV), 64, 0, s, qkv, pending.partials, pending.splits, p, q_out, (float*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd, 2 + 2 * kv.v_extra);
   return launched(1);
 }
 
