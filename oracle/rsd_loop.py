@@ -22,6 +22,16 @@ needs, under one deterministic policy, so it can be compared bit for bit:
   * the ascending list of rejected rows, and token / FLOPs counters (Section 3.3: 2N FLOPs per
     inference token of an N-parameter model, PRM included).
 
+Merged PRM (`prm_shares_draft`).  Appendix B.3 builds the PRM as a projection layer on top of the
+final transformer layer of a language model, and the discussion of model merging (Section 4, "PRM
+overhead") asks for one model that is both policy and PRM.  When the PRM's trunk IS the draft's
+trunk, the reward of y^_i needs no second pass over (z_i, y^_i): the draft's cache already covers
+everything but the last token of y^_i, so one more single-token forward of the draft at that token
+gives the hidden state the reward head reads.  The draft cursor is not advanced by it (the token
+is fed again as the first input of the next decode), so the cursors and every token are exactly
+those of the loop with a separate PRM whose trunk weights equal the draft's; the PRM keeps no
+cache at all.
+
 Queued rejections (`min_target_rows` > 1).  Rows never interact, so nothing in Algorithm 1 says that
 all rows must take their i-th step together.  The paper counts the cost of the target by the tokens
 it generates (Section 3.3), but a batched target pass reads all of M's weights whether one row or
@@ -55,6 +65,7 @@ class LoopConfig:
     page_tokens: int = 16
     omega_kind: int = 1            # Table 1 row: 0 constant, 1 binary step, 2 clip, 3 r/(1+r), 4 logistic
     omega_b: float = 0.0           # alpha of the logistic; the first parameter is the delta of each step
+    prm_shares_draft: bool = False  # the PRM is a reward head on the draft's trunk (merged serving, see below)
     pool_pages: tuple = (1 << 30, 1 << 30, 1 << 30)
     keep_logits: bool = False
 
@@ -123,17 +134,20 @@ class OracleRSD:
             if len(row.z) + self.cfg.max_step_tokens > self.cfg.max_seq_tokens:
                 row.live = False        # no room for even one step: the row never starts
         live_rows = [b for b, row in enumerate(self.rows) if row.live]
+        shared = self.cfg.prm_shares_draft
         for b in live_rows:
             self._reserve(DRAFT, b, len(self.rows[b].z) - 1)
         for b in live_rows:
-            self._reserve(PRM, b, len(self.rows[b].z))
+            if not shared:
+                self._reserve(PRM, b, len(self.rows[b].z))
         for b in live_rows:
             row = self.rows[b]
             n = len(row.z)
             self._ingest(DRAFT, b, n - 1, row.z)
-            self._ingest(PRM, b, n, row.z)
             self.counters["ingest_tokens"][DRAFT] += n - 1
-            self.counters["ingest_tokens"][PRM] += n
+            if not shared:
+                self._ingest(PRM, b, n, row.z)
+                self.counters["ingest_tokens"][PRM] += n
 
     def _generate_step(self, which: int, b: int, forced=None, trace=None) -> list:
         """One step from model `which` given the row's context z (Algorithm 1: m(x, y_{1:i-1}) or
@@ -184,9 +198,11 @@ class OracleRSD:
         for b in run_rows:
             res["drafted"][b] = 1
 
-        # draft step y^_i for every live row that is not waiting for the target
+        # draft step y^_i for every live row that is not waiting for the target (with a merged PRM the
+        # draft also caches the step's last token when it scores it: one more position)
+        shared = cfg.prm_shares_draft
         for b in run_rows:
-            self._reserve(DRAFT, b, len(self.rows[b].z) - 1 + cfg.max_step_tokens)
+            self._reserve(DRAFT, b, len(self.rows[b].z) - 1 + cfg.max_step_tokens + (1 if shared else 0))
         for b in run_rows:
             tr = dict(sampled=[], margin=[], logits=[])
             f = forced_draft[b] if forced_draft is not None else None
@@ -195,9 +211,19 @@ class OracleRSD:
 
         # reward r_i = r(y^_i | z_i), read at the last token of the draft step
         for b in run_rows:
-            self._reserve(PRM, b, len(self.rows[b].z) + len(res["draft_tokens"][b]))
+            if not shared:
+                self._reserve(PRM, b, len(self.rows[b].z) + len(res["draft_tokens"][b]))
         for b in run_rows:
             row = self.rows[b]
+            if shared:
+                # the draft's cache holds z_i and all of y^_i but its last token: push that token
+                # through the draft's trunk, read the reward head, leave the cursor where it was
+                pos = row.kv_len[DRAFT]
+                assert pos == len(row.z) + len(res["draft_tokens"][b]) - 1
+                h = self.models[DRAFT].forward(row.caches[DRAFT], [res["draft_tokens"][b][-1]], pos)
+                row.reward = self.models[PRM].reward(h[0])
+                self.counters["score_tokens"] += 1
+                continue
             seq = row.z + res["draft_tokens"][b]
             n_known = len(row.z) - row.kv_len[PRM]      # committed tokens the PRM has not cached yet
             h = self._ingest(PRM, b, len(seq), seq)
@@ -217,7 +243,8 @@ class OracleRSD:
                 # drop the draft step from the draft and PRM caches; the target will write y_i
                 row.waiting = True
                 row.kv_len[DRAFT] = len(row.z) - 1
-                row.kv_len[PRM] = len(row.z)
+                if not shared:
+                    row.kv_len[PRM] = len(row.z)
                 self.counters["discarded_draft_tokens"] += len(res["draft_tokens"][b])
         wait_rows = [b for b in range(B) if self.rows[b].live and self.rows[b].waiting]
         res["rej_idx"] = wait_rows

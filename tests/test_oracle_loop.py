@@ -321,3 +321,44 @@ def test_queued_flush_rule_and_cursors(tiny_weights):
     # every live row waits -> flush although fewer than min_target_rows wait
     r = loop.step(0.5, forced_accept=[0, 0, 0, 0], min_target_rows=100)
     assert r["flushed"] and r["rej_idx"] == [0, 1, 2, 3]
+
+
+def test_merged_prm_equals_a_separate_prm_with_the_drafts_trunk(tiny_weights):
+    """A PRM that is a reward head on the draft's trunk (Appendix B.3: a projection layer on top of the
+    final transformer layer) scored from the draft's own cache plus one single-token forward must give
+    the rewards of a separately cached PRM whose trunk weights are the draft's -- and with them the same
+    gate decisions, tokens, draft / target cursors and pages -- while the PRM keeps no cache and bills
+    one processed token per scored step."""
+    d, p, t = tiny_weights
+    dm, tm = OracleModel(d, DRAFT), OracleModel(t, TARGET)
+    twin = dict(d)                      # the draft's trunk ...
+    twin["head"], twin["head_kind"], twin["final_norm"] = p["head"], p["head_kind"], p["final_norm"]   # ... the PRM's head
+    pm_twin = OracleModel(twin, PRM)
+    pm_head_only = OracleModel(dict(p, layers=[]), PRM)      # merged mode never touches PRM layers
+    cfg = dict(max_step_tokens=5, max_steps=4, max_seq_tokens=64, step_end_id=2, step_end_mod=4, temperature=0.7, seed=8)
+    tok, off = ri.prompts(12, 4, 4, 9, 1024)
+    prompts = [tok[off[b]:off[b + 1]].tolist() for b in range(4)]
+    sep = OracleRSD(dm, pm_twin, tm, LoopConfig(**cfg))
+    sep.prefill(prompts)
+    delta = float(np.median(sep.step(0.0)["rewards"]))
+    sep = OracleRSD(dm, pm_twin, tm, LoopConfig(**cfg))
+    mrg = OracleRSD(dm, pm_head_only, tm, LoopConfig(prm_shares_draft=True, **cfg))
+    sep.prefill(prompts)
+    mrg.prefill(prompts)
+    saw = set()
+    for _ in range(cfg["max_steps"]):
+        a, b = sep.step(delta), mrg.step(delta)
+        assert np.allclose(a["rewards"], b["rewards"], rtol=0, atol=1e-12)
+        assert np.array_equal(a["accept"], b["accept"]) and np.array_equal(a["live"], b["live"])
+        assert [list(x) for x in a["step_tokens"]] == [list(x) for x in b["step_tokens"]]
+        saw |= set(int(x) for x, n in zip(a["accept"], a["step_len"]) if n)
+        sa, sb = sep.state(), mrg.state()
+        for w in (DRAFT, TARGET):
+            assert np.array_equal(sa["kv_len"][w], sb["kv_len"][w])
+        assert sa["pages"][TARGET] == sb["pages"][TARGET]
+        assert not sb["kv_len"][PRM].any() and not sb["n_pages"][PRM].any()
+    assert saw == {0, 1}
+    for key in ("gen_tokens", "steps", "accepted_steps", "rejected_steps", "discarded_draft_tokens"):
+        assert sep.counters[key] == mrg.counters[key]
+    assert mrg.counters["ingest_tokens"][PRM] == 0
+    assert mrg.counters["score_tokens"] == mrg.counters["steps"]     # one token per scored step (lock-step)
