@@ -209,6 +209,7 @@ def workload_config(args) -> dict:
                         + (f"delta {args.delta}" if getattr(args, "delta", None) is not None else "delta at the 70% accept quantile"),
             "batch": B, "max_step_tokens": args.cap or cap, "replicas": args.gpus,
             "kv_cache": "fp16 hi+lo pairs" if kv_extended(args) else "fp16",
+            "prm": "head on the draft's trunk (prm_shares_draft)" if getattr(args, "merged_prm", False) else "separate model",
             "schedule": "lock-step rsd_step" if getattr(args, "queue", 1) == 1 else
                         f"rsd_step_queued, target pass once {args.queue} rows wait",
             "l2": "weights and KV read per decode iteration exceed the 126 MB L2 (no flush needed)"}
@@ -249,12 +250,20 @@ def run_ours(args, rank: int, world: int):
         cap = args.cap          # profiling aid: shorter steps (recorded in the config line)
     shapes = [ri.SHAPES[d], ri.SHAPES[p], ri.SHAPES[t]]
     heads = (ri.HEAD_LM, ri.HEAD_REWARD_SIGMOID, ri.HEAD_LM)
-    models = [Model(sh, ri.gpu_model_tensors(sh, slot, 0, True, hk), hk)
+    merged = bool(args.merged_prm)
+    if merged and shapes[1] != shapes[0]:
+        raise SystemExit("--merged-prm needs a PRM of the draft's shape")
+    models = [Model(sh, ri.gpu_model_tensors(sh, slot, 0, True, hk), hk, head_only=merged and slot == 1)
               for slot, (sh, hk) in enumerate(zip(shapes, heads))]
+    if merged:                      # only the PRM's embedding row count, final norm and head are read
+        for k in ("wqkv", "wo", "wgu", "wdown", "norm1", "norm2"):
+            models[1].t[k] = []
+        torch.cuda.empty_cache()
     n_steps = args.warmup + args.steps
     S = hi + n_steps * cap
     eng = Engine(*models, max_batch=B, max_seq_tokens=S, max_step_tokens=cap, max_steps=n_steps + 1,
-                 step_end_id=13, temperature=0.7, seed=0, kv_extended=kv_extended(args))
+                 step_end_id=13, temperature=0.7, seed=0, kv_extended=kv_extended(args),
+                 prm_shares_draft=int(merged))
     tokens, offsets = rank_prompts(rank, B, lo, hi, shapes[0].vocab)
     pinned_tokens = torch.from_numpy(tokens).pin_memory()
 
@@ -508,6 +517,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--delta", type=float, default=None, help="fixed threshold instead of the 70 %% accept quantile")
     ap.add_argument("--cap", type=int, default=0, help="override the step cap (profiling aid)")
+    ap.add_argument("--merged-prm", action="store_true", dest="merged_prm",
+                    help="prm_shares_draft: the PRM is a head on the draft's trunk (not the headline configuration)")
     ap.add_argument("--queue", type=int, default=1,
                     help="min_target_rows of rsd_step_queued (1 = rsd_step, the headline configuration)")
     ap.add_argument("--kv-extended", type=int, default=None, choices=[0, 1], dest="kv_extended",

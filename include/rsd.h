@@ -96,6 +96,14 @@ typedef struct {
                                  fp16 hi + lo pairs (twice the KV bytes) and queries / softmax weights
                                  enter as hi + lo pairs (attention accurate to ~2^-20); for deep models
                                  whose logits must stay within 3e-2 of an fp64 reference               */
+  int32_t prm_shares_draft;   /* 1: merged serving (Appendix B.3: the PRM is a projection layer on a language
+                                 model's final layer; Section 4 on merging PRM and policy): the PRM is its
+                                 final_norm and scalar head on the DRAFT's trunk.  r_i is read after one
+                                 single-token pass of the draft over the last token of the draft step,
+                                 from the draft's own cache; the PRM keeps no cache and its separate
+                                 scoring pass disappears.  The prm descriptor must repeat the draft's
+                                 dimensions and dtype; its layer arrays and kv_pool[RSD_PRM] may be NULL.
+                                 Results equal those of a separate PRM whose trunk weights are the draft's */
   /* caller-allocated device memory, sizes as reported by rsd_query_sizes (or larger)        */
   void* kv_pool[3];           /* RSD_DRAFT / RSD_PRM / RSD_TARGET                            */
   size_t kv_bytes[3];

@@ -38,7 +38,7 @@ class rsd_config(ctypes.Structure):
     _fields_ = [(n, c_int32) for n in ("max_batch", "max_seq_tokens", "max_step_tokens", "max_steps", "page_tokens",
                                         "step_end_id", "eos_id", "step_end_mod")] + \
                [("temperature", c_float), ("seed", c_uint64), ("omega_kind", c_int32), ("omega_alpha", c_float),
-                ("max_chunk_tokens", c_int32), ("debug_flags", c_int32), ("kv_extended", c_int32),
+                ("max_chunk_tokens", c_int32), ("debug_flags", c_int32), ("kv_extended", c_int32), ("prm_shares_draft", c_int32),
                 ("kv_pool", c_void_p * 3), ("kv_bytes", c_size_t * 3), ("workspace", c_void_p),
                 ("workspace_bytes", c_size_t)]
 
@@ -125,9 +125,10 @@ class Model:
     """A transformer's weights as torch CUDA tensors plus the rsd_model descriptor pointing at them.
 
     tensors: tok_embed [V, d], final_norm [d], head [V, d] or [d], and per-layer lists wqkv
-    [(H+2KV)hd, d], wo [d, Hhd], wgu [2F, d], wdown [d, F], norm1 [d], norm2 [d]."""
+    [(H+2KV)hd, d], wo [d, Hhd], wgu [2F, d], wdown [d, F], norm1 [d], norm2 [d].
+    head_only: a PRM that is a head on the draft's trunk (prm_shares_draft) carries no layers."""
 
-    def __init__(self, shape, tensors: dict, head_kind: int):
+    def __init__(self, shape, tensors: dict, head_kind: int, head_only: bool = False):
         import torch
         self.shape, self.t, self.head_kind = shape, tensors, head_kind
         dt = tensors["tok_embed"].dtype
@@ -136,6 +137,9 @@ class Model:
         L = shape.n_layers
         self._arrays = {}
         for k in ("wqkv", "wo", "wgu", "wdown", "norm1", "norm2"):
+            if head_only:
+                self._arrays[k] = None
+                continue
             assert len(tensors[k]) == L
             for w in tensors[k]:
                 assert w.is_cuda and w.is_contiguous() and w.dtype == dt
@@ -144,8 +148,8 @@ class Model:
                               shape.d_ffn, shape.vocab, self.dtype, shape.rope_theta, shape.rms_eps, head_kind,
                               tensors["tok_embed"].data_ptr(), tensors["final_norm"].data_ptr(),
                               tensors["head"].data_ptr(),
-                              *[ctypes.cast(self._arrays[k], POINTER(c_void_p)) for k in
-                                ("wqkv", "wo", "wgu", "wdown", "norm1", "norm2")])
+                              *[ctypes.cast(self._arrays[k], POINTER(c_void_p)) if self._arrays[k] is not None
+                                else POINTER(c_void_p)() for k in ("wqkv", "wo", "wgu", "wdown", "norm1", "norm2")])
 
 
 class Engine:
@@ -153,7 +157,8 @@ class Engine:
 
     def __init__(self, draft: Model, prm: Model, target: Model, *, max_batch, max_seq_tokens, max_step_tokens,
                  max_steps, step_end_id, eos_id=-1, step_end_mod=0, temperature=0.0, seed=0, omega_kind=1,
-                 omega_alpha=0.0, max_chunk_tokens=0, debug_flags=0, kv_bytes=None, kv_extended=0):
+                 omega_alpha=0.0, max_chunk_tokens=0, debug_flags=0, kv_bytes=None, kv_extended=0,
+                 prm_shares_draft=0):
         import torch
         if not torch.cuda.is_available():
             raise RsdError(-4, "no CUDA device: this library has no CPU fallback")
@@ -161,7 +166,8 @@ class Engine:
         self.B_max, self.S, self.C = max_batch, max_seq_tokens, max_step_tokens
         self.max_pages = (max_seq_tokens + 15) // 16
         cfg = rsd_config(max_batch, max_seq_tokens, max_step_tokens, max_steps, 16, step_end_id, eos_id, step_end_mod,
-                         temperature, seed, omega_kind, omega_alpha, max_chunk_tokens, debug_flags, kv_extended)
+                         temperature, seed, omega_kind, omega_alpha, max_chunk_tokens, debug_flags, kv_extended,
+                         prm_shares_draft)
         _check(lib().rsd_query_sizes(draft.desc, prm.desc, target.desc, cfg))
         if kv_bytes is not None:
             for i in range(3):

@@ -173,7 +173,7 @@ size_t layout_workspace(const rsd_config& cfg, const rsd_model* const ms[3], rsd
 #define TAKE(type, n) (type*)P(L.take(sizeof(type) * (size_t)(n)))
   // row state
   RowState st{};
-  st.B = 0; st.S = S; st.C = C; st.max_pages = max_pages;
+  st.B = 0; st.S = S; st.C = C; st.max_pages = max_pages; st.prm_shared = cfg.prm_shares_draft ? 1 : 0;
   st.z_len = TAKE(int32_t, B); st.live = TAKE(int32_t, B); st.n_steps = TAKE(int32_t, B);
   st.tok = TAKE(int32_t, (size_t)B * S);
   for (int w = 0; w < 3; ++w) {
@@ -573,6 +573,7 @@ int rsd_query_sizes(const rsd_model* draft, const rsd_model* prm, const rsd_mode
   }
   const int max_pages = (cfg->max_seq_tokens + kPageTokens - 1) / kPageTokens;
   for (int i = 0; i < 3; ++i) cfg->kv_bytes[i] = kv_pool_bytes(*ms[i], cfg->max_batch * max_pages, cfg->kv_extended);
+  if (cfg->prm_shares_draft) cfg->kv_bytes[RSD_PRM] = 0;   // the PRM reads the draft's cache
   cfg->workspace_bytes = layout_workspace(*cfg, ms, nullptr);
   return RSD_OK;
 }
@@ -583,7 +584,7 @@ int rsd_create(const rsd_config* cfg, rsd_ctx** out) {
   *out = nullptr;
   int rc = check_config(cfg, &why);
   if (rc) return fail(nullptr, rc, "config: %s", why);
-  if (!cfg->workspace || !cfg->kv_pool[0] || !cfg->kv_pool[1] || !cfg->kv_pool[2])
+  if (!cfg->workspace || !cfg->kv_pool[0] || (!cfg->kv_pool[1] && !cfg->prm_shares_draft) || !cfg->kv_pool[2])
     return fail(nullptr, RSD_ERR_ARG, "workspace and KV pools must be provided by the caller%s");
   int dev_count = 0;
   if (cudaGetDeviceCount(&dev_count) != cudaSuccess || dev_count == 0)
@@ -611,10 +612,13 @@ int rsd_load_models(rsd_ctx* c, const rsd_model* draft, const rsd_model* prm, co
   for (int i = 0; i < 3; ++i) {
     int rc = check_model(ms[i], &why);
     if (rc) return fail(c, rc, "model: %s", why);
-    if (!ms[i]->tok_embed || !ms[i]->final_norm || !ms[i]->head || !ms[i]->wqkv || !ms[i]->wo || !ms[i]->wgu ||
-        !ms[i]->wdown || !ms[i]->norm1 || !ms[i]->norm2)
+    const bool head_only = i == RSD_PRM && c->cfg.prm_shares_draft;
+    if (!ms[i]->tok_embed || !ms[i]->final_norm || !ms[i]->head ||
+        (!head_only && (!ms[i]->wqkv || !ms[i]->wo || !ms[i]->wgu || !ms[i]->wdown || !ms[i]->norm1 || !ms[i]->norm2)))
       return fail(c, RSD_ERR_ARG, "model: null weight pointer%s");
   }
+  if (c->cfg.prm_shares_draft && (prm->d_model != draft->d_model || prm->dtype != draft->dtype))
+    return fail(c, RSD_ERR_ARG, "prm_shares_draft: the PRM head must have the draft's width and dtype%s");
   if (draft->head_kind != RSD_HEAD_LM || target->head_kind != RSD_HEAD_LM || prm->head_kind == RSD_HEAD_LM)
     return fail(c, RSD_ERR_ARG, "draft and target need lm heads, the PRM a scalar head%s");
   const size_t need = layout_workspace(c->cfg, ms, nullptr);
@@ -624,6 +628,16 @@ int rsd_load_models(rsd_ctx* c, const rsd_model* draft, const rsd_model* prm, co
   for (int w = 0; w < 3; ++w) {
     ModelHost& M = c->mdl[w];
     M.m = *ms[w];
+    if (w == RSD_PRM && c->cfg.prm_shares_draft) {
+      // head on the draft's trunk: no layers, no cache of its own
+      M.m.wqkv = M.m.wo = M.m.wgu = M.m.wdown = M.m.norm1 = M.m.norm2 = nullptr;
+      M.elem = M.m.dtype == RSD_BF16 ? 2 : 4;
+      M.split = M.m.dtype == RSD_BF16;
+      M.n_params = count_params(M.m);
+      M.pool_pages = 0;
+      c->st.pool_pages[w] = 0;
+      continue;
+    }
     const int L = M.m.n_layers;
     M.wqkv.assign(ms[w]->wqkv, ms[w]->wqkv + L); M.wo.assign(ms[w]->wo, ms[w]->wo + L);
     M.wgu.assign(ms[w]->wgu, ms[w]->wgu + L); M.wdown.assign(ms[w]->wdown, ms[w]->wdown + L);
@@ -694,8 +708,9 @@ int rsd_prefill(rsd_ctx* c, const int32_t* tokens, const int32_t* offsets, int32
   RSD_LAUNCH((init_rows_kernel), B, 128, 0, s, c->st, c->st.pass_tok_id, c->st.pass_tok_row, B);
   CU(launched(1));
   CU(cudaStreamSynchronize(s));  // the staging buffers are reused below
+  const bool merged = c->cfg.prm_shares_draft != 0;
   CU(launch_reserve_pages(c->st, RSD_DRAFT, kReservePrefillDraft, 1, s));
-  CU(launch_reserve_pages(c->st, RSD_PRM, kReservePrefillPrm, 1, s));
+  if (!merged) CU(launch_reserve_pages(c->st, RSD_PRM, kReservePrefillPrm, 1, s));
   Scalars sc;
   CU(launch_build_pass(c->st, RSD_DRAFT, kPassIngestDraft, 1, s));
   rc = read_scalars(c, s, &sc);
@@ -703,14 +718,37 @@ int rsd_prefill(rsd_ctx* c, const int32_t* tokens, const int32_t* offsets, int32
   rc = run_ingest(c, RSD_DRAFT, sc.n_tok, false, s);
   if (rc) return rc;
   c->ctr.ingest_tokens[RSD_DRAFT] += sc.n_tok;
-  CU(launch_build_pass(c->st, RSD_PRM, kPassScorePrm, 1, s));
-  rc = read_scalars(c, s, &sc);
-  if (rc) return rc;
-  rc = run_ingest(c, RSD_PRM, sc.n_tok, false, s);
-  if (rc) return rc;
-  c->ctr.ingest_tokens[RSD_PRM] += sc.n_tok;
+  if (!merged) {
+    CU(launch_build_pass(c->st, RSD_PRM, kPassScorePrm, 1, s));
+    rc = read_scalars(c, s, &sc);
+    if (rc) return rc;
+    rc = run_ingest(c, RSD_PRM, sc.n_tok, false, s);
+    if (rc) return rc;
+    c->ctr.ingest_tokens[RSD_PRM] += sc.n_tok;
+  }
   CU(cudaStreamSynchronize(s));
   c->prefilled = true;
+  return RSD_OK;
+}
+
+// Merged PRM: r_i from the draft's trunk.  The draft's cache holds z_i and y^_i up to the step's last
+// token; that token goes through the draft once more (its keys and values land beyond the cursor,
+// which does not move) and the PRM's final norm and head read the hidden state.
+static int score_with_draft_trunk(rsd_ctx* c, cudaStream_t s) {
+  const ModelHost& D = c->mdl[RSD_DRAFT];
+  const rsd_model& prm = c->mdl[RSD_PRM].m;
+  const int B = c->st.B;
+  CU(launch_score_prepare(c->st, s));
+  PassView p{c->st.pass_tok_id, c->st.pass_tok_row, c->st.pass_tok_pos, B, c->st.n_active};
+  int rc;
+  const bool was_in_decode = c->in_decode;
+  c->in_decode = true;             // GEMM timing: treated like a decode iteration that is not sampled
+  if (fused_decode_ok(D)) rc = forward_decode_fused(c, RSD_DRAFT, p, prm.final_norm, s);
+  else rc = forward_pass(c, RSD_DRAFT, p, s);
+  c->in_decode = was_in_decode;
+  if (rc) return rc;
+  CU(launch_reward(prm.dtype, c->x, prm.final_norm, prm.head, prm.head_kind, c->st.last_idx, 0, B, prm.d_model,
+                   prm.rms_eps, c->st.rewards, B, s));
   return RSD_OK;
 }
 
@@ -737,11 +775,17 @@ static int step_impl(rsd_ctx* c, float delta, int min_target_rows, void* cuda_st
   if ((rc = decode_phase(c, RSD_DRAFT, 0, B, s))) return rc;
   PHASE(2);
   // PRM: score y^_i at its last token
-  CU(launch_reserve_pages(c->st, RSD_PRM, kReserveScorePrm, 1, s));
-  CU(launch_build_pass(c->st, RSD_PRM, kPassScorePrm, 1, s));
-  if ((rc = read_scalars(c, s, &sc))) return rc;
-  const int n_prm = sc.n_tok;
-  if ((rc = run_ingest(c, RSD_PRM, n_prm, true, s))) return rc;
+  const bool merged = c->cfg.prm_shares_draft != 0;
+  int n_prm = 0;
+  if (merged) {
+    if ((rc = score_with_draft_trunk(c, s))) return rc;
+  } else {
+    CU(launch_reserve_pages(c->st, RSD_PRM, kReserveScorePrm, 1, s));
+    CU(launch_build_pass(c->st, RSD_PRM, kPassScorePrm, 1, s));
+    if ((rc = read_scalars(c, s, &sc))) return rc;
+    n_prm = sc.n_tok;
+    if ((rc = run_ingest(c, RSD_PRM, n_prm, true, s))) return rc;
+  }
   PHASE(3);
   // gate, compaction of the waiting rows; once enough of them wait: target catch-up and decode
   CU(launch_gate(c->st, delta, c->lp, s));
@@ -790,10 +834,10 @@ static int step_impl(rsd_ctx* c, float delta, int min_target_rows, void* cuda_st
     }
   }
   // counters (Section 3.3 accounting): draft tokens when they are generated, steps when they are committed
-  uint64_t gen_d = 0, gen_t = 0, n_acc = 0, n_tgt = 0, discarded = 0;
+  uint64_t gen_d = 0, gen_t = 0, n_acc = 0, n_tgt = 0, discarded = 0, n_scored = 0;
   for (int b = 0; b < B; ++b) {
     const int code = h_role[b] & 3;
-    if (code) gen_d += h_gen0[b];
+    if (code) { gen_d += h_gen0[b]; ++n_scored; }
     if (code == 1) ++n_acc;
     if (code == 2) discarded += h_gen0[b];
     if (h_role[b] & 4) { gen_t += h_gen1[b]; ++n_tgt; }
@@ -801,9 +845,9 @@ static int step_impl(rsd_ctx* c, float delta, int min_target_rows, void* cuda_st
   c->ctr.gen_tokens[RSD_DRAFT] += gen_d;
   c->ctr.gen_tokens[RSD_TARGET] += gen_t;
   c->ctr.ingest_tokens[RSD_DRAFT] += n_sync;
-  c->ctr.ingest_tokens[RSD_PRM] += (uint64_t)n_prm - gen_d;
+  c->ctr.ingest_tokens[RSD_PRM] += merged ? 0 : (uint64_t)n_prm - gen_d;
   c->ctr.ingest_tokens[RSD_TARGET] += target_runs ? n_catch : 0;
-  c->ctr.score_tokens += gen_d;
+  c->ctr.score_tokens += merged ? n_scored : gen_d;   // merged PRM: one token per scored step
   c->ctr.steps += n_acc + n_tgt; c->ctr.accepted_steps += n_acc; c->ctr.rejected_steps += n_tgt;
   c->ctr.discarded_draft_tokens += discarded;
   if (step_tokens) memcpy(step_tokens, h_tokens, sizeof(int32_t) * (size_t)B * c->C);

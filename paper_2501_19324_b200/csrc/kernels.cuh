@@ -137,6 +137,7 @@ cudaError_t launch_gate_compact_large(const float* rewards, const uint8_t* live,
 // ---- row state ------------------------------------------------------------------------------
 struct RowState {
   int B, S, C, max_pages;      // rows in use, tokens per row, step cap, pages per row
+  int prm_shared;              // 1: the PRM is a head on the draft's trunk and keeps no cache
   int32_t *z_len, *live, *n_steps, *tok;
   int32_t *kv_len[3], *n_pages[3], *page_table[3];
   int32_t* next_page;          // [3]
@@ -178,6 +179,9 @@ inline __host__ __device__ bool target_pass_due(int n_waiting, int n_live, int m
   return n_waiting > 0 && n_waiting >= (want < n_live ? want : n_live);
 }
 cudaError_t launch_decode_begin(const RowState& st, int phase, cudaStream_t s);
+// Merged PRM: one slot per row that took a draft step, carrying the step's last token at the draft's
+// cursor (which stays where it is); n_active = number of such rows, last_idx[b] = b for them.
+cudaError_t launch_score_prepare(const RowState& st, cudaStream_t s);
 cudaError_t launch_decode_prepare(const RowState& st, int which, int n_slots, cudaStream_t s);
 // best: packed winners left by launch_sample (cleared here).
 cudaError_t launch_decode_update(const RowState& st, int which, int phase, unsigned long long* best,

@@ -24,7 +24,7 @@ __global__ void __launch_bounds__(1024) reserve_pages_kernel(RowState st, int wh
     switch (mode) {
       case kReservePrefillDraft: need = live ? z - 1 : 0; break;
       case kReservePrefillPrm: need = live ? z : 0; break;
-      case kReserveStepDraft: need = runs ? z - 1 + st.C : 0; break;
+      case kReserveStepDraft: need = runs ? z - 1 + st.C + st.prm_shared : 0; break;   // merged PRM: + the step's last token
       case kReserveScorePrm: need = runs ? z + st.gen_len[0][b] : 0; break;
       case kReserveTarget:
         need = (live && st.waiting[b] && target_pass_due(st.n_rej[0], st.n_live[0], min_target_rows)) ? z - 1 + st.C : 0;
@@ -142,6 +142,32 @@ __global__ void __launch_bounds__(1024) decode_begin_kernel(RowState st, int pha
 
 cudaError_t launch_decode_begin(const RowState& st, int phase, cudaStream_t s) {
   RSD_LAUNCH((decode_begin_kernel), 1, 1024, 0, s, st, phase);
+  return launched(1);
+}
+
+__global__ void __launch_bounds__(1024) score_prepare_kernel(RowState st) {
+  RSD_PDL_SYNC();
+  const int b = threadIdx.x;
+  int part = 0;
+  if (b < st.B) {
+    const int n = st.gen_len[0][b];
+    part = st.live[b] != 0 && st.waiting[b] == 0 && n > 0;
+    if (part) {
+      st.pass_tok_id[b] = st.gen_tok[0][(size_t)b * st.C + n - 1];
+      st.pass_tok_pos[b] = st.kv_len[0][b];     // position of the step's last token; the cursor does not move
+      st.pass_tok_row[b] = b;
+      st.last_idx[b] = b;
+    } else {
+      st.pass_tok_row[b] = -1;
+      st.last_idx[b] = -1;
+    }
+  }
+  const int total = __syncthreads_count(part);
+  if (b == 0) st.n_active[0] = total;
+}
+
+cudaError_t launch_score_prepare(const RowState& st, cudaStream_t s) {
+  RSD_LAUNCH((score_prepare_kernel), 1, 1024, 0, s, st);
   return launched(1);
 }
 
@@ -287,7 +313,7 @@ __global__ void __launch_bounds__(1024) gate_kernel(RowState st, float delta, Lo
         waits = true;
         st.waiting[b] = 1;
         st.kv_len[0][b] = st.z_len[b] - 1;   // draft: drop y^_i, keep z_i minus its newest token
-        st.kv_len[1][b] = st.z_len[b];       // PRM: drop y^_i
+        if (!st.prm_shared) st.kv_len[1][b] = st.z_len[b];   // PRM: drop y^_i
       }
     } else if (!live) {
       st.rewards[b] = 0.f;

@@ -14,9 +14,10 @@ def build_pair(shapes, *, bf16, seed=0, prompts, loop_kwargs, engine_kwargs=None
     """shapes = (draft, prm, target) ModelShape.  Returns (engine, oracle_loop)."""
     from paper_2501_19324_b200 import Engine, Model, RSD_DEBUG_KEEP_LOGITS
     heads = (ri.HEAD_LM, ri.HEAD_REWARD_SIGMOID, ri.HEAD_LM)
-    gpu_models = [Model(sh, ri.gpu_model_tensors(sh, slot, seed, bf16, hk), hk)
+    merged = bool(loop_kwargs.get("prm_shares_draft"))     # the PRM is its head on the draft's trunk
+    gpu_models = [Model(sh, ri.gpu_model_tensors(sh, slot, seed, bf16, hk), hk, head_only=merged and slot == PRM)
                   for slot, (sh, hk) in enumerate(zip(shapes, heads))]
-    cpu_models = [OracleModel(ri.cpu_model_weights(sh, slot, seed, bf16, hk), slot)
+    cpu_models = [OracleModel(ri.cpu_model_weights(sh, slot, seed, bf16, hk, with_layers=not (merged and slot == PRM)), slot)
                   for slot, (sh, hk) in enumerate(zip(shapes, heads))]
     tokens, offsets = prompts
     B = len(offsets) - 1
@@ -24,6 +25,8 @@ def build_pair(shapes, *, bf16, seed=0, prompts, loop_kwargs, engine_kwargs=None
     kw.update({k: loop_kwargs[k] for k in ("max_seq_tokens", "max_step_tokens", "max_steps", "step_end_id",
                                            "eos_id", "step_end_mod", "temperature", "seed") if k in loop_kwargs})
     # loop_kwargs may also carry oracle-only settings (omega_kind, omega_b); the engine takes its own
+    if merged:
+        kw["prm_shares_draft"] = 1
     kw.update(engine_kwargs or {})
     eng = Engine(*gpu_models, **kw)
     loop = OracleRSD(*cpu_models, LoopConfig(keep_logits=True, **loop_kwargs))

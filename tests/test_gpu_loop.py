@@ -225,3 +225,26 @@ def test_queued_with_min_rows_one_is_rsd_step_and_bad_arguments():
         assert not out["waiting"].any()
     assert lib().rsd_step_queued(b.ctx, 0.5, 0, None, *ptr) == -1
     assert b"min_target_rows" in lib().rsd_last_error(b.ctx)
+
+
+@pytest.mark.parametrize("shapes,bf16,tol", [(TINY, False, TOL32), (MINI, True, TOL16)])
+def test_merged_prm_on_the_drafts_trunk(shapes, bf16, tol):
+    """prm_shares_draft: the reward comes from one more single-token pass of the draft and the PRM's head;
+    step-by-step parity with the oracle in the same mode (rewards, gate, tokens, cursors -- the PRM's stay
+    at zero -- pages, counters)."""
+    prompts = ri.prompts(41, 5, 6, 30, shapes[0].vocab)
+    kw = dict(max_step_tokens=6, max_steps=4, max_seq_tokens=96, step_end_id=3, step_end_mod=5, temperature=0.7,
+              seed=6, prm_shares_draft=True)
+    eng, loop = build_pair(shapes, bf16=bf16, prompts=prompts, loop_kwargs=kw)
+    probe = loop.step(0.0)["rewards"]
+    delta = float(np.median(probe))
+    eng, loop = build_pair(shapes, bf16=bf16, prompts=prompts, loop_kwargs=kw)
+    stats, seen = {}, set()
+    for _ in range(4):
+        g, o = parity_step(eng, loop, delta, stats=stats, **tol)
+        seen |= set(int(a) for a, n in zip(o["accept"], o["step_len"]) if n)
+    assert seen == {0, 1}
+    st = eng.state()
+    assert not st["kv_len"][1].any() and not st["n_pages"][1].any()
+    compare_counters(eng, loop)
+    print("merged PRM", "bf16" if bf16 else "fp32", stats)
