@@ -113,7 +113,9 @@ typedef struct {
 
 enum {
   RSD_DEBUG_KEEP_LOGITS = 1, /* keep every decode iteration's logits for rsd_debug_get_logits      */
-  RSD_DEBUG_NO_GRAPHS = 2    /* launch decode iterations kernel by kernel instead of as CUDA graphs */
+  RSD_DEBUG_NO_GRAPHS = 2,   /* launch decode iterations kernel by kernel instead of as CUDA graphs */
+  RSD_DEBUG_NO_MEGA = 4      /* run the layers of a decode iteration as separate kernels instead of the one
+                                persistent kernel (bf16 models, up to 64 rows)                        */
 };
 
 /* Fills cfg->kv_bytes[] (enough pages for max_batch rows of max_seq_tokens) and

@@ -16,6 +16,8 @@ RSD_F32, RSD_BF16 = 0, 1
 RSD_DRAFT, RSD_PRM, RSD_TARGET = 0, 1, 2
 RSD_HEAD_LM, RSD_HEAD_REWARD_SIGMOID, RSD_HEAD_REWARD_RAW = 0, 1, 2
 RSD_DEBUG_KEEP_LOGITS = 1
+RSD_DEBUG_NO_GRAPHS = 2
+RSD_DEBUG_NO_MEGA = 4
 ERRORS = {0: "RSD_OK", -1: "RSD_ERR_ARG", -2: "RSD_ERR_STATE", -3: "RSD_ERR_OOM_PAGES", -4: "RSD_ERR_CUDA",
           -5: "RSD_ERR_TIMEOUT", -6: "RSD_ERR_UNSUPPORTED"}
 

@@ -65,6 +65,10 @@ struct rsd_ctx {
   float* o_rewards = nullptr;
   uint8_t *o_accept = nullptr, *o_live = nullptr, *o_role = nullptr, *o_waiting = nullptr;
   float* norm_ssq = nullptr;   // [B][chunks] sums of squares of the residual stream (decode path)
+  // persistent decode kernel: parameter block per model (draft, target), built for the batch size mega_B
+  void* mega_block[3] = {nullptr, nullptr, nullptr};
+  int mega_B[3] = {0, 0, 0};
+  int32_t* mega_sync = nullptr;
   char* pinned = nullptr;
   size_t pinned_bytes = 0;
   void* gemm_scratch = nullptr;
@@ -213,7 +217,10 @@ size_t layout_workspace(const rsd_config& cfg, const rsd_model* const ms[3], rsd
   void* act = TAKE(float, (size_t)T * dm.f);
   float* logits = TAKE(float, (size_t)B * dm.v);
   unsigned long long* sample_best = TAKE(unsigned long long, B);
-  float* norm_ssq = TAKE(float, (size_t)B * norm_chunks(dm.d));
+  float* norm_ssq = TAKE(float, (size_t)B * 2 * norm_chunks(dm.d));   // room for 128-column chunks
+  void* mega_block[3] = {nullptr, nullptr, nullptr};
+  for (int w = 0; w < 3; w += 2) mega_block[w] = TAKE(char, mega_block_bytes(ms[w]->n_layers));
+  int32_t* mega_sync = TAKE(int32_t, 1024);
   float2* rope[3];
   for (int w = 0; w < 3; ++w) rope[w] = TAKE(float2, (size_t)S * (ms[w]->head_dim / 2));
   float* dbg[2] = {nullptr, nullptr};
@@ -244,6 +251,8 @@ size_t layout_workspace(const rsd_config& cfg, const rsd_model* const ms[3], rsd
     c->act_lo = (char*)act + (size_t)T * dm.f * 2;
     c->sample_best = sample_best;
     c->norm_ssq = norm_ssq;
+    for (int w = 0; w < 3; ++w) { c->mega_block[w] = mega_block[w]; c->mega_B[w] = 0; }
+    c->mega_sync = mega_sync;
     for (int w = 0; w < 3; ++w) c->mdl[w].rope = rope[w];
     c->dbg_logits[0] = dbg[0]; c->dbg_logits[1] = dbg[1];
     c->d_scalars = scal;
@@ -438,6 +447,53 @@ __global__ void scatter_logits_kernel(const float* logits, const int32_t* slot_r
   for (int i = threadIdx.x; i < V; i += blockDim.x) dst[i] = src[i];
 }
 
+MegaShape mega_shape(const ModelHost& M) {
+  const rsd_model& m = M.m;
+  return MegaShape{m.n_layers, m.d_model, m.n_heads, m.n_kv_heads, m.head_dim, m.d_ffn, m.dtype == RSD_BF16 && M.split, m.rms_eps};
+}
+
+// The persistent decode kernel serves bf16 models with 16-bit caches at up to 64 rows.
+bool mega_wanted(const rsd_ctx* c, int which) {
+  const ModelHost& M = c->mdl[which];
+  if (c->cfg.debug_flags & RSD_DEBUG_NO_MEGA) return false;
+  if (which == RSD_PRM || !fused_decode_ok(M) || (M.kv_dtype != 2 && M.kv_dtype != 3)) return false;
+  if (!mega_supported(mega_shape(M), c->st.B)) return false;
+  const MegaShape sh = mega_shape(M);
+  return mega_partials_floats(sh, c->st.B) * sizeof(float) + 4096 + 256 <= c->gemm_scratch_bytes && c->st.B * sh.KV <= 1000;
+}
+
+// (Re)builds the kernel's parameter block of model `which` for the current batch size.
+int ensure_mega(rsd_ctx* c, int which, cudaStream_t s) {
+  if (!mega_wanted(c, which)) { c->mega_B[which] = 0; return RSD_OK; }
+  if (c->mega_B[which] == c->st.B) return RSD_OK;
+  const ModelHost& M = c->mdl[which];
+  const int B = c->st.B;
+  MegaBuild a{};
+  a.shape = mega_shape(M);
+  a.B = B; a.max_pages = c->max_pages;
+  a.embed = M.m.tok_embed;
+  a.wqkv = M.m.wqkv; a.wo = M.m.wo; a.wgu = M.m.wgu; a.wdown = M.m.wdown; a.norm1 = M.m.norm1; a.norm2 = M.m.norm2;
+  a.kv_pool = M.kv_pool; a.layer_stride = M.layer_stride;
+  a.x = c->x; a.h = c->h; a.h_lo = c->h_lo; a.attn = c->attn; a.attn_lo = c->attn_lo; a.act = c->act; a.act_lo = c->act_lo;
+  a.partials = const_cast<float*>(gemm_partials(c->gemm_scratch));
+  a.ssq = c->norm_ssq;
+  // the decode-attention scratch holds the context-split partials: (max, sum) pairs first, outputs after them
+  const size_t head = ((sizeof(int32_t) * 2 * (size_t)c->B_max + 255) / 256) * 256;
+  int h_max = 0;
+  for (int w = 0; w < 3; ++w) h_max = std::max(h_max, c->mdl[w].m.n_heads);
+  a.part_ml = (float*)((char*)c->attn_scratch + head);
+  a.part_o = a.part_ml + (size_t)c->B_max * h_max * 32 * 2;
+  a.sync_words = c->mega_sync;
+  a.err = (int*)((char*)c->gemm_scratch + 4096);
+  a.rope = M.rope;
+  a.page_table = c->st.page_table[which];
+  cudaError_t e = mega_build(c->mega_block[which], a, s);
+  if (e == cudaErrorNotSupported) { c->mega_B[which] = 0; return RSD_OK; }
+  CU(e);
+  c->mega_B[which] = B;
+  return RSD_OK;
+}
+
 // Enqueues one decode iteration: (prepare, model pass, final norm, lm_head, sample, append).
 int decode_iteration(rsd_ctx* c, int which, int phase, int n_slots, cudaStream_t s) {
   const ModelHost& M = c->mdl[which];
@@ -445,7 +501,12 @@ int decode_iteration(rsd_ctx* c, int which, int phase, int n_slots, cudaStream_t
   CU(launch_decode_prepare(c->st, which, n_slots, s));
   PassView p{c->st.pass_tok_id, c->st.pass_tok_row, c->st.pass_tok_pos, n_slots, c->st.n_active};
   int rc;
-  if (fused_decode_ok(M)) {
+  if (c->mega_B[which] > 0 && c->mega_B[which] == c->st.B && n_slots == c->st.B) {
+    // the whole layer stack in one persistent kernel
+    CU(launch_decode_mega(c->mega_block[which], c->st.B, M.kv_dtype == 3, p, m.final_norm, s));
+    const RowScale rs{c->norm_ssq, m.d_model / 128, 1.f / (float)m.d_model, m.rms_eps};
+    rc = gemm(c, M, m.head, c->h, c->h_lo, c->logits, n_slots, m.vocab, m.d_model, 0, p.n_active, nullptr, s, rs);
+  } else if (fused_decode_ok(M)) {
     if ((rc = forward_decode_fused(c, which, p, m.final_norm, s))) return rc;
     const RowScale rs{c->norm_ssq, norm_chunks(m.d_model), 1.f / (float)m.d_model, m.rms_eps};
     rc = gemm(c, M, m.head, c->h, c->h_lo, c->logits, n_slots, m.vocab, m.d_model, 0, p.n_active, nullptr, s, rs);
@@ -499,7 +560,7 @@ int decode_phase(rsd_ctx* c, int which, int phase, int n_slots, cudaStream_t s) 
   CU(launch_decode_begin(c->st, phase, s));
   if (n_slots <= 0) return RSD_OK;
   const bool graphs = !(c->cfg.debug_flags & RSD_DEBUG_NO_GRAPHS);
-  if (graphs) n_slots = c->st.B;   // fixed shape: slots beyond the phase's rows are idle
+  if (graphs || c->mega_B[which] == c->st.B) n_slots = c->st.B;   // fixed shape: slots beyond the phase's rows are idle
   c->in_decode = true;
   int rc = RSD_OK;
   for (int j = 0; j < c->C && rc == RSD_OK; ++j) {
@@ -665,6 +726,7 @@ int rsd_load_models(rsd_ctx* c, const rsd_model* draft, const rsd_model* prm, co
   CU(cudaMemsetAsync(c->d_scalars, 0, 16 * sizeof(int32_t), s));
   CU(cudaMemsetAsync(c->gemm_scratch, 0, c->gemm_scratch_bytes, s));
   CU(cudaMemsetAsync(c->sample_best, 0, sizeof(unsigned long long) * c->B_max, s));
+  CU(cudaMemsetAsync(c->mega_sync, 0, sizeof(int32_t) * 1024, s));
   int rc = clear_forcing(c, s);
   if (rc) return rc;
   CU(cudaStreamSynchronize(s));
@@ -709,6 +771,7 @@ int rsd_prefill(rsd_ctx* c, const int32_t* tokens, const int32_t* offsets, int32
   CU(launched(1));
   CU(cudaStreamSynchronize(s));  // the staging buffers are reused below
   const bool merged = c->cfg.prm_shares_draft != 0;
+  if ((rc = ensure_mega(c, RSD_DRAFT, s)) || (rc = ensure_mega(c, RSD_TARGET, s))) return rc;
   CU(launch_reserve_pages(c->st, RSD_DRAFT, kReservePrefillDraft, 1, s));
   if (!merged) CU(launch_reserve_pages(c->st, RSD_PRM, kReservePrefillPrm, 1, s));
   Scalars sc;

@@ -110,6 +110,40 @@ cudaError_t launch_attn_decode(int kv_dtype, const float* q, const void* pool_la
                                void* out, void* out_lo, int out_dtype, int B, int H, int KV, int hd, int max_ctx, void* scratch,
                                size_t scratch_bytes, const int32_t* n_active, cudaStream_t s);
 
+// ---- persistent decode kernel: the whole layer stack of one decode iteration in one launch -------------
+struct MegaShape {
+  int n_layers, d, H, KV, hd, F;
+  bool bf16;
+  float eps;
+};
+// Everything the kernel needs for one model and one batch size; the arrays and buffers stay the caller's.
+struct MegaBuild {
+  MegaShape shape;
+  int B, max_pages;
+  const void* embed;
+  const void* const *wqkv, *const *wo, *const *wgu, *const *wdown, *const *norm1, *const *norm2;
+  char* kv_pool;
+  size_t layer_stride;
+  float* x;                                        // [B, d] residual stream
+  void *h, *h_lo, *attn, *attn_lo, *act, *act_lo;  // bf16 operand pairs [B, d], [B, H*hd], [B, F]
+  float* partials;                                 // K-split partial sums (mega_partials_floats)
+  float* ssq;                                      // [B, d / 128] sums of squares of the residual stream
+  float *part_o, *part_ml;                         // attention context-split partials [B, H, 16, hd] and [B, H, 16, 2]
+  int32_t* sync_words;                             // 1024 ints, zero: grid barrier and split arrival counters
+  int* err;                                        // raised to -5 when a bounded wait expires
+  const float2* rope;
+  const int32_t* page_table;
+};
+bool mega_supported(const MegaShape& m, int B);
+size_t mega_block_bytes(int n_layers);
+size_t mega_partials_floats(const MegaShape& m, int B);
+// Writes the kernel's parameter block (tensor maps, work plan, pointers) to dev_block (256-byte aligned).
+cudaError_t mega_build(void* dev_block, const MegaBuild& a, cudaStream_t s);
+// Runs embedding + all layers for the B slots of p (p.T == B).  On return x is the final residual stream,
+// h / h_lo hold x * final_gain and ssq the sums of squares per 128-column chunk.
+cudaError_t launch_decode_mega(const void* dev_block, int B, int kv_extended, PassView p, const void* final_gain,
+                               cudaStream_t s);
+
 struct SampleArgs {
   const float* logits;         // [n_slots, V]
   int n_slots, V, v_limit;

@@ -248,3 +248,44 @@ def test_merged_prm_on_the_drafts_trunk(shapes, bf16, tol):
     assert not st["kv_len"][1].any() and not st["n_pages"][1].any()
     compare_counters(eng, loop)
     print("merged PRM", "bf16" if bf16 else "fp32", stats)
+
+
+@pytest.mark.parametrize("B,ext", [(5, 0), (20, 0), (40, 0), (6, 1)])
+def test_persistent_decode_kernel_against_the_oracle_and_the_separate_kernels(B, ext):
+    """bf16 models at up to 64 rows decode with one persistent kernel per iteration (all layers, grid barriers
+    between the phases).  It must meet the oracle like the kernel-by-kernel path (RSD_DEBUG_NO_MEGA), agree with
+    that path far inside the bf16 bound, and launch far fewer kernels.  Batch sizes cover the 16-, 32- and 64-row
+    operand tiles; ext = hi + lo KV cache."""
+    from paper_2501_19324_b200 import lib, RSD_DEBUG_KEEP_LOGITS, RSD_DEBUG_NO_MEGA
+    from oracle.rsd_loop import DRAFT, TARGET
+    prompts = ri.prompts(50 + B, B, 5, 40, MINI[0].vocab)
+    kw = dict(max_step_tokens=5, max_steps=3, max_seq_tokens=80, step_end_id=3, step_end_mod=5, temperature=0.7, seed=8)
+    probe_eng, probe = build_pair(MINI, bf16=True, prompts=prompts, loop_kwargs=kw,
+                                  engine_kwargs=dict(debug_flags=RSD_DEBUG_KEEP_LOGITS | RSD_DEBUG_NO_MEGA))
+    delta = float(np.median(probe.step(0.0)["rewards"]))
+    probe_eng.close()
+    runs = {}
+    for name, flags in (("mega", RSD_DEBUG_KEEP_LOGITS), ("separate", RSD_DEBUG_KEEP_LOGITS | RSD_DEBUG_NO_MEGA)):
+        eng, loop = build_pair(MINI, bf16=True, prompts=prompts, loop_kwargs=kw,
+                               engine_kwargs=dict(debug_flags=flags, kv_extended=ext))
+        before = lib().rsd_debug_launch_count()
+        stats, logits, seen = {}, [], set()
+        for _ in range(3):
+            g, o = parity_step(eng, loop, delta, stats=stats, **TOL16)
+            seen |= set(int(a) for a, n in zip(o["accept"], o["step_len"]) if n)
+            logits.append((eng.logits(DRAFT).copy(), eng.logits(TARGET).copy(), o))
+        compare_counters(eng, loop)
+        runs[name] = dict(stats=stats, logits=logits, launches=lib().rsd_debug_launch_count() - before, seen=seen)
+        eng.close()
+    assert runs["mega"]["seen"] == {0, 1}                      # both models decoded
+    assert runs["mega"]["launches"] < 0.6 * runs["separate"]["launches"]
+    worst = 0.0
+    for (d0, t0, o), (d1, t1, _) in zip(runs["mega"]["logits"], runs["separate"]["logits"]):
+        for key, a, b in (("draft_trace", d0, d1), ("target_trace", t0, t1)):
+            for r in range(B):
+                if o[key][r] is not None:
+                    n = len(o[key][r]["logits"])
+                    worst = max(worst, float(np.abs(a[r, :n] - b[r, :n]).max()))
+    assert worst <= 2e-3, worst
+    print("persistent decode kernel", B, ext, runs["mega"]["stats"], "vs separate kernels", worst,
+          "launches", runs["mega"]["launches"], runs["separate"]["launches"])
