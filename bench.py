@@ -228,6 +228,35 @@ def combine_ranks(ms, e2e_ms, tokens, e2e_tokens, world, device):
     return float(t[0]), float(t[1]), float(n[0]), float(n[1])
 
 
+def debug_flags(args) -> int:
+    from paper_2501_19324_b200 import RSD_DEBUG_PERSISTENT_DECODE, RSD_DEBUG_MEGA_PROFILE
+    return (RSD_DEBUG_PERSISTENT_DECODE if (args.mega or args.mega_profile) else 0) | (RSD_DEBUG_MEGA_PROFILE if args.mega_profile else 0)
+
+
+def mega_phase_table(eng, which: int, n_layers: int) -> dict:
+    """Mean duration (us) of each phase of the persistent decode kernel's last launch, work and barrier wait
+    apart, as seen by its first CTA."""
+    st = eng.mega_profile(which).astype(np.int64)
+    names = ["qkv", "attention", "wo", "resid_norm_1", "gate_up_swiglu", "down", "resid_norm_2"]
+    out = {"total_us": float(st[-1] - st[0]) / 1e3, "embed_us": float(st[1] - st[0]) / 1e3}
+    work = {n: [] for n in names}
+    wait = {n: [] for n in names}
+    # stamps: [start, (work end, barrier end) of the embedding phase, then of every layer phase ..., kernel end]
+    i = 3
+    for l in range(n_layers):
+        for n in names:
+            if i >= len(st):
+                break
+            work[n].append(st[i] - st[i - 1])
+            if i + 1 < len(st) and not (l == n_layers - 1 and n == names[-1]):
+                wait[n].append(st[i + 1] - st[i])
+            i += 2
+    for n in names:
+        out[n] = {"work_us": float(np.mean(work[n])) / 1e3 if work[n] else None,
+                  "barrier_us": float(np.mean(wait[n])) / 1e3 if wait[n] else None}
+    return out
+
+
 def rank_prompts(rank, B, lo, hi, vocab):
     """Every replica works on its own prompts (seed 1 + rank)."""
     return ri.prompts(1 + rank, B, lo, hi, vocab)
@@ -263,7 +292,7 @@ def run_ours(args, rank: int, world: int):
     S = hi + n_steps * cap
     eng = Engine(*models, max_batch=B, max_seq_tokens=S, max_step_tokens=cap, max_steps=n_steps + 1,
                  step_end_id=13, temperature=0.7, seed=0, kv_extended=kv_extended(args),
-                 prm_shares_draft=int(merged))
+                 prm_shares_draft=int(merged), debug_flags=debug_flags(args))
     tokens, offsets = rank_prompts(rank, B, lo, hi, shapes[0].vocab)
     pinned_tokens = torch.from_numpy(tokens).pin_memory()
 
@@ -318,6 +347,14 @@ def run_ours(args, rank: int, world: int):
     e2e_ms = e2e_start.elapsed_time(e2e_end)
     ms, e2e_ms, timed_tokens, e2e_tokens = combine_ranks(ms, e2e_ms, timed_tokens, e2e_tokens, world, "cuda")
     counters = eng.counters()
+    mega_tables = None
+    if args.mega_profile and rank == 0:
+        mega_tables = {}
+        for name, which in (("draft", 0), ("target", 2)):
+            try:
+                mega_tables[name] = mega_phase_table(eng, which, shapes[which].n_layers)
+            except Exception as e:       # the model does not run the persistent kernel
+                mega_tables[name] = str(e)
 
     if rank == 0:
         hbm, tf, how = peaks()
@@ -346,6 +383,8 @@ def run_ours(args, rank: int, world: int):
                "phase_ms_per_step": phases,
                "flops_paper": counters["flops_paper"], "clocks": clocks,
                "gen_tokens": counters["gen_tokens"]}
+        if mega_tables is not None:
+            out["mega_profile"] = mega_tables
         if world == 1 and not args.no_cpu_baseline:
             level = 0 if (args.workload == "mini" or (args.workload == "cfg2" and mem_available_gb() > 60)) else 1
             smp = OracleSample(args.workload, level)
@@ -519,6 +558,10 @@ def main():
     ap.add_argument("--cap", type=int, default=0, help="override the step cap (profiling aid)")
     ap.add_argument("--merged-prm", action="store_true", dest="merged_prm",
                     help="prm_shares_draft: the PRM is a head on the draft's trunk (not the headline configuration)")
+    ap.add_argument("--mega", action="store_true",
+                    help="decode with the persistent decode kernel instead of kernel by kernel (not the headline path)")
+    ap.add_argument("--mega-profile", action="store_true", dest="mega_profile",
+                    help="record and print the phase timeline of the persistent decode kernel's last launches")
     ap.add_argument("--queue", type=int, default=1,
                     help="min_target_rows of rsd_step_queued (1 = rsd_step, the headline configuration)")
     ap.add_argument("--kv-extended", type=int, default=None, choices=[0, 1], dest="kv_extended",

@@ -114,8 +114,12 @@ typedef struct {
 enum {
   RSD_DEBUG_KEEP_LOGITS = 1, /* keep every decode iteration's logits for rsd_debug_get_logits      */
   RSD_DEBUG_NO_GRAPHS = 2,   /* launch decode iterations kernel by kernel instead of as CUDA graphs */
-  RSD_DEBUG_NO_MEGA = 4      /* run the layers of a decode iteration as separate kernels instead of the one
-                                persistent kernel (bf16 models, up to 64 rows)                        */
+  RSD_DEBUG_PERSISTENT_DECODE = 4, /* alternative decode path for bf16 models at up to 64 rows: the layers of a
+                                decode iteration run as ONE persistent kernel (one CTA per SM, grid barriers
+                                between the phases) instead of kernel by kernel.  Same results; slower than
+                                the default on the measured shapes, kept for study                    */
+  RSD_DEBUG_MEGA_PROFILE = 8 /* the persistent decode kernel records global-timer stamps around its grid
+                                barriers (rsd_debug_mega_profile)                                     */
 };
 
 /* Fills cfg->kv_bytes[] (enough pages for max_batch rows of max_seq_tokens) and
@@ -213,6 +217,13 @@ int rsd_debug_gemm_timing(rsd_ctx*, int32_t stride, double* ms, double* bytes, u
 int rsd_debug_phase_ms(rsd_ctx*, int32_t enable, double* out);
 /* Number of kernels this library has enqueued in this process so far.                          */
 uint64_t rsd_debug_launch_count(void);
+/* Timeline of the last launch of the persistent decode kernel of model `which` (RSD_DRAFT or RSD_TARGET),
+ * recorded by its first CTA when RSD_DEBUG_MEGA_PROFILE is set: stamps[0] = kernel start, then for every
+ * grid barrier the global-timer value (ns) when the CTA's phase work was done and when the barrier let it
+ * go, in phase order (embedding; per layer: qkv, attention, wo, residual + norm, gate/up + SwiGLU, down,
+ * residual + norm), last the kernel's end.  stamps (HOST, `capacity` words) receives *n_out values.
+ * Synchronises the device.  RSD_ERR_STATE when the flag was not set.                            */
+int rsd_debug_mega_profile(rsd_ctx*, int which, uint64_t* stamps, int32_t capacity, int32_t* n_out);
 
 /* ---- single kernels (sweeps and unit parity); all pointers DEVICE unless noted ------------ */
 

@@ -17,7 +17,8 @@ RSD_DRAFT, RSD_PRM, RSD_TARGET = 0, 1, 2
 RSD_HEAD_LM, RSD_HEAD_REWARD_SIGMOID, RSD_HEAD_REWARD_RAW = 0, 1, 2
 RSD_DEBUG_KEEP_LOGITS = 1
 RSD_DEBUG_NO_GRAPHS = 2
-RSD_DEBUG_NO_MEGA = 4
+RSD_DEBUG_PERSISTENT_DECODE = 4
+RSD_DEBUG_MEGA_PROFILE = 8
 ERRORS = {0: "RSD_OK", -1: "RSD_ERR_ARG", -2: "RSD_ERR_STATE", -3: "RSD_ERR_OOM_PAGES", -4: "RSD_ERR_CUDA",
           -5: "RSD_ERR_TIMEOUT", -6: "RSD_ERR_UNSUPPORTED"}
 
@@ -53,7 +54,7 @@ class rsd_counters(ctypes.Structure):
 
 EXPORTS = ["rsd_query_sizes", "rsd_create", "rsd_load_models", "rsd_prefill", "rsd_step", "rsd_step_queued", "rsd_flops_counters",
            "rsd_reset", "rsd_destroy", "rsd_last_error", "rsd_debug_force", "rsd_debug_get_logits",
-           "rsd_debug_get_sampled", "rsd_debug_get_state", "rsd_debug_gemm_timing", "rsd_debug_launch_count", "rsd_debug_phase_ms", "rsd_k_gemm", "rsd_k_gemm_scratch_bytes",
+           "rsd_debug_get_sampled", "rsd_debug_get_state", "rsd_debug_gemm_timing", "rsd_debug_launch_count", "rsd_debug_mega_profile", "rsd_debug_phase_ms", "rsd_k_gemm", "rsd_k_gemm_scratch_bytes",
            "rsd_k_attn_decode", "rsd_k_attn_decode_scratch_bytes", "rsd_k_attn_chunk", "rsd_k_gate_compact", "rsd_k_gate_compact_static", "rsd_k_gate_compact_static_error", "rsd_k_rmsnorm",
            "rsd_k_rope", "rsd_k_swiglu", "rsd_k_sample", "rsd_k_philox"]
 
@@ -86,6 +87,7 @@ def lib():
         L.rsd_debug_gemm_timing.argtypes = [vp, c_int32, vp, vp, vp]
         L.rsd_debug_phase_ms.argtypes = [vp, c_int32, vp]
         L.rsd_debug_launch_count.argtypes = []
+        L.rsd_debug_mega_profile.argtypes = [vp, c_int32, vp, c_int32, vp]
         L.rsd_debug_launch_count.restype = c_uint64
         L.rsd_k_gemm.argtypes = [vp, vp, vp, vp, c_int32, c_int32, c_int32, c_int32, c_int32, c_int32, vp, c_size_t, vp]
         L.rsd_k_gemm_scratch_bytes.argtypes = [c_int32, c_int32, c_int32]
@@ -242,6 +244,13 @@ class Engine:
         return dict(zip(self.PHASES, list(out)))
 
     # -- parity hooks ---------------------------------------------------------------------------
+    def mega_profile(self, which: int) -> np.ndarray:
+        """Global-timer stamps (ns) of the last persistent-decode launch of model `which` (RSD_DEBUG_MEGA_PROFILE)."""
+        out = np.zeros(1024, dtype=np.uint64)
+        n = ctypes.c_int32(0)
+        _check(lib().rsd_debug_mega_profile(self.ctx, which, out.ctypes.data, 1024, ctypes.byref(n)), self.ctx)
+        return out[:n.value]
+
     def force_tokens(self, which: int, steps: list):
         """steps[b]: list of token ids forced on row b in the next step (empty = free-running)."""
         tok = np.zeros((self.B, self.C), np.int32)

@@ -69,6 +69,7 @@ struct rsd_ctx {
   void* mega_block[3] = {nullptr, nullptr, nullptr};
   int mega_B[3] = {0, 0, 0};
   int32_t* mega_sync = nullptr;
+  unsigned long long* mega_prof[3] = {nullptr, nullptr, nullptr};   // RSD_DEBUG_MEGA_PROFILE
   char* pinned = nullptr;
   size_t pinned_bytes = 0;
   void* gemm_scratch = nullptr;
@@ -221,6 +222,9 @@ size_t layout_workspace(const rsd_config& cfg, const rsd_model* const ms[3], rsd
   void* mega_block[3] = {nullptr, nullptr, nullptr};
   for (int w = 0; w < 3; w += 2) mega_block[w] = TAKE(char, mega_block_bytes(ms[w]->n_layers));
   int32_t* mega_sync = TAKE(int32_t, 1024);
+  unsigned long long* mega_prof[3] = {nullptr, nullptr, nullptr};
+  if (cfg.debug_flags & RSD_DEBUG_MEGA_PROFILE)
+    for (int w = 0; w < 3; w += 2) mega_prof[w] = TAKE(unsigned long long, 1024);
   float2* rope[3];
   for (int w = 0; w < 3; ++w) rope[w] = TAKE(float2, (size_t)S * (ms[w]->head_dim / 2));
   float* dbg[2] = {nullptr, nullptr};
@@ -253,6 +257,7 @@ size_t layout_workspace(const rsd_config& cfg, const rsd_model* const ms[3], rsd
     c->norm_ssq = norm_ssq;
     for (int w = 0; w < 3; ++w) { c->mega_block[w] = mega_block[w]; c->mega_B[w] = 0; }
     c->mega_sync = mega_sync;
+    for (int w = 0; w < 3; ++w) c->mega_prof[w] = mega_prof[w];
     for (int w = 0; w < 3; ++w) c->mdl[w].rope = rope[w];
     c->dbg_logits[0] = dbg[0]; c->dbg_logits[1] = dbg[1];
     c->d_scalars = scal;
@@ -452,10 +457,10 @@ MegaShape mega_shape(const ModelHost& M) {
   return MegaShape{m.n_layers, m.d_model, m.n_heads, m.n_kv_heads, m.head_dim, m.d_ffn, m.dtype == RSD_BF16 && M.split, m.rms_eps};
 }
 
-// The persistent decode kernel serves bf16 models with 16-bit caches at up to 64 rows.
+// The persistent decode kernel (opt-in) serves bf16 models with 16-bit caches at up to 64 rows.
 bool mega_wanted(const rsd_ctx* c, int which) {
   const ModelHost& M = c->mdl[which];
-  if (c->cfg.debug_flags & RSD_DEBUG_NO_MEGA) return false;
+  if (!(c->cfg.debug_flags & RSD_DEBUG_PERSISTENT_DECODE)) return false;
   if (which == RSD_PRM || !fused_decode_ok(M) || (M.kv_dtype != 2 && M.kv_dtype != 3)) return false;
   if (!mega_supported(mega_shape(M), c->st.B)) return false;
   const MegaShape sh = mega_shape(M);
@@ -487,6 +492,7 @@ int ensure_mega(rsd_ctx* c, int which, cudaStream_t s) {
   a.err = (int*)((char*)c->gemm_scratch + 4096);
   a.rope = M.rope;
   a.page_table = c->st.page_table[which];
+  a.prof = c->mega_prof[which];
   cudaError_t e = mega_build(c->mega_block[which], a, s);
   if (e == cudaErrorNotSupported) { c->mega_B[which] = 0; return RSD_OK; }
   CU(e);
@@ -1036,6 +1042,18 @@ int rsd_debug_gemm_timing(rsd_ctx* c, int32_t stride, double* ms, double* bytes,
 }
 
 uint64_t rsd_debug_launch_count(void) { return launches_total(); }
+
+int rsd_debug_mega_profile(rsd_ctx* c, int which, uint64_t* stamps, int32_t capacity, int32_t* n_out) {
+  if (!c || !stamps || !n_out || capacity < 1 || which < 0 || which > 2) return RSD_ERR_ARG;
+  if (!c->mega_prof[which]) return fail(c, RSD_ERR_STATE, "RSD_DEBUG_MEGA_PROFILE was not set%s");
+  CU(cudaDeviceSynchronize());
+  unsigned long long n = 0;
+  CU(cudaMemcpy(&n, c->mega_prof[which] + 1023, sizeof(n), cudaMemcpyDeviceToHost));
+  const int take = (int)std::min<unsigned long long>(std::min<unsigned long long>(n, 1022), (unsigned long long)capacity);
+  CU(cudaMemcpy(stamps, c->mega_prof[which], sizeof(uint64_t) * take, cudaMemcpyDeviceToHost));
+  *n_out = take;
+  return RSD_OK;
+}
 
 int rsd_debug_phase_ms(rsd_ctx* c, int32_t enable, double* out) {
   if (!c) return RSD_ERR_ARG;

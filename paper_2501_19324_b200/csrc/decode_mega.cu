@@ -46,7 +46,8 @@ constexpr int kPhaseThreads = 320;    // everyone but the W producer meets at th
 constexpr int kWStageBytes = 128 * 64 * 2;
 constexpr int kGenScratchBytes = 8 * 8 * 128 * 4 + 2 * 8 * 8 * 4 + 8 * 128 * 4;   // attention: outputs, (max, sum), q
 constexpr uint32_t kGridSpinLimit = 1u << 22;
-constexpr int kMaxAttnSplits = 16;
+constexpr int kMaxStamps = 1022;
+constexpr int kXchBytes = 64 * 65 * 4;
 
 struct GemmPlan {
   int N, K, n_tiles, splits, kbps, total_kb;
@@ -75,6 +76,7 @@ struct alignas(128) MegaParams {
   int* err;
   const float2* rope;
   const int32_t* page_table;
+  unsigned long long* prof;            // debug: CTA 0 stamps the global timer before and after every grid barrier
 };
 
 // ---- small helpers ------------------------------------------------------------------------------
@@ -87,23 +89,34 @@ __device__ __forceinline__ unsigned ld_acquire(const unsigned* p) {
   return v;
 }
 __device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async;" ::: "memory"); }
+__device__ __forceinline__ unsigned long long global_timer() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
 
 struct Shared {
   uint8_t* wring;
   uint8_t* xring;
-  float* gen;            // general scratch (attention) / gate-up exchange
+  float* gen;            // attention scratch; aliases the X ring, which is idle outside the GEMM phases
+  float* xch;            // gate/up exchange of the SwiGLU epilogue [64][65]
   float* row_scale;      // [64]
   uint64_t *full_w, *empty_w, *full_x, *empty_x, *acc_full, *acc_empty;
   uint32_t* tmem_slot;
   volatile int* abort_flag;
   volatile int* go;
   volatile int* flag;
+  int* pref;             // [B + 1] prefix sums of the rows' page counts, [B + 1] = the largest count
 };
 
-// Bounded wait that also gives up when another role has stopped the CTA.
+// Bounded wait that also gives up when another role has stopped the CTA.  Waiters sleep in hardware between
+// polls (about 2 us at most, so ~2 s in all before the wait is given up).
+constexpr uint32_t kSleepNs = 2000;
+constexpr uint32_t kSleepPolls = 1u << 20;
 __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, const Shared& sh, int* err) {
-  for (uint32_t i = 0; i < kWaitLimit; ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
+  if (mbar_try_wait(bar, parity)) return true;
+  for (uint32_t i = 0; i < kSleepPolls; ++i) {
+    if (mbar_try_wait_sleep(bar, parity, kSleepNs)) return true;
     if (*sh.abort_flag) return false;
   }
   *sh.abort_flag = 1;
@@ -111,34 +124,42 @@ __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, const S
   return false;
 }
 
-// Grid-wide barrier for everyone but the W producer: self-resetting arrival counter plus a generation word.
-__device__ __forceinline__ void grid_sync(const MegaParams& P, const Shared& sh) {
-  __threadfence();
+// Grid-wide barrier for everyone but the W producer.  grid_bar[0] counts arrivals and only grows during a
+// launch: barrier number k is passed once it reads k * gridDim.x.  Thread 0 arrives with a one-way release
+// reduction and polls with acquire loads; the CTA barriers on both sides extend the ordering to the other
+// threads.  The last CTA to leave the kernel puts the counter back to zero (finish_grid_sync).
+__device__ __forceinline__ void grid_sync(const MegaParams& P, const Shared& sh, unsigned& epoch, int& n_stamps) {
+  if (P.prof != nullptr && blockIdx.x == 0 && threadIdx.x == 0 && n_stamps < kMaxStamps) P.prof[n_stamps++] = global_timer();
   fence_async_proxy();          // activations written with plain stores are read by TMA after the barrier
   bar_sync(1, kPhaseThreads);
   if (threadIdx.x == 0) {
     if (!*sh.abort_flag) {
-      __threadfence();
-      const unsigned gen = ld_acquire(P.grid_bar + 1);
-      const unsigned old = atomicAdd(P.grid_bar, 1u);
-      if (old == gridDim.x - 1) {
-        P.grid_bar[0] = 0u;
-        __threadfence();
-        atomicAdd(P.grid_bar + 1, 1u);
-      } else {
-        bool ok = false;
-        for (uint32_t i = 0; i < kGridSpinLimit; ++i) {
-          if (ld_acquire(P.grid_bar + 1) != gen) { ok = true; break; }
-          if ((i & 255u) == 255u && __ldcg(P.err) != 0) break;
-        }
-        if (!ok) { *sh.abort_flag = 1; atomicCAS(P.err, 0, -5); }
+      ++epoch;
+      const unsigned target = epoch * gridDim.x;
+      asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(P.grid_bar) : "memory");
+      bool ok = false;
+      for (uint32_t i = 0; i < kGridSpinLimit; ++i) {
+        if (ld_acquire(P.grid_bar) >= target) { ok = true; break; }
+        if ((i & 255u) == 255u && __ldcg(P.err) != 0) break;
       }
-      __threadfence();
+      if (!ok) { *sh.abort_flag = 1; atomicCAS(P.err, 0, -5); }
     }
     *sh.go = *sh.abort_flag ? 0 : 1;
   }
   bar_sync(1, kPhaseThreads);
   fence_async_proxy();
+  if (P.prof != nullptr && blockIdx.x == 0 && threadIdx.x == 0 && n_stamps < kMaxStamps) P.prof[n_stamps++] = global_timer();
+}
+
+// Called by thread 0 of every CTA after its last barrier: the last one to come resets both counters.
+__device__ __forceinline__ void finish_grid_sync(const MegaParams& P) {
+  __threadfence();
+  const unsigned old = atomicAdd(P.grid_bar + 1, 1u);
+  if (old == gridDim.x - 1) {
+    P.grid_bar[0] = 0u;
+    P.grid_bar[1] = 0u;
+    __threadfence();
+  }
 }
 
 struct Item { int tile, split, kb0, kb1; };
@@ -226,29 +247,37 @@ __device__ __forceinline__ void mma_f16(float& d0, float& d1, float& d2, float& 
 __device__ __forceinline__ uint4 ldcg_u4(const __half* p) { return __ldcg(reinterpret_cast<const uint4*>(p)); }
 __device__ __forceinline__ uint2 ldcg_u2(const __half* p) { return __ldcg(reinterpret_cast<const uint2*>(p)); }
 
-// Sum over the K-split partial sums of the qkv product, element (slot, col).
-__device__ __forceinline__ float qkv_sum(const MegaParams& P, int slot, int col) {
+// Sums over the K-split partial sums of the qkv product for two columns of one slot.  All loads of a group of
+// eight splits (sixteen loads) are in flight together; the sums stay in split order.
+__device__ __forceinline__ void qkv_sum2(const MegaParams& P, int slot, int col_a, int col_b, float& a, float& b) {
   const GemmPlan& g = P.plan[0];
   const size_t stride = (size_t)P.B * g.N;
-  const float* p = P.partials + (size_t)slot * g.N + col;
-  float v = 0.f;
-  int s = 0;
-  for (; s + 4 <= g.splits; s += 4) {
-    float t[4];
+  const float* pa = P.partials + (size_t)slot * g.N + col_a;
+  const float* pb = P.partials + (size_t)slot * g.N + col_b;
+  const int splits = g.splits;
+  a = 0.f; b = 0.f;
+  for (int s0 = 0; s0 < splits; s0 += 8) {
+    float ta[8], tb[8];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) t[u] = __ldcg(p + (size_t)(s + u) * stride);
+    for (int u = 0; u < 8; ++u) {
+      const bool in = s0 + u < splits;
+      ta[u] = in ? __ldcg(pa + (size_t)(s0 + u) * stride) : 0.f;
+      tb[u] = in ? __ldcg(pb + (size_t)(s0 + u) * stride) : 0.f;
+    }
 #pragma unroll
-    for (int u = 0; u < 4; ++u) v += t[u];
+    for (int u = 0; u < 8; ++u) { a += ta[u]; b += tb[u]; }
   }
-  for (; s < g.splits; ++s) v += __ldcg(p + (size_t)s * stride);
-  return v;
 }
 
-// Work item = (row slot, KV head, context split), served by the eight general warps of the CTA: the rotated
-// queries of the head group are rebuilt from the qkv partial sums, the split that owns the newest page
-// also rotates the new key and writes it and the new value into the page, then every warp walks its share
-// of the 16-token pages with m16n8k16 MMAs (queries of the group as rows).  The last split of a (slot, head)
-// pair to finish merges all of them.
+// The (row slot, KV head, page) triples of the iteration are laid end to end (slot-major, then head, then
+// page) and cut into equal chunks, one per CTA, so every CTA walks the same number of pages whatever the
+// rows' context lengths.  A chunk is a few segments, each a page range of one (slot, head) pair, served by
+// the eight general warps: the rotated queries of the head group are rebuilt from the qkv partial sums, the
+// segment that holds the pair's newest page also rotates the new key and writes it and the new value into
+// that page, then every warp walks its share of the 16-token pages with m16n8k16 MMAs (queries of the group
+// as rows).  A pair cut into several segments is merged by the last of them to finish.
+constexpr int kMaxParts = 32;
+
 template <bool EXT>
 __device__ __forceinline__ void attn_phase(const MegaParams& P, const MegaLayer& Ly, const PassView& pv, const Shared& sh) {
   constexpr int HD = 128, KB = HD / 32, NT = HD / 8;
@@ -256,7 +285,7 @@ __device__ __forceinline__ void attn_phase(const MegaParams& P, const MegaLayer&
   if (tid >= kGenThreads) return;
   const int warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, t = lane & 3;
-  const int H = P.H, KV = P.KV, G = H / KV, S = P.attn_splits;
+  const int H = P.H, KV = P.KV, G = H / KV;
   float* s_o = sh.gen;                       // [8 warps][8 heads][HD]
   float* s_m = s_o + 8 * 8 * HD;             // [8][8]
   float* s_l = s_m + 64;                     // [8][8]
@@ -266,35 +295,55 @@ __device__ __forceinline__ void attn_phase(const MegaParams& P, const MegaLayer&
   const size_t block_elems = (size_t)KV * kPageTokens * HD;
   const size_t page_elems = (EXT ? 4 : 2) * block_elems;
   const float scale = rsqrtf((float)HD);
-  const int n_items = P.B * KV * S;
-  for (int it = blockIdx.x; it < n_items; it += gridDim.x) {
-    const int split = it % S, pair = it / S, kvh = pair % KV, slot = pair / KV;
+  const int U = sh.pref[P.B] * KV;
+  // pages per CTA: an even share, at least one page per warp, and no pair in more than kMaxParts pieces
+  const int chunk = max(max((U + (int)gridDim.x - 1) / (int)gridDim.x, 8), (sh.pref[P.B + 1] + kMaxParts - 3) / (kMaxParts - 2));
+  const int u_end = min(U, ((int)blockIdx.x + 1) * chunk);
+  int slot = 0;
+  for (int u = (int)blockIdx.x * chunk; u < u_end;) {
+    while (sh.pref[slot + 1] * KV <= u) ++slot;
+    const int n_pages = sh.pref[slot + 1] - sh.pref[slot];
+    const int rel = u - sh.pref[slot] * KV;
+    const int kvh = rel / n_pages, p_begin = rel - kvh * n_pages;
+    const int p_end = min(n_pages, p_begin + (u_end - u));
+    const int pair_u0 = sh.pref[slot] * KV + kvh * n_pages;
+    const int first_cta = pair_u0 / chunk;
+    const int S = (pair_u0 + n_pages - 1) / chunk - first_cta + 1;      // pieces of this pair
+    const int split = (int)blockIdx.x - first_cta;
+    const int pair = slot * KV + kvh;
+    u += p_end - p_begin;
     const int row = pv.tok_row[slot];
-    if (row < 0) continue;
     const int pos = pv.tok_pos[slot], ctx = pos + 1;
     const int h0 = kvh * G;
-    const int n_pages = (ctx + kPageTokens - 1) / kPageTokens;
-    const int pps = (n_pages + S - 1) / S;
-    const int p_begin = split * pps, p_end = min(n_pages, p_begin + pps);
-    const int last_split = (n_pages - 1) / pps;
     const int32_t* pt = P.page_table + (size_t)row * P.max_pages;
     const float2* cs = P.rope + (size_t)pos * (HD / 2);
+    // page indices of this warp's visits are requested first, so that they arrive under the rebuild below
+    int pg[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int pp = p_begin + warp + 8 * i;
+      pg[i] = pp < p_end ? __ldg(pt + pp) : 0;
+    }
     // rotated queries of the group
     for (int idx = tid; idx < G * (HD / 2); idx += kGenThreads) {
       const int gg = idx >> 6, i = idx & 63;
-      const float a = qkv_sum(P, slot, (h0 + gg) * HD + i), b = qkv_sum(P, slot, (h0 + gg) * HD + i + HD / 2);
+      float a, b;
+      qkv_sum2(P, slot, (h0 + gg) * HD + i, (h0 + gg) * HD + i + HD / 2, a, b);
       const float2 c = cs[i];
       sq[gg * HD + i] = a * c.x - b * c.y;
       sq[gg * HD + i + HD / 2] = b * c.x + a * c.y;
     }
-    if (split == last_split) {
-      // the new token's key (rotated) and value go into their page before the page is read
+    if (p_end == n_pages) {
+      // the new token's key (rotated) and value go into their page before the page is read; the three upper
+      // warps do it, which have the fewest queries to rebuild
       const int page = pt[pos / kPageTokens], tslot = pos % kPageTokens;
       __half* kbase = pool_w + (size_t)page * page_elems;
       __half* vbase = kbase + block_elems;
-      if (tid < HD / 2) {
-        const int i = tid;
-        const float a = qkv_sum(P, slot, (H + kvh) * HD + i), b = qkv_sum(P, slot, (H + kvh) * HD + i + HD / 2);
+      const int r = kGenThreads - 1 - tid;        // 0..255 from the top thread down
+      if (r < HD / 2) {
+        const int i = r;
+        float a, b;
+        qkv_sum2(P, slot, (H + kvh) * HD + i, (H + kvh) * HD + i + HD / 2, a, b);
         const float2 c = cs[i];
         const float ra = a * c.x - b * c.y, rb = b * c.x + a * c.y;
         __half* k = kbase + ((size_t)kvh * kPageTokens + tslot) * HD;
@@ -305,12 +354,17 @@ __device__ __forceinline__ void attn_phase(const MegaParams& P, const MegaLayer&
           k[2 * block_elems + i] = __float2half_rn(ra - __half2float(ka));
           k[2 * block_elems + i + HD / 2] = __float2half_rn(rb - __half2float(kb2));
         }
-      } else if (tid < HD / 2 + HD) {
-        const int i = tid - HD / 2;
-        const float v = qkv_sum(P, slot, (H + KV + kvh) * HD + i);
-        const __half vh = __float2half_rn(v);
-        vbase[((size_t)kvh * HD + i) * kPageTokens + tslot] = vh;
-        if (EXT) vbase[2 * block_elems + ((size_t)kvh * HD + i) * kPageTokens + tslot] = __float2half_rn(v - __half2float(vh));
+      } else if (r < HD) {
+        const int i = r - HD / 2;                 // value dims i and i + 64
+        float v0, v1;
+        qkv_sum2(P, slot, (H + KV + kvh) * HD + i, (H + KV + kvh) * HD + i + HD / 2, v0, v1);
+        const __half h0v = __float2half_rn(v0), h1v = __float2half_rn(v1);
+        vbase[((size_t)kvh * HD + i) * kPageTokens + tslot] = h0v;
+        vbase[((size_t)kvh * HD + i + HD / 2) * kPageTokens + tslot] = h1v;
+        if (EXT) {
+          vbase[2 * block_elems + ((size_t)kvh * HD + i) * kPageTokens + tslot] = __float2half_rn(v0 - __half2float(h0v));
+          vbase[2 * block_elems + ((size_t)kvh * HD + i + HD / 2) * kPageTokens + tslot] = __float2half_rn(v1 - __half2float(h1v));
+        }
       }
     }
     bar_sync(3, kGenThreads);
@@ -335,11 +389,13 @@ __device__ __forceinline__ void attn_phase(const MegaParams& P, const MegaLayer&
     float dump0 = 0.f, dump1 = 0.f;
     float m_run = -INFINITY, l_run = 0.f;
     const int tok0 = 4 * (g >> 1) + (g & 1), tok1 = tok0 + 2;
-    int page = (p_begin + warp < p_end) ? pt[p_begin + warp] : 0;
-    for (int p = p_begin + warp; p < p_end; p += 8) {
+    int visit = 0;
+    int page_next = 0;
+    for (int p = p_begin + warp; p < p_end; p += 8, ++visit) {
+      const int page = visit == 0 ? pg[0] : (visit == 1 ? pg[1] : (visit == 2 ? pg[2] : (visit == 3 ? pg[3] : page_next)));
       const __half* kb = pool + (size_t)page * page_elems + (size_t)kvh * kPageTokens * HD;
       const __half* vb = pool + (size_t)page * page_elems + block_elems + (size_t)kvh * HD * kPageTokens;
-      if (p + 8 < p_end) page = pt[p + 8];
+      if (visit >= 3 && p + 8 < p_end) page_next = pt[p + 8];
       uint4 k0[KB], k1[KB];
       uint2 vv[NT], vl[EXT ? NT : 1];
 #pragma unroll
@@ -433,7 +489,7 @@ __device__ __forceinline__ void attn_phase(const MegaParams& P, const MegaLayer&
       if (S == 1) {
         store_operand<__nv_bfloat16>(P.attn_hi, P.attn_lo, ((size_t)slot * H + h) * HD + dd, O / L);
       } else {
-        const size_t base = ((size_t)slot * H + h) * S + split;
+        const size_t base = ((size_t)slot * H + h) * kMaxParts + split;
         P.part_o[base * HD + dd] = O;
         if (dd == 0) { P.part_ml[base * 2] = M; P.part_ml[base * 2 + 1] = L; }
       }
@@ -451,33 +507,50 @@ __device__ __forceinline__ void attn_phase(const MegaParams& P, const MegaLayer&
         __threadfence();
         for (int idx = tid; idx < G * HD; idx += kGenThreads) {
           const int gg = idx / HD, dd = idx % HD, h = h0 + gg;
-          const size_t base = ((size_t)slot * H + h) * S;
-          float M = -INFINITY;
-          for (int s = 0; s < S; ++s) M = fmaxf(M, __ldcg(P.part_ml + (base + s) * 2));
-          float L = 0.f, O = 0.f;
-          for (int s = 0; s < S; ++s) {
-            const float m = __ldcg(P.part_ml + (base + s) * 2);
-            if (m > -INFINITY) {
-              const float e = __expf(m - M);
-              L += __ldcg(P.part_ml + (base + s) * 2 + 1) * e;
-              O += __ldcg(P.part_o + (base + s) * HD + dd) * e;
+          const size_t base = ((size_t)slot * H + h) * kMaxParts;
+          float M = -INFINITY, L = 0.f, O = 0.f;
+          for (int s0 = 0; s0 < S; s0 += 4) {
+            float2 ml[4];
+            float ov[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              const bool in = s0 + u < S;
+              ml[u] = in ? __ldcg(reinterpret_cast<const float2*>(P.part_ml + (base + s0 + u) * 2)) : make_float2(-INFINITY, 0.f);
+              ov[u] = in ? __ldcg(P.part_o + (base + s0 + u) * HD + dd) : 0.f;
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              if (ml[u].x > -INFINITY) {
+                const float Mn = fmaxf(M, ml[u].x);
+                const float e_old = __expf(M - Mn), e_new = __expf(ml[u].x - Mn);
+                L = L * e_old + ml[u].y * e_new;
+                O = O * e_old + ov[u] * e_new;
+                M = Mn;
+              }
             }
           }
           store_operand<__nv_bfloat16>(P.attn_hi, P.attn_lo, ((size_t)slot * H + h) * HD + dd, O / L);
         }
       }
     }
-    bar_sync(3, kGenThreads);   // the scratch is free for the next item
+    bar_sync(3, kGenThreads);   // the scratch is free for the next segment
   }
 }
 
 // ---- GEMM phase ----------------------------------------------------------------------------------------
+// Ring positions as (stage, parity) pairs that are stepped, never divided: the loops below run in one thread
+// each, where every dependent instruction costs its full latency.
+struct RingPos {
+  uint32_t stage = 0, parity = 0;
+  __device__ __forceinline__ void step(uint32_t n) {
+    if (++stage == n) { stage = 0; parity ^= 1u; }
+  }
+};
 struct PipeState {
-  uint32_t xi = 0;   // X stages issued          (X producer)
-  uint32_t wc = 0;   // W stages consumed        (MMA issuer)
-  uint32_t xc = 0;   // X stages consumed        (MMA issuer)
-  uint32_t ac = 0;   // accumulators produced    (MMA issuer)
-  uint32_t ae = 0;   // accumulators read        (epilogue warps)
+  RingPos xi;        // next X stage to fill         (X producer)
+  RingPos wc, xc;    // next W / X stage to consume  (MMA issuer)
+  uint32_t ac = 0;   // accumulators produced        (MMA issuer)
+  uint32_t ae = 0;   // accumulators read            (epilogue warps)
 };
 
 // which: 0 qkv, 1 wo, 2 gate/up (+ SwiGLU), 3 down.
@@ -487,7 +560,8 @@ __device__ __forceinline__ void gemm_phase(const MegaParams& P, int which, const
   const GemmPlan& g = P.plan[which];
   const int n_items = g.n_tiles * g.splits;
   const int rows = P.rows, mt = P.mt;
-  const uint32_t xstage = (uint32_t)mt * 128u;
+  const uint32_t xstage = (uint32_t)mt * 128u, n_sw = (uint32_t)P.sw, n_sx = (uint32_t)P.sx;
+  int* const err = P.err;
   if (warp == kWarpX) {
     if (lane == 0 && !*sh.abort_flag) {
       const int src = which == 1 ? 1 : (which == 3 ? 2 : 0);
@@ -497,14 +571,14 @@ __device__ __forceinline__ void gemm_phase(const MegaParams& P, int which, const
         const Item im = item_of(g, it);
         bool ok = true;
         for (int kb = im.kb0; kb < im.kb1 && ok; ++kb) {
-          const uint32_t s = ps.xi % (uint32_t)P.sx;
-          ok = wait_bar(&sh.empty_x[s], ((ps.xi / (uint32_t)P.sx) & 1u) ^ 1u, sh, P.err);
+          const uint32_t s = ps.xi.stage;
+          ok = wait_bar(&sh.empty_x[s], ps.xi.parity ^ 1u, sh, err);
           if (!ok) break;
           uint8_t* dst = sh.xring + (size_t)s * xstage;
           mbar_expect_tx(&sh.full_x[s], xstage);
           tma_load_2d(dst, mhi, &sh.full_x[s], kb * 64, 0);
           tma_load_2d(dst + (size_t)rows * 128, mlo, &sh.full_x[s], kb * 64, 0);
-          ++ps.xi;
+          ps.xi.step(n_sx);
         }
         if (!ok) break;
       }
@@ -515,27 +589,37 @@ __device__ __forceinline__ void gemm_phase(const MegaParams& P, int which, const
   if (warp == kWarpMma) {
     if (lane == 0 && !*sh.abort_flag) {
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(mt >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+      // shared-memory descriptors (K-major, 128-byte swizzle): the high word is constant, the low word is the
+      // tile address in 16-byte units (plus 2 per 16-element k slice) with the unused leading offset set to 1
+      const uint32_t desc_hi = (uint32_t)(1024 >> 4) | (1u << 14) | (2u << 29);
+      const uint32_t a_lo0 = ((smem_u32(sh.wring) >> 4) & 0x3FFFu) | (1u << 16);
+      const uint32_t b_lo0 = ((smem_u32(sh.xring) >> 4) & 0x3FFFu) | (1u << 16);
+      const uint32_t b_step = xstage >> 4;
       for (int it = blockIdx.x; it < n_items; it += gridDim.x) {
         const Item im = item_of(g, it);
         const uint32_t b = ps.ac & 1u;
-        bool ok = wait_bar(&sh.acc_empty[b], ((ps.ac >> 1) & 1u) ^ 1u, sh, P.err);
+        bool ok = wait_bar(&sh.acc_empty[b], ((ps.ac >> 1) & 1u) ^ 1u, sh, err);
         if (!ok) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + b * (uint32_t)mt;
+        uint32_t acc = 0u;
         for (int kb = im.kb0; kb < im.kb1; ++kb) {
-          const uint32_t ws = ps.wc % (uint32_t)P.sw, xs = ps.xc % (uint32_t)P.sx;
-          ok = wait_bar(&sh.full_w[ws], (ps.wc / (uint32_t)P.sw) & 1u, sh, P.err) &&
-               wait_bar(&sh.full_x[xs], (ps.xc / (uint32_t)P.sx) & 1u, sh, P.err);
+          const uint32_t ws = ps.wc.stage, xs = ps.xc.stage;
+          ok = wait_bar(&sh.full_w[ws], ps.wc.parity, sh, err) && wait_bar(&sh.full_x[xs], ps.xc.parity, sh, err);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t a = smem_u32(sh.wring + (size_t)ws * kWStageBytes);
-          const uint32_t bb = smem_u32(sh.xring + (size_t)xs * xstage);
+          const uint32_t a_lo = a_lo0 + ws * (kWStageBytes >> 4), b_lo = b_lo0 + xs * b_step;
 #pragma unroll
-          for (int k = 0; k < 4; ++k)
-            umma_bf16(d_tmem, smem_desc_sw128(a + k * 32), smem_desc_sw128(bb + k * 32), idesc, (kb > im.kb0 || k > 0) ? 1u : 0u);
+          for (int k = 0; k < 4; ++k) {
+            const uint64_t da = ((uint64_t)desc_hi << 32) | (uint64_t)(a_lo + 2 * k);
+            const uint64_t db = ((uint64_t)desc_hi << 32) | (uint64_t)(b_lo + 2 * k);
+            umma_bf16(d_tmem, da, db, idesc, acc);
+            acc = 1u;
+          }
           umma_commit(&sh.empty_w[ws]);
           umma_commit(&sh.empty_x[xs]);
-          ++ps.wc; ++ps.xc;
+          ps.wc.step(n_sw);
+          ps.xc.step(n_sx);
         }
         if (!ok) break;
         umma_commit(&sh.acc_full[b]);
@@ -562,7 +646,7 @@ __device__ __forceinline__ void gemm_phase(const MegaParams& P, int which, const
   for (int it = blockIdx.x; it < n_items; it += gridDim.x) {
     const Item im = item_of(g, it);
     const uint32_t b = ps.ae & 1u;
-    const bool ok = wait_bar(&sh.acc_full[b], (ps.ae >> 1) & 1u, sh, P.err);
+    const bool ok = wait_bar(&sh.acc_full[b], (ps.ae >> 1) & 1u, sh, err);
     ++ps.ae;
     tc_fence_after();
     const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + b * (uint32_t)mt;
@@ -589,7 +673,7 @@ __device__ __forceinline__ void gemm_phase(const MegaParams& P, int which, const
       }
     } else {
       // gate rows in TMEM lanes 0-63 (warps 0, 1), the matching up rows in lanes 64-127 (warps 2, 3)
-      float* xch = sh.gen;                         // [64][65]
+      float* xch = sh.xch;                         // [64][65]
       const int l = (warp & 1) * 32 + lane;        // feature within the 64-row half
       if (ok && warp >= 2) {
         for (int c = 0; c < rows && c < B; c += 16) {
@@ -642,8 +726,9 @@ decode_mega_kernel(const MegaParams* __restrict__ Pp, const MegaLayer* __restric
   Shared sh;
   sh.wring = smem;
   sh.xring = sh.wring + (size_t)P.sw * kWStageBytes;
-  sh.gen = (float*)(sh.xring + (size_t)P.sx * P.mt * 128);
-  sh.row_scale = (float*)((uint8_t*)sh.gen + kGenScratchBytes);
+  sh.gen = (float*)sh.xring;
+  sh.xch = (float*)(sh.xring + (size_t)P.sx * P.mt * 128);
+  sh.row_scale = (float*)((uint8_t*)sh.xch + kXchBytes);
   sh.full_w = (uint64_t*)(sh.row_scale + 64);
   sh.empty_w = sh.full_w + P.sw;
   sh.full_x = sh.empty_w + P.sw;
@@ -654,6 +739,7 @@ decode_mega_kernel(const MegaParams* __restrict__ Pp, const MegaLayer* __restric
   sh.abort_flag = (volatile int*)(sh.tmem_slot + 1);
   sh.go = sh.abort_flag + 1;
   sh.flag = sh.abort_flag + 2;
+  sh.pref = (int*)(sh.abort_flag + 4);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
@@ -664,6 +750,25 @@ decode_mega_kernel(const MegaParams* __restrict__ Pp, const MegaLayer* __restric
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == kWarpMma) tmem_alloc(sh.tmem_slot, (uint32_t)P.tmem_cols);
+  if (warp == 1) {
+    // page counts of the rows of this iteration (idle slots: none), as prefix sums; B <= 64
+    int n0 = 0, n1 = 0;
+    if (lane < P.B && pv.tok_row[lane] >= 0) n0 = (pv.tok_pos[lane] + 1 + kPageTokens - 1) / kPageTokens;
+    if (lane + 32 < P.B && pv.tok_row[lane + 32] >= 0) n1 = (pv.tok_pos[lane + 32] + 1 + kPageTokens - 1) / kPageTokens;
+    int i0 = n0, i1 = n1;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int a = __shfl_up_sync(0xFFFFFFFFu, i0, o), b = __shfl_up_sync(0xFFFFFFFFu, i1, o);
+      if (lane >= o) { i0 += a; i1 += b; }
+    }
+    const int tot0 = __shfl_sync(0xFFFFFFFFu, i0, 31);
+    int mx = max(n0, n1);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = max(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+    if (lane == 0) { sh.pref[0] = 0; sh.pref[P.B + 1] = mx; }
+    if (lane < P.B) sh.pref[lane + 1] = i0;
+    if (lane + 32 < P.B) sh.pref[lane + 33] = tot0 + i1;
+  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -674,7 +779,11 @@ decode_mega_kernel(const MegaParams* __restrict__ Pp, const MegaLayer* __restric
     // ---------------- W producer: streams every weight tile of this CTA's work items, in order ----------------
     if (lane == 0) {
       uint32_t wi = 0;
+      RingPos wpos;
       bool ok = true;
+      const uint32_t n_sw = (uint32_t)P.sw;
+      int* const err = P.err;
+      const int F = P.F;
       for (int l = 0; l < L && ok; ++l) {
         for (int which = 0; which < 4 && ok; ++which) {
           const GemmPlan& g = P.plan[which];
@@ -683,17 +792,18 @@ decode_mega_kernel(const MegaParams* __restrict__ Pp, const MegaLayer* __restric
           for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
             const Item im = item_of(g, it);
             for (int kb = im.kb0; kb < im.kb1; ++kb) {
-              const uint32_t s = wi % (uint32_t)P.sw;
-              ok = wait_bar(&sh.empty_w[s], ((wi / (uint32_t)P.sw) & 1u) ^ 1u, sh, P.err);
+              const uint32_t s = wpos.stage;
+              ok = wait_bar(&sh.empty_w[s], wpos.parity ^ 1u, sh, err);
               if (!ok) break;
               uint8_t* dst = sh.wring + (size_t)s * kWStageBytes;
               mbar_expect_tx(&sh.full_w[s], kWStageBytes);
               if (which == 2) {
                 tma_load_2d(dst, map, &sh.full_w[s], kb * 64, im.tile * 64);
-                tma_load_2d(dst + kWStageBytes / 2, map, &sh.full_w[s], kb * 64, P.F + im.tile * 64);
+                tma_load_2d(dst + kWStageBytes / 2, map, &sh.full_w[s], kb * 64, F + im.tile * 64);
               } else {
                 tma_load_2d(dst, map, &sh.full_w[s], kb * 64, im.tile * 128);
               }
+              wpos.step(n_sw);
               ++wi;
             }
           }
@@ -701,36 +811,46 @@ decode_mega_kernel(const MegaParams* __restrict__ Pp, const MegaLayer* __restric
       }
       if (!ok) {
         // copies already requested must land before the CTA goes away
-        const uint32_t n_back = min(wi, (uint32_t)P.sw);
-        for (uint32_t i = wi - n_back; i < wi; ++i) {
-          uint64_t* bar = &sh.full_w[i % (uint32_t)P.sw];
-          const uint32_t parity = (i / (uint32_t)P.sw) & 1u;
+        for (uint32_t i = 0; i < min(wi, n_sw); ++i) {
+          // stage filled i + 1 steps ago
+          uint32_t st = wpos.stage, par = wpos.parity;
+          for (uint32_t k = 0; k <= i; ++k) {
+            if (st == 0) { st = n_sw - 1; par ^= 1u; } else --st;
+          }
           for (uint32_t k = 0; k < (1u << 16); ++k)
-            if (mbar_try_wait(bar, parity)) break;
+            if (mbar_try_wait(&sh.full_w[st], par)) break;
         }
       }
     }
   } else {
     PipeState ps;
+    int n_stamps = 1;
+    unsigned epoch = 0;
+    if (P.prof != nullptr && blockIdx.x == 0 && threadIdx.x == 0) P.prof[0] = global_timer();
     rn_phase(P, pv, 0, layers[0].norm1, true);
-    grid_sync(P, sh);
+    grid_sync(P, sh, epoch, n_stamps);
     for (int l = 0; l < L; ++l) {
       const MegaLayer& Ly = layers[l];
       if (*sh.go) gemm_phase(P, 0, sh, tmem_base, ps);
-      grid_sync(P, sh);
+      grid_sync(P, sh, epoch, n_stamps);
       if (*sh.go) attn_phase<EXT>(P, Ly, pv, sh);
-      grid_sync(P, sh);
+      grid_sync(P, sh, epoch, n_stamps);
       if (*sh.go) gemm_phase(P, 1, sh, tmem_base, ps);
-      grid_sync(P, sh);
+      grid_sync(P, sh, epoch, n_stamps);
       if (*sh.go) rn_phase(P, pv, P.plan[1].splits, Ly.norm2, false);
-      grid_sync(P, sh);
+      grid_sync(P, sh, epoch, n_stamps);
       if (*sh.go) gemm_phase(P, 2, sh, tmem_base, ps);
-      grid_sync(P, sh);
+      grid_sync(P, sh, epoch, n_stamps);
       if (*sh.go) gemm_phase(P, 3, sh, tmem_base, ps);
-      grid_sync(P, sh);
+      grid_sync(P, sh, epoch, n_stamps);
       if (*sh.go) rn_phase(P, pv, P.plan[3].splits, l + 1 < L ? layers[l + 1].norm1 : final_gain, false);
-      if (l + 1 < L) grid_sync(P, sh);
+      if (l + 1 < L) grid_sync(P, sh, epoch, n_stamps);
     }
+    if (P.prof != nullptr && blockIdx.x == 0 && threadIdx.x == 0) {
+      if (n_stamps < kMaxStamps) P.prof[n_stamps++] = global_timer();
+      P.prof[kMaxStamps + 1] = (unsigned long long)n_stamps;
+    }
+    if (threadIdx.x == 0 && !*sh.abort_flag) finish_grid_sync(P);
   }
   tc_fence_before();
   __syncthreads();
@@ -760,11 +880,16 @@ struct Geometry { int rows, sw, sx; size_t smem; };
 Geometry geometry(int B) {
   Geometry g;
   g.rows = B <= 16 ? 16 : (B <= 32 ? 32 : 64);
-  g.sx = 4;                                          // X ring; the rest of the budget goes to the W ring
-  const size_t fixed = 1024 + (size_t)kGenScratchBytes + 64 * 4 + 1024;
-  const size_t xbytes = (size_t)g.sx * 2 * g.rows * 128;
-  g.sw = (int)std::min<size_t>(12, (227 * 1024 - fixed - xbytes) / kWStageBytes);
-  g.smem = fixed + xbytes + (size_t)g.sw * kWStageBytes;
+  // The X ring is as deep as the W ring: a weight tile can only be consumed together with its activation
+  // tile, and both arrive with the same latency.  What is left over goes to the W ring.
+  const size_t fixed = 1024 + kXchBytes + 64 * 4 + 1024;
+  const size_t avail = 227 * 1024 - fixed;
+  const size_t xstage = (size_t)2 * g.rows * 128;
+  size_t n = avail / (kWStageBytes + xstage);
+  while (n * xstage < (size_t)kGenScratchBytes) ++n;        // the attention scratch lives in the X ring
+  g.sx = (int)n;
+  g.sw = (int)std::min<size_t>(16, (avail - n * xstage) / kWStageBytes);
+  g.smem = fixed + n * xstage + (size_t)g.sw * kWStageBytes;
   return g;
 }
 
@@ -818,7 +943,7 @@ cudaError_t mega_build(void* dev_block, const MegaBuild& a, cudaStream_t s) {
   P->plan[2] = make_plan(2 * m.F, m.d, 128, n_ctas);
   P->plan[2].splits = 1; P->plan[2].kbps = P->plan[2].total_kb;   // SwiGLU in the epilogue needs whole sums
   P->plan[3] = make_plan(m.d, m.F, 128, n_ctas);
-  P->attn_splits = std::max(1, std::min(kMaxAttnSplits, n_ctas / (a.B * m.KV)));
+  P->attn_splits = 0;
   const Geometry geo = geometry(a.B);
   P->sx = geo.sx; P->sw = geo.sw;
   if (P->sw < 3) return cudaErrorNotSupported;
@@ -829,7 +954,7 @@ cudaError_t mega_build(void* dev_block, const MegaBuild& a, cudaStream_t s) {
   P->act_hi = (__nv_bfloat16*)a.act; P->act_lo = (__nv_bfloat16*)a.act_lo;
   P->partials = a.partials; P->ssq = a.ssq; P->part_o = a.part_o; P->part_ml = a.part_ml;
   P->attn_cnt = a.sync_words + 16; P->grid_bar = (unsigned*)a.sync_words; P->err = a.err;
-  P->rope = a.rope; P->page_table = a.page_table;
+  P->rope = a.rope; P->page_table = a.page_table; P->prof = a.prof;
   const void* xs[6] = {a.h, a.h_lo, a.attn, a.attn_lo, a.act, a.act_lo};
   const int xk[6] = {m.d, m.d, hq, hq, m.F, m.F};
   for (int i = 0; i < 6; ++i)

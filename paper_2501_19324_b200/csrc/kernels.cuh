@@ -133,6 +133,8 @@ struct MegaBuild {
   int* err;                                        // raised to -5 when a bounded wait expires
   const float2* rope;
   const int32_t* page_table;
+  unsigned long long* prof;                        // null, or 1024 words: CTA 0's global-timer stamps around every grid
+                                                   // barrier of the last launch ([1023] = number of stamps)
 };
 bool mega_supported(const MegaShape& m, int B);
 size_t mega_block_bytes(int n_layers);

@@ -252,20 +252,20 @@ def test_merged_prm_on_the_drafts_trunk(shapes, bf16, tol):
 
 @pytest.mark.parametrize("B,ext", [(5, 0), (20, 0), (40, 0), (6, 1)])
 def test_persistent_decode_kernel_against_the_oracle_and_the_separate_kernels(B, ext):
-    """bf16 models at up to 64 rows decode with one persistent kernel per iteration (all layers, grid barriers
-    between the phases).  It must meet the oracle like the kernel-by-kernel path (RSD_DEBUG_NO_MEGA), agree with
-    that path far inside the bf16 bound, and launch far fewer kernels.  Batch sizes cover the 16-, 32- and 64-row
+    """RSD_DEBUG_PERSISTENT_DECODE: bf16 models at up to 64 rows decode with one persistent kernel per iteration
+    (all layers, grid barriers between the phases).  It must meet the oracle like the default kernel-by-kernel
+    path, agree with that path far inside the bf16 bound, and launch far fewer kernels.  Batch sizes cover the 16-, 32- and 64-row
     operand tiles; ext = hi + lo KV cache."""
-    from paper_2501_19324_b200 import lib, RSD_DEBUG_KEEP_LOGITS, RSD_DEBUG_NO_MEGA
+    from paper_2501_19324_b200 import lib, RSD_DEBUG_KEEP_LOGITS, RSD_DEBUG_PERSISTENT_DECODE
     from oracle.rsd_loop import DRAFT, TARGET
     prompts = ri.prompts(50 + B, B, 5, 40, MINI[0].vocab)
     kw = dict(max_step_tokens=5, max_steps=3, max_seq_tokens=80, step_end_id=3, step_end_mod=5, temperature=0.7, seed=8)
     probe_eng, probe = build_pair(MINI, bf16=True, prompts=prompts, loop_kwargs=kw,
-                                  engine_kwargs=dict(debug_flags=RSD_DEBUG_KEEP_LOGITS | RSD_DEBUG_NO_MEGA))
+                                  engine_kwargs=dict(debug_flags=RSD_DEBUG_KEEP_LOGITS))
     delta = float(np.median(probe.step(0.0)["rewards"]))
     probe_eng.close()
     runs = {}
-    for name, flags in (("mega", RSD_DEBUG_KEEP_LOGITS), ("separate", RSD_DEBUG_KEEP_LOGITS | RSD_DEBUG_NO_MEGA)):
+    for name, flags in (("mega", RSD_DEBUG_KEEP_LOGITS | RSD_DEBUG_PERSISTENT_DECODE), ("separate", RSD_DEBUG_KEEP_LOGITS)):
         eng, loop = build_pair(MINI, bf16=True, prompts=prompts, loop_kwargs=kw,
                                engine_kwargs=dict(debug_flags=flags, kv_extended=ext))
         before = lib().rsd_debug_launch_count()
