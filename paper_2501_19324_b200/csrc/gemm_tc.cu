@@ -183,9 +183,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
       }
       asm volatile("bar.sync 1, 128;" ::: "memory");   // the four epilogue warps only
     }
-    bool ok = false;
-    for (uint32_t i = 0; i < kWaitLimit && !ok; ++i) {
-      ok = mbar_try_wait(tmem_full, 0);
+    // the four epilogue warps sleep in hardware between polls (about 1 us at most): busy polling by 128 threads
+    // crowds the shared-memory pipe that the producer and the MMA issuer need for their own barriers
+    bool ok = mbar_try_wait(tmem_full, 0);
+    for (uint32_t i = 0; i < (1u << 21) && !ok; ++i) {
+      ok = mbar_try_wait_sleep(tmem_full, 0, 1000);
       if (!ok && flags[0]) break;                        // the CTA was stopped (idle phase or an expired wait)
     }
     if (!ok && flags[0] == 0) {
