@@ -295,6 +295,14 @@ int rsd_k_rope(float* v, const int32_t* pos, int32_t T, int32_t n_heads, int32_t
                void* cuda_stream);
 /* out[t, f] = silu(gu[t, f]) * gu[t, F + f]; gu fp32 [T, 2F], out of element type `dtype`.     */
 int rsd_k_swiglu(const float* gu, void* out, int32_t T, int32_t F, int32_t dtype, void* cuda_stream);
+/* Gate/up projection of the SwiGLU MLP with the nonlinearity in the GEMM epilogue (tcgen05 path, bf16):
+ * act[m, f] = silu(g[m, f]) * u[m, f], [g | u] = (x + x_lo)[M, K] * Wgu[2F, K]^T with Wgu rows = Wgate | Wup,
+ * written as the split-precision pair act_hi = bf16(act), act_lo = bf16(act - act_hi), both [M, F].
+ * F % 64 == 0, K % 8 == 0, 16-byte aligned rows; x_lo must be given.  `scratch`: at least
+ * rsd_k_gemm_scratch_bytes(M, 2F, K) bytes, zero on first use (it carries the kernel's error flag).
+ * RSD_ERR_UNSUPPORTED for other shapes.                                                         */
+int rsd_k_gemm_gu(const void* Wgu, const void* x, const void* x_lo, void* act_hi, void* act_lo, int32_t M, int32_t F,
+                  int32_t K, void* scratch, size_t scratch_bytes, void* cuda_stream);
 /* token[b] = argmax over v < v_limit of logits[b, v] / T + g, g = -log(-log u) with u the Philox
  * uniform of (seed; counter = (v / 4, pos[b] + 1, row[b], model_id), word v % 4), or the plain
  * argmax when temperature == 0; ties to the lowest id.  pos[b] is the position of the token fed to

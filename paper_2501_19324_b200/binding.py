@@ -56,7 +56,7 @@ EXPORTS = ["rsd_query_sizes", "rsd_create", "rsd_load_models", "rsd_prefill", "r
            "rsd_reset", "rsd_destroy", "rsd_last_error", "rsd_debug_force", "rsd_debug_get_logits",
            "rsd_debug_get_sampled", "rsd_debug_get_state", "rsd_debug_gemm_timing", "rsd_debug_launch_count", "rsd_debug_mega_profile", "rsd_debug_phase_ms", "rsd_k_gemm", "rsd_k_gemm_scratch_bytes",
            "rsd_k_attn_decode", "rsd_k_attn_decode_scratch_bytes", "rsd_k_attn_chunk", "rsd_k_gate_compact", "rsd_k_gate_compact_static", "rsd_k_gate_compact_static_error", "rsd_k_rmsnorm",
-           "rsd_k_rope", "rsd_k_swiglu", "rsd_k_sample", "rsd_k_philox"]
+           "rsd_k_rope", "rsd_k_swiglu", "rsd_k_gemm_gu", "rsd_k_sample", "rsd_k_philox"]
 
 _lib = None
 
@@ -104,6 +104,7 @@ def lib():
         L.rsd_k_rmsnorm.argtypes = [vp, vp, vp, c_int32, c_int32, c_float, c_int32, vp]
         L.rsd_k_rope.argtypes = [vp, vp, c_int32, c_int32, c_int32, c_float, vp]
         L.rsd_k_swiglu.argtypes = [vp, vp, c_int32, c_int32, c_int32, vp]
+        L.rsd_k_gemm_gu.argtypes = [vp, vp, vp, vp, vp, c_int32, c_int32, c_int32, vp, c_size_t, vp]
         L.rsd_k_sample.argtypes = [vp, c_int32, c_int32, c_int32, c_float, c_uint64, c_int32, vp, vp, vp, vp, c_size_t, vp]
         L.rsd_k_philox.argtypes = [vp, vp, vp, c_int32, vp]
         _lib = L
@@ -374,6 +375,19 @@ def k_swiglu(gu, out_dtype):
     dt = RSD_BF16 if out_dtype == torch.bfloat16 else RSD_F32
     _check(lib().rsd_k_swiglu(_ptr(gu), _ptr(out), T, F2 // 2, dt, _stream()))
     return out
+
+
+def k_gemm_gu(Wgu, x_hi, x_lo):
+    """Gate/up projection + SwiGLU on the tensor-core path: returns (act_hi, act_lo), bf16 [M, F]."""
+    import torch
+    M, K = x_hi.shape
+    F = Wgu.shape[0] // 2
+    hi = torch.zeros(M, F, dtype=torch.bfloat16, device=x_hi.device)
+    lo = torch.zeros(M, F, dtype=torch.bfloat16, device=x_hi.device)
+    nbytes = lib().rsd_k_gemm_scratch_bytes(M, 2 * F, K)
+    scratch = torch.zeros(nbytes, dtype=torch.uint8, device=x_hi.device)
+    _check(lib().rsd_k_gemm_gu(_ptr(Wgu), _ptr(x_hi), _ptr(x_lo), _ptr(hi), _ptr(lo), M, F, K, _ptr(scratch), nbytes, _stream()))
+    return hi, lo
 
 
 def k_sample(logits, v_limit, temperature, seed, model_id, row, pos):

@@ -337,6 +337,25 @@ int gemm(rsd_ctx* c, const ModelHost& M, const void* W, const void* xin, const v
   return RSD_OK;
 }
 
+// Gate/up projection + SwiGLU in one kernel (bf16 models); timed like gemm().
+int gemm_gu(rsd_ctx* c, const ModelHost& M, const void* Wgu, const void* xin, const void* xin_lo, void* act, void* act_lo,
+            int Mrows, int F, int K, const int32_t* n_active, cudaStream_t s, RowScale rs = RowScale()) {
+  const bool pick = c->in_decode ? c->time_this_iter
+                                 : (c->time_stride > 0 && (c->gemm_calls++ % (uint64_t)c->time_stride) == 0);
+  const bool timed = pick && c->ev_used < c->ev_bytes.size();
+  if (timed) CU(cudaEventRecord(c->ev[2 * c->ev_used], s));
+  CU(launch_gemm_gu(Wgu, xin, xin_lo, act, act_lo, Mrows, F, K, c->gemm_scratch, c->gemm_scratch_bytes, n_active, s, rs));
+  if (timed) {
+    CU(cudaEventRecord(c->ev[2 * c->ev_used + 1], s));
+    // algorithmic bytes: the stacked weight matrix and the input pair once, the output pair once
+    c->ev_bytes[c->ev_used] = 2.0 * F * K * M.elem + 2.0 * Mrows * K * M.elem + 2.0 * Mrows * F * M.elem;
+    ++c->ev_used;
+  }
+  return RSD_OK;
+}
+
+bool gu_fused_ok(const ModelHost& M) { return M.m.dtype == RSD_BF16 && M.split && gemm_gu_supported(1, 1, M.m.d_ffn, M.m.d_model); }
+
 int forward_pass(rsd_ctx* c, int which, PassView p, cudaStream_t s) {
   const ModelHost& M = c->mdl[which];
   const rsd_model& m = M.m;
@@ -370,10 +389,15 @@ int forward_pass(rsd_ctx* c, int which, PassView p, cudaStream_t s) {
     rc = gemm(c, M, M.wo[l], c->attn, attn_lo, c->x, T, d, H * hd, 1, p.n_active, defer_small ? &x_pending : nullptr, s);
     if (rc) return rc;
     CU(launch_rmsnorm(m.dtype, c->x, M.norm2[l], c->h, h_lo, T, d, m.rms_eps, nullptr, p.n_active, x_pending, s));
-    SplitSum gu_pending;
-    rc = gemm(c, M, M.wgu[l], c->h, h_lo, c->gu, T, 2 * F, d, 0, p.n_active, &gu_pending, s);
-    if (rc) return rc;
-    CU(launch_swiglu(m.dtype, c->gu, gu_pending, c->act, act_lo, T, F, p.n_active, s));
+    if (gu_fused_ok(M)) {
+      rc = gemm_gu(c, M, M.wgu[l], c->h, h_lo, c->act, act_lo, T, F, d, p.n_active, s);
+      if (rc) return rc;
+    } else {
+      SplitSum gu_pending;
+      rc = gemm(c, M, M.wgu[l], c->h, h_lo, c->gu, T, 2 * F, d, 0, p.n_active, &gu_pending, s);
+      if (rc) return rc;
+      CU(launch_swiglu(m.dtype, c->gu, gu_pending, c->act, act_lo, T, F, p.n_active, s));
+    }
     // the last layer's result must be complete in x when the pass ends
     const bool last = l + 1 == m.n_layers;
     x_pending = SplitSum();
@@ -412,9 +436,14 @@ int forward_decode_fused(rsd_ctx* c, int which, PassView p, const void* final_ga
     if (rc) return rc;
     CU(launch_reduce_norm(x_pending.partials, x_pending.splits, c->x, M.norm2[l], c->h, c->h_lo, c->norm_ssq, T, d,
                           p.n_active, s));
-    rc = gemm(c, M, M.wgu[l], c->h, c->h_lo, c->gu, T, 2 * F, d, 0, p.n_active, &gu_pending, s, rs);
-    if (rc) return rc;
-    CU(launch_swiglu(m.dtype, c->gu, gu_pending, c->act, c->act_lo, T, F, p.n_active, s));
+    if (gu_fused_ok(M)) {
+      rc = gemm_gu(c, M, M.wgu[l], c->h, c->h_lo, c->act, c->act_lo, T, F, d, p.n_active, s, rs);
+      if (rc) return rc;
+    } else {
+      rc = gemm(c, M, M.wgu[l], c->h, c->h_lo, c->gu, T, 2 * F, d, 0, p.n_active, &gu_pending, s, rs);
+      if (rc) return rc;
+      CU(launch_swiglu(m.dtype, c->gu, gu_pending, c->act, c->act_lo, T, F, p.n_active, s));
+    }
     x_pending = SplitSum();
     rc = gemm(c, M, M.wdown[l], c->act, c->act_lo, c->x, T, d, F, 1, p.n_active, &x_pending, s);
     if (rc) return rc;
@@ -1146,6 +1175,15 @@ int rsd_k_rope(float* v, const int32_t* pos, int32_t T, int32_t n_heads, int32_t
 int rsd_k_swiglu(const float* gu, void* out, int32_t T, int32_t F, int32_t dtype, void* cuda_stream) {
   if (!gu || !out || T < 0 || F < 1) return RSD_ERR_ARG;
   KCU(launch_swiglu(dtype, gu, SplitSum(), out, nullptr, T, F, nullptr, (cudaStream_t)cuda_stream));
+  return RSD_OK;
+}
+
+int rsd_k_gemm_gu(const void* Wgu, const void* x, const void* x_lo, void* act_hi, void* act_lo, int32_t M, int32_t F,
+                  int32_t K, void* scratch, size_t scratch_bytes, void* cuda_stream) {
+  if (!Wgu || !x || !x_lo || !act_hi || !act_lo || M < 0 || F < 1 || K < 1) return RSD_ERR_ARG;
+  if (!gemm_gu_supported(RSD_BF16, M > 0 ? M : 1, F, K)) return RSD_ERR_UNSUPPORTED;
+  if (!scratch || scratch_bytes < gemm_scratch_bytes(M)) return RSD_ERR_ARG;
+  KCU(launch_gemm_gu(Wgu, x, x_lo, act_hi, act_lo, M, F, K, scratch, scratch_bytes, nullptr, (cudaStream_t)cuda_stream));
   return RSD_OK;
 }
 

@@ -43,34 +43,47 @@ constexpr int kCounterBytes = 4096;
 constexpr int kMaxSplitTiles = kCounterBytes / 4;
 constexpr int kMaxSplitCtas = 640;
 
-template <int MT> struct TcCfg {
+// DEEP: a ring of eight (six for 128-row x tiles) stages for one CTA per SM, for grids that do not reach two CTAs per SM anyway (a lone
+// CTA needs about twice the bytes in flight to keep its share of the HBM stream going).
+template <int MT, bool DEEP = false> struct TcCfg {
   // tiles of up to 128 x-rows leave room for two CTAs per SM (one streams while the other starts
   // up or drains); the 256-row tile of the dense regime takes the SM alone
-  static constexpr int kCtasPerSm = MT <= 128 ? 2 : 1;
-  static constexpr int kStages = MT <= 32 ? 5 : (MT == 64 ? 4 : (MT == 128 ? 3 : 4));
+  static constexpr int kCtasPerSm = DEEP ? 1 : (MT <= 128 ? 2 : 1);
+  static constexpr int kStages = DEEP ? (MT <= 64 ? 8 : 6) : (MT <= 32 ? 5 : (MT == 64 ? 4 : (MT == 128 ? 3 : 4)));
   static constexpr int kABytes = kTileN * kTileK * 2;
   static constexpr int kBBytes = MT * kTileK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
   static constexpr int kTmemCols = MT < 32 ? 32 : MT;
   static constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + 256 + 512;   // barriers, row scales
+  // gate/up mode: two exchange buffers [64 features][MT / 4 rows + 1] between the gate and the up warps; they
+  // reuse the pipeline stages once the last MMA has read them
+  static constexpr size_t kXchBytes = 2 * 64 * (size_t)(MT / 4 + 1) * 4;
+  static_assert(kSmemBytes <= 227 * 1024, "shared memory of one CTA");
+  static_assert(kXchBytes <= (size_t)kStages * kStageBytes, "exchange buffers must fit in the stage ring");
   // instruction descriptor: fp32 accumulate, bf16 A and B, both K-major, N = MT, M = 128
   static constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(MT >> 3) << 17) | ((uint32_t)(kTileN >> 4) << 24);
 };
 
 // SPLIT: the x operand is a pair (hi, lo) of bf16 matrices whose sum is the activation; the tile
 // holds MT/2 rows of hi followed by the same MT/2 rows of lo, and the epilogue adds the two halves.
-template <int MT, bool SPLIT>
-__global__ void __launch_bounds__(192, TcCfg<MT>::kCtasPerSm)
+// GU (gate/up mode, SPLIT only): W is the stacked matrix [Wgate | Wup] of 2 * N rows; a CTA's 128-row tile is
+// 64 gate rows and the 64 up rows of the same features (two TMA boxes of 64 rows), there is no K split, and the
+// epilogue writes act = silu(gate) * up as the bf16 hi + lo operand pair [M, N] of the down projection instead
+// of Y.  The gate values sit in TMEM lanes 0-63 (warps 0, 1), the up values in lanes 64-127 (warps 2, 3); the
+// two warp pairs swap one half of the x rows each through shared memory, so all four warps compute.
+template <int MT, bool SPLIT, bool GU = false, bool DEEP = false>
+__global__ void __launch_bounds__(192, TcCfg<MT, DEEP>::kCtasPerSm)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x,
                const __grid_constant__ CUtensorMap tm_x_lo, float* __restrict__ Y,
                int M, int N, int K, int accumulate, int splits, int kb_per_split, float* __restrict__ partials,
-               int* __restrict__ err, const int32_t* __restrict__ n_active, RowScale rs) {
+               int* __restrict__ err, const int32_t* __restrict__ n_active, RowScale rs,
+               __nv_bfloat16* __restrict__ act_hi = nullptr, __nv_bfloat16* __restrict__ act_lo = nullptr) {
   // Programmatic dependent launch: the next kernel may be scheduled at once; this kernel sets itself
   // up and starts streaming its WEIGHT tiles (never written by any kernel) while its predecessors are
   // still running, and only then waits for them (griddepcontrol.wait) before it touches activations,
   // outputs or the idle flag.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  using Cfg = TcCfg<MT>;
+  using Cfg = TcCfg<MT, DEEP>;
   constexpr int kRows = SPLIT ? MT / 2 : MT;   // distinct x rows per tile
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -82,7 +95,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
   float* row_scale = (float*)(smem + (size_t)Cfg::kStages * Cfg::kStageBytes + 256);   // [kRows <= 128]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n0 = blockIdx.x * kTileN, m0 = blockIdx.y * kRows, split = blockIdx.z;
+  const int n0 = blockIdx.x * (GU ? kTileN / 2 : kTileN), m0 = blockIdx.y * kRows, split = blockIdx.z;
+  float* xch = (float*)smem;   // GU only: the exchange buffers reuse the pipeline stages, which are drained by then
   const int total_kb = (K + kTileK - 1) / kTileK;
   const int kb0 = split * kb_per_split;
   const int kb1 = min(total_kb, kb0 + kb_per_split);
@@ -109,7 +123,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
       const int pre = min(n_kb, Cfg::kStages);
       for (int i = 0; i < pre; ++i) {
         mbar_expect_tx(&full[i], Cfg::kStageBytes);
-        tma_load_2d(smem + (size_t)i * Cfg::kStageBytes, &tm_w, &full[i], (kb0 + i) * kTileK, n0);
+        uint8_t* a = smem + (size_t)i * Cfg::kStageBytes;
+        if (GU) {
+          tma_load_2d(a, &tm_w, &full[i], (kb0 + i) * kTileK, n0);
+          tma_load_2d(a + Cfg::kABytes / 2, &tm_w, &full[i], (kb0 + i) * kTileK, N + n0);
+        } else {
+          tma_load_2d(a, &tm_w, &full[i], (kb0 + i) * kTileK, n0);
+        }
       }
       issued = pre;
       asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -131,7 +151,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
           if (!ok || flags[0]) { ok = false; break; }
           uint8_t* a = smem + (size_t)s * Cfg::kStageBytes;
           mbar_expect_tx(&full[s], Cfg::kStageBytes);
-          tma_load_2d(a, &tm_w, &full[s], (kb0 + i) * kTileK, n0);
+          if (GU) {
+            tma_load_2d(a, &tm_w, &full[s], (kb0 + i) * kTileK, n0);
+            tma_load_2d(a + Cfg::kABytes / 2, &tm_w, &full[s], (kb0 + i) * kTileK, N + n0);
+          } else {
+            tma_load_2d(a, &tm_w, &full[s], (kb0 + i) * kTileK, n0);
+          }
           tma_load_2d(a + Cfg::kABytes, &tm_x, &full[s], (kb0 + i) * kTileK, m0);
           if (SPLIT) tma_load_2d(a + Cfg::kABytes + kRows * kTileK * 2, &tm_x_lo, &full[s], (kb0 + i) * kTileK, m0);
           issued = i + 1;
@@ -199,7 +224,50 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
     const int n = n0 + n_local;
     const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16);
     const int m_valid = min(kRows, M - m0);
-    if (ok) {
+    if (GU) {
+      // SwiGLU epilogue.  Rows [0, half) of the tile are finished by the gate warps (they receive the up values
+      // of those rows), rows [half, kRows) by the up warps (they receive the gate values).
+      constexpr int kHalf = kRows / 2, kLd = kHalf + 1;
+      const bool is_gate = warp < 2;
+      const int l = (warp & 1) * 32 + lane;                    // feature within the 64-row half
+      float* send = xch + (is_gate ? 64 * kLd : 0) + l * kLd;  // [0]: up values of the low rows, [1]: gate values of the high rows
+      const float* recv = xch + (is_gate ? 0 : 64 * kLd) + l * kLd;
+      const int send0 = is_gate ? kHalf : 0, own0 = is_gate ? 0 : kHalf;
+      if (ok) {
+#pragma unroll 1
+        for (int c = 0; c < kHalf; c += 16) {
+          float v[16], w[16];
+          tmem_ld16(taddr + send0 + c, v);
+          tmem_ld16(taddr + kRows + send0 + c, w);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) send[c + j] = v[j] + w[j];
+        }
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (ok && n0 + l < N) {
+#pragma unroll 1
+        for (int c = 0; c < kHalf; c += 16) {
+          if (own0 + c >= m_valid) break;
+          float v[16], w[16];
+          tmem_ld16(taddr + own0 + c, v);
+          tmem_ld16(taddr + kRows + own0 + c, w);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const int r = own0 + c + j;
+            if (r < m_valid) {
+              const float sc = rs.ssq != nullptr ? row_scale[r] : 1.f;
+              const float mine = (v[j] + w[j]) * sc, other = recv[c + j] * sc;
+              const float gate = is_gate ? mine : other, up = is_gate ? other : mine;
+              const float a = gate / (1.f + expf(-gate)) * up;
+              const size_t o = (size_t)(m0 + r) * N + n0 + l;
+              const __nv_bfloat16 h = __float2bfloat16_rn(a);
+              act_hi[o] = h;
+              act_lo[o] = __float2bfloat16_rn(a - __bfloat162float(h));
+            }
+          }
+        }
+      }
+    } else if (ok) {
       // with several K-splits each CTA stores its partial sums as rows of a [split][M][N] array;
       // a reduction kernel adds the splits in order afterwards (deterministic)
       float* dst = splits == 1 ? Y : partials + (size_t)split * M * N;
@@ -372,7 +440,8 @@ cudaError_t launch_mt(const CUtensorMap& tw, const CUtensorMap& tx, const CUtens
   }
   dim3 grid(p.n_tiles, p.m_tiles, p.splits);
   RSD_LAUNCH((gemm_tc_kernel<MT, SPLIT>), grid, 192, TcCfg<MT>::kSmemBytes, s, tw, tx, txl, y, M, N, K, accumulate, p.splits,
-                                                                     p.kb_per_split, partials, err, n_active, rs);
+                                                                     p.kb_per_split, partials, err, n_active, rs,
+                                                                     (__nv_bfloat16*)nullptr, (__nv_bfloat16*)nullptr);
   if (p.splits > 1 && !defer_reduce) {
     const size_t total4 = (size_t)M * N / 4;
     const int blocks = (int)std::min<size_t>((total4 + 255) / 256, 148 * 8);
@@ -391,6 +460,55 @@ bool tc_tensor_map(const void* ptr, int rows, int cols, int box_rows, CUtensorMa
 
 bool gemm_tc_supported(int dtype, int M, int N, int K) {
   return dtype == 1 && M >= 1 && N >= 1 && K >= 8 && K % 8 == 0;
+}
+
+template <int MT, bool DEEP>
+static cudaError_t launch_gu_mt(const CUtensorMap& tw, const CUtensorMap& tx, const CUtensorMap& txl, int M, int F, int K, int rows,
+                                int* err, const int32_t* n_active, RowScale rs, __nv_bfloat16* act_hi, __nv_bfloat16* act_lo,
+                                cudaStream_t s) {
+  constexpr size_t smem = TcCfg<MT, DEEP>::kSmemBytes;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<MT, true, true, DEEP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  const int total_kb = (K + kTileK - 1) / kTileK;
+  dim3 grid(F / 64, (M + rows - 1) / rows, 1);
+  RSD_LAUNCH((gemm_tc_kernel<MT, true, true, DEEP>), grid, 192, smem, s, tw, tx, txl, (float*)nullptr, M, F, K, 0, 1, total_kb,
+             (float*)nullptr, err, n_active, rs, act_hi, act_lo);
+  return launched(1);
+}
+
+bool gemm_gu_supported(int dtype, int M, int F, int K) {
+  return dtype == 1 && M >= 1 && F >= 64 && F % 64 == 0 && K >= 8 && K % 8 == 0;
+}
+
+// act (hi + lo, bf16 [M, F]) = silu(g) * u with [g | u] = rowscale * (x_hi + x_lo)[M, K] * Wgu[2F, K]^T.
+cudaError_t launch_gemm_gu(const void* Wgu, const void* x, const void* x_lo, void* act_hi, void* act_lo, int M, int F, int K,
+                           void* scratch, size_t scratch_bytes, const int32_t* n_active, cudaStream_t s, RowScale rs) {
+  if (M <= 0) return cudaSuccess;
+  if (!gemm_gu_supported(1, M, F, K) || !x_lo || !act_hi || !act_lo) return cudaErrorNotSupported;
+  if (!scratch || scratch_bytes < (size_t)kCounterBytes + 256) return cudaErrorInvalidValue;
+  if (((uintptr_t)Wgu & 15) || ((uintptr_t)x & 15) || ((uintptr_t)x_lo & 15)) return cudaErrorMisalignedAddress;
+  // at least 32 x rows per tile: each warp pair finishes one half of them, 16 at a time
+  const int rows = M <= 32 ? 32 : (M <= 64 ? 64 : 128);
+  if (rs.ssq != nullptr && rows > 128) return cudaErrorInvalidValue;
+  CUtensorMap tw, tx, txl;
+  if (!get_map(Wgu, 2 * F, K, kTileN / 2, &tw) || !get_map(x, M, K, rows, &tx) || !get_map(x_lo, M, K, rows, &txl))
+    return cudaErrorNotSupported;
+  int* err = (int*)((char*)scratch + kCounterBytes);
+  auto* hi = (__nv_bfloat16*)act_hi;
+  auto* lo = (__nv_bfloat16*)act_lo;
+  // fewer than ~1.5 CTAs per SM: one CTA per SM with a deep ring streams faster than a thin second wave
+  const bool deep = (F / 64) * ((M + rows - 1) / rows) <= 222;
+  switch (rows) {
+    case 32: return deep ? launch_gu_mt<64, true>(tw, tx, txl, M, F, K, rows, err, n_active, rs, hi, lo, s)
+                         : launch_gu_mt<64, false>(tw, tx, txl, M, F, K, rows, err, n_active, rs, hi, lo, s);
+    case 64: return deep ? launch_gu_mt<128, true>(tw, tx, txl, M, F, K, rows, err, n_active, rs, hi, lo, s)
+                         : launch_gu_mt<128, false>(tw, tx, txl, M, F, K, rows, err, n_active, rs, hi, lo, s);
+    default: return launch_gu_mt<256, false>(tw, tx, txl, M, F, K, rows, err, n_active, rs, hi, lo, s);
+  }
 }
 
 // Layout of the scratch: [0, 4096) tile counters (kept zero between launches), then one int error

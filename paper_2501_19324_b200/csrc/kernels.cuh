@@ -74,6 +74,12 @@ cudaError_t launch_gemm_tc(const void* W, const void* x, const void* x_lo, float
                            void* scratch, size_t scratch_bytes, const int32_t* n_active, int* deferred_splits,
                            cudaStream_t s, RowScale rs = RowScale());
 const float* gemm_partials(const void* scratch);
+// Gate/up projection with SwiGLU in the epilogue (bf16, split-precision operand): act_hi + act_lo [M, F] =
+// silu(g) * u with [g | u] = rowscale * (x + x_lo)[M, K] * Wgu[2F, K]^T, Wgu rows = Wgate | Wup.  No K split and no
+// fp32 gate/up array: the tile of a CTA is 64 gate rows and the 64 matching up rows.  F % 64 == 0.
+bool gemm_gu_supported(int dtype, int M, int F, int K);
+cudaError_t launch_gemm_gu(const void* Wgu, const void* x, const void* x_lo, void* act_hi, void* act_lo, int M, int F, int K,
+                           void* scratch, size_t scratch_bytes, const int32_t* n_active, cudaStream_t s, RowScale rs = RowScale());
 
 // impl: 0 = by shape, 1 = SIMT split-K GEMV, 2 = tcgen05.
 cudaError_t launch_gemm(int dtype, const void* W, const void* x, const void* x_lo, float* y, int M, int N, int K,

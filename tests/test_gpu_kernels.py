@@ -295,3 +295,29 @@ def test_extended_precision_attention(hd, H, KV):
     for t in range(0, len(rows), 3):
         for h in range(0, H, max(1, H // 4)):
             np.testing.assert_allclose(gotc[t, h], ref(rows[t], poss[t], qc[t, h], h), rtol=0, atol=2e-5)
+
+
+@pytest.mark.parametrize("M,F,K", [(1, 64, 64), (5, 192, 512), (32, 1408, 512), (33, 128, 520), (70, 2048, 768),
+                                   (129, 704, 1408), (300, 320, 256), (32, 8960, 1536)])
+def test_gate_up_gemm_with_swiglu_epilogue(M, F, K):
+    """Gate/up projection with SwiGLU inside the GEMM epilogue (tile = 64 gate rows + the 64 matching up rows):
+    against matmul + silu(g) * u written out in fp64.  Ragged M (all three tile heights and several x tiles), F of
+    one to many tiles, K not a multiple of 64; the hi + lo output pair must carry the result to ~16 bits."""
+    rng = np.random.default_rng(M * 13 + F)
+    W = ri.cpu_tensor(3, 7, 2 * F, K, True) * 8.0          # pre-activations of order one, so silu is exercised
+    W = dev(W, torch.bfloat16).float().cpu().numpy()
+    x = rng.normal(size=(M, K)).astype(np.float32)
+    xf = dev(x)
+    hi = xf.to(torch.bfloat16)
+    lo = (xf - hi.float()).to(torch.bfloat16)
+    gu = oracle.matmul(W, (hi.float() + lo.float()).cpu().numpy()).astype(np.float64)
+    g, u = gu[:, :F], gu[:, F:]
+    want = g / (1.0 + np.exp(-g)) * u
+    a_hi, a_lo = rb.k_gemm_gu(dev(W, torch.bfloat16), hi, lo)
+    got = a_hi.float().cpu().numpy().astype(np.float64) + a_lo.float().cpu().numpy()
+    scale = max(1.0, float(np.abs(want).max()))
+    np.testing.assert_allclose(got, want, rtol=0, atol=(3e-5 * np.sqrt(K) + 2e-5) * scale)
+    assert np.array_equal(a_hi.float().cpu().numpy(), torch.from_numpy(got.astype(np.float32)).to(torch.bfloat16).float().numpy()) or \
+        np.abs(a_hi.float().cpu().numpy() - got).max() <= 2 ** -8 * scale
+    again_hi, again_lo = rb.k_gemm_gu(dev(W, torch.bfloat16), hi, lo)
+    assert torch.equal(again_hi, a_hi) and torch.equal(again_lo, a_lo)
