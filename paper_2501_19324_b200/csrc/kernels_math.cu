@@ -120,17 +120,16 @@ reduce_norm_kernel(const float* __restrict__ partials, int splits, float* __rest
     float4 v = *reinterpret_cast<const float4*>(x + o);
     if (splits > 1) {
       const size_t stride = (size_t)M * d;
-      int sidx = 0;
-      for (; sidx + 4 <= splits; sidx += 4) {
-        float4 a[4];
+      // twelve loads in flight at a time (tail predicated): each group is one L2 round trip, and 10-24 splits
+      // are the rule; the sums stay in split order
+      for (int s0 = 0; s0 < splits; s0 += 12) {
+        float4 a[12];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) a[u] = __ldcg(reinterpret_cast<const float4*>(partials + (size_t)(sidx + u) * stride + o));
+        for (int u = 0; u < 12; ++u)
+          a[u] = s0 + u < splits ? __ldcg(reinterpret_cast<const float4*>(partials + (size_t)(s0 + u) * stride + o))
+                                 : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int u = 0; u < 4; ++u) { v.x += a[u].x; v.y += a[u].y; v.z += a[u].z; v.w += a[u].w; }
-      }
-      for (; sidx < splits; ++sidx) {
-        const float4 a = __ldcg(reinterpret_cast<const float4*>(partials + (size_t)sidx * stride + o));
-        v.x += a.x; v.y += a.y; v.z += a.z; v.w += a.w;
+        for (int u = 0; u < 12; ++u) { v.x += a[u].x; v.y += a[u].y; v.z += a[u].z; v.w += a[u].w; }
       }
       *reinterpret_cast<float4*>(x + o) = v;
     }
@@ -265,17 +264,15 @@ cudaError_t launch_rope_table(float2* table, int n_pos, int hd, float theta, cud
 __device__ __forceinline__ float split_sum(const float* __restrict__ direct, const float* __restrict__ partials, int splits,
                                            size_t idx, size_t stride) {
   if (splits <= 1) return direct[idx];
-  // loads go out eight at a time so their latencies overlap; the sums stay in split order
+  // loads go out twelve at a time (tail predicated) so their latencies overlap; the sums stay in split order
   float v = 0.f;
-  int sidx = 0;
-  for (; sidx + 8 <= splits; sidx += 8) {
-    float t[8];
+  for (int s0 = 0; s0 < splits; s0 += 12) {
+    float t[12];
 #pragma unroll
-    for (int u = 0; u < 8; ++u) t[u] = __ldcg(partials + (size_t)(sidx + u) * stride + idx);
+    for (int u = 0; u < 12; ++u) t[u] = s0 + u < splits ? __ldcg(partials + (size_t)(s0 + u) * stride + idx) : 0.f;
 #pragma unroll
-    for (int u = 0; u < 8; ++u) v += t[u];
+    for (int u = 0; u < 12; ++u) v += t[u];
   }
-  for (; sidx < splits; ++sidx) v += __ldcg(partials + (size_t)sidx * stride + idx);
   return v;
 }
 
