@@ -257,6 +257,27 @@ def mega_phase_table(eng, which: int, n_layers: int) -> dict:
     return out
 
 
+def decode_iteration_roofline(phases, iters, steps, shapes, hbm, queue):
+    """Whole decode iterations against the HBM roofline: the bytes an iteration must read at least (every layer's
+    weights and the lm head once; the KV cache, which comes on top, is left out) over the measured time of an
+    iteration inside the step loop (phase time / iterations; a rejected row's draft step ran to the cap before it
+    was dropped).  Only meaningful for the lock-step schedule."""
+    if queue != 1:
+        return None
+    out = {}
+    for name, slot, key in (("draft", 0, "draft_decode"), ("target", 2, "target_decode")):
+        sh = shapes[slot]
+        weight_bytes = 2.0 * (sh.n_params() - sh.vocab * sh.d_model)       # bf16; the embedding table is not streamed
+        n = iters[name]
+        if n <= 0 or phases.get(key, 0) <= 0:
+            out[name] = None
+            continue
+        ms = phases[key] * steps / n
+        gbs = weight_bytes / (ms * 1e-3) / 1e9
+        out[name] = {"ms": ms, "weight_gb": weight_bytes / 1e9, "gbs": gbs, "frac_of_hbm": gbs / hbm, "iterations": n}
+    return out
+
+
 def rank_prompts(rank, B, lo, hi, vocab):
     """Every replica works on its own prompts (seed 1 + rank)."""
     return ri.prompts(1 + rank, B, lo, hi, vocab)
@@ -329,11 +350,19 @@ def run_ours(args, rank: int, world: int):
     t_start = torch.cuda.Event(enable_timing=True); t_end = torch.cuda.Event(enable_timing=True)
     t_start.record()
     timed_tokens = 0
+    iters = {"draft": 0, "target": 0}
     for _ in range(args.steps):
         r = eng.step(delta, args.queue)                    # host outputs: D2H inside the call
         timed_tokens += int(r["step_len"].sum())
         accepted += int(r["accept"].sum())
         live_steps += int((r["step_len"] > 0).sum())
+        # decode iterations of the step: a phase runs until its longest row ends
+        took = r["step_len"] > 0
+        rejected = took & (r["accept"] == 0)
+        if took.any():
+            iters["draft"] += cap if rejected.any() else int(r["step_len"][took].max())
+        if rejected.any():
+            iters["target"] += int(r["step_len"][rejected].max())
     t_end.record()
     barrier()
     e2e_end.record()
@@ -381,6 +410,7 @@ def run_ours(args, rank: int, world: int):
                             "peak_source": how, "timed_launches": gt["launches"],
                             "timing": f"CUDA events around every {args.time_stride}th GEMM launch of the timed steps"},
                "phase_ms_per_step": phases,
+               "decode_iteration": decode_iteration_roofline(phases, iters, args.steps, shapes, hbm, args.queue),
                "flops_paper": counters["flops_paper"], "clocks": clocks,
                "gen_tokens": counters["gen_tokens"]}
         if mega_tables is not None:

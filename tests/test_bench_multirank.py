@@ -57,3 +57,21 @@ def test_reference_arm_only_rank_zero_prints():
     line = json.loads(r.stdout.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["value"] > 0 and line["cpu_baseline"]["kind"] == "oracle"
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["n_gpus"] == 2
+
+
+def test_decode_iteration_roofline_arithmetic():
+    """bench.py's whole-iteration roofline: weight bytes of the model (embedding table excluded) over the measured
+    time of one decode iteration, by hand for the 1.5B shape."""
+    sys.path.insert(0, ROOT)
+    import bench
+    import rsd_inputs as ri
+    shapes = [ri.SHAPES["1.5b"], ri.SHAPES["1.5b"], ri.SHAPES["7b"]]
+    phases = {"draft_decode": 256.0, "target_decode": 448.0}          # ms per step
+    r = bench.decode_iteration_roofline(phases, {"draft": 3 * 128, "target": 2 * 128}, 3, shapes, 6538.0, 1)
+    # 28 layers x 46,792,704 matrix parameters + norm gains + lm head of 151936 x 1536, two bytes each
+    want_bytes = 2.0 * (28 * (46_792_704 + 2 * 1536) + 1536 + 151936 * 1536)
+    assert abs(r["draft"]["weight_gb"] * 1e9 - want_bytes) < 1.0
+    assert abs(r["draft"]["ms"] - 2.0) < 1e-12 and abs(r["target"]["ms"] - 5.25) < 1e-12
+    assert abs(r["draft"]["frac_of_hbm"] - want_bytes / 2.0e-3 / 1e9 / 6538.0) < 1e-9
+    assert bench.decode_iteration_roofline(phases, {"draft": 1, "target": 0}, 3, shapes, 6538.0, 1)["target"] is None
+    assert bench.decode_iteration_roofline(phases, {"draft": 1, "target": 1}, 3, shapes, 6538.0, 8) is None
