@@ -80,9 +80,11 @@ struct rsd_ctx {
   int last_n_rej = 0;
   // one CUDA graph per decode phase (draft, target): a whole decode iteration, replayed per token
   cudaStream_t cap_stream = nullptr;
-  cudaGraphExec_t dec_graph[2] = {nullptr, nullptr};
-  int dec_graph_B[2] = {0, 0};
-  uint64_t dec_graph_kernels[2] = {0, 0};
+  // slot = phase * 4 + bucket of the number of rows that take part (all, a half, a quarter, an eighth or fewer)
+  cudaGraphExec_t dec_graph[8] = {};
+  int dec_graph_B[8] = {};
+  uint64_t dec_graph_kernels[8] = {};
+  int attn_rows_hint = 0;      // rows expected to be active in the running decode phase (0: all slots)
   bool time_this_iter = false, in_decode = false;
   // per-phase timing of rsd_step (rsd_debug_phase_ms)
   bool time_phases = false;
@@ -387,7 +389,7 @@ int forward_pass(rsd_ctx* c, int which, PassView p, cudaStream_t s) {
       // decode pass: one query per row slot
       CU(launch_attn_decode(M.kv_dtype, c->q, kv.pool_layer, kv.page_table, kv.max_pages, p.tok_row, p.tok_pos, 1,
                             c->attn, attn_lo, m.dtype, T, H, KV, hd, c->S, c->attn_scratch, c->attn_scratch_bytes,
-                            p.n_active, s));
+                            p.n_active, s, c->attn_rows_hint));
     } else {
       CU(launch_attn_chunk(M.kv_dtype, c->q, p, kv, c->attn, attn_lo, m.dtype, H, KV, hd, s));
     }
@@ -436,7 +438,7 @@ int forward_decode_fused(rsd_ctx* c, int which, PassView p, const void* final_ga
     CU(launch_rope_kv(M.kv_dtype, c->qkv, qkv_pending, p, c->q, kv, M.rope, H, KV, hd, s));
     CU(launch_attn_decode(M.kv_dtype, c->q, kv.pool_layer, kv.page_table, kv.max_pages, p.tok_row, p.tok_pos, 1,
                           c->attn, c->attn_lo, m.dtype, T, H, KV, hd, c->S, c->attn_scratch, c->attn_scratch_bytes,
-                          p.n_active, s));
+                          p.n_active, s, c->attn_rows_hint));
     rc = gemm(c, M, M.wo[l], c->attn, c->attn_lo, c->x, T, d, H * hd, 1, p.n_active, &x_pending, s);
     if (rc) return rc;
     CU(launch_reduce_norm(x_pending.partials, x_pending.splits, c->x, M.norm2[l], c->h, c->h_lo, c->norm_ssq, T, d,
@@ -571,10 +573,10 @@ int decode_iteration(rsd_ctx* c, int which, int phase, int n_slots, cudaStream_t
 
 // Captures one decode iteration of `which` over all B slots into a graph (idle slots are skipped
 // inside the kernels), so that a token costs one graph launch instead of some 300 kernel launches.
-int ensure_decode_graph(rsd_ctx* c, int which, int phase) {
+int ensure_decode_graph(rsd_ctx* c, int which, int phase, int g) {
   const int B = c->st.B;
-  if (c->dec_graph[phase] && c->dec_graph_B[phase] == B) return RSD_OK;
-  if (c->dec_graph[phase]) { cudaGraphExecDestroy(c->dec_graph[phase]); c->dec_graph[phase] = nullptr; }
+  if (c->dec_graph[g] && c->dec_graph_B[g] == B) return RSD_OK;
+  if (c->dec_graph[g]) { cudaGraphExecDestroy(c->dec_graph[g]); c->dec_graph[g] = nullptr; }
   if (!c->cap_stream) CU(cudaStreamCreateWithFlags(&c->cap_stream, cudaStreamNonBlocking));
   const uint64_t before = launches_total();
   CU(cudaStreamBeginCapture(c->cap_stream, cudaStreamCaptureModeThreadLocal));
@@ -586,11 +588,11 @@ int ensure_decode_graph(rsd_ctx* c, int which, int phase) {
   cudaError_t e = cudaStreamEndCapture(c->cap_stream, &graph);
   if (rc) { if (graph) cudaGraphDestroy(graph); return rc; }
   CU(e);
-  c->dec_graph_kernels[phase] = launches_total() - before;
-  e = cudaGraphInstantiate(&c->dec_graph[phase], graph, 0);
+  c->dec_graph_kernels[g] = launches_total() - before;
+  e = cudaGraphInstantiate(&c->dec_graph[g], graph, 0);
   cudaGraphDestroy(graph);
   CU(e);
-  c->dec_graph_B[phase] = B;
+  c->dec_graph_B[g] = B;
   return RSD_OK;
 }
 
@@ -600,6 +602,12 @@ int decode_phase(rsd_ctx* c, int which, int phase, int n_slots, cudaStream_t s) 
   CU(launch_decode_begin(c->st, phase, s));
   if (n_slots <= 0) return RSD_OK;
   const bool graphs = !(c->cfg.debug_flags & RSD_DEBUG_NO_GRAPHS);
+  // The attention kernel splits every row's context over so many CTAs that the ACTIVE rows fill the machine; the
+  // rows of the phase are known here, so the iteration is captured once per power-of-two bucket of that number.
+  int bucket = 0, rows_eff = c->st.B;
+  while (bucket < 3 && n_slots * 2 <= rows_eff) { rows_eff = (rows_eff + 1) / 2; ++bucket; }
+  c->attn_rows_hint = rows_eff;
+  const int g = phase * 4 + bucket;
   if (graphs || c->mega_B[which] == c->st.B) n_slots = c->st.B;   // fixed shape: slots beyond the phase's rows are idle
   c->in_decode = true;
   int rc = RSD_OK;
@@ -607,15 +615,15 @@ int decode_phase(rsd_ctx* c, int which, int phase, int n_slots, cudaStream_t s) 
     const bool timed_iter = c->time_stride > 0 && (j % 16) == 5;
     // the first iteration ever runs kernel by kernel (it also sets every kernel's attributes), then
     // the iteration is captured once and replayed
-    const bool have_graph = graphs && c->dec_graph[phase] && c->dec_graph_B[phase] == c->st.B;
+    const bool have_graph = graphs && c->dec_graph[g] && c->dec_graph_B[g] == c->st.B;
     if (graphs && !have_graph && j > 0) {
-      rc = ensure_decode_graph(c, which, phase);
+      rc = ensure_decode_graph(c, which, phase, g);
       if (rc) break;
     }
-    if (graphs && !timed_iter && c->dec_graph[phase] && c->dec_graph_B[phase] == c->st.B) {
-      cudaError_t e = cudaGraphLaunch(c->dec_graph[phase], s);
+    if (graphs && !timed_iter && c->dec_graph[g] && c->dec_graph_B[g] == c->st.B) {
+      cudaError_t e = cudaGraphLaunch(c->dec_graph[g], s);
       if (e != cudaSuccess) { c->in_decode = false; CU(e); }
-      note_replayed_launches(c->dec_graph_kernels[phase]);
+      note_replayed_launches(c->dec_graph_kernels[g]);
     } else {
       c->time_this_iter = timed_iter;
       rc = decode_iteration(c, which, phase, n_slots, s);
@@ -628,6 +636,7 @@ int decode_phase(rsd_ctx* c, int which, int phase, int n_slots, cudaStream_t s) 
     }
   }
   c->in_decode = false;
+  c->attn_rows_hint = 0;
   return rc;
 }
 

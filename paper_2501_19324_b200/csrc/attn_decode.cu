@@ -234,15 +234,26 @@ attn_merge_kernel(const float* __restrict__ part_o, const float* __restrict__ pa
   const int slot = blockIdx.y, h = blockIdx.x, dd = threadIdx.x;
   if ((slot_row && slot_row[slot] < 0) || len_or_pos[slot] + len_offset <= 0) return;
   const size_t base = ((size_t)slot * H + h) * n_splits;
-  float M = -INFINITY;
-  for (int s = 0; s < n_splits; ++s) M = fmaxf(M, part_ml[(base + s) * 2]);
-  float L = 0.f, O = 0.f;
-  for (int s = 0; s < n_splits; ++s) {
-    const float m = part_ml[(base + s) * 2];
-    if (m > -INFINITY) {
-      const float e = __expf(m - M);
-      L += part_ml[(base + s) * 2 + 1] * e;
-      O += part_o[(base + s) * HD + dd] * e;
+  // four splits at a time with every load of the group in flight together; running maximum as in the kernel above
+  float M = -INFINITY, L = 0.f, O = 0.f;
+  for (int s0 = 0; s0 < n_splits; s0 += 4) {
+    float2 ml[4];
+    float ov[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const bool in = s0 + u < n_splits;
+      ml[u] = in ? *reinterpret_cast<const float2*>(part_ml + (base + s0 + u) * 2) : make_float2(-INFINITY, 0.f);
+      ov[u] = in ? part_o[(base + s0 + u) * HD + dd] : 0.f;
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      if (ml[u].x > -INFINITY) {
+        const float Mn = fmaxf(M, ml[u].x);
+        const float e_old = __expf(M - Mn), e_new = __expf(ml[u].x - Mn);
+        L = L * e_old + ml[u].y * e_new;
+        O = O * e_old + ov[u] * e_new;
+        M = Mn;
+      }
     }
   }
   store_operand<OT>(out, out_lo, ((size_t)slot * H + h) * HD + dd, O / L);
@@ -278,7 +289,7 @@ size_t attn_decode_scratch_bytes(int B, int H, int hd, int max_ctx) {
 cudaError_t launch_attn_decode(int kv_dtype, const float* q, const void* pool_layer, const int32_t* page_table,
                                int max_pages, const int32_t* slot_row, const int32_t* len_or_pos, int len_offset,
                                void* out, void* out_lo, int out_dtype, int B, int H, int KV, int hd, int max_ctx,
-                               void* scratch, size_t scratch_bytes, const int32_t* n_active, cudaStream_t s) {
+                               void* scratch, size_t scratch_bytes, const int32_t* n_active, cudaStream_t s, int active_rows) {
   if (B <= 0) return cudaSuccess;
   if (!scratch || scratch_bytes < attn_decode_scratch_bytes(B, H, hd, max_ctx)) return cudaErrorInvalidValue;
   const int G = H / KV;
@@ -295,7 +306,7 @@ cudaError_t launch_attn_decode(int kv_dtype, const float* q, const void* pool_la
   const size_t head = ((sizeof(int32_t) * 2 * (size_t)B + 255) / 256) * 256;
   float* part_ml = (float*)((char*)scratch + head);
   float* part_o = part_ml + (size_t)B * H * kMaxSplits * 2;
-  const int splits = pick_splits(B, KV, max_ctx);
+  const int splits = pick_splits(active_rows > 0 ? std::min(active_rows, B) : B, KV, max_ctx);
   dim3 grid(KV, B, splits);
 #define RSD_DEC(HD, KT, OT, EXTV)                                                                                          \
   do {                                                                                                               \

@@ -95,7 +95,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
   float* row_scale = (float*)(smem + (size_t)Cfg::kStages * Cfg::kStageBytes + 256);   // [kRows <= 128]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n0 = blockIdx.x * (GU ? kTileN / 2 : kTileN), m0 = blockIdx.y * kRows, split = blockIdx.z;
+  // Tile order.  CTAs start in the order of their linear index; with n fastest, the CTAs in flight together would
+  // hold as many different weight tiles as there are SMs and the weight matrix would come from HBM once per row
+  // tile of x.  With several row tiles the index is therefore walked in groups of eight row tiles, row tile
+  // fastest: the CTAs in flight share eight x tiles and a few weight tiles, both of which stay in L2.
+  int tile_n = blockIdx.x, tile_m = blockIdx.y;
+  if (gridDim.y > 1) {
+    constexpr int kGroup = 8;
+    const int lin = blockIdx.y * gridDim.x + blockIdx.x, per_group = kGroup * gridDim.x;
+    const int g0 = (lin / per_group) * kGroup, rem = lin % per_group;
+    const int gsz = min(kGroup, (int)gridDim.y - g0);
+    tile_m = g0 + rem % gsz;
+    tile_n = rem / gsz;
+  }
+  const int n0 = tile_n * (GU ? kTileN / 2 : kTileN), m0 = tile_m * kRows, split = blockIdx.z;
   float* xch = (float*)smem;   // GU only: the exchange buffers reuse the pipeline stages, which are drained by then
   const int total_kb = (K + kTileK - 1) / kTileK;
   const int kb0 = split * kb_per_split;

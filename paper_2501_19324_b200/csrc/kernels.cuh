@@ -110,11 +110,12 @@ cudaError_t launch_swiglu(int dtype, const float* gu, SplitSum pending, void* ou
 // Decode attention (one query per row) with split-KV partial results merged in a second pass.
 size_t attn_decode_scratch_bytes(int B, int H, int hd, int max_ctx);
 // Slot i attends positions [0, len_or_pos[i] + len_offset) of row slot_row[i] (slot i itself when
-// slot_row is null); slot_row[i] < 0 skips the slot.
+// slot_row is null); slot_row[i] < 0 skips the slot.  active_rows (0 = B): how many of the B slots are expected to
+// carry a row; the context splits are chosen so that those fill the machine (idle slots cost nothing).
 cudaError_t launch_attn_decode(int kv_dtype, const float* q, const void* pool_layer, const int32_t* page_table,
                                int max_pages, const int32_t* slot_row, const int32_t* len_or_pos, int len_offset,
                                void* out, void* out_lo, int out_dtype, int B, int H, int KV, int hd, int max_ctx, void* scratch,
-                               size_t scratch_bytes, const int32_t* n_active, cudaStream_t s);
+                               size_t scratch_bytes, const int32_t* n_active, cudaStream_t s, int active_rows = 0);
 
 // ---- persistent decode kernel: the whole layer stack of one decode iteration in one launch -------------
 struct MegaShape {
