@@ -52,7 +52,7 @@ __device__ __forceinline__ void mma_c<__half>(float (&d)[4], uint32_t a0, uint32
 // EXT: hi + lo pairs for the queries and the softmax weights, low halves of the values in a third block
 // of every page (see the decode kernel).
 template <int HD, typename KT, typename OT, bool EXT>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, EXT ? 1 : 2)   // two CTAs per SM: one alone (7 warps) cannot hide the page loads
 attn_chunk_kernel(const float* __restrict__ q, PassView p, const KT* __restrict__ pool, const int32_t* __restrict__ page_table,
                   int max_pages, OT* __restrict__ out, OT* __restrict__ out_lo, int H, int KV) {
   RSD_PDL_SYNC();
