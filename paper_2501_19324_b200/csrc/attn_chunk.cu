@@ -49,17 +49,33 @@ __device__ __forceinline__ void mma_c<__half>(float (&d)[4], uint32_t a0, uint32
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// The pages of the row travel through a ring of shared-memory stages filled with cp.async by all warps of the CTA
+// (the warps are the query heads of one KV head, so they all need the same keys and values): the copies of the next
+// pages are in flight while the MMAs of the current page run, and every warp reads its fragments from shared
+// memory instead of waiting for global memory page by page.  Key rows are padded by 16 bytes against bank conflicts.
 // EXT: hi + lo pairs for the queries and the softmax weights, low halves of the values in a third block
 // of every page (see the decode kernel).
 template <int HD, typename KT, typename OT, bool EXT>
-__global__ void __launch_bounds__(256, EXT ? 1 : 2)   // two CTAs per SM: one alone (7 warps) cannot hide the page loads
+__global__ void __launch_bounds__(256)
 attn_chunk_kernel(const float* __restrict__ q, PassView p, const KT* __restrict__ pool, const int32_t* __restrict__ page_table,
                   int max_pages, OT* __restrict__ out, OT* __restrict__ out_lo, int H, int KV) {
   RSD_PDL_SYNC();
   constexpr int KB = HD / 32, NT = HD / 8;
+  constexpr int NS = EXT ? 2 : 4;              // ring stages (a stage: keys + values of one page, EXT: and their low halves)
+  constexpr int KP = HD + 8;                   // padded key row
+  __shared__ __align__(16) KT s_k[NS][kPageTokens][KP];
+  __shared__ __align__(16) KT s_v[NS][HD][kPageTokens];
+  __shared__ __align__(16) KT s_kl[EXT ? NS : 1][EXT ? kPageTokens : 1][EXT ? KP : 8];
+  __shared__ __align__(16) KT s_vl[EXT ? NS : 1][EXT ? HD : 1][EXT ? kPageTokens : 8];
   const int G = H / KV;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  if (warp >= G) return;
+  const int n_thr = blockDim.x;                // 32 * G: every thread belongs to a working warp
   const int kvh = blockIdx.y, h = kvh * G + warp;
   const int t0 = blockIdx.x * 16;
   const int n_tile = min(16, p.T - t0);
@@ -110,21 +126,44 @@ attn_chunk_kernel(const float* __restrict__ q, PassView p, const KT* __restrict_
     float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
     const int32_t* pt = page_table + (size_t)r * max_pages;
     const int n_pages = pos_last / kPageTokens + 1;
+    // one page -> one ring stage: 2 * HD pieces of 16 bytes for the keys (16 rows of HD) and as many for the values
+    auto issue_page = [&](int pg) {
+      if (pg < n_pages) {
+        const int st = pg % NS;
+        const KT* kb = pool + (size_t)pt[pg] * page_elems + (size_t)kvh * kPageTokens * HD;
+        const KT* vb = pool + (size_t)pt[pg] * page_elems + block_elems + (size_t)kvh * HD * kPageTokens;
+        for (int c = threadIdx.x; c < 2 * HD; c += n_thr) {
+          const int r = c / (HD / 8), pc = c % (HD / 8);
+          cp_async16(&s_k[st][r][pc * 8], kb + r * HD + pc * 8);
+          cp_async16(&s_v[st][0][0] + c * 8, vb + c * 8);
+          if (EXT) {
+            cp_async16(&s_kl[st][r][pc * 8], kb + 2 * block_elems + r * HD + pc * 8);
+            cp_async16(&s_vl[st][0][0] + c * 8, vb + 2 * block_elems + c * 8);
+          }
+        }
+      }
+      cp_async_commit();                       // one group per page, empty beyond the last
+    };
+    __syncthreads();                           // every warp has left the previous segment's stages
+#pragma unroll
+    for (int i = 0; i < NS - 1; ++i) issue_page(i);
     for (int pg = 0; pg < n_pages; ++pg) {
-      const KT* kb = pool + (size_t)pt[pg] * page_elems + (size_t)kvh * kPageTokens * HD;
-      const KT* vb = pool + (size_t)pt[pg] * page_elems + (size_t)KV * kPageTokens * HD + (size_t)kvh * HD * kPageTokens;
+      cp_async_wait<NS - 2>();                 // this thread's copies of page pg have landed
+      __syncthreads();                         // everyone's have, and everyone is done with page pg - 1
+      issue_page(pg + NS - 1);                 // into the stage of page pg - 1
+      const int st = pg % NS;
       float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int j = 0; j < KB; ++j) {
-        const uint4 k0 = *reinterpret_cast<const uint4*>(kb + tok0 * HD + 32 * j + 8 * t);
-        const uint4 k1 = *reinterpret_cast<const uint4*>(kb + tok1 * HD + 32 * j + 8 * t);
+        const uint4 k0 = *reinterpret_cast<const uint4*>(&s_k[st][tok0][32 * j + 8 * t]);
+        const uint4 k1 = *reinterpret_cast<const uint4*>(&s_k[st][tok1][32 * j + 8 * t]);
         mma_c<KT>(s0, qa[j][0][0], qa[j][0][1], qa[j][0][2], qa[j][0][3], k0.x, k0.y);
         mma_c<KT>(s0, qa[j][1][0], qa[j][1][1], qa[j][1][2], qa[j][1][3], k0.z, k0.w);
         mma_c<KT>(s1, qa[j][0][0], qa[j][0][1], qa[j][0][2], qa[j][0][3], k1.x, k1.y);
         mma_c<KT>(s1, qa[j][1][0], qa[j][1][1], qa[j][1][2], qa[j][1][3], k1.z, k1.w);
         if (EXT) {
-          const uint4 e0 = *reinterpret_cast<const uint4*>(kb + 2 * block_elems + tok0 * HD + 32 * j + 8 * t);
-          const uint4 e1 = *reinterpret_cast<const uint4*>(kb + 2 * block_elems + tok1 * HD + 32 * j + 8 * t);
+          const uint4 e0 = *reinterpret_cast<const uint4*>(&s_kl[EXT ? st : 0][EXT ? tok0 : 0][EXT ? 32 * j + 8 * t : 0]);
+          const uint4 e1 = *reinterpret_cast<const uint4*>(&s_kl[EXT ? st : 0][EXT ? tok1 : 0][EXT ? 32 * j + 8 * t : 0]);
           mma_c<KT>(s0, qa[j][0][0], qa[j][0][1], qa[j][0][2], qa[j][0][3], e0.x, e0.y);
           mma_c<KT>(s0, qa[j][1][0], qa[j][1][1], qa[j][1][2], qa[j][1][3], e0.z, e0.w);
           mma_c<KT>(s1, qa[j][0][0], qa[j][0][1], qa[j][0][2], qa[j][0][3], e1.x, e1.y);
@@ -173,11 +212,11 @@ attn_chunk_kernel(const float* __restrict__ q, PassView p, const KT* __restrict_
       }
 #pragma unroll
       for (int i = 0; i < NT; ++i) {
-        const uint2 vv = *reinterpret_cast<const uint2*>(vb + (size_t)(8 * i + g) * kPageTokens + 4 * t);
+        const uint2 vv = *reinterpret_cast<const uint2*>(&s_v[st][8 * i + g][4 * t]);
         o[i][0] *= ca; o[i][1] *= ca; o[i][2] *= cb; o[i][3] *= cb;
         mma_c<KT>(o[i], a0, a1, a2, a3, vv.x & mlo, vv.y & mhi);
         if (EXT) {
-          const uint2 vl = *reinterpret_cast<const uint2*>(vb + 2 * block_elems + (size_t)(8 * i + g) * kPageTokens + 4 * t);
+          const uint2 vl = *reinterpret_cast<const uint2*>(&s_vl[EXT ? st : 0][EXT ? 8 * i + g : 0][EXT ? 4 * t : 0]);
           mma_c<KT>(o[i], l0p, l1p, l2p, l3p, vv.x & mlo, vv.y & mhi);
           mma_c<KT>(o[i], a0, a1, a2, a3, vl.x & mlo, vl.y & mhi);
         }
