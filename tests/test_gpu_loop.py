@@ -289,3 +289,27 @@ def test_persistent_decode_kernel_against_the_oracle_and_the_separate_kernels(B,
     assert worst <= 2e-3, worst
     print("persistent decode kernel", B, ext, runs["mega"]["stats"], "vs separate kernels", worst,
           "launches", runs["mega"]["launches"], runs["separate"]["launches"])
+
+
+def test_persistent_decode_kernel_phase_timeline():
+    """rsd_debug_mega_profile: with RSD_DEBUG_MEGA_PROFILE the persistent kernel's first CTA stamps the global timer
+    at its start, before and after each of its 7 * layers grid barriers and at its end, in order; without the flag
+    the call is refused."""
+    from paper_2501_19324_b200 import RSD_DEBUG_KEEP_LOGITS, RSD_DEBUG_PERSISTENT_DECODE, RSD_DEBUG_MEGA_PROFILE
+    from paper_2501_19324_b200.binding import RsdError
+    from oracle.rsd_loop import DRAFT, TARGET
+    prompts = ri.prompts(77, 4, 5, 20, MINI[0].vocab)
+    kw = dict(max_step_tokens=3, max_steps=2, max_seq_tokens=48, step_end_id=3, temperature=0.7, seed=2)
+    eng, loop = build_pair(MINI, bf16=True, prompts=prompts, loop_kwargs=kw,
+                           engine_kwargs=dict(debug_flags=RSD_DEBUG_KEEP_LOGITS | RSD_DEBUG_PERSISTENT_DECODE | RSD_DEBUG_MEGA_PROFILE))
+    parity_step(eng, loop, 2.0, **TOL16)                   # delta above the reward range: both models decode
+    for which, shape in ((DRAFT, MINI[0]), (TARGET, MINI[2])):
+        st = eng.mega_profile(which).astype(np.int64)
+        assert len(st) == 14 * shape.n_layers + 2, len(st)
+        assert (np.diff(st) >= 0).all() and st[-1] > st[0]
+        assert st[-1] - st[0] < 50_000_000                 # one launch of a two- or three-layer model: far below 50 ms
+    eng.close()
+    eng, loop = build_pair(MINI, bf16=True, prompts=prompts, loop_kwargs=kw)
+    with pytest.raises(RsdError):
+        eng.mega_profile(DRAFT)
+    eng.close()
