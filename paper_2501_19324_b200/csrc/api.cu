@@ -356,9 +356,9 @@ int gemm_gu(rsd_ctx* c, const ModelHost& M, const void* Wgu, const void* xin, co
   return RSD_OK;
 }
 
-// Up to 128 rows the fused kernel wins (one kernel and the fp32 gate/up array less); in the dense passes a CTA
-// computes one large tile and cannot hide the heavier epilogue (measured at 4096 rows: 586 us against 367 + 64 us),
-// so those keep the plain GEMM + SwiGLU kernel.
+// Up to 128 rows the one-tile-per-CTA fused kernel wins (one kernel and the fp32 gate/up array less); with more rows
+// a CTA of that kernel cannot hide the heavier epilogue (measured at 4096 rows: 586 us against 367 + 64 us): there
+// the caller takes the persistent kernel when it can (no idle flag), else the plain GEMM + SwiGLU kernel.
 bool gu_fused_ok(const ModelHost& M, int rows) {
   return rows <= 128 && M.m.dtype == RSD_BF16 && M.split && gemm_gu_supported(1, rows, M.m.d_ffn, M.m.d_model);
 }
@@ -396,7 +396,9 @@ int forward_pass(rsd_ctx* c, int which, PassView p, cudaStream_t s) {
     rc = gemm(c, M, M.wo[l], c->attn, attn_lo, c->x, T, d, H * hd, 1, p.n_active, defer_small ? &x_pending : nullptr, s);
     if (rc) return rc;
     CU(launch_rmsnorm(m.dtype, c->x, M.norm2[l], c->h, h_lo, T, d, m.rms_eps, nullptr, p.n_active, x_pending, s));
-    if (gu_fused_ok(M, T)) {
+    // up to 128 rows: fused kernel; dense passes (no idle flag): the persistent kernel hides the SwiGLU epilogue
+    // under the next tile's MMAs
+    if (gu_fused_ok(M, T) || (T > 128 && p.n_active == nullptr && gu_fused_ok(M, 128))) {
       rc = gemm_gu(c, M, M.wgu[l], c->h, h_lo, c->act, act_lo, T, F, d, p.n_active, s);
       if (rc) return rc;
     } else {

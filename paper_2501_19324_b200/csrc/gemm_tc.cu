@@ -324,6 +324,205 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
   }
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// Persistent form of the kernel above for the dense regime (more than 128 rows of x, split-precision operand, no
+// K split): a CTA per SM walks the output tiles (128 weight rows x 128 x rows, the same grouped order), the TMA
+// ring runs on from tile to tile, and the accumulator alternates between the two halves of tensor memory, so
+// the epilogue of one tile (TMEM -> registers -> global) overlaps the MMAs of the next instead of ending the CTA.
+// GU: gate/up tiles with the SwiGLU epilogue as above; the exchange buffers get shared memory of their own, since
+// the ring is busy with the next tile.
+// ---------------------------------------------------------------------------------------------------------
+struct PersistCfg {
+  static constexpr int kMT = 256, kRows = 128, kStages = 4;
+  static constexpr int kABytes = kTileN * kTileK * 2, kBBytes = kMT * kTileK * 2, kStageBytes = kABytes + kBBytes;
+  static constexpr int kHalf = kRows / 2, kLd = kHalf + 1;
+  static constexpr size_t kXchBytes = 2 * 64 * (size_t)kLd * 4;
+  static constexpr size_t smem(bool gu) { return 1024 + (size_t)kStages * kStageBytes + 256 + (gu ? kXchBytes : 0); }
+  static constexpr uint32_t kIdesc = TcCfg<256>::kIdesc;
+};
+
+template <bool GU>
+__global__ void __launch_bounds__(192, 1)
+gemm_tc_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x,
+                          const __grid_constant__ CUtensorMap tm_x_lo, float* __restrict__ Y, int M, int N, int K,
+                          int accumulate, int n_tiles_n, int n_tiles_m, int* __restrict__ err,
+                          __nv_bfloat16* __restrict__ act_hi, __nv_bfloat16* __restrict__ act_lo) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  using C = PersistCfg;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  uint64_t* full = (uint64_t*)(smem + (size_t)C::kStages * C::kStageBytes);
+  uint64_t* empty = full + C::kStages;
+  uint64_t* acc_full = empty + C::kStages;
+  uint64_t* acc_empty = acc_full + 2;
+  uint32_t* tmem_slot = (uint32_t*)(acc_empty + 2);
+  volatile uint32_t* stop = tmem_slot + 1;
+  float* xch = (float*)(smem + (size_t)C::kStages * C::kStageBytes + 256);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int total_kb = (K + kTileK - 1) / kTileK, n_tiles = n_tiles_n * n_tiles_m;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < C::kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 4); }
+    *stop = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 5) tmem_alloc(tmem_slot, 512);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  // tile t -> (row tile of x, tile of W): groups of eight row tiles, row tile fastest
+  auto tile_of = [&](int t, int& tm, int& tn) {
+    const int per_group = 8 * n_tiles_n, g0 = (t / per_group) * 8, rem = t % per_group, gsz = min(8, n_tiles_m - g0);
+    tm = g0 + rem % gsz;
+    tn = rem / gsz;
+  };
+  auto fail = [&]() { if (*stop == 0) { if (err) atomicCAS(err, 0, -5); *stop = 1; } };
+
+  if (warp == 4) {
+    if (lane == 0) {
+      uint32_t it = 0;
+      for (int t = blockIdx.x; t < n_tiles && !*stop; t += gridDim.x) {
+        int tm, tn;
+        tile_of(t, tm, tn);
+        const int n0 = tn * (GU ? kTileN / 2 : kTileN), m0 = tm * C::kRows;
+        for (int kb = 0; kb < total_kb; ++kb, ++it) {
+          const uint32_t s = it % C::kStages;
+          if (!mbar_wait(&empty[s], ((it / C::kStages) & 1u) ^ 1u) || *stop) { fail(); break; }
+          uint8_t* a = smem + (size_t)s * C::kStageBytes;
+          mbar_expect_tx(&full[s], C::kStageBytes);
+          if (GU) {
+            tma_load_2d(a, &tm_w, &full[s], kb * kTileK, n0);
+            tma_load_2d(a + C::kABytes / 2, &tm_w, &full[s], kb * kTileK, N + n0);
+          } else {
+            tma_load_2d(a, &tm_w, &full[s], kb * kTileK, n0);
+          }
+          tma_load_2d(a + C::kABytes, &tm_x, &full[s], kb * kTileK, m0);
+          tma_load_2d(a + C::kABytes + C::kRows * kTileK * 2, &tm_x_lo, &full[s], kb * kTileK, m0);
+        }
+      }
+      if (*stop) {   // copies in flight must land before the CTA goes away
+        for (uint32_t i = (it > (uint32_t)C::kStages ? it - C::kStages : 0); i < it; ++i)
+          for (uint32_t k = 0; k < (1u << 16); ++k)
+            if (mbar_try_wait(&full[i % C::kStages], (i / C::kStages) & 1u)) break;
+      }
+    }
+  } else if (warp == 5) {
+    if (lane == 0) {
+      uint32_t it = 0, n_acc = 0;
+      for (int t = blockIdx.x; t < n_tiles && !*stop; t += gridDim.x, ++n_acc) {
+        const uint32_t b = n_acc & 1u;
+        if (!mbar_wait(&acc_empty[b], ((n_acc >> 1) & 1u) ^ 1u) || *stop) { fail(); break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + b * (uint32_t)C::kMT;
+        bool ok = true;
+        for (int kb = 0; kb < total_kb; ++kb, ++it) {
+          const uint32_t s = it % C::kStages;
+          if (!mbar_wait(&full[s], (it / C::kStages) & 1u) || *stop) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t a = smem_u32(smem + (size_t)s * C::kStageBytes), bb = a + C::kABytes;
+#pragma unroll
+          for (int k = 0; k < kTileK / kUmmaK; ++k)
+            umma_bf16(d_tmem, smem_desc_sw128(a + k * kUmmaK * 2), smem_desc_sw128(bb + k * kUmmaK * 2), C::kIdesc,
+                      (kb > 0 || k > 0) ? 1u : 0u);
+          umma_commit(&empty[s]);
+        }
+        if (!ok) { fail(); break; }
+        umma_commit(&acc_full[b]);
+      }
+    }
+  } else {
+    // ---------------- epilogue warps ----------------
+    uint32_t n_acc = 0;
+    for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++n_acc) {
+      int tm, tn;
+      tile_of(t, tm, tn);
+      const int n0 = tn * (GU ? kTileN / 2 : kTileN), m0 = tm * C::kRows;
+      const uint32_t b = n_acc & 1u;
+      bool ok = mbar_try_wait(&acc_full[b], (n_acc >> 1) & 1u);
+      for (uint32_t i = 0; i < (1u << 21) && !ok && !*stop; ++i) ok = mbar_try_wait_sleep(&acc_full[b], (n_acc >> 1) & 1u, 1000);
+      if (!ok) fail();
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + b * (uint32_t)C::kMT;
+      const int m_valid = min(C::kRows, M - m0);
+      if (!GU) {
+        const int n = n0 + warp * 32 + lane;
+        if (ok) {
+          for (int c = 0; c < m_valid; c += 16) {
+            float v[16], w[16];
+            tmem_ld16(taddr + c, v);
+            tmem_ld16(taddr + C::kRows + c, w);
+            if (n < N) {
+#pragma unroll
+              for (int j = 0; j < 16; ++j) {
+                if (c + j < m_valid) {
+                  float* y = Y + (size_t)(m0 + c + j) * N + n;
+                  const float r = v[j] + w[j];
+                  *y = accumulate ? (*y + r) : r;
+                }
+              }
+            }
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&acc_empty[b]);
+      } else {
+        const bool is_gate = warp < 2;
+        const int l = (warp & 1) * 32 + lane;
+        float* send = xch + (is_gate ? 64 * C::kLd : 0) + l * C::kLd;
+        const float* recv = xch + (is_gate ? 0 : 64 * C::kLd) + l * C::kLd;
+        const int send0 = is_gate ? C::kHalf : 0, own0 = is_gate ? 0 : C::kHalf;
+        if (ok) {
+#pragma unroll 1
+          for (int c = 0; c < C::kHalf; c += 16) {
+            float v[16], w[16];
+            tmem_ld16(taddr + send0 + c, v);
+            tmem_ld16(taddr + C::kRows + send0 + c, w);
+#pragma unroll
+            for (int j = 0; j < 16; ++j) send[c + j] = v[j] + w[j];
+          }
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (ok && n0 + l < N) {
+#pragma unroll 1
+          for (int c = 0; c < C::kHalf; c += 16) {
+            if (own0 + c >= m_valid) break;
+            float v[16], w[16];
+            tmem_ld16(taddr + own0 + c, v);
+            tmem_ld16(taddr + C::kRows + own0 + c, w);
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const int r = own0 + c + j;
+              if (r < m_valid) {
+                const float mine = v[j] + w[j], other = recv[c + j];
+                const float gate = is_gate ? mine : other, up = is_gate ? other : mine;
+                const float a = gate / (1.f + expf(-gate)) * up;
+                const size_t o = (size_t)(m0 + r) * N + n0 + l;
+                const __nv_bfloat16 h = __float2bfloat16_rn(a);
+                act_hi[o] = h;
+                act_lo[o] = __float2bfloat16_rn(a - __bfloat162float(h));
+              }
+            }
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&acc_empty[b]);
+        asm volatile("bar.sync 1, 128;" ::: "memory");   // the exchange buffers are free for the next tile
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 5) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
 // y[m, n] (+)= sum over splits of partials[s][m][n], splits added in order; 4 columns per thread.
 __global__ void __launch_bounds__(256)
 splitk_reduce_kernel(const float* __restrict__ partials, float* __restrict__ Y, int M, int N, int splits, int accumulate,
@@ -475,6 +674,36 @@ bool gemm_tc_supported(int dtype, int M, int N, int K) {
   return dtype == 1 && M >= 1 && N >= 1 && K >= 8 && K % 8 == 0;
 }
 
+static int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) n = 0;
+  }
+  return n;
+}
+
+// Dense regime (M > 128 rows, split-precision operand, no K split, no row scale, no idle flag): persistent kernel.
+template <bool GU>
+static cudaError_t launch_persistent(const CUtensorMap& tw, const CUtensorMap& tx, const CUtensorMap& txl, float* y, int M, int N,
+                                     int K, int accumulate, int* err, __nv_bfloat16* act_hi, __nv_bfloat16* act_lo, cudaStream_t s) {
+  constexpr size_t smem = PersistCfg::smem(GU);
+  static_assert(PersistCfg::smem(true) <= 227 * 1024, "shared memory of one CTA");
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_tc_persistent_kernel<GU>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  const int n_sm = sm_count();
+  if (n_sm <= 0) return cudaErrorInvalidDevice;
+  const int tiles_n = GU ? N / 64 : (N + kTileN - 1) / kTileN, tiles_m = (M + PersistCfg::kRows - 1) / PersistCfg::kRows;
+  const int grid = std::min(tiles_n * tiles_m, n_sm);
+  RSD_LAUNCH((gemm_tc_persistent_kernel<GU>), grid, 192, smem, s, tw, tx, txl, y, M, N, K, accumulate, tiles_n, tiles_m, err,
+             act_hi, act_lo);
+  return launched(1);
+}
+
 template <int MT, bool DEEP>
 static cudaError_t launch_gu_mt(const CUtensorMap& tw, const CUtensorMap& tx, const CUtensorMap& txl, int M, int F, int K, int rows,
                                 int* err, const int32_t* n_active, RowScale rs, __nv_bfloat16* act_hi, __nv_bfloat16* act_lo,
@@ -511,6 +740,8 @@ cudaError_t launch_gemm_gu(const void* Wgu, const void* x, const void* x_lo, voi
   if (!get_map(Wgu, 2 * F, K, kTileN / 2, &tw) || !get_map(x, M, K, rows, &tx) || !get_map(x_lo, M, K, rows, &txl))
     return cudaErrorNotSupported;
   int* err = (int*)((char*)scratch + kCounterBytes);
+  if (M > 128 && rs.ssq == nullptr && n_active == nullptr)
+    return launch_persistent<true>(tw, tx, txl, nullptr, M, F, K, 0, err, (__nv_bfloat16*)act_hi, (__nv_bfloat16*)act_lo, s);
   auto* hi = (__nv_bfloat16*)act_hi;
   auto* lo = (__nv_bfloat16*)act_lo;
   // fewer than ~1.5 CTAs per SM: one CTA per SM with a deep ring streams faster than a thin second wave
@@ -556,6 +787,8 @@ cudaError_t launch_gemm_tc(const void* W, const void* x, const void* x_lo, float
   else txl = tx;
   int* err = (int*)((char*)scratch + kCounterBytes);
   float* partials = (float*)((char*)scratch + kCounterBytes + 256);
+  if (split_operand && M > 128 && p.splits == 1 && rs.ssq == nullptr && n_active == nullptr)
+    return launch_persistent<false>(tw, tx, txl, y, M, N, K, accumulate, err, nullptr, nullptr, s);
 #define RSD_TC(MT, SP) return launch_mt<MT, SP>(tw, tx, txl, y, M, N, K, accumulate, p, partials, err, n_active, defer, rs, s)
   if (split_operand) {
     switch (p.mt) {
