@@ -61,10 +61,11 @@ def test_gemm_simt(M, N, K, bf16):
 
 @pytest.mark.parametrize("M,N,K", [(16, 128, 64), (5, 256, 512), (17, 1536, 1536), (32, 2048, 1536), (33, 1000, 520),
                                    (64, 1536, 8960), (100, 384, 1408), (128, 640, 768), (129, 256, 2048),
-                                   (300, 4096, 512), (1000, 1280, 768), (8, 17920, 1536)])
+                                   (300, 4096, 512), (1000, 1280, 768), (8, 17920, 1536), (200, 384, 520), (2500, 1024, 192)])
 def test_gemm_tcgen05(M, N, K):
     """Tensor-core path: ragged M, N not a multiple of the 128-row tile, K not a multiple of 64,
-    split-K with the last-arriver reduction, several x tiles, accumulate into y."""
+    split-K with the last-arriver reduction, several x tiles (more than 128 rows with a split operand take the
+    persistent kernel: several tiles per CTA, more row tiles than one group of eight), accumulate into y."""
     rng = np.random.default_rng(M * 7 + N)
     W = ri.cpu_tensor(2, 5, N, K, True)
     x = rng.normal(size=(M, K)).astype(np.float32)
@@ -298,7 +299,7 @@ def test_extended_precision_attention(hd, H, KV):
 
 
 @pytest.mark.parametrize("M,F,K", [(1, 64, 64), (5, 192, 512), (32, 1408, 512), (33, 128, 520), (70, 2048, 768),
-                                   (129, 704, 1408), (300, 320, 256), (32, 8960, 1536)])
+                                   (129, 704, 1408), (300, 320, 256), (32, 8960, 1536), (200, 128, 520), (2100, 640, 128)])
 def test_gate_up_gemm_with_swiglu_epilogue(M, F, K):
     """Gate/up projection with SwiGLU inside the GEMM epilogue (tile = 64 gate rows + the 64 matching up rows):
     against matmul + silu(g) * u written out in fp64.  Ragged M (all three tile heights and several x tiles), F of
