@@ -575,7 +575,7 @@ int decode_iteration(rsd_ctx* c, int which, int phase, int n_slots, cudaStream_t
 
 // Captures one decode iteration of `which` over all B slots into a graph (idle slots are skipped
 // inside the kernels), so that a token costs one graph launch instead of some 300 kernel launches.
-int ensure_decode_graph(rsd_ctx* c, int which, int phase, int g) {
+int ensure_decode_graph(rsd_ctx* c, int which, int phase, int g, int n_slots) {
   const int B = c->st.B;
   if (c->dec_graph[g] && c->dec_graph_B[g] == B) return RSD_OK;
   if (c->dec_graph[g]) { cudaGraphExecDestroy(c->dec_graph[g]); c->dec_graph[g] = nullptr; }
@@ -584,7 +584,7 @@ int ensure_decode_graph(rsd_ctx* c, int which, int phase, int g) {
   CU(cudaStreamBeginCapture(c->cap_stream, cudaStreamCaptureModeThreadLocal));
   const bool was_in_decode = c->in_decode, was_timed = c->time_this_iter;
   c->in_decode = true; c->time_this_iter = false;          // no event records inside the capture
-  const int rc = decode_iteration(c, which, phase, B, c->cap_stream);
+  const int rc = decode_iteration(c, which, phase, n_slots, c->cap_stream);
   c->in_decode = was_in_decode; c->time_this_iter = was_timed;
   cudaGraph_t graph = nullptr;
   cudaError_t e = cudaStreamEndCapture(c->cap_stream, &graph);
@@ -610,7 +610,10 @@ int decode_phase(rsd_ctx* c, int which, int phase, int n_slots, cudaStream_t s) 
   while (bucket < 3 && n_slots * 2 <= rows_eff) { rows_eff = (rows_eff + 1) / 2; ++bucket; }
   c->attn_rows_hint = rows_eff;
   const int g = phase * 4 + bucket;
-  if (graphs || c->mega_B[which] == c->st.B) n_slots = c->st.B;   // fixed shape: slots beyond the phase's rows are idle
+  // fixed shape per bucket: the rows of the phase sit in the first slots, so the iteration runs over the bucket's
+  // slot count (the persistent kernel is built for all B slots); slots beyond the phase's rows are idle
+  if (c->mega_B[which] == c->st.B) n_slots = c->st.B;
+  else if (graphs) n_slots = rows_eff;
   c->in_decode = true;
   int rc = RSD_OK;
   for (int j = 0; j < c->C && rc == RSD_OK; ++j) {
@@ -619,7 +622,7 @@ int decode_phase(rsd_ctx* c, int which, int phase, int n_slots, cudaStream_t s) 
     // the iteration is captured once and replayed
     const bool have_graph = graphs && c->dec_graph[g] && c->dec_graph_B[g] == c->st.B;
     if (graphs && !have_graph && j > 0) {
-      rc = ensure_decode_graph(c, which, phase, g);
+      rc = ensure_decode_graph(c, which, phase, g, n_slots);
       if (rc) break;
     }
     if (graphs && !timed_iter && c->dec_graph[g] && c->dec_graph_B[g] == c->st.B) {
