@@ -196,10 +196,22 @@ def run_reference(args, rank: int):
 
 
 def kv_extended(args) -> int:
-    """The 72B-shape target keeps its logits within 3e-2 of the fp64 definition only with the
-    hi + lo KV cache, so that workload runs with it unless told otherwise."""
+    """rsd_config.kv_extended: 0 lets the library decide per model by depth (the 80-layer target of cfg4 gets
+    the hi + lo KV cache that keeps its logits within 3e-2 of the fp64 definition), 1 forces the pairs, 2 the
+    plain fp16 cache."""
     v = getattr(args, "kv_extended", None)
-    return int(v) if v is not None else int(args.workload == "cfg4")
+    return int(v) if v is not None else 0
+
+
+def kv_cache_label(args) -> str:
+    setting = kv_extended(args)
+    names = WORKLOADS[args.workload][:3]
+    ext = [setting == 1 or (setting == 0 and ri.SHAPES[n].n_layers > 48) for n in names]
+    if all(ext):
+        return "fp16 hi+lo pairs"
+    if not any(ext):
+        return "fp16"
+    return "fp16; fp16 hi+lo pairs for " + ", ".join(r for r, e in zip(("draft", "PRM", "target"), ext) if e)
 
 
 def workload_config(args) -> dict:
@@ -208,7 +220,7 @@ def workload_config(args) -> dict:
                         f"step <= {cap} tokens, Gumbel-max T=0.7, "
                         + (f"delta {args.delta}" if getattr(args, "delta", None) is not None else "delta at the 70% accept quantile"),
             "batch": B, "max_step_tokens": args.cap or cap, "replicas": args.gpus,
-            "kv_cache": "fp16 hi+lo pairs" if kv_extended(args) else "fp16",
+            "kv_cache": kv_cache_label(args),
             "prm": "head on the draft's trunk (prm_shares_draft)" if getattr(args, "merged_prm", False) else "separate model",
             "schedule": "lock-step rsd_step" if getattr(args, "queue", 1) == 1 else
                         f"rsd_step_queued, target pass once {args.queue} rows wait",
@@ -594,8 +606,8 @@ def main():
                     help="record and print the phase timeline of the persistent decode kernel's last launches")
     ap.add_argument("--queue", type=int, default=1,
                     help="min_target_rows of rsd_step_queued (1 = rsd_step, the headline configuration)")
-    ap.add_argument("--kv-extended", type=int, default=None, choices=[0, 1], dest="kv_extended",
-                    help="KV cache as fp16 hi+lo pairs (default: on for cfg4 only)")
+    ap.add_argument("--kv-extended", type=int, default=None, choices=[0, 1, 2], dest="kv_extended",
+                    help="KV cache: 0 by model depth (default: hi+lo pairs beyond 48 layers), 1 fp16 hi+lo pairs, 2 plain fp16")
     ap.add_argument("--only", default="", help="with --sweep gemm: a single M,K,N point, plain launches")
     ap.add_argument("--sweep", default="", choices=["", "gemm", "attn", "gate", "score"],
                     help="kernel sweep on config-2 shapes instead of the step-loop benchmark")

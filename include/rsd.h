@@ -37,7 +37,8 @@ enum {
   RSD_OK = 0,
   RSD_ERR_ARG = -1,         /* bad argument / inconsistent shapes                         */
   RSD_ERR_STATE = -2,       /* call out of order (e.g. step before prefill)               */
-  RSD_ERR_OOM_PAGES = -3,   /* a KV page pool or the workspace is too small               */
+  RSD_ERR_OOM_PAGES = -3,   /* a KV page pool or the workspace is too small; the rows' state is
+                               unchanged, but only rsd_prefill / rsd_reset are valid afterwards */
   RSD_ERR_CUDA = -4,        /* a CUDA call failed; only rsd_destroy is valid afterwards   */
   RSD_ERR_TIMEOUT = -5,     /* a bounded device-side wait expired                         */
   RSD_ERR_UNSUPPORTED = -6  /* shape or option the kernels do not cover                   */
@@ -91,11 +92,13 @@ typedef struct {
   float omega_alpha;          /* alpha of RSD_OMEGA_LOGISTIC                                 */
   int32_t max_chunk_tokens;   /* tokens pushed through a model per multi-token pass; 0 = 4096 */
   int32_t debug_flags;        /* RSD_DEBUG_*                                                 */
-  int32_t kv_extended;        /* bf16 models only.  0: fp16 keys and values, fp16 queries and softmax
-                                 weights in the attention products.  1: keys and values are cached as
-                                 fp16 hi + lo pairs (twice the KV bytes) and queries / softmax weights
-                                 enter as hi + lo pairs (attention accurate to ~2^-20); for deep models
-                                 whose logits must stay within 3e-2 of an fp64 reference               */
+  int32_t kv_extended;        /* bf16 models only; per model.  1: keys and values are cached as fp16 hi + lo
+                                 pairs (twice the KV bytes) and queries / softmax weights enter the attention
+                                 products as hi + lo pairs (attention accurate to ~2^-20).  2: plain fp16 keys
+                                 and values, fp16 queries and softmax weights.  0 (default): by depth -- plain
+                                 fp16 for models of up to 48 layers, the pairs for deeper ones, whose logits
+                                 would otherwise leave the 3e-2 band around an exact reference (measured at 80
+                                 layers: 5.7e-2 with the plain cache, 1.7e-3 with the pairs)                  */
   int32_t prm_shares_draft;   /* 1: merged serving (Appendix B.3: the PRM is a projection layer on a language
                                  model's final layer; Section 4 on merging PRM and policy): the PRM is its
                                  final_norm and scalar head on the DRAFT's trunk.  r_i is read after one
@@ -133,7 +136,9 @@ int rsd_create(const rsd_config* cfg, rsd_ctx** out);
 /* rsd_load_models(draft, prm, target): records the three borrowed weight sets, validates shapes
  * (GQA divisibility, head_dim 64 or 128, K dimensions a multiple of the vector width) and lays
  * out the workspace.  Sampling is restricted to ids below the smallest of the three vocabularies
- * so every token is valid for every embedding.                                               */
+ * so every token is valid for every embedding.  Once per context: a second successful load is
+ * refused with RSD_ERR_STATE (the captured decode graphs keep the first models' pointers); use a
+ * new context for other models.                                                              */
 int rsd_load_models(rsd_ctx*, const rsd_model* draft, const rsd_model* prm, const rsd_model* target);
 
 /* rsd_prefill(prompts): starts B rows from ragged prompts (z_1 = x).  `tokens` is a HOST array of
@@ -285,7 +290,8 @@ int rsd_k_gate_compact(const float* rewards, const uint8_t* live, float delta, u
 #define RSD_GATE_STATIC_MAX_ROWS (1 << 20)
 int rsd_k_gate_compact_static(const float* rewards, const uint8_t* live, float delta, uint8_t* accept,
                               int32_t* rej_idx, int32_t* n_rej, int32_t B, void* cuda_stream);
-const char* rsd_k_gate_compact_static_error(void); /* library-owned text of its last failure      */
+const char* rsd_k_gate_compact_static_error(void); /* text of its last failure (any thread's), copied for
+                                                      the calling thread: valid until that thread's next call */
 
 /* out[t, :] = x[t, :] * gain / sqrt(mean(x^2) + eps), x fp32 [T, d], out of element type `dtype`. */
 int rsd_k_rmsnorm(const float* x, const void* gain, void* out, int32_t T, int32_t d, float eps,

@@ -143,9 +143,17 @@ double count_params(const rsd_model& m) {
   return (double)m.vocab * d + m.n_layers * per_layer + d + head;
 }
 
+// Whether model m caches keys and values as fp16 hi + lo pairs.  Setting 0 decides by depth: the rounding of
+// 16-bit keys and values grows with the number of layers, and beyond 48 layers the logits of a bf16 model
+// leave the 3e-2 band around an exact reference (80 layers: 5.7e-2), so deep models get the pairs.
+bool kv_extended_for(const rsd_model& m, int setting) {
+  if (m.dtype != RSD_BF16) return false;
+  return setting == 1 || (setting == 0 && m.n_layers > 48);
+}
+
 size_t kv_pool_bytes(const rsd_model& m, int pages, int kv_extended) {
   const size_t elem = m.dtype == RSD_BF16 ? 2 : 4;
-  const size_t blocks = (m.dtype == RSD_BF16 && kv_extended) ? 4 : 2;   // keys, values (, their low halves)
+  const size_t blocks = kv_extended_for(m, kv_extended) ? 4 : 2;   // keys, values (, their low halves)
   return (size_t)pages * m.n_layers * blocks * m.n_kv_heads * kPageTokens * m.head_dim * elem;
 }
 
@@ -280,6 +288,7 @@ int check_config(const rsd_config* cfg, const char** why) {
   if (cfg->temperature < 0.f) { *why = "temperature"; return RSD_ERR_ARG; }
   if (cfg->omega_kind < 0 || cfg->omega_kind > 4) { *why = "omega_kind"; return RSD_ERR_ARG; }
   if (cfg->step_end_mod < 0) { *why = "step_end_mod"; return RSD_ERR_ARG; }
+  if (cfg->kv_extended < 0 || cfg->kv_extended > 2) { *why = "kv_extended out of 0..2"; return RSD_ERR_ARG; }
   return RSD_OK;
 }
 
@@ -722,6 +731,8 @@ int rsd_create(const rsd_config* cfg, rsd_ctx** out) {
 int rsd_load_models(rsd_ctx* c, const rsd_model* draft, const rsd_model* prm, const rsd_model* target) {
   if (!c) return RSD_ERR_ARG;
   if (c->poisoned) return fail(c, RSD_ERR_STATE, "context unusable after a CUDA error%s");
+  // captured decode graphs, parameter blocks and tensor maps hold the first models' pointers and shapes
+  if (c->loaded) return fail(c, RSD_ERR_STATE, "models are loaded once per context: create a new context for other models%s");
   const rsd_model* ms[3] = {draft, prm, target};
   const char* why;
   for (int i = 0; i < 3; ++i) {
@@ -760,7 +771,7 @@ int rsd_load_models(rsd_ctx* c, const rsd_model* draft, const rsd_model* prm, co
     M.m.wqkv = M.wqkv.data(); M.m.wo = M.wo.data(); M.m.wgu = M.wgu.data(); M.m.wdown = M.wdown.data();
     M.m.norm1 = M.norm1.data(); M.m.norm2 = M.norm2.data();
     M.elem = M.m.dtype == RSD_BF16 ? 2 : 4;
-    M.kv_dtype = M.m.dtype == RSD_BF16 ? (c->cfg.kv_extended ? 3 : 2) : 0;
+    M.kv_dtype = M.m.dtype == RSD_BF16 ? (kv_extended_for(M.m, c->cfg.kv_extended) ? 3 : 2) : 0;
     // hi + lo operands for every bf16 model: with plain bf16 operands a 7B-shape PRM misses the
     // 1e-2 reward bound (1.1e-2 measured), a 1.5B-shape one would pass (1.5e-3)
     M.split = M.m.dtype == RSD_BF16;

@@ -84,17 +84,20 @@ __global__ void __launch_bounds__(1024) build_pass_kernel(RowState st, int which
   int total;
   const int off = block_exclusive_scan(cnt, scan, &total);
   if (b < kMaxBatch) { s_off[b] = off; s_start[b] = start; }
+  if (total > st.pass_capacity) {
+    // the list does not fit: raise the error and leave cursors and the list as they were
+    if (b == 0) { st.n_tok[0] = 0; st.err[0] = -3; }
+    return;
+  }
   if (b == 0) {
     s_off[kMaxBatch] = total;
     st.n_tok[0] = total;
-    if (total > st.pass_capacity) st.err[0] = -3;
   }
   if (b < st.B) {
     st.last_idx[b] = cnt > 0 ? off + cnt - 1 : -1;
     st.kv_len[which][b] = start + cnt;
   }
   __syncthreads();
-  if (total > st.pass_capacity) return;
   for (int t = threadIdx.x; t < total; t += blockDim.x) {
     // largest row with s_off[row] <= t (rows with no tokens share an offset with their successor)
     int lo = 0, hi = st.B - 1;

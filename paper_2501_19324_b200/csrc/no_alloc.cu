@@ -31,7 +31,14 @@ std::string g_error;
 
 extern "C" {
 
-const char* rsd_k_gate_compact_static_error(void) { return g_error.c_str(); }
+// The text is copied under the lock into a buffer of the calling thread, so a failing call on another host
+// thread cannot reallocate it under the reader; it stays valid until this thread asks again.
+const char* rsd_k_gate_compact_static_error(void) {
+  thread_local std::string copy;
+  std::lock_guard<std::mutex> lock(g_mutex);
+  copy = g_error;
+  return copy.c_str();
+}
 
 int rsd_k_gate_compact_static(const float* rewards, const uint8_t* live, float delta, uint8_t* accept,
                               int32_t* rej_idx, int32_t* n_rej, int32_t B, void* cuda_stream) {

@@ -25,6 +25,8 @@ SIGMA = 0.02
 WEIGHT_SCALE = float(np.float32(SIGMA / (2.0 * math.sqrt(8.0 * (65536.0 ** 2 - 1.0) / 12.0))))
 
 KIND_EMBED, KIND_HEAD, KIND_WQ, KIND_WK, KIND_WV, KIND_WO, KIND_WGATE, KIND_WUP, KIND_WDOWN = range(9)
+KIND_NORM1, KIND_NORM2, KIND_FINAL_NORM = 9, 10, 11
+GAIN_SPREAD = 5.0   # RMSNorm gains = 1 + GAIN_SPREAD * (a weight-recipe draw of sigma 0.02): 1 +- 0.1
 SLOT_DRAFT, SLOT_PRM, SLOT_TARGET = 0, 1, 2
 HEAD_LM, HEAD_REWARD_SIGMOID, HEAD_REWARD_RAW = 0, 1, 2
 
@@ -140,6 +142,24 @@ def cpu_tensor(seed: int, tid: int, rows: int, cols: int, bf16: bool, first_row:
     return out
 
 
+def _round_bf16(a: np.ndarray) -> np.ndarray:
+    """fp32 array rounded to the nearest bfloat16 (ties to even), returned as fp32."""
+    u = np.ascontiguousarray(a, dtype=np.float32).view(np.uint32)
+    r = ((u >> np.uint32(16)) & np.uint32(1)) + np.uint32(0x7FFF)
+    return (((u + r) >> np.uint32(16)) << np.uint32(16)).view(np.float32)
+
+
+def cpu_gain(seed: int, tid: int, d: int, bf16: bool) -> np.ndarray:
+    """RMSNorm gain vector [d]: 1 + GAIN_SPREAD * draw (about 1 +- 0.1, never near zero: the draw is
+    bounded by 4.9 sigma), a distinct tensor id per norm, so that a gain taken from the wrong layer, a
+    skipped norm or a gain applied twice changes the result.  Computed on the host in fp32 (one multiply,
+    one add, each rounded once) and, for 16-bit models, rounded to bfloat16; the GPU copy is an upload of
+    these very values."""
+    draw = cpu_tensor(seed, tid, 1, d, False)[0]
+    g = (np.float32(1.0) + np.float32(GAIN_SPREAD) * draw).astype(np.float32)
+    return _round_bf16(g) if bf16 else g
+
+
 def layer_tensor_dims(shape: ModelShape) -> dict:
     d, hd = shape.d_model, shape.head_dim
     return {
@@ -150,13 +170,14 @@ def layer_tensor_dims(shape: ModelShape) -> dict:
 
 
 def cpu_layer_weights(shape: ModelShape, slot: int, layer: int, seed: int, bf16: bool) -> dict:
-    """Un-fused weight matrices of one layer (fp32 host arrays; RMSNorm gains are 1)."""
+    """Un-fused weight matrices of one layer and its two RMSNorm gain vectors (fp32 host arrays)."""
     dims = layer_tensor_dims(shape)
     w = {k: cpu_tensor(seed, tensor_id(slot, layer, k), r, c, bf16) for k, (r, c) in dims.items()}
     return {
         "wq": w[KIND_WQ], "wk": w[KIND_WK], "wv": w[KIND_WV], "wo": w[KIND_WO],
         "wgate": w[KIND_WGATE], "wup": w[KIND_WUP], "wdown": w[KIND_WDOWN],
-        "norm1": np.ones(shape.d_model, dtype=np.float32), "norm2": np.ones(shape.d_model, dtype=np.float32),
+        "norm1": cpu_gain(seed, tensor_id(slot, layer, KIND_NORM1), shape.d_model, bf16),
+        "norm2": cpu_gain(seed, tensor_id(slot, layer, KIND_NORM2), shape.d_model, bf16),
     }
 
 
@@ -168,7 +189,7 @@ def cpu_model_weights(shape: ModelShape, slot: int, seed: int, bf16: bool, head_
     out = {
         "shape": shape, "head_kind": head_kind,
         "tok_embed": cpu_tensor(seed, tensor_id(slot, 0, KIND_EMBED), shape.vocab, d, bf16),
-        "final_norm": np.ones(d, dtype=np.float32),
+        "final_norm": cpu_gain(seed, tensor_id(slot, 0, KIND_FINAL_NORM), d, bf16),
         "head": cpu_tensor(seed, tensor_id(slot, 0, KIND_HEAD), head_rows, d, bf16),
         "layers": [],
     }
@@ -192,11 +213,12 @@ def gpu_model_tensors(shape: ModelShape, slot: int, seed: int, bf16: bool, head_
                                         WEIGHT_SCALE, stream)
         assert rc == 0, f"fill kernel launch failed: {rc}"
 
-    def ones(n):
-        return torch.ones(n, dtype=dt, device="cuda")
+    def gain(layer, kind):
+        # the host's values, uploaded: bf16 values are exact in fp32, so the cast back is exact
+        return torch.from_numpy(cpu_gain(seed, tensor_id(slot, layer, kind), shape.d_model, bf16)).to(dt).cuda()
 
     d, hd, H, KV, F = shape.d_model, shape.head_dim, shape.n_heads, shape.n_kv_heads, shape.d_ffn
-    out = {"tok_embed": torch.empty(shape.vocab, d, dtype=dt, device="cuda"), "final_norm": ones(d),
+    out = {"tok_embed": torch.empty(shape.vocab, d, dtype=dt, device="cuda"), "final_norm": gain(0, KIND_FINAL_NORM),
            "wqkv": [], "wo": [], "wgu": [], "wdown": [], "norm1": [], "norm2": []}
     fill(out["tok_embed"], 0, shape.vocab, d, tensor_id(slot, 0, KIND_EMBED))
     head_rows = shape.vocab if head_kind == HEAD_LM else 1
@@ -215,7 +237,7 @@ def gpu_model_tensors(shape: ModelShape, slot: int, seed: int, bf16: bool, head_
         wdown = torch.empty(d, F, dtype=dt, device="cuda")
         fill(wdown, 0, d, F, tensor_id(slot, l, KIND_WDOWN))
         out["wqkv"].append(wqkv); out["wo"].append(wo); out["wgu"].append(wgu); out["wdown"].append(wdown)
-        out["norm1"].append(ones(d)); out["norm2"].append(ones(d))
+        out["norm1"].append(gain(l, KIND_NORM1)); out["norm2"].append(gain(l, KIND_NORM2))
     return out
 
 

@@ -44,11 +44,13 @@ def compare_state(eng, loop):
     assert g["next_page"] == o["next_page"]
 
 
-def parity_step(eng, loop, delta, *, tol_logits, tol_reward, margin_tok, margin_gate, stats=None, min_target_rows=1):
+def parity_step(eng, loop, delta, *, tol_logits, tol_reward, margin_tok, margin_gate, stats=None, min_target_rows=1,
+                accept_pattern=None):
     """One step on both sides.  The GPU is forced onto the oracle's tokens; its own samples and its
-    own gate decisions are checked wherever the oracle's margins are clear."""
+    own gate decisions are checked wherever the oracle's margins are clear.  accept_pattern (per row
+    0 / 1 / None) imposes gate decisions on BOTH sides, to steer how many rows the target serves."""
     B = len(loop.rows)
-    o = loop.step(delta, min_target_rows=min_target_rows)
+    o = loop.step(delta, min_target_rows=min_target_rows, forced_accept=accept_pattern)
     eng.force_tokens(DRAFT, o["draft_tokens"])
     eng.force_tokens(TARGET, o["target_tokens"])
     # the gate is left to the GPU except where the oracle's reward sits within the margin of delta
@@ -56,6 +58,8 @@ def parity_step(eng, loop, delta, *, tol_logits, tol_reward, margin_tok, margin_
     for b in range(B):
         if o["drafted"][b] and abs(o["rewards"][b] - delta) <= margin_gate:
             amb[b] = int(o["accept"][b])
+        if accept_pattern is not None and accept_pattern[b] is not None:
+            amb[b] = int(accept_pattern[b])
     eng.force_accept(amb)
     g = eng.step(delta, min_target_rows)
     live_before = (o["step_len"] > 0) | (o["drafted"] > 0) | (o["waiting"] > 0)

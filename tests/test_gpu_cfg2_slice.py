@@ -31,21 +31,55 @@ def test_config2_shapes_reduced_slice():
 
 
 def test_config3_shapes_prm_at_target_shape():
-    """Config-3 slice: 1.5B-shape draft, 7B-shape PRM and 7B-shape target; two rows, one accepted and
-    one rejected step of at most 3 tokens."""
+    """Config-3 slice: 1.5B-shape draft, 7B-shape PRM and 7B-shape target, full depth and vocabulary; four rows,
+    three steps of at most 3 tokens, one step at each threshold of the configuration's sweep (delta = 0.5, 0.7,
+    0.9).  The gate is left to the GPU wherever the oracle's reward is more than 1e-2 away from delta: a random-init
+    7B-shape PRM spreads its rewards over most of [0, 1], so the sweep accepts fewer and fewer rows."""
     import os
     if os.sysconf("SC_PAGE_SIZE") * os.sysconf("SC_PHYS_PAGES") < 90e9:
         pytest.skip("the oracle needs ~65 GB of host memory for two 7B-shape fp32 weight sets")
     shapes = (ri.SHAPES["1.5b"], ri.SHAPES["7b"], ri.SHAPES["7b"])
-    prompts = ri.prompts(2, 2, 6, 9, shapes[0].vocab)
-    base = dict(max_step_tokens=3, max_steps=2, max_seq_tokens=24, step_end_id=13, temperature=0.7, seed=3)
+    prompts = ri.prompts(2, 4, 5, 8, shapes[0].vocab)
+    base = dict(max_step_tokens=3, max_steps=3, max_seq_tokens=24, step_end_id=13, temperature=0.7, seed=3)
     eng, loop = build_pair(shapes, bf16=True, prompts=prompts, loop_kwargs=base)
     stats = {}
-    parity_step(eng, loop, 0.0, stats=stats, **TOL16)
-    g, o = parity_step(eng, loop, 1.5, stats=stats, **TOL16)
-    assert o["rej_idx"] == [0, 1]
+    accepted = []
+    for delta in (0.5, 0.7, 0.9):
+        g, o = parity_step(eng, loop, delta, stats=stats, **TOL16)
+        accepted.append(int(g["accept"].sum()))
+        assert np.all(o["rewards"] >= 0) and np.all(o["rewards"] <= 1)
     compare_counters(eng, loop)
-    print("config-3 shapes, 2 rows x 2 steps x <=3 tokens:", stats)
+    c = eng.counters()
+    assert c["accepted_steps"] == sum(accepted) and c["rejected_steps"] == 12 - sum(accepted)
+    assert c["rejected_steps"] > 0                      # the target ran (catch-up over prompt and accepted steps)
+    print("config-3 shapes, 4 rows x 3 steps x <=3 tokens, delta 0.5 / 0.7 / 0.9: accepted", accepted, stats)
+    eng.close()
+
+
+def test_config4_width_loop_level():
+    """Config 4 at the loop level: batch 8, a target of the 72B shape's width (d 8192, 64 / 8 heads, ffn 29568,
+    vocabulary 152064 -- larger than the draft's and the PRM's 151936, so sampling is confined to the shared ids)
+    with the 1.5B-width draft and PRM, all cut to two layers so that the oracle can hold them; the full depth of
+    the 72B shape is covered by the layer-major test below.  Mixed accept / reject steps with the gate left to
+    the GPU: logits, rewards, tokens, the rejected-row list, cursors and page tables against the oracle."""
+    import dataclasses
+    small = dataclasses.replace(ri.SHAPES["1.5b"], n_layers=2)
+    wide = dataclasses.replace(ri.SHAPES["72b"], n_layers=2)
+    shapes = (small, small, wide)
+    prompts = ri.prompts(4, 8, 5, 20, small.vocab)
+    base = dict(max_step_tokens=3, max_steps=3, max_seq_tokens=40, step_end_id=13, temperature=0.7, seed=11)
+    eng, loop = build_pair(shapes, bf16=True, prompts=prompts, loop_kwargs=base)
+    assert loop.v_limit == small.vocab < wide.vocab
+    delta = float(np.sort(loop.step(0.0)["rewards"])[2])          # the quantile rule: about 70 % accepted
+    eng, loop = build_pair(shapes, bf16=True, prompts=prompts, loop_kwargs=base)
+    stats, seen = {}, set()
+    for _ in range(3):
+        g, o = parity_step(eng, loop, delta, stats=stats, **TOL16)
+        seen |= set(int(a) for a, n in zip(o["accept"], o["step_len"]) if n)
+    assert seen == {0, 1}
+    compare_counters(eng, loop)
+    print("config-4 width (two layers), 8 rows x 3 steps x <=3 tokens:", stats)
+    eng.close()
 
 
 def test_config4_shape_target_layer_major():
@@ -70,7 +104,7 @@ def test_config4_shape_target_layer_major():
     draft_step = rng.integers(0, sd.vocab, size=4).tolist()
     target_step = rng.integers(0, sd.vocab, size=4).tolist()
     got = {}
-    for ext in (0, 1):          # 16-bit cache as benchmarked, and the extended-precision cache
+    for ext in (2, 0):          # plain 16-bit cache forced, and the library's default for an 80-layer model (hi + lo pairs)
         eng = Engine(*models, max_batch=1, max_seq_tokens=32, max_step_tokens=4, max_steps=2, step_end_id=13,
                      temperature=0.0, seed=0, debug_flags=RSD_DEBUG_KEEP_LOGITS, max_chunk_tokens=64, kv_extended=ext)
         eng.prefill(prompt, np.array([0, 7], np.int32))
@@ -94,18 +128,21 @@ def test_config4_shape_target_layer_major():
         ls = OracleModel._layer_struct(lw)
         oracle.lib().orc_layer_forward(om._cshape, ls, x.ctypes.data, len(seq), 0, cache.k[0].ctypes.data,
                                        cache.v[0].ctypes.data)
-    errs = {0: [], 1: []}
+    errs = {2: [], 0: []}
     for j in range(4):
         want = om.logits(x[len(prompt) - 1 + j])
-        for ext in (0, 1):
+        for ext in (2, 0):
             errs[ext].append(float(np.abs(got[ext][j].astype(np.float64) - want).max()))
-    print("config-4 target shape, 1 row, 7-token prompt + 4-token step: max logit errors, 16-bit KV", errs[0],
-          "extended KV", errs[1])
+    print("config-4 target shape, 1 row, 7-token prompt + 4-token step: max logit errors, plain 16-bit KV", errs[2],
+          "default (hi + lo pairs at this depth)", errs[0])
     # With keys, values, queries and softmax weights all at 11-bit mantissas (fp16) the residual stream
     # picks up about 5e-4 of relative error per layer, most of it from the rounded keys; over 80 layers
     # and 152 K logits of standard deviation 1.8 that is about 5e-2 at the worst logit, above the 3e-2
     # asked of bf16 arithmetic (28 layers: 1.5e-2).  kv_extended = 1 keeps keys and values as hi + lo
     # pairs and splits queries and softmax weights: the attention is then exact to fp32 rounding and
-    # this shape lands near 2e-3, at twice the KV bytes.
-    assert max(errs[1]) <= 1e-2
-    assert max(errs[0]) <= 6e-2
+    # this shape lands near 2e-3, at twice the KV bytes.  The library therefore picks the pairs by itself for
+    # models deeper than 48 layers (kv_extended = 0): the default configuration, which is also the one the
+    # benchmark times for this shape, meets the bound asked of bf16 arithmetic.  The plain cache, which a
+    # caller has to force (kv_extended = 2), is characterised only.
+    assert max(errs[0]) <= 1e-2
+    assert max(errs[2]) <= 6e-2 and max(errs[2]) > max(errs[0])

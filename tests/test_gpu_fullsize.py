@@ -62,3 +62,52 @@ def test_config2_full_size_properties_and_sampled_output():
     assert delta2 == delta and np.array_equal(q0["step_tokens"], r0["step_tokens"])
     assert np.array_equal(q1["step_tokens"], r1["step_tokens"]) and np.array_equal(q1["accept"], r1["accept"])
     eng2.close()
+
+
+
+def test_target_decode_in_the_benchmarked_launch_configuration():
+    """The else-branch of Algorithm 1 (y_i <- M(x, y_{1:i-1})) batched the way the benchmark runs it: a context of
+    32 rows, the rejected rows compacted into the first slots, the target's decode iteration captured once per
+    power-of-two bucket of their number (5 rows -> the 8-slot graph, 9 -> 16 slots, 17 -> 32 slots) and replayed
+    from the second token on; the three patterns run one after the other on ONE context, as the buckets alternate
+    in a benchmark run.  The target has the full 7B shape (28 layers, d 3584, vocabulary 151936); draft and PRM
+    keep the 1.5B width at two layers, since they are not the subject and the oracle's time is better spent on
+    the target.  Two of the rejected rows carry 9- to 14-token prompts (a real catch-up pass), the others 2-token
+    prompts, which keeps the oracle affordable while every slot of the bucket is occupied.  Compared: every logit
+    column of every target (and draft) iteration of every row at 3e-2, rewards, tokens, the rejected-row list,
+    cursors and page tables bit for bit."""
+    import dataclasses
+    from helpers import build_pair, parity_step, compare_counters, compare_state
+    from oracle.rsd_loop import OracleRSD
+    small = dataclasses.replace(ri.SHAPES["1.5b"], n_layers=2)
+    shapes = (small, small, ri.SHAPES["7b"])
+    B, cap = 32, 3
+    kw = dict(max_step_tokens=cap, max_steps=2, max_seq_tokens=32, step_end_id=13, temperature=0.7, seed=3)
+    eng = loop = None
+    for n_rejected in (5, 17, 9):
+        rng = np.random.default_rng(100 + n_rejected)
+        rejected = sorted(rng.choice(B, size=n_rejected, replace=False).tolist())
+        long_rows = [rejected[0], rejected[-1]]                  # first and last slot of the compacted list
+        lens = np.full(B, 2, dtype=np.int32)
+        lens[long_rows] = rng.integers(9, 15, size=2)
+        offsets = np.zeros(B + 1, dtype=np.int32)
+        offsets[1:] = np.cumsum(lens)
+        tokens = rng.integers(0, small.vocab, size=int(offsets[-1])).astype(np.int32)
+        if eng is None:
+            eng, loop = build_pair(shapes, bf16=True, prompts=(tokens, offsets), loop_kwargs=kw)
+        else:
+            eng.prefill(tokens, offsets)                         # drops the previous pattern's rows
+            loop = OracleRSD(*loop.models, loop.cfg)
+            loop.prefill([tokens[offsets[b]:offsets[b + 1]].tolist() for b in range(B)])
+        compare_state(eng, loop)
+        pattern = [0 if b in rejected else 1 for b in range(B)]
+        stats = {}
+        g, o = parity_step(eng, loop, 0.5, stats=stats, accept_pattern=pattern, tol_logits=3e-2, tol_reward=1e-2,
+                           margin_tok=5e-2, margin_gate=1e-2)
+        assert o["rej_idx"] == rejected and eng.state()["rej_idx"] == rejected
+        assert not g["accept"][rejected].any() and g["accept"].sum() == B - n_rejected
+        compare_counters(eng, loop)
+        assert eng.counters()["gen_tokens"][2] == int(g["step_len"][rejected].sum())
+        assert eng.counters()["ingest_tokens"][2] == int((lens[rejected] - 1).sum())
+        print(f"7B-shape target, 32-row context, {n_rejected} rejected rows:", stats)
+    eng.close()

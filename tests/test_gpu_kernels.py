@@ -27,18 +27,42 @@ def test_input_generators_agree_bit_for_bit():
         assert np.array_equal(g["wgu"][1].float().cpu().numpy(), np.concatenate([l["wgate"], l["wup"]]))
         assert np.array_equal(g["wo"][1].float().cpu().numpy(), l["wo"])
         assert np.array_equal(g["wdown"][1].float().cpu().numpy(), l["wdown"])
+        for k in ("norm1", "norm2"):
+            assert np.array_equal(g[k][1].float().cpu().numpy(), l[k]) and np.abs(l[k] - 1).max() > 0.1
+        assert np.array_equal(g["final_norm"].float().cpu().numpy(), c["final_norm"])
+
+
+def philox_numpy(ctr, key):
+    """Philox4x32-10 over an array of counters [n, 4] (uint32), written out with numpy integer arithmetic: ten rounds of
+    two 32 x 32 -> 64-bit products whose halves are mixed with the other words and the key, the key advancing by the
+    two Weyl constants.  A third statement of the algorithm beside the oracle's and the kernel's; the test checks it
+    against the oracle before using it on every counter."""
+    c = [ctr[:, i].astype(np.uint64) for i in range(4)]
+    k0, k1 = np.uint64(key[0]), np.uint64(key[1])
+    mask = np.uint64(0xFFFFFFFF)
+    for _ in range(10):
+        p0 = np.uint64(0xD2511F53) * c[0]
+        p1 = np.uint64(0xCD9E8D57) * c[2]
+        c = [(p1 >> np.uint64(32)) ^ c[1] ^ k0, p1 & mask, (p0 >> np.uint64(32)) ^ c[3] ^ k1, p0 & mask]
+        k0 = (k0 + np.uint64(0x9E3779B9)) & mask
+        k1 = (k1 + np.uint64(0xBB67AE85)) & mask
+    return np.stack(c, axis=1).astype(np.uint32)
 
 
 def test_philox_matches_oracle_on_many_counters():
+    """2^20 random counters (plus all-zero and all-one words): every block of the kernel against the numpy
+    restatement, which itself is checked against the oracle's C implementation on 512 of them."""
     rng = np.random.default_rng(0)
-    n = 1 << 16
+    n = 1 << 20
     ctr = rng.integers(0, 2 ** 32, size=(n, 4), dtype=np.uint64).astype(np.uint32)
     ctr[0] = 0
     ctr[1] = 0xFFFFFFFF
     key = np.array([0x12345678, 0x9ABCDEF0], dtype=np.uint32)
+    want = philox_numpy(ctr, key)
+    for i in list(range(64)) + list(rng.integers(0, n, size=448)):
+        assert np.array_equal(want[i], oracle.philox4x32_10(ctr[i], key))
     got = rb.k_philox(dev(ctr.view(np.int32)), dev(key.view(np.int32))).cpu().numpy().view(np.uint32)
-    for i in list(range(64)) + list(rng.integers(0, n, size=192)):
-        assert np.array_equal(got[i], oracle.philox4x32_10(ctr[i], key))
+    assert np.array_equal(got, want)
     zero = rb.k_philox(dev(np.zeros((1, 4), np.int32)), dev(np.zeros(2, np.int32))).cpu().numpy().view(np.uint32)
     assert [hex(v) for v in zero[0]] == ["0x6627e8d5", "0xe169c58d", "0xbc57ac4c", "0x9b00dbd8"]
 
@@ -88,9 +112,8 @@ def test_gemm_tcgen05(M, N, K):
     got2 = rb.k_gemm(Wd, hi, impl=2, x_lo=lo).cpu().numpy()
     np.testing.assert_allclose(got2, want2, rtol=0, atol=tol)
     assert np.abs(want2 - oracle.matmul(W, x)).max() < 1e-3 * np.sqrt(K) * 0.02 + 1e-4   # hi + lo ~ x
-    if M <= 4 or True:
-        got3 = rb.k_gemm(Wd, hi, impl=1, x_lo=lo).cpu().numpy()                # SIMT path, same operands
-        np.testing.assert_allclose(got3, want2, rtol=0, atol=tol)
+    got3 = rb.k_gemm(Wd, hi, impl=1, x_lo=lo).cpu().numpy()                    # SIMT path, same operands
+    np.testing.assert_allclose(got3, want2, rtol=0, atol=tol)
 
 
 def test_rmsnorm_rope_swiglu():
@@ -139,16 +162,51 @@ def test_sampling_matches_oracle(temperature):
 
 
 def test_gate_compaction_all_masks_and_large():
-    # every mask of 12 rows: brute-force serial loop against the ballot / prefix path
+    """Brute force (a serial loop over the rows) against the ballot / prefix path: EVERY accept mask of 12 rows, one
+    call per mask as the step loop calls it, and every mask of 16 rows laid end to end in one call of 2^20 rows."""
     B = 12
-    for mask in range(0, 1 << B, 37):
-        r = np.array([(0.9 if (mask >> b) & 1 else 0.1) for b in range(B)], dtype=np.float32)
-        live = np.array([1 if b % 5 else 0 for b in range(B)], dtype=np.uint8)
-        acc, rej, n = rb.k_gate_compact(dev(r), dev(live), 0.5)
-        want_rej = [b for b in range(B) if live[b] and r[b] < 0.5]
-        assert int(n.item()) == len(want_rej)
-        assert rej.cpu().numpy()[:len(want_rej)].tolist() == want_rej
-        assert acc.cpu().numpy().tolist() == [int(live[b] and r[b] >= 0.5) for b in range(B)]
+    n_masks = 1 << B
+    bits = (np.arange(n_masks)[:, None] >> np.arange(B)[None, :]) & 1               # [mask, row]
+    r = np.where(bits == 1, np.float32(0.9), np.float32(0.1)).astype(np.float32)
+    live = np.tile(np.array([1 if b % 5 else 0 for b in range(B)], dtype=np.uint8), (n_masks, 1))
+    r_d, live_d = dev(r), dev(live)
+    acc_d = torch.zeros(n_masks, B, dtype=torch.uint8, device="cuda")
+    rej_d = torch.full((n_masks, B), -1, dtype=torch.int32, device="cuda")
+    n_d = torch.zeros(n_masks, dtype=torch.int32, device="cuda")
+    scratch = torch.zeros(64, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream().cuda_stream
+    for m in range(n_masks):
+        rc = rb.lib().rsd_k_gate_compact(r_d.data_ptr() + 4 * B * m, live_d.data_ptr() + B * m, 0.5, acc_d.data_ptr() + B * m,
+                                         rej_d.data_ptr() + 4 * B * m, n_d.data_ptr() + 4 * m, B, scratch.data_ptr(), 64, stream)
+        assert rc == 0
+    acc, rej, n = acc_d.cpu().numpy(), rej_d.cpu().numpy(), n_d.cpu().numpy()
+    for m in range(n_masks):
+        want_rej = []
+        for b in range(B):                                  # the serial definition
+            if live[m, b] and not (r[m, b] >= np.float32(0.5)):
+                want_rej.append(b)
+        assert n[m] == len(want_rej), m
+        assert rej[m, :len(want_rej)].tolist() == want_rej, m
+        assert acc[m].tolist() == [int(live[m, b] and r[m, b] >= np.float32(0.5)) for b in range(B)], m
+    # all 2^16 masks of 16 rows as consecutive segments of one call: the ascending global list, cut at the
+    # segment boundaries, is every segment's own ascending list
+    B = 16
+    n_masks = 1 << B
+    bits = (np.arange(n_masks)[:, None] >> np.arange(B)[None, :]) & 1
+    r = np.where(bits == 1, np.float32(0.9), np.float32(0.1)).astype(np.float32).reshape(-1)
+    live = np.tile(np.array([0 if b in (3, 11) else 1 for b in range(B)], dtype=np.uint8), n_masks)
+    acc, rej, n = rb.k_gate_compact(dev(r), dev(live), 0.5)
+    acc, rej, n = acc.cpu().numpy(), rej.cpu().numpy(), int(n.item())
+    want = []
+    for i in range(n_masks * B):
+        if live[i] and not (r[i] >= np.float32(0.5)):
+            want.append(i)
+    assert n == len(want) and np.array_equal(rej[:n], np.array(want, dtype=np.int32))
+    assert np.array_equal(acc, ((live == 1) & (r >= np.float32(0.5))).astype(np.uint8))
+    seg = rej[:n] // B
+    for m in (0, 1, 0x5A5A, 0xFFFF, 0x8001):
+        want_rej = [b for b in range(B) if live[m * B + b] and not ((m >> b) & 1)]
+        assert (rej[:n][seg == m] - m * B).tolist() == want_rej
     rng = np.random.default_rng(3)
     for B, p in [(1, 0.5), (1023, 0.3), (1024, 0.9), (1025, 0.1), (70001, 0.7), (1 << 20, 0.5)]:
         r = rng.random(B).astype(np.float32)

@@ -176,6 +176,15 @@ def test_call_order_and_argument_errors():
     assert r["accept"].all() and (r["step_len"] > 0).all()
     with pytest.raises(RsdError):                        # a PRM must not carry an lm head, and vice versa
         Engine(models[0], models[0], models[2], max_batch=2, max_seq_tokens=48, max_step_tokens=8, max_steps=2, step_end_id=13)
+    # models are loaded once per context: the captured decode graphs hold their pointers
+    from paper_2501_19324_b200 import lib
+    assert lib().rsd_load_models(eng.ctx, models[0].desc, models[1].desc, models[2].desc) == -2
+    assert b"once per context" in lib().rsd_last_error(eng.ctx)
+    r = eng.step(0.0)                                    # the refusal left the context as it was
+    assert (r["step_len"] > 0).all()
+    with pytest.raises(RsdError) as e:                   # kv_extended takes 0 (by depth), 1 or 2
+        Engine(*models, max_batch=2, max_seq_tokens=48, max_step_tokens=8, max_steps=2, step_end_id=13, kv_extended=3)
+    assert e.value.code == -1
 
 
 @pytest.mark.parametrize("delta,min_rows", [(0.47, 3), (0.49, 4)])

@@ -54,6 +54,27 @@ def test_bf16_rounding_matches_library():
     assert np.array_equal(r, want)
 
 
+def test_norm_gains_are_seeded_distinct_and_away_from_one():
+    """RMSNorm gains are 1 + 5 * (a weight-recipe draw): near 1 +- 0.1, a different vector for every norm of every
+    layer and model, exactly representable in bfloat16 for 16-bit models."""
+    sh = ri.SHAPES["tiny_draft"]
+    for bf16 in (False, True):
+        w = ri.cpu_model_weights(sh, ri.SLOT_DRAFT, 0, bf16, ri.HEAD_LM)
+        p = ri.cpu_model_weights(sh, ri.SLOT_PRM, 0, bf16, ri.HEAD_REWARD_SIGMOID)
+        gains = [w["final_norm"], p["final_norm"]] + [lw[k] for lw in w["layers"] + p["layers"] for k in ("norm1", "norm2")]
+        for g in gains:
+            assert g.shape == (sh.d_model,) and g.dtype == np.float32
+            assert 0.5 < g.min() and g.max() < 1.5 and 0.05 < g.std() < 0.15
+            if bf16:
+                assert np.array_equal(g, torch.from_numpy(g).to(torch.bfloat16).float().numpy())
+        for i in range(len(gains)):
+            for j in range(i + 1, len(gains)):
+                assert np.abs(gains[i] - gains[j]).max() > 0.1
+    draw = ri.cpu_tensor(0, ri.tensor_id(0, 1, ri.KIND_NORM2), 1, sh.d_model, False)[0]
+    want = np.float32(1.0) + np.float32(5.0) * draw
+    assert np.array_equal(ri.cpu_model_weights(sh, 0, 0, False, ri.HEAD_LM)["layers"][1]["norm2"], want)
+
+
 def test_prompts_shape_and_range():
     tok, off = ri.prompts(1, 32, 128, 512, 151936)
     lens = np.diff(off)
