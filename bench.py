@@ -87,17 +87,15 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.rows.append([c.strip() for c in line.split(",")])
 
-    def stop(self) -> dict:
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except subprocess.TimeoutExpired:
-            self.proc.kill()
+    def mark(self) -> int:
+        """Number of samples taken so far; two marks bracket a region for summary()."""
+        return len(self.rows)
+
+    def summary(self, lo: int = 0, hi: int | None = None) -> dict:
+        """Median SM clock, maximum clock and the throttle reasons seen in samples [lo, hi)."""
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
+        for r in self.rows[lo:hi]:
             if len(r) < 7:
                 continue
             try:
@@ -109,6 +107,16 @@ class ClockSampler:
                     reasons.add(n)
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
                 "samples": len(sm), "reasons": sorted(reasons)}
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        return self.summary()
 
 
 def cpu_cores() -> int:
@@ -269,11 +277,14 @@ def mega_phase_table(eng, which: int, n_layers: int) -> dict:
     return out
 
 
-def decode_iteration_roofline(phases, iters, steps, shapes, hbm, queue):
-    """Whole decode iterations against the HBM roofline: the bytes an iteration must read at least (every layer's
-    weights and the lm head once; the KV cache, which comes on top, is left out) over the measured time of an
-    iteration inside the step loop (phase time / iterations; a rejected row's draft step ran to the cap before it
-    was dropped).  Only meaningful for the lock-step schedule."""
+def decode_iteration_roofline(phases, iters, kv_bytes, steps, shapes, hbm, queue):
+    """Whole decode iterations against the HBM roofline.  One iteration of model X is one replay of its captured
+    graph (every layer, the lm head, sampling).  Algorithmic bytes of an iteration: every layer's weights and the
+    lm head once (the embedding table is gathered, not streamed) plus the keys and values of every attended
+    position (kv_bytes: summed on the host from the rows' context lengths).  Time: the phase's device time from
+    CUDA events on the launching stream over the timed steps / the iterations it ran (a phase runs until its
+    longest row ends; a rejected row's draft step ran to the cap before it was dropped).  Only meaningful for the
+    lock-step schedule."""
     if queue != 1:
         return None
     out = {}
@@ -285,8 +296,11 @@ def decode_iteration_roofline(phases, iters, steps, shapes, hbm, queue):
             out[name] = None
             continue
         ms = phases[key] * steps / n
-        gbs = weight_bytes / (ms * 1e-3) / 1e9
-        out[name] = {"ms": ms, "weight_gb": weight_bytes / 1e9, "gbs": gbs, "frac_of_hbm": gbs / hbm, "iterations": n}
+        per_iter = weight_bytes + kv_bytes[name] / n
+        gbs = per_iter / (ms * 1e-3) / 1e9
+        out[name] = {"ms": ms, "weight_gb": weight_bytes / 1e9, "kv_gb": kv_bytes[name] / n / 1e9, "gbs": gbs,
+                     "frac_of_hbm": gbs / hbm, "frac_of_hbm_weights_only": weight_bytes / (ms * 1e-3) / 1e9 / hbm,
+                     "iterations": n}
     return out
 
 
@@ -321,7 +335,7 @@ def run_ours(args, rank: int, world: int):
         for k in ("wqkv", "wo", "wgu", "wdown", "norm1", "norm2"):
             models[1].t[k] = []
         torch.cuda.empty_cache()
-    n_steps = args.warmup + args.steps
+    n_steps = args.warmup + args.steps + 1        # + one untimed step in which single GEMM launches are timed
     S = hi + n_steps * cap
     eng = Engine(*models, max_batch=B, max_seq_tokens=S, max_step_tokens=cap, max_steps=n_steps + 1,
                  step_end_id=13, temperature=0.7, seed=0, kv_extended=kv_extended(args),
@@ -342,6 +356,31 @@ def run_ours(args, rank: int, world: int):
             dist.barrier()
         torch.cuda.synchronize()
 
+    # host-side book-keeping of context lengths, for the algorithmic bytes and flops of the phases
+    z = np.diff(offsets).astype(np.int64)          # committed tokens per row
+    prm_len = z.copy()                             # positions the PRM has cached
+    kv_tok = [sh.kv_bytes_per_token(2) for sh in shapes]
+    kv_bytes = {"draft": 0.0, "target": 0.0}
+    prm_ctx_sum = 0                                # sum over the PRM's processed tokens of the positions each attends
+
+    def account(r, timed):
+        nonlocal prm_ctx_sum
+        took = r["step_len"] > 0
+        acc = took & (r["accept"] == 1)
+        rej = took & (r["accept"] == 0)
+        for b in np.nonzero(took)[0]:
+            n_draft = int(r["step_len"][b]) if acc[b] else cap      # a rejected draft step ran to the cap
+            if timed:
+                kv_bytes["draft"] += kv_tok[0] * (n_draft * int(z[b]) + n_draft * (n_draft - 1) // 2)
+                lo_p, hi_p = int(prm_len[b]), int(z[b]) + n_draft   # PRM: positions [lo_p, hi_p), token p attends p + 1
+                prm_ctx_sum += (hi_p * (hi_p + 1) - lo_p * (lo_p + 1)) // 2
+            if rej[b] and timed:
+                n = int(r["step_len"][b])
+                kv_bytes["target"] += kv_tok[2] * (n * int(z[b]) + n * (n - 1) // 2)
+            if acc[b]:
+                prm_len[b] = z[b] + r["step_len"][b]
+            z[b] += r["step_len"][b]
+
     sampler = ClockSampler(local)
     launches0 = lib().rsd_debug_launch_count()
     barrier()
@@ -355,11 +394,14 @@ def run_ours(args, rank: int, world: int):
     for _ in range(args.warmup):
         r = eng.step(delta, args.queue)
         e2e_tokens += int(r["step_len"].sum())
-    eng.gemm_timing(args.time_stride)
-    eng.phase_ms(True)
+        account(r, False)
+    eng.gemm_timing(0)                                   # no event records inside the timed steps: every decode
+    eng.phase_ms(True)                                   # iteration replays its captured graph
+    c0 = eng.counters()
     barrier()
     launches1 = lib().rsd_debug_launch_count()
     t_start = torch.cuda.Event(enable_timing=True); t_end = torch.cuda.Event(enable_timing=True)
+    clk_lo = sampler.mark()
     t_start.record()
     timed_tokens = 0
     iters = {"draft": 0, "target": 0}
@@ -375,19 +417,28 @@ def run_ours(args, rank: int, world: int):
             iters["draft"] += cap if rejected.any() else int(r["step_len"][took].max())
         if rejected.any():
             iters["target"] += int(r["step_len"][rejected].max())
+        account(r, True)
     t_end.record()
     barrier()
     e2e_end.record()
     torch.cuda.synchronize()
     launches2 = lib().rsd_debug_launch_count()
-    clocks = sampler.stop()
-    gt = eng.gemm_timing(0)
+    clocks = sampler.summary(clk_lo, sampler.mark())
+    c1 = eng.counters()
     phases = {k: v / args.steps for k, v in eng.phase_ms(False).items()}
+    # one more step, outside every timed region: single GEMM launches bracketed by CUDA events (decode
+    # iterations chosen for it run kernel by kernel instead of replaying their graph)
+    gt = {"ms": 0.0, "bytes": 0.0, "launches": 0}
+    if args.time_stride > 0:
+        eng.gemm_timing(args.time_stride)
+        eng.step(delta, args.queue)
+        gt = eng.gemm_timing(0)
+    sampler.stop()
     e2e_tokens += timed_tokens
     ms = t_start.elapsed_time(t_end)
     e2e_ms = e2e_start.elapsed_time(e2e_end)
     ms, e2e_ms, timed_tokens, e2e_tokens = combine_ranks(ms, e2e_ms, timed_tokens, e2e_tokens, world, "cuda")
-    counters = eng.counters()
+    counters = c1
     mega_tables = None
     if args.mega_profile and rank == 0:
         mega_tables = {}
@@ -399,30 +450,60 @@ def run_ours(args, rank: int, world: int):
 
     if rank == 0:
         hbm, tf, how = peaks()
-        achieved = gt["bytes"] / (gt["ms"] * 1e-3) / 1e9 if gt["ms"] > 0 else None
+        dec = decode_iteration_roofline(phases, iters, kv_bytes, args.steps, shapes, hbm, args.queue)
+        gemm_gbs = gt["bytes"] / (gt["ms"] * 1e-3) / 1e9 if gt["ms"] > 0 else None
         ratio = gemm_traffic_ratio()
-        traffic = (ratio * gt["bytes"] / gt["launches"]) if (ratio and gt["launches"]) else None
+        gemm_sub = {"what": "single weight-GEMM launches (decode, scoring, catch-up) in one extra, untimed step: CUDA events "
+                            f"around every {args.time_stride}th launch; the decode iterations picked for it run kernel by kernel",
+                    "GBps": gemm_gbs, "frac_of_hbm": (gemm_gbs / hbm) if gemm_gbs else None, "timed_launches": gt["launches"],
+                    "algorithmic_bytes_per_launch": (gt["bytes"] / gt["launches"]) if gt["launches"] else None,
+                    "dram_traffic_over_algorithmic": ratio,
+                    "traffic_source": "ncu capture of one decode-shaped launch (profiles/)" if ratio else
+                                      "none: the kernel changed since the counters were taken"}
+        # dominant phase: the target's decode iterations
+        tgt = dec["target"] if dec else None
+        if tgt:
+            roofline = {"bound": "hbm", "kernel": "target decode iteration: one replay of the captured graph (28 layers of qkv / "
+                        "attention / wo / gate-up + SwiGLU / down, lm head, sampling)",
+                        "achieved": tgt["gbs"], "peak": hbm, "unit": "GB/s", "frac": tgt["frac_of_hbm"], "traffic": None,
+                        "algorithmic_bytes_per_launch": (tgt["weight_gb"] + tgt["kv_gb"]) * 1e9,
+                        "launches": tgt["iterations"], "avg_launch_ms": tgt["ms"],
+                        "traffic_note": "no DRAM counters for a whole iteration; see gemm.dram_traffic_over_algorithmic for "
+                                        "the kernel class that moves 97 % of its bytes",
+                        "peak_source": how, "timing": "CUDA events on the launching stream around the phase, inside the timed steps",
+                        "gemm": gemm_sub}
+        else:
+            roofline = {"bound": "hbm", "kernel": "weight GEMM launches (no target decode phase ran, or queued schedule)",
+                        "achieved": gemm_gbs, "peak": hbm, "unit": "GB/s", "frac": (gemm_gbs / hbm) if gemm_gbs else None,
+                        "traffic": None, "peak_source": how, "gemm": gemm_sub}
+        # dense regime: the PRM's scoring pass (one ragged multi-token pass per step)
+        prm = shapes[1]
+        prm_tokens = (c1["score_tokens"] + c1["ingest_tokens"][1]) - (c0["score_tokens"] + c0["ingest_tokens"][1])
+        prm_layer_params = prm.n_params(ri.HEAD_REWARD_SIGMOID) - prm.vocab * prm.d_model
+        prm_flops = 2.0 * prm_layer_params * prm_tokens + 4.0 * prm.n_layers * prm.n_heads * prm.head_dim * prm_ctx_sum
+        prm_ms = phases["prm_scoring"] * args.steps
+        dense = None
+        if not merged and prm_ms > 0 and prm_tokens > 0:
+            tfs = prm_flops / (prm_ms * 1e-3) / 1e12
+            dense = {"bound": "tensor", "kernel": "PRM scoring phase (page reservation, pass list, every layer's GEMMs, chunk "
+                     "attention, norms, reward head)", "achieved": tfs, "peak": tf, "unit": "TFLOP/s", "frac": tfs / tf,
+                     "flops": "algorithmic: 2 * layer parameters * tokens + 4 * L * H * hd * attended positions (no factor "
+                              "for split-precision operands)",
+                     "tokens_per_step": prm_tokens / args.steps, "ms_per_step": phases["prm_scoring"],
+                     "peak_source": how + " (sustained bf16)"}
         out = {"metric": METRIC, "value": timed_tokens / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
                "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
                "data": "synthetic", "config": workload_config(args),
                "accept_rate": accepted / max(1, live_steps), "delta": delta,
                "e2e": {"value": e2e_tokens / (e2e_ms * 1e-3), "unit": UNIT,
-                       "h2d_bytes_per_step": int(tokens.nbytes + offsets.nbytes) // n_steps,
+                       "h2d_bytes_per_step": int(tokens.nbytes + offsets.nbytes) // (args.warmup + args.steps),
                        "d2h_bytes_per_step": B * (cap * 4 + 4 + 4 + 1 + 1) + 3 * 32,
                        "covers": "prefill from host prompts + all warm-up and timed steps"},
                "gpu_launches": int(launches2 - launches1),
-               "roofline": {"bound": "hbm", "kernel": "weight GEMM (decode, prefill, scoring)", "achieved": achieved,
-                            "peak": hbm, "unit": "GB/s", "frac": (achieved / hbm) if achieved else None,
-                            "traffic": traffic,
-                            "algorithmic_bytes_per_launch": (gt["bytes"] / gt["launches"]) if gt["launches"] else None,
-                            "traffic_source": "ncu capture of one decode-shaped launch (profiles/), traffic / algorithmic = "
-                                              + (f"{ratio}" if ratio else "n/a: kernel changed since the capture")
-                                              + ", scaled to the average launch",
-                            "peak_source": how, "timed_launches": gt["launches"],
-                            "timing": f"CUDA events around every {args.time_stride}th GEMM launch of the timed steps"},
+               "roofline": roofline, "roofline_dense": dense,
                "phase_ms_per_step": phases,
-               "decode_iteration": decode_iteration_roofline(phases, iters, args.steps, shapes, hbm, args.queue),
+               "decode_iteration": dec,
                "flops_paper": counters["flops_paper"], "clocks": clocks,
                "gen_tokens": counters["gen_tokens"]}
         if mega_tables is not None:
@@ -442,9 +523,12 @@ def run_ours(args, rank: int, world: int):
 # ------------------------------------------------------------------------------------------------
 # Kernel sweeps: each point is one JSON line with its fraction of the HBM or bf16 roofline
 # ------------------------------------------------------------------------------------------------
-def _graph_time_us(fn, variants, iters=20):
-    """Device time per call of fn(v), v cycling over `variants` (distinct buffers, so that repeated
-    calls do not hit L2), measured by replaying a CUDA graph of `iters` calls."""
+def _graph_time_us(fn, variants, iters=20, sampler=None, min_seconds=0.3):
+    """Device time per call of fn(v), v cycling over `variants` (distinct buffers, so that repeated calls do not
+    hit L2): a CUDA graph of `iters` calls is replayed at least seven times and for at least `min_seconds`, each
+    replay timed by its own pair of CUDA events; the result is the MEDIAN replay.  Returns (us per call, detail)
+    where detail carries the number of replays, the fastest replay and -- when a ClockSampler is given -- the SM
+    clocks and throttle reasons sampled while this point ran."""
     import torch
     torch.cuda.synchronize()          # inputs were filled on the default stream: finish before the side stream reads them
     side = torch.cuda.Stream()
@@ -457,12 +541,32 @@ def _graph_time_us(fn, variants, iters=20):
             for i in range(iters):
                 fn(variants[i % len(variants)])
     torch.cuda.synchronize()
-    g.replay()
+    for _ in range(3):                # warm-up replays
+        g.replay()
     torch.cuda.synchronize()
-    s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    s.record(); g.replay(); e.record()
-    torch.cuda.synchronize()
-    return s.elapsed_time(e) * 1e3 / iters
+    lo = sampler.mark() if sampler is not None else 0
+    times = []
+    t0 = time.perf_counter()
+    while len(times) < 7 or (time.perf_counter() - t0 < min_seconds and len(times) < 20000):
+        batch = []
+        for _ in range(7 if not times else 32):
+            s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            s.record(); g.replay(); e.record()
+            batch.append((s, e))
+        torch.cuda.synchronize()
+        times += [a.elapsed_time(b) for a, b in batch]
+    detail = {"replays": len(times), "us_min": min(times) * 1e3 / iters, "calls_per_replay": iters}
+    if sampler is not None:
+        detail["clocks"] = sampler.summary(lo, sampler.mark())
+    return float(np.median(times)) * 1e3 / iters, detail
+
+
+def _sweep_sampler():
+    import torch
+    sampler = ClockSampler(torch.cuda.current_device())
+    sampler.start()
+    time.sleep(0.5)
+    return sampler
 
 
 def sweep_gemm(args):
@@ -481,6 +585,7 @@ def sweep_gemm(args):
         torch.cuda.synchronize()
         print(json.dumps({"sweep": "gemm", "only": [M, K, N], "algorithmic_bytes": N * K * 2 + 2 * M * K * 2 + M * N * 4}))
         return
+    sampler = _sweep_sampler()
     for K, N in ((1536, 8960), (3584, 18944)):
         nbuf = max(2, int(400e6 // (N * K * 2)))
         Ws = [(torch.randn(N, K, device="cuda") * 0.02).to(torch.bfloat16) for _ in range(nbuf)]
@@ -495,12 +600,14 @@ def sweep_gemm(args):
             def call(W):
                 rb._check(rb.lib().rsd_k_gemm(rb._ptr(W), rb._ptr(hi), rb._ptr(lo), rb._ptr(y), M, N, K, 1, 0, 0,
                                               rb._ptr(scratch), nbytes, rb._stream()))
-            us = _graph_time_us(call, Ws)
+            us, detail = _graph_time_us(call, Ws, sampler=sampler)
             byts = N * K * 2 + 2 * M * K * 2 + M * N * 4
-            flops = 2.0 * 2 * M * N * K          # hi and lo rows both go through the tensor cores
+            flops = 2.0 * M * N * K              # the contraction itself; the hi + lo operand rows double the tensor-core work
             print(json.dumps({"sweep": "gemm", "M": M, "K": K, "N": N, "us": us, "GBps": byts / us * 1e-3,
-                              "hbm_frac": byts / us * 1e-3 / hbm, "TFLOPs_mma": flops / us * 1e-6,
-                              "bf16_frac": flops / us * 1e-6 / tf, "peak_source": how}), flush=True)
+                              "hbm_frac": byts / us * 1e-3 / hbm, "TFLOPs_algorithmic": flops / us * 1e-6,
+                              "bf16_frac_algorithmic": flops / us * 1e-6 / tf, "TFLOPs_mma": 2 * flops / us * 1e-6,
+                              "peak_source": how, **detail}), flush=True)
+    sampler.stop()
 
 
 def sweep_attn(args):
@@ -508,6 +615,7 @@ def sweep_attn(args):
     from paper_2501_19324_b200 import binding as rb
     hbm, _, how = peaks()
     hd = 128
+    sampler = _sweep_sampler()
     for H, KV in ((12, 2), (28, 4)):
         for ctx in (512, 1024, 2048, 4096, 8192, 16384):
             for B in (1, 2, 4, 8, 16, 32, 64, 128, 256):
@@ -528,17 +636,19 @@ def sweep_attn(args):
                     rb._check(rb.lib().rsd_k_attn_decode(rb._ptr(q), rb._ptr(pool), rb._ptr(table), rb._ptr(ctx_len),
                                                          rb._ptr(out), B, H, KV, hd, ctx // 16, 2, rb._ptr(scratch),
                                                          nbytes, rb._stream()))
-                us = _graph_time_us(call, pools, iters=10)
+                us, detail = _graph_time_us(call, pools, iters=10, sampler=sampler)
                 print(json.dumps({"sweep": "attn_decode", "H": H, "KV": KV, "ctx": ctx, "batch": B, "us": us,
                                   "GBps": pool_bytes / us * 1e-3, "hbm_frac": pool_bytes / us * 1e-3 / hbm,
-                                  "pages": "randomly permuted", "peak_source": how}), flush=True)
+                                  "pages": "randomly permuted", "peak_source": how, **detail}), flush=True)
                 del pools
+    sampler.stop()
 
 
 def sweep_gate(args):
     import torch
     from paper_2501_19324_b200 import binding as rb
     hbm, _, how = peaks()
+    sampler = _sweep_sampler()
     for B in (256, 1 << 20):
         for p in (0.1, 0.3, 0.5, 0.7, 0.9):
             r = torch.rand(B, device="cuda")
@@ -551,11 +661,12 @@ def sweep_gate(args):
             def call(_):
                 rb._check(rb.lib().rsd_k_gate_compact(rb._ptr(r), rb._ptr(live), float(1 - p), rb._ptr(acc), rb._ptr(rej),
                                                       rb._ptr(n), B, rb._ptr(scratch), scratch.numel(), rb._stream()))
-            us = _graph_time_us(call, [0])
+            us, detail = _graph_time_us(call, [0], sampler=sampler)
             byts = B * (4 + 1 + 1) + int(B * (1 - p)) * 4
             print(json.dumps({"sweep": "gate_compact", "rows": B, "accept_p": p, "us": us, "GBps": byts / us * 1e-3,
                               "hbm_frac": byts / us * 1e-3 / hbm, "bound": "latency" if B <= 1024 else "hbm",
-                              "peak_source": how}), flush=True)
+                              "peak_source": how, **detail}), flush=True)
+    sampler.stop()
 
 
 def sweep_score(args):
@@ -569,22 +680,36 @@ def sweep_score(args):
               Model(prm, ri.gpu_model_tensors(prm, 1, 0, True, ri.HEAD_REWARD_SIGMOID), ri.HEAD_REWARD_SIGMOID),
               Model(small_t, ri.gpu_model_tensors(small_t, 2, 0, True, ri.HEAD_LM), ri.HEAD_LM)]
     layer_params = prm.n_params(ri.HEAD_REWARD_SIGMOID) - prm.vocab * prm.d_model
+    sampler = _sweep_sampler()
+    n_rep = 7
     for B in (1, 2, 4, 8, 16, 32, 64, 128):
-        eng = Engine(*models, max_batch=B, max_seq_tokens=256 + 3 * 128, max_step_tokens=128, max_steps=4,
+        eng = Engine(*models, max_batch=B, max_seq_tokens=256 + (n_rep + 2) * 128, max_step_tokens=128, max_steps=n_rep + 2,
                      step_end_id=13, temperature=0.7, seed=0)
         tokens, offsets = ri.prompts(3, B, 256, 256, small_d.vocab)
         eng.prefill(tokens, offsets)
         eng.step(0.0)
         eng.phase_ms(True)
-        eng.step(0.0)
-        ms = eng.phase_ms(False)["prm_scoring"]
-        T = B * 128
-        flops = 2.0 * layer_params * T
-        print(json.dumps({"sweep": "prm_scoring", "batch": B, "step_tokens": 128, "ms": ms,
-                          "TFLOPs_algorithmic": flops / ms * 1e-9, "bf16_frac_algorithmic": flops / ms * 1e-9 / tf,
-                          "note": "split-precision operands double the tensor-core work per algorithmic flop",
-                          "peak_source": how}), flush=True)
+        lo = sampler.mark()
+        ms_all, flops_all = [], []
+        for i in range(n_rep):
+            r = eng.step(0.0)
+            ms_all.append(eng.phase_ms(True)["prm_scoring"])
+            # scored tokens sit at positions z .. z + len - 1 of their rows: contraction flops of the layers plus the
+            # attention products (QK^T and PV: 4 * H * hd flops per attended position and layer)
+            z0 = 256 + (i + 1) * 128
+            T = int(r["step_len"].sum())
+            ctx_sum = sum(int(n) * z0 + int(n) * (int(n) + 1) // 2 for n in r["step_len"])
+            flops_all.append(2.0 * layer_params * T + 4.0 * prm.n_layers * prm.n_heads * prm.head_dim * ctx_sum)
+        eng.phase_ms(False)
+        k = int(np.argsort(ms_all)[len(ms_all) // 2])
+        ms, flops = ms_all[k], flops_all[k]
+        print(json.dumps({"sweep": "prm_scoring", "batch": B, "step_tokens": 128, "ms": ms, "ms_min": min(ms_all),
+                          "steps_timed": n_rep, "TFLOPs_algorithmic": flops / ms * 1e-9,
+                          "bf16_frac_algorithmic": flops / ms * 1e-9 / tf,
+                          "note": "median step; algorithmic flops = 2 * layer parameters * tokens + attention products",
+                          "peak_source": how, "clocks": sampler.summary(lo, sampler.mark())}), flush=True)
         eng.close()
+    sampler.stop()
 
 
 def main():

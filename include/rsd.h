@@ -98,7 +98,7 @@ typedef struct {
                                  and values, fp16 queries and softmax weights.  0 (default): by depth -- plain
                                  fp16 for models of up to 48 layers, the pairs for deeper ones, whose logits
                                  would otherwise leave the 3e-2 band around an exact reference (measured at 80
-                                 layers: 5.7e-2 with the plain cache, 1.7e-3 with the pairs)                  */
+                                 layers: 5e-2 to 7e-2 with the plain cache, 2e-3 with the pairs)                  */
   int32_t prm_shares_draft;   /* 1: merged serving (Appendix B.3: the PRM is a projection layer on a language
                                  model's final layer; Section 4 on merging PRM and policy): the PRM is its
                                  final_norm and scalar head on the DRAFT's trunk.  r_i is read after one

@@ -145,7 +145,7 @@ double count_params(const rsd_model& m) {
 
 // Whether model m caches keys and values as fp16 hi + lo pairs.  Setting 0 decides by depth: the rounding of
 // 16-bit keys and values grows with the number of layers, and beyond 48 layers the logits of a bf16 model
-// leave the 3e-2 band around an exact reference (80 layers: 5.7e-2), so deep models get the pairs.
+// leave the 3e-2 band around an exact reference (80 layers: 5e-2 to 7e-2), so deep models get the pairs.
 bool kv_extended_for(const rsd_model& m, int setting) {
   if (m.dtype != RSD_BF16) return false;
   return setting == 1 || (setting == 0 && m.n_layers > 48);
@@ -407,7 +407,7 @@ int forward_pass(rsd_ctx* c, int which, PassView p, cudaStream_t s) {
     CU(launch_rmsnorm(m.dtype, c->x, M.norm2[l], c->h, h_lo, T, d, m.rms_eps, nullptr, p.n_active, x_pending, s));
     // up to 128 rows: fused kernel; dense passes (no idle flag): the persistent kernel hides the SwiGLU epilogue
     // under the next tile's MMAs
-    if (gu_fused_ok(M, T) || (T > 128 && p.n_active == nullptr && gu_fused_ok(M, 128))) {
+    if (gu_fused_ok(M, T) || (T > 128 && p.n_active == nullptr && m.dtype == RSD_BF16 && gemm_gu_supported(1, T, F, d))) {
       rc = gemm_gu(c, M, M.wgu[l], c->h, h_lo, c->act, act_lo, T, F, d, p.n_active, s);
       if (rc) return rc;
     } else {
@@ -772,9 +772,12 @@ int rsd_load_models(rsd_ctx* c, const rsd_model* draft, const rsd_model* prm, co
     M.m.norm1 = M.norm1.data(); M.m.norm2 = M.norm2.data();
     M.elem = M.m.dtype == RSD_BF16 ? 2 : 4;
     M.kv_dtype = M.m.dtype == RSD_BF16 ? (kv_extended_for(M.m, c->cfg.kv_extended) ? 3 : 2) : 0;
-    // hi + lo operands for every bf16 model: with plain bf16 operands a 7B-shape PRM misses the
-    // 1e-2 reward bound (1.1e-2 measured), a 1.5B-shape one would pass (1.5e-3)
-    M.split = M.m.dtype == RSD_BF16;
+    // hi + lo operands for the bf16 policies (logits within 3e-2 need them: plain bf16 GEMM inputs alone cost
+    // 5.7e-2 at the 1.5B shape).  The PRM's one scalar is far less sensitive: with plain bf16 operands a
+    // 1.5B-shape PRM errs by 1.5e-3 against the 1e-2 asked, a 7B-shape one by 1.1e-2; the error grows with the
+    // width, so PRMs of up to 2048 columns take plain operands (half the tensor-core work of a scoring pass),
+    // wider ones the pairs.
+    M.split = M.m.dtype == RSD_BF16 && !(w == RSD_PRM && M.m.d_model <= 2048);
     M.n_params = count_params(M.m);
     M.kv_pool = (char*)c->cfg.kv_pool[w];
     const size_t page_bytes = (size_t)(M.kv_dtype == 3 ? 4 : 2) * M.m.n_kv_heads * kPageTokens * M.m.head_dim * M.elem;

@@ -332,23 +332,28 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
 // GU: gate/up tiles with the SwiGLU epilogue as above; the exchange buffers get shared memory of their own, since
 // the ring is busy with the next tile.
 // ---------------------------------------------------------------------------------------------------------
-struct PersistCfg {
-  static constexpr int kMT = 256, kRows = 128, kStages = 4;
-  static constexpr int kABytes = kTileN * kTileK * 2, kBBytes = kMT * kTileK * 2, kStageBytes = kABytes + kBBytes;
+// SPLIT: the x tile is 128 rows of hi followed by the same 128 rows of lo (the epilogue adds the halves); otherwise it is
+// 256 plain rows.  Either way the instruction's N is 256 and an accumulator takes 256 columns of tensor memory.
+template <bool SPLIT, bool GU> struct PersistCfg {
+  static constexpr int kMT = 256, kRows = SPLIT ? 128 : 256;
   static constexpr int kHalf = kRows / 2, kLd = kHalf + 1;
-  static constexpr size_t kXchBytes = 2 * 64 * (size_t)kLd * 4;
-  static constexpr size_t smem(bool gu) { return 1024 + (size_t)kStages * kStageBytes + 256 + (gu ? kXchBytes : 0); }
+  static constexpr size_t kXchBytes = GU ? 2 * 64 * (size_t)kLd * 4 : 0;
+  // the exchange buffers of the plain gate/up tile (2 x 64 x 129 floats) leave room for three stages
+  static constexpr int kStages = (GU && !SPLIT) ? 3 : 4;
+  static constexpr int kABytes = kTileN * kTileK * 2, kBBytes = kMT * kTileK * 2, kStageBytes = kABytes + kBBytes;
+  static constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + 256 + kXchBytes;
   static constexpr uint32_t kIdesc = TcCfg<256>::kIdesc;
+  static_assert(kSmemBytes <= 227 * 1024, "shared memory of one CTA");
 };
 
-template <bool GU>
+template <bool GU, bool SPLIT>
 __global__ void __launch_bounds__(192, 1)
 gemm_tc_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x,
                           const __grid_constant__ CUtensorMap tm_x_lo, float* __restrict__ Y, int M, int N, int K,
                           int accumulate, int n_tiles_n, int n_tiles_m, int* __restrict__ err,
                           __nv_bfloat16* __restrict__ act_hi, __nv_bfloat16* __restrict__ act_lo) {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  using C = PersistCfg;
+  using C = PersistCfg<SPLIT, GU>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint64_t* full = (uint64_t*)(smem + (size_t)C::kStages * C::kStageBytes);
@@ -399,7 +404,7 @@ gemm_tc_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid
             tma_load_2d(a, &tm_w, &full[s], kb * kTileK, n0);
           }
           tma_load_2d(a + C::kABytes, &tm_x, &full[s], kb * kTileK, m0);
-          tma_load_2d(a + C::kABytes + C::kRows * kTileK * 2, &tm_x_lo, &full[s], kb * kTileK, m0);
+          if (SPLIT) tma_load_2d(a + C::kABytes + C::kRows * kTileK * 2, &tm_x_lo, &full[s], kb * kTileK, m0);
         }
       }
       if (*stop) {   // copies in flight must land before the CTA goes away
@@ -450,16 +455,20 @@ gemm_tc_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid
         const int n = n0 + warp * 32 + lane;
         if (ok) {
           for (int c = 0; c < m_valid; c += 16) {
-            float v[16], w[16];
+            float v[16];
             tmem_ld16(taddr + c, v);
-            tmem_ld16(taddr + C::kRows + c, w);
+            if (SPLIT) {
+              float w[16];
+              tmem_ld16(taddr + C::kRows + c, w);
+#pragma unroll
+              for (int j = 0; j < 16; ++j) v[j] += w[j];
+            }
             if (n < N) {
 #pragma unroll
               for (int j = 0; j < 16; ++j) {
                 if (c + j < m_valid) {
                   float* y = Y + (size_t)(m0 + c + j) * N + n;
-                  const float r = v[j] + w[j];
-                  *y = accumulate ? (*y + r) : r;
+                  *y = accumulate ? (*y + v[j]) : v[j];
                 }
               }
             }
@@ -477,11 +486,16 @@ gemm_tc_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid
         if (ok) {
 #pragma unroll 1
           for (int c = 0; c < C::kHalf; c += 16) {
-            float v[16], w[16];
+            float v[16];
             tmem_ld16(taddr + send0 + c, v);
-            tmem_ld16(taddr + C::kRows + send0 + c, w);
+            if (SPLIT) {
+              float w[16];
+              tmem_ld16(taddr + C::kRows + send0 + c, w);
 #pragma unroll
-            for (int j = 0; j < 16; ++j) send[c + j] = v[j] + w[j];
+              for (int j = 0; j < 16; ++j) v[j] += w[j];
+            }
+#pragma unroll
+            for (int j = 0; j < 16; ++j) send[c + j] = v[j];
           }
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");
@@ -489,20 +503,25 @@ gemm_tc_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid
 #pragma unroll 1
           for (int c = 0; c < C::kHalf; c += 16) {
             if (own0 + c >= m_valid) break;
-            float v[16], w[16];
+            float v[16];
             tmem_ld16(taddr + own0 + c, v);
-            tmem_ld16(taddr + C::kRows + own0 + c, w);
+            if (SPLIT) {
+              float w[16];
+              tmem_ld16(taddr + C::kRows + own0 + c, w);
+#pragma unroll
+              for (int j = 0; j < 16; ++j) v[j] += w[j];
+            }
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
               const int r = own0 + c + j;
               if (r < m_valid) {
-                const float mine = v[j] + w[j], other = recv[c + j];
+                const float mine = v[j], other = recv[c + j];
                 const float gate = is_gate ? mine : other, up = is_gate ? other : mine;
                 const float a = gate / (1.f + expf(-gate)) * up;
                 const size_t o = (size_t)(m0 + r) * N + n0 + l;
                 const __nv_bfloat16 h = __float2bfloat16_rn(a);
                 act_hi[o] = h;
-                act_lo[o] = __float2bfloat16_rn(a - __bfloat162float(h));
+                if (SPLIT) act_lo[o] = __float2bfloat16_rn(a - __bfloat162float(h));
               }
             }
           }
@@ -683,23 +702,23 @@ static int sm_count() {
   return n;
 }
 
-// Dense regime (M > 128 rows, split-precision operand, no K split, no row scale, no idle flag): persistent kernel.
-template <bool GU>
+// Dense regime (M > 128 rows, no K split, no row scale, no idle flag): persistent kernel.
+template <bool GU, bool SPLIT>
 static cudaError_t launch_persistent(const CUtensorMap& tw, const CUtensorMap& tx, const CUtensorMap& txl, float* y, int M, int N,
                                      int K, int accumulate, int* err, __nv_bfloat16* act_hi, __nv_bfloat16* act_lo, cudaStream_t s) {
-  constexpr size_t smem = PersistCfg::smem(GU);
-  static_assert(PersistCfg::smem(true) <= 227 * 1024, "shared memory of one CTA");
+  using C = PersistCfg<SPLIT, GU>;
+  constexpr size_t smem = C::kSmemBytes;
   static bool configured = false;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_tc_persistent_kernel<GU>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(gemm_tc_persistent_kernel<GU, SPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     configured = true;
   }
   const int n_sm = sm_count();
   if (n_sm <= 0) return cudaErrorInvalidDevice;
-  const int tiles_n = GU ? N / 64 : (N + kTileN - 1) / kTileN, tiles_m = (M + PersistCfg::kRows - 1) / PersistCfg::kRows;
+  const int tiles_n = GU ? N / 64 : (N + kTileN - 1) / kTileN, tiles_m = (M + C::kRows - 1) / C::kRows;
   const int grid = std::min(tiles_n * tiles_m, n_sm);
-  RSD_LAUNCH((gemm_tc_persistent_kernel<GU>), grid, 192, smem, s, tw, tx, txl, y, M, N, K, accumulate, tiles_n, tiles_m, err,
+  RSD_LAUNCH((gemm_tc_persistent_kernel<GU, SPLIT>), grid, 192, smem, s, tw, tx, txl, y, M, N, K, accumulate, tiles_n, tiles_m, err,
              act_hi, act_lo);
   return launched(1);
 }
@@ -730,18 +749,25 @@ bool gemm_gu_supported(int dtype, int M, int F, int K) {
 cudaError_t launch_gemm_gu(const void* Wgu, const void* x, const void* x_lo, void* act_hi, void* act_lo, int M, int F, int K,
                            void* scratch, size_t scratch_bytes, const int32_t* n_active, cudaStream_t s, RowScale rs) {
   if (M <= 0) return cudaSuccess;
-  if (!gemm_gu_supported(1, M, F, K) || !x_lo || !act_hi || !act_lo) return cudaErrorNotSupported;
+  if (!gemm_gu_supported(1, M, F, K) || !act_hi) return cudaErrorNotSupported;
   if (!scratch || scratch_bytes < (size_t)kCounterBytes + 256) return cudaErrorInvalidValue;
   if (((uintptr_t)Wgu & 15) || ((uintptr_t)x & 15) || ((uintptr_t)x_lo & 15)) return cudaErrorMisalignedAddress;
+  int* err = (int*)((char*)scratch + kCounterBytes);
+  CUtensorMap tw, tx, txl;
+  if (x_lo == nullptr) {
+    // plain bf16 operand: the persistent kernel only (more than 128 rows, no row scale, no idle flag)
+    if (!(M > 128 && rs.ssq == nullptr && n_active == nullptr)) return cudaErrorNotSupported;
+    if (!get_map(Wgu, 2 * F, K, kTileN / 2, &tw) || !get_map(x, M, K, 256, &tx)) return cudaErrorNotSupported;
+    return launch_persistent<true, false>(tw, tx, tx, nullptr, M, F, K, 0, err, (__nv_bfloat16*)act_hi, nullptr, s);
+  }
+  if (!act_lo) return cudaErrorNotSupported;
   // at least 32 x rows per tile: each warp pair finishes one half of them, 16 at a time
   const int rows = M <= 32 ? 32 : (M <= 64 ? 64 : 128);
   if (rs.ssq != nullptr && rows > 128) return cudaErrorInvalidValue;
-  CUtensorMap tw, tx, txl;
   if (!get_map(Wgu, 2 * F, K, kTileN / 2, &tw) || !get_map(x, M, K, rows, &tx) || !get_map(x_lo, M, K, rows, &txl))
     return cudaErrorNotSupported;
-  int* err = (int*)((char*)scratch + kCounterBytes);
   if (M > 128 && rs.ssq == nullptr && n_active == nullptr)
-    return launch_persistent<true>(tw, tx, txl, nullptr, M, F, K, 0, err, (__nv_bfloat16*)act_hi, (__nv_bfloat16*)act_lo, s);
+    return launch_persistent<true, true>(tw, tx, txl, nullptr, M, F, K, 0, err, (__nv_bfloat16*)act_hi, (__nv_bfloat16*)act_lo, s);
   auto* hi = (__nv_bfloat16*)act_hi;
   auto* lo = (__nv_bfloat16*)act_lo;
   // fewer than ~1.5 CTAs per SM: one CTA per SM with a deep ring streams faster than a thin second wave
@@ -787,8 +813,10 @@ cudaError_t launch_gemm_tc(const void* W, const void* x, const void* x_lo, float
   else txl = tx;
   int* err = (int*)((char*)scratch + kCounterBytes);
   float* partials = (float*)((char*)scratch + kCounterBytes + 256);
-  if (split_operand && M > 128 && p.splits == 1 && rs.ssq == nullptr && n_active == nullptr)
-    return launch_persistent<false>(tw, tx, txl, y, M, N, K, accumulate, err, nullptr, nullptr, s);
+  if (M > 128 && p.splits == 1 && rs.ssq == nullptr && n_active == nullptr) {
+    if (split_operand) return launch_persistent<false, true>(tw, tx, txl, y, M, N, K, accumulate, err, nullptr, nullptr, s);
+    return launch_persistent<false, false>(tw, tx, txl, y, M, N, K, accumulate, err, nullptr, nullptr, s);
+  }
 #define RSD_TC(MT, SP) return launch_mt<MT, SP>(tw, tx, txl, y, M, N, K, accumulate, p, partials, err, n_active, defer, rs, s)
   if (split_operand) {
     switch (p.mt) {

@@ -362,3 +362,98 @@ def test_merged_prm_equals_a_separate_prm_with_the_drafts_trunk(tiny_weights):
         assert sep.counters[key] == mrg.counters[key]
     assert mrg.counters["ingest_tokens"][PRM] == 0
     assert mrg.counters["score_tokens"] == mrg.counters["steps"]     # one token per scored step (lock-step)
+
+
+# ---------------------------------------------------------------------------------------------------------
+# RSD combined with speculative decoding for the rejected steps (Section 4, "Combine RSD with SD")
+# ---------------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("temperature,k", [(0.0, 1), (0.0, 4), (0.7, 3), (0.7, 8)])
+def test_speculative_rejected_steps_equal_plain_target_decoding(tiny_weights, temperature, k):
+    """However many tokens the draft proposes per round and whatever it proposes, the step a rejected row
+    receives is the target's own: every committed step equals plain full-recompute decoding with the
+    target from the committed context, and the whole run equals the loop without speculative decoding."""
+    dm, pm, tm = tiny_models(tiny_weights)
+    base = dict(max_step_tokens=7, max_steps=3, max_seq_tokens=64, step_end_id=2, step_end_mod=5,
+                temperature=temperature, seed=13)
+    tok, off = ri.prompts(6, 3, 4, 9, 1024)
+    prompts = [tok[off[b]:off[b + 1]].tolist() for b in range(3)]
+    sd = OracleRSD(dm, pm, tm, LoopConfig(sd_tokens=k, **base))
+    ref = OracleRSD(dm, pm, tm, LoopConfig(**base))
+    sd.prefill(prompts); ref.prefill(prompts)
+    pattern = [[0, 1, 0], [0, 0, 1], [1, 0, 0]]
+    ctx = [list(p) for p in prompts]
+    for i in range(3):
+        a = sd.step(0.5, forced_accept=pattern[i])
+        r = ref.step(0.5, forced_accept=pattern[i])
+        for b in range(3):
+            assert list(a["step_tokens"][b]) == list(r["step_tokens"][b])
+            if not pattern[i][b]:
+                want = plain_decode(tm, TARGET, b, ctx[b], len(a["step_tokens"][b]), sd.cfg, 1024)
+                assert want == list(a["step_tokens"][b])
+                rounds = a["sd_rounds"][b]
+                assert sum(rd["emitted"] for rd in rounds) == len(want)
+                assert all(1 <= rd["emitted"] <= len(rd["props"]) <= k for rd in rounds)
+                # a round writes its matching prefix and, unless the step or the round ended there, one more token
+                for rd in rounds:
+                    assert rd["emitted"] in (rd["matched"], rd["matched"] + 1)
+                # the same logits chose the tokens: traces agree with the plain loop's
+                assert a["target_trace"][b]["sampled"] == r["target_trace"][b]["sampled"]
+            ctx[b] += list(a["step_tokens"][b])
+        sa, sr = sd.state(), ref.state()
+        assert np.array_equal(sa["z_len"], sr["z_len"]) and np.array_equal(sa["kv_len"][PRM], sr["kv_len"][PRM])
+        assert np.array_equal(sa["kv_len"][TARGET], sr["kv_len"][TARGET])
+        for b in range(3):
+            if not pattern[i][b]:        # the draft proposed along: it has cached the step, the plain loop's draft has not
+                assert sa["kv_len"][DRAFT][b] == sa["z_len"][b] - 1 and sr["kv_len"][DRAFT][b] < sa["kv_len"][DRAFT][b]
+        assert sa["pages"] == sr["pages"]
+    cs, cr = sd.counters, ref.counters
+    assert cs["gen_tokens"] == cr["gen_tokens"] and cs["steps"] == cr["steps"]
+    assert cs["sd_verified"] == cs["sd_proposed"] >= cs["gen_tokens"][TARGET] >= cs["sd_rounds"] > 0
+    # the draft never has to catch up on a step it proposed along with
+    assert cs["ingest_tokens"][DRAFT] < cr["ingest_tokens"][DRAFT]
+
+
+def test_speculative_rounds_accept_exactly_the_matching_prefix(tiny_weights):
+    """Proposals planted around the target's true continuation: a round keeps the proposals up to the
+    first one that differs from the target's choice and writes the target's token there; rounds, matches
+    and evaluated positions follow by hand."""
+    dm, pm, tm = tiny_models(tiny_weights)
+    cfg = LoopConfig(max_step_tokens=9, max_steps=1, max_seq_tokens=32, step_end_id=1 << 20, temperature=0.7, seed=5,
+                     sd_tokens=4)
+    prompt = ri.prompts(9, 1, 6, 6, 1024)[0].tolist()
+    truth = plain_decode(tm, TARGET, 0, prompt, 9, cfg, 1024)
+    bad = lambda t: (t + 1) % 1024
+    # round 1 at offset 0: all four right -> 4 written; round 2 at offset 4: wrong at once -> 1 written;
+    # round 3 at offset 5: two right, third wrong -> 3 written; round 4 at offset 8: one slot left, right -> 1 written
+    planted = [truth[0:4], [bad(truth[4]), 7, 7, 7], [truth[5], truth[6], bad(truth[7]), truth[8]], [truth[8]]]
+    loop = OracleRSD(dm, pm, tm, cfg)
+    loop.prefill([prompt])
+    r = loop.step(0.5, forced_accept=[0], forced_sd_props=[planted])
+    assert list(r["step_tokens"][0]) == truth
+    assert [(rd["emitted"], rd["matched"]) for rd in r["sd_rounds"][0]] == [(4, 4), (1, 0), (3, 2), (1, 1)]
+    assert [len(rd["props"]) for rd in r["sd_rounds"][0]] == [4, 4, 4, 1]
+    c = loop.counters
+    assert (c["sd_rounds"], c["sd_proposed"], c["sd_verified"], c["sd_matched"]) == (4, 13, 13, 7)
+    assert c["gen_tokens"][TARGET] == 9 and c["gen_tokens"][DRAFT] == 9
+    st = loop.state()
+    assert st["kv_len"][TARGET][0] == st["kv_len"][DRAFT][0] == len(prompt) + 9 - 1
+    # Section 3.3 accounting: the draft is billed its step and its proposals, the target every evaluated position
+    nd, npr, nt = (m.n_params for m in (dm, pm, tm))
+    want = 2.0 * nd * (9 + 13) + 2.0 * nt * 13 + 2.0 * npr * (c["score_tokens"] + c["ingest_tokens"][PRM])
+    assert loop.flops_paper() == want
+
+
+def test_speculative_rounds_with_an_agreeing_draft(tiny_weights):
+    """When the draft IS the target (same weights) and decoding is greedy, every proposal matches: a step of
+    n tokens takes ceil(n / k) rounds and as many target passes instead of n."""
+    d, p, t = tiny_weights
+    dm, pm = OracleModel(d, DRAFT), OracleModel(p, PRM)
+    tm = OracleModel(d, TARGET)                       # the draft's weights under the target's id
+    cfg = LoopConfig(max_step_tokens=10, max_steps=1, max_seq_tokens=40, step_end_id=1 << 20, temperature=0.0, seed=0,
+                     sd_tokens=4)
+    prompt = ri.prompts(12, 1, 8, 8, 1024)[0].tolist()
+    loop = OracleRSD(dm, pm, tm, cfg)
+    loop.prefill([prompt])
+    r = loop.step(0.5, forced_accept=[0])
+    assert list(r["step_tokens"][0]) == list(r["draft_tokens"][0]) == plain_decode(tm, TARGET, 0, prompt, 10, cfg, 1024)
+    assert [(rd["emitted"], rd["matched"]) for rd in r["sd_rounds"][0]] == [(4, 4), (4, 4), (2, 2)]
