@@ -107,6 +107,15 @@ typedef struct {
                                  scoring pass disappears.  The prm descriptor must repeat the draft's
                                  dimensions and dtype; its layer arrays and kv_pool[RSD_PRM] may be NULL.
                                  Results equal those of a separate PRM whose trunk weights are the draft's */
+  int32_t sd_tokens;          /* k, 0..16.  k > 0: RSD combined with speculative decoding (Section 4, "Combine RSD
+                                 with SD": during a rejected step, draft + target speculative decoding can
+                                 regenerate the step).  The target's step of a rejected row is then written in
+                                 rounds: the draft proposes up to k tokens, the target evaluates its own choice at
+                                 all k positions in ONE pass and the choices are written while every earlier one
+                                 equalled the proposal (at least one, at most k tokens per round).  Sampling
+                                 noise is keyed by (model, row, position), so the step is token for token the
+                                 one plain target decoding writes; only the number of target passes changes.
+                                 The workspace grows with k (logits of k positions per row)                   */
   /* caller-allocated device memory, sizes as reported by rsd_query_sizes (or larger)        */
   void* kv_pool[3];           /* RSD_DRAFT / RSD_PRM / RSD_TARGET                            */
   size_t kv_bytes[3];
@@ -179,6 +188,10 @@ typedef struct {
   uint64_t score_tokens;
   uint64_t steps, accepted_steps, rejected_steps, discarded_draft_tokens;
   double flops_paper, flops_all_tokens;
+  /* speculative decoding of rejected steps (sd_tokens > 0): rounds summed over rows, tokens the draft proposed,
+     proposals the target's choice equalled, positions the target evaluated.  flops_paper then bills the draft
+     its proposals as well and the target every evaluated position instead of every generated token.          */
+  uint64_t sd_rounds, sd_proposed, sd_matched, sd_verified;
 } rsd_counters;
 int rsd_flops_counters(rsd_ctx*, rsd_counters* out);
 
@@ -193,6 +206,11 @@ const char* rsd_last_error(const rsd_ctx*); /* ctx may be NULL: error of the las
  * ids remain readable through rsd_debug_get_sampled.  accept [B] (HOST, may be NULL; 0/1, other
  * values = do not force) overrides the gate when which == RSD_PRM (tokens/len ignored).      */
 int rsd_debug_force(rsd_ctx*, int which, const int32_t* tokens, const int32_t* len, const uint8_t* accept);
+
+/* Speculative decoding of rejected steps, for the NEXT step only: props [B, max_step_tokens, sd_tokens] (HOST)
+ * replaces what the draft proposes -- entry (b, r, j) is proposal j of row b's r-th round -- for rows with
+ * on[b] != 0 (HOST [B]).  Needs sd_tokens > 0 and RSD_DEBUG_KEEP_LOGITS, else RSD_ERR_STATE.                 */
+int rsd_debug_force_sd(rsd_ctx*, const int32_t* props, const uint8_t* on);
 
 /* Logits of the last rsd_step's decode iterations of model `which`, when RSD_DEBUG_KEEP_LOGITS
  * is set: out is a HOST array [B, max_step_tokens, vocab(which)] (row b, iteration j).        */

@@ -42,18 +42,19 @@ class rsd_config(ctypes.Structure):
                                         "step_end_id", "eos_id", "step_end_mod")] + \
                [("temperature", c_float), ("seed", c_uint64), ("omega_kind", c_int32), ("omega_alpha", c_float),
                 ("max_chunk_tokens", c_int32), ("debug_flags", c_int32), ("kv_extended", c_int32), ("prm_shares_draft", c_int32),
-                ("kv_pool", c_void_p * 3), ("kv_bytes", c_size_t * 3), ("workspace", c_void_p),
+                ("sd_tokens", c_int32), ("kv_pool", c_void_p * 3), ("kv_bytes", c_size_t * 3), ("workspace", c_void_p),
                 ("workspace_bytes", c_size_t)]
 
 
 class rsd_counters(ctypes.Structure):
     _fields_ = [("gen_tokens", c_uint64 * 3), ("ingest_tokens", c_uint64 * 3), ("score_tokens", c_uint64),
                 ("steps", c_uint64), ("accepted_steps", c_uint64), ("rejected_steps", c_uint64),
-                ("discarded_draft_tokens", c_uint64), ("flops_paper", c_double), ("flops_all_tokens", c_double)]
+                ("discarded_draft_tokens", c_uint64), ("flops_paper", c_double), ("flops_all_tokens", c_double),
+                ("sd_rounds", c_uint64), ("sd_proposed", c_uint64), ("sd_matched", c_uint64), ("sd_verified", c_uint64)]
 
 
 EXPORTS = ["rsd_query_sizes", "rsd_create", "rsd_load_models", "rsd_prefill", "rsd_step", "rsd_step_queued", "rsd_flops_counters",
-           "rsd_reset", "rsd_destroy", "rsd_last_error", "rsd_debug_force", "rsd_debug_get_logits",
+           "rsd_reset", "rsd_destroy", "rsd_last_error", "rsd_debug_force", "rsd_debug_force_sd", "rsd_debug_get_logits",
            "rsd_debug_get_sampled", "rsd_debug_get_state", "rsd_debug_gemm_timing", "rsd_debug_launch_count", "rsd_debug_mega_profile", "rsd_debug_phase_ms", "rsd_k_gemm", "rsd_k_gemm_scratch_bytes",
            "rsd_k_attn_decode", "rsd_k_attn_decode_scratch_bytes", "rsd_k_attn_chunk", "rsd_k_gate_compact", "rsd_k_gate_compact_static", "rsd_k_gate_compact_static_error", "rsd_k_rmsnorm",
            "rsd_k_rope", "rsd_k_swiglu", "rsd_k_gemm_gu", "rsd_k_sample", "rsd_k_philox"]
@@ -81,6 +82,7 @@ def lib():
         L.rsd_last_error.argtypes = [vp]
         L.rsd_last_error.restype = ctypes.c_char_p
         L.rsd_debug_force.argtypes = [vp, c_int32, vp, vp, vp]
+        L.rsd_debug_force_sd.argtypes = [vp, vp, vp]
         L.rsd_debug_get_logits.argtypes = [vp, c_int32, vp]
         L.rsd_debug_get_sampled.argtypes = [vp, c_int32, vp]
         L.rsd_debug_get_state.argtypes = [vp] * 8
@@ -163,16 +165,17 @@ class Engine:
     def __init__(self, draft: Model, prm: Model, target: Model, *, max_batch, max_seq_tokens, max_step_tokens,
                  max_steps, step_end_id, eos_id=-1, step_end_mod=0, temperature=0.0, seed=0, omega_kind=1,
                  omega_alpha=0.0, max_chunk_tokens=0, debug_flags=0, kv_bytes=None, kv_extended=0,
-                 prm_shares_draft=0):
+                 prm_shares_draft=0, sd_tokens=0):
         import torch
         if not torch.cuda.is_available():
             raise RsdError(-4, "no CUDA device: this library has no CPU fallback")
         self.models = (draft, prm, target)
         self.B_max, self.S, self.C = max_batch, max_seq_tokens, max_step_tokens
         self.max_pages = (max_seq_tokens + 15) // 16
+        self.sd_tokens = sd_tokens
         cfg = rsd_config(max_batch, max_seq_tokens, max_step_tokens, max_steps, 16, step_end_id, eos_id, step_end_mod,
                          temperature, seed, omega_kind, omega_alpha, max_chunk_tokens, debug_flags, kv_extended,
-                         prm_shares_draft)
+                         prm_shares_draft, sd_tokens)
         _check(lib().rsd_query_sizes(draft.desc, prm.desc, target.desc, cfg))
         if kv_bytes is not None:
             for i in range(3):
@@ -223,7 +226,8 @@ class Engine:
         return dict(gen_tokens=list(c.gen_tokens), ingest_tokens=list(c.ingest_tokens), score_tokens=c.score_tokens,
                     steps=c.steps, accepted_steps=c.accepted_steps, rejected_steps=c.rejected_steps,
                     discarded_draft_tokens=c.discarded_draft_tokens, flops_paper=c.flops_paper,
-                    flops_all_tokens=c.flops_all_tokens)
+                    flops_all_tokens=c.flops_all_tokens, sd_rounds=c.sd_rounds, sd_proposed=c.sd_proposed,
+                    sd_matched=c.sd_matched, sd_verified=c.sd_verified)
 
     def reset(self):
         _check(lib().rsd_reset(self.ctx), self.ctx)
@@ -261,6 +265,20 @@ class Engine:
                 tok[b, :len(s)] = s
                 ln[b] = len(s)
         _check(lib().rsd_debug_force(self.ctx, which, tok.ctypes.data, ln.ctypes.data, None), self.ctx)
+
+    def force_sd_proposals(self, rounds: list):
+        """rounds[b]: None, or the list of row b's rounds, each a list of proposed token ids (speculative decoding
+        of rejected steps); imposed on the draft's proposals in the next step."""
+        k = self.sd_tokens
+        props = np.zeros((self.B, self.C, k), np.int32)
+        on = np.zeros(self.B, np.uint8)
+        for b, rs in enumerate(rounds):
+            if rs is None:
+                continue
+            on[b] = 1
+            for r, p in enumerate(rs):
+                props[b, r, :len(p)] = p
+        _check(lib().rsd_debug_force_sd(self.ctx, props.ctypes.data, on.ctypes.data), self.ctx)
 
     def force_accept(self, mask):
         m = np.array([255 if v is None else int(v) for v in mask], dtype=np.uint8)

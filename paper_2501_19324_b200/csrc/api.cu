@@ -33,6 +33,7 @@ struct ModelHost {
 // Host-visible scalars mirrored from the device after each phase boundary.
 struct Scalars {
   int32_t n_tok, n_rej, err, n_active, n_slots, next_page[3], iter, n_live;
+  int32_t sd_rounds, sd_proposed, sd_matched, sd_round, sd_j, pad;   // speculative decoding of rejected steps
 };
 
 struct Layout {
@@ -80,10 +81,13 @@ struct rsd_ctx {
   int last_n_rej = 0;
   // one CUDA graph per decode phase (draft, target): a whole decode iteration, replayed per token
   cudaStream_t cap_stream = nullptr;
-  // slot = phase * 4 + bucket of the number of rows that take part (all, a half, a quarter, an eighth or fewer)
-  cudaGraphExec_t dec_graph[8] = {};
-  int dec_graph_B[8] = {};
-  uint64_t dec_graph_kernels[8] = {};
+  // slot = phase * 4 + bucket of the number of rows that take part (all, a half, a quarter, an eighth or fewer);
+  // 8 + bucket: a proposal iteration of the draft, 12 + bucket: the target's pass over a round's proposals
+  // (speculative decoding of rejected steps)
+  cudaGraphExec_t dec_graph[16] = {};
+  int dec_graph_B[16] = {};
+  uint64_t dec_graph_kernels[16] = {};
+  int sd_k = 0, slots_max = 0;
   int attn_rows_hint = 0;      // rows expected to be active in the running decode phase (0: all slots)
   bool time_this_iter = false, in_decode = false;
   // per-phase timing of rsd_step (rsd_debug_phase_ms)
@@ -181,7 +185,9 @@ size_t layout_workspace(const rsd_config& cfg, const rsd_model* const ms[3], rsd
   const int B = cfg.max_batch, S = cfg.max_seq_tokens, C = cfg.max_step_tokens;
   const int max_pages = (S + kPageTokens - 1) / kPageTokens;
   const int chunk = cfg.max_chunk_tokens > 0 ? cfg.max_chunk_tokens : 4096;
-  const int T = std::max(B, chunk);
+  const int sd_k = cfg.sd_tokens > 0 ? cfg.sd_tokens : 0;
+  const int slots = B * std::max(1, sd_k);      // token slots of one pass of a decode phase (a round's proposals)
+  const int T = std::max(slots, chunk);
   const Dims dm = max_dims(ms);
   char* base = c ? (char*)cfg.workspace : nullptr;
   auto P = [&](size_t off) -> char* { return base ? base + off : nullptr; };
@@ -214,6 +220,10 @@ size_t layout_workspace(const rsd_config& cfg, const rsd_model* const ms[3], rsd
   int32_t* scal = TAKE(int32_t, 16);
   st.n_tok = scal + 0; st.n_rej = scal + 1; st.err = scal + 2; st.n_active = scal + 3; st.n_slots = scal + 4; st.iter = scal + 8;
   st.next_page = scal + 5; st.n_live = scal + 9;
+  st.sd_k = sd_k; st.sd_stats = scal + 10;
+  st.sd_out_idx = TAKE(int32_t, slots);
+  st.sd_forced_on = TAKE(uint8_t, B);
+  st.sd_forced_props = (sd_k > 0 && (cfg.debug_flags & RSD_DEBUG_KEEP_LOGITS)) ? TAKE(int32_t, (size_t)B * C * sd_k) : nullptr;
   st.pass_capacity = B * S;
   st.pass_tok_id = TAKE(int32_t, (size_t)B * S);
   st.pass_tok_row = TAKE(int32_t, (size_t)B * S);
@@ -226,9 +236,9 @@ size_t layout_workspace(const rsd_config& cfg, const rsd_model* const ms[3], rsd
   void* attn = TAKE(float, (size_t)T * dm.hq);
   float* gu = TAKE(float, (size_t)T * 2 * dm.f);
   void* act = TAKE(float, (size_t)T * dm.f);
-  float* logits = TAKE(float, (size_t)B * dm.v);
-  unsigned long long* sample_best = TAKE(unsigned long long, B);
-  float* norm_ssq = TAKE(float, (size_t)B * 2 * norm_chunks(dm.d));   // room for 128-column chunks
+  float* logits = TAKE(float, (size_t)slots * dm.v);
+  unsigned long long* sample_best = TAKE(unsigned long long, slots);
+  float* norm_ssq = TAKE(float, (size_t)slots * 2 * norm_chunks(dm.d));   // room for 128-column chunks
   void* mega_block[3] = {nullptr, nullptr, nullptr};
   for (int w = 0; w < 3; w += 2) mega_block[w] = TAKE(char, mega_block_bytes(ms[w]->n_layers));
   int32_t* mega_sync = TAKE(int32_t, 1024);
@@ -253,11 +263,12 @@ size_t layout_workspace(const rsd_config& cfg, const rsd_model* const ms[3], rsd
   void* gscr = TAKE(char, gs);
   int h_max = 0;
   for (int w = 0; w < 3; ++w) h_max = std::max(h_max, ms[w]->n_heads);
-  const size_t as = attn_decode_scratch_bytes(B, h_max, dm.hd, S);
+  const size_t as = attn_decode_scratch_bytes(slots, h_max, dm.hd, S);
   void* ascr = TAKE(char, as);
 #undef TAKE
   if (c) {
     c->st = st; c->B_max = B; c->S = S; c->C = C; c->max_pages = max_pages; c->chunk = chunk; c->T_max = T;
+    c->sd_k = sd_k; c->slots_max = slots;
     c->x = x; c->h = h; c->qkv = qkv; c->q = q; c->attn = attn; c->gu = gu; c->act = act; c->logits = logits;
     // each operand buffer was sized at 4 bytes per element: a bf16 hi array followed by its lo array
     c->h_lo = (char*)h + (size_t)T * dm.d * 2;
@@ -289,6 +300,7 @@ int check_config(const rsd_config* cfg, const char** why) {
   if (cfg->omega_kind < 0 || cfg->omega_kind > 4) { *why = "omega_kind"; return RSD_ERR_ARG; }
   if (cfg->step_end_mod < 0) { *why = "step_end_mod"; return RSD_ERR_ARG; }
   if (cfg->kv_extended < 0 || cfg->kv_extended > 2) { *why = "kv_extended out of 0..2"; return RSD_ERR_ARG; }
+  if (cfg->sd_tokens < 0 || cfg->sd_tokens > 16) { *why = "sd_tokens out of 0..16"; return RSD_ERR_ARG; }
   return RSD_OK;
 }
 
@@ -547,28 +559,47 @@ int ensure_mega(rsd_ctx* c, int which, cudaStream_t s) {
   return RSD_OK;
 }
 
-// Enqueues one decode iteration: (prepare, model pass, final norm, lm_head, sample, append).
-int decode_iteration(rsd_ctx* c, int which, int phase, int n_slots, cudaStream_t s) {
+__global__ void scatter_logits_sd_kernel(const float* logits, const int32_t* tok_row, const int32_t* out_idx, float* dbg,
+                                         int V, int C, const int32_t* n_active) {
+  RSD_PDL_SYNC();
+  if (*n_active == 0) return;
+  const int row = tok_row[blockIdx.x];
+  if (row < 0) return;
+  const float* src = logits + (size_t)blockIdx.x * V;
+  float* dst = dbg + ((size_t)row * C + out_idx[blockIdx.x]) * V;
+  for (int i = threadIdx.x; i < V; i += blockDim.x) dst[i] = src[i];
+}
+
+// Model pass + final norm + lm head over the T token slots of p: logits [T, vocab] in c->logits.
+int model_logits(rsd_ctx* c, int which, PassView p, bool allow_mega, cudaStream_t s) {
   const ModelHost& M = c->mdl[which];
   const rsd_model& m = M.m;
-  CU(launch_decode_prepare(c->st, which, n_slots, s));
-  PassView p{c->st.pass_tok_id, c->st.pass_tok_row, c->st.pass_tok_pos, n_slots, c->st.n_active};
+  const int T = p.T;
   int rc;
-  if (c->mega_B[which] > 0 && c->mega_B[which] == c->st.B && n_slots == c->st.B) {
+  if (allow_mega && c->mega_B[which] > 0 && c->mega_B[which] == c->st.B && T == c->st.B) {
     // the whole layer stack in one persistent kernel
     CU(launch_decode_mega(c->mega_block[which], c->st.B, M.kv_dtype == 3, p, m.final_norm, s));
     const RowScale rs{c->norm_ssq, m.d_model / 128, 1.f / (float)m.d_model, m.rms_eps};
-    rc = gemm(c, M, m.head, c->h, c->h_lo, c->logits, n_slots, m.vocab, m.d_model, 0, p.n_active, nullptr, s, rs);
+    rc = gemm(c, M, m.head, c->h, c->h_lo, c->logits, T, m.vocab, m.d_model, 0, p.n_active, nullptr, s, rs);
   } else if (fused_decode_ok(M)) {
     if ((rc = forward_decode_fused(c, which, p, m.final_norm, s))) return rc;
     const RowScale rs{c->norm_ssq, norm_chunks(m.d_model), 1.f / (float)m.d_model, m.rms_eps};
-    rc = gemm(c, M, m.head, c->h, c->h_lo, c->logits, n_slots, m.vocab, m.d_model, 0, p.n_active, nullptr, s, rs);
+    rc = gemm(c, M, m.head, c->h, c->h_lo, c->logits, T, m.vocab, m.d_model, 0, p.n_active, nullptr, s, rs);
   } else {
     if ((rc = forward_pass(c, which, p, s))) return rc;
-    CU(launch_rmsnorm(m.dtype, c->x, m.final_norm, c->h, M.split ? c->h_lo : nullptr, n_slots, m.d_model, m.rms_eps,
+    CU(launch_rmsnorm(m.dtype, c->x, m.final_norm, c->h, M.split ? c->h_lo : nullptr, T, m.d_model, m.rms_eps,
                       nullptr, p.n_active, SplitSum(), s));
-    rc = gemm(c, M, m.head, c->h, c->h_lo, c->logits, n_slots, m.vocab, m.d_model, 0, p.n_active, nullptr, s);
+    rc = gemm(c, M, m.head, c->h, c->h_lo, c->logits, T, m.vocab, m.d_model, 0, p.n_active, nullptr, s);
   }
+  return rc;
+}
+
+// Enqueues one decode iteration: (prepare, model pass, final norm, lm_head, sample, append).
+int decode_iteration(rsd_ctx* c, int which, int phase, int n_slots, cudaStream_t s) {
+  const rsd_model& m = c->mdl[which].m;
+  CU(launch_decode_prepare(c->st, which, n_slots, s));
+  PassView p{c->st.pass_tok_id, c->st.pass_tok_row, c->st.pass_tok_pos, n_slots, c->st.n_active};
+  int rc = model_logits(c, which, p, true, s);
   if (rc) return rc;
   if (c->dbg_logits[phase]) {
     RSD_LAUNCH((scatter_logits_kernel), n_slots, 256, 0, s, c->logits, c->st.pass_tok_row, c->dbg_logits[phase], m.vocab, c->C,
@@ -582,9 +613,55 @@ int decode_iteration(rsd_ctx* c, int which, int phase, int n_slots, cudaStream_t
   return RSD_OK;
 }
 
-// Captures one decode iteration of `which` over all B slots into a graph (idle slots are skipped
-// inside the kernels), so that a token costs one graph launch instead of some 300 kernel launches.
-int ensure_decode_graph(rsd_ctx* c, int which, int phase, int g, int n_slots) {
+// Speculative decoding of rejected steps, one proposal iteration of the draft over the waiting rows' slots: the
+// token at the draft's cursor goes through the draft, the sampled token becomes the round's next proposal.
+int sd_propose_iteration(rsd_ctx* c, int n_slots, cudaStream_t s) {
+  const rsd_model& m = c->mdl[RSD_DRAFT].m;
+  CU(launch_sd_propose_prepare(c->st, n_slots, s));
+  PassView p{c->st.pass_tok_id, c->st.pass_tok_row, c->st.pass_tok_pos, n_slots, c->st.n_active};
+  int rc = model_logits(c, RSD_DRAFT, p, false, s);
+  if (rc) return rc;
+  SampleArgs a{c->logits, n_slots, m.vocab, c->v_limit, c->cfg.temperature, c->cfg.seed, RSD_DRAFT,
+               c->st.pass_tok_row, c->st.pass_tok_pos, nullptr, c->st.n_active, c->sample_best};
+  CU(launch_sample(a, s));
+  CU(launch_sd_propose_update(c->st, c->sample_best, n_slots, s));
+  return RSD_OK;
+}
+
+// ... and the target's pass over a round: sd_k token slots per row slot (the last written token and all proposals
+// but the last), the target's choice at every one of them, then the prefix rule.
+int sd_verify_pass(rsd_ctx* c, int n_slots, cudaStream_t s) {
+  const rsd_model& m = c->mdl[RSD_TARGET].m;
+  CU(launch_sd_verify_prepare(c->st, n_slots, s));
+  const int T = n_slots * c->sd_k;
+  PassView p{c->st.pass_tok_id, c->st.pass_tok_row, c->st.pass_tok_pos, T, c->st.n_active};
+  int rc = model_logits(c, RSD_TARGET, p, false, s);
+  if (rc) return rc;
+  if (c->dbg_logits[1]) {
+    RSD_LAUNCH((scatter_logits_sd_kernel), T, 256, 0, s, c->logits, c->st.pass_tok_row, c->st.sd_out_idx, c->dbg_logits[1],
+               m.vocab, c->C, c->st.n_active);
+    CU(launched(1));
+  }
+  SampleArgs a{c->logits, T, m.vocab, c->v_limit, c->cfg.temperature, c->cfg.seed, RSD_TARGET,
+               c->st.pass_tok_row, c->st.pass_tok_pos, nullptr, c->st.n_active, c->sample_best};
+  CU(launch_sample(a, s));
+  CU(launch_sd_accept(c->st, c->sample_best, n_slots, c->lp, s));
+  return RSD_OK;
+}
+
+enum IterKind { kIterDecode = 0, kIterSdPropose = 1, kIterSdVerify = 2 };
+
+int enqueue_iteration(rsd_ctx* c, IterKind kind, int which, int phase, int n_slots, cudaStream_t s) {
+  switch (kind) {
+    case kIterSdPropose: return sd_propose_iteration(c, n_slots, s);
+    case kIterSdVerify: return sd_verify_pass(c, n_slots, s);
+    default: return decode_iteration(c, which, phase, n_slots, s);
+  }
+}
+
+// Captures one iteration of `kind` over n_slots slots into a graph (idle slots are skipped inside the
+// kernels), so that a token costs one graph launch instead of some 300 kernel launches.
+int ensure_decode_graph(rsd_ctx* c, IterKind kind, int which, int phase, int g, int n_slots) {
   const int B = c->st.B;
   if (c->dec_graph[g] && c->dec_graph_B[g] == B) return RSD_OK;
   if (c->dec_graph[g]) { cudaGraphExecDestroy(c->dec_graph[g]); c->dec_graph[g] = nullptr; }
@@ -593,7 +670,7 @@ int ensure_decode_graph(rsd_ctx* c, int which, int phase, int g, int n_slots) {
   CU(cudaStreamBeginCapture(c->cap_stream, cudaStreamCaptureModeThreadLocal));
   const bool was_in_decode = c->in_decode, was_timed = c->time_this_iter;
   c->in_decode = true; c->time_this_iter = false;          // no event records inside the capture
-  const int rc = decode_iteration(c, which, phase, n_slots, c->cap_stream);
+  const int rc = enqueue_iteration(c, kind, which, phase, n_slots, c->cap_stream);
   c->in_decode = was_in_decode; c->time_this_iter = was_timed;
   cudaGraph_t graph = nullptr;
   cudaError_t e = cudaStreamEndCapture(c->cap_stream, &graph);
@@ -631,7 +708,7 @@ int decode_phase(rsd_ctx* c, int which, int phase, int n_slots, cudaStream_t s) 
     // the iteration is captured once and replayed
     const bool have_graph = graphs && c->dec_graph[g] && c->dec_graph_B[g] == c->st.B;
     if (graphs && !have_graph && j > 0) {
-      rc = ensure_decode_graph(c, which, phase, g, n_slots);
+      rc = ensure_decode_graph(c, kIterDecode, which, phase, g, n_slots);
       if (rc) break;
     }
     if (graphs && !timed_iter && c->dec_graph[g] && c->dec_graph_B[g] == c->st.B) {
@@ -648,6 +725,45 @@ int decode_phase(rsd_ctx* c, int which, int phase, int n_slots, cudaStream_t s) 
       rc = read_scalars(c, s, &sc);
       if (rc == RSD_OK && sc.n_active == 0) break;
     }
+  }
+  c->in_decode = false;
+  c->attn_rows_hint = 0;
+  return rc;
+}
+
+// The target phase with speculative decoding: rounds of sd_k proposal iterations of the draft and one pass of the
+// target over all of them, until every waiting row's step has ended.  A round writes at least one token per row, so
+// there are at most C rounds; the host looks at the number of unfinished rows after each.  The first round runs
+// kernel by kernel, the following ones replay two captured graphs (proposal iteration, target pass) per bucket.
+int decode_phase_sd(rsd_ctx* c, int n_slots, cudaStream_t s) {
+  CU(launch_decode_begin(c->st, 1, s));
+  if (n_slots <= 0) return RSD_OK;
+  const bool graphs = !(c->cfg.debug_flags & RSD_DEBUG_NO_GRAPHS);
+  int bucket = 0, rows_eff = c->st.B;
+  while (bucket < 3 && n_slots * 2 <= rows_eff) { rows_eff = (rows_eff + 1) / 2; ++bucket; }
+  if (graphs) n_slots = rows_eff;
+  c->in_decode = true;
+  int rc = RSD_OK;
+  auto run = [&](IterKind kind, int g, bool direct) -> int {
+    c->attn_rows_hint = kind == kIterSdVerify ? rows_eff * c->sd_k : rows_eff;
+    if (graphs && !direct) {
+      int r = ensure_decode_graph(c, kind, kind == kIterSdVerify ? RSD_TARGET : RSD_DRAFT, 1, g, n_slots);
+      if (r) return r;
+      cudaError_t e = cudaGraphLaunch(c->dec_graph[g], s);
+      if (e != cudaSuccess) { c->in_decode = false; CU(e); }
+      note_replayed_launches(c->dec_graph_kernels[g]);
+      return RSD_OK;
+    }
+    return enqueue_iteration(c, kind, 0, 1, n_slots, s);
+  };
+  for (int round = 0; round < c->C && rc == RSD_OK; ++round) {
+    const bool direct = round == 0;
+    for (int j = 0; j < c->sd_k && rc == RSD_OK; ++j) rc = run(kIterSdPropose, 8 + bucket, direct);
+    if (rc == RSD_OK) rc = run(kIterSdVerify, 12 + bucket, direct);
+    if (rc != RSD_OK) break;
+    Scalars sc;
+    rc = read_scalars(c, s, &sc);
+    if (rc == RSD_OK && sc.n_active == 0) break;
   }
   c->in_decode = false;
   c->attn_rows_hint = 0;
@@ -676,6 +792,7 @@ int clear_forcing(rsd_ctx* c, cudaStream_t s) {
   CU(cudaMemsetAsync(c->st.forced_len[0], 0, sizeof(int32_t) * c->B_max, s));
   CU(cudaMemsetAsync(c->st.forced_len[1], 0, sizeof(int32_t) * c->B_max, s));
   CU(cudaMemsetAsync(c->st.forced_accept, 255, c->B_max, s));
+  CU(cudaMemsetAsync(c->st.sd_forced_on, 0, c->B_max, s));
   return RSD_OK;
 }
 
@@ -793,7 +910,7 @@ int rsd_load_models(rsd_ctx* c, const rsd_model* draft, const rsd_model* prm, co
     CU(launch_rope_table(c->mdl[w].rope, c->S, c->mdl[w].m.head_dim, c->mdl[w].m.rope_theta, s));
   CU(cudaMemsetAsync(c->d_scalars, 0, 16 * sizeof(int32_t), s));
   CU(cudaMemsetAsync(c->gemm_scratch, 0, c->gemm_scratch_bytes, s));
-  CU(cudaMemsetAsync(c->sample_best, 0, sizeof(unsigned long long) * c->B_max, s));
+  CU(cudaMemsetAsync(c->sample_best, 0, sizeof(unsigned long long) * c->slots_max, s));
   CU(cudaMemsetAsync(c->mega_sync, 0, sizeof(int32_t) * 1024, s));
   int rc = clear_forcing(c, s);
   if (rc) return rc;
@@ -929,7 +1046,7 @@ static int step_impl(rsd_ctx* c, float delta, int min_target_rows, void* cuda_st
   PHASE(4);
   if (target_runs && (rc = run_ingest(c, RSD_TARGET, n_catch, false, s))) return rc;
   PHASE(5);
-  if (target_runs && (rc = decode_phase(c, RSD_TARGET, 1, n_rej, s))) return rc;
+  if (target_runs && (rc = c->sd_k > 0 ? decode_phase_sd(c, n_rej, s) : decode_phase(c, RSD_TARGET, 1, n_rej, s))) return rc;
   PHASE(6);
   // commit and read the results back
   CU(launch_commit(c->st, c->lp, target_runs ? 1 : 0, c->o_tokens, c->o_len, c->o_rewards, c->o_accept, c->o_live,
@@ -981,6 +1098,9 @@ static int step_impl(rsd_ctx* c, float delta, int min_target_rows, void* cuda_st
   c->ctr.score_tokens += merged ? n_scored : gen_d;   // merged PRM: one token per scored step
   c->ctr.steps += n_acc + n_tgt; c->ctr.accepted_steps += n_acc; c->ctr.rejected_steps += n_tgt;
   c->ctr.discarded_draft_tokens += discarded;
+  // speculative decoding of rejected steps: the device keeps running totals since the last reset
+  c->ctr.sd_rounds = (uint64_t)sc.sd_rounds; c->ctr.sd_proposed = (uint64_t)sc.sd_proposed;
+  c->ctr.sd_matched = (uint64_t)sc.sd_matched; c->ctr.sd_verified = (uint64_t)sc.sd_proposed;
   if (step_tokens) memcpy(step_tokens, h_tokens, sizeof(int32_t) * (size_t)B * c->C);
   if (step_len) memcpy(step_len, h_len, sizeof(int32_t) * B);
   if (rewards) memcpy(rewards, h_rew, sizeof(float) * B);
@@ -1005,10 +1125,12 @@ int rsd_flops_counters(rsd_ctx* c, rsd_counters* out) {
   if (!c->loaded) return fail(c, RSD_ERR_STATE, "no models loaded%s");
   rsd_counters r = c->ctr;
   const double nd = c->mdl[RSD_DRAFT].n_params, np = c->mdl[RSD_PRM].n_params, nt = c->mdl[RSD_TARGET].n_params;
-  r.flops_paper = 2.0 * nd * (double)r.gen_tokens[RSD_DRAFT] + 2.0 * nt * (double)r.gen_tokens[RSD_TARGET] +
+  // with speculative decoding the draft is billed its proposals too and the target every position it evaluated
+  const double target_tokens = c->sd_k > 0 ? (double)r.sd_verified : (double)r.gen_tokens[RSD_TARGET];
+  r.flops_paper = 2.0 * nd * (double)(r.gen_tokens[RSD_DRAFT] + r.sd_proposed) + 2.0 * nt * target_tokens +
                   2.0 * np * (double)(r.score_tokens + r.ingest_tokens[RSD_PRM]);
-  r.flops_all_tokens = 2.0 * nd * (double)(r.gen_tokens[RSD_DRAFT] + r.ingest_tokens[RSD_DRAFT]) +
-                       2.0 * nt * (double)(r.gen_tokens[RSD_TARGET] + r.ingest_tokens[RSD_TARGET]) +
+  r.flops_all_tokens = 2.0 * nd * (double)(r.gen_tokens[RSD_DRAFT] + r.sd_proposed + r.ingest_tokens[RSD_DRAFT]) +
+                       2.0 * nt * (target_tokens + (double)r.ingest_tokens[RSD_TARGET]) +
                        2.0 * np * (double)(r.score_tokens + r.ingest_tokens[RSD_PRM]);
   *out = r;
   return RSD_OK;
@@ -1045,6 +1167,16 @@ int rsd_debug_force(rsd_ctx* c, int which, const int32_t* tokens, const int32_t*
   const int p = which == RSD_DRAFT ? 0 : 1;
   CU(cudaMemcpy(c->st.forced_tok[p], tokens, sizeof(int32_t) * (size_t)B * c->C, cudaMemcpyHostToDevice));
   CU(cudaMemcpy(c->st.forced_len[p], len, sizeof(int32_t) * B, cudaMemcpyHostToDevice));
+  return RSD_OK;
+}
+
+int rsd_debug_force_sd(rsd_ctx* c, const int32_t* props, const uint8_t* on) {
+  if (!c || !props || !on) return RSD_ERR_ARG;
+  if (!c->prefilled) return fail(c, RSD_ERR_STATE, "forcing needs rows%s");
+  if (!c->st.sd_forced_props) return fail(c, RSD_ERR_STATE, "needs sd_tokens > 0 and RSD_DEBUG_KEEP_LOGITS%s");
+  const int B = c->st.B;
+  CU(cudaMemcpy(c->st.sd_forced_props, props, sizeof(int32_t) * (size_t)B * c->C * c->sd_k, cudaMemcpyHostToDevice));
+  CU(cudaMemcpy(c->st.sd_forced_on, on, B, cudaMemcpyHostToDevice));
   return RSD_OK;
 }
 

@@ -201,6 +201,13 @@ struct RowState {
   int32_t *err;                // first error raised on the device
   int32_t *pass_tok_id, *pass_tok_row, *pass_tok_pos;  // flat pass lists
   int pass_capacity;
+  // speculative decoding of rejected steps (sd_k proposals per round; 0 = off)
+  int sd_k;
+  int32_t* sd_stats;           // [5] rounds, proposed tokens, matched tokens (summed over rows since the last reset),
+                               // index of the running round, index of the next proposal within it
+  int32_t* sd_out_idx;         // [slots * sd_k] per verify slot: index of its token within the row's step, or -1
+  int32_t* sd_forced_props;    // null, or [B][C][sd_k]: proposals imposed on the draft (parity hook), by row, round, index
+  uint8_t* sd_forced_on;       // [B] 1: row b takes its proposals from sd_forced_props
 };
 
 enum ReserveMode { kReservePrefillDraft, kReservePrefillPrm, kReserveStepDraft, kReserveScorePrm, kReserveTarget };
@@ -230,6 +237,17 @@ cudaError_t launch_decode_prepare(const RowState& st, int which, int n_slots, cu
 cudaError_t launch_decode_update(const RowState& st, int which, int phase, unsigned long long* best,
                                  int n_slots, const LoopParams& lp, cudaStream_t s);
 cudaError_t launch_gate(const RowState& st, float delta, const LoopParams& lp, cudaStream_t s);
+// Speculative decoding of the waiting rows' steps (slot i <-> row slot_row[i], as in the target's decode phase).
+// A round: sd_k draft iterations, each bracketed by propose_prepare (slot i feeds the token at the draft's cursor,
+// while the round still has proposals to make for its row) and propose_update (the sampled token becomes proposal j:
+// written after the fed token in the row's buffer, the draft's cursor moves on); then ONE target pass over
+// n_slots * sd_k token slots laid out by verify_prepare (slot i * sd_k + j feeds the j-th token from the target's
+// cursor on; unused slots idle), sampling at every slot, and accept: the target's choices are written one by one
+// while the ones before equalled the proposals; both cursors end at the last written token.
+cudaError_t launch_sd_propose_prepare(const RowState& st, int n_slots, cudaStream_t s);
+cudaError_t launch_sd_propose_update(const RowState& st, unsigned long long* best, int n_slots, cudaStream_t s);
+cudaError_t launch_sd_verify_prepare(const RowState& st, int n_slots, cudaStream_t s);
+cudaError_t launch_sd_accept(const RowState& st, unsigned long long* best, int n_slots, const LoopParams& lp, cudaStream_t s);
 // target_ran: the waiting rows' steps were written by the target in this call.  out_role[b]: bits 0-1 =
 // accept code of this call, bit 2 = the row committed a target step; out_waiting[b]: still waiting.
 cudaError_t launch_commit(const RowState& st, const LoopParams& lp, int target_ran, int32_t* out_tokens,

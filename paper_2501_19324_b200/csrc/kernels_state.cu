@@ -133,7 +133,7 @@ __global__ void __launch_bounds__(1024) decode_begin_kernel(RowState st, int pha
   }
   int total;
   block_exclusive_scan(part, scan, &total);
-  if (b == 0) { st.n_active[0] = total; st.iter[0] = 0; }
+  if (b == 0) { st.n_active[0] = total; st.iter[0] = 0; st.sd_stats[3] = 0; st.sd_stats[4] = 0; }
   const int n_slots = phase == 0 ? st.B : st.n_rej[0];
   if (b == 0) st.n_slots[0] = n_slots;
   if (b < st.B) st.slot_row[b] = phase == 0 ? b : (b < n_slots ? st.rej_idx[b] : -1);
@@ -242,6 +242,158 @@ cudaError_t launch_decode_update(const RowState& st, int which, int phase, unsig
                                  int n_slots, const LoopParams& lp, cudaStream_t s) {
   if (n_slots <= 0) return cudaSuccess;
   RSD_LAUNCH((decode_update_kernel), 1, 1024, 0, s, st, which, phase, best, n_slots, lp);
+  return launched(1);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Speculative decoding of rejected steps (the paper's discussion of combining RSD with speculative decoding:
+// a rejected step is regenerated by draft + target).  Slot i serves row slot_row[i]; gen_len[1][row] tokens
+// of the row's step are written so far; the row's last written token sits at the cursor of both caches.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ int sd_round_tokens(const RowState& st, int row) {
+  // proposals (and evaluated positions) of the running round for this row: up to sd_k, not beyond the step cap
+  return min(st.sd_k, st.C - st.gen_len[1][row]);
+}
+
+__global__ void __launch_bounds__(1024) sd_propose_prepare_kernel(RowState st, int n_slots) {
+  RSD_PDL_SYNC();
+  if (st.n_active[0] == 0) return;
+  const int j = st.sd_stats[4];   // proposal index within the round, kept on the device so one graph serves every j
+  const int i = threadIdx.x;
+  if (i >= n_slots) return;
+  const int row = st.slot_row[i];
+  if (row >= 0 && st.gen_active[row] && j < sd_round_tokens(st, row)) {
+    const int pos = st.kv_len[0][row];
+    st.pass_tok_id[i] = st.tok[(size_t)row * st.S + pos];
+    st.pass_tok_pos[i] = pos;
+    st.pass_tok_row[i] = row;
+  } else {
+    st.pass_tok_row[i] = -1;
+  }
+}
+
+cudaError_t launch_sd_propose_prepare(const RowState& st, int n_slots, cudaStream_t s) {
+  if (n_slots <= 0) return cudaSuccess;
+  RSD_LAUNCH((sd_propose_prepare_kernel), 1, 1024, 0, s, st, n_slots);
+  return launched(1);
+}
+
+__global__ void __launch_bounds__(1024)
+sd_propose_update_kernel(RowState st, unsigned long long* best, int n_slots) {
+  RSD_PDL_SYNC();
+  if (st.n_active[0] == 0) return;
+  const int j = st.sd_stats[4];
+  const int i = threadIdx.x;
+  __syncthreads();                              // every thread has read j
+  if (i == 0) st.sd_stats[4] = j + 1;
+  if (i >= n_slots) return;
+  const int row = st.pass_tok_row[i];
+  const unsigned long long packed = best[i];
+  best[i] = 0ull;
+  if (row < 0) return;
+  int t = packed ? (int)(0xFFFFFFFFu - (uint32_t)(packed & 0xFFFFFFFFull)) : 0;
+  if (st.sd_forced_props != nullptr && st.sd_forced_on[row])
+    t = st.sd_forced_props[((size_t)row * st.C + st.sd_stats[3]) * st.sd_k + j];
+  const int pos = st.pass_tok_pos[i];
+  st.tok[(size_t)row * st.S + pos + 1] = t;     // proposal j of the round; the target's choice replaces it later
+  st.kv_len[0][row] = pos + 1;
+}
+
+cudaError_t launch_sd_propose_update(const RowState& st, unsigned long long* best, int n_slots, cudaStream_t s) {
+  if (n_slots <= 0) return cudaSuccess;
+  RSD_LAUNCH((sd_propose_update_kernel), 1, 1024, 0, s, st, best, n_slots);
+  return launched(1);
+}
+
+// One block; thread i lays out the sd_k token slots of decode slot i.
+__global__ void __launch_bounds__(1024) sd_verify_prepare_kernel(RowState st, int n_slots) {
+  RSD_PDL_SYNC();
+  if (st.n_active[0] == 0) return;
+  const int i = threadIdx.x;
+  if (i >= n_slots) return;
+  const int row = st.slot_row[i];
+  const bool on = row >= 0 && st.gen_active[row];
+  const int kk = on ? sd_round_tokens(st, row) : 0;
+  const int pos0 = on ? st.kv_len[2][row] : 0;
+  const int e = on ? st.gen_len[1][row] : 0;
+  for (int j = 0; j < st.sd_k; ++j) {
+    const int t = i * st.sd_k + j;
+    if (j < kk) {
+      st.pass_tok_id[t] = st.tok[(size_t)row * st.S + pos0 + j];   // the last written token, then the proposals
+      st.pass_tok_pos[t] = pos0 + j;
+      st.pass_tok_row[t] = row;
+      st.sd_out_idx[t] = e + j;
+    } else {
+      st.pass_tok_row[t] = -1;
+      st.sd_out_idx[t] = -1;
+    }
+  }
+}
+
+cudaError_t launch_sd_verify_prepare(const RowState& st, int n_slots, cudaStream_t s) {
+  if (n_slots <= 0) return cudaSuccess;
+  RSD_LAUNCH((sd_verify_prepare_kernel), 1, 1024, 0, s, st, n_slots);
+  return launched(1);
+}
+
+__global__ void __launch_bounds__(1024)
+sd_accept_kernel(RowState st, unsigned long long* best, int n_slots, LoopParams lp) {
+  RSD_PDL_SYNC();
+  if (st.n_active[0] == 0) return;
+  const int i = threadIdx.x;
+  int ended = 0, proposed = 0, matched = 0, rounds = 0;
+  if (i < n_slots) {
+    const int row = st.slot_row[i];
+    const bool on = row >= 0 && st.gen_active[row];
+    if (on) {
+      const int kk = sd_round_tokens(st, row);
+      const int pos0 = st.kv_len[2][row];
+      const int e = st.gen_len[1][row];
+      const int flen = st.forced_len[1][row];
+      const int limit = flen > 0 ? flen : st.C;
+      int n_emit = 0;
+      bool done = false;
+      for (int j = 0; j < kk; ++j) {
+        const unsigned long long packed = best[i * st.sd_k + j];
+        int t = packed ? (int)(0xFFFFFFFFu - (uint32_t)(packed & 0xFFFFFFFFull)) : 0;
+        st.sampled[1][(size_t)row * st.C + e + j] = t;
+        if (flen > 0) t = st.forced_tok[1][(size_t)row * st.C + e + j];
+        const int prop = st.tok[(size_t)row * st.S + pos0 + 1 + j];
+        st.tok[(size_t)row * st.S + pos0 + 1 + j] = t;
+        st.gen_tok[1][(size_t)row * st.C + e + j] = t;
+        ++n_emit;
+        if (ends_step(t, lp) || e + n_emit == limit) done = true;
+        if (t == prop) ++matched;
+        if (done || t != prop) break;
+      }
+      // both caches hold the positions whose input tokens stand: the old last token and all written but the newest
+      st.kv_len[2][row] = pos0 + n_emit;
+      st.kv_len[0][row] = pos0 + n_emit;
+      st.gen_len[1][row] = e + n_emit;
+      if (done) { st.gen_active[row] = 0; ended = 1; }
+      proposed = kk;
+      rounds = 1;
+    }
+    for (int j = 0; j < st.sd_k; ++j) best[i * st.sd_k + j] = 0ull;
+  }
+  __shared__ int sums[4];
+  if (threadIdx.x < 4) sums[threadIdx.x] = 0;
+  __syncthreads();
+  if (rounds) { atomicAdd(&sums[0], rounds); atomicAdd(&sums[1], proposed); atomicAdd(&sums[2], matched); atomicAdd(&sums[3], ended); }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    st.sd_stats[0] += sums[0];
+    st.sd_stats[1] += sums[1];
+    st.sd_stats[2] += sums[2];
+    st.sd_stats[3] += 1;
+    st.sd_stats[4] = 0;
+    st.n_active[0] -= sums[3];
+  }
+}
+
+cudaError_t launch_sd_accept(const RowState& st, unsigned long long* best, int n_slots, const LoopParams& lp, cudaStream_t s) {
+  if (n_slots <= 0) return cudaSuccess;
+  RSD_LAUNCH((sd_accept_kernel), 1, 1024, 0, s, st, best, n_slots, lp);
   return launched(1);
 }
 

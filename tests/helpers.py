@@ -23,7 +23,7 @@ def build_pair(shapes, *, bf16, seed=0, prompts, loop_kwargs, engine_kwargs=None
     B = len(offsets) - 1
     kw = dict(max_batch=B, debug_flags=RSD_DEBUG_KEEP_LOGITS)
     kw.update({k: loop_kwargs[k] for k in ("max_seq_tokens", "max_step_tokens", "max_steps", "step_end_id",
-                                           "eos_id", "step_end_mod", "temperature", "seed") if k in loop_kwargs})
+                                           "eos_id", "step_end_mod", "temperature", "seed", "sd_tokens") if k in loop_kwargs})
     # loop_kwargs may also carry oracle-only settings (omega_kind, omega_b); the engine takes its own
     if merged:
         kw["prm_shares_draft"] = 1
@@ -61,6 +61,10 @@ def parity_step(eng, loop, delta, *, tol_logits, tol_reward, margin_tok, margin_
         if accept_pattern is not None and accept_pattern[b] is not None:
             amb[b] = int(accept_pattern[b])
     eng.force_accept(amb)
+    if loop.cfg.sd_tokens > 0 and any(r is not None for r in o["sd_rounds"]):
+        # speculative decoding of rejected steps: the draft's proposals are imposed too, so that the rounds (and
+        # their counters) are the oracle's even where a proposal was a near tie
+        eng.force_sd_proposals([None if r is None else [rd["props"] for rd in r] for r in o["sd_rounds"]])
     g = eng.step(delta, min_target_rows)
     live_before = (o["step_len"] > 0) | (o["drafted"] > 0) | (o["waiting"] > 0)
     # rewards, gate, outputs
@@ -109,6 +113,7 @@ def compare_counters(eng, loop):
     g, o = eng.counters(), loop.counters
     for k in ("gen_tokens", "ingest_tokens"):
         assert list(g[k]) == list(o[k]), (k, g[k], o[k])
-    for k in ("score_tokens", "steps", "accepted_steps", "rejected_steps", "discarded_draft_tokens"):
+    for k in ("score_tokens", "steps", "accepted_steps", "rejected_steps", "discarded_draft_tokens",
+              "sd_rounds", "sd_proposed", "sd_matched", "sd_verified"):
         assert g[k] == o[k], (k, g[k], o[k])
     assert abs(g["flops_paper"] - loop.flops_paper()) <= 1e-9 * max(1.0, loop.flops_paper())

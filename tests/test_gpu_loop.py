@@ -322,3 +322,66 @@ def test_persistent_decode_kernel_phase_timeline():
     with pytest.raises(RsdError):
         eng.mega_profile(DRAFT)
     eng.close()
+
+
+@pytest.mark.parametrize("shapes,bf16,tol,k", [(TINY, False, TOL32, 3), (MINI, True, TOL16, 4), (TINY, False, TOL32, 1)])
+def test_speculative_decoding_of_rejected_steps(shapes, bf16, tol, k):
+    """sd_tokens = k (the paper's discussion of combining RSD with speculative decoding): the steps of rejected rows
+    are written in rounds of k draft proposals and one target pass.  Step by step against the oracle in the same
+    mode: logits of every written token, tokens, cursors of all three caches (the draft's now follow the target's),
+    pages, the rounds' counters; and the committed sequences equal those of the plain loop."""
+    prompts = ri.prompts(61, 6, 6, 30, shapes[0].vocab)
+    kw = dict(max_step_tokens=7, max_steps=4, max_seq_tokens=96, step_end_id=3, step_end_mod=5, temperature=0.7,
+              seed=6, sd_tokens=k)
+    eng, loop = build_pair(shapes, bf16=bf16, prompts=prompts, loop_kwargs=kw)
+    delta = float(np.median(loop.step(0.0)["rewards"]))
+    eng, loop = build_pair(shapes, bf16=bf16, prompts=prompts, loop_kwargs=kw)
+    _, plain = build_pair(shapes, bf16=bf16, prompts=prompts, loop_kwargs=dict(kw, sd_tokens=0))
+    stats, seen = {}, set()
+    for _ in range(4):
+        g, o = parity_step(eng, loop, delta, stats=stats, **tol)
+        seen |= set(int(a) for a, n in zip(o["accept"], o["step_len"]) if n)
+        plain.step(delta)
+    assert seen == {0, 1}
+    assert [r.z for r in loop.rows] == [r.z for r in plain.rows]
+    compare_counters(eng, loop)
+    c = eng.counters()
+    assert c["sd_rounds"] > 0 and c["sd_verified"] == c["sd_proposed"] >= c["gen_tokens"][2]
+    print("speculative decoding of rejected steps, k =", k, stats, {q: c[q] for q in c if q.startswith("sd_")})
+    eng.close()
+
+
+def test_speculative_rounds_keep_the_matching_prefix_on_gpu():
+    """Proposals planted around the target's true continuation (known from a first, plain run of the oracle): all
+    right, wrong at once, right-right-wrong, a short last round.  The GPU must write the matching prefix plus the
+    target's own token, round by round: tokens, cursors and the round counters against the oracle's."""
+    from oracle.rsd_loop import OracleRSD, LoopConfig
+    shapes = TINY
+    prompts = ri.prompts(62, 3, 5, 12, shapes[0].vocab)
+    kw = dict(max_step_tokens=9, max_steps=1, max_seq_tokens=40, step_end_id=1 << 20, temperature=0.7, seed=5, sd_tokens=4)
+    _, probe = build_pair(shapes, bf16=False, prompts=prompts, loop_kwargs=dict(kw, sd_tokens=0))
+    truth = [list(y) for y in probe.step(2.0)["step_tokens"]]          # delta above the range: the target's steps
+    bad = lambda t: (t + 1) % 1024
+    planted = []
+    for b in range(3):
+        t = truth[b]
+        planted.append([t[0:4], [bad(t[4]), 7, 7, 7], [t[5], t[6], bad(t[7]), t[8]], [t[8]]])
+    planted[2] = None                                                   # row 2 keeps the draft's own proposals
+    eng, loop = build_pair(shapes, bf16=False, prompts=prompts, loop_kwargs=kw)
+    o = loop.step(2.0, forced_sd_props=planted)
+    eng.force_tokens(0, o["draft_tokens"])
+    eng.force_tokens(2, o["target_tokens"])
+    eng.force_sd_proposals([None if r is None else [rd["props"] for rd in r] for r in o["sd_rounds"]])
+    g = eng.step(2.0)
+    for b in range(3):
+        assert g["step_tokens"][b].tolist() == truth[b] == list(o["step_tokens"][b])
+    for b in range(2):
+        assert [(rd["emitted"], rd["matched"]) for rd in o["sd_rounds"][b]] == [(4, 4), (1, 0), (3, 2), (1, 1)]
+    from helpers import compare_state
+    compare_state(eng, loop)
+    compare_counters(eng, loop)
+    smp = eng.sampled(2)
+    for b in range(3):                                   # the target's own choices were the truth everywhere
+        clear = [j for j in range(9) if o["target_trace"][b]["margin"][j] > 1e-3]
+        assert [smp[b, j] for j in clear] == [truth[b][j] for j in clear]
+    eng.close()
