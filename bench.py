@@ -232,6 +232,8 @@ def workload_config(args) -> dict:
             "prm": "head on the draft's trunk (prm_shares_draft)" if getattr(args, "merged_prm", False) else "separate model",
             "schedule": "lock-step rsd_step" if getattr(args, "queue", 1) == 1 else
                         f"rsd_step_queued, target pass once {args.queue} rows wait",
+            "rejected_steps": "target decoding" if not getattr(args, "sd", 0) else
+                              f"speculative decoding, {args.sd} draft proposals per target pass",
             "l2": "weights and KV read per decode iteration exceed the 126 MB L2 (no flush needed)"}
 
 
@@ -277,7 +279,7 @@ def mega_phase_table(eng, which: int, n_layers: int) -> dict:
     return out
 
 
-def decode_iteration_roofline(phases, iters, kv_bytes, steps, shapes, hbm, queue):
+def decode_iteration_roofline(phases, iters, kv_bytes, steps, shapes, hbm, queue, sd=0):
     """Whole decode iterations against the HBM roofline.  One iteration of model X is one replay of its captured
     graph (every layer, the lm head, sampling).  Algorithmic bytes of an iteration: every layer's weights and the
     lm head once (the embedding table is gathered, not streamed) plus the keys and values of every attended
@@ -292,7 +294,7 @@ def decode_iteration_roofline(phases, iters, kv_bytes, steps, shapes, hbm, queue
         sh = shapes[slot]
         weight_bytes = 2.0 * (sh.n_params() - sh.vocab * sh.d_model)       # bf16; the embedding table is not streamed
         n = iters[name]
-        if n <= 0 or phases.get(key, 0) <= 0:
+        if n <= 0 or phases.get(key, 0) <= 0 or (sd and name == "target"):   # rounds of speculative decoding are not iterations
             out[name] = None
             continue
         ms = phases[key] * steps / n
@@ -339,7 +341,7 @@ def run_ours(args, rank: int, world: int):
     S = hi + n_steps * cap
     eng = Engine(*models, max_batch=B, max_seq_tokens=S, max_step_tokens=cap, max_steps=n_steps + 1,
                  step_end_id=13, temperature=0.7, seed=0, kv_extended=kv_extended(args),
-                 prm_shares_draft=int(merged), debug_flags=debug_flags(args))
+                 prm_shares_draft=int(merged), debug_flags=debug_flags(args), sd_tokens=args.sd)
     tokens, offsets = rank_prompts(rank, B, lo, hi, shapes[0].vocab)
     pinned_tokens = torch.from_numpy(tokens).pin_memory()
 
@@ -450,7 +452,7 @@ def run_ours(args, rank: int, world: int):
 
     if rank == 0:
         hbm, tf, how = peaks()
-        dec = decode_iteration_roofline(phases, iters, kv_bytes, args.steps, shapes, hbm, args.queue)
+        dec = decode_iteration_roofline(phases, iters, kv_bytes, args.steps, shapes, hbm, args.queue, args.sd)
         gemm_gbs = gt["bytes"] / (gt["ms"] * 1e-3) / 1e9 if gt["ms"] > 0 else None
         ratio = gemm_traffic_ratio()
         gemm_sub = {"what": "single weight-GEMM launches (decode, scoring, catch-up) in one extra, untimed step: CUDA events "
@@ -506,6 +508,13 @@ def run_ours(args, rank: int, world: int):
                "decode_iteration": dec,
                "flops_paper": counters["flops_paper"], "clocks": clocks,
                "gen_tokens": counters["gen_tokens"]}
+        if args.sd:
+            # speculative decoding of the rejected steps: what the rounds did (random-init draft and target agree on
+            # next to no token, so a round writes about one token: the figure shows the mechanism's cost, not its gain)
+            d_sd = {k: c1[k] - c0[k] for k in ("sd_rounds", "sd_proposed", "sd_matched", "sd_verified")}
+            d_sd["target_tokens"] = c1["gen_tokens"][2] - c0["gen_tokens"][2]
+            d_sd["tokens_per_round"] = d_sd["target_tokens"] / max(1, d_sd["sd_rounds"])
+            out["speculative_decoding"] = d_sd
         if mega_tables is not None:
             out["mega_profile"] = mega_tables
         if world == 1 and not args.no_cpu_baseline:
@@ -674,18 +683,27 @@ def sweep_score(args):
     the PRM-scoring phase of one rsd_step."""
     import torch
     from paper_2501_19324_b200 import Engine, Model
+    from paper_2501_19324_b200 import lib as rb_lib
     _, tf, how = peaks()
-    small_d, small_t, prm = ri.SHAPES["mini_draft"], ri.SHAPES["mini_target"], ri.SHAPES["1.5b"]
+    small_d, small_t = ri.SHAPES["mini_draft"], ri.SHAPES["mini_target"]
+    prm = ri.SHAPES[args.prm_shape]
     models = [Model(small_d, ri.gpu_model_tensors(small_d, 0, 0, True, ri.HEAD_LM), ri.HEAD_LM),
               Model(prm, ri.gpu_model_tensors(prm, 1, 0, True, ri.HEAD_REWARD_SIGMOID), ri.HEAD_REWARD_SIGMOID),
               Model(small_t, ri.gpu_model_tensors(small_t, 2, 0, True, ri.HEAD_LM), ri.HEAD_LM)]
     layer_params = prm.n_params(ri.HEAD_REWARD_SIGMOID) - prm.vocab * prm.d_model
     sampler = _sweep_sampler()
     n_rep = 7
-    for B in (1, 2, 4, 8, 16, 32, 64, 128):
-        eng = Engine(*models, max_batch=B, max_seq_tokens=256 + (n_rep + 2) * 128, max_step_tokens=128, max_steps=n_rep + 2,
+    batches = (1, 2, 4, 8, 16, 32, 64, 128)
+    prompt_len = 256
+    if args.only:
+        # one point, one timed step (the form a launch-list capture of the scoring pass uses): "batch" or "batch,prompt"
+        v = [int(x) for x in args.only.split(",")]
+        batches, n_rep = (v[0],), 1
+        prompt_len = v[1] if len(v) > 1 else 256
+    for B in batches:
+        eng = Engine(*models, max_batch=B, max_seq_tokens=prompt_len + (n_rep + 2) * 128, max_step_tokens=128, max_steps=n_rep + 2,
                      step_end_id=13, temperature=0.7, seed=0)
-        tokens, offsets = ri.prompts(3, B, 256, 256, small_d.vocab)
+        tokens, offsets = ri.prompts(3, B, prompt_len, prompt_len, small_d.vocab)
         eng.prefill(tokens, offsets)
         eng.step(0.0)
         eng.phase_ms(True)
@@ -696,7 +714,7 @@ def sweep_score(args):
             ms_all.append(eng.phase_ms(True)["prm_scoring"])
             # scored tokens sit at positions z .. z + len - 1 of their rows: contraction flops of the layers plus the
             # attention products (QK^T and PV: 4 * H * hd flops per attended position and layer)
-            z0 = 256 + (i + 1) * 128
+            z0 = prompt_len + (i + 1) * 128
             T = int(r["step_len"].sum())
             ctx_sum = sum(int(n) * z0 + int(n) * (int(n) + 1) // 2 for n in r["step_len"])
             flops_all.append(2.0 * layer_params * T + 4.0 * prm.n_layers * prm.n_heads * prm.head_dim * ctx_sum)
@@ -707,7 +725,8 @@ def sweep_score(args):
                           "steps_timed": n_rep, "TFLOPs_algorithmic": flops / ms * 1e-9,
                           "bf16_frac_algorithmic": flops / ms * 1e-9 / tf,
                           "note": "median step; algorithmic flops = 2 * layer parameters * tokens + attention products",
-                          "peak_source": how, "clocks": sampler.summary(lo, sampler.mark())}), flush=True)
+                          "peak_source": how, "clocks": sampler.summary(lo, sampler.mark()),
+                          "library_launches_so_far": int(rb_lib().rsd_debug_launch_count())}), flush=True)
         eng.close()
     sampler.stop()
 
@@ -729,11 +748,16 @@ def main():
                     help="decode with the persistent decode kernel instead of kernel by kernel (not the headline path)")
     ap.add_argument("--mega-profile", action="store_true", dest="mega_profile",
                     help="record and print the phase timeline of the persistent decode kernel's last launches")
+    ap.add_argument("--sd", type=int, default=0,
+                    help="sd_tokens: rejected steps by speculative decoding with this many proposals per round (0 = off, the headline)")
     ap.add_argument("--queue", type=int, default=1,
                     help="min_target_rows of rsd_step_queued (1 = rsd_step, the headline configuration)")
     ap.add_argument("--kv-extended", type=int, default=None, choices=[0, 1, 2], dest="kv_extended",
                     help="KV cache: 0 by model depth (default: hi+lo pairs beyond 48 layers), 1 fp16 hi+lo pairs, 2 plain fp16")
-    ap.add_argument("--only", default="", help="with --sweep gemm: a single M,K,N point, plain launches")
+    ap.add_argument("--only", default="", help="with --sweep gemm: a single M,K,N point, plain launches; with --sweep score: "
+                                               "a single batch[,prompt length], one timed step")
+    ap.add_argument("--prm-shape", default="1.5b", dest="prm_shape", choices=["1.5b", "7b"],
+                    help="with --sweep score: shape of the PRM")
     ap.add_argument("--sweep", default="", choices=["", "gemm", "attn", "gate", "score"],
                     help="kernel sweep on config-2 shapes instead of the step-loop benchmark")
     args = ap.parse_args()

@@ -261,6 +261,15 @@ int rsd_debug_mega_profile(rsd_ctx*, int which, uint64_t* stamps, int32_t capaci
 int rsd_k_gemm(const void* W, const void* x, const void* x_lo, float* y, int32_t M, int32_t N, int32_t K, int32_t dtype,
                int32_t accumulate, int32_t impl, void* scratch, size_t scratch_bytes, void* cuda_stream);
 size_t rsd_k_gemm_scratch_bytes(int32_t M, int32_t N, int32_t K);
+/* Failure path of the tcgen05 GEMM without a fault: launches one CTA of the kernel in a mode in which its copy
+ * engine issues nothing, so the first pipeline stage never fills, the MMA warp's bounded wait (cut to a few thousand
+ * polls here) runs out, the CTA raises the error flag, releases its other warps, frees its tensor memory and
+ * returns with nothing in flight.  Returns RSD_ERR_TIMEOUT (the expected outcome; rsd_last_error(NULL) names the
+ * wait) after clearing the flag, so the same scratch serves rsd_k_gemm afterwards.  W [128, 64] and x [16, 64]
+ * bf16 and y [16, 128] fp32 are DEVICE buffers that are mapped but neither read nor written; scratch as for
+ * rsd_k_gemm with M = 16.  Synchronises the stream.                                                          */
+int rsd_debug_gemm_wait_probe(const void* W, const void* x, float* y, void* scratch, size_t scratch_bytes,
+                              void* cuda_stream);
 
 /* Paged-KV grouped-query decode attention: one query per row.  q [B, H, hd] fp32; kv pool of pages,
  * each page = keys [KV][16 tokens][hd] followed by values transposed [KV][hd][16 tokens], of
@@ -322,7 +331,8 @@ int rsd_k_swiglu(const float* gu, void* out, int32_t T, int32_t F, int32_t dtype
 /* Gate/up projection of the SwiGLU MLP with the nonlinearity in the GEMM epilogue (tcgen05 path, bf16):
  * act[m, f] = silu(g[m, f]) * u[m, f], [g | u] = (x + x_lo)[M, K] * Wgu[2F, K]^T with Wgu rows = Wgate | Wup,
  * written as the split-precision pair act_hi = bf16(act), act_lo = bf16(act - act_hi), both [M, F].
- * F % 64 == 0, K % 8 == 0, 16-byte aligned rows; x_lo must be given.  `scratch`: at least
+ * F % 64 == 0, K % 8 == 0, 16-byte aligned rows.  x_lo and act_lo may both be NULL when M > 128: the operand is
+ * then plain bf16 and only act_hi = bf16(act) is written (half the tensor-core work).  `scratch`: at least
  * rsd_k_gemm_scratch_bytes(M, 2F, K) bytes, zero on first use (it carries the kernel's error flag).
  * RSD_ERR_UNSUPPORTED for other shapes.                                                         */
 int rsd_k_gemm_gu(const void* Wgu, const void* x, const void* x_lo, void* act_hi, void* act_lo, int32_t M, int32_t F,

@@ -55,7 +55,7 @@ class rsd_counters(ctypes.Structure):
 
 EXPORTS = ["rsd_query_sizes", "rsd_create", "rsd_load_models", "rsd_prefill", "rsd_step", "rsd_step_queued", "rsd_flops_counters",
            "rsd_reset", "rsd_destroy", "rsd_last_error", "rsd_debug_force", "rsd_debug_force_sd", "rsd_debug_get_logits",
-           "rsd_debug_get_sampled", "rsd_debug_get_state", "rsd_debug_gemm_timing", "rsd_debug_launch_count", "rsd_debug_mega_profile", "rsd_debug_phase_ms", "rsd_k_gemm", "rsd_k_gemm_scratch_bytes",
+           "rsd_debug_get_sampled", "rsd_debug_get_state", "rsd_debug_gemm_timing", "rsd_debug_launch_count", "rsd_debug_mega_profile", "rsd_debug_phase_ms", "rsd_k_gemm", "rsd_k_gemm_scratch_bytes", "rsd_debug_gemm_wait_probe",
            "rsd_k_attn_decode", "rsd_k_attn_decode_scratch_bytes", "rsd_k_attn_chunk", "rsd_k_gate_compact", "rsd_k_gate_compact_static", "rsd_k_gate_compact_static_error", "rsd_k_rmsnorm",
            "rsd_k_rope", "rsd_k_swiglu", "rsd_k_gemm_gu", "rsd_k_sample", "rsd_k_philox"]
 
@@ -92,6 +92,7 @@ def lib():
         L.rsd_debug_mega_profile.argtypes = [vp, c_int32, vp, c_int32, vp]
         L.rsd_debug_launch_count.restype = c_uint64
         L.rsd_k_gemm.argtypes = [vp, vp, vp, vp, c_int32, c_int32, c_int32, c_int32, c_int32, c_int32, vp, c_size_t, vp]
+        L.rsd_debug_gemm_wait_probe.argtypes = [vp, vp, vp, vp, c_size_t, vp]
         L.rsd_k_gemm_scratch_bytes.argtypes = [c_int32, c_int32, c_int32]
         L.rsd_k_gemm_scratch_bytes.restype = c_size_t
         L.rsd_k_attn_decode.argtypes = [vp, vp, vp, vp, vp, c_int32, c_int32, c_int32, c_int32, c_int32, c_int32,

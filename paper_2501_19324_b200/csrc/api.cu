@@ -65,6 +65,8 @@ struct rsd_ctx {
   int32_t *o_tokens = nullptr, *o_len = nullptr;
   float* o_rewards = nullptr;
   uint8_t *o_accept = nullptr, *o_live = nullptr, *o_role = nullptr, *o_waiting = nullptr;
+  int32_t* o_gen = nullptr;
+  size_t o_block_bytes = 0;
   float* norm_ssq = nullptr;   // [B][chunks] sums of squares of the residual stream (decode path)
   // persistent decode kernel: parameter block per model (draft, target), built for the batch size mega_B
   void* mega_block[3] = {nullptr, nullptr, nullptr};
@@ -88,6 +90,7 @@ struct rsd_ctx {
   int dec_graph_B[16] = {};
   uint64_t dec_graph_kernels[16] = {};
   int sd_k = 0, slots_max = 0;
+
   int attn_rows_hint = 0;      // rows expected to be active in the running decode phase (0: all slots)
   bool time_this_iter = false, in_decode = false;
   // per-phase timing of rsd_step (rsd_debug_phase_ms)
@@ -259,6 +262,8 @@ size_t layout_workspace(const rsd_config& cfg, const rsd_model* const ms[3], rsd
   uint8_t* o_live = TAKE(uint8_t, B);
   uint8_t* o_role = TAKE(uint8_t, B);
   uint8_t* o_waiting = TAKE(uint8_t, B);
+  int32_t* o_gen = TAKE(int32_t, 2 * (size_t)B);   // tokens each row generated in the draft / target phase of the call
+  const size_t o_end = L.bytes;                    // the step's outputs form one block [o_tokens, o_end): one copy
   const size_t gs = gemm_scratch_bytes_any();
   void* gscr = TAKE(char, gs);
   int h_max = 0;
@@ -283,7 +288,8 @@ size_t layout_workspace(const rsd_config& cfg, const rsd_model* const ms[3], rsd
     c->dbg_logits[0] = dbg[0]; c->dbg_logits[1] = dbg[1];
     c->d_scalars = scal;
     c->o_tokens = o_tokens; c->o_len = o_len; c->o_rewards = o_rewards; c->o_accept = o_accept; c->o_live = o_live;
-    c->o_role = o_role; c->o_waiting = o_waiting;
+    c->o_role = o_role; c->o_waiting = o_waiting; c->o_gen = o_gen;
+    c->o_block_bytes = o_end - (size_t)((char*)o_tokens - base);
     c->gemm_scratch = gscr; c->gemm_scratch_bytes = gs;
     c->attn_scratch = ascr; c->attn_scratch_bytes = as;
   }
@@ -833,7 +839,8 @@ int rsd_create(const rsd_config* cfg, rsd_ctx** out) {
   rsd_ctx* c = new (std::nothrow) rsd_ctx();
   if (!c) return fail(nullptr, RSD_ERR_ARG, "out of host memory%s");
   c->cfg = *cfg;
-  c->pinned_bytes = 4096 + (size_t)cfg->max_batch * (cfg->max_step_tokens * 4 + 64);
+  // scalars, then a mirror of the step's output block (every array of it rounded up to 256 bytes)
+  c->pinned_bytes = 4096 + (size_t)cfg->max_batch * (cfg->max_step_tokens * 4 + 64) + 16 * 256;
   if (cudaHostAlloc((void**)&c->pinned, c->pinned_bytes, cudaHostAllocDefault) != cudaSuccess) {
     delete c;
     return fail(nullptr, RSD_ERR_CUDA, "pinned host allocation failed%s");
@@ -1050,26 +1057,21 @@ static int step_impl(rsd_ctx* c, float delta, int min_target_rows, void* cuda_st
   PHASE(6);
   // commit and read the results back
   CU(launch_commit(c->st, c->lp, target_runs ? 1 : 0, c->o_tokens, c->o_len, c->o_rewards, c->o_accept, c->o_live,
-                   c->o_role, c->o_waiting, s));
+                   c->o_role, c->o_waiting, c->o_gen, s));
+  // one device-to-host copy brings the whole output block; the arrays sit in it at their workspace offsets
   char* hp = c->pinned + 256;
-  int32_t* h_tokens = (int32_t*)hp; hp += sizeof(int32_t) * (size_t)B * c->C;
-  int32_t* h_len = (int32_t*)hp; hp += sizeof(int32_t) * B;
-  int32_t* h_gen0 = (int32_t*)hp; hp += sizeof(int32_t) * B;
-  int32_t* h_gen1 = (int32_t*)hp; hp += sizeof(int32_t) * B;
-  float* h_rew = (float*)hp; hp += sizeof(float) * B;
-  uint8_t* h_acc = (uint8_t*)hp; hp += B;
-  uint8_t* h_live = (uint8_t*)hp; hp += B;
-  uint8_t* h_role = (uint8_t*)hp; hp += B;
-  uint8_t* h_wait = (uint8_t*)hp; hp += B;
-  CU(cudaMemcpyAsync(h_tokens, c->o_tokens, sizeof(int32_t) * (size_t)B * c->C, cudaMemcpyDeviceToHost, s));
-  CU(cudaMemcpyAsync(h_len, c->o_len, sizeof(int32_t) * B, cudaMemcpyDeviceToHost, s));
-  CU(cudaMemcpyAsync(h_gen0, c->st.gen_len[0], sizeof(int32_t) * B, cudaMemcpyDeviceToHost, s));
-  CU(cudaMemcpyAsync(h_gen1, c->st.gen_len[1], sizeof(int32_t) * B, cudaMemcpyDeviceToHost, s));
-  CU(cudaMemcpyAsync(h_rew, c->o_rewards, sizeof(float) * B, cudaMemcpyDeviceToHost, s));
-  CU(cudaMemcpyAsync(h_acc, c->o_accept, B, cudaMemcpyDeviceToHost, s));
-  CU(cudaMemcpyAsync(h_live, c->o_live, B, cudaMemcpyDeviceToHost, s));
-  CU(cudaMemcpyAsync(h_role, c->o_role, B, cudaMemcpyDeviceToHost, s));
-  CU(cudaMemcpyAsync(h_wait, c->o_waiting, B, cudaMemcpyDeviceToHost, s));
+  if (256 + c->o_block_bytes > c->pinned_bytes) return fail(c, RSD_ERR_STATE, "output mirror too small%s");
+  CU(cudaMemcpyAsync(hp, c->o_tokens, c->o_block_bytes, cudaMemcpyDeviceToHost, s));
+  auto mirror = [&](const void* dev) { return hp + ((const char*)dev - (const char*)c->o_tokens); };
+  const int32_t* h_tokens = (const int32_t*)mirror(c->o_tokens);
+  const int32_t* h_len = (const int32_t*)mirror(c->o_len);
+  const int32_t* h_gen0 = (const int32_t*)mirror(c->o_gen);
+  const int32_t* h_gen1 = h_gen0 + B;
+  const float* h_rew = (const float*)mirror(c->o_rewards);
+  const uint8_t* h_acc = (const uint8_t*)mirror(c->o_accept);
+  const uint8_t* h_live = (const uint8_t*)mirror(c->o_live);
+  const uint8_t* h_role = (const uint8_t*)mirror(c->o_role);
+  const uint8_t* h_wait = (const uint8_t*)mirror(c->o_waiting);
   if ((rc = clear_forcing(c, s))) return rc;
   PHASE(7);
 #undef PHASE
@@ -1143,6 +1145,7 @@ int rsd_destroy(rsd_ctx* c) {
   for (cudaEvent_t e : c->ph_ev) if (e) cudaEventDestroy(e);
   for (auto& g : c->dec_graph) if (g) cudaGraphExecDestroy(g);
   if (c->cap_stream) cudaStreamDestroy(c->cap_stream);
+
   if (c->pinned) cudaFreeHost(c->pinned);
   delete c;
   return RSD_OK;
@@ -1286,6 +1289,19 @@ int rsd_k_gemm(const void* W, const void* x, const void* x_lo, float* y, int32_t
   return RSD_OK;
 }
 
+int rsd_debug_gemm_wait_probe(const void* W, const void* x, float* y, void* scratch, size_t scratch_bytes, void* cuda_stream) {
+  if (!W || !x || !y || !scratch || scratch_bytes < gemm_scratch_bytes(16)) return RSD_ERR_ARG;
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  KCU(launch_gemm_wait_probe(W, x, y, scratch, scratch_bytes, s));
+  int32_t flag = 0;
+  KCU(cudaMemcpyAsync(&flag, (char*)scratch + 4096, sizeof(flag), cudaMemcpyDeviceToHost, s));
+  KCU(cudaStreamSynchronize(s));
+  if (flag == 0) return RSD_OK;                       // the wait did not run out: not what the probe is for
+  KCU(cudaMemsetAsync((char*)scratch + 4096, 0, sizeof(flag), s));   // the scratch is usable again
+  g_create_error = "a bounded wait inside the tensor-core GEMM expired";
+  return RSD_ERR_TIMEOUT;
+}
+
 size_t rsd_k_attn_decode_scratch_bytes(int32_t B, int32_t H, int32_t hd, int32_t max_ctx) {
   return attn_decode_scratch_bytes(B, H, hd, max_ctx);
 }
@@ -1345,8 +1361,10 @@ int rsd_k_swiglu(const float* gu, void* out, int32_t T, int32_t F, int32_t dtype
 
 int rsd_k_gemm_gu(const void* Wgu, const void* x, const void* x_lo, void* act_hi, void* act_lo, int32_t M, int32_t F,
                   int32_t K, void* scratch, size_t scratch_bytes, void* cuda_stream) {
-  if (!Wgu || !x || !x_lo || !act_hi || !act_lo || M < 0 || F < 1 || K < 1) return RSD_ERR_ARG;
+  if (!Wgu || !x || !act_hi || M < 0 || F < 1 || K < 1) return RSD_ERR_ARG;
+  if ((x_lo == nullptr) != (act_lo == nullptr)) return RSD_ERR_ARG;      // plain operand in, plain operand out
   if (!gemm_gu_supported(RSD_BF16, M > 0 ? M : 1, F, K)) return RSD_ERR_UNSUPPORTED;
+  if (x_lo == nullptr && M <= 128) return RSD_ERR_UNSUPPORTED;
   if (!scratch || scratch_bytes < gemm_scratch_bytes(M)) return RSD_ERR_ARG;
   KCU(launch_gemm_gu(Wgu, x, x_lo, act_hi, act_lo, M, F, K, scratch, scratch_bytes, nullptr, (cudaStream_t)cuda_stream));
   return RSD_OK;

@@ -71,7 +71,11 @@ template <int MT, bool DEEP = false> struct TcCfg {
 // epilogue writes act = silu(gate) * up as the bf16 hi + lo operand pair [M, N] of the down projection instead
 // of Y.  The gate values sit in TMEM lanes 0-63 (warps 0, 1), the up values in lanes 64-127 (warps 2, 3); the
 // two warp pairs swap one half of the x rows each through shared memory, so all four warps compute.
-template <int MT, bool SPLIT, bool GU = false, bool DEEP = false>
+// PROBE (one instantiation, reached only through the wait-probe entry): the producer warp issues NO copy, so the
+// first stage never fills; the MMA warp's wait, cut to a few thousand polls, runs out, and the kernel must take its
+// failure path -- error flag raised, epilogue warps released, tensor memory freed, clean return -- with nothing in
+// flight.  This is how the failure path is exercised without a fault or an endless wait.
+template <int MT, bool SPLIT, bool GU = false, bool DEEP = false, bool PROBE = false>
 __global__ void __launch_bounds__(192, TcCfg<MT, DEEP>::kCtasPerSm)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x,
                const __grid_constant__ CUtensorMap tm_x_lo, float* __restrict__ Y,
@@ -129,7 +133,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
 
   if (warp == 4) {
     // ---------------- TMA producer ----------------
-    if (lane == 0) {
+    if (lane == 0 && !PROBE) {
       int issued = 0;
       bool ok = true;
       // weight tiles of the first ring of stages go out before the predecessors have finished
@@ -189,7 +193,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
       bool ok = true;
       for (int i = 0; i < n_kb; ++i) {
         const int s = i % Cfg::kStages;
-        ok = mbar_wait(&full[s], (i / Cfg::kStages) & 1);
+        ok = mbar_wait(&full[s], (i / Cfg::kStages) & 1, PROBE ? 4096u : kWaitLimit);
         if (!ok || flags[0]) { ok = false; break; }
         tc_fence_after();
         const uint32_t a = smem_u32(smem + (size_t)s * Cfg::kStageBytes);
@@ -304,12 +308,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
             if (c + j < m_valid) v[j] *= row_scale[c + j];
         }
         if (n < N) {
+          // when adding into y, all sixteen old values are requested before the first store: written as
+          // "*y += v" row by row, every load would wait for the store before it (the compiler cannot rule out
+          // that two rows alias) and the epilogue would crawl at one memory round trip per element
+          if (accumulate && splits == 1) {
+            float old[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) old[j] = c + j < m_valid ? dst[(size_t)(m0 + c + j) * N + n] : 0.f;
+#pragma unroll
+            for (int j = 0; j < 16; ++j) v[j] += old[j];
+          }
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
-            if (c + j < m_valid) {
-              float* y = dst + (size_t)(m0 + c + j) * N + n;
-              *y = (accumulate && splits == 1) ? (*y + v[j]) : v[j];
-            }
+            if (c + j < m_valid) dst[(size_t)(m0 + c + j) * N + n] = v[j];
           }
         }
       }
@@ -464,12 +475,17 @@ gemm_tc_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid
               for (int j = 0; j < 16; ++j) v[j] += w[j];
             }
             if (n < N) {
+              // all sixteen old values first, then the stores (see the one-tile kernel's epilogue)
+              if (accumulate) {
+                float old[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) old[j] = c + j < m_valid ? Y[(size_t)(m0 + c + j) * N + n] : 0.f;
+#pragma unroll
+                for (int j = 0; j < 16; ++j) v[j] += old[j];
+              }
 #pragma unroll
               for (int j = 0; j < 16; ++j) {
-                if (c + j < m_valid) {
-                  float* y = Y + (size_t)(m0 + c + j) * N + n;
-                  *y = accumulate ? (*y + v[j]) : v[j];
-                }
+                if (c + j < m_valid) Y[(size_t)(m0 + c + j) * N + n] = v[j];
               }
             }
           }
@@ -687,6 +703,26 @@ cudaError_t launch_mt(const CUtensorMap& tw, const CUtensorMap& tx, const CUtens
 // Row-major bf16 matrix [rows, cols] as a TMA tensor map with a 64-column x box_rows box under the 128-byte swizzle.
 bool tc_tensor_map(const void* ptr, int rows, int cols, int box_rows, CUtensorMap* out) {
   return get_map(ptr, rows, cols, box_rows, out);
+}
+
+// Launches the PROBE instantiation on a 128 x 16 x 64 problem whose copies are never issued (W and x are mapped but
+// not read): the kernel's bounded wait expires and *err (the int at byte 4096 of the scratch) becomes -5.
+cudaError_t launch_gemm_wait_probe(const void* W, const void* x, float* y, void* scratch, size_t scratch_bytes, cudaStream_t s) {
+  if (!scratch || scratch_bytes < gemm_scratch_bytes(16)) return cudaErrorInvalidValue;
+  CUtensorMap tw, tx;
+  if (!get_map(W, 128, 64, kTileN, &tw) || !get_map(x, 16, 64, 16, &tx)) return cudaErrorNotSupported;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<16, false, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)TcCfg<16>::kSmemBytes);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  int* err = (int*)((char*)scratch + kCounterBytes);
+  float* partials = (float*)((char*)scratch + kCounterBytes + 256);
+  RSD_LAUNCH((gemm_tc_kernel<16, false, false, false, true>), dim3(1, 1, 1), 192, TcCfg<16>::kSmemBytes, s, tw, tx, tx, y, 16, 128, 64, 0, 1, 1,
+             partials, err, (const int32_t*)nullptr, RowScale(), (__nv_bfloat16*)nullptr, (__nv_bfloat16*)nullptr);
+  return launched(1);
 }
 
 bool gemm_tc_supported(int dtype, int M, int N, int K) {

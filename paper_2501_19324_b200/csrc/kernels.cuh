@@ -74,6 +74,9 @@ cudaError_t launch_gemm_tc(const void* W, const void* x, const void* x_lo, float
                            void* scratch, size_t scratch_bytes, const int32_t* n_active, int* deferred_splits,
                            cudaStream_t s, RowScale rs = RowScale());
 const float* gemm_partials(const void* scratch);
+// Failure-path probe of the tensor-core GEMM: one CTA whose copies are never issued; its bounded wait runs out and
+// the error flag at byte 4096 of the scratch becomes -5.  W [128, 64] and x [16, 64] bf16, y [16, 128] fp32 (untouched).
+cudaError_t launch_gemm_wait_probe(const void* W, const void* x, float* y, void* scratch, size_t scratch_bytes, cudaStream_t s);
 // Gate/up projection with SwiGLU in the epilogue (bf16, split-precision operand): act_hi + act_lo [M, F] =
 // silu(g) * u with [g | u] = rowscale * (x + x_lo)[M, K] * Wgu[2F, K]^T, Wgu rows = Wgate | Wup.  No K split and no
 // fp32 gate/up array: the tile of a CTA is 64 gate rows and the 64 matching up rows.  F % 64 == 0.
@@ -249,9 +252,10 @@ cudaError_t launch_sd_propose_update(const RowState& st, unsigned long long* bes
 cudaError_t launch_sd_verify_prepare(const RowState& st, int n_slots, cudaStream_t s);
 cudaError_t launch_sd_accept(const RowState& st, unsigned long long* best, int n_slots, const LoopParams& lp, cudaStream_t s);
 // target_ran: the waiting rows' steps were written by the target in this call.  out_role[b]: bits 0-1 =
-// accept code of this call, bit 2 = the row committed a target step; out_waiting[b]: still waiting.
+// accept code of this call, bit 2 = the row committed a target step; out_waiting[b]: still waiting;
+// out_gen [2, B]: tokens the draft / the target generated for the row in this call.
 cudaError_t launch_commit(const RowState& st, const LoopParams& lp, int target_ran, int32_t* out_tokens,
                           int32_t* out_len, float* out_rewards, uint8_t* out_accept, uint8_t* out_live,
-                          uint8_t* out_role, uint8_t* out_waiting, cudaStream_t s);
+                          uint8_t* out_role, uint8_t* out_waiting, int32_t* out_gen, cudaStream_t s);
 
 }  // namespace rsd

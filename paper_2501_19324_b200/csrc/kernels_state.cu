@@ -551,7 +551,7 @@ cudaError_t launch_gate_compact_large(const float* rewards, const uint8_t* live,
 // ---------------------------------------------------------------------------------------------
 __global__ void commit_kernel(RowState st, LoopParams lp, int target_ran, int32_t* out_tokens, int32_t* out_len,
                               float* out_rewards, uint8_t* out_accept, uint8_t* out_live, uint8_t* out_role,
-                              uint8_t* out_waiting) {
+                              uint8_t* out_waiting, int32_t* out_gen) {
   RSD_PDL_SYNC();
   const int b = blockIdx.x;
   const bool live = st.live[b] != 0;
@@ -570,6 +570,8 @@ __global__ void commit_kernel(RowState st, LoopParams lp, int target_ran, int32_
   has_eos = __syncthreads_or(has_eos);
   if (threadIdx.x == 0) {
     out_len[b] = n;
+    out_gen[b] = st.gen_len[0][b];
+    out_gen[gridDim.x + b] = st.gen_len[1][b];
     out_rewards[b] = live ? st.rewards[b] : 0.f;
     out_accept[b] = (live && code == 1) ? 1 : 0;
     out_role[b] = (uint8_t)((live ? code : 0) | (phase == 1 ? 4 : 0));
@@ -590,10 +592,10 @@ __global__ void commit_kernel(RowState st, LoopParams lp, int target_ran, int32_
 
 cudaError_t launch_commit(const RowState& st, const LoopParams& lp, int target_ran, int32_t* out_tokens,
                           int32_t* out_len, float* out_rewards, uint8_t* out_accept, uint8_t* out_live,
-                          uint8_t* out_role, uint8_t* out_waiting, cudaStream_t s) {
+                          uint8_t* out_role, uint8_t* out_waiting, int32_t* out_gen, cudaStream_t s) {
   if (st.B <= 0) return cudaSuccess;
   RSD_LAUNCH((commit_kernel), st.B, 128, 0, s, st, lp, target_ran, out_tokens, out_len, out_rewards, out_accept,
-             out_live, out_role, out_waiting);
+             out_live, out_role, out_waiting, out_gen);
   return launched(1);
 }
 

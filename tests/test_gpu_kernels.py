@@ -380,3 +380,28 @@ def test_gate_up_gemm_with_swiglu_epilogue(M, F, K):
         np.abs(a_hi.float().cpu().numpy() - got).max() <= 2 ** -8 * scale
     again_hi, again_lo = rb.k_gemm_gu(dev(W, torch.bfloat16), hi, lo)
     assert torch.equal(again_hi, a_hi) and torch.equal(again_lo, a_lo)
+
+
+def test_bounded_wait_runs_out_and_the_kernel_leaves_cleanly():
+    """RSD_ERR_TIMEOUT without a fault: one CTA of the tensor-core GEMM whose copies are never issued.  Its wait
+    (a few thousand polls in this mode) expires, the error flag is raised and reported, tensor memory is freed: the
+    very next GEMMs on the same scratch are correct, many times over (a leaked allocation would stall them)."""
+    rng = np.random.default_rng(5)
+    W = dev(rng.normal(size=(128, 64)).astype(np.float32), torch.bfloat16)
+    x = dev(rng.normal(size=(16, 64)).astype(np.float32), torch.bfloat16)
+    y = torch.full((16, 128), 7.0, dtype=torch.float32, device="cuda")
+    nbytes = rb.lib().rsd_k_gemm_scratch_bytes(16, 128, 64)
+    scratch = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream().cuda_stream
+    for _ in range(3):
+        rc = rb.lib().rsd_debug_gemm_wait_probe(W.data_ptr(), x.data_ptr(), y.data_ptr(), scratch.data_ptr(), nbytes, stream)
+        assert rc == -5
+        assert b"bounded wait" in rb.lib().rsd_last_error(None)
+        assert int(scratch[4096:4100].view(torch.int32).item()) == 0           # cleared for the next use
+        assert torch.all(y == 7.0)                                             # nothing was computed or written
+    want = oracle.matmul(W.float().cpu().numpy(), x.float().cpu().numpy())
+    for _ in range(40):                                  # 40 x 32 columns: more than the 512 a leak of 3 x 32 would leave
+        got = torch.zeros(16, 128, dtype=torch.float32, device="cuda")
+        assert rb.lib().rsd_k_gemm(W.data_ptr(), x.data_ptr(), None, got.data_ptr(), 16, 128, 64, 1, 0, 2, scratch.data_ptr(),
+                                   nbytes, stream) == 0
+        np.testing.assert_allclose(got.cpu().numpy(), want, rtol=0, atol=3e-4)
