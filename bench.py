@@ -692,7 +692,7 @@ def sweep_score(args):
               Model(small_t, ri.gpu_model_tensors(small_t, 2, 0, True, ri.HEAD_LM), ri.HEAD_LM)]
     layer_params = prm.n_params(ri.HEAD_REWARD_SIGMOID) - prm.vocab * prm.d_model
     sampler = _sweep_sampler()
-    n_rep = 7
+    n_rep = 15                                   # at least 7 timed steps, more while they take under half a second
     batches = (1, 2, 4, 8, 16, 32, 64, 128)
     prompt_len = 256
     if args.only:
@@ -709,7 +709,10 @@ def sweep_score(args):
         eng.phase_ms(True)
         lo = sampler.mark()
         ms_all, flops_all = [], []
+        t_begin = time.perf_counter()
         for i in range(n_rep):
+            if i >= min(7, n_rep) and time.perf_counter() - t_begin > 0.5:
+                break
             r = eng.step(0.0)
             ms_all.append(eng.phase_ms(True)["prm_scoring"])
             # scored tokens sit at positions z .. z + len - 1 of their rows: contraction flops of the layers plus the
@@ -722,7 +725,7 @@ def sweep_score(args):
         k = int(np.argsort(ms_all)[len(ms_all) // 2])
         ms, flops = ms_all[k], flops_all[k]
         print(json.dumps({"sweep": "prm_scoring", "batch": B, "step_tokens": 128, "ms": ms, "ms_min": min(ms_all),
-                          "steps_timed": n_rep, "TFLOPs_algorithmic": flops / ms * 1e-9,
+                          "steps_timed": len(ms_all), "TFLOPs_algorithmic": flops / ms * 1e-9,
                           "bf16_frac_algorithmic": flops / ms * 1e-9 / tf,
                           "note": "median step; algorithmic flops = 2 * layer parameters * tokens + attention products",
                           "peak_source": how, "clocks": sampler.summary(lo, sampler.mark()),

@@ -107,15 +107,16 @@ typedef struct {
                                  scoring pass disappears.  The prm descriptor must repeat the draft's
                                  dimensions and dtype; its layer arrays and kv_pool[RSD_PRM] may be NULL.
                                  Results equal those of a separate PRM whose trunk weights are the draft's */
-  int32_t sd_tokens;          /* k, 0..16.  k > 0: RSD combined with speculative decoding (Section 4, "Combine RSD
-                                 with SD": during a rejected step, draft + target speculative decoding can
-                                 regenerate the step).  The target's step of a rejected row is then written in
-                                 rounds: the draft proposes up to k tokens, the target evaluates its own choice at
-                                 all k positions in ONE pass and the choices are written while every earlier one
-                                 equalled the proposal (at least one, at most k tokens per round).  Sampling
-                                 noise is keyed by (model, row, position), so the step is token for token the
-                                 one plain target decoding writes; only the number of target passes changes.
-                                 The workspace grows with k (logits of k positions per row)                   */
+  int32_t sd_tokens;          /* k, 0..16.  k > 0: RSD combined with speculative decoding (Section 4, discussion
+                                 item on combining RSD with SD: a rejected step, which the target must write
+                                 anyway, is rewritten by draft-then-verify decoding).  The target's step of a
+                                 rejected row is then written in rounds: the draft proposes up to k tokens, the
+                                 target evaluates its own choice at all k positions in ONE pass and the choices
+                                 are written while every earlier one equalled the proposal (at least one, at
+                                 most k tokens per round).  Sampling noise is keyed by (model, row, position), so
+                                 the step is token for token the one plain target decoding writes; only the
+                                 number of target passes changes.  The workspace grows with k (logits of k
+                                 positions per row)                                                           */
   /* caller-allocated device memory, sizes as reported by rsd_query_sizes (or larger)        */
   void* kv_pool[3];           /* RSD_DRAFT / RSD_PRM / RSD_TARGET                            */
   size_t kv_bytes[3];
@@ -254,7 +255,7 @@ int rsd_debug_mega_profile(rsd_ctx*, int which, uint64_t* stamps, int32_t capaci
  * x_lo (bf16 only, may be NULL) is the low half of a split-precision activation: x = bf16(a),
  * x_lo = bf16(a - x), both multiplied on the tensor cores and added, so `a` enters with ~16 bits.
  * impl: 0 = pick by shape, 1 = split-K SIMT GEMV path, 2 = tcgen05/TMEM/TMA path (bf16 only,
- * K % 64 == 0, 16-byte aligned rows).  `scratch` (scratch_bytes from rsd_k_gemm_scratch_bytes)
+ * K % 8 == 0, 16-byte aligned rows), 3 = the same with one CTA per output tile (no split along K).  `scratch` (scratch_bytes from rsd_k_gemm_scratch_bytes)
  * holds split-K partial sums and tile counters; its first 4 KiB + 256 B must be zero before the
  * first call; the counters are left zero by every call and the int at byte 4096 becomes non-zero
  * if a bounded device-side wait of the tcgen05 path expired (RSD_ERR_TIMEOUT condition).                                                      */

@@ -40,8 +40,8 @@ draft step dropped, while the accepted rows go on drafting, until `min_target_ro
 nothing else is left to run); then the target writes y_i for all of them in one pass.  Each row's
 own sequence of steps is the one Algorithm 1 gives it: only the order in time changes.
 
-RSD combined with speculative decoding (`sd_tokens` = k > 0; Section 4, "Combine RSD with SD": a rejected
-step may be regenerated by draft + target speculative decoding instead of by the target alone).  The step
+RSD combined with speculative decoding (`sd_tokens` = k > 0; Section 4, the discussion item on combining
+RSD with SD: the target need not write a rejected step alone, draft + target speculative decoding can).  The step
 of a rejected row is then written in rounds.  In a round the draft proposes up to k tokens after the
 tokens written so far; the target evaluates, in ONE pass over the last written token and all but the
 last proposal, its own choice at each of those positions; the choices are taken one by one while every

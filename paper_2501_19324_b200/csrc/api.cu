@@ -1279,10 +1279,10 @@ size_t rsd_k_gemm_scratch_bytes(int32_t M, int32_t N, int32_t K) {
 
 int rsd_k_gemm(const void* W, const void* x, const void* x_lo, float* y, int32_t M, int32_t N, int32_t K, int32_t dtype,
                int32_t accumulate, int32_t impl, void* scratch, size_t scratch_bytes, void* cuda_stream) {
-  if (!W || !x || !y || M < 0 || N < 1 || K < 1 || (dtype != RSD_F32 && dtype != RSD_BF16) || impl < 0 || impl > 2)
+  if (!W || !x || !y || M < 0 || N < 1 || K < 1 || (dtype != RSD_F32 && dtype != RSD_BF16) || impl < 0 || impl > 3)
     return RSD_ERR_ARG;
   if (K % (dtype == RSD_BF16 ? 8 : 4)) return RSD_ERR_UNSUPPORTED;
-  if (impl == 2 && !gemm_tc_supported(dtype, M, N, K)) return RSD_ERR_UNSUPPORTED;
+  if (impl >= 2 && !gemm_tc_supported(dtype, M, N, K)) return RSD_ERR_UNSUPPORTED;
   if (impl != 1 && (!scratch || scratch_bytes < gemm_scratch_bytes(M))) return RSD_ERR_ARG;
   if (x_lo && dtype != RSD_BF16) return RSD_ERR_ARG;
   KCU(launch_gemm(dtype, W, x, x_lo, y, M, N, K, accumulate, impl, scratch, scratch_bytes, nullptr, nullptr, (cudaStream_t)cuda_stream));

@@ -675,18 +675,19 @@ TcPlan plan_tc(int M, int N, int K, bool split_operand) {
   return p;
 }
 
-template <int MT, bool SPLIT>
+template <int MT, bool SPLIT, bool DEEP = false>
 cudaError_t launch_mt(const CUtensorMap& tw, const CUtensorMap& tx, const CUtensorMap& txl, float* y, int M, int N, int K,
                       int accumulate, const TcPlan& p, float* partials, int* err, const int32_t* n_active,
                       bool defer_reduce, RowScale rs, cudaStream_t s) {
+  using Cfg = TcCfg<MT, DEEP>;
   static bool configured = false;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<MT, SPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TcCfg<MT>::kSmemBytes);
+    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<MT, SPLIT, false, DEEP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::kSmemBytes);
     if (e != cudaSuccess) return e;
     configured = true;
   }
   dim3 grid(p.n_tiles, p.m_tiles, p.splits);
-  RSD_LAUNCH((gemm_tc_kernel<MT, SPLIT>), grid, 192, TcCfg<MT>::kSmemBytes, s, tw, tx, txl, y, M, N, K, accumulate, p.splits,
+  RSD_LAUNCH((gemm_tc_kernel<MT, SPLIT, false, DEEP>), grid, 192, Cfg::kSmemBytes, s, tw, tx, txl, y, M, N, K, accumulate, p.splits,
                                                                      p.kb_per_split, partials, err, n_active, rs,
                                                                      (__nv_bfloat16*)nullptr, (__nv_bfloat16*)nullptr);
   if (p.splits > 1 && !defer_reduce) {
@@ -832,14 +833,15 @@ const float* gemm_partials(const void* scratch) { return (const float*)((const c
 
 cudaError_t launch_gemm_tc(const void* W, const void* x, const void* x_lo, float* y, int M, int N, int K, int accumulate,
                            void* scratch, size_t scratch_bytes, const int32_t* n_active, int* deferred_splits,
-                           cudaStream_t s, RowScale rs) {
+                           cudaStream_t s, RowScale rs, bool no_k_split) {
   if (deferred_splits) *deferred_splits = 1;
   if (M <= 0) return cudaSuccess;
   if (rs.ssq != nullptr && accumulate) return cudaErrorInvalidValue;
   if (!scratch || scratch_bytes < gemm_scratch_bytes(M)) return cudaErrorInvalidValue;
   if (((uintptr_t)W & 15) || ((uintptr_t)x & 15) || ((uintptr_t)x_lo & 15)) return cudaErrorMisalignedAddress;
   const bool split_operand = x_lo != nullptr;
-  const TcPlan p = plan_tc(M, N, K, split_operand);
+  TcPlan p = plan_tc(M, N, K, split_operand);
+  if (no_k_split) { p.splits = 1; p.kb_per_split = (K + kTileK - 1) / kTileK; }
   if (rs.ssq != nullptr && p.rows > 128) return cudaErrorInvalidValue;   // one epilogue thread per x row of the tile
   if (deferred_splits) *deferred_splits = p.splits;
   const bool defer = deferred_splits != nullptr;
@@ -854,6 +856,17 @@ cudaError_t launch_gemm_tc(const void* W, const void* x, const void* x_lo, float
     return launch_persistent<false, false>(tw, tx, txl, y, M, N, K, accumulate, err, nullptr, nullptr, s);
   }
 #define RSD_TC(MT, SP) return launch_mt<MT, SP>(tw, tx, txl, y, M, N, K, accumulate, p, partials, err, n_active, defer, rs, s)
+  // a grid of at most one CTA per SM: the deep ring (a lone CTA needs more bytes in flight to keep its stream going)
+  if (split_operand && p.n_tiles * p.m_tiles * p.splits <= 148 && p.mt <= 128) {
+#define RSD_TCD(MT) return launch_mt<MT, true, true>(tw, tx, txl, y, M, N, K, accumulate, p, partials, err, n_active, defer, rs, s)
+    switch (p.mt) {
+      case 16: RSD_TCD(16);
+      case 32: RSD_TCD(32);
+      case 64: RSD_TCD(64);
+      default: RSD_TCD(128);
+    }
+#undef RSD_TCD
+  }
   if (split_operand) {
     switch (p.mt) {
       case 16: RSD_TC(16, true);
@@ -879,8 +892,8 @@ cudaError_t launch_gemm(int dtype, const void* W, const void* x, const void* x_l
   if (deferred_splits) *deferred_splits = 1;
   const bool tc_ok = gemm_tc_supported(dtype, M, N, K) && scratch && scratch_bytes >= gemm_scratch_bytes(M);
   // the tensor-core path wins for every M (an M = 1 GEMV included: TMA streaming beats the SIMT loads)
-  if (impl == 2 || (impl == 0 && tc_ok))
-    return launch_gemm_tc(W, x, x_lo, y, M, N, K, accumulate, scratch, scratch_bytes, n_active, deferred_splits, s, rs);
+  if (impl == 2 || impl == 3 || (impl == 0 && tc_ok))
+    return launch_gemm_tc(W, x, x_lo, y, M, N, K, accumulate, scratch, scratch_bytes, n_active, deferred_splits, s, rs, impl == 3);
   if (rs.ssq != nullptr) return cudaErrorNotSupported;
   return launch_gemm_simt(dtype, W, x, dtype == 1 ? x_lo : nullptr, y, M, N, K, accumulate, n_active, s);
 }

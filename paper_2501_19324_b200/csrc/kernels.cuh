@@ -72,7 +72,7 @@ size_t gemm_scratch_bytes_any();
 // 1 means y holds the finished result.
 cudaError_t launch_gemm_tc(const void* W, const void* x, const void* x_lo, float* y, int M, int N, int K, int accumulate,
                            void* scratch, size_t scratch_bytes, const int32_t* n_active, int* deferred_splits,
-                           cudaStream_t s, RowScale rs = RowScale());
+                           cudaStream_t s, RowScale rs = RowScale(), bool no_k_split = false);
 const float* gemm_partials(const void* scratch);
 // Failure-path probe of the tensor-core GEMM: one CTA whose copies are never issued; its bounded wait runs out and
 // the error flag at byte 4096 of the scratch becomes -5.  W [128, 64] and x [16, 64] bf16, y [16, 128] fp32 (untouched).
@@ -84,7 +84,7 @@ bool gemm_gu_supported(int dtype, int M, int F, int K);
 cudaError_t launch_gemm_gu(const void* Wgu, const void* x, const void* x_lo, void* act_hi, void* act_lo, int M, int F, int K,
                            void* scratch, size_t scratch_bytes, const int32_t* n_active, cudaStream_t s, RowScale rs = RowScale());
 
-// impl: 0 = by shape, 1 = SIMT split-K GEMV, 2 = tcgen05.
+// impl: 0 = by shape, 1 = SIMT split-K GEMV, 2 = tcgen05, 3 = tcgen05 without a K split.
 cudaError_t launch_gemm(int dtype, const void* W, const void* x, const void* x_lo, float* y, int M, int N, int K,
                         int accumulate, int impl, void* scratch, size_t scratch_bytes, const int32_t* n_active,
                         int* deferred_splits, cudaStream_t s, RowScale rs = RowScale());
