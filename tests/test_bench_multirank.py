@@ -67,11 +67,18 @@ def test_decode_iteration_roofline_arithmetic():
     import rsd_inputs as ri
     shapes = [ri.SHAPES["1.5b"], ri.SHAPES["1.5b"], ri.SHAPES["7b"]]
     phases = {"draft_decode": 256.0, "target_decode": 448.0}          # ms per step
-    r = bench.decode_iteration_roofline(phases, {"draft": 3 * 128, "target": 2 * 128}, 3, shapes, 6538.0, 1)
+    kv = {"draft": 3 * 128 * 1.0e9, "target": 0.0}                    # KV bytes read over all iterations of the phase
+    r = bench.decode_iteration_roofline(phases, {"draft": 3 * 128, "target": 2 * 128}, kv, 3, shapes, 6538.0, 1)
     # 28 layers x 46,792,704 matrix parameters + norm gains + lm head of 151936 x 1536, two bytes each
     want_bytes = 2.0 * (28 * (46_792_704 + 2 * 1536) + 1536 + 151936 * 1536)
     assert abs(r["draft"]["weight_gb"] * 1e9 - want_bytes) < 1.0
     assert abs(r["draft"]["ms"] - 2.0) < 1e-12 and abs(r["target"]["ms"] - 5.25) < 1e-12
-    assert abs(r["draft"]["frac_of_hbm"] - want_bytes / 2.0e-3 / 1e9 / 6538.0) < 1e-9
-    assert bench.decode_iteration_roofline(phases, {"draft": 1, "target": 0}, 3, shapes, 6538.0, 1)["target"] is None
-    assert bench.decode_iteration_roofline(phases, {"draft": 1, "target": 1}, 3, shapes, 6538.0, 8) is None
+    # an iteration's bytes: the weights once plus its share of the KV reads (1 GB per draft iteration here)
+    assert abs(r["draft"]["kv_gb"] - 1.0) < 1e-12 and r["target"]["kv_gb"] == 0.0
+    assert abs(r["draft"]["frac_of_hbm"] - (want_bytes + 1.0e9) / 2.0e-3 / 1e9 / 6538.0) < 1e-9
+    assert abs(r["draft"]["frac_of_hbm_weights_only"] - want_bytes / 2.0e-3 / 1e9 / 6538.0) < 1e-9
+    none = {"draft": 0.0, "target": 0.0}
+    assert bench.decode_iteration_roofline(phases, {"draft": 1, "target": 0}, none, 3, shapes, 6538.0, 1)["target"] is None
+    assert bench.decode_iteration_roofline(phases, {"draft": 1, "target": 1}, none, 3, shapes, 6538.0, 8) is None
+    # rounds of speculative decoding are not decode iterations: no target figure in that mode
+    assert bench.decode_iteration_roofline(phases, {"draft": 1, "target": 1}, none, 3, shapes, 6538.0, 1, sd=4)["target"] is None
