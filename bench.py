@@ -45,14 +45,25 @@ WORKLOADS = {
 }
 
 
-def gemm_traffic_ratio():
-    """DRAM traffic / algorithmic bytes of the tensor-core GEMM from the committed ncu capture, or None
-    when the kernel source has changed since the counters were taken."""
+TRAFFIC_SOURCES = ("gemm_tc.cu", "tc_ptx.cuh", "attn_decode.cu", "kernels_math.cu", "kernels_state.cu", "common.cuh")
+
+
+def kernel_sources_sha() -> str:
+    """One hash over the sources of every kernel of a decode iteration."""
     import hashlib
+    h = hashlib.sha256()
+    for f in TRAFFIC_SOURCES:
+        h.update(open(os.path.join(ROOT, "paper_2501_19324_b200", "csrc", f), "rb").read())
+    return h.hexdigest()
+
+
+def iteration_traffic_ratio():
+    """DRAM traffic / algorithmic bytes of one target decode iteration from the committed ncu capture (taken at a
+    step cap of 8 tokens, where the iteration's kernels are those of the full-size step; traffic grows with the
+    weights and the KV read, as the algorithmic bytes do), or None when a kernel source has changed since."""
     try:
-        d = json.load(open(os.path.join(ROOT, "profiles", "gemm_tc_traffic.json")))
-        src = open(os.path.join(ROOT, d["source"]), "rb").read()
-        return d["ratio"] if hashlib.sha256(src).hexdigest() == d["sha256"] else None
+        d = json.load(open(os.path.join(ROOT, "profiles", "target_decode_iteration_traffic.json")))
+        return d["ratio"] if kernel_sources_sha() == d["sha256"] else None
     except (OSError, KeyError, ValueError):
         return None
 
@@ -142,7 +153,8 @@ def mem_available_gb() -> float:
 class OracleSample:
     """One row of the workload pushed through the oracle's step loop for one short step.
 
-    level 0: 8-token prompt, 2-token step, forced rejection, so draft, PRM and target all run;
+    level 0: 24-token prompt, 6-token step, forced rejection, so draft, PRM and target all run (about 10 s of
+    host time at the 1.5B / 1.5B / 7B shapes);
     level 1: 4-token prompt, 1-token step, accepted (draft and PRM only) -- used when many steps are
     requested or the host has too little memory for the target's fp32 weights."""
 
@@ -156,7 +168,7 @@ class OracleSample:
         for slot, (sh, hk) in enumerate(zip(self.shapes, heads)):
             with_layers = not (slot == 2 and level == 1)
             self.models.append(OracleModel(ri.cpu_model_weights(sh, slot, 0, True, hk, with_layers=with_layers), slot))
-        self.prompt_len, self.cap = (8, 2) if level == 0 else (4, 1)
+        self.prompt_len, self.cap = (24, 6) if level == 0 else (4, 1)
         self.delta = 2.0 if level == 0 else 0.0
         self.desc = (f"1 row, {self.prompt_len}-token prompt, one step of {self.cap} token(s), "
                      + ("delta above the PRM range so the target re-decodes it" if level == 0 else
@@ -454,24 +466,24 @@ def run_ours(args, rank: int, world: int):
         hbm, tf, how = peaks()
         dec = decode_iteration_roofline(phases, iters, kv_bytes, args.steps, shapes, hbm, args.queue, args.sd)
         gemm_gbs = gt["bytes"] / (gt["ms"] * 1e-3) / 1e9 if gt["ms"] > 0 else None
-        ratio = gemm_traffic_ratio()
+        ratio = iteration_traffic_ratio()
         gemm_sub = {"what": "single weight-GEMM launches (decode, scoring, catch-up) in one extra, untimed step: CUDA events "
                             f"around every {args.time_stride}th launch; the decode iterations picked for it run kernel by kernel",
                     "GBps": gemm_gbs, "frac_of_hbm": (gemm_gbs / hbm) if gemm_gbs else None, "timed_launches": gt["launches"],
-                    "algorithmic_bytes_per_launch": (gt["bytes"] / gt["launches"]) if gt["launches"] else None,
-                    "dram_traffic_over_algorithmic": ratio,
-                    "traffic_source": "ncu capture of one decode-shaped launch (profiles/)" if ratio else
-                                      "none: the kernel changed since the counters were taken"}
+                    "algorithmic_bytes_per_launch": (gt["bytes"] / gt["launches"]) if gt["launches"] else None}
         # dominant phase: the target's decode iterations
         tgt = dec["target"] if dec else None
         if tgt:
             roofline = {"bound": "hbm", "kernel": "target decode iteration: one replay of the captured graph (28 layers of qkv / "
                         "attention / wo / gate-up + SwiGLU / down, lm head, sampling)",
-                        "achieved": tgt["gbs"], "peak": hbm, "unit": "GB/s", "frac": tgt["frac_of_hbm"], "traffic": None,
+                        "achieved": tgt["gbs"], "peak": hbm, "unit": "GB/s", "frac": tgt["frac_of_hbm"],
+                        "traffic": (ratio * (tgt["weight_gb"] + tgt["kv_gb"]) * 1e9) if ratio else None,
                         "algorithmic_bytes_per_launch": (tgt["weight_gb"] + tgt["kv_gb"]) * 1e9,
                         "launches": tgt["iterations"], "avg_launch_ms": tgt["ms"],
-                        "traffic_note": "no DRAM counters for a whole iteration; see gemm.dram_traffic_over_algorithmic for "
-                                        "the kernel class that moves 97 % of its bytes",
+                        "traffic_source": ("ncu dram__bytes_read + dram__bytes_write summed over the kernels of one iteration at a "
+                                           f"step cap of 8 (profiles/), traffic / algorithmic = {ratio:.4f}, scaled to this "
+                                           "run's bytes per iteration") if ratio else
+                                          "none: a kernel source changed since the counters were taken",
                         "peak_source": how, "timing": "CUDA events on the launching stream around the phase, inside the timed steps",
                         "gemm": gemm_sub}
         else:
@@ -517,6 +529,27 @@ def run_ours(args, rank: int, world: int):
             out["speculative_decoding"] = d_sd
         if mega_tables is not None:
             out["mega_profile"] = mega_tables
+        if world == 1 and args.queue == 1 and not args.sd and not args.no_alt:
+            # the same rows under the queued schedule (rejected rows wait until half the batch does, then one target
+            # pass serves them all): every row's sequence of steps is unchanged, the target's weight passes are
+            # shared by more rows.  Reported beside the headline, which stays the lock-step rsd_step.
+            q_rows = max(2, B // 2)
+            calls_w, calls_t = 3, max(1, min(args.steps, n_steps - 4))
+            eng.prefill(tokens, offsets)
+            for _ in range(calls_w):
+                eng.step(delta, q_rows)
+            qs, qe = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            qs.record()
+            q_tokens = 0
+            for _ in range(calls_t):
+                q_tokens += int(eng.step(delta, q_rows)["step_len"].sum())
+            qe.record()
+            torch.cuda.synchronize()
+            q_ms = qs.elapsed_time(qe)
+            out["other_schedules"] = {f"rsd_step_queued(min_target_rows={q_rows})": {
+                "value": q_tokens / (q_ms * 1e-3), "unit": UNIT, "calls": calls_t, "warmup_calls": calls_w,
+                "ms_per_call": q_ms / calls_t}}
         if world == 1 and not args.no_cpu_baseline:
             level = 0 if (args.workload == "mini" or (args.workload == "cfg2" and mem_available_gb() > 60)) else 1
             smp = OracleSample(args.workload, level)
@@ -743,6 +776,7 @@ def main():
     ap.add_argument("--workload", default="cfg2", choices=sorted(WORKLOADS))
     ap.add_argument("--time-stride", type=int, default=16, dest="time_stride")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-alt", action="store_true", dest="no_alt", help="skip the extra measurement of the queued schedule")
     ap.add_argument("--delta", type=float, default=None, help="fixed threshold instead of the 70 %% accept quantile")
     ap.add_argument("--cap", type=int, default=0, help="override the step cap (profiling aid)")
     ap.add_argument("--merged-prm", action="store_true", dest="merged_prm",

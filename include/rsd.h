@@ -178,6 +178,20 @@ int rsd_step(rsd_ctx*, float delta, void* cuda_stream, int32_t* step_tokens, int
 int rsd_step_queued(rsd_ctx*, float delta, int32_t min_target_rows, void* cuda_stream, int32_t* step_tokens,
                     int32_t* step_len, float* rewards, uint8_t* accept, uint8_t* live, uint8_t* waiting);
 
+/* rsd_step / rsd_step_queued (min_target_rows = 1 is rsd_step) with DEVICE output arrays (any may be NULL), filled
+ * on the stream in order with the call's kernels: for callers that keep the step's results on the GPU.  The call
+ * still synchronises the stream while it runs (the host sizes the ragged passes from device counters).        */
+int rsd_step_device(rsd_ctx*, float delta, int32_t min_target_rows, void* cuda_stream, int32_t* step_tokens,
+                    int32_t* step_len, float* rewards, uint8_t* accept, uint8_t* live, uint8_t* waiting);
+
+/* Reward of each row's latest step that the TARGET wrote (HOST out [B]; NaN for a row without one, or whose step has
+ * not been scored yet).  Algorithm 1 gates on the draft step's reward only; the paper's comparison of draft-step and
+ * target-step rewards inside RSD (Section 2, figure on reward distributions) reads this value too.  It costs
+ * nothing: the PRM has to cache a target-written step before it scores the row's next draft step, and the reward
+ * head is read at that step's last token on the way, so the value appears one call after the step was written.
+ * Not available with prm_shares_draft (no PRM pass).  Synchronises the device.                                 */
+int rsd_get_target_step_rewards(rsd_ctx*, float* out);
+
 /* Counters of the work done since rsd_prefill / rsd_reset.  Index 0 draft, 1 PRM, 2 target.
  * flops_paper follows Section 3.3: 2N per inference token of an N-parameter model (all
  * parameters, embedding and head included), counting every token the draft or the target

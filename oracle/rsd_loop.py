@@ -265,7 +265,7 @@ class OracleRSD:
                    draft_tokens=[[] for _ in range(B)], target_tokens=[[] for _ in range(B)],
                    draft_trace=[None] * B, target_trace=[None] * B, rej_idx=[], z_len_before=np.zeros(B, np.int32),
                    drafted=np.zeros(B, np.uint8), waiting=np.zeros(B, np.uint8), flushed=False,
-                   sd_rounds=[None] * B)
+                   sd_rounds=[None] * B, target_rewards=np.full(B, np.nan))
         run_rows = [b for b in range(B) if self.rows[b].live and not self.rows[b].waiting]
         for b in range(B):
             res["z_len_before"][b] = len(self.rows[b].z)
@@ -302,6 +302,11 @@ class OracleRSD:
             n_known = len(row.z) - row.kv_len[PRM]      # committed tokens the PRM has not cached yet
             h = self._ingest(PRM, b, len(seq), seq)
             row.reward = self.models[PRM].reward(h[-1])
+            if n_known > 0:
+                # the row's previous step was written by the target: the PRM caches it only now, and the hidden
+                # state at its last token gives that step's reward r(y_{i-1} | z_{i-1}) on the way (the paper's
+                # comparison of draft-step and target-step rewards inside RSD reads such values); not used by the gate
+                res["target_rewards"][b] = self.models[PRM].reward(h[n_known - 1])
             self.counters["ingest_tokens"][PRM] += n_known
             self.counters["score_tokens"] += len(res["draft_tokens"][b])
 

@@ -53,7 +53,7 @@ class rsd_counters(ctypes.Structure):
                 ("sd_rounds", c_uint64), ("sd_proposed", c_uint64), ("sd_matched", c_uint64), ("sd_verified", c_uint64)]
 
 
-EXPORTS = ["rsd_query_sizes", "rsd_create", "rsd_load_models", "rsd_prefill", "rsd_step", "rsd_step_queued", "rsd_flops_counters",
+EXPORTS = ["rsd_query_sizes", "rsd_create", "rsd_load_models", "rsd_prefill", "rsd_step", "rsd_step_queued", "rsd_step_device", "rsd_get_target_step_rewards", "rsd_flops_counters",
            "rsd_reset", "rsd_destroy", "rsd_last_error", "rsd_debug_force", "rsd_debug_force_sd", "rsd_debug_get_logits",
            "rsd_debug_get_sampled", "rsd_debug_get_state", "rsd_debug_gemm_timing", "rsd_debug_launch_count", "rsd_debug_mega_profile", "rsd_debug_phase_ms", "rsd_k_gemm", "rsd_k_gemm_scratch_bytes", "rsd_debug_gemm_wait_probe",
            "rsd_k_attn_decode", "rsd_k_attn_decode_scratch_bytes", "rsd_k_attn_chunk", "rsd_k_gate_compact", "rsd_k_gate_compact_static", "rsd_k_gate_compact_static_error", "rsd_k_rmsnorm",
@@ -76,6 +76,8 @@ def lib():
         L.rsd_prefill.argtypes = [vp, vp, vp, c_int32, vp]
         L.rsd_step.argtypes = [vp, c_float, vp, vp, vp, vp, vp, vp]
         L.rsd_step_queued.argtypes = [vp, c_float, c_int32, vp, vp, vp, vp, vp, vp, vp]
+        L.rsd_step_device.argtypes = [vp, c_float, c_int32, vp, vp, vp, vp, vp, vp, vp]
+        L.rsd_get_target_step_rewards.argtypes = [vp, vp]
         L.rsd_flops_counters.argtypes = [vp, POINTER(rsd_counters)]
         L.rsd_reset.argtypes = [vp]
         L.rsd_destroy.argtypes = [vp]
@@ -219,6 +221,27 @@ class Engine:
         else:
             _check(lib().rsd_step_queued(self.ctx, delta, min_target_rows, _stream(), *ptrs,
                                          out["waiting"].ctypes.data), self.ctx)
+        return out
+
+    def step_device(self, delta: float, min_target_rows: int = 1) -> dict:
+        """rsd_step_device: the step's outputs as torch CUDA tensors, filled on the current stream."""
+        import torch
+        B, C = self.B, self.C
+        out = dict(step_tokens=torch.zeros(B, C, dtype=torch.int32, device="cuda"),
+                   step_len=torch.zeros(B, dtype=torch.int32, device="cuda"),
+                   rewards=torch.zeros(B, dtype=torch.float32, device="cuda"),
+                   accept=torch.zeros(B, dtype=torch.uint8, device="cuda"),
+                   live=torch.zeros(B, dtype=torch.uint8, device="cuda"),
+                   waiting=torch.zeros(B, dtype=torch.uint8, device="cuda"))
+        _check(lib().rsd_step_device(self.ctx, delta, min_target_rows, _stream(),
+                                     *[_ptr(out[k]) for k in ("step_tokens", "step_len", "rewards", "accept", "live", "waiting")]),
+               self.ctx)
+        return out
+
+    def target_step_rewards(self) -> np.ndarray:
+        """Reward of each row's latest target-written step (NaN where there is none yet)."""
+        out = np.zeros(self.B, np.float32)
+        _check(lib().rsd_get_target_step_rewards(self.ctx, out.ctypes.data), self.ctx)
         return out
 
     def counters(self) -> dict:

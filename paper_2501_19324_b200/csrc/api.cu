@@ -220,6 +220,8 @@ size_t layout_workspace(const rsd_config& cfg, const rsd_model* const ms[3], rsd
   st.rej_idx = TAKE(int32_t, B);
   st.slot_row = TAKE(int32_t, B);
   st.last_idx = TAKE(int32_t, B);
+  st.prev_idx = TAKE(int32_t, B);
+  st.target_rewards = TAKE(float, B);
   int32_t* scal = TAKE(int32_t, 16);
   st.n_tok = scal + 0; st.n_rej = scal + 1; st.err = scal + 2; st.n_active = scal + 3; st.n_slots = scal + 4; st.iter = scal + 8;
   st.next_page = scal + 5; st.n_live = scal + 9;
@@ -501,6 +503,9 @@ int run_ingest(rsd_ctx* c, int which, int n_total, bool want_reward, cudaStream_
       const rsd_model& m = c->mdl[which].m;
       CU(launch_reward(m.dtype, c->x, m.final_norm, m.head, m.head_kind, c->st.last_idx, c0, Tc, m.d_model, m.rms_eps,
                        c->st.rewards, c->st.B, s));
+      // rows whose previous step came from the target: that step's reward, read at its last token on the way
+      CU(launch_reward(m.dtype, c->x, m.final_norm, m.head, m.head_kind, c->st.prev_idx, c0, Tc, m.d_model, m.rms_eps,
+                       c->st.target_rewards, c->st.B, s));
     }
   }
   return RSD_OK;
@@ -789,6 +794,8 @@ __global__ void init_rows_kernel(RowState st, const int32_t* flat, const int32_t
     for (int p = 0; p < 2; ++p) { st.gen_len[p][b] = 0; st.forced_len[p][b] = 0; }
     st.forced_accept[b] = 255;
     st.rewards[b] = 0.f;
+    st.target_rewards[b] = __int_as_float(0x7FC00000);   // NaN: no target-written step has been scored yet
+    st.prev_idx[b] = -1;
     st.accept[b] = 0;
     st.waiting[b] = 0;
   }
@@ -1008,7 +1015,8 @@ static int score_with_draft_trunk(rsd_ctx* c, cudaStream_t s) {
 }
 
 static int step_impl(rsd_ctx* c, float delta, int min_target_rows, void* cuda_stream, int32_t* step_tokens,
-                     int32_t* step_len, float* rewards, uint8_t* accept, uint8_t* live, uint8_t* waiting) {
+                     int32_t* step_len, float* rewards, uint8_t* accept, uint8_t* live, uint8_t* waiting,
+                     bool device_outputs = false) {
   if (!c) return RSD_ERR_ARG;
   if (c->poisoned) return fail(c, RSD_ERR_STATE, "context unusable after a CUDA error%s");
   if (!c->prefilled) return fail(c, RSD_ERR_STATE, "rsd_step before rsd_prefill%s");
@@ -1072,6 +1080,15 @@ static int step_impl(rsd_ctx* c, float delta, int min_target_rows, void* cuda_st
   const uint8_t* h_live = (const uint8_t*)mirror(c->o_live);
   const uint8_t* h_role = (const uint8_t*)mirror(c->o_role);
   const uint8_t* h_wait = (const uint8_t*)mirror(c->o_waiting);
+  if (device_outputs) {
+    // the caller's arrays are device memory: filled on the stream, in stream order with the call's kernels
+    if (step_tokens) CU(cudaMemcpyAsync(step_tokens, c->o_tokens, sizeof(int32_t) * (size_t)B * c->C, cudaMemcpyDeviceToDevice, s));
+    if (step_len) CU(cudaMemcpyAsync(step_len, c->o_len, sizeof(int32_t) * B, cudaMemcpyDeviceToDevice, s));
+    if (rewards) CU(cudaMemcpyAsync(rewards, c->o_rewards, sizeof(float) * B, cudaMemcpyDeviceToDevice, s));
+    if (accept) CU(cudaMemcpyAsync(accept, c->o_accept, B, cudaMemcpyDeviceToDevice, s));
+    if (live) CU(cudaMemcpyAsync(live, c->o_live, B, cudaMemcpyDeviceToDevice, s));
+    if (waiting) CU(cudaMemcpyAsync(waiting, c->o_waiting, B, cudaMemcpyDeviceToDevice, s));
+  }
   if ((rc = clear_forcing(c, s))) return rc;
   PHASE(7);
 #undef PHASE
@@ -1103,6 +1120,7 @@ static int step_impl(rsd_ctx* c, float delta, int min_target_rows, void* cuda_st
   // speculative decoding of rejected steps: the device keeps running totals since the last reset
   c->ctr.sd_rounds = (uint64_t)sc.sd_rounds; c->ctr.sd_proposed = (uint64_t)sc.sd_proposed;
   c->ctr.sd_matched = (uint64_t)sc.sd_matched; c->ctr.sd_verified = (uint64_t)sc.sd_proposed;
+  if (device_outputs) return RSD_OK;
   if (step_tokens) memcpy(step_tokens, h_tokens, sizeof(int32_t) * (size_t)B * c->C);
   if (step_len) memcpy(step_len, h_len, sizeof(int32_t) * B);
   if (rewards) memcpy(rewards, h_rew, sizeof(float) * B);
@@ -1120,6 +1138,11 @@ int rsd_step(rsd_ctx* c, float delta, void* cuda_stream, int32_t* step_tokens, i
 int rsd_step_queued(rsd_ctx* c, float delta, int32_t min_target_rows, void* cuda_stream, int32_t* step_tokens,
                     int32_t* step_len, float* rewards, uint8_t* accept, uint8_t* live, uint8_t* waiting) {
   return step_impl(c, delta, min_target_rows, cuda_stream, step_tokens, step_len, rewards, accept, live, waiting);
+}
+
+int rsd_step_device(rsd_ctx* c, float delta, int32_t min_target_rows, void* cuda_stream, int32_t* step_tokens,
+                    int32_t* step_len, float* rewards, uint8_t* accept, uint8_t* live, uint8_t* waiting) {
+  return step_impl(c, delta, min_target_rows, cuda_stream, step_tokens, step_len, rewards, accept, live, waiting, true);
 }
 
 int rsd_flops_counters(rsd_ctx* c, rsd_counters* out) {
@@ -1188,6 +1211,14 @@ int rsd_debug_get_logits(rsd_ctx* c, int which, float* out) {
   const int p = which == RSD_DRAFT ? 0 : (which == RSD_TARGET ? 1 : -1);
   if (p < 0 || !c->dbg_logits[p]) return fail(c, RSD_ERR_STATE, "logits were not kept%s");
   CU(cudaMemcpy(out, c->dbg_logits[p], sizeof(float) * (size_t)c->st.B * c->C * c->mdl[which].m.vocab, cudaMemcpyDeviceToHost));
+  return RSD_OK;
+}
+
+int rsd_get_target_step_rewards(rsd_ctx* c, float* out) {
+  if (!c || !out) return RSD_ERR_ARG;
+  if (!c->prefilled) return fail(c, RSD_ERR_STATE, "no rows%s");
+  CU(cudaDeviceSynchronize());
+  CU(cudaMemcpy(out, c->st.target_rewards, sizeof(float) * c->st.B, cudaMemcpyDeviceToHost));
   return RSD_OK;
 }
 

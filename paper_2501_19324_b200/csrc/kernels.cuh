@@ -200,6 +200,9 @@ struct RowState {
   int32_t *slot_row, *n_slots; // decode slots of the current phase
   int32_t *iter;               // iteration counter of the current decode phase
   int32_t *last_idx;           // [B] flat index of each row's last token in the current pass
+  int32_t *prev_idx;           // [B] PRM scoring pass: flat index of the row's last COMMITTED token when the pass
+                               // caches it (the row's previous step came from the target), else -1
+  float* target_rewards;       // [B] reward of the row's latest target-written step (NaN until one was scored)
   int32_t *n_tok;              // tokens of the current pass
   int32_t *err;                // first error raised on the device
   int32_t *pass_tok_id, *pass_tok_row, *pass_tok_pos;  // flat pass lists

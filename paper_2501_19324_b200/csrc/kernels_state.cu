@@ -96,6 +96,11 @@ __global__ void __launch_bounds__(1024) build_pass_kernel(RowState st, int which
   if (b < st.B) {
     st.last_idx[b] = cnt > 0 ? off + cnt - 1 : -1;
     st.kv_len[which][b] = start + cnt;
+    if (mode == kPassScorePrm) {
+      // the pass also caches a step the target wrote last time: its last token is the row's last committed one
+      const int z = st.z_len[b];
+      st.prev_idx[b] = (cnt > 0 && start < z) ? off + (z - 1 - start) : -1;
+    }
   }
   __syncthreads();
   for (int t = threadIdx.x; t < total; t += blockDim.x) {

@@ -80,6 +80,14 @@ def parity_step(eng, loop, delta, *, tol_logits, tol_reward, margin_tok, margin_
         assert g["step_tokens"][b, :n].tolist() == list(o["step_tokens"][b])
         assert not g["step_tokens"][b, n:].any()
     assert eng.state()["rej_idx"] == o["rej_idx"]
+    # rewards of steps the target wrote in an earlier call, read when the PRM cached them in this one
+    fresh = ~np.isnan(o["target_rewards"])
+    if fresh.any():
+        got_t = eng.target_step_rewards()
+        err_t = np.abs(got_t[fresh].astype(np.float64) - o["target_rewards"][fresh])
+        assert err_t.max() <= tol_reward, f"target-step reward error {err_t.max()}"
+        if stats is not None:
+            stats["target_step_rewards"] = stats.get("target_step_rewards", 0) + int(fresh.sum())
     # logits and free samples of both decode phases
     max_err = 0.0
     n_tok = n_cmp = 0

@@ -1,7 +1,7 @@
-"""Config 2 at its full size, in the launch configuration bench.py times (batch 32, prompts of 128 to 512
-tokens, steps of up to 128 tokens, CUDA graphs): properties that hold at any size, and the one output
-the oracle can afford to compute on its own -- the first draft logits of the row with the shortest
-prompt."""
+"""Configs 2, 3 and 4 at their full sizes, in the launch configuration bench.py times (batch 32 / 64 / 8, prompts of
+128-512 / 256 / 256 tokens, steps of up to 128 / 256 / 256 tokens, CUDA graphs): properties that hold at any size,
+and for config 2 the one output the oracle can afford to compute on its own -- the first draft logits of the row with
+the shortest prompt; plus the 7B-shape target against the oracle in the bucketed launch configuration."""
 import numpy as np
 import pytest
 
@@ -10,18 +10,24 @@ import rsd_inputs as ri
 pytestmark = [pytest.mark.gpu, pytest.mark.slow]
 
 
-def test_config2_full_size_properties_and_sampled_output():
+@pytest.mark.parametrize("config", ["cfg2", "cfg3", "cfg4"])
+def test_full_size_properties_and_sampled_output(config):
+    import torch
     from oracle import OracleModel
     from paper_2501_19324_b200 import Engine, Model, RSD_DEBUG_KEEP_LOGITS, RSD_DRAFT
-    shapes = [ri.SHAPES["1.5b"], ri.SHAPES["1.5b"], ri.SHAPES["7b"]]
+    names, B, lo, hi, cap = {"cfg2": (("1.5b", "1.5b", "7b"), 32, 128, 512, 128),
+                             "cfg3": (("1.5b", "7b", "7b"), 64, 256, 256, 256),
+                             "cfg4": (("1.5b", "1.5b", "72b"), 8, 256, 256, 256)}[config]
+    if config == "cfg4" and torch.cuda.mem_get_info()[1] < 170e9:
+        pytest.skip("needs a 180 GB GPU for the 72B-shape weights")
+    shapes = [ri.SHAPES[n] for n in names]
     heads = (ri.HEAD_LM, ri.HEAD_REWARD_SIGMOID, ri.HEAD_LM)
     models = [Model(sh, ri.gpu_model_tensors(sh, slot, 0, True, hk), hk) for slot, (sh, hk) in enumerate(zip(shapes, heads))]
-    B, cap = 32, 128
-    tokens, offsets = ri.prompts(1, B, 128, 512, shapes[0].vocab)
+    tokens, offsets = ri.prompts(1, B, lo, hi, shapes[0].vocab)
     lens = np.diff(offsets)
 
     def run(debug):
-        eng = Engine(*models, max_batch=B, max_seq_tokens=512 + 3 * cap, max_step_tokens=cap, max_steps=3,
+        eng = Engine(*models, max_batch=B, max_seq_tokens=hi + 3 * cap, max_step_tokens=cap, max_steps=3,
                      step_end_id=13, temperature=0.7, seed=0, debug_flags=debug)
         eng.prefill(tokens, offsets)
         r0 = eng.step(0.0)                                  # delta = 0: draft-only decoding
@@ -29,7 +35,8 @@ def test_config2_full_size_properties_and_sampled_output():
         r1 = eng.step(delta)
         return eng, r0, r1, delta
 
-    eng, r0, r1, delta = run(RSD_DEBUG_KEEP_LOGITS)
+    # the logits of every iteration are kept only where the oracle looks at them (config 2)
+    eng, r0, r1, delta = run(RSD_DEBUG_KEEP_LOGITS if config == "cfg2" else 0)
     c = eng.counters()
     # delta = 0 accepted every row and never touched the target
     assert r0["accept"].all() and (r0["step_len"] == cap).sum() >= B - 2
@@ -46,6 +53,15 @@ def test_config2_full_size_properties_and_sampled_output():
         assert sorted(pages) == list(range(st["next_page"][w]))
     assert c["gen_tokens"][2] == int(r1["step_len"][r1["accept"] == 0].sum())
     assert c["gen_tokens"][0] == int(r0["step_len"].sum()) + int(c["score_tokens"] - r0["step_len"].sum())
+    assert c["rejected_steps"] == int((r1["accept"] == 0).sum()) > 0 and c["accepted_steps"] == B + int(r1["accept"].sum())
+    if config != "cfg2":
+        eng.close()
+        eng2, q0, q1, delta2 = run(0)                        # determinism of the whole run
+        assert delta2 == delta and np.array_equal(q0["step_tokens"], r0["step_tokens"])
+        assert np.array_equal(q1["step_tokens"], r1["step_tokens"]) and np.array_equal(q1["accept"], r1["accept"])
+        eng2.close()
+        print(f"full-size {config}: accepted {int(r1['accept'].sum())}/{B}, delta {delta:.4f}")
+        return
     # sampled output: first draft logits of the shortest prompt against the oracle's full recompute
     b = int(np.argmin(lens))
     got = eng.logits(RSD_DRAFT)[b, 0]                        # logits of step 2's first token ... of the last step

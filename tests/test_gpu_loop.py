@@ -351,6 +351,28 @@ def test_speculative_decoding_of_rejected_steps(shapes, bf16, tol, k):
     eng.close()
 
 
+@pytest.mark.parametrize("extra,min_rows", [(dict(), 3), (dict(prm_shares_draft=True), 1)])
+def test_speculative_decoding_with_queued_rows_and_with_a_merged_prm(extra, min_rows):
+    """sd_tokens together with the other two scheduling modes: rejected rows that wait for a shared target pass
+    (rsd_step_queued), and a PRM that is a head on the draft's trunk (its scoring pass leaves one more position in
+    the draft's cache beyond the cursor, which the proposals then overwrite)."""
+    prompts = ri.prompts(63, 6, 5, 20, 1024)
+    kw = dict(max_step_tokens=6, max_steps=5, max_seq_tokens=96, step_end_id=3, step_end_mod=5, temperature=0.7,
+              seed=12, sd_tokens=3, **extra)
+    eng, loop = build_pair(TINY, bf16=False, prompts=prompts, loop_kwargs=kw)
+    delta = float(np.median(loop.step(0.0)["rewards"]))
+    eng, loop = build_pair(TINY, bf16=False, prompts=prompts, loop_kwargs=kw)
+    served = 0
+    for _ in range(12):
+        if not any(r.live for r in loop.rows):
+            break
+        g, o = parity_step(eng, loop, delta, min_target_rows=min_rows, **TOL32)
+        served += sum(1 for r in o["sd_rounds"] if r)
+    assert served > 0
+    compare_counters(eng, loop)
+    eng.close()
+
+
 def test_speculative_rounds_keep_the_matching_prefix_on_gpu():
     """Proposals planted around the target's true continuation (known from a first, plain run of the oracle): all
     right, wrong at once, right-right-wrong, a short last round.  The GPU must write the matching prefix plus the
@@ -385,3 +407,32 @@ def test_speculative_rounds_keep_the_matching_prefix_on_gpu():
         clear = [j for j in range(9) if o["target_trace"][b]["margin"][j] > 1e-3]
         assert [smp[b, j] for j in clear] == [truth[b][j] for j in clear]
     eng.close()
+
+
+def test_device_outputs_and_target_step_rewards():
+    """rsd_step_device fills device arrays with what rsd_step returns on the host, and the reward of a step the
+    target wrote shows up one call later (the PRM caches that step before it scores the next draft step): NaN
+    before, equal to the oracle's value afterwards."""
+    prompts = ri.prompts(71, 5, 6, 20, 1024)
+    kw = dict(max_step_tokens=6, max_steps=4, max_seq_tokens=64, step_end_id=3, step_end_mod=5, temperature=0.7, seed=9)
+    a, loop = build_pair(TINY, bf16=False, prompts=prompts, loop_kwargs=kw)
+    b, _ = build_pair(TINY, bf16=False, prompts=prompts, loop_kwargs=kw)
+    assert np.isnan(a.target_step_rewards()).all()
+    delta = float(np.median(loop.step(0.0)["rewards"]))
+    _, loop = build_pair(TINY, bf16=False, prompts=prompts, loop_kwargs=kw)
+    seen = 0
+    for i in range(4):
+        o = loop.step(delta)
+        host = a.step(delta)
+        dev = b.step_device(delta)
+        for k in ("step_tokens", "step_len", "rewards", "accept", "live"):
+            assert np.array_equal(host[k], dev[k].cpu().numpy()), k
+        fresh = ~np.isnan(o["target_rewards"])
+        got = a.target_step_rewards()
+        if fresh.any():
+            assert np.abs(got[fresh] - o["target_rewards"][fresh]).max() <= 1e-5
+            seen += int(fresh.sum())
+        if i == 0:
+            assert np.isnan(got).all()                                   # nothing the target wrote has been scored yet
+    assert seen > 0
+    a.close(); b.close()

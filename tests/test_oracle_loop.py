@@ -81,6 +81,12 @@ def test_rollback_and_mixed_accept_match_plain_decoding(tiny_weights):
             # the reward is that of the draft's step given the committed context
             seq = ctx[b] + list(r["draft_tokens"][b])
             assert abs(pm.reward(pm.forward_full(seq)[-1]) - r["rewards"][b]) < 1e-9
+            # the reward of a step the target wrote is read one call later, when the PRM caches that step:
+            # the PRM's score at the last token of the context as it stood after the target's step
+            if i > 0 and not pattern[i - 1][b]:
+                assert abs(pm.reward(pm.forward_full(ctx[b])[-1]) - r["target_rewards"][b]) < 1e-9
+            else:
+                assert np.isnan(r["target_rewards"][b])
             ctx[b] += list(r["step_tokens"][b])
         st = loop.state()
         assert np.array_equal(st["z_len"], [len(c) for c in ctx])
