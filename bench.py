@@ -443,9 +443,12 @@ def run_ours(args, rank: int, world: int):
     # one more step, outside every timed region: single GEMM launches bracketed by CUDA events (decode
     # iterations chosen for it run kernel by kernel instead of replaying their graph)
     gt = {"ms": 0.0, "bytes": 0.0, "launches": 0}
+    gd = {}
     if args.time_stride > 0:
         eng.gemm_timing(args.time_stride)
+        eng.gemm_timing_dense()
         eng.step(delta, args.queue)
+        gd = eng.gemm_timing_dense()
         gt = eng.gemm_timing(0)
     sampler.stop()
     e2e_tokens += timed_tokens
@@ -505,6 +508,14 @@ def run_ours(args, rank: int, world: int):
                               "for split-precision operands)",
                      "tokens_per_step": prm_tokens / args.steps, "ms_per_step": phases["prm_scoring"],
                      "peak_source": how + " (sustained bf16)"}
+            dense["gemm"] = {"what": "the dense weight-GEMM launches (more than 128 rows: scoring, sync and catch-up passes) of "
+                                     "the extra, untimed step, CUDA events around single launches; algorithmic flops 2 M N K; "
+                                     "'plain' = bf16 operand (the PRM), 'split' = hi + lo operand pair (draft, target: twice "
+                                     "the tensor-core work per algorithmic flop)"}
+            for k, v in gd.items():
+                if v["launches"]:
+                    g_tfs = v["flops"] / (v["ms"] * 1e-3) / 1e12
+                    dense["gemm"][k] = {"TFLOPs": g_tfs, "frac": g_tfs / tf, "timed_launches": v["launches"]}
         out = {"metric": METRIC, "value": timed_tokens / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
                "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",

@@ -248,6 +248,12 @@ int rsd_debug_get_state(rsd_ctx*, int32_t* z_len, int32_t* kv_len, int32_t* n_pa
  * the number of timed launches -- then clears the totals and installs the new stride.  HOST outputs,
  * any may be NULL.  Synchronises the device.                                                   */
 int rsd_debug_gemm_timing(rsd_ctx*, int32_t stride, double* ms, double* bytes, uint64_t* launches);
+/* The dense launches (more than 128 rows of x: prefill, PRM scoring, sync and catch-up passes) among the launches
+ * timed by rsd_debug_gemm_timing since the previous call of THIS function, in two classes -- index 0: plain bf16
+ * operand, index 1: hi + lo operand pair (twice the tensor-core work per algorithmic flop) --: summed device time in
+ * ms, summed algorithmic flops 2 M N K and the number of launches; the totals are cleared.  Call it before the
+ * rsd_debug_gemm_timing call that closes the period.  HOST arrays of two elements, any may be NULL.               */
+int rsd_debug_gemm_timing_dense(rsd_ctx*, double* ms, double* flops, uint64_t* launches);
 /* Device time of the phases of rsd_step, from CUDA events on the caller's stream, summed over the
  * steps since the previous call: out[7] (HOST, may be NULL) = draft sync, draft decode, PRM scoring,
  * gate + routing, target catch-up, target decode, commit, in ms.  Each call returns and clears the

@@ -55,7 +55,7 @@ class rsd_counters(ctypes.Structure):
 
 EXPORTS = ["rsd_query_sizes", "rsd_create", "rsd_load_models", "rsd_prefill", "rsd_step", "rsd_step_queued", "rsd_step_device", "rsd_get_target_step_rewards", "rsd_flops_counters",
            "rsd_reset", "rsd_destroy", "rsd_last_error", "rsd_debug_force", "rsd_debug_force_sd", "rsd_debug_get_logits",
-           "rsd_debug_get_sampled", "rsd_debug_get_state", "rsd_debug_gemm_timing", "rsd_debug_launch_count", "rsd_debug_mega_profile", "rsd_debug_phase_ms", "rsd_k_gemm", "rsd_k_gemm_scratch_bytes", "rsd_debug_gemm_wait_probe",
+           "rsd_debug_get_sampled", "rsd_debug_get_state", "rsd_debug_gemm_timing", "rsd_debug_gemm_timing_dense", "rsd_debug_launch_count", "rsd_debug_mega_profile", "rsd_debug_phase_ms", "rsd_k_gemm", "rsd_k_gemm_scratch_bytes", "rsd_debug_gemm_wait_probe",
            "rsd_k_attn_decode", "rsd_k_attn_decode_scratch_bytes", "rsd_k_attn_chunk", "rsd_k_gate_compact", "rsd_k_gate_compact_static", "rsd_k_gate_compact_static_error", "rsd_k_rmsnorm",
            "rsd_k_rope", "rsd_k_swiglu", "rsd_k_gemm_gu", "rsd_k_sample", "rsd_k_philox"]
 
@@ -89,6 +89,7 @@ def lib():
         L.rsd_debug_get_sampled.argtypes = [vp, c_int32, vp]
         L.rsd_debug_get_state.argtypes = [vp] * 8
         L.rsd_debug_gemm_timing.argtypes = [vp, c_int32, vp, vp, vp]
+        L.rsd_debug_gemm_timing_dense.argtypes = [vp, vp, vp, vp]
         L.rsd_debug_phase_ms.argtypes = [vp, c_int32, vp]
         L.rsd_debug_launch_count.argtypes = []
         L.rsd_debug_mega_profile.argtypes = [vp, c_int32, vp, c_int32, vp]
@@ -263,6 +264,13 @@ class Engine:
         _check(lib().rsd_debug_gemm_timing(self.ctx, stride, ctypes.addressof(ms), ctypes.addressof(by),
                                            ctypes.addressof(n)), self.ctx)
         return dict(ms=ms.value, bytes=by.value, launches=n.value)
+
+    def gemm_timing_dense(self) -> dict:
+        """Dense GEMM launches (more than 128 rows) timed since the last call, by operand class:
+        {"plain": {ms, flops, launches}, "split": {...}}."""
+        ms, fl, n = (c_double * 2)(), (c_double * 2)(), (c_uint64 * 2)()
+        _check(lib().rsd_debug_gemm_timing_dense(self.ctx, ms, fl, n), self.ctx)
+        return {k: dict(ms=ms[i], flops=fl[i], launches=n[i]) for i, k in enumerate(("plain", "split"))}
 
     PHASES = ("draft_sync", "draft_decode", "prm_scoring", "gate_routing", "target_catchup", "target_decode", "commit")
 

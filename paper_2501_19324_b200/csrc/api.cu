@@ -2,6 +2,7 @@
 // prefill / one step (Algorithm 1 batched over rows) as kernel launches on the caller's stream.
 #include "../../include/rsd.h"
 
+#include <cmath>
 #include <cstdio>
 #include <cstring>
 #include <new>
@@ -102,9 +103,13 @@ struct rsd_ctx {
   uint64_t gemm_calls = 0;
   std::vector<cudaEvent_t> ev;          // pairs: start, stop
   std::vector<double> ev_bytes;
+  std::vector<double> ev_flops;         // != 0: a dense launch (more than 128 rows), its algorithmic flops 2 M N K;
+                                        // negative when the operand is a hi + lo pair (twice the tensor-core work)
   size_t ev_used = 0;
   double timed_ms = 0, timed_bytes = 0;
   uint64_t timed_launches = 0;
+  double dense_ms[2] = {0, 0}, dense_flops[2] = {0, 0};  // the dense launches among them: [0] plain operand, [1] hi + lo
+  uint64_t dense_launches[2] = {0, 0};
   std::string err;
 };
 
@@ -340,6 +345,10 @@ int drain_gemm_events(rsd_ctx* c) {
     c->timed_ms += ms;
     c->timed_bytes += c->ev_bytes[i];
     ++c->timed_launches;
+    if (c->ev_flops[i] != 0) {
+      const int k = c->ev_flops[i] < 0 ? 1 : 0;
+      c->dense_ms[k] += ms; c->dense_flops[k] += std::abs(c->ev_flops[i]); ++c->dense_launches[k];
+    }
   }
   c->ev_used = 0;
   return RSD_OK;
@@ -363,6 +372,7 @@ int gemm(rsd_ctx* c, const ModelHost& M, const void* W, const void* xin, const v
     // algorithmic bytes: the weight matrix and the input once, the output once (twice when added to)
     c->ev_bytes[c->ev_used] = (double)N * K * M.elem + (double)Mrows * K * M.elem +
                               (double)Mrows * N * 4.0 * (accumulate ? 2.0 : 1.0);
+    c->ev_flops[c->ev_used] = Mrows > 128 ? (M.split ? -1.0 : 1.0) * 2.0 * Mrows * (double)N * K : 0.0;
     ++c->ev_used;
   }
   return RSD_OK;
@@ -380,6 +390,7 @@ int gemm_gu(rsd_ctx* c, const ModelHost& M, const void* Wgu, const void* xin, co
     CU(cudaEventRecord(c->ev[2 * c->ev_used + 1], s));
     // algorithmic bytes: the stacked weight matrix and the input pair once, the output pair once
     c->ev_bytes[c->ev_used] = 2.0 * F * K * M.elem + 2.0 * Mrows * K * M.elem + 2.0 * Mrows * F * M.elem;
+    c->ev_flops[c->ev_used] = Mrows > 128 ? (M.split ? -1.0 : 1.0) * 2.0 * Mrows * 2.0 * F * K : 0.0;
     ++c->ev_used;
   }
   return RSD_OK;
@@ -1249,6 +1260,20 @@ int rsd_debug_get_state(rsd_ctx* c, int32_t* z_len, int32_t* kv_len, int32_t* n_
   return RSD_OK;
 }
 
+int rsd_debug_gemm_timing_dense(rsd_ctx* c, double* ms, double* flops, uint64_t* launches) {
+  if (!c) return RSD_ERR_ARG;
+  CU(cudaDeviceSynchronize());
+  int rc = drain_gemm_events(c);
+  if (rc) return rc;
+  for (int k = 0; k < 2; ++k) {
+    if (ms) ms[k] = c->dense_ms[k];
+    if (flops) flops[k] = c->dense_flops[k];
+    if (launches) launches[k] = c->dense_launches[k];
+    c->dense_ms[k] = 0; c->dense_flops[k] = 0; c->dense_launches[k] = 0;
+  }
+  return RSD_OK;
+}
+
 int rsd_debug_gemm_timing(rsd_ctx* c, int32_t stride, double* ms, double* bytes, uint64_t* launches) {
   if (!c || stride < 0) return RSD_ERR_ARG;
   CU(cudaDeviceSynchronize());
@@ -1264,6 +1289,7 @@ int rsd_debug_gemm_timing(rsd_ctx* c, int32_t stride, double* ms, double* bytes,
     c->ev.resize(2 * pairs);
     for (auto& e : c->ev) CU(cudaEventCreate(&e));
     c->ev_bytes.assign(pairs, 0.0);
+    c->ev_flops.assign(pairs, 0.0);
   }
   c->time_stride = stride;
   return RSD_OK;
