@@ -223,6 +223,15 @@ def kv_extended(args) -> int:
     return int(v) if v is not None else 0
 
 
+def chunk_tokens(args) -> int:
+    """max_chunk_tokens of the run: configs 2 and 3 score more than 4096 tokens per step (32 x 128 draft tokens plus the
+    target-written steps the PRM still has to cache; 64 x 256), so their passes take 8192-token chunks instead of
+    the library's 4096 (one dense pass instead of a full one and a thin one); 0 = the library's default."""
+    if getattr(args, "chunk", 0):
+        return args.chunk
+    return 8192 if args.workload in ("cfg2", "cfg3") else 0
+
+
 def kv_cache_label(args) -> str:
     setting = kv_extended(args)
     names = WORKLOADS[args.workload][:3]
@@ -240,7 +249,7 @@ def workload_config(args) -> dict:
                         f"step <= {cap} tokens, Gumbel-max T=0.7, "
                         + (f"delta {args.delta}" if getattr(args, "delta", None) is not None else "delta at the 70% accept quantile"),
             "batch": B, "max_step_tokens": args.cap or cap, "replicas": args.gpus,
-            "kv_cache": kv_cache_label(args),
+            "kv_cache": kv_cache_label(args), "max_chunk_tokens": chunk_tokens(args) or 4096,
             "prm": "head on the draft's trunk (prm_shares_draft)" if getattr(args, "merged_prm", False) else "separate model",
             "schedule": "lock-step rsd_step" if getattr(args, "queue", 1) == 1 else
                         f"rsd_step_queued, target pass once {args.queue} rows wait",
@@ -353,7 +362,8 @@ def run_ours(args, rank: int, world: int):
     S = hi + n_steps * cap
     eng = Engine(*models, max_batch=B, max_seq_tokens=S, max_step_tokens=cap, max_steps=n_steps + 1,
                  step_end_id=13, temperature=0.7, seed=0, kv_extended=kv_extended(args),
-                 prm_shares_draft=int(merged), debug_flags=debug_flags(args), sd_tokens=args.sd)
+                 prm_shares_draft=int(merged), debug_flags=debug_flags(args), sd_tokens=args.sd,
+                 max_chunk_tokens=chunk_tokens(args))
     tokens, offsets = rank_prompts(rank, B, lo, hi, shapes[0].vocab)
     pinned_tokens = torch.from_numpy(tokens).pin_memory()
 
@@ -796,6 +806,8 @@ def main():
                     help="decode with the persistent decode kernel instead of kernel by kernel (not the headline path)")
     ap.add_argument("--mega-profile", action="store_true", dest="mega_profile",
                     help="record and print the phase timeline of the persistent decode kernel's last launches")
+    ap.add_argument("--chunk", type=int, default=0,
+                    help="max_chunk_tokens: tokens per multi-token pass (default: 8192 for cfg2 / cfg3, else the library's 4096)")
     ap.add_argument("--sd", type=int, default=0,
                     help="sd_tokens: rejected steps by speculative decoding with this many proposals per round (0 = off, the headline)")
     ap.add_argument("--queue", type=int, default=1,

@@ -357,8 +357,11 @@ template <bool SPLIT, bool GU> struct PersistCfg {
   static_assert(kSmemBytes <= 227 * 1024, "shared memory of one CTA");
 };
 
+// warps 0..7: epilogue, warp 8: TMA producer, warp 9: MMA issuer and owner of the tensor-memory allocation
+constexpr int kPersistEpiWarps = 8, kPersistThreads = 32 * (kPersistEpiWarps + 2);
+
 template <bool GU, bool SPLIT>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(kPersistThreads, 1)
 gemm_tc_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x,
                           const __grid_constant__ CUtensorMap tm_x_lo, float* __restrict__ Y, int M, int N, int K,
                           int accumulate, int n_tiles_n, int n_tiles_m, int* __restrict__ err,
@@ -378,11 +381,11 @@ gemm_tc_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid
   const int total_kb = (K + kTileK - 1) / kTileK, n_tiles = n_tiles_n * n_tiles_m;
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 4); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], kPersistEpiWarps); }
     *stop = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 5) tmem_alloc(tmem_slot, 512);
+  if (warp == kPersistEpiWarps + 1) tmem_alloc(tmem_slot, 512);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -396,7 +399,7 @@ gemm_tc_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid
   };
   auto fail = [&]() { if (*stop == 0) { if (err) atomicCAS(err, 0, -5); *stop = 1; } };
 
-  if (warp == 4) {
+  if (warp == kPersistEpiWarps) {
     if (lane == 0) {
       uint32_t it = 0;
       for (int t = blockIdx.x; t < n_tiles && !*stop; t += gridDim.x) {
@@ -424,7 +427,7 @@ gemm_tc_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid
             if (mbar_try_wait(&full[i % C::kStages], (i / C::kStages) & 1u)) break;
       }
     }
-  } else if (warp == 5) {
+  } else if (warp == kPersistEpiWarps + 1) {
     if (lane == 0) {
       uint32_t it = 0, n_acc = 0;
       for (int t = blockIdx.x; t < n_tiles && !*stop; t += gridDim.x, ++n_acc) {
@@ -450,6 +453,10 @@ gemm_tc_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid
     }
   } else {
     // ---------------- epilogue warps ----------------
+    // eight of them: warp w reads the tensor-memory lanes of quarter w % 4 (the hardware's rule), the two warps of a
+    // quarter take alternate groups of sixteen columns, which halves the time an accumulator stays occupied
+    const int quarter = warp & 3, col0 = (warp >> 2) * 16;
+    constexpr int kColStep = 16 * (kPersistEpiWarps / 4);
     uint32_t n_acc = 0;
     for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++n_acc) {
       int tm, tn;
@@ -460,12 +467,12 @@ gemm_tc_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid
       for (uint32_t i = 0; i < (1u << 21) && !ok && !*stop; ++i) ok = mbar_try_wait_sleep(&acc_full[b], (n_acc >> 1) & 1u, 1000);
       if (!ok) fail();
       tc_fence_after();
-      const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + b * (uint32_t)C::kMT;
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + b * (uint32_t)C::kMT;
       const int m_valid = min(C::kRows, M - m0);
       if (!GU) {
-        const int n = n0 + warp * 32 + lane;
+        const int n = n0 + quarter * 32 + lane;
         if (ok) {
-          for (int c = 0; c < m_valid; c += 16) {
+          for (int c = col0; c < m_valid; c += kColStep) {
             float v[16];
             tmem_ld16(taddr + c, v);
             if (SPLIT) {
@@ -494,14 +501,14 @@ gemm_tc_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid
         __syncwarp();
         if (lane == 0) mbar_arrive(&acc_empty[b]);
       } else {
-        const bool is_gate = warp < 2;
-        const int l = (warp & 1) * 32 + lane;
+        const bool is_gate = quarter < 2;
+        const int l = (quarter & 1) * 32 + lane;
         float* send = xch + (is_gate ? 64 * C::kLd : 0) + l * C::kLd;
         const float* recv = xch + (is_gate ? 0 : 64 * C::kLd) + l * C::kLd;
         const int send0 = is_gate ? C::kHalf : 0, own0 = is_gate ? 0 : C::kHalf;
         if (ok) {
 #pragma unroll 1
-          for (int c = 0; c < C::kHalf; c += 16) {
+          for (int c = col0; c < C::kHalf; c += kColStep) {
             float v[16];
             tmem_ld16(taddr + send0 + c, v);
             if (SPLIT) {
@@ -514,10 +521,10 @@ gemm_tc_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid
             for (int j = 0; j < 16; ++j) send[c + j] = v[j];
           }
         }
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        asm volatile("bar.sync 1, %0;" ::"n"(32 * kPersistEpiWarps) : "memory");
         if (ok && n0 + l < N) {
 #pragma unroll 1
-          for (int c = 0; c < C::kHalf; c += 16) {
+          for (int c = col0; c < C::kHalf; c += kColStep) {
             if (own0 + c >= m_valid) break;
             float v[16];
             tmem_ld16(taddr + own0 + c, v);
@@ -545,13 +552,13 @@ gemm_tc_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&acc_empty[b]);
-        asm volatile("bar.sync 1, 128;" ::: "memory");   // the exchange buffers are free for the next tile
+        asm volatile("bar.sync 1, %0;" ::"n"(32 * kPersistEpiWarps) : "memory");   // the exchange buffers are free for the next tile
       }
     }
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 5) {
+  if (warp == kPersistEpiWarps + 1) {
     __syncwarp();
     tc_fence_after();
     tmem_dealloc(tmem_base, 512);
@@ -755,8 +762,8 @@ static cudaError_t launch_persistent(const CUtensorMap& tw, const CUtensorMap& t
   if (n_sm <= 0) return cudaErrorInvalidDevice;
   const int tiles_n = GU ? N / 64 : (N + kTileN - 1) / kTileN, tiles_m = (M + C::kRows - 1) / C::kRows;
   const int grid = std::min(tiles_n * tiles_m, n_sm);
-  RSD_LAUNCH((gemm_tc_persistent_kernel<GU, SPLIT>), grid, 192, smem, s, tw, tx, txl, y, M, N, K, accumulate, tiles_n, tiles_m, err,
-             act_hi, act_lo);
+  RSD_LAUNCH((gemm_tc_persistent_kernel<GU, SPLIT>), grid, kPersistThreads, smem, s, tw, tx, txl, y, M, N, K, accumulate, tiles_n,
+             tiles_m, err, act_hi, act_lo);
   return launched(1);
 }
 

@@ -332,15 +332,118 @@ __global__ void rope_kv_kernel(const float* __restrict__ qkv, const float* __res
   }
 }
 
+// The same for the long passes (prefill, scoring, sync, catch-up: thousands of tokens, no K-split sums): a block takes
+// kRopeTokens consecutive list entries.  Their rows, positions and pages are looked up once into shared memory, so the
+// data loads of all entries go out together instead of after a chain of three dependent loads per (token, head)
+// block; and when the entries are consecutive positions of one row inside one page (the rule in a long pass), a thread
+// writes the eight transposed value elements of a (head, dim) as ONE 16-byte store instead of eight 2-byte ones.
+constexpr int kRopeTokens = 8;
+
+template <typename KT>
+__global__ void __launch_bounds__(256)
+rope_kv_long_kernel(const float* __restrict__ qkv, PassView p, float* __restrict__ q_out, KT* pool,
+                    const int32_t* __restrict__ page_table, int max_pages, const float2* __restrict__ rope, int H, int KV,
+                    int hd, int pf) {
+  RSD_PDL_SYNC();
+  __shared__ int s_row[kRopeTokens], s_pos[kRopeTokens], s_page[kRopeTokens];
+  __shared__ int s_run;            // 1: the entries are eight consecutive positions of one row within one page
+  const int t0 = blockIdx.x * kRopeTokens;
+  const int n_tok = min(kRopeTokens, p.T - t0);
+  if (threadIdx.x < kRopeTokens) {
+    const int i = threadIdx.x;
+    int row = -1, pos = 0, page = 0;
+    if (i < n_tok) {
+      row = p.tok_row[t0 + i];
+      pos = p.tok_pos[t0 + i];
+      if (row >= 0) page = page_table[(size_t)row * max_pages + pos / kPageTokens];
+    }
+    s_row[i] = row; s_pos[i] = pos; s_page[i] = page;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int run = n_tok == kRopeTokens && s_row[0] >= 0 && (s_pos[0] % kRopeTokens) == 0;
+    for (int i = 1; i < kRopeTokens && run; ++i) run = s_row[i] == s_row[0] && s_pos[i] == s_pos[0] + i;
+    s_run = run;
+  }
+  __syncthreads();
+  const int half = hd / 2;
+  const int width = (H + 2 * KV) * hd;
+  const size_t block = (size_t)KV * kPageTokens * hd;
+  const int n_rot = (H + KV) * half;            // rotated pairs of one token
+  // queries and keys: one (token, head, pair) per step
+  for (int idx = threadIdx.x; idx < n_tok * n_rot; idx += blockDim.x) {
+    const int tk = idx / n_rot, e = idx % n_rot;
+    if (s_row[tk] < 0) continue;
+    const int head = e / half, i = e % half;
+    const int t = t0 + tk, pos = s_pos[tk];
+    const float a = qkv[(size_t)t * width + head * hd + i], b = qkv[(size_t)t * width + head * hd + i + half];
+    const float2 c = rope[(size_t)pos * half + i];
+    const float ra = a * c.x - b * c.y, rb = b * c.x + a * c.y;
+    if (head < H) {
+      q_out[(size_t)t * H * hd + head * hd + i] = ra;
+      q_out[(size_t)t * H * hd + head * hd + i + half] = rb;
+    } else {
+      KT* k = pool + (size_t)s_page[tk] * pf * block + ((size_t)(head - H) * kPageTokens + pos % kPageTokens) * hd;
+      const KT ka = from_f32<KT>(ra), kb2 = from_f32<KT>(rb);
+      k[i] = ka;
+      k[i + half] = kb2;
+      if (pf == 4) {
+        k[2 * block + i] = from_f32<KT>(ra - to_f32(ka));
+        k[2 * block + i + half] = from_f32<KT>(rb - to_f32(kb2));
+      }
+    }
+  }
+  // values, transposed inside the page: [KV][hd][16 tokens]
+  if (s_run && sizeof(KT) == 2) {
+    const int slot0 = s_pos[0] % kPageTokens;                     // 0 or 8: the 16-byte store is aligned
+    KT* vbase = pool + (size_t)s_page[0] * pf * block + block;
+    for (int e = threadIdx.x; e < KV * hd; e += blockDim.x) {
+      __align__(16) KT hi8[kRopeTokens];
+      __align__(16) KT lo8[kRopeTokens];
+#pragma unroll
+      for (int tk = 0; tk < kRopeTokens; ++tk) {
+        const float v = qkv[(size_t)(t0 + tk) * width + (size_t)(H + KV) * hd + e];
+        hi8[tk] = from_f32<KT>(v);
+        lo8[tk] = from_f32<KT>(v - to_f32(hi8[tk]));
+      }
+      *reinterpret_cast<uint4*>(vbase + (size_t)e * kPageTokens + slot0) = *reinterpret_cast<const uint4*>(hi8);
+      if (pf == 4) *reinterpret_cast<uint4*>(vbase + 2 * block + (size_t)e * kPageTokens + slot0) = *reinterpret_cast<const uint4*>(lo8);
+    }
+  } else {
+    for (int idx = threadIdx.x; idx < n_tok * KV * hd; idx += blockDim.x) {
+      const int tk = idx / (KV * hd), e = idx % (KV * hd);
+      if (s_row[tk] < 0) continue;
+      const float v = qkv[(size_t)(t0 + tk) * width + (size_t)(H + KV) * hd + e];
+      KT* vbase = pool + (size_t)s_page[tk] * pf * block + block;
+      const int slot = s_pos[tk] % kPageTokens;
+      const KT vh = from_f32<KT>(v);
+      vbase[(size_t)e * kPageTokens + slot] = vh;
+      if (pf == 4) vbase[2 * block + (size_t)e * kPageTokens + slot] = from_f32<KT>(v - to_f32(vh));
+    }
+  }
+}
+
 cudaError_t launch_rope_kv(int kv_dtype, const float* qkv, SplitSum pending, PassView p, float* q_out, KvView kv,
                            const float2* rope, int H, int KV, int hd, cudaStream_t s) {
   if (p.T <= 0) return cudaSuccess;
+  const int pf = 2 + 2 * kv.v_extra;
+  if (pending.splits <= 1 && p.n_active == nullptr && p.T >= 64) {
+    // long pass: eight list entries per block
+    const int blocks = (p.T + kRopeTokens - 1) / kRopeTokens;
+    if (kv_dtype == 2 || kv_dtype == 3)
+      RSD_LAUNCH((rope_kv_long_kernel<__half>), blocks, 256, 0, s, qkv, p, q_out, (__half*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd, pf);
+    else if (kv_dtype == 1)
+      RSD_LAUNCH((rope_kv_long_kernel<__nv_bfloat16>), blocks, 256, 0, s, qkv, p, q_out, (__nv_bfloat16*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd, pf);
+    else
+      RSD_LAUNCH((rope_kv_long_kernel<float>), blocks, 256, 0, s, qkv, p, q_out, (float*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd, pf);
+    return launched(1);
+  }
   if (kv_dtype == 2 || kv_dtype == 3)
-    RSD_LAUNCH((rope_kv_kernel<__half>), dim3(p.T, H + 2 * KV), 64, 0, s, qkv, pending.partials, pending.splits, p, q_out, (__half*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd, 2 + 2 * kv.v_extra);
+    RSD_LAUNCH((rope_kv_kernel<__half>), dim3(p.T, H + 2 * KV), 64, 0, s, qkv, pending.partials, pending.splits, p, q_out, (__half*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd, pf);
   else if (kv_dtype == 1)
-    RSD_LAUNCH((rope_kv_kernel<__nv_bfloat16>), dim3(p.T, H + 2 * KV), 64, 0, s, qkv, pending.partials, pending.splits, p, q_out, (__nv_bfloat16*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd, 2 + 2 * kv.v_extra);
+    RSD_LAUNCH((rope_kv_kernel<__nv_bfloat16>), dim3(p.T, H + 2 * KV), 64, 0, s, qkv, pending.partials, pending.splits, p, q_out, (__nv_bfloat16*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd, pf);
   else
-    RSD_LAUNCH((rope_kv_kernel<float>), dim3(p.T, H + 2 * KV), 64, 0, s, qkv, pending.partials, pending.splits, p, q_out, (float*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd, 2 + 2 * kv.v_extra);
+    RSD_LAUNCH((rope_kv_kernel<float>), dim3(p.T, H + 2 * KV), 64, 0, s, qkv, pending.partials, pending.splits, p, q_out, (float*)kv.pool_layer, kv.page_table, kv.max_pages, rope, H, KV, hd, pf);
   return launched(1);
 }
 
