@@ -707,6 +707,52 @@ def sweep_attn(args):
     sampler.stop()
 
 
+def sweep_chunk(args):
+    """Causal chunk attention (prefill / scoring / catch-up) over a paged prefix: `rows` rows, each with `new` query
+    tokens after `prefix` cached positions, fp16 cache, pages randomly permuted.  --only rows,new,prefix,H,KV runs a
+    single point with plain launches (the form an ncu capture uses)."""
+    import torch
+    from paper_2501_19324_b200 import binding as rb
+    _, tf, how = peaks()
+    hd = 128
+    points = [(H, KV, B, new, prefix) for (H, KV) in ((12, 2), (28, 4))
+              for (B, new, prefix) in ((32, 128, 256), (32, 128, 1024), (16, 256, 2048), (16, 256, 3072), (8, 512, 0))]
+    only = None
+    if args.only:
+        B, new, prefix, H, KV = (int(v) for v in args.only.split(","))
+        points, only = [(H, KV, B, new, prefix)], True
+    sampler = None if only else _sweep_sampler()
+    for H, KV, B, new, prefix in points:
+        ctx = prefix + new
+        n_pages_row = (ctx + 15) // 16
+        n_pages = B * n_pages_row
+        pool = torch.randn(n_pages * 2 * KV * 16 * hd, device="cuda", dtype=torch.float16)
+        table = torch.randperm(n_pages, device="cuda", dtype=torch.int32).view(B, n_pages_row).contiguous()
+        rows = torch.arange(B, device="cuda", dtype=torch.int32).repeat_interleave(new)
+        pos = (torch.arange(new, device="cuda", dtype=torch.int32) + prefix).repeat(B)
+        T = B * new
+        q = torch.randn(T, H, hd, device="cuda")
+        out = torch.zeros_like(q)
+
+        def call(_):
+            rb._check(rb.lib().rsd_k_attn_chunk(rb._ptr(q), rb._ptr(pool), rb._ptr(table), rb._ptr(rows), rb._ptr(pos),
+                                                rb._ptr(out), T, H, KV, hd, n_pages_row, 2, rb._stream()))
+        flops = 4.0 * H * hd * B * (new * prefix + new * (new + 1) // 2)
+        kv_bytes = B * ctx * 2 * KV * hd * 2
+        if only:
+            for _ in range(4):
+                call(0)
+            torch.cuda.synchronize()
+            print(json.dumps({"sweep": "chunk_attn", "only": [B, new, prefix, H, KV], "flops": flops, "kv_bytes": kv_bytes}))
+            return
+        us, detail = _graph_time_us(call, [0], iters=5, sampler=sampler)
+        print(json.dumps({"sweep": "chunk_attn", "H": H, "KV": KV, "rows": B, "new_tokens": new, "prefix": prefix, "us": us,
+                          "TFLOPs": flops / us * 1e-6, "bf16_frac": flops / us * 1e-6 / tf, "kv_bytes": kv_bytes,
+                          "peak_source": how, **detail}), flush=True)
+    if sampler is not None:
+        sampler.stop()
+
+
 def sweep_gate(args):
     import torch
     from paper_2501_19324_b200 import binding as rb
@@ -818,11 +864,11 @@ def main():
                                                "a single batch[,prompt length], one timed step")
     ap.add_argument("--prm-shape", default="1.5b", dest="prm_shape", choices=["1.5b", "7b"],
                     help="with --sweep score: shape of the PRM")
-    ap.add_argument("--sweep", default="", choices=["", "gemm", "attn", "gate", "score"],
+    ap.add_argument("--sweep", default="", choices=["", "gemm", "attn", "chunk", "gate", "score"],
                     help="kernel sweep on config-2 shapes instead of the step-loop benchmark")
     args = ap.parse_args()
     if args.sweep:
-        {"gemm": sweep_gemm, "attn": sweep_attn, "gate": sweep_gate, "score": sweep_score}[args.sweep](args)
+        {"gemm": sweep_gemm, "attn": sweep_attn, "chunk": sweep_chunk, "gate": sweep_gate, "score": sweep_score}[args.sweep](args)
         return
     args.warmup = max(args.warmup, 0)
     rank = int(os.environ.get("RANK", 0))

@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "librsd.so")
-SOURCES = ["api.cu", "kernels_math.cu", "kernels_state.cu", "gemm_tc.cu", "attn_decode.cu", "attn_chunk.cu", "decode_mega.cu", "no_alloc.cu"]
+SOURCES = ["api.cu", "kernels_math.cu", "kernels_state.cu", "gemm_tc.cu", "attn_decode.cu", "attn_chunk.cu", "attn_chunk_tc.cu", "decode_mega.cu", "no_alloc.cu"]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "--use_fast_math=false"]
 

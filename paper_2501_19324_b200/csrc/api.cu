@@ -431,7 +431,8 @@ int forward_pass(rsd_ctx* c, int which, PassView p, cudaStream_t s) {
                             c->attn, attn_lo, m.dtype, T, H, KV, hd, c->S, c->attn_scratch, c->attn_scratch_bytes,
                             p.n_active, s, c->attn_rows_hint));
     } else {
-      CU(launch_attn_chunk(M.kv_dtype, c->q, p, kv, c->attn, attn_lo, m.dtype, H, KV, hd, s));
+      CU(launch_attn_chunk(M.kv_dtype, c->q, p, kv, c->attn, attn_lo, m.dtype, H, KV, hd, s,
+                           (int*)((char*)c->gemm_scratch + 4096)));
     }
     rc = gemm(c, M, M.wo[l], c->attn, attn_lo, c->x, T, d, H * hd, 1, p.n_active, defer_small ? &x_pending : nullptr, s);
     if (rc) return rc;

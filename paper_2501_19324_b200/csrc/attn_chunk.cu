@@ -245,8 +245,10 @@ attn_chunk_kernel(const float* __restrict__ q, PassView p, const KT* __restrict_
 }  // namespace
 
 cudaError_t launch_attn_chunk(int kv_dtype, const float* q, PassView p, KvView kv, void* out, void* out_lo,
-                              int out_dtype, int H, int KV, int hd, cudaStream_t s) {
+                              int out_dtype, int H, int KV, int hd, cudaStream_t s, int* err) {
   if (p.T <= 0) return cudaSuccess;
+  if (attn_chunk_tc_supported(kv_dtype, H, KV, hd, p.T))
+    return launch_attn_chunk_tc(q, p, kv, out, out_lo, out_dtype, H, KV, err, s);
   const int G = H / KV;
   if (kv_dtype == 3) kv.v_extra = 1;
   if (kv_dtype == 0 || G > 8)

@@ -713,6 +713,49 @@ bool tc_tensor_map(const void* ptr, int rows, int cols, int box_rows, CUtensorMa
   return get_map(ptr, rows, cols, box_rows, out);
 }
 
+// One layer's slab of fp16 KV pages as a tensor of 4096-byte blocks (per page: the keys of every KV head
+// [16 tokens][128 dims], then the values [128 dims][16 tokens]), one box per block:
+//   keys    (64 dims, 8 tokens, 2 dim halves, 2 token groups, block)   128-byte swizzle: lands as
+//           [token group][dim half][8 tokens][64 dims], the order the score MMA wants its operand in
+//   values  (16 tokens, 128 dims, block)                               32-byte swizzle
+// The block extent is a bound on what a coordinate may name, not an allocation size: only the boxes a kernel asks
+// for are touched.
+bool tc_tensor_map_kv(const void* pool_layer, int values, CUtensorMap* out) {
+  static std::mutex mu;
+  static std::unordered_map<MapKey, CUtensorMap, MapKeyHash> cache;
+  std::lock_guard<std::mutex> lock(mu);
+  MapKey key{pool_layer, values, 0, 0};
+  auto it = cache.find(key);
+  if (it != cache.end()) { *out = it->second; return true; }
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  CUtensorMap m;
+  const cuuint64_t blocks = 1ull << 30;
+  CUresult r;
+  if (values) {
+    cuuint64_t dims[3] = {16, 128, blocks};
+    cuuint64_t strides[2] = {32, 4096};
+    cuuint32_t box[3] = {16, 128, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    r = fn(&m, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void*>(pool_layer), dims, strides, box, estr,
+           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  } else {
+    cuuint64_t dims[5] = {64, 8, 2, 2, blocks};
+    cuuint64_t strides[4] = {256, 128, 2048, 4096};      // token, dim half, token group, block
+    cuuint32_t box[5] = {64, 8, 2, 2, 1};
+    cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    r = fn(&m, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 5, const_cast<void*>(pool_layer), dims, strides, box, estr,
+           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  }
+  if (r != CUDA_SUCCESS) return false;
+  if (cache.size() > 65536) cache.clear();
+  cache.emplace(key, m);
+  *out = m;
+  return true;
+}
+
 // Launches the PROBE instantiation on a 128 x 16 x 64 problem whose copies are never issued (W and x are mapped but
 // not read): the kernel's bounded wait expires and *err (the int at byte 4096 of the scratch) becomes -5.
 cudaError_t launch_gemm_wait_probe(const void* W, const void* x, float* y, void* scratch, size_t scratch_bytes, cudaStream_t s) {

@@ -104,9 +104,14 @@ cudaError_t launch_rope_only(float* v, const int32_t* pos, int T, int n_heads, i
 // Causal attention of every slot over positions [0, tok_pos] of its row, read from the pages.
 cudaError_t launch_attn_generic(int kv_dtype, const float* q, PassView p, KvView kv, void* out, void* out_lo,
                                 int out_dtype, int H, int KV, int hd, cudaStream_t s);
-// Tensor-core version of the above for 16-bit caches with H / KV <= 8 (falls back otherwise).
+// Tensor-core versions of the above for 16-bit caches with H / KV <= 8 (falls back otherwise): the tcgen05 kernel for
+// fp16 caches with head_dim 128 and at least 64 list entries (attn_chunk_tc.cu), else the mma.sync kernel.
+// err (nullable): raised to -5 when a bounded wait of the tcgen05 kernel expires.
 cudaError_t launch_attn_chunk(int kv_dtype, const float* q, PassView p, KvView kv, void* out, void* out_lo,
-                              int out_dtype, int H, int KV, int hd, cudaStream_t s);
+                              int out_dtype, int H, int KV, int hd, cudaStream_t s, int* err = nullptr);
+bool attn_chunk_tc_supported(int kv_dtype, int H, int KV, int hd, int T);
+cudaError_t launch_attn_chunk_tc(const float* q, PassView p, KvView kv, void* out, void* out_lo, int out_dtype, int H, int KV,
+                                 int* err, cudaStream_t s);
 cudaError_t launch_swiglu(int dtype, const float* gu, SplitSum pending, void* out, void* out_lo, int T, int F,
                           const int32_t* n_active, cudaStream_t s);
 

@@ -97,4 +97,9 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
 // Row-major bf16 matrix [rows, cols] as a TMA tensor map (box = 64 columns x box_rows rows, 128-byte swizzle);
 // host side, cached by (pointer, shape).  Defined with the tensor-core GEMM.
 bool tc_tensor_map(const void* ptr, int rows, int cols, int box_rows, CUtensorMap* out);
+// One layer's slab of fp16 KV pages (head_dim 128) as a tensor of 4096-byte blocks, one TMA box per block: keys
+// (values = 0) land as [2 token groups][2 dim halves][8 tokens][64 dims] under the 128-byte swizzle, values
+// (values = 1) as [128 dims][16 tokens] under the 32-byte swizzle; the last coordinate is the block,
+// (2 * page + values) * KV + head.
+bool tc_tensor_map_kv(const void* pool_layer, int values, CUtensorMap* out);
 }  // namespace rsd
