@@ -678,33 +678,44 @@ def sweep_attn(args):
     from paper_2501_19324_b200 import binding as rb
     hbm, _, how = peaks()
     hd = 128
-    sampler = _sweep_sampler()
-    for H, KV in ((12, 2), (28, 4)):
-        for ctx in (512, 1024, 2048, 4096, 8192, 16384):
-            for B in (1, 2, 4, 8, 16, 32, 64, 128, 256):
-                n_pages = B * (ctx // 16)
-                pool_bytes = n_pages * 2 * KV * 16 * hd * 2
-                if pool_bytes > 24e9:
-                    continue
-                reps = max(1, min(4, int(300e6 // pool_bytes) + 1))
-                pools = [torch.randn(n_pages * 2 * KV * 16 * hd, device="cuda", dtype=torch.float16) for _ in range(reps)]
-                table = torch.randperm(n_pages, device="cuda", dtype=torch.int32).view(B, ctx // 16).contiguous()
-                q = torch.randn(B, H, hd, device="cuda")
-                ctx_len = torch.full((B,), ctx, dtype=torch.int32, device="cuda")
-                out = torch.empty_like(q)
-                nbytes = rb.lib().rsd_k_attn_decode_scratch_bytes(B, H, hd, ctx)
-                scratch = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
+    points = [(H, KV, ctx, B) for (H, KV) in ((12, 2), (28, 4)) for ctx in (512, 1024, 2048, 4096, 8192, 16384)
+              for B in (1, 2, 4, 8, 16, 32, 64, 128, 256)]
+    only = bool(args.only)
+    if only:          # --only batch,ctx,H,KV: a single point with plain launches (the form an ncu capture uses)
+        B, ctx, H, KV = (int(v) for v in args.only.split(","))
+        points = [(H, KV, ctx, B)]
+    sampler = None if only else _sweep_sampler()
+    for H, KV, ctx, B in points:
+        n_pages = B * (ctx // 16)
+        pool_bytes = n_pages * 2 * KV * 16 * hd * 2
+        if pool_bytes > 24e9:
+            continue
+        reps = max(1, min(4, int(300e6 // pool_bytes) + 1))
+        pools = [torch.randn(n_pages * 2 * KV * 16 * hd, device="cuda", dtype=torch.float16) for _ in range(reps)]
+        table = torch.randperm(n_pages, device="cuda", dtype=torch.int32).view(B, ctx // 16).contiguous()
+        q = torch.randn(B, H, hd, device="cuda")
+        ctx_len = torch.full((B,), ctx, dtype=torch.int32, device="cuda")
+        out = torch.empty_like(q)
+        nbytes = rb.lib().rsd_k_attn_decode_scratch_bytes(B, H, hd, ctx)
+        scratch = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
 
-                def call(pool):
-                    rb._check(rb.lib().rsd_k_attn_decode(rb._ptr(q), rb._ptr(pool), rb._ptr(table), rb._ptr(ctx_len),
-                                                         rb._ptr(out), B, H, KV, hd, ctx // 16, 2, rb._ptr(scratch),
-                                                         nbytes, rb._stream()))
-                us, detail = _graph_time_us(call, pools, iters=10, sampler=sampler)
-                print(json.dumps({"sweep": "attn_decode", "H": H, "KV": KV, "ctx": ctx, "batch": B, "us": us,
-                                  "GBps": pool_bytes / us * 1e-3, "hbm_frac": pool_bytes / us * 1e-3 / hbm,
-                                  "pages": "randomly permuted", "peak_source": how, **detail}), flush=True)
-                del pools
-    sampler.stop()
+        def call(pool):
+            rb._check(rb.lib().rsd_k_attn_decode(rb._ptr(q), rb._ptr(pool), rb._ptr(table), rb._ptr(ctx_len),
+                                                 rb._ptr(out), B, H, KV, hd, ctx // 16, 2, rb._ptr(scratch),
+                                                 nbytes, rb._stream()))
+        if only:
+            for i in range(6):
+                call(pools[i % len(pools)])
+            torch.cuda.synchronize()
+            print(json.dumps({"sweep": "attn_decode", "only": [B, ctx, H, KV], "kv_bytes": pool_bytes}))
+            return
+        us, detail = _graph_time_us(call, pools, iters=10, sampler=sampler)
+        print(json.dumps({"sweep": "attn_decode", "H": H, "KV": KV, "ctx": ctx, "batch": B, "us": us,
+                          "GBps": pool_bytes / us * 1e-3, "hbm_frac": pool_bytes / us * 1e-3 / hbm,
+                          "pages": "randomly permuted", "peak_source": how, **detail}), flush=True)
+        del pools
+    if sampler is not None:
+        sampler.stop()
 
 
 def sweep_chunk(args):
@@ -861,7 +872,8 @@ def main():
     ap.add_argument("--kv-extended", type=int, default=None, choices=[0, 1, 2], dest="kv_extended",
                     help="KV cache: 0 by model depth (default: hi+lo pairs beyond 48 layers), 1 fp16 hi+lo pairs, 2 plain fp16")
     ap.add_argument("--only", default="", help="with --sweep gemm: a single M,K,N point, plain launches; with --sweep score: "
-                                               "a single batch[,prompt length], one timed step")
+                                               "a single batch[,prompt length], one timed step; with --sweep attn: batch,ctx,H,KV; "
+                                               "with --sweep chunk: rows,new,prefix,H,KV (plain launches)")
     ap.add_argument("--prm-shape", default="1.5b", dest="prm_shape", choices=["1.5b", "7b"],
                     help="with --sweep score: shape of the PRM")
     ap.add_argument("--sweep", default="", choices=["", "gemm", "attn", "chunk", "gate", "score"],

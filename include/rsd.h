@@ -307,8 +307,12 @@ size_t rsd_k_attn_decode_scratch_bytes(int32_t B, int32_t H, int32_t hd, int32_t
 /* Causal attention of a ragged list of T new tokens over the same paged cache (prefill, PRM step scoring,
  * catch-up): entry t belongs to row tok_row[t] (entries sorted by row, then position; tok_row < 0 is
  * skipped) and attends positions [0, tok_pos[t]] of that row, whose keys and values (those of the new
- * tokens included) are already in the pages.  q and out are [T, H, hd] fp32.  16-bit caches with
- * H / KV <= 8 take the tensor-core kernel, everything else the generic one.                        */
+ * tokens included) are already in the pages.  q and out are [T, H, hd] fp32.  fp16 caches with
+ * hd = 128, H / KV <= 8 and T >= 64 take the tcgen05 kernel (operands and accumulators in tensor
+ * memory, pages fetched by TMA: kv_pool must be 16-byte aligned), other 16-bit caches with
+ * H / KV <= 8 the mma.sync kernel, everything else the generic one.  (Inside rsd_prefill / rsd_step
+ * a bounded device-side wait of the tcgen05 kernel that runs out makes the call return
+ * RSD_ERR_TIMEOUT; this stand-alone entry has no error word to report it in.)                      */
 int rsd_k_attn_chunk(const float* q, const void* kv_pool, const int32_t* page_table, const int32_t* tok_row,
                      const int32_t* tok_pos, float* out, int32_t T, int32_t H, int32_t KV, int32_t hd,
                      int32_t max_pages, int32_t dtype, void* cuda_stream);

@@ -297,7 +297,8 @@ def test_decode_attention_against_definition(dtype, hd, H, KV):
 
 
 @pytest.mark.parametrize("dtype,hd,H,KV", [(torch.float16, 128, 12, 2), (torch.float16, 128, 28, 4), (torch.float16, 64, 4, 2),
-                                          (torch.float32, 64, 4, 2), (torch.float16, 128, 64, 8)])
+                                          (torch.float32, 64, 4, 2), (torch.float16, 128, 64, 8), (torch.float16, 128, 8, 4),
+                                          (torch.float16, 128, 3, 3), (torch.bfloat16, 128, 12, 2)])
 def test_chunk_attention_against_definition(dtype, hd, H, KV):
     """Ragged chunks of several rows in one list: tiles that straddle rows, a chunk that starts in the
     middle of a page, long prefixes, one idle entry; every query against brute-force causal softmax."""
@@ -315,7 +316,7 @@ def test_chunk_attention_against_definition(dtype, hd, H, KV):
     T = len(rows)
     q = rng.normal(size=(T, H, hd)).astype(np.float32)
     got = rb.k_attn_chunk(dev(q), pool, table, dev(np.array(rows, np.int32)), dev(np.array(poss, np.int32)), KV).cpu().numpy()
-    tol = 2e-5 if dtype == torch.float32 else 2e-3
+    tol = {torch.float32: 2e-5, torch.float16: 2e-3, torch.bfloat16: 1.5e-2}[dtype]
     for t in range(T):
         b, p = rows[t], poss[t]
         if b < 0:
