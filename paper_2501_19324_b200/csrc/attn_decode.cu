@@ -11,8 +11,13 @@
 //   O += P V     with the same MMA: values are stored transposed inside a page ([hd][16 tokens]), so a
 //        B fragment is one 64-bit load; the order of the tokens inside a page is permuted identically
 //        for P and V.
-// The warps' partial (max, sum, O) meet in shared memory; with several context splits the CTA writes
-// its partial to scratch and a second kernel merges the splits.
+// The warps' partial (max, sum, O) meet in shared memory.  With 2 to 8 context splits the splits of a (slot, KV
+// head) are the CTAs of one thread-block cluster: each leaves its partial in its own shared memory, and after a
+// cluster barrier every CTA merges a slice of the G x HD outputs out of all the CTAs' shared memory (in split
+// order) and writes it: no second launch and no trip through global memory.  With more splits than a cluster
+// holds the CTA writes its partial to scratch and a second kernel merges them.
+#include <cooperative_groups.h>
+
 #include "common.cuh"
 #include "kernels.cuh"
 
@@ -63,7 +68,7 @@ __device__ __forceinline__ void mma_16816<__half>(float& d0, float& d1, float& d
 // part_o: [slot][head][split][HD] un-normalised outputs; part_ml: [slot][head][split][2] (max, sum).
 // EXT: queries and softmax weights enter the products as hi + lo pairs and every page carries the low
 // halves of its keys and values in two more blocks: the attention is accurate to about 2^-20.
-template <int HD, typename KT, typename OT, bool EXT>
+template <int HD, typename KT, typename OT, bool EXT, bool CL>
 __global__ void __launch_bounds__(128, EXT ? 2 : 4)
 attn_decode_kernel(const float* __restrict__ q, const KT* __restrict__ pool, const int32_t* __restrict__ page_table,
                    int max_pages, const int32_t* __restrict__ slot_row, const int32_t* __restrict__ len_or_pos, int len_offset,
@@ -201,6 +206,7 @@ attn_decode_kernel(const float* __restrict__ q, const KT* __restrict__ pool, con
     s_o[warp][g][8 * i + 2 * t + 1] = o[i][1];
   }
   __syncthreads();
+  __shared__ float c_m[8], c_l[8];               // cluster mode: this CTA's (max, sum) per head; its O goes to s_o[0]
   for (int idx = threadIdx.x; idx < G * HD; idx += blockDim.x) {
     const int gg = idx / HD, dd = idx % HD;
     float M = fmaxf(fmaxf(s_m[0][gg], s_m[1][gg]), fmaxf(s_m[2][gg], s_m[3][gg]));
@@ -214,13 +220,54 @@ attn_decode_kernel(const float* __restrict__ q, const KT* __restrict__ pool, con
       }
     }
     const int h = h0 + gg;
-    if (n_splits == 1) {
+    if (CL) {
+      // (gg, dd) is this thread's alone: it has read the four warps' values and may overwrite the first
+      s_o[0][gg][dd] = O;
+      if (dd == 0) { c_m[gg] = M; c_l[gg] = L; }
+    } else if (n_splits == 1) {
       store_operand<OT>(out, out_lo, ((size_t)slot * H + h) * HD + dd, O / L);
     } else {
       const size_t base = ((size_t)slot * H + h) * n_splits + split;
       part_o[base * HD + dd] = O;
       if (dd == 0) { part_ml[base * 2] = M; part_ml[base * 2 + 1] = L; }
     }
+  }
+  if (CL) {
+    // Every CTA of the cluster gets here (the early returns above depend on the slot alone, which the cluster
+    // shares).  Rank = split.  A CTA merges the outputs [rank * per, rank * per + per) of the G x HD.
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
+    cluster.sync();
+    const int n_rank = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
+    const int total = G * HD, per = (total + n_rank - 1) / n_rank;
+    const int end = min(total, (rank + 1) * per);
+    for (int idx = rank * per + threadIdx.x; idx < end; idx += blockDim.x) {
+      const int gg = idx / HD, dd = idx % HD;
+      float pm[8], pl[8], po[8];
+#pragma unroll
+      for (int r = 0; r < 8; ++r) {
+        if (r < n_rank) {
+          pm[r] = *cluster.map_shared_rank(&c_m[gg], r);
+          pl[r] = *cluster.map_shared_rank(&c_l[gg], r);
+          po[r] = *cluster.map_shared_rank(&s_o[0][gg][dd], r);
+        } else {
+          pm[r] = -INFINITY; pl[r] = 0.f; po[r] = 0.f;
+        }
+      }
+      float M = -INFINITY, L = 0.f, O = 0.f;
+#pragma unroll
+      for (int r = 0; r < 8; ++r) {
+        if (pm[r] > -INFINITY) {
+          const float Mn = fmaxf(M, pm[r]);
+          const float e_old = __expf(M - Mn), e_new = __expf(pm[r] - Mn);
+          L = L * e_old + pl[r] * e_new;
+          O = O * e_old + po[r] * e_new;
+          M = Mn;
+        }
+      }
+      store_operand<OT>(out, out_lo, ((size_t)slot * H + h0 + gg) * HD + dd, O / L);
+    }
+    cluster.sync();                              // nobody leaves while its shared memory may still be read
   }
 }
 
@@ -270,12 +317,39 @@ __global__ void decode_slots_kernel(const int32_t* slot_row, const int32_t* len_
   pos[i] = ctx - 1;
 }
 
+constexpr int kClusterSplits = 8;   // the portable cluster size
+
 int pick_splits(int B, int KV, int max_ctx) {
   const int ctas = B * KV;
   int splits = (4 * 148) / ctas;   // one wave of at most four CTAs per SM: a second, partial wave would double the time
   const int max_by_ctx = std::max(1, (max_ctx / kPageTokens) / 4);   // at least 4 pages per split (one per warp)
   splits = std::min(splits, max_by_ctx);
-  return std::max(1, std::min(splits, kMaxSplits));
+  splits = std::max(1, std::min(splits, kMaxSplits));
+  // a few splits more than a cluster holds are not worth the second launch: 8 splits of 16 or more (slot, KV head)
+  // pairs already put a CTA on most SMs
+  if (splits > kClusterSplits && ctas * kClusterSplits >= 128) splits = kClusterSplits;
+  return splits;
+}
+
+// Launch with programmatic stream serialisation and, when cluster_z > 1, clusters of cluster_z CTAs along z.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_decode(void (*kernel)(KArgs...), dim3 grid, int cluster_z, cudaStream_t s, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(128);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.numAttrs = 1;
+  if (cluster_z > 1) {
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = 1; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = (unsigned)cluster_z;
+    cfg.numAttrs = 2;
+  }
+  cfg.attrs = attr;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(std::forward<Args>(args))...);
 }
 
 }  // namespace
@@ -307,13 +381,17 @@ cudaError_t launch_attn_decode(int kv_dtype, const float* q, const void* pool_la
   float* part_ml = (float*)((char*)scratch + head);
   float* part_o = part_ml + (size_t)B * H * kMaxSplits * 2;
   const int splits = pick_splits(active_rows > 0 ? std::min(active_rows, B) : B, KV, max_ctx);
+  const bool clustered = splits >= 2 && splits <= kClusterSplits;
   dim3 grid(KV, B, splits);
 #define RSD_DEC(HD, KT, OT, EXTV)                                                                                          \
   do {                                                                                                               \
-    RSD_LAUNCH((attn_decode_kernel<HD, KT, OT, EXTV>), grid, 128, 0, s, q, (const KT*)pool_layer, page_table, max_pages, slot_row,     \
-                                                        len_or_pos, len_offset, (OT*)out, (OT*)out_lo, part_o, part_ml, \
-                                                        H, KV, splits, n_active);                                    \
-    if (splits > 1)                                                                                                  \
+    if (clustered)                                                                                                   \
+      (void)launch_decode(attn_decode_kernel<HD, KT, OT, EXTV, true>, grid, splits, s, q, (const KT*)pool_layer, page_table,       \
+                          max_pages, slot_row, len_or_pos, len_offset, (OT*)out, (OT*)out_lo, part_o, part_ml, H, KV, splits, n_active); \
+    else                                                                                                             \
+      (void)launch_decode(attn_decode_kernel<HD, KT, OT, EXTV, false>, grid, 1, s, q, (const KT*)pool_layer, page_table,           \
+                          max_pages, slot_row, len_or_pos, len_offset, (OT*)out, (OT*)out_lo, part_o, part_ml, H, KV, splits, n_active); \
+    if (splits > 1 && !clustered)                                                                                    \
       RSD_LAUNCH((attn_merge_kernel<HD, OT>), dim3(H, B), HD, 0, s, part_o, part_ml, slot_row, len_or_pos, len_offset, (OT*)out, \
                                                           (OT*)out_lo, H, splits, n_active);                         \
   } while (0)
@@ -323,7 +401,7 @@ cudaError_t launch_attn_decode(int kv_dtype, const float* q, const void* pool_la
   else { if (hd == 128) RSD_DEC_O(128, __nv_bfloat16, false); else RSD_DEC_O(64, __nv_bfloat16, false); }
 #undef RSD_DEC_O
 #undef RSD_DEC
-  return launched(splits > 1 ? 2 : 1);
+  return launched(splits > 1 && !clustered ? 2 : 1);
 }
 
 }  // namespace rsd
