@@ -329,6 +329,35 @@ def test_chunk_attention_against_definition(dtype, hd, H, KV):
             np.testing.assert_allclose(got[t, h], want, rtol=0, atol=tol)
 
 
+@pytest.mark.parametrize("H,KV", [(28, 4), (12, 2)])
+def test_chunk_attention_long_prefix(H, KV):
+    """Prefixes of more than a hundred pages (the page ids of a row are fetched in batches of 32, several batches a
+    pass), a chunk that ends in the middle of a page, two rows in one tile; fp16 cache, head_dim 128."""
+    rng = np.random.default_rng(21)
+    hd = 128
+    ctx = [2603, 531]
+    new = [90, 70]
+    B = len(ctx)
+    max_pages = 170
+    pool, table, Ks, Vs = paged_kv(rng, B, KV, hd, ctx, torch.float16, max_pages)
+    rows, poss = [], []
+    for b in range(B):
+        for p in range(ctx[b] - new[b], ctx[b]):
+            rows.append(b); poss.append(p)
+    T = len(rows)
+    q = rng.normal(size=(T, H, hd)).astype(np.float32)
+    got = rb.k_attn_chunk(dev(q), pool, table, dev(np.array(rows, np.int32)), dev(np.array(poss, np.int32)), KV).cpu().numpy()
+    assert np.isfinite(got).all()
+    for t in range(0, T, 3):
+        b, p = rows[t], poss[t]
+        for h in range(0, H, max(1, H // 5)):
+            g = h // (H // KV)
+            s = Ks[b][:p + 1, g].astype(np.float64) @ q[t, h].astype(np.float64) / np.sqrt(hd)
+            w = np.exp(s - s.max()); w /= w.sum()
+            want = w @ Vs[b][:p + 1, g].astype(np.float64)
+            np.testing.assert_allclose(got[t, h], want, rtol=0, atol=2e-3)
+
+
 @pytest.mark.parametrize("hd,H,KV", [(128, 12, 2), (128, 64, 8), (64, 4, 2), (128, 16, 1)])
 def test_extended_precision_attention(hd, H, KV):
     """fp16 cache with keys and values kept as hi + lo pairs, queries and softmax weights as hi + lo
