@@ -250,6 +250,9 @@ def workload_config(args) -> dict:
                         + (f"delta {args.delta}" if getattr(args, "delta", None) is not None else "delta at the 70% accept quantile"),
             "batch": B, "max_step_tokens": args.cap or cap, "replicas": args.gpus,
             "kv_cache": kv_cache_label(args), "max_chunk_tokens": chunk_tokens(args) or 4096,
+            "dense_operands": "bf16 hi + lo pairs" if getattr(args, "no_f16_dense", False) else
+                              "passes of more than 128 tokens: fp16 copies of the layer weights (made at load, models up to 20 GB) "
+                              "x one fp16 activation; decode and the 72B-shape target: bf16 weights x bf16 hi + lo pairs",
             "prm": "head on the draft's trunk (prm_shares_draft)" if getattr(args, "merged_prm", False) else "separate model",
             "schedule": "lock-step rsd_step" if getattr(args, "queue", 1) == 1 else
                         f"rsd_step_queued, target pass once {args.queue} rows wait",
@@ -273,7 +276,9 @@ def combine_ranks(ms, e2e_ms, tokens, e2e_tokens, world, device):
 
 def debug_flags(args) -> int:
     from paper_2501_19324_b200 import RSD_DEBUG_PERSISTENT_DECODE, RSD_DEBUG_MEGA_PROFILE
-    return (RSD_DEBUG_PERSISTENT_DECODE if (args.mega or args.mega_profile) else 0) | (RSD_DEBUG_MEGA_PROFILE if args.mega_profile else 0)
+    from paper_2501_19324_b200.binding import RSD_DEBUG_NO_F16_DENSE
+    return ((RSD_DEBUG_PERSISTENT_DECODE if (args.mega or args.mega_profile) else 0) | (RSD_DEBUG_MEGA_PROFILE if args.mega_profile else 0)
+            | (RSD_DEBUG_NO_F16_DENSE if getattr(args, "no_f16_dense", False) else 0))
 
 
 def mega_phase_table(eng, which: int, n_layers: int) -> dict:
@@ -865,6 +870,8 @@ def main():
                     help="record and print the phase timeline of the persistent decode kernel's last launches")
     ap.add_argument("--chunk", type=int, default=0,
                     help="max_chunk_tokens: tokens per multi-token pass (default: 8192 for cfg2 / cfg3, else the library's 4096)")
+    ap.add_argument("--no-f16-dense", action="store_true", dest="no_f16_dense",
+                    help="keep bf16 hi + lo operand pairs in the dense passes (no fp16 weight copies)")
     ap.add_argument("--sd", type=int, default=0,
                     help="sd_tokens: rejected steps by speculative decoding with this many proposals per round (0 = off, the headline)")
     ap.add_argument("--queue", type=int, default=1,

@@ -131,8 +131,12 @@ enum {
                                 decode iteration run as ONE persistent kernel (one CTA per SM, grid barriers
                                 between the phases) instead of kernel by kernel.  Same results; slower than
                                 the default on the measured shapes, kept for study                    */
-  RSD_DEBUG_MEGA_PROFILE = 8 /* the persistent decode kernel records global-timer stamps around its grid
+  RSD_DEBUG_MEGA_PROFILE = 8, /* the persistent decode kernel records global-timer stamps around its grid
                                 barriers (rsd_debug_mega_profile)                                     */
+  RSD_DEBUG_NO_F16_DENSE = 16 /* keep bf16 hi + lo operand pairs in the passes of more than 128 tokens too
+                                (by default a bf16 model that uses the pairs gets fp16 copies of its layer
+                                matrices in the workspace, up to 20 GB a model, and those passes run on them
+                                with one fp16 activation operand: half the tensor-core work)             */
 };
 
 /* Fills cfg->kv_bytes[] (enough pages for max_batch rows of max_seq_tokens) and

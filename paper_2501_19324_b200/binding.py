@@ -19,6 +19,7 @@ RSD_DEBUG_KEEP_LOGITS = 1
 RSD_DEBUG_NO_GRAPHS = 2
 RSD_DEBUG_PERSISTENT_DECODE = 4
 RSD_DEBUG_MEGA_PROFILE = 8
+RSD_DEBUG_NO_F16_DENSE = 16
 ERRORS = {0: "RSD_OK", -1: "RSD_ERR_ARG", -2: "RSD_ERR_STATE", -3: "RSD_ERR_OOM_PAGES", -4: "RSD_ERR_CUDA",
           -5: "RSD_ERR_TIMEOUT", -6: "RSD_ERR_UNSUPPORTED"}
 

@@ -24,6 +24,22 @@ struct ModelHost {
   size_t elem = 4;
   int kv_dtype = 0;      // element type of this model's KV cache: 0 fp32, 2 fp16 (for bf16 weights)
   bool split = false;    // bf16 GEMM inputs are kept as hi + lo pairs
+  // Dense passes (more than 128 tokens) of a split model run on fp16 copies of its layer matrices with ONE fp16
+  // activation operand instead of the bf16 pair: half the tensor-core work at an 11-bit significand.
+  bool f16_dense = false;
+  char* w16 = nullptr;                  // the copies: per layer wqkv, wo, wgu, wdown back to back
+  size_t w16_layer = 0;                 // elements of one layer's four matrices
+  // fp16 copy of matrix `which` (0 wqkv, 1 wo, 2 wgu, 3 wdown) of layer l
+  const void* w16_of(int l, int which) const {
+    const size_t d = m.d_model, hq = (size_t)m.n_heads * m.head_dim, qkv = (size_t)(m.n_heads + 2 * m.n_kv_heads) * m.head_dim;
+    const size_t off[4] = {0, qkv * d, qkv * d + d * hq, qkv * d + d * hq + 2 * (size_t)m.d_ffn * d};
+    return w16 + ((size_t)l * w16_layer + off[which]) * 2;
+  }
+  size_t w16_elems(int which) const {
+    const size_t d = m.d_model, hq = (size_t)m.n_heads * m.head_dim, qkv = (size_t)(m.n_heads + 2 * m.n_kv_heads) * m.head_dim;
+    const size_t n[4] = {qkv * d, d * hq, 2 * (size_t)m.d_ffn * d, d * (size_t)m.d_ffn};
+    return n[which];
+  }
   float2* rope = nullptr;
   char* kv_pool = nullptr;
   size_t layer_stride = 0;  // bytes of one layer's slab
@@ -187,6 +203,25 @@ Dims max_dims(const rsd_model* const ms[3]) {
   return r;
 }
 
+// Elements of one layer's four weight matrices.
+size_t layer_weight_elems(const rsd_model& m) {
+  const size_t d = m.d_model, hq = (size_t)m.n_heads * m.head_dim, qkv = (size_t)(m.n_heads + 2 * m.n_kv_heads) * m.head_dim;
+  return qkv * d + d * hq + 2 * (size_t)m.d_ffn * d + d * (size_t)m.d_ffn;
+}
+
+// Which models get fp16 copies of their layer matrices for the dense passes: bf16 models that keep hi + lo operands
+// (so not the narrow PRMs, which already run plain bf16), whose chunk attention is the kernel that can write a single
+// fp16 operand (fp16 cache without the low halves, head_dim 128, groups of up to 8 heads), and whose copies stay
+// within 20 GB (a 72B-shape model's would not fit beside the model itself).
+bool wants_f16_dense(const rsd_config& cfg, const rsd_model& m, int which) {
+  if (cfg.debug_flags & RSD_DEBUG_NO_F16_DENSE) return false;
+  if (m.dtype != RSD_BF16) return false;
+  if (which == RSD_PRM && (cfg.prm_shares_draft || m.d_model <= 2048)) return false;
+  if (kv_extended_for(m, cfg.kv_extended)) return false;
+  if (m.head_dim != 128 || m.n_heads % m.n_kv_heads != 0 || m.n_heads / m.n_kv_heads > 8) return false;
+  return layer_weight_elems(m) * 2 * (size_t)m.n_layers <= ((size_t)20 << 30);
+}
+
 // Lays out the workspace; with c == nullptr only the size is computed.
 size_t layout_workspace(const rsd_config& cfg, const rsd_model* const ms[3], rsd_ctx* c) {
   Layout L;
@@ -257,6 +292,9 @@ size_t layout_workspace(const rsd_config& cfg, const rsd_model* const ms[3], rsd
     for (int w = 0; w < 3; w += 2) mega_prof[w] = TAKE(unsigned long long, 1024);
   float2* rope[3];
   for (int w = 0; w < 3; ++w) rope[w] = TAKE(float2, (size_t)S * (ms[w]->head_dim / 2));
+  char* w16[3] = {nullptr, nullptr, nullptr};
+  for (int w = 0; w < 3; ++w)
+    if (wants_f16_dense(cfg, *ms[w], w)) w16[w] = TAKE(char, layer_weight_elems(*ms[w]) * 2 * (size_t)ms[w]->n_layers);
   float* dbg[2] = {nullptr, nullptr};
   if (cfg.debug_flags & RSD_DEBUG_KEEP_LOGITS) {
     dbg[0] = TAKE(float, (size_t)B * C * ms[RSD_DRAFT]->vocab);
@@ -292,6 +330,7 @@ size_t layout_workspace(const rsd_config& cfg, const rsd_model* const ms[3], rsd
     c->mega_sync = mega_sync;
     for (int w = 0; w < 3; ++w) c->mega_prof[w] = mega_prof[w];
     for (int w = 0; w < 3; ++w) c->mdl[w].rope = rope[w];
+    for (int w = 0; w < 3; ++w) c->mdl[w].w16 = w16[w];
     c->dbg_logits[0] = dbg[0]; c->dbg_logits[1] = dbg[1];
     c->d_scalars = scal;
     c->o_tokens = o_tokens; c->o_len = o_len; c->o_rewards = o_rewards; c->o_accept = o_accept; c->o_live = o_live;
@@ -403,6 +442,57 @@ bool gu_fused_ok(const ModelHost& M, int rows) {
   return rows <= 128 && M.m.dtype == RSD_BF16 && M.split && gemm_gu_supported(1, rows, M.m.d_ffn, M.m.d_model);
 }
 
+// One dense GEMM of the fp16 pass, timed like gemm() (class "plain": its tensor-core work is the algorithm's).
+int gemm_f16(rsd_ctx* c, const void* W16, const void* x16, float* y, int Mrows, int N, int K, int accumulate, cudaStream_t s) {
+  const bool pick = c->time_stride > 0 && (c->gemm_calls++ % (uint64_t)c->time_stride) == 0;
+  const bool timed = pick && c->ev_used < c->ev_bytes.size();
+  if (timed) CU(cudaEventRecord(c->ev[2 * c->ev_used], s));
+  CU(launch_gemm_f16_dense(W16, x16, y, Mrows, N, K, accumulate, c->gemm_scratch, c->gemm_scratch_bytes, s));
+  if (timed) {
+    CU(cudaEventRecord(c->ev[2 * c->ev_used + 1], s));
+    c->ev_bytes[c->ev_used] = (double)N * K * 2 + (double)Mrows * K * 2 + (double)Mrows * N * 4.0 * (accumulate ? 2.0 : 1.0);
+    c->ev_flops[c->ev_used] = 2.0 * Mrows * (double)N * K;
+    ++c->ev_used;
+  }
+  return RSD_OK;
+}
+
+// The layer stack of a pass of more than 128 tokens on the fp16 copies of the weights: every GEMM operand (normed
+// residual, attention output, SwiGLU output) is written once, as fp16, by the kernel that produces it.  x holds the
+// embedded tokens on entry and the last layer's residual stream on exit, as in forward_pass.
+int forward_pass_f16(rsd_ctx* c, int which, PassView p, cudaStream_t s) {
+  const ModelHost& M = c->mdl[which];
+  const rsd_model& m = M.m;
+  const int d = m.d_model, H = m.n_heads, KV = m.n_kv_heads, hd = m.head_dim, F = m.d_ffn;
+  const int T = p.T;
+  for (int l = 0; l < m.n_layers; ++l) {
+    KvView kv{M.kv_pool + (size_t)l * M.layer_stride, c->st.page_table[which], c->max_pages, 0};
+    CU(launch_rmsnorm(m.dtype, c->x, M.norm1[l], c->h, nullptr, T, d, m.rms_eps, nullptr, nullptr, SplitSum(), s, true));
+    int rc = gemm_f16(c, M.w16_of(l, 0), c->h, c->qkv, T, (H + 2 * KV) * hd, d, 0, s);
+    if (rc) return rc;
+    CU(launch_rope_kv(M.kv_dtype, c->qkv, SplitSum(), p, c->q, kv, M.rope, H, KV, hd, s));
+    CU(launch_attn_chunk(M.kv_dtype, c->q, p, kv, c->attn, nullptr, 2, H, KV, hd, s, (int*)((char*)c->gemm_scratch + 4096)));
+    rc = gemm_f16(c, M.w16_of(l, 1), c->attn, c->x, T, d, H * hd, 1, s);
+    if (rc) return rc;
+    CU(launch_rmsnorm(m.dtype, c->x, M.norm2[l], c->h, nullptr, T, d, m.rms_eps, nullptr, nullptr, SplitSum(), s, true));
+    {
+      const bool pick = c->time_stride > 0 && (c->gemm_calls++ % (uint64_t)c->time_stride) == 0;
+      const bool timed = pick && c->ev_used < c->ev_bytes.size();
+      if (timed) CU(cudaEventRecord(c->ev[2 * c->ev_used], s));
+      CU(launch_gemm_gu_f16_dense(M.w16_of(l, 2), c->h, c->act, T, F, d, c->gemm_scratch, c->gemm_scratch_bytes, s));
+      if (timed) {
+        CU(cudaEventRecord(c->ev[2 * c->ev_used + 1], s));
+        c->ev_bytes[c->ev_used] = 2.0 * F * d * 2 + (double)T * d * 2 + (double)T * F * 2;
+        c->ev_flops[c->ev_used] = 2.0 * T * 2.0 * F * d;
+        ++c->ev_used;
+      }
+    }
+    rc = gemm_f16(c, M.w16_of(l, 3), c->act, c->x, T, d, F, 1, s);
+    if (rc) return rc;
+  }
+  return RSD_OK;
+}
+
 int forward_pass(rsd_ctx* c, int which, PassView p, cudaStream_t s) {
   const ModelHost& M = c->mdl[which];
   const rsd_model& m = M.m;
@@ -410,6 +500,9 @@ int forward_pass(rsd_ctx* c, int which, PassView p, cudaStream_t s) {
   const int T = p.T;
   if (T <= 0) return RSD_OK;
   CU(launch_embed(m.dtype, m.tok_embed, p, c->x, d, s));
+  // dense pass of a model with fp16 weight copies: one fp16 activation operand, no low halves
+  const bool f16 = M.f16_dense && p.n_active == nullptr && T > 128 && gemm_gu_supported(1, T, F, d);
+  if (f16) return forward_pass_f16(c, which, p, s);
   void* h_lo = M.split ? c->h_lo : nullptr;
   void* attn_lo = M.split ? c->attn_lo : nullptr;
   void* act_lo = M.split ? c->act_lo : nullptr;
@@ -921,6 +1014,8 @@ int rsd_load_models(rsd_ctx* c, const rsd_model* draft, const rsd_model* prm, co
     // width, so PRMs of up to 2048 columns take plain operands (half the tensor-core work of a scoring pass),
     // wider ones the pairs.
     M.split = M.m.dtype == RSD_BF16 && !(w == RSD_PRM && M.m.d_model <= 2048);
+    M.f16_dense = M.split && M.w16 != nullptr && wants_f16_dense(c->cfg, M.m, w);
+    M.w16_layer = layer_weight_elems(M.m);
     M.n_params = count_params(M.m);
     M.kv_pool = (char*)c->cfg.kv_pool[w];
     const size_t page_bytes = (size_t)(M.kv_dtype == 3 ? 4 : 2) * M.m.n_kv_heads * kPageTokens * M.m.head_dim * M.elem;
@@ -934,6 +1029,16 @@ int rsd_load_models(rsd_ctx* c, const rsd_model* draft, const rsd_model* prm, co
   cudaStream_t s = 0;
   for (int w = 0; w < 3; ++w)
     CU(launch_rope_table(c->mdl[w].rope, c->S, c->mdl[w].m.head_dim, c->mdl[w].m.rope_theta, s));
+  // fp16 copies of the layer matrices for the dense passes (exact for |w| >= 2^-14, to 2^-25 absolute below)
+  for (int w = 0; w < 3; ++w) {
+    const ModelHost& M = c->mdl[w];
+    if (!M.f16_dense) continue;
+    for (int l = 0; l < M.m.n_layers; ++l) {
+      const void* src[4] = {M.wqkv[l], M.wo[l], M.wgu[l], M.wdown[l]};
+      for (int k = 0; k < 4; ++k)
+        CU(launch_bf16_to_f16(src[k], const_cast<void*>(M.w16_of(l, k)), M.w16_elems(k), s));
+    }
+  }
   CU(cudaMemsetAsync(c->d_scalars, 0, 16 * sizeof(int32_t), s));
   CU(cudaMemsetAsync(c->gemm_scratch, 0, c->gemm_scratch_bytes, s));
   CU(cudaMemsetAsync(c->sample_best, 0, sizeof(unsigned long long) * c->slots_max, s));

@@ -249,6 +249,7 @@ cudaError_t launch_attn_chunk(int kv_dtype, const float* q, PassView p, KvView k
   if (p.T <= 0) return cudaSuccess;
   if (attn_chunk_tc_supported(kv_dtype, H, KV, hd, p.T))
     return launch_attn_chunk_tc(q, p, kv, out, out_lo, out_dtype, H, KV, err, s);
+  if (out_dtype == 2) return cudaErrorNotSupported;   // a single fp16 operand is written by the tcgen05 kernel only
   const int G = H / KV;
   if (kv_dtype == 3) kv.v_extra = 1;
   if (kv_dtype == 0 || G > 8)

@@ -169,6 +169,13 @@ template <> __device__ __forceinline__ void store16<float>(float* hi, float*, si
 #pragma unroll
   for (int i = 0; i < 4; ++i) *reinterpret_cast<float4*>(hi + o + 4 * i) = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
 }
+template <> __device__ __forceinline__ void store16<__half>(__half* hi, __half*, size_t o, const float* v) {
+  __align__(16) __half2 h[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) h[i] = __floats2half2_rn(v[2 * i], v[2 * i + 1]);
+  *reinterpret_cast<uint4*>(hi + o) = *reinterpret_cast<const uint4*>(h);
+  *reinterpret_cast<uint4*>(hi + o + 8) = *reinterpret_cast<const uint4*>(h + 4);
+}
 template <> __device__ __forceinline__ void store16<__nv_bfloat16>(__nv_bfloat16* hi, __nv_bfloat16* lo, size_t o, const float* v) {
   __align__(16) __nv_bfloat16 h[16];
   __align__(16) __nv_bfloat16 l[16];
@@ -562,8 +569,16 @@ cudaError_t launch_attn_chunk_tc(const float* q, PassView p, KvView kv, void* ou
   dim3 grid((p.T + QT - 1) / QT, KV);
   CUtensorMap tm_k, tm_v;
   if (!tc_tensor_map_kv(kv.pool_layer, 0, &tm_k) || !tc_tensor_map_kv(kv.pool_layer, 1, &tm_v)) return cudaErrorInvalidValue;
-  static bool configured[2] = {false, false};
-  if (out_dtype == 1) {
+  static bool configured[3] = {false, false, false};
+  if (out_dtype == 2) {      // one fp16 operand (out_lo unused)
+    if (!configured[2]) {
+      cudaError_t e = cudaFuncSetAttribute(attn_chunk_tc_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+      if (e != cudaSuccess) return e;
+      configured[2] = true;
+    }
+    RSD_LAUNCH((attn_chunk_tc_kernel<__half>), grid, kThreads, kSmemBytes, s, tm_k, tm_v, q, p, (const __half*)kv.pool_layer,
+               kv.page_table, kv.max_pages, (__half*)out, (__half*)nullptr, H, KV, QT, err);
+  } else if (out_dtype == 1) {
     if (!configured[1]) {
       cudaError_t e = cudaFuncSetAttribute(attn_chunk_tc_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
       if (e != cudaSuccess) return e;

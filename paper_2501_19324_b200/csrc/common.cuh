@@ -60,6 +60,9 @@ template <> __device__ __forceinline__ void store_operand<__nv_bfloat16>(__nv_bf
   if (lo != nullptr) lo[i] = __float2bfloat16_rn(v - __bfloat162float(h));
 }
 
+// A single fp16 operand (the dense passes that run on fp16 copies of the weights): no low half.
+template <> __device__ __forceinline__ void store_operand<__half>(__half* hi, __half*, size_t i, float v) { hi[i] = __float2half_rn(v); }
+
 // 16-byte vector of elements of type T, unpacked to fp32.
 template <typename T> struct Vec16;
 template <> struct Vec16<float> {

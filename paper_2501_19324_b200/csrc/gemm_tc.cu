@@ -365,9 +365,12 @@ __global__ void __launch_bounds__(kPersistThreads, 1)
 gemm_tc_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x,
                           const __grid_constant__ CUtensorMap tm_x_lo, float* __restrict__ Y, int M, int N, int K,
                           int accumulate, int n_tiles_n, int n_tiles_m, int* __restrict__ err,
-                          __nv_bfloat16* __restrict__ act_hi, __nv_bfloat16* __restrict__ act_lo) {
+                          __nv_bfloat16* __restrict__ act_hi, __nv_bfloat16* __restrict__ act_lo, int f16) {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   using C = PersistCfg<SPLIT, GU>;
+  // f16: both operands are fp16 (weights re-encoded at load, one fp16 activation operand); the MMA's operand-format
+  // fields become 0 and a gate/up tile writes its activations as fp16.  Otherwise bf16 throughout.
+  const uint32_t idesc = f16 ? (C::kIdesc & ~((1u << 7) | (1u << 10))) : C::kIdesc;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint64_t* full = (uint64_t*)(smem + (size_t)C::kStages * C::kStageBytes);
@@ -443,7 +446,7 @@ gemm_tc_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid
           const uint32_t a = smem_u32(smem + (size_t)s * C::kStageBytes), bb = a + C::kABytes;
 #pragma unroll
           for (int k = 0; k < kTileK / kUmmaK; ++k)
-            umma_bf16(d_tmem, smem_desc_sw128(a + k * kUmmaK * 2), smem_desc_sw128(bb + k * kUmmaK * 2), C::kIdesc,
+            umma_bf16(d_tmem, smem_desc_sw128(a + k * kUmmaK * 2), smem_desc_sw128(bb + k * kUmmaK * 2), idesc,
                       (kb > 0 || k > 0) ? 1u : 0u);
           umma_commit(&empty[s]);
         }
@@ -542,9 +545,13 @@ gemm_tc_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid
                 const float gate = is_gate ? mine : other, up = is_gate ? other : mine;
                 const float a = gate / (1.f + expf(-gate)) * up;
                 const size_t o = (size_t)(m0 + r) * N + n0 + l;
-                const __nv_bfloat16 h = __float2bfloat16_rn(a);
-                act_hi[o] = h;
-                if (SPLIT) act_lo[o] = __float2bfloat16_rn(a - __bfloat162float(h));
+                if (!SPLIT && f16) {
+                  reinterpret_cast<__half*>(act_hi)[o] = __float2half_rn(a);
+                } else {
+                  const __nv_bfloat16 h = __float2bfloat16_rn(a);
+                  act_hi[o] = h;
+                  if (SPLIT) act_lo[o] = __float2bfloat16_rn(a - __bfloat162float(h));
+                }
               }
             }
           }
@@ -792,7 +799,8 @@ static int sm_count() {
 // Dense regime (M > 128 rows, no K split, no row scale, no idle flag): persistent kernel.
 template <bool GU, bool SPLIT>
 static cudaError_t launch_persistent(const CUtensorMap& tw, const CUtensorMap& tx, const CUtensorMap& txl, float* y, int M, int N,
-                                     int K, int accumulate, int* err, __nv_bfloat16* act_hi, __nv_bfloat16* act_lo, cudaStream_t s) {
+                                     int K, int accumulate, int* err, __nv_bfloat16* act_hi, __nv_bfloat16* act_lo, cudaStream_t s,
+                                     int f16 = 0) {
   using C = PersistCfg<SPLIT, GU>;
   constexpr size_t smem = C::kSmemBytes;
   static bool configured = false;
@@ -806,7 +814,7 @@ static cudaError_t launch_persistent(const CUtensorMap& tw, const CUtensorMap& t
   const int tiles_n = GU ? N / 64 : (N + kTileN - 1) / kTileN, tiles_m = (M + C::kRows - 1) / C::kRows;
   const int grid = std::min(tiles_n * tiles_m, n_sm);
   RSD_LAUNCH((gemm_tc_persistent_kernel<GU, SPLIT>), grid, kPersistThreads, smem, s, tw, tx, txl, y, M, N, K, accumulate, tiles_n,
-             tiles_m, err, act_hi, act_lo);
+             tiles_m, err, act_hi, act_lo, f16);
   return launched(1);
 }
 
@@ -934,6 +942,32 @@ cudaError_t launch_gemm_tc(const void* W, const void* x, const void* x_lo, float
     default: RSD_TC(256, false);
   }
 #undef RSD_TC
+}
+
+// Dense products (more than 128 rows) with fp16 weights and ONE fp16 activation operand: the persistent kernel with
+// the operand formats switched.  y [M, N] fp32 (+)= x [M, K] W [N, K]^T.
+cudaError_t launch_gemm_f16_dense(const void* W16, const void* x16, float* y, int M, int N, int K, int accumulate,
+                                  void* scratch, size_t scratch_bytes, cudaStream_t s) {
+  if (M <= 128 || !gemm_tc_supported(1, M, N, K)) return cudaErrorNotSupported;
+  if (!scratch || scratch_bytes < gemm_scratch_bytes(M)) return cudaErrorInvalidValue;
+  if (((uintptr_t)W16 & 15) || ((uintptr_t)x16 & 15)) return cudaErrorMisalignedAddress;
+  TcPlan p = plan_tc(M, N, K, false);
+  CUtensorMap tw, tx;
+  if (!get_map(W16, N, K, kTileN, &tw) || !get_map(x16, M, K, p.rows, &tx)) return cudaErrorNotSupported;
+  int* err = (int*)((char*)scratch + kCounterBytes);
+  return launch_persistent<false, false>(tw, tx, tx, y, M, N, K, accumulate, err, nullptr, nullptr, s, 1);
+}
+
+// act [M, F] fp16 = silu(g) * u with [g | u] = x [M, K] Wgu [2F, K]^T, fp16 operands, more than 128 rows.
+cudaError_t launch_gemm_gu_f16_dense(const void* Wgu16, const void* x16, void* act16, int M, int F, int K, void* scratch,
+                                     size_t scratch_bytes, cudaStream_t s) {
+  if (M <= 128 || !gemm_gu_supported(1, M, F, K) || !act16) return cudaErrorNotSupported;
+  if (!scratch || scratch_bytes < (size_t)kCounterBytes + 256) return cudaErrorInvalidValue;
+  if (((uintptr_t)Wgu16 & 15) || ((uintptr_t)x16 & 15)) return cudaErrorMisalignedAddress;
+  int* err = (int*)((char*)scratch + kCounterBytes);
+  CUtensorMap tw, tx;
+  if (!get_map(Wgu16, 2 * F, K, kTileN / 2, &tw) || !get_map(x16, M, K, 256, &tx)) return cudaErrorNotSupported;
+  return launch_persistent<true, false>(tw, tx, tx, nullptr, M, F, K, 0, err, (__nv_bfloat16*)act16, nullptr, s, 1);
 }
 
 cudaError_t launch_gemm(int dtype, const void* W, const void* x, const void* x_lo, float* y, int M, int N, int K,

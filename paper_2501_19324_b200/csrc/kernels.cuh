@@ -53,12 +53,13 @@ struct KvView {
                                // the values (x = hi + lo, both fp16), laid out like the first two
 };
 
+cudaError_t launch_bf16_to_f16(const void* src, void* dst, size_t n, cudaStream_t s);
 cudaError_t launch_embed(int dtype, const void* embed, PassView p, float* x, int d, cudaStream_t s);
 // out[t] = rmsnorm(x[src ? src[t] : t]); rows with src[t] < 0 are skipped.
 // out (and out_lo when given, bf16 only: the low half of a split-precision operand)
 // pending (splits > 1): x[t] += sum of the partial sums [splits][T][d] first (x is written back).
 cudaError_t launch_rmsnorm(int dtype, float* x, const void* gain, void* out, void* out_lo, int T, int d, float eps,
-                           const int32_t* src, const int32_t* n_active, SplitSum pending, cudaStream_t s);
+                           const int32_t* src, const int32_t* n_active, SplitSum pending, cudaStream_t s, bool out_f16 = false);
 // x_lo (nullable, bf16 only): second operand matrix added to x (split-precision activations).
 cudaError_t launch_gemm_simt(int dtype, const void* W, const void* x, const void* x_lo, float* y, int M, int N, int K,
                              int accumulate, const int32_t* n_active, cudaStream_t s);
@@ -81,6 +82,11 @@ cudaError_t launch_gemm_wait_probe(const void* W, const void* x, float* y, void*
 // silu(g) * u with [g | u] = rowscale * (x + x_lo)[M, K] * Wgu[2F, K]^T, Wgu rows = Wgate | Wup.  No K split and no
 // fp32 gate/up array: the tile of a CTA is 64 gate rows and the 64 matching up rows.  F % 64 == 0.
 bool gemm_gu_supported(int dtype, int M, int F, int K);
+// Dense passes (more than 128 rows) on fp16 copies of the weights with one fp16 activation operand.
+cudaError_t launch_gemm_f16_dense(const void* W16, const void* x16, float* y, int M, int N, int K, int accumulate,
+                                  void* scratch, size_t scratch_bytes, cudaStream_t s);
+cudaError_t launch_gemm_gu_f16_dense(const void* Wgu16, const void* x16, void* act16, int M, int F, int K, void* scratch,
+                                     size_t scratch_bytes, cudaStream_t s);
 cudaError_t launch_gemm_gu(const void* Wgu, const void* x, const void* x_lo, void* act_hi, void* act_lo, int M, int F, int K,
                            void* scratch, size_t scratch_bytes, const int32_t* n_active, cudaStream_t s, RowScale rs = RowScale());
 

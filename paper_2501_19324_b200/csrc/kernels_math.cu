@@ -86,11 +86,36 @@ __global__ void rmsnorm_kernel(float* __restrict__ x, const GT* __restrict__ gai
   }
 }
 
+// bf16 -> fp16, element by element (n a multiple of 8: weight matrices are).
+__global__ void bf16_to_f16_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, size_t n8) {
+  RSD_PDL_SYNC();
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n8; i += (size_t)gridDim.x * blockDim.x) {
+    uint4 v = src[i];
+    const __nv_bfloat162* b = reinterpret_cast<const __nv_bfloat162*>(&v);
+    uint4 o;
+    __half2* h = reinterpret_cast<__half2*>(&o);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) h[k] = __floats2half2_rn(__low2float(b[k]), __high2float(b[k]));
+    dst[i] = o;
+  }
+}
+
+cudaError_t launch_bf16_to_f16(const void* src, void* dst, size_t n, cudaStream_t s) {
+  if (n == 0) return cudaSuccess;
+  if (n % 8 != 0 || ((uintptr_t)src & 15) || ((uintptr_t)dst & 15)) return cudaErrorInvalidValue;
+  const size_t n8 = n / 8;
+  const int blocks = (int)std::min<size_t>((n8 + 255) / 256, 148 * 16);
+  RSD_LAUNCH((bf16_to_f16_kernel), blocks, 256, 0, s, (const uint4*)src, (uint4*)dst, n8);
+  return launched(1);
+}
+
 cudaError_t launch_rmsnorm(int dtype, float* x, const void* gain, void* out, void* out_lo, int T, int d, float eps,
-                           const int32_t* src, const int32_t* n_active, SplitSum pending, cudaStream_t s) {
+                           const int32_t* src, const int32_t* n_active, SplitSum pending, cudaStream_t s, bool out_f16) {
   if (T <= 0) return cudaSuccess;
   const int threads = d >= 2048 ? 512 : 256;
-  if (dtype == 1)
+  if (dtype == 1 && out_f16)
+    RSD_LAUNCH((rmsnorm_kernel<__half, __nv_bfloat16>), T, threads, 0, s, x, (const __nv_bfloat16*)gain, (__half*)out, (__half*)nullptr, d, eps, src, n_active, pending.partials, pending.splits, T);
+  else if (dtype == 1)
     RSD_LAUNCH((rmsnorm_kernel<__nv_bfloat16, __nv_bfloat16>), T, threads, 0, s, x, (const __nv_bfloat16*)gain, (__nv_bfloat16*)out, (__nv_bfloat16*)out_lo, d, eps, src, n_active, pending.partials, pending.splits, T);
   else
     RSD_LAUNCH((rmsnorm_kernel<float, float>), T, threads, 0, s, x, (const float*)gain, (float*)out, nullptr, d, eps, src, n_active, pending.partials, pending.splits, T);

@@ -127,3 +127,34 @@ def test_target_decode_in_the_benchmarked_launch_configuration():
         assert eng.counters()["ingest_tokens"][2] == int((lens[rejected] - 1).sum())
         print(f"7B-shape target, 32-row context, {n_rejected} rejected rows:", stats)
     eng.close()
+
+
+def test_dense_pass_on_fp16_weight_copies_at_the_7b_shape():
+    """Passes of more than 128 tokens run on fp16 copies of the layer matrices with ONE fp16 activation operand
+    (instead of bf16 weights x bf16 hi + lo pairs).  A 150-token prompt beside a 3-token one makes the prefill of
+    every model such a pass; PRM and target have the full 7B shape (28 layers, d 3584), the draft the 1.5B width at
+    two layers.  Row 0's first step is rejected, so the target decodes from the cache the fp16 pass wrote: every
+    logit column of every draft and target iteration within 3e-2 of the oracle, the 7B-shape PRM's rewards (read
+    over the cache its fp16 prefill wrote) within 1e-2, tokens, cursors and page tables bit for bit."""
+    import dataclasses
+    import os
+    from helpers import build_pair, parity_step, compare_counters, compare_state
+    if os.sysconf("SC_PAGE_SIZE") * os.sysconf("SC_PHYS_PAGES") < 90e9:
+        pytest.skip("the oracle needs ~65 GB of host memory for two 7B-shape fp32 weight sets")
+    small = dataclasses.replace(ri.SHAPES["1.5b"], n_layers=2)
+    shapes = (small, ri.SHAPES["7b"], ri.SHAPES["7b"])
+    rng = np.random.default_rng(77)
+    lens = np.array([150, 3], dtype=np.int32)
+    offsets = np.zeros(3, dtype=np.int32)
+    offsets[1:] = np.cumsum(lens)
+    tokens = rng.integers(0, small.vocab, size=int(offsets[-1])).astype(np.int32)
+    kw = dict(max_step_tokens=3, max_steps=2, max_seq_tokens=176, step_end_id=13, temperature=0.7, seed=5)
+    eng, loop = build_pair(shapes, bf16=True, prompts=(tokens, offsets), loop_kwargs=kw)
+    compare_state(eng, loop)
+    stats = {}
+    g, o = parity_step(eng, loop, 0.5, stats=stats, accept_pattern=[0, 1], tol_logits=3e-2, tol_reward=1e-2,
+                       margin_tok=5e-2, margin_gate=1e-2)
+    assert o["rej_idx"] == [0] and eng.state()["rej_idx"] == [0]
+    compare_counters(eng, loop)
+    print("fp16 dense passes, 7B-shape PRM and target after a 150-token prompt:", stats)
+    eng.close()
