@@ -525,8 +525,9 @@ def run_ours(args, rank: int, world: int):
                      "peak_source": how + " (sustained bf16)"}
             dense["gemm"] = {"what": "the dense weight-GEMM launches (more than 128 rows: scoring, sync and catch-up passes) of "
                                      "the extra, untimed step, CUDA events around single launches; algorithmic flops 2 M N K; "
-                                     "'plain' = bf16 operand (the PRM), 'split' = hi + lo operand pair (draft, target: twice "
-                                     "the tensor-core work per algorithmic flop)"}
+                                     "'plain' = one 16-bit operand per activation (bf16 for the narrow PRM; fp16 against fp16 "
+                                     "weight copies for the models that otherwise use pairs), 'split' = bf16 hi + lo pair (twice "
+                                     "the tensor-core work per algorithmic flop: --no-f16-dense, or models too large for copies)"}
             for k, v in gd.items():
                 if v["launches"]:
                     g_tfs = v["flops"] / (v["ms"] * 1e-3) / 1e12
@@ -675,6 +676,25 @@ def sweep_gemm(args):
                               "hbm_frac": byts / us * 1e-3 / hbm, "TFLOPs_algorithmic": flops / us * 1e-6,
                               "bf16_frac_algorithmic": flops / us * 1e-6 / tf, "TFLOPs_mma": 2 * flops / us * 1e-6,
                               "peak_source": how, **detail}), flush=True)
+        # the dense form of the long passes: fp16 weights x one fp16 activation operand (rsd_k_gemm impl 4)
+        W16 = [(torch.randn(N, K, device="cuda") * 0.02).to(torch.float16) for _ in range(nbuf)]
+        for M in (256, 512, 1024, 4096, 8192):
+            x16 = torch.randn(M, K, device="cuda").to(torch.float16)
+            y = torch.zeros(M, N, device="cuda")
+            nbytes = rb.lib().rsd_k_gemm_scratch_bytes(M, N, K)
+            scratch = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
+
+            def call16(W):
+                rb._check(rb.lib().rsd_k_gemm(rb._ptr(W), rb._ptr(x16), None, rb._ptr(y), M, N, K, 1, 0, 4,
+                                              rb._ptr(scratch), nbytes, rb._stream()))
+            us, detail = _graph_time_us(call16, W16, sampler=sampler)
+            byts = N * K * 2 + M * K * 2 + M * N * 4
+            flops = 2.0 * M * N * K
+            print(json.dumps({"sweep": "gemm_f16_dense", "M": M, "K": K, "N": N, "us": us, "GBps": byts / us * 1e-3,
+                              "hbm_frac": byts / us * 1e-3 / hbm, "TFLOPs_algorithmic": flops / us * 1e-6,
+                              "bf16_frac_algorithmic": flops / us * 1e-6 / tf, "TFLOPs_mma": flops / us * 1e-6,
+                              "peak_source": how, **detail}), flush=True)
+        del W16
     sampler.stop()
 
 

@@ -140,7 +140,11 @@ enum {
 };
 
 /* Fills cfg->kv_bytes[] (enough pages for max_batch rows of max_seq_tokens) and
- * cfg->workspace_bytes for these three models.  Host only.  RSD_ERR_ARG on bad shapes.       */
+ * cfg->workspace_bytes for these three models.  Host only.  RSD_ERR_ARG on bad shapes.
+ * The workspace includes room for fp16 copies of the layer matrices of the bf16 models whose
+ * passes of more than 128 tokens run on them (see RSD_DEBUG_NO_F16_DENSE): up to the size of
+ * the model's layers again, for models of up to 20 GB.  rsd_load_models fills the copies; the
+ * caller's weights are only ever read.                                                        */
 int rsd_query_sizes(const rsd_model* draft, const rsd_model* prm, const rsd_model* target, rsd_config* cfg);
 
 /* Creates a context on the current CUDA device from a filled rsd_config.  The KV pools and the
@@ -279,7 +283,9 @@ int rsd_debug_mega_profile(rsd_ctx*, int which, uint64_t* stamps, int32_t capaci
  * x_lo (bf16 only, may be NULL) is the low half of a split-precision activation: x = bf16(a),
  * x_lo = bf16(a - x), both multiplied on the tensor cores and added, so `a` enters with ~16 bits.
  * impl: 0 = pick by shape, 1 = split-K SIMT GEMV path, 2 = tcgen05/TMEM/TMA path (bf16 only,
- * K % 8 == 0, 16-byte aligned rows), 3 = the same with one CTA per output tile (no split along K).  `scratch` (scratch_bytes from rsd_k_gemm_scratch_bytes)
+ * K % 8 == 0, 16-byte aligned rows), 3 = the same with one CTA per output tile (no split along K),
+ * 4 = the dense form of the passes of more than 128 tokens: W and x hold FP16 (dtype still RSD_BF16: the element
+ * size), x_lo NULL, M > 128, one fp16 operand per activation on the persistent tcgen05 kernel.  `scratch` (scratch_bytes from rsd_k_gemm_scratch_bytes)
  * holds split-K partial sums and tile counters; its first 4 KiB + 256 B must be zero before the
  * first call; the counters are left zero by every call and the int at byte 4096 becomes non-zero
  * if a bounded device-side wait of the tcgen05 path expired (RSD_ERR_TIMEOUT condition).                                                      */

@@ -351,7 +351,7 @@ def k_gemm(W, x, y=None, accumulate=False, impl=0, x_lo=None):
         y = torch.zeros(M, N, dtype=torch.float32, device=x.device)
     nbytes = lib().rsd_k_gemm_scratch_bytes(M, N, K)
     scratch = torch.zeros(nbytes, dtype=torch.uint8, device=x.device)
-    dt = RSD_BF16 if W.dtype == torch.bfloat16 else RSD_F32
+    dt = RSD_BF16 if W.dtype in (torch.bfloat16, torch.float16) else RSD_F32     # fp16: impl 4 only (the element size)
     _check(lib().rsd_k_gemm(_ptr(W), _ptr(x), _ptr(x_lo) if x_lo is not None else None, _ptr(y), M, N, K, dt, int(accumulate), impl, _ptr(scratch), nbytes,
                             _stream()))
     if nbytes >= 4100 and int(scratch[4096:4100].view(torch.int32).item()) != 0:

@@ -1442,8 +1442,16 @@ size_t rsd_k_gemm_scratch_bytes(int32_t M, int32_t N, int32_t K) {
 
 int rsd_k_gemm(const void* W, const void* x, const void* x_lo, float* y, int32_t M, int32_t N, int32_t K, int32_t dtype,
                int32_t accumulate, int32_t impl, void* scratch, size_t scratch_bytes, void* cuda_stream) {
-  if (!W || !x || !y || M < 0 || N < 1 || K < 1 || (dtype != RSD_F32 && dtype != RSD_BF16) || impl < 0 || impl > 3)
+  if (!W || !x || !y || M < 0 || N < 1 || K < 1 || (dtype != RSD_F32 && dtype != RSD_BF16) || impl < 0 || impl > 4)
     return RSD_ERR_ARG;
+  if (impl == 4) {
+    // the dense form of the long passes: W and x hold fp16, one operand per activation, more than 128 rows
+    if (x_lo || dtype != RSD_BF16) return RSD_ERR_ARG;
+    if (M <= 128 || K % 8 || !gemm_tc_supported(dtype, M, N, K)) return RSD_ERR_UNSUPPORTED;
+    if (!scratch || scratch_bytes < gemm_scratch_bytes(M)) return RSD_ERR_ARG;
+    KCU(launch_gemm_f16_dense(W, x, y, M, N, K, accumulate, scratch, scratch_bytes, (cudaStream_t)cuda_stream));
+    return RSD_OK;
+  }
   if (K % (dtype == RSD_BF16 ? 8 : 4)) return RSD_ERR_UNSUPPORTED;
   if (impl >= 2 && !gemm_tc_supported(dtype, M, N, K)) return RSD_ERR_UNSUPPORTED;
   if (impl != 1 && (!scratch || scratch_bytes < gemm_scratch_bytes(M))) return RSD_ERR_ARG;

@@ -386,6 +386,25 @@ def test_extended_precision_attention(hd, H, KV):
             np.testing.assert_allclose(gotc[t, h], ref(rows[t], poss[t], qc[t, h], h), rtol=0, atol=2e-5)
 
 
+@pytest.mark.parametrize("M,N,K", [(129, 256, 64), (300, 1000, 520), (512, 1536, 1536), (2100, 640, 128), (4096, 2048, 1536)])
+def test_dense_gemm_on_fp16_operands(M, N, K):
+    """The dense form of the long passes (rsd_k_gemm impl 4): fp16 weights x one fp16 activation operand, more than
+    128 rows, with and without adding into y; against the exact product of the fp16 values in fp64."""
+    rng = np.random.default_rng(31)
+    W = (rng.normal(size=(N, K)) * 0.05).astype(np.float16)
+    x = rng.normal(size=(M, K)).astype(np.float16)
+    want = x.astype(np.float64) @ W.astype(np.float64).T
+    Wd, xd = torch.from_numpy(W).cuda(), torch.from_numpy(x).cuda()
+    got = rb.k_gemm(Wd, xd, impl=4).cpu().numpy()
+    tol = 2e-5 * np.sqrt(K) + 1e-6                      # fp32 accumulation of K products of order 0.05
+    np.testing.assert_allclose(got, want, rtol=0, atol=tol)
+    y0 = rng.normal(size=(M, N)).astype(np.float32)
+    got2 = rb.k_gemm(Wd, xd, y=torch.from_numpy(y0.copy()).cuda(), accumulate=True, impl=4).cpu().numpy()
+    np.testing.assert_allclose(got2, want + y0, rtol=0, atol=tol + 1e-6)
+    with pytest.raises(rb.RsdError):
+        rb.k_gemm(Wd, xd[:128].contiguous(), impl=4)    # the form is for more than 128 rows
+
+
 @pytest.mark.parametrize("M,F,K", [(1, 64, 64), (5, 192, 512), (32, 1408, 512), (33, 128, 520), (70, 2048, 768),
                                    (129, 704, 1408), (300, 320, 256), (32, 8960, 1536), (200, 128, 520), (2100, 640, 128)])
 def test_gate_up_gemm_with_swiglu_epilogue(M, F, K):
