@@ -10,11 +10,16 @@ import rsd_inputs as ri
 pytestmark = [pytest.mark.gpu, pytest.mark.slow]
 
 
-@pytest.mark.parametrize("config", ["cfg2", "cfg3", "cfg4"])
+@pytest.mark.parametrize("config", ["cfg2", "cfg2-pairs", "cfg3", "cfg4"])
 def test_full_size_properties_and_sampled_output(config):
     import torch
     from oracle import OracleModel
     from paper_2501_19324_b200 import Engine, Model, RSD_DEBUG_KEEP_LOGITS, RSD_DRAFT
+    from paper_2501_19324_b200.binding import RSD_DEBUG_NO_F16_DENSE
+    # "-pairs": the passes of more than 128 tokens keep bf16 weights x bf16 hi + lo operand pairs (the form the
+    # 72B-shape target always takes) instead of the fp16 weight copies x one fp16 operand
+    pairs = RSD_DEBUG_NO_F16_DENSE if config.endswith("-pairs") else 0
+    config = config.split("-")[0]
     names, B, lo, hi, cap = {"cfg2": (("1.5b", "1.5b", "7b"), 32, 128, 512, 128),
                              "cfg3": (("1.5b", "7b", "7b"), 64, 256, 256, 256),
                              "cfg4": (("1.5b", "1.5b", "72b"), 8, 256, 256, 256)}[config]
@@ -28,7 +33,7 @@ def test_full_size_properties_and_sampled_output(config):
 
     def run(debug):
         eng = Engine(*models, max_batch=B, max_seq_tokens=hi + 3 * cap, max_step_tokens=cap, max_steps=3,
-                     step_end_id=13, temperature=0.7, seed=0, debug_flags=debug)
+                     step_end_id=13, temperature=0.7, seed=0, debug_flags=debug | pairs)
         eng.prefill(tokens, offsets)
         r0 = eng.step(0.0)                                  # delta = 0: draft-only decoding
         delta = float(np.sort(r0["rewards"])[int(0.3 * B)])
