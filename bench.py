@@ -644,7 +644,17 @@ def sweep_gemm(args):
     hbm, tf, how = peaks()
     if args.only:
         # one point, launched plainly (no graph): the form an ncu capture of the GEMM kernel uses
-        M, K, N = (int(v) for v in args.only.split(","))
+        vals = [int(v) for v in args.only.split(",")]
+        M, K, N = vals[:3]
+        if len(vals) > 3 and vals[3] == 16:
+            # M,K,N,16: the dense fp16 form (fp16 weights x one fp16 activation operand, rsd_k_gemm impl 4)
+            Ws = [(torch.randn(N, K, device="cuda") * 0.02).to(torch.float16) for _ in range(3)]
+            x16 = torch.randn(M, K, device="cuda").to(torch.float16)
+            for W in Ws + Ws:
+                rb.k_gemm(W, x16, impl=4)
+            torch.cuda.synchronize()
+            print(json.dumps({"sweep": "gemm_f16_dense", "only": [M, K, N], "flops": 2.0 * M * N * K}))
+            return
         Ws = [(torch.randn(N, K, device="cuda") * 0.02).to(torch.bfloat16) for _ in range(3)]
         x = torch.randn(M, K, device="cuda")
         hi = x.to(torch.bfloat16)
